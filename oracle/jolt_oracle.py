@@ -1,0 +1,530 @@
+"""Plain fp64 CPU oracle for the JoLT / FlashJoLT hot path.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, obviously-correct statement of
+what the library computes.  It shares no code with the CUDA path, imports nothing
+from the package, and may be imported only by the tests, by the smoke check and by
+the benchmark's CPU-baseline leg.  Everything is numpy in float64 unless a passage
+below fixes a narrower type (fp16 storage of factors and scales, fp32 decision
+precision of the quantiser).
+
+Each function names the passage of the paper it follows:
+
+* Sec. 4 "Partial Tucker backbone"  -> feature_factor, token_unfold, token_factor_exact,
+  core_tensor, compress_cell, decompress_cell
+* Sec. 5 "FlashJoLT" (randomized token-mode SVD after Halko et al.) -> token_factor_randomized,
+  tail_mass_spectrum, cap_policy
+* Sec. 4 "Rotated residual"         -> rotation_signs, hadamard_matrix, rotate, unrotate,
+  quantize_rows, dequantize_rows, pack_codes, unpack_codes
+* Eq. (1)                            -> eq1_bytes, stored_bytes
+* Eq. (2)                            -> eps2_table, tau_table
+* Eq. (3), Eq. (4)                   -> dual_allocate
+
+Pins (tests/test_oracle_*.py): full-rank exactness, exact low-rank recovery, orthonormality,
+energy split, ST-HOSVD sandwich bound, norm preservation and involution of the rotation,
+popcount-vs-Sylvester construction, quantiser error bound, pack/unpack identity on exhaustive
+small patterns, Eq. (1) closed form and the printed 268.4 MB figure, the printed cap-policy
+values, randomized == exact when the sketch covers the rank, and brute-force optimality of
+the dual.  The paper's real-cache error figures (0.009 / 0.006 at 2x) need its models and
+datasets: parity unpinned for those numbers.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+
+# --------------------------------------------------------------------------------------
+# Counter-based random numbers (the method draws a Gaussian sketch and rotation signs;
+# both sides implement this generator separately from the same written definition).
+# --------------------------------------------------------------------------------------
+
+_U64 = np.uint64
+_GOLD = _U64(0x9E3779B97F4A7C15)
+_M1 = _U64(0xBF58476D1CE4E5B9)
+_M2 = _U64(0x94D049BB133111EB)
+
+STREAM_SKETCH = 0
+STREAM_SIGNS = 1
+STREAM_PROBE = 2
+STREAM_EPS = 3
+
+
+def mix64(z):
+    """SplitMix64 finaliser applied to (z + golden-ratio increment), all mod 2^64."""
+    z = np.asarray(z, dtype=_U64)
+    with np.errstate(over="ignore"):
+        z = z + _GOLD
+        z = (z ^ (z >> _U64(30))) * _M1
+        z = (z ^ (z >> _U64(27))) * _M2
+        z = z ^ (z >> _U64(31))
+    return z
+
+
+def stream_base(seed: int, cell: int, stream: int):
+    """Key of one random stream: mix64(mix64(seed) ^ (4*cell + stream))."""
+    s = mix64(_U64(seed & 0xFFFFFFFFFFFFFFFF))
+    return mix64(s ^ _U64(4 * cell + stream))
+
+
+def random_u64(seed: int, cell: int, stream: int, count: int, start: int = 0):
+    base = stream_base(seed, cell, stream)
+    idx = np.arange(start, start + count, dtype=_U64)
+    with np.errstate(over="ignore"):
+        return mix64(base + idx)
+
+
+def gaussian_from_u64(r):
+    """Box-Muller, cosine branch, one normal per 64-bit word, evaluated in fp64.
+
+    u1 = (hi32 + 0.5) / 2^32, u2 = (lo32 + 0.5) / 2^32, z = sqrt(-2 ln u1) cos(2 pi u2).
+    """
+    hi = (r >> _U64(32)).astype(np.float64)
+    lo = (r & _U64(0xFFFFFFFF)).astype(np.float64)
+    u1 = (hi + 0.5) * (1.0 / 4294967296.0)
+    u2 = (lo + 0.5) * (1.0 / 4294967296.0)
+    return np.sqrt(-2.0 * np.log(u1)) * np.cos((2.0 * math.pi) * u2)
+
+
+def gaussian_sketch(seed: int, cell: int, n_rows: int, n_cols: int, stream: int = STREAM_SKETCH):
+    """Seeded Gaussian test matrix Omega (n_rows x n_cols), entry (i, j) from counter i*n_cols + j,
+    rounded to fp32 (the value both sides then use), returned as float64."""
+    r = random_u64(seed, cell, stream, n_rows * n_cols)
+    g = gaussian_from_u64(r).astype(np.float32)
+    return g.astype(np.float64).reshape(n_rows, n_cols)
+
+
+def rotation_signs(seed: int, cell: int, d: int = 128):
+    """Sign vector s in {+1,-1}^d: feature f takes bit (f mod 64) of word f // 64; bit set -> -1."""
+    words = random_u64(seed, cell, STREAM_SIGNS, (d + 63) // 64)
+    f = np.arange(d)
+    bits = (words[f // 64] >> (f % 64).astype(_U64)) & _U64(1)
+    return np.where(bits == 1, -1.0, 1.0)
+
+
+# --------------------------------------------------------------------------------------
+# Rotation: randomized Hadamard along the feature axis (Sec. 4, "Rotated residual")
+# --------------------------------------------------------------------------------------
+
+
+def hadamard_matrix(d: int):
+    """Sylvester-ordered Hadamard matrix, H[i, j] = (-1)^popcount(i & j)."""
+    i = np.arange(d)
+    a = i[:, None] & i[None, :]
+    pc = np.zeros_like(a)
+    while a.any():
+        pc += a & 1
+        a = a >> 1
+    return np.where(pc % 2 == 0, 1.0, -1.0)
+
+
+def rotate(R, signs):
+    """r' = H (s . r) / sqrt(d) along the last axis."""
+    d = R.shape[-1]
+    return ((R * signs) @ hadamard_matrix(d)) / math.sqrt(d)
+
+
+def unrotate(Rp, signs):
+    """Inverse of rotate: r = s . (H r') / sqrt(d)  (H symmetric, H H = d I)."""
+    d = Rp.shape[-1]
+    return ((Rp @ hadamard_matrix(d)) / math.sqrt(d)) * signs
+
+
+# --------------------------------------------------------------------------------------
+# Uniform b-bit quantiser with per-group absmax scale, and bit packing
+# --------------------------------------------------------------------------------------
+
+
+def fp16_round(x):
+    """Round to nearest-even fp16, returned in float64."""
+    with np.errstate(over="ignore"):
+        return np.asarray(x, dtype=np.float64).astype(np.float16).astype(np.float64)
+
+
+def quantize_rows(Rp, bits: int, group: int = 32):
+    """Mid-rise symmetric quantiser on groups of `group` consecutive rotated features.
+
+    a = max |r'| over the group; Delta = fp16(a / 2^(b-1)); Delta == 0 -> all codes 2^(b-1);
+    otherwise u = clamp(floor(r' * (1/Delta)), -2^(b-1), 2^(b-1)-1) + 2^(b-1).
+    The decision (reciprocal, product, floor) is taken in fp32, the precision of the kernel.
+    Returns (codes uint8 [..., d], scales float16 [..., d/group]).
+    """
+    assert bits in (1, 2, 3, 4, 8)
+    shp = Rp.shape
+    d = shp[-1]
+    assert d % group == 0
+    g = Rp.reshape(shp[:-1] + (d // group, group))
+    half = float(1 << (bits - 1))
+    a32 = np.abs(g).max(axis=-1).astype(np.float32)
+    with np.errstate(over="ignore"):
+        delta16 = (a32 * np.float32(1.0 / half)).astype(np.float16)
+    delta32 = delta16.astype(np.float32)
+    zero = delta32 == 0
+    with np.errstate(divide="ignore", over="ignore", invalid="ignore"):
+        inv = np.where(zero, np.float32(0), np.float32(1.0) / np.where(zero, np.float32(1), delta32)).astype(np.float32)
+        q = np.floor(g.astype(np.float32) * inv[..., None])
+    q = np.clip(q, -half, half - 1.0) + half
+    q = np.where(zero[..., None], half, q)
+    return q.astype(np.uint8).reshape(shp), delta16
+
+
+def dequantize_rows(codes, scales, bits: int, group: int = 32):
+    """r^' = Delta * (u - 2^(b-1) + 1/2)."""
+    shp = codes.shape
+    d = shp[-1]
+    half = float(1 << (bits - 1))
+    g = codes.reshape(shp[:-1] + (d // group, group)).astype(np.float64)
+    return ((g - half + 0.5) * scales.astype(np.float64)[..., None]).reshape(shp)
+
+
+def pack_codes(codes, bits: int, group: int = 32):
+    """Per group of 32 codes: `bits` little-endian uint32 words; code j occupies bits
+    [j*b, j*b + b) of the group's 32*b-bit little-endian string.  Returns uint32 [..., d/32*b]."""
+    assert group == 32
+    shp = codes.shape
+    d = shp[-1]
+    g = codes.reshape(-1, d // 32, 32).astype(np.uint64)
+    out = np.zeros((g.shape[0], d // 32, bits), dtype=np.uint64)
+    for j in range(32):
+        pos = j * bits
+        w, off = divmod(pos, 32)
+        v = g[:, :, j] << np.uint64(off)
+        out[:, :, w] |= v & np.uint64(0xFFFFFFFF)
+        if off + bits > 32:
+            out[:, :, w + 1] |= v >> np.uint64(32)
+    return out.astype(np.uint32).reshape(shp[:-1] + (d // 32 * bits,))
+
+
+def unpack_codes(words, bits: int, d: int):
+    shp = words.shape
+    w = words.reshape(-1, d // 32, bits).astype(np.uint64)
+    out = np.zeros((w.shape[0], d // 32, 32), dtype=np.uint8)
+    mask = np.uint64((1 << bits) - 1)
+    for j in range(32):
+        pos = j * bits
+        k, off = divmod(pos, 32)
+        v = w[:, :, k] >> np.uint64(off)
+        if off + bits > 32:
+            v = v | (w[:, :, k + 1] << np.uint64(32 - off))
+        out[:, :, j] = (v & mask).astype(np.uint8)
+    return out.reshape(shp[:-1] + (d,))
+
+
+# --------------------------------------------------------------------------------------
+# Partial Tucker backbone (Sec. 4): ST-HOSVD, feature mode first, then token mode
+# --------------------------------------------------------------------------------------
+
+
+def mode3_gram(X):
+    """C = X_(3) X_(3)^T, the d x d Gram of the feature unfolding; X is [m, T, d]."""
+    A = X.reshape(-1, X.shape[-1])
+    return A.T @ A
+
+
+def feature_factor(X, r_f: int):
+    """Leading r_f mode-3 singular vectors (eigenvectors of the mode-3 Gram, descending)."""
+    lam, V = np.linalg.eigh(mode3_gram(X))
+    order = np.argsort(-lam, kind="stable")
+    lam = np.maximum(lam[order], 0.0)
+    return V[:, order[:r_f]], lam
+
+
+def token_unfold(Y):
+    """Mode-2 unfolding A in R^{T x (m r)}: column index h*r + j."""
+    m, T, r = Y.shape
+    return np.transpose(Y, (1, 0, 2)).reshape(T, m * r)
+
+
+def token_factor_exact(A, r_t: int):
+    """Leading r_t left singular vectors of A and all its singular values."""
+    U, s, _ = np.linalg.svd(A, full_matrices=False)
+    return U[:, :r_t], s
+
+
+def _orth(S):
+    Q, _ = np.linalg.qr(S)
+    return Q
+
+
+def token_factor_randomized(A, r_t: int, Omega, power_iters: int):
+    """Randomized range finder + small SVD (Sec. 5; Halko et al. Alg. 4.4 / 5.1).
+
+    Q = orth(A Omega); q times {Z = orth(A^T Q); Q = orth(A Z)}; B = Q^T A;
+    B = U~ S V~^T; U_T = Q U~[:, :r_t].  Returns (U_T, sigma[k], Q, U~, B).
+    """
+    Q = _orth(A @ Omega)
+    for _ in range(power_iters):
+        Z = _orth(A.T @ Q)
+        Q = _orth(A @ Z)
+    B = Q.T @ A
+    Ut, s, _ = np.linalg.svd(B, full_matrices=False)
+    return Q @ Ut[:, :r_t], s, Q, Ut, B
+
+
+def sketch_width(r_t: int, oversample: int, T: int, N: int):
+    return min(r_t + oversample, T, N)
+
+
+def core_tensor(X, U_T, U_F):
+    """G = X x_2 U_T^T x_3 U_F^T, shape [m, r_t, r_f]."""
+    return np.einsum("htf,tr,fs->hrs", X, U_T, U_F, optimize=True)
+
+
+def reconstruct(G, U_T, U_F):
+    """X~ = G x_2 U_T x_3 U_F."""
+    return np.einsum("hrs,tr,fs->htf", G, U_T, U_F, optimize=True)
+
+
+CORE_TARGET_EXP = 10  # stored core is scaled so that max |G| lies in [2^10, 2^11)
+
+
+def core_scale_exponent(G):
+    """Per-cell power-of-two exponent e with max|G| * 2^-e in [2^10, 2^11); 0 for a zero core."""
+    mx = float(np.abs(G).max()) if G.size else 0.0
+    if mx == 0.0 or not math.isfinite(mx):
+        return 0
+    return int(math.floor(math.log2(mx))) - CORE_TARGET_EXP
+
+
+def stored_backbone(Gs16, e: int, UT16, UF16):
+    """Decoder's backbone from the STORED (fp16) quantities:
+    P_h = fp16(G~_h U~_F^T) (scaled units), X~ = 2^e * U~_T P_h."""
+    P = fp16_round(np.einsum("hrs,fs->hrf", Gs16, UF16, optimize=True))
+    return math.ldexp(1.0, e) * np.einsum("tr,hrf->htf", UT16, P, optimize=True)
+
+
+@dataclass
+class CompressedCell:
+    m: int
+    T: int
+    d: int
+    r_t: int
+    r_f: int
+    bits: int
+    group: int
+    e: int                      # core scale exponent
+    Gs16: np.ndarray            # [m, r_t, r_f] fp16 values (as float64), scaled by 2^-e
+    UT16: np.ndarray            # [T, r_t]
+    UF16: np.ndarray            # [d, r_f]
+    signs: np.ndarray           # [d]
+    words: np.ndarray | None    # uint32 [m, T, d/32*bits]
+    scales: np.ndarray | None   # float16 [m, T, d/32]
+    out_dtype: str = "f16"
+    ideal: dict = field(default_factory=dict)   # unrounded quantities for the invariant tests
+
+
+def compress_cell(X, r_t: int, r_f: int, bits: int, *, seed: int = 0, cell: int = 0,
+                  token_mode: str = "randomized", oversample: int = 10, power_iters: int = 1,
+                  group: int = 32, out_dtype: str = "f16", factors=None) -> CompressedCell:
+    """One (layer group, K|V) cell: partial Tucker backbone + rotated b-bit residual.
+
+    X is [m, T, d] (any float dtype; converted exactly to fp64).  r_t = 0 means no backbone
+    (R = X).  bits = 0 means no residual.  `factors=(U_T, U_F)` injects given factors
+    (stage-isolated parity); otherwise they are computed as the paper states.
+    """
+    X = np.asarray(X, dtype=np.float64)
+    m, T, d = X.shape
+    ideal = {}
+    signs = rotation_signs(seed, cell, d)
+    if r_t > 0:
+        if factors is not None:
+            U_T, U_F = (np.asarray(f, dtype=np.float64) for f in factors)
+            lam = None
+            sig = None
+        else:
+            U_F, lam = feature_factor(X, r_f)
+            Y = np.einsum("htf,fs->hts", X, U_F, optimize=True)
+            A = token_unfold(Y)
+            N = A.shape[1]
+            if token_mode == "exact":
+                U_T, sig = token_factor_exact(A, r_t)
+            elif token_mode == "randomized":
+                k = sketch_width(r_t, oversample, T, N)
+                Omega = gaussian_sketch(seed, cell, N, k)
+                U_T, sig, _, _, _ = token_factor_randomized(A, r_t, Omega, power_iters)
+            else:
+                raise ValueError(token_mode)
+        G = core_tensor(X, U_T, U_F)
+        ideal.update(U_T=U_T, U_F=U_F, G=G, lam=lam, sigma=sig)
+        e = core_scale_exponent(G)
+        Gs16 = fp16_round(G * math.ldexp(1.0, -e))
+        UT16 = fp16_round(U_T)
+        UF16 = fp16_round(U_F)
+        Xt = stored_backbone(Gs16, e, UT16, UF16)
+    else:
+        e = 0
+        Gs16 = np.zeros((m, 0, r_f))
+        UT16 = np.zeros((T, 0))
+        UF16 = np.zeros((d, r_f))
+        Xt = np.zeros_like(X)
+    R = X - Xt
+    ideal["R_stored"] = R
+    words = scales = None
+    if bits > 0:
+        Rp = rotate(R, signs)
+        codes, scales = quantize_rows(Rp, bits, group)
+        words = pack_codes(codes, bits, group)
+        ideal["codes"] = codes
+    return CompressedCell(m, T, d, r_t, r_f, bits, group, e, Gs16, UT16, UF16, signs, words, scales,
+                          out_dtype, ideal)
+
+
+def decompress_cell(c: CompressedCell):
+    """X^ = X~ + s . H(r^') / sqrt(d), rounded to the output dtype."""
+    if c.r_t > 0:
+        Xh = stored_backbone(c.Gs16, c.e, c.UT16, c.UF16)
+    else:
+        Xh = np.zeros((c.m, c.T, c.d))
+    if c.bits > 0:
+        codes = unpack_codes(c.words, c.bits, c.d)
+        Xh = Xh + unrotate(dequantize_rows(codes, c.scales, c.bits, c.group), c.signs)
+    if c.out_dtype == "f16":
+        return fp16_round(Xh)
+    return Xh.astype(np.float32).astype(np.float64)
+
+
+def rel_frobenius(X, Xh):
+    X = np.asarray(X, dtype=np.float64)
+    return float(np.linalg.norm(X - Xh) / np.linalg.norm(X))
+
+
+# --------------------------------------------------------------------------------------
+# Byte model, error model, cap policy, tail-mass accounting, Lagrangian dual
+# --------------------------------------------------------------------------------------
+
+
+def eq1_bytes(m, T, d, r_t, r_f, bits, c: int = 2):
+    """Eq. (1): (m r_T r_d + T r_T + d_h r_d) c + (b/8) m T d_h."""
+    return (m * r_t * r_f + T * r_t + d * r_f) * c + (bits * m * T * d) // 8
+
+
+def stored_bytes(m, T, d, r_t, r_f, bits, c: int = 2, group: int = 32):
+    """Eq. (1) plus the per-group fp16 scales the paper calls negligible (2 M / group bytes if b > 0)."""
+    s = eq1_bytes(m, T, d, r_t, r_f, bits, c)
+    if bits > 0:
+        s += 2 * (m * T * d) // group
+    return s
+
+
+def cap_policy(T: int, ratio: float):
+    """q_cap = min(max(q_min(R), ceil(T/32)), 512), q_min = 32 for R <= 4, 64 for R >= 5 (Sec. 5)."""
+    q_min = 32 if ratio <= 4 else 64
+    return min(max(q_min, -(-T // 32)), 512)
+
+
+def tail_mass_spectrum(sigma_top, total_sq):
+    """Append the omitted Frobenius mass past q_cap as one synthetic singular value (Sec. 5)."""
+    sigma_top = np.asarray(sigma_top, dtype=np.float64)
+    rest = max(0.0, float(total_sq) - float(np.sum(sigma_top ** 2)))
+    return np.concatenate([sigma_top, [math.sqrt(rest)]])
+
+
+def eps2_table(bits_list, n: int = 1 << 20, seed: int = 0, group: int = 32):
+    """Eq. (2) calibration: relative squared error of a Gaussian round trip through the quantiser."""
+    g = gaussian_from_u64(random_u64(seed, 0, STREAM_EPS, n)).reshape(-1, 128)
+    out = {}
+    tot = float(np.sum(g * g))
+    for b in bits_list:
+        if b == 0:
+            out[0] = 1.0
+            continue
+        codes, sc = quantize_rows(g, b, group)
+        gh = dequantize_rows(codes, sc, b, group)
+        out[b] = float(np.sum((g - gh) ** 2)) / tot
+    return out
+
+
+def tau_table(lam, sigma2_sq, total_sq, r_t_grid, r_f_grid):
+    """tau(r_t, r_f) = min(1, [tail_3(r_f) + tail_2(r_t)] / ||X||^2).
+
+    lam: mode-3 Gram eigenvalues (descending); sigma2_sq: squared mode-2 singular values
+    (descending, possibly ending in the synthetic tail value)."""
+    lam = np.asarray(lam, dtype=np.float64)
+    s2 = np.asarray(sigma2_sq, dtype=np.float64)
+    tau = np.zeros((len(r_t_grid), len(r_f_grid)))
+    for i, rt in enumerate(r_t_grid):
+        t2 = float(np.sum(s2[rt:]))
+        for j, rf in enumerate(r_f_grid):
+            t3 = float(np.sum(lam[rf:]))
+            tau[i, j] = min(1.0, (t2 + t3) / total_sq)
+    return tau
+
+
+def cell_options(m, T, d, tau, r_t_grid, r_f_grid, bits_list, eps2, include_scales=True):
+    """All (r_t, r_f, b) options of one cell as parallel lists (error, bytes, triple), in the
+    fixed enumeration order r_t-major, then r_f, then bits."""
+    errs, costs, trip = [], [], []
+    for i, rt in enumerate(r_t_grid):
+        for j, rf in enumerate(r_f_grid):
+            for b in bits_list:
+                errs.append(eps2[b] * tau[i, j])
+                costs.append(stored_bytes(m, T, d, rt, rf, b) if include_scales else eq1_bytes(m, T, d, rt, rf, b))
+                trip.append((rt, rf, b))
+    return np.array(errs), np.array(costs, dtype=np.float64), trip
+
+
+def _argmin_lagrangian(errs, costs, lam):
+    """Per-cell argmin of e + lambda s; ties go to the smaller cost, then the earlier option."""
+    val = errs + lam * costs
+    best = 0
+    for i in range(1, len(val)):
+        if val[i] < val[best] or (val[i] == val[best] and costs[i] < costs[best]):
+            best = i
+    return best
+
+
+def dual_allocate(cells, budget: float, halvings: int = 200):
+    """Lagrangian dual of Eq. (3) by bisection on lambda (Eq. (4)).
+
+    cells: list of (errs, costs) arrays.  Returns (choice index per cell, total cost, lambda,
+    feasible flag).  lambda = 0 is tried first; the upper end is found by doubling; the feasible
+    (cost <= budget) end of the bracket is returned.  If even the cheapest options exceed the
+    budget the cheapest allocation is returned with feasible = False.
+    """
+    def solve(lam):
+        ch = [_argmin_lagrangian(e, c, lam) for e, c in cells]
+        return ch, float(sum(c[i] for (e, c), i in zip(cells, ch)))
+
+    ch, cost = solve(0.0)
+    if cost <= budget:
+        return ch, cost, 0.0, True
+    min_cost = float(sum(c.min() for e, c in cells))
+    if min_cost > budget:
+        ch = [int(np.lexsort((e, c))[0]) for e, c in cells]
+        return ch, min_cost, math.inf, False
+    lo, hi = 0.0, 1e-12
+    ch_hi, cost_hi = solve(hi)
+    while cost_hi > budget:
+        lo = hi
+        hi *= 2.0
+        ch_hi, cost_hi = solve(hi)
+    for _ in range(halvings):
+        mid = 0.5 * (lo + hi)
+        if mid == lo or mid == hi:
+            break
+        ch_m, cost_m = solve(mid)
+        if cost_m <= budget:
+            hi, ch_hi, cost_hi = mid, ch_m, cost_m
+        else:
+            lo = mid
+    return ch_hi, cost_hi, hi, True
+
+
+def plan_spectra(X, q_cap: int, *, seed: int = 0, cell: int = 0, oversample: int = 10,
+                 power_iters: int = 1, token_mode: str = "randomized"):
+    """Spectra the allocator consumes for one cell: mode-3 Gram eigenvalues, squared mode-2
+    singular values of the UNPROJECTED unfolding (top q_cap + synthetic tail when randomized),
+    and ||X||^2."""
+    X = np.asarray(X, dtype=np.float64)
+    m, T, d = X.shape
+    lam = feature_factor(X, d)[1]
+    total = float(np.sum(X * X))
+    A = token_unfold(X)
+    if token_mode == "exact":
+        s = np.linalg.svd(A, compute_uv=False)
+        return lam, s ** 2, total
+    k = sketch_width(q_cap, oversample, T, A.shape[1])
+    Omega = gaussian_sketch(seed, cell, A.shape[1], k, stream=STREAM_PROBE)
+    _, s, _, _, _ = token_factor_randomized(A, q_cap, Omega, power_iters)
+    spec = tail_mass_spectrum(s[:q_cap], total)
+    return lam, spec ** 2, total
