@@ -1,0 +1,175 @@
+/*
+ * jolt.h -- C ABI of the B200 (sm_100a) JoLT / FlashJoLT KV-cache compressor.
+ *
+ * One *cell* is a (layer group g, tensor t in {K, V}) pair (paper Sec. 4, first paragraph).  Its data is
+ * the tensor X in R^{m x T x d_h}, m = (layers in the group) * n_kv_heads, merged index
+ * h = layer_in_group * n_kv_heads + head.  Cell index everywhere: 2*g + (0 for K, 1 for V).
+ *
+ * Every function returns 0 (JOLT_OK) or a negative jolt_status.  No exception, abort or trap crosses
+ * this boundary.  Device pointers are borrowed; the handle owns every compressed buffer.
+ * All work is issued on the CUDA stream passed in (a cudaStream_t cast to void*, NULL = default
+ * stream); jolt_plan and jolt_compress synchronise that stream before they return (they read back
+ * spectra / a status word), jolt_decompress only when the destination is host memory.
+ */
+#ifndef JOLT_H
+#define JOLT_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  JOLT_OK = 0,
+  JOLT_EINVAL = -1,        /* bad argument (null pointer, shape, plan outside its range)            */
+  JOLT_EUNSUPPORTED = -2,  /* valid request that this build does not implement (e.g. head_dim != 128) */
+  JOLT_EBUDGET = -3,       /* even the cheapest grid point exceeds the byte budget; plan = cheapest   */
+  JOLT_ENUMERIC = -4,      /* Cholesky pivot <= 0, eigen-solver not converged, non-finite scale       */
+  JOLT_ENOMEM = -5,        /* host or device allocation failed                                        */
+  JOLT_ECUDA = -6,         /* a CUDA runtime / driver call failed (see jolt_last_error)               */
+  JOLT_ETIMEOUT = -7       /* a bounded device-side wait ran out (kernel returned, context is usable) */
+} jolt_status;
+
+enum { JOLT_F16 = 0, JOLT_F32 = 1 };                 /* element type of the K / V tensors           */
+enum { JOLT_MEM_DEVICE = 0, JOLT_MEM_HOST = 1 };      /* where the K / V tensors live                */
+enum { JOLT_TOKEN_EXACT = 0, JOLT_TOKEN_RANDOMIZED = 1 };
+enum { JOLT_K = 0, JOLT_V = 1 };
+
+/* Shape and strides shared by the K and the V tensor (paper Sec. 4: "partition the L layers into G
+ * contiguous groups").  Element (layer l, head n, token t, feature f) sits at
+ * l*stride_layer + n*stride_head + t*stride_token + f (in elements; the feature stride is 1).
+ * head_dim must be 128; seq_len a multiple of 128; stride_token a multiple of 8.
+ * group_start has n_groups + 1 ascending entries, group_start[0] = 0, group_start[n_groups] = n_layers. */
+typedef struct {
+  int32_t n_layers, n_kv_heads, seq_len, head_dim;
+  int32_t dtype;                    /* JOLT_F16 | JOLT_F32 */
+  int32_t mem_space;                /* JOLT_MEM_DEVICE | JOLT_MEM_HOST (host: the call stages the copies) */
+  int64_t stride_layer, stride_head, stride_token;
+  int32_t n_groups;
+  const int32_t *group_start;       /* host array */
+} jolt_layout;
+
+/* Ranks and residual bit-width of one cell: the (r_T, r_d, b) of paper Eq. (1).
+ * r_t in [0, min(T, m*r_f)], r_t = 0 means no backbone (R = X); r_f in [1, 128] (ignored when r_t = 0);
+ * bits in {0, 1, 2, 3, 4, 8}, 0 = no residual stored.  r_t = 0 together with bits = 0 is JOLT_EINVAL. */
+typedef struct { int32_t r_t, r_f, bits; } jolt_cell_plan;
+
+/* Options of the token-mode solver (paper Sec. 5) and of the allocator's grid (paper Sec. 4, Eq. (3)). */
+typedef struct {
+  int32_t token_mode;               /* JOLT_TOKEN_EXACT | JOLT_TOKEN_RANDOMIZED                          */
+  int32_t oversample;               /* p: sketch width k = min(r_t + p, T, m*r_f); default 10             */
+  int32_t power_iters;              /* q >= 0 power iterations of the range finder                        */
+  int32_t quant_group;              /* must be 32                                                         */
+  uint64_t seed;                    /* seeds the Gaussian sketch and the rotation signs                   */
+  const int32_t *bits_set;          /* host array of allowed bit-widths for jolt_plan; NULL = {0,2,4,8}   */
+  int32_t n_bits;
+  int32_t rank_step;                /* rank grid = multiples of rank_step (default 16)                    */
+  int32_t r_t_min, r_f_min;         /* floors of the grid (default rank_step)                             */
+  int32_t q_cap;                    /* <= 0: the paper's cap policy min(max(q_min(R), ceil(T/32)), 512)   */
+  const double *eps2;               /* host table eps^2(b) for b = 0..8 (Eq. (2)); NULL = built-in        */
+  int32_t count_scale_bytes;        /* 1 (default): the fp16 group scales count toward the budget         */
+} jolt_options;
+
+typedef struct jolt_handle jolt_handle;
+
+/* Fill *o with the defaults listed above (randomized token mode, p = 10, q = 1, seed 0). */
+void jolt_default_options(jolt_options *o);
+
+/* jolt_plan -- paper Sec. 4 "Joint Lagrangian allocation", Eq. (1)-(4), with the spectra of Sec. 5.
+ * Measures, per cell, the mode-3 Gram eigenvalues and the leading q_cap token-mode singular values
+ * (randomized, plus the tail-mass value) on the GPU, copies them to the host, and runs the Lagrangian
+ * dual by bisection so that sum of stored bytes <= byte_budget.
+ * dK, dV: the tensors described by `layout`.  out: host array of 2*n_groups plans.
+ * achieved_bytes (may be NULL): total stored bytes of the returned plan.
+ * Errors: JOLT_EBUDGET leaves the cheapest plan in `out`; other errors leave `out` untouched. */
+int jolt_plan(const jolt_layout *layout, const void *dK, const void *dV, double byte_budget,
+              const jolt_options *opts, void *stream, jolt_cell_plan *out, double *achieved_bytes);
+
+/* jolt_compress -- paper Sec. 4 "Partial Tucker backbone" + "Rotated residual", Sec. 5 for the
+ * randomized token factor.  For every cell: U_F from the mode-3 Gram, U_T (exact or randomized),
+ * core G, residual against the stored fp16 backbone, sign-flip + 128-point Hadamard rotation along
+ * features, per-32-feature absmax mid-rise quantisation to `bits` bits, bit-packing.
+ * plan: host array of 2*n_groups cell plans.  *out receives a new handle (free with jolt_free).
+ * On error *out is NULL. */
+int jolt_compress(const jolt_layout *layout, const void *dK, const void *dV, const jolt_cell_plan *plan,
+                  const jolt_options *opts, void *stream, jolt_handle **out);
+
+/* Test hook: as jolt_compress but with the factors given instead of computed.
+ * UT[c], UF[c]: host fp32 arrays, row-major T x r_t and 128 x r_f, for cell c (entries for cells
+ * with r_t = 0 are ignored).  The library rounds them to fp16, forms the core and proceeds. */
+int jolt_compress_with_factors(const jolt_layout *layout, const void *dK, const void *dV,
+                               const jolt_cell_plan *plan, const jolt_options *opts,
+                               const float *const *UT, const float *const *UF, void *stream,
+                               jolt_handle **out);
+
+/* jolt_decompress -- paper Sec. 4 "decoding simply inverts the rotation", Sec. 7 (decode reconstructs
+ * the cache from its factors): X^ = U_T (G U_F^T) + s . H(dequant(codes)) / sqrt(d), written in
+ * out_layout->dtype to dK_out / dV_out (shape must equal the compressed shape; strides may differ). */
+int jolt_decompress(const jolt_handle *h, const jolt_layout *out_layout, void *dK_out, void *dV_out,
+                    void *stream);
+
+/* Release a handle and all buffers it owns.  NULL is accepted. */
+int jolt_free(jolt_handle *h);
+
+/* Stored bytes of the compressed cache: factors + core + packed codes + scales, i.e. Eq. (1) plus
+ * the scale term, summed over cells. */
+int jolt_compressed_bytes(const jolt_handle *h, int64_t *bytes);
+
+/* Read one stored component of one cell back to host memory (tests, serialisation).
+ * which: 0 = core (fp16 bits, [m][r_t][r_f]), 1 = U_T (fp16, [T][r_t]), 2 = U_F (fp16, [128][r_f]),
+ * 3 = packed codes (uint32, [m][T][4*bits]), 4 = scales (fp16, [m][T][4]), 5 = core exponent (int32),
+ * 6 = token-mode singular values (fp32, k entries, 0 entries if injected), 7 = mode-3 eigenvalues
+ * (fp32, 128).  dst_bytes is the capacity of dst; *written gets the size of the component. */
+int jolt_get_component(const jolt_handle *h, int32_t cell, int32_t which, void *dst, int64_t dst_bytes,
+                       int64_t *written);
+
+/* Host-only allocator (no GPU): the Lagrangian dual of Eq. (3)/(4) on caller-supplied spectra.
+ * For cell c: lam3[c*128 .. +128) mode-3 Gram eigenvalues (descending); sig2sq + sig2_off[c] points at
+ * sig2_len[c] squared token-mode singular values (descending; last one may be the synthetic tail
+ * value); total_sq[c] = ||X||^2.  m[c], T, d describe the cell.  Grid and eps2 come from opts.
+ * r_t_max[c] bounds the token rank grid.  out: n_cells plans. */
+int jolt_allocate(int32_t n_cells, const int32_t *m, int32_t T, int32_t d, const double *lam3,
+                  const double *sig2sq, const int64_t *sig2_off, const int32_t *sig2_len,
+                  const double *total_sq, const int32_t *r_t_max, double byte_budget,
+                  const jolt_options *opts, jolt_cell_plan *out, double *achieved_bytes);
+
+/* Stored bytes of one cell at a given plan (Eq. (1), c = 2, plus 2*M/32 scale bytes if bits > 0 and
+ * count_scale_bytes). */
+int64_t jolt_cell_bytes(int32_t m, int32_t T, int32_t d, int32_t r_t, int32_t r_f, int32_t bits,
+                        int32_t count_scale_bytes);
+
+/* The cap policy of paper Sec. 5: min(max(q_min(R), ceil(T/32)), 512). */
+int32_t jolt_cap_policy(int32_t T, double ratio);
+
+/* Built-in eps^2(b) calibration (Gaussian round trip through the quantiser), b = 0..8; entries for
+ * unsupported widths are NaN. */
+int jolt_eps2_table(double out[9]);
+
+/* Seeded draws of the method, exposed so that tests can compare them with an independent
+ * implementation: n_rows x n_cols Gaussian sketch (host fp32 out) and the 128 rotation signs. */
+int jolt_sketch_host(uint64_t seed, int32_t cell, int32_t stream_id, int64_t n_rows, int32_t n_cols, float *out);
+int jolt_signs_host(uint64_t seed, int32_t cell, float out[128]);
+
+/* Free cached device workspace held by the library for the current device. */
+int jolt_release_workspace(void);
+
+/* Number of kernel launches the library has issued since load (all streams). */
+int64_t jolt_launch_count(void);
+
+/* Selects the kernel family: 0 = portable SIMT kernels only, 1 (default) = tcgen05 / TMA kernels
+ * where the shapes allow.  Returns the previous value. */
+int jolt_set_fast_path(int enabled);
+
+/* Wall-clock-free per-stage device timing of the last compress / decompress on this thread
+ * (milliseconds, CUDA events): out[0..n) in stage order, names via jolt_stage_name. */
+int jolt_last_stage_ms(float *out, int32_t cap, int32_t *n);
+const char *jolt_stage_name(int32_t i);
+
+const char *jolt_strerror(int status);
+const char *jolt_last_error(void);   /* thread-local detail of the last failure */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JOLT_H */

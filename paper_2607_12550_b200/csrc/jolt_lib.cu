@@ -1,0 +1,1176 @@
+// C-ABI entry points and host orchestration of the JoLT compressor.  Every stage of the path is a
+// kernel launched from here; nothing is computed on the host except the allocator (Eq. (3)/(4)),
+// argument checks and task tables.
+#include <algorithm>
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <functional>
+#include <memory>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "allocator.h"
+#include "common.cuh"
+#include "rowquant.cuh"
+#include "simt_gemm.cuh"
+#include "small_solvers.cuh"
+
+using namespace jolt;
+
+namespace jolt {
+thread_local std::string g_err;
+std::atomic<long long> g_launches{0};
+std::atomic<int> g_fast{1};
+
+int fail(int code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  g_err = buf;
+  return code;
+}
+
+// ------------------------------------------------------------------ stage timing
+static const char *kStageNames[] = {"stage_in", "sketch_gen", "gram", "eig_feat", "sketch", "orth", "power", "project",
+                                    "small_svd", "factors", "store", "backbone", "residual_quant", "decode_backbone",
+                                    "decode_rows", "stage_out"};
+constexpr int kNumStages = sizeof(kStageNames) / sizeof(kStageNames[0]);
+struct StageTimer {
+  cudaEvent_t ev[kNumStages + 1];
+  bool have = false;
+  int order[kNumStages + 1];
+  int n = 0;
+  float ms[kNumStages];
+  void init() {
+    if (have) return;
+    for (auto &e : ev) cudaEventCreate(&e);
+    have = true;
+  }
+  void begin(cudaStream_t s) { init(); n = 0; for (auto &m : ms) m = 0.f; cudaEventRecord(ev[0], s); }
+  void mark(int stage, cudaStream_t s) { if (n < kNumStages) { order[n] = stage; ++n; cudaEventRecord(ev[n], s); } }
+  void finish() {
+    for (int i = 0; i < n; ++i) { float t = 0; if (cudaEventElapsedTime(&t, ev[i], ev[i + 1]) == cudaSuccess) ms[order[i]] += t; }
+  }
+};
+thread_local StageTimer g_timer;
+enum { ST_IN = 0, ST_SKGEN, ST_GRAM, ST_EIGF, ST_SKETCH, ST_ORTH, ST_POWER, ST_PROJ, ST_SVD, ST_FACT, ST_STORE, ST_BACK,
+       ST_RQ, ST_DBACK, ST_DROWS, ST_OUT };
+
+// ------------------------------------------------------------------ workspace cache (per device)
+struct Workspace { void *base = nullptr; size_t cap = 0; };
+static std::mutex g_ws_mu;
+static Workspace g_ws[64];
+
+static int ws_reserve(int dev, size_t bytes, void **out) {
+  std::lock_guard<std::mutex> lk(g_ws_mu);
+  Workspace &w = g_ws[dev];
+  if (w.cap < bytes) {
+    if (w.base) { cudaDeviceSynchronize(); cudaFree(w.base); w.base = nullptr; w.cap = 0; }
+    const size_t want = bytes + (bytes >> 3);
+    if (cudaMalloc(&w.base, want) != cudaSuccess) {
+      cudaGetLastError();
+      if (cudaMalloc(&w.base, bytes) != cudaSuccess) { cudaGetLastError(); w.base = nullptr; return fail(JOLT_ENOMEM, "workspace of %zu bytes", bytes); }
+      w.cap = bytes;
+    } else w.cap = want;
+  }
+  *out = w.base;
+  return JOLT_OK;
+}
+
+struct Bump {
+  char *base = nullptr;
+  size_t off = 0;
+  template <typename T> T *take(size_t n) {
+    off = (off + 255) & ~(size_t)255;
+    T *p = base ? (T *)(base + off) : nullptr;
+    off += n * sizeof(T);
+    return p;
+  }
+};
+
+// ------------------------------------------------------------------ small kernels
+__global__ void gen_sketch_kernel(const CellDesc *cells, float *const *omega, const long long *counts, int stream_id,
+                                  uint64_t seed) {
+  const int ci = blockIdx.y;
+  const long long n = counts[ci];
+  const uint64_t base = stream_base(seed, cells[ci].cell, stream_id);
+  float *o = omega[ci];
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    o[i] = (float)gaussian_from_u64(mix64(base + (uint64_t)i));
+}
+
+__global__ void reduce_partials_kernel(const double *const *partials, double *const *out, const int *counts, int n_elems) {
+  const int ci = blockIdx.y;
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n_elems) return;
+  const double *p = partials[ci];
+  double s = 0;
+  for (int h = 0; h < counts[ci]; ++h) s += p[(size_t)h * n_elems + e];
+  out[ci][e] = s;
+}
+
+__global__ void set_identity_kernel(float *const *U, const int *ld) {
+  const int ci = blockIdx.y;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < kD * ld[ci]) U[ci][i] = ((i / ld[ci]) == (i % ld[ci])) ? 1.f : 0.f;
+}
+
+struct StoreJob {
+  const float *G32; const float *UT32; const float *UF32;
+  __half *G16, *UT16, *UF16;
+  int *e;
+  long long nG, nUT, nUF;
+  int round_inputs;   // 1: UT32/UF32 are rounded to fp16 in place as well (injected factors)
+};
+
+__global__ void core_exponent_kernel(const StoreJob *jobs) {
+  const StoreJob j = jobs[blockIdx.x];
+  float mx = 0.f;
+  for (long long i = threadIdx.x; i < j.nG; i += blockDim.x) mx = fmaxf(mx, fabsf(j.G32[i]));
+  for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  __shared__ float red[32];
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < (int)blockDim.x / 32; ++i) mx = fmaxf(mx, red[i]);
+    int e = 0;
+    if (mx > 0.f && isfinite(mx)) e = ilogbf(mx) - kCoreTargetExp;
+    *j.e = e;
+  }
+}
+
+__global__ void store_factors_kernel(const StoreJob *jobs) {
+  const StoreJob j = jobs[blockIdx.y];
+  const int e = *j.e;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  for (long long i = i0; i < j.nG; i += stride) j.G16[i] = __float2half_rn(ldexpf(j.G32[i], -e));
+  for (long long i = i0; i < j.nUT; i += stride) j.UT16[i] = __float2half_rn(j.UT32[i]);
+  for (long long i = i0; i < j.nUF; i += stride) j.UF16[i] = __float2half_rn(j.UF32[i]);
+}
+
+__global__ void round_to_half_inplace_kernel(float *const *ptrs, const long long *counts) {
+  const int ci = blockIdx.y;
+  float *p = ptrs[ci];
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < counts[ci]; i += (long long)gridDim.x * blockDim.x)
+    p[i] = __half2float(__float2half_rn(p[i]));
+}
+
+}  // namespace jolt
+
+// ------------------------------------------------------------------ handle
+struct CellStore {
+  CellDesc c;          // X is null after compress
+  __half *G16 = nullptr, *UT16 = nullptr, *UF16 = nullptr;
+  int *e = nullptr;
+  uint32_t *words = nullptr;
+  __half *scales = nullptr;
+  float *sigma = nullptr;  // k (or T for the exact path)
+  float *lam = nullptr;    // 128
+  int n_sigma = 0;
+};
+
+struct jolt_handle {
+  int device = 0;
+  int n_layers = 0, n_kv_heads = 0, T = 0, n_groups = 0;
+  std::vector<int> group_start;
+  std::vector<CellStore> cells;
+  void *blob = nullptr;
+  size_t blob_bytes = 0;
+  uint64_t seed = 0;
+  int64_t stored_bytes = 0;
+};
+
+// ------------------------------------------------------------------ validation
+static int check_layout(const jolt_layout *L) {
+  if (!L) return fail(JOLT_EINVAL, "layout is null");
+  if (L->head_dim != kD) return fail(L->head_dim > 0 ? JOLT_EUNSUPPORTED : JOLT_EINVAL, "head_dim %d (only 128 is built)", L->head_dim);
+  if (L->n_layers <= 0 || L->n_kv_heads <= 0 || L->seq_len <= 0) return fail(JOLT_EINVAL, "non-positive shape");
+  if (L->seq_len % 128) return fail(JOLT_EUNSUPPORTED, "seq_len %d is not a multiple of 128", L->seq_len);
+  if (L->dtype != JOLT_F16 && L->dtype != JOLT_F32) return fail(JOLT_EINVAL, "dtype %d", L->dtype);
+  if (L->mem_space != JOLT_MEM_DEVICE && L->mem_space != JOLT_MEM_HOST) return fail(JOLT_EINVAL, "mem_space %d", L->mem_space);
+  if (L->stride_token < kD || L->stride_token % 8) return fail(JOLT_EINVAL, "stride_token %lld", (long long)L->stride_token);
+  if (L->stride_head % 8 || L->stride_layer % 8 || L->stride_head <= 0 || L->stride_layer <= 0) return fail(JOLT_EINVAL, "strides must be positive multiples of 8");
+  if (L->n_groups <= 0 || !L->group_start) return fail(JOLT_EINVAL, "layer grouping missing");
+  if (L->group_start[0] != 0 || L->group_start[L->n_groups] != L->n_layers) return fail(JOLT_EINVAL, "group_start must run from 0 to n_layers");
+  for (int g = 0; g < L->n_groups; ++g)
+    if (L->group_start[g + 1] <= L->group_start[g]) return fail(JOLT_EINVAL, "group_start must ascend");
+  return JOLT_OK;
+}
+
+static size_t layout_span_elems(const jolt_layout *L) {
+  return (size_t)(L->n_layers - 1) * L->stride_layer + (size_t)(L->n_kv_heads - 1) * L->stride_head +
+         (size_t)(L->seq_len - 1) * L->stride_token + kD;
+}
+
+static int check_options(const jolt_options *o) {
+  if (!o) return fail(JOLT_EINVAL, "options are null");
+  if (o->token_mode != JOLT_TOKEN_EXACT && o->token_mode != JOLT_TOKEN_RANDOMIZED) return fail(JOLT_EINVAL, "token_mode %d", o->token_mode);
+  if (o->oversample < 0 || o->power_iters < 0 || o->power_iters > 8) return fail(JOLT_EINVAL, "oversample / power_iters out of range");
+  if (o->quant_group != kGroup) return fail(JOLT_EUNSUPPORTED, "quant_group %d (only 32 is built)", o->quant_group);
+  return JOLT_OK;
+}
+
+static bool bits_ok(int b) { return b == 0 || b == 1 || b == 2 || b == 3 || b == 4 || b == 8; }
+
+#define CU(x)                                                                                   \
+  do {                                                                                          \
+    cudaError_t e__ = (x);                                                                      \
+    if (e__ != cudaSuccess) return fail(JOLT_ECUDA, "%s: %s", #x, cudaGetErrorString(e__));      \
+  } while (0)
+#define LAUNCHED() (++g_launches)
+
+// ------------------------------------------------------------------ launch program
+// All argument tables of a call are built on the host first, uploaded with one copy, and then the
+// kernels are launched back to back: the stream never waits for the host between stages.
+namespace {
+
+struct Program {
+  std::vector<char> host;
+  struct Step { int stage; std::function<void(char *, cudaStream_t)> run; };
+  std::vector<Step> steps;
+  template <typename T> size_t push(const std::vector<T> &v) {
+    size_t off = (host.size() + 15) & ~(size_t)15;
+    host.resize(off + v.size() * sizeof(T));
+    if (!v.empty()) memcpy(host.data() + off, v.data(), v.size() * sizeof(T));
+    return off;
+  }
+  void add(int stage, std::function<void(char *, cudaStream_t)> f) { steps.push_back({stage, std::move(f)}); }
+};
+
+GemmTask mk(const void *A, int ta, long long a_rs, long long a_cs, const void *B, int tb, long long b_rs, long long b_cs,
+            void *C, int tc, long long c_rs, int M, int N, int K) {
+  GemmTask t;
+  memset(&t, 0, sizeof t);
+  t.A = A; t.B = B; t.C = C; t.M = M; t.N = N; t.K = K; t.nseg = 1; t.seg_inner = 1;
+  t.a_rs = a_rs; t.a_cs = a_cs; t.b_rs = b_rs; t.b_cs = b_cs; t.c_rs = c_rs; t.c_cs = 1;
+  t.ta = ta; t.tb = tb; t.tc = tc; t.alpha = 1.f; t.alpha_exp = nullptr; t.accumulate = 0;
+  return t;
+}
+
+void add_gemm(Program &P, int stage, const std::vector<GemmTask> &tasks, bool f64) {
+  if (tasks.empty()) return;
+  int mM = 0, mN = 0;
+  for (auto &t : tasks) { mM = std::max(mM, t.M); mN = std::max(mN, t.N); }
+  if (mM == 0 || mN == 0) return;
+  const size_t off = P.push(tasks);
+  const int n = (int)tasks.size();
+  P.add(stage, [=](char *dev, cudaStream_t s) {
+    const GemmTask *d = (const GemmTask *)(dev + off);
+    for (int z0 = 0; z0 < n; z0 += 32768) {
+      dim3 grid((mN + 63) / 64, (mM + 63) / 64, std::min(32768, n - z0));
+      if (f64) simt_gemm_kernel<double><<<grid, 256, 0, s>>>(d + z0);
+      else simt_gemm_kernel<float><<<grid, 256, 0, s>>>(d + z0);
+      LAUNCHED();
+    }
+  });
+}
+
+void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks) {
+  if (tasks.empty()) return;
+  int mn = 0;
+  for (auto &t : tasks) mn = std::max(mn, t.n);
+  const size_t off = P.push(tasks);
+  const int n = (int)tasks.size();
+  const size_t shm = (size_t)(2 * ((mn + 1) / 2) + 32) * sizeof(double);
+  P.add(stage, [=](char *dev, cudaStream_t s) {
+    jacobi_eig_kernel<<<n, kEigThreads, shm, s>>>((const EigTask *)(dev + off));
+    LAUNCHED();
+  });
+}
+
+void add_chol(Program &P, int stage, const std::vector<CholTask> &tasks) {
+  if (tasks.empty()) return;
+  const size_t off = P.push(tasks);
+  const int n = (int)tasks.size();
+  P.add(stage, [=](char *dev, cudaStream_t s) {
+    cholesky_inv_kernel<<<n, 1024, 0, s>>>((const CholTask *)(dev + off));
+    LAUNCHED();
+  });
+}
+
+inline const void *x_head(const CellDesc &c, int h) {
+  const int l = h / c.n_heads, hd = h % c.n_heads;
+  const long long off = (long long)l * c.sl + (long long)hd * c.sh;
+  return (const char *)c.X + off * (c.dtype == DT_F16 ? 2 : 4);
+}
+
+struct CellWork {      // device scratch of one cell
+  CellDesc c;
+  bool active = false;       // has a backbone to compute
+  double *gram_part = nullptr, *C = nullptr, *Cv = nullptr, *Cw = nullptr;
+  float *UF32 = nullptr, *lam = nullptr;
+  float *omega = nullptr, *W = nullptr, *S = nullptr, *S2 = nullptr, *Zp = nullptr, *Z = nullptr, *Z2 = nullptr;
+  double *Gs = nullptr, *Linv = nullptr; float *LinvT = nullptr;
+  double *BBt = nullptr, *BBv = nullptr, *BBw = nullptr;
+  float *Ut = nullptr, *sigma = nullptr;
+  float *UT32 = nullptr, *G32 = nullptr;
+  float *Y = nullptr; double *Gt = nullptr, *Gtv = nullptr, *Gtw = nullptr;
+  __half *P16 = nullptr;
+  float *Xt = nullptr;
+  int *status = nullptr;
+  int n_sigma = 0;
+};
+
+enum FactorMode { FM_RANDOMIZED = 0, FM_EXACT = 1, FM_INJECTED = 2 };
+
+// Scratch layout of one cell; run with b.base == nullptr to size it.
+void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
+  const bool real = b.base != nullptr;
+  const CellDesc &c = w.c;
+  const size_t M = (size_t)c.m * c.T * kD;
+  if (w.active) {
+    const size_t k = c.k, N = c.N, T = c.T;
+    w.UF32 = b.take<float>(kD * (size_t)c.r_f);
+    if (!(real && w.lam)) w.lam = b.take<float>(kD);
+    w.UT32 = b.take<float>(T * c.r_t);
+    w.G32 = b.take<float>((size_t)c.m * c.r_t * c.r_f);
+    w.Zp = b.take<float>((size_t)c.m * kD * std::max<size_t>(k, c.r_t));
+    if (mode != FM_INJECTED) {
+      w.gram_part = b.take<double>((size_t)c.m * kD * kD);
+      w.C = b.take<double>(kD * kD); w.Cv = b.take<double>(kD * kD); w.Cw = b.take<double>(kD);
+    }
+    if (mode == FM_RANDOMIZED) {
+      w.omega = b.take<float>(N * k);
+      w.W = b.take<float>((size_t)c.m * kD * k);
+      w.S = b.take<float>(T * k); w.S2 = b.take<float>(T * k);
+      w.Z = b.take<float>(N * k); w.Z2 = b.take<float>(N * k);
+      w.Gs = b.take<double>(k * k); w.Linv = b.take<double>(k * k); w.LinvT = b.take<float>(k * k);
+      w.BBt = b.take<double>(k * k); w.BBv = b.take<double>(k * k); w.BBw = b.take<double>(k);
+      w.Ut = b.take<float>(k * std::max<size_t>(c.r_t, 1));
+      if (!(real && w.sigma)) w.sigma = b.take<float>(k);
+      w.n_sigma = (int)k;
+    } else if (mode == FM_EXACT) {
+      w.Y = b.take<float>((size_t)c.m * T * c.r_f);
+      w.Gt = b.take<double>(T * T); w.Gtv = b.take<double>(T * T); w.Gtw = b.take<double>(T);
+      if (!(real && w.sigma)) w.sigma = b.take<float>(T);
+      w.n_sigma = (int)T;
+    }
+  }
+  if (need_backbone_scratch && c.r_t > 0) {
+    w.P16 = b.take<__half>((size_t)c.m * c.r_t * kD);
+    w.Xt = b.take<float>(M);
+  }
+}
+
+// orth(S) for every active cell by CholeskyQR2: twice {Gs = S^T S (fp64), Gs = L L^T, S <- S L^-T}.
+// `rows` selects T (token side) or N (feature side); in/out in buf0, buf1 is scratch.
+void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side) {
+  for (int pass = 0; pass < 2; ++pass) {
+    std::vector<GemmTask> g1, g2;
+    std::vector<CholTask> ch;
+    for (auto &w : ws) {
+      if (!w.active) continue;
+      const int k = w.c.k, rows = token_side ? w.c.T : w.c.N;
+      float *src = token_side ? (pass == 0 ? w.S : w.S2) : (pass == 0 ? w.Z : w.Z2);
+      float *dst = token_side ? (pass == 0 ? w.S2 : w.S) : (pass == 0 ? w.Z2 : w.Z);
+      g1.push_back(mk(src, DT_F32, 1, k, src, DT_F32, k, 1, w.Gs, DT_F64, k, k, k, rows));
+      CholTask c; c.G = w.Gs; c.Linv = w.Linv; c.LinvT32 = w.LinvT; c.n = k; c.status = w.status;
+      ch.push_back(c);
+      g2.push_back(mk(src, DT_F32, k, 1, w.LinvT, DT_F32, k, 1, dst, DT_F32, k, rows, k, k));
+    }
+    add_gemm(P, stage, g1, true);
+    add_chol(P, stage, ch);
+    add_gemm(P, stage, g2, false);
+  }
+}
+
+// W_h = U_F R_h for every head (R = Omega or Z, N x k row blocks of r_f), then S = sum_h X_h W_h.
+void add_sketch(Program &P, int stage, std::vector<CellWork> &ws, bool from_omega) {
+  std::vector<GemmTask> g1, g2;
+  for (auto &w : ws) {
+    if (!w.active) continue;
+    const CellDesc &c = w.c;
+    const float *R = from_omega ? w.omega : w.Z;
+    for (int h = 0; h < c.m; ++h)
+      g1.push_back(mk(w.UF32, DT_F32, c.r_f, 1, R + (size_t)h * c.r_f * c.k, DT_F32, c.k, 1,
+                      w.W + (size_t)h * kD * c.k, DT_F32, c.k, kD, c.k, c.r_f));
+    GemmTask t = mk(c.X, c.dtype, c.st, 1, w.W, DT_F32, c.k, 1, w.S, DT_F32, c.k, c.T, c.k, kD);
+    t.nseg = c.m; t.seg_inner = c.n_heads;
+    t.a_so = c.sl; t.a_si = c.sh;
+    t.b_so = (long long)c.n_heads * kD * c.k; t.b_si = (long long)kD * c.k;
+    g2.push_back(t);
+  }
+  add_gemm(P, stage, g1, false);
+  add_gemm(P, stage, g2, false);
+}
+
+// Z_h = U_F^T (X_h^T Q) for every head: rows h*r_f.. of the N x k matrix Z.  Q (T x cols) is `Qsel`.
+void add_project(Program &P, int stage, std::vector<CellWork> &ws) {
+  std::vector<GemmTask> g1, g2;
+  for (auto &w : ws) {
+    if (!w.active) continue;
+    const CellDesc &c = w.c;
+    for (int h = 0; h < c.m; ++h) {
+      g1.push_back(mk(x_head(c, h), c.dtype, 1, c.st, w.S, DT_F32, c.k, 1, w.Zp + (size_t)h * kD * c.k, DT_F32, c.k,
+                      kD, c.k, c.T));
+      g2.push_back(mk(w.UF32, DT_F32, 1, c.r_f, w.Zp + (size_t)h * kD * c.k, DT_F32, c.k, 1,
+                      w.Z + (size_t)h * c.r_f * c.k, DT_F32, c.k, c.r_f, c.k, kD));
+    }
+  }
+  add_gemm(P, stage, g1, false);
+  add_gemm(P, stage, g2, false);
+}
+
+// Stages that produce U_F (fp32), U_T (fp32) and the core (fp32) of every active cell.
+void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool probe, int power_iters, uint64_t seed, bool fast) {
+  (void)fast;
+  std::vector<int> act;
+  for (size_t i = 0; i < ws.size(); ++i) if (ws[i].active) act.push_back((int)i);
+  if (act.empty()) return;
+  const int na = (int)act.size();
+  if (mode == FM_RANDOMIZED) {
+    std::vector<CellDesc> cd; std::vector<float *> om; std::vector<long long> cnt;
+    for (int i : act) { cd.push_back(ws[i].c); om.push_back(ws[i].omega); cnt.push_back((long long)ws[i].c.N * ws[i].c.k); }
+    const size_t o1 = P.push(cd), o2 = P.push(om), o3 = P.push(cnt);
+    const int sid = probe ? STREAM_PROBE : STREAM_SKETCH;
+    P.add(ST_SKGEN, [=](char *dev, cudaStream_t s) {
+      gen_sketch_kernel<<<dim3(148, na), 256, 0, s>>>((const CellDesc *)(dev + o1), (float *const *)(dev + o2),
+                                                      (const long long *)(dev + o3), sid, seed);
+      LAUNCHED();
+    });
+  }
+  if (mode != FM_INJECTED) {
+    // mode-3 Gram: per-head partials in fp64, deterministic reduction, Jacobi
+    std::vector<GemmTask> g;
+    std::vector<const double *> parts; std::vector<double *> outs; std::vector<int> counts;
+    std::vector<EigTask> eg;
+    for (int i : act) {
+      CellWork &w = ws[i];
+      const CellDesc &c = w.c;
+      for (int h = 0; h < c.m; ++h)
+        g.push_back(mk(x_head(c, h), c.dtype, 1, c.st, x_head(c, h), c.dtype, c.st, 1, w.gram_part + (size_t)h * kD * kD,
+                       DT_F64, kD, kD, kD, c.T));
+      parts.push_back(w.gram_part); outs.push_back(w.C); counts.push_back(c.m);
+      EigTask e; memset(&e, 0, sizeof e);
+      e.A = w.C; e.Vt = w.Cv; e.w = w.Cw; e.n = kD; e.status = w.status; e.w_out = w.lam; e.w_sqrt = 0;
+      if (!probe) { e.U_out = w.UF32; e.ld_out = c.r_f; e.r_out = c.r_f; }
+      eg.push_back(e);
+    }
+    add_gemm(P, ST_GRAM, g, true);
+    const size_t o1 = P.push(parts), o2 = P.push(outs), o3 = P.push(counts);
+    P.add(ST_GRAM, [=](char *dev, cudaStream_t s) {
+      reduce_partials_kernel<<<dim3(kD * kD / 256, na), 256, 0, s>>>((const double *const *)(dev + o1), (double *const *)(dev + o2),
+                                                                   (const int *)(dev + o3), kD * kD);
+      LAUNCHED();
+    });
+    add_eig(P, ST_EIGF, eg);
+    if (probe) {
+      std::vector<float *> us; std::vector<int> lds;
+      for (int i : act) { us.push_back(ws[i].UF32); lds.push_back(ws[i].c.r_f); }
+      const size_t p1 = P.push(us), p2 = P.push(lds);
+      P.add(ST_EIGF, [=](char *dev, cudaStream_t s) {
+        set_identity_kernel<<<dim3(kD * kD / 256, na), 256, 0, s>>>((float *const *)(dev + p1), (const int *)(dev + p2));
+        LAUNCHED();
+      });
+    }
+  }
+  if (mode == FM_RANDOMIZED) {
+    add_sketch(P, ST_SKETCH, ws, true);
+    add_orth(P, ST_ORTH, ws, true);
+    for (int it = 0; it < power_iters; ++it) {
+      add_project(P, ST_POWER, ws);
+      add_orth(P, ST_POWER, ws, false);
+      add_sketch(P, ST_POWER, ws, false);
+      add_orth(P, ST_POWER, ws, true);
+    }
+    add_project(P, ST_PROJ, ws);          // Z now holds B^T (N x k)
+    std::vector<GemmTask> g; std::vector<EigTask> eg; std::vector<GemmTask> g2;
+    for (int i : act) {
+      CellWork &w = ws[i];
+      const CellDesc &c = w.c;
+      g.push_back(mk(w.Z, DT_F32, 1, c.k, w.Z, DT_F32, c.k, 1, w.BBt, DT_F64, c.k, c.k, c.k, c.N));
+      EigTask e; memset(&e, 0, sizeof e);
+      e.A = w.BBt; e.Vt = w.BBv; e.w = w.BBw; e.n = c.k; e.status = w.status; e.w_out = w.sigma; e.w_sqrt = 1;
+      if (!probe) { e.U_out = w.Ut; e.ld_out = c.r_t; e.r_out = c.r_t; }
+      eg.push_back(e);
+      if (!probe) {
+        g2.push_back(mk(w.S, DT_F32, c.k, 1, w.Ut, DT_F32, c.r_t, 1, w.UT32, DT_F32, c.r_t, c.T, c.r_t, c.k));
+        for (int h = 0; h < c.m; ++h)   // G_h = Ut_r^T (B restricted to head h) : r_t x r_f
+          g2.push_back(mk(w.Ut, DT_F32, 1, c.r_t, w.Z + (size_t)h * c.r_f * c.k, DT_F32, 1, c.k,
+                          w.G32 + (size_t)h * c.r_t * c.r_f, DT_F32, c.r_f, c.r_t, c.r_f, c.k));
+      }
+    }
+    add_gemm(P, ST_SVD, g, true);
+    add_eig(P, ST_SVD, eg);
+    add_gemm(P, ST_FACT, g2, false);
+  } else if (mode == FM_EXACT) {
+    std::vector<GemmTask> g1, g2, g3; std::vector<EigTask> eg;
+    for (int i : act) {
+      CellWork &w = ws[i];
+      const CellDesc &c = w.c;
+      for (int h = 0; h < c.m; ++h)
+        g1.push_back(mk(x_head(c, h), c.dtype, c.st, 1, w.UF32, DT_F32, c.r_f, 1, w.Y + (size_t)h * c.T * c.r_f, DT_F32,
+                        c.r_f, c.T, c.r_f, kD));
+      GemmTask t = mk(w.Y, DT_F32, c.r_f, 1, w.Y, DT_F32, 1, c.r_f, w.Gt, DT_F64, c.T, c.T, c.T, c.r_f);
+      t.nseg = c.m; t.seg_inner = c.m; t.a_si = (long long)c.T * c.r_f; t.b_si = (long long)c.T * c.r_f;
+      g2.push_back(t);
+      EigTask e; memset(&e, 0, sizeof e);
+      e.A = w.Gt; e.Vt = w.Gtv; e.w = w.Gtw; e.n = c.T; e.status = w.status; e.w_out = w.sigma; e.w_sqrt = 1;
+      if (!probe) { e.U_out = w.UT32; e.ld_out = c.r_t; e.r_out = c.r_t; }
+      eg.push_back(e);
+      if (!probe) for (int h = 0; h < c.m; ++h)
+        g3.push_back(mk(w.UT32, DT_F32, 1, c.r_t, w.Y + (size_t)h * c.T * c.r_f, DT_F32, c.r_f, 1,
+                        w.G32 + (size_t)h * c.r_t * c.r_f, DT_F32, c.r_f, c.r_t, c.r_f, c.T));
+    }
+    add_gemm(P, ST_SKETCH, g1, false);
+    add_gemm(P, ST_SKETCH, g2, true);
+    add_eig(P, ST_SVD, eg);
+    add_gemm(P, ST_FACT, g3, false);
+  } else if (mode == FM_INJECTED) {
+    // core from given factors: Zp_h = X_h^T U_T (128 x r_t), G_h = Zp_h^T U_F (r_t x r_f)
+    std::vector<GemmTask> g1, g2;
+    for (int i : act) {
+      CellWork &w = ws[i];
+      const CellDesc &c = w.c;
+      for (int h = 0; h < c.m; ++h) {
+        g1.push_back(mk(x_head(c, h), c.dtype, 1, c.st, w.UT32, DT_F32, c.r_t, 1, w.Zp + (size_t)h * kD * c.r_t, DT_F32,
+                        c.r_t, kD, c.r_t, c.T));
+        g2.push_back(mk(w.Zp + (size_t)h * kD * c.r_t, DT_F32, 1, c.r_t, w.UF32, DT_F32, c.r_f, 1,
+                        w.G32 + (size_t)h * c.r_t * c.r_f, DT_F32, c.r_f, c.r_t, c.r_f, kD));
+      }
+    }
+    add_gemm(P, ST_FACT, g1, true);
+    add_gemm(P, ST_FACT, g2, true);
+  }
+}
+
+// P_h = fp16(G16_h U_F16^T), X~_h = 2^e U_T16 P_h (fp32 scratch) for cells with a backbone.
+struct BackboneRef { CellDesc c; const __half *G16, *UT16, *UF16; const int *e; __half *P16; float *Xt; };
+void add_backbone(Program &P, int stage, const std::vector<BackboneRef> &refs) {
+  std::vector<GemmTask> g1, g2;
+  for (auto &r : refs) {
+    const CellDesc &c = r.c;
+    if (c.r_t == 0) continue;
+    for (int h = 0; h < c.m; ++h) {
+      g1.push_back(mk(r.G16 + (size_t)h * c.r_t * c.r_f, DT_F16, c.r_f, 1, r.UF16, DT_F16, 1, c.r_f,
+                      r.P16 + (size_t)h * c.r_t * kD, DT_F16, kD, c.r_t, kD, c.r_f));
+      GemmTask t = mk(r.UT16, DT_F16, c.r_t, 1, r.P16 + (size_t)h * c.r_t * kD, DT_F16, kD, 1,
+                      r.Xt + (size_t)h * c.T * kD, DT_F32, kD, c.T, kD, c.r_t);
+      t.alpha_exp = r.e;
+      g2.push_back(t);
+    }
+  }
+  add_gemm(P, stage, g1, false);
+  add_gemm(P, stage, g2, false);
+}
+
+int run_program(Program &P, char *d_tables, cudaStream_t st) {
+  if (!P.host.empty()) CU(cudaMemcpyAsync(d_tables, P.host.data(), P.host.size(), cudaMemcpyHostToDevice, st));
+  int cur = -1;
+  for (auto &s : P.steps) {
+    if (cur != -1 && s.stage != cur) g_timer.mark(cur, st);
+    cur = s.stage;
+    s.run(d_tables, st);
+  }
+  if (cur != -1) g_timer.mark(cur, st);
+  CU(cudaGetLastError());
+  return JOLT_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ call context
+namespace {
+
+static Workspace g_tab[64];
+static int tab_reserve(int dev, size_t bytes, void **out) {
+  std::lock_guard<std::mutex> lk(g_ws_mu);
+  Workspace &w = g_tab[dev];
+  if (w.cap < bytes) {
+    if (w.base) { cudaDeviceSynchronize(); cudaFree(w.base); w.base = nullptr; w.cap = 0; }
+    const size_t want = std::max<size_t>(bytes * 2, 1 << 20);
+    if (cudaMalloc(&w.base, want) != cudaSuccess) { cudaGetLastError(); return fail(JOLT_ENOMEM, "task tables of %zu bytes", want); }
+    w.cap = want;
+  }
+  *out = w.base;
+  return JOLT_OK;
+}
+
+struct TensorRef { const void *K, *V; };
+
+int make_cells(const jolt_layout *L, const void *K, const void *V, const jolt_cell_plan *plan, int oversample,
+               std::vector<CellDesc> &cells) {
+  cells.clear();
+  const int esz = L->dtype == JOLT_F16 ? 2 : 4;
+  for (int g = 0; g < L->n_groups; ++g)
+    for (int which = 0; which < 2; ++which) {
+      CellDesc c;
+      memset(&c, 0, sizeof c);
+      const char *base = (const char *)(which == 0 ? K : V);
+      c.X = base ? base + (size_t)L->group_start[g] * L->stride_layer * esz : nullptr;
+      c.dtype = L->dtype == JOLT_F16 ? DT_F16 : DT_F32;
+      c.n_heads = L->n_kv_heads;
+      c.m = (L->group_start[g + 1] - L->group_start[g]) * L->n_kv_heads;
+      c.T = L->seq_len;
+      c.sl = L->stride_layer; c.sh = L->stride_head; c.st = L->stride_token;
+      const jolt_cell_plan &p = plan[2 * g + which];
+      c.r_t = p.r_t; c.r_f = p.r_t > 0 ? p.r_f : 0; c.bits = p.bits;
+      c.N = c.m * c.r_f;
+      c.k = std::min(std::min(c.r_t + oversample, c.T), c.N);
+      c.cell = 2 * g + which;
+      cells.push_back(c);
+    }
+  return JOLT_OK;
+}
+
+int check_plan(const std::vector<CellDesc> &cells, const jolt_cell_plan *plan) {
+  for (size_t i = 0; i < cells.size(); ++i) {
+    const jolt_cell_plan &p = plan[i];
+    if (!bits_ok(p.bits)) return fail(JOLT_EINVAL, "cell %zu: bits %d", i, p.bits);
+    if (p.r_t < 0) return fail(JOLT_EINVAL, "cell %zu: r_t %d", i, p.r_t);
+    if (p.r_t == 0 && p.bits == 0) return fail(JOLT_EINVAL, "cell %zu stores nothing (r_t = 0 and bits = 0)", i);
+    if (p.r_t > 0) {
+      if (p.r_f < 1 || p.r_f > kD) return fail(JOLT_EINVAL, "cell %zu: r_f %d", i, p.r_f);
+      if (p.r_t > cells[i].T || p.r_t > cells[i].m * p.r_f) return fail(JOLT_EINVAL, "cell %zu: r_t %d exceeds min(T, m r_f)", i, p.r_t);
+    }
+  }
+  return JOLT_OK;
+}
+
+struct StatusReader {
+  int *d = nullptr;
+  std::vector<int> h;
+};
+
+int status_to_code(const std::vector<int> &st) {
+  for (size_t i = 0; i < st.size(); i += 4) {
+    if (st[i] & 1) return fail(JOLT_ENUMERIC, "cell %zu: eigen-solver did not converge", i / 4);
+    if (st[i] & 4) return fail(JOLT_ENUMERIC, "cell %zu: quantisation step is not finite in fp16", i / 4);
+    if (st[i] & 8) return fail(JOLT_ETIMEOUT, "cell %zu: a bounded device-side wait ran out", i / 4);
+  }
+  return JOLT_OK;
+}
+
+}  // namespace
+
+#include "fast_path.cuh"
+
+// ------------------------------------------------------------------ compress
+static int compress_impl(const jolt_layout *L, const void *K, const void *V, const jolt_cell_plan *plan,
+                         const jolt_options *o, const float *const *inUT, const float *const *inUF, void *stream,
+                         jolt_handle **out) {
+  if (out) *out = nullptr;
+  if (!out || !plan || !K || !V) return fail(JOLT_EINVAL, "null argument");
+  int rc;
+  if ((rc = check_layout(L)) || (rc = check_options(o))) return rc;
+  const bool injected = inUT != nullptr || inUF != nullptr;
+  if (injected && (!inUT || !inUF)) return fail(JOLT_EINVAL, "both factor arrays are needed");
+  cudaStream_t st = (cudaStream_t)stream;
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
+  const int mode = injected ? FM_INJECTED : (o->token_mode == JOLT_TOKEN_EXACT ? FM_EXACT : FM_RANDOMIZED);
+  std::vector<CellDesc> cells;
+  make_cells(L, K, V, plan, o->oversample, cells);
+  if ((rc = check_plan(cells, plan))) return rc;
+  if (mode == FM_EXACT) {
+    for (auto &c : cells) {
+      if (c.r_t > 0 && c.T > 1024) return fail(JOLT_EUNSUPPORTED, "exact token factor is built for T <= 1024 (got %d)", c.T);
+      c.k = c.r_t;
+    }
+  }
+  if (injected) for (auto &c : cells) c.k = c.r_t;
+  const int nc = (int)cells.size();
+  const size_t esz = L->dtype == JOLT_F16 ? 2 : 4;
+  const size_t span = layout_span_elems(L) * esz;
+
+  // ---- handle blob
+  std::unique_ptr<jolt_handle> H(new jolt_handle);
+  H->device = dev; H->n_layers = L->n_layers; H->n_kv_heads = L->n_kv_heads; H->T = L->seq_len; H->n_groups = L->n_groups;
+  H->group_start.assign(L->group_start, L->group_start + L->n_groups + 1);
+  H->seed = o->seed;
+  H->cells.resize(nc);
+  for (int pass = 0; pass < 2; ++pass) {
+    Bump b;
+    b.base = (char *)H->blob;
+    int64_t stored = 0;
+    for (int i = 0; i < nc; ++i) {
+      CellStore &cs = H->cells[i];
+      const CellDesc &c = cells[i];
+      cs.c = c; cs.c.X = nullptr;
+      const size_t M = (size_t)c.m * c.T * kD;
+      cs.e = b.take<int>(4);
+      cs.lam = b.take<float>(kD);
+      cs.n_sigma = c.r_t > 0 && !injected ? (mode == FM_EXACT ? c.T : c.k) : 0;
+      cs.sigma = b.take<float>(std::max(cs.n_sigma, 1));
+      cs.G16 = b.take<__half>((size_t)c.m * c.r_t * c.r_f);
+      cs.UT16 = b.take<__half>((size_t)c.T * c.r_t);
+      cs.UF16 = b.take<__half>((size_t)kD * c.r_f);
+      cs.words = b.take<uint32_t>(M / 32 * c.bits);
+      cs.scales = b.take<__half>(c.bits ? M / 32 : 0);
+      stored += cell_bytes(c.m, c.T, kD, c.r_t, c.r_f, c.bits, true);
+    }
+    if (pass == 0) {
+      H->blob_bytes = b.off + 256;
+      H->stored_bytes = stored;
+      if (cudaMallocAsync(&H->blob, H->blob_bytes, st) != cudaSuccess) { cudaGetLastError(); return fail(JOLT_ENOMEM, "compressed cache of %zu bytes", H->blob_bytes); }
+    }
+  }
+  auto free_blob = [&]() { cudaFreeAsync(H->blob, st); H->blob = nullptr; };
+
+  // ---- workspace
+  std::vector<CellWork> ws(nc);
+  const bool fast = g_fast.load() != 0;
+  size_t ws_bytes = 0;
+  void *ws_base = nullptr;
+  int *d_status = nullptr;
+  char *stage_K = nullptr, *stage_V = nullptr;
+  for (int pass = 0; pass < 2; ++pass) {
+    Bump b;
+    b.base = (char *)ws_base;
+    d_status = b.take<int>(4 * (size_t)nc);
+    if (L->mem_space == JOLT_MEM_HOST) { stage_K = b.take<char>(span); stage_V = b.take<char>(span); }
+    for (int i = 0; i < nc; ++i) {
+      CellWork &w = ws[i];
+      w.c = cells[i];
+      w.active = cells[i].r_t > 0;
+      if (pass == 1) { w.lam = H->cells[i].lam; w.sigma = H->cells[i].n_sigma ? H->cells[i].sigma : nullptr; w.status = d_status + 4 * i; }
+      carve(b, w, mode, true);
+      if (pass == 1 && !w.n_sigma) w.n_sigma = H->cells[i].n_sigma;
+    }
+    fast_carve(b, ws, fast);
+    if (pass == 0) {
+      ws_bytes = b.off + 256;
+      if ((rc = ws_reserve(dev, ws_bytes, &ws_base))) { free_blob(); return rc; }
+    }
+  }
+  if (L->mem_space == JOLT_MEM_HOST) {
+    // re-point the cells at the staged device copies
+    for (int i = 0; i < nc; ++i) {
+      const char *hb = (const char *)(i % 2 == 0 ? K : V);
+      const char *db = i % 2 == 0 ? stage_K : stage_V;
+      ws[i].c.X = db + ((const char *)ws[i].c.X - hb);
+      cells[i].X = ws[i].c.X;
+    }
+  }
+
+  // ---- program
+  Program P;
+  build_factor_program(P, ws, mode, false, o->power_iters, o->seed, fast);
+  std::vector<StoreJob> sj;
+  std::vector<BackboneRef> br;
+  for (int i = 0; i < nc; ++i) {
+    const CellDesc &c = cells[i];
+    const CellStore &cs = H->cells[i];
+    if (c.r_t == 0) continue;
+    StoreJob j;
+    j.G32 = ws[i].G32; j.UT32 = ws[i].UT32; j.UF32 = ws[i].UF32;
+    j.G16 = cs.G16; j.UT16 = cs.UT16; j.UF16 = cs.UF16; j.e = cs.e;
+    j.nG = (long long)c.m * c.r_t * c.r_f; j.nUT = (long long)c.T * c.r_t; j.nUF = (long long)kD * c.r_f; j.round_inputs = 0;
+    sj.push_back(j);
+    br.push_back({ws[i].c, cs.G16, cs.UT16, cs.UF16, cs.e, ws[i].P16, ws[i].Xt});
+  }
+  if (!sj.empty()) {
+    const size_t off = P.push(sj);
+    const int n = (int)sj.size();
+    P.add(ST_STORE, [=](char *dev_t, cudaStream_t s) {
+      core_exponent_kernel<<<n, 1024, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
+      store_factors_kernel<<<dim3(64, n), 256, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
+    });
+  }
+  std::vector<RowJob> rj(nc);
+  long long rows = 0;
+  bool any_bits = false;
+  for (int i = 0; i < nc; ++i) {
+    RowJob &j = rj[i];
+    memset(&j, 0, sizeof j);
+    j.c = ws[i].c; j.Xt = cells[i].r_t > 0 ? ws[i].Xt : nullptr;
+    j.words = H->cells[i].words; j.scales = H->cells[i].scales; j.status = d_status + 4 * i; j.row0 = rows;
+    rows += (long long)cells[i].m * cells[i].T;
+    any_bits |= cells[i].bits > 0;
+  }
+  if (!fast_residual(P, ws, br, rj, H.get(), o->seed, fast)) {
+    add_backbone(P, ST_BACK, br);
+    if (any_bits) {
+      const size_t off = P.push(rj);
+      const uint64_t seed = o->seed;
+      P.add(ST_RQ, [=](char *dev_t, cudaStream_t s) {
+        residual_quant_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, s>>>((const RowJob *)(dev_t + off), nc, rows, seed);
+        LAUNCHED();
+      });
+    }
+  }
+  void *d_tab = nullptr;
+  if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) { free_blob(); return rc; }
+
+  // ---- run
+  g_timer.begin(st);
+  cudaError_t ce = cudaMemsetAsync(d_status, 0, sizeof(int) * 4 * nc, st);
+  if (ce == cudaSuccess && L->mem_space == JOLT_MEM_HOST) {
+    ce = cudaMemcpyAsync(stage_K, K, span, cudaMemcpyHostToDevice, st);
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(stage_V, V, span, cudaMemcpyHostToDevice, st);
+    g_timer.mark(ST_IN, st);
+  }
+  if (ce == cudaSuccess && injected) {
+    std::vector<float *> ptrs; std::vector<long long> cnts;
+    for (int i = 0; i < nc && ce == cudaSuccess; ++i) {
+      const CellDesc &c = cells[i];
+      if (c.r_t == 0) continue;
+      if (!inUT[i] || !inUF[i]) { free_blob(); return fail(JOLT_EINVAL, "cell %d: factor pointer is null", i); }
+      ce = cudaMemcpyAsync(ws[i].UT32, inUT[i], sizeof(float) * c.T * c.r_t, cudaMemcpyHostToDevice, st);
+      if (ce == cudaSuccess) ce = cudaMemcpyAsync(ws[i].UF32, inUF[i], sizeof(float) * kD * c.r_f, cudaMemcpyHostToDevice, st);
+    }
+  }
+  if (ce != cudaSuccess) { free_blob(); return fail(JOLT_ECUDA, "staging copy: %s", cudaGetErrorString(ce)); }
+  if ((rc = run_program(P, (char *)d_tab, st))) { free_blob(); return rc; }
+  std::vector<int> hstat(4 * nc);
+  ce = cudaMemcpyAsync(hstat.data(), d_status, sizeof(int) * 4 * nc, cudaMemcpyDeviceToHost, st);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+  if (ce != cudaSuccess) { cudaGetLastError(); free_blob(); return fail(JOLT_ECUDA, "compress: %s", cudaGetErrorString(ce)); }
+  g_timer.finish();
+  if ((rc = status_to_code(hstat))) { free_blob(); return rc; }
+  *out = H.release();
+  return JOLT_OK;
+}
+
+extern "C" int jolt_compress(const jolt_layout *L, const void *K, const void *V, const jolt_cell_plan *plan,
+                             const jolt_options *o, void *stream, jolt_handle **out) {
+  return compress_impl(L, K, V, plan, o, nullptr, nullptr, stream, out);
+}
+
+extern "C" int jolt_compress_with_factors(const jolt_layout *L, const void *K, const void *V, const jolt_cell_plan *plan,
+                                          const jolt_options *o, const float *const *UT, const float *const *UF,
+                                          void *stream, jolt_handle **out) {
+  if (!UT || !UF) { if (out) *out = nullptr; return fail(JOLT_EINVAL, "factor arrays are null"); }
+  return compress_impl(L, K, V, plan, o, UT, UF, stream, out);
+}
+
+// ------------------------------------------------------------------ decompress
+extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void *Kout, void *Vout, void *stream) {
+  if (!H || !Kout || !Vout) return fail(JOLT_EINVAL, "null argument");
+  int rc;
+  if ((rc = check_layout(L))) return rc;
+  if (L->n_layers != H->n_layers || L->n_kv_heads != H->n_kv_heads || L->seq_len != H->T || L->n_groups != H->n_groups)
+    return fail(JOLT_EINVAL, "output layout does not match the compressed cache");
+  for (int g = 0; g <= L->n_groups; ++g)
+    if (L->group_start[g] != H->group_start[g]) return fail(JOLT_EINVAL, "output grouping does not match");
+  cudaStream_t st = (cudaStream_t)stream;
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
+  if (dev != H->device) return fail(JOLT_EINVAL, "handle belongs to device %d, current device is %d", H->device, dev);
+  const int nc = (int)H->cells.size();
+  const size_t esz = L->dtype == JOLT_F16 ? 2 : 4;
+  const size_t span = layout_span_elems(L) * esz;
+  const bool fast = g_fast.load() != 0;
+  std::vector<CellWork> ws(nc);
+  void *ws_base = nullptr;
+  char *stage_K = nullptr, *stage_V = nullptr;
+  int *d_status = nullptr;
+  for (int pass = 0; pass < 2; ++pass) {
+    Bump b;
+    b.base = (char *)ws_base;
+    d_status = b.take<int>(4 * (size_t)nc);
+    if (L->mem_space == JOLT_MEM_HOST) { stage_K = b.take<char>(span); stage_V = b.take<char>(span); }
+    for (int i = 0; i < nc; ++i) {
+      ws[i].c = H->cells[i].c;
+      ws[i].active = false;
+      ws[i].status = d_status ? d_status + 4 * i : nullptr;
+      carve(b, ws[i], FM_INJECTED, !fast_decode_ok(ws[i].c, L, fast));
+    }
+    fast_carve_decode(b, ws, fast);
+    if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) return rc;
+  }
+  char *Kd = L->mem_space == JOLT_MEM_HOST ? stage_K : (char *)Kout;
+  char *Vd = L->mem_space == JOLT_MEM_HOST ? stage_V : (char *)Vout;
+  Program P;
+  std::vector<BackboneRef> br;
+  std::vector<RowJob> rj(nc);
+  long long rows = 0;
+  for (int i = 0; i < nc; ++i) {
+    const CellStore &cs = H->cells[i];
+    const CellDesc &c = cs.c;
+    if (c.r_t > 0) br.push_back({c, cs.G16, cs.UT16, cs.UF16, cs.e, ws[i].P16, ws[i].Xt});
+    RowJob &j = rj[i];
+    memset(&j, 0, sizeof j);
+    j.c = c; j.Xt = c.r_t > 0 ? ws[i].Xt : nullptr; j.words = cs.words; j.scales = cs.scales; j.status = d_status + 4 * i;
+    const int g = i / 2;
+    j.out = (i % 2 == 0 ? Kd : Vd) + (size_t)L->group_start[g] * L->stride_layer * esz;
+    j.out_dtype = L->dtype == JOLT_F16 ? DT_F16 : DT_F32;
+    j.osl = L->stride_layer; j.osh = L->stride_head; j.ost = L->stride_token;
+    j.row0 = rows;
+    rows += (long long)c.m * c.T;
+  }
+  if (!fast_decode(P, ws, br, rj, H, L, fast)) {
+    add_backbone(P, ST_DBACK, br);
+    const size_t off = P.push(rj);
+    const uint64_t seed = H->seed;
+    P.add(ST_DROWS, [=](char *dev_t, cudaStream_t s) {
+      dequant_add_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, s>>>((const RowJob *)(dev_t + off), nc, rows, seed);
+      LAUNCHED();
+    });
+  }
+  void *d_tab = nullptr;
+  if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
+  g_timer.begin(st);
+  CU(cudaMemsetAsync(d_status, 0, sizeof(int) * 4 * nc, st));
+  if ((rc = run_program(P, (char *)d_tab, st))) return rc;
+  if (L->mem_space == JOLT_MEM_HOST) {
+    CU(cudaMemcpyAsync(Kout, stage_K, span, cudaMemcpyDeviceToHost, st));
+    CU(cudaMemcpyAsync(Vout, stage_V, span, cudaMemcpyDeviceToHost, st));
+    g_timer.mark(ST_OUT, st);
+    CU(cudaStreamSynchronize(st));
+    g_timer.finish();
+  }
+  return JOLT_OK;
+}
+
+extern "C" int jolt_free(jolt_handle *H) {
+  if (!H) return JOLT_OK;
+  if (H->blob) {
+    int cur = 0;
+    cudaGetDevice(&cur);
+    if (cur != H->device) cudaSetDevice(H->device);
+    cudaFreeAsync(H->blob, 0);
+    if (cur != H->device) cudaSetDevice(cur);
+  }
+  delete H;
+  return JOLT_OK;
+}
+
+extern "C" int jolt_compressed_bytes(const jolt_handle *H, int64_t *bytes) {
+  if (!H || !bytes) return fail(JOLT_EINVAL, "null argument");
+  *bytes = H->stored_bytes;
+  return JOLT_OK;
+}
+
+extern "C" int jolt_get_component(const jolt_handle *H, int32_t cell, int32_t which, void *dst, int64_t cap, int64_t *written) {
+  if (!H || !written) return fail(JOLT_EINVAL, "null argument");
+  if (cell < 0 || cell >= (int)H->cells.size()) return fail(JOLT_EINVAL, "cell %d out of range", cell);
+  const CellStore &cs = H->cells[cell];
+  const CellDesc &c = cs.c;
+  const size_t M = (size_t)c.m * c.T * kD;
+  const void *src = nullptr;
+  size_t n = 0;
+  switch (which) {
+    case 0: src = cs.G16; n = 2 * (size_t)c.m * c.r_t * c.r_f; break;
+    case 1: src = cs.UT16; n = 2 * (size_t)c.T * c.r_t; break;
+    case 2: src = cs.UF16; n = 2 * (size_t)kD * c.r_f; break;
+    case 3: src = cs.words; n = 4 * (M / 32 * c.bits); break;
+    case 4: src = cs.scales; n = c.bits ? 2 * (M / 32) : 0; break;
+    case 5: src = cs.e; n = 4; break;
+    case 6: src = cs.sigma; n = 4 * (size_t)cs.n_sigma; break;
+    case 7: src = cs.lam; n = 4 * (size_t)kD; break;
+    default: return fail(JOLT_EINVAL, "component %d", which);
+  }
+  *written = (int64_t)n;
+  if (!dst) return JOLT_OK;
+  if ((int64_t)n > cap) return fail(JOLT_EINVAL, "destination holds %lld bytes, component has %zu", (long long)cap, n);
+  if (n) CU(cudaMemcpy(dst, src, n, cudaMemcpyDeviceToHost));
+  return JOLT_OK;
+}
+
+// ------------------------------------------------------------------ plan
+static void fill_defaults(jolt_options *o) {
+  memset(o, 0, sizeof *o);
+  o->token_mode = JOLT_TOKEN_RANDOMIZED; o->oversample = 10; o->power_iters = 1; o->quant_group = kGroup; o->seed = 0;
+  o->bits_set = nullptr; o->n_bits = 0; o->rank_step = 16; o->r_t_min = 16; o->r_f_min = 16; o->q_cap = 0; o->eps2 = nullptr;
+  o->count_scale_bytes = 1;
+}
+extern "C" void jolt_default_options(jolt_options *o) { if (o) fill_defaults(o); }
+
+extern "C" int64_t jolt_cell_bytes(int32_t m, int32_t T, int32_t d, int32_t r_t, int32_t r_f, int32_t bits, int32_t scales) {
+  return cell_bytes(m, T, d, r_t, r_f, bits, scales != 0);
+}
+extern "C" int32_t jolt_cap_policy(int32_t T, double ratio) { return cap_policy(T, ratio); }
+
+static const double *builtin_eps2() {
+  static double tab[9];
+  static std::once_flag once;
+  std::call_once(once, [] { eps2_calibration(tab); });
+  return tab;
+}
+extern "C" int jolt_eps2_table(double out[9]) {
+  if (!out) return fail(JOLT_EINVAL, "null argument");
+  memcpy(out, builtin_eps2(), sizeof(double) * 9);
+  return JOLT_OK;
+}
+
+extern "C" int jolt_allocate(int32_t n_cells, const int32_t *m, int32_t T, int32_t d, const double *lam3, const double *sig2sq,
+                             const int64_t *sig2_off, const int32_t *sig2_len, const double *total_sq, const int32_t *r_t_max,
+                             double budget, const jolt_options *o, jolt_cell_plan *out, double *achieved) {
+  if (n_cells <= 0 || !m || !lam3 || !sig2sq || !sig2_off || !sig2_len || !total_sq || !r_t_max || !o || !out)
+    return fail(JOLT_EINVAL, "null argument");
+  if (d != kD) return fail(JOLT_EUNSUPPORTED, "head_dim %d", d);
+  static const int32_t def_bits[4] = {0, 2, 4, 8};
+  const int32_t *bits = o->bits_set ? o->bits_set : def_bits;
+  const int nb = o->bits_set ? o->n_bits : 4;
+  if (nb <= 0) return fail(JOLT_EINVAL, "empty bits set");
+  for (int i = 0; i < nb; ++i) if (!bits_ok(bits[i])) return fail(JOLT_EINVAL, "bits %d", bits[i]);
+  const int step = o->rank_step > 0 ? o->rank_step : 16;
+  const int rt0 = o->r_t_min > 0 ? o->r_t_min : step, rf0 = o->r_f_min > 0 ? o->r_f_min : step;
+  const double *eps2 = o->eps2 ? o->eps2 : builtin_eps2();
+  std::vector<CellOptions> cells(n_cells);
+  for (int c = 0; c < n_cells; ++c) {
+    const double *l3 = lam3 + (size_t)c * kD;
+    const double *s2 = sig2sq + sig2_off[c];
+    const int ns = sig2_len[c];
+    if (!(total_sq[c] > 0)) return fail(JOLT_EINVAL, "cell %d has zero energy", c);
+    for (int rt = rt0; rt <= r_t_max[c]; rt += step) {
+      double t2 = 0;
+      for (int i = rt; i < ns; ++i) t2 += s2[i];
+      for (int rf = rf0; rf <= kD; rf += step) {
+        if (rt > m[c] * rf) continue;
+        double t3 = 0;
+        for (int i = rf; i < kD; ++i) t3 += l3[i];
+        const double tau = std::min(1.0, (t2 + t3) / total_sq[c]);
+        for (int bi = 0; bi < nb; ++bi) {
+          cells[c].err.push_back(eps2[bits[bi]] * tau);
+          cells[c].cost.push_back((double)cell_bytes(m[c], T, d, rt, rf, bits[bi], o->count_scale_bytes != 0));
+          cells[c].trip.push_back({rt, rf, bits[bi]});
+        }
+      }
+    }
+    if (cells[c].err.empty()) return fail(JOLT_EINVAL, "cell %d: empty rank grid (r_t_max %d)", c, r_t_max[c]);
+  }
+  std::vector<size_t> choice;
+  double total = 0;
+  const bool ok = dual_allocate(cells, budget, choice, total);
+  for (int c = 0; c < n_cells; ++c) out[c] = cells[c].trip[choice[c]];
+  if (achieved) *achieved = total;
+  return ok ? JOLT_OK : fail(JOLT_EBUDGET, "cheapest allocation needs %.0f bytes, budget is %.0f", total, budget);
+}
+
+extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, double budget, const jolt_options *o, void *stream,
+                         jolt_cell_plan *out, double *achieved) {
+  if (!out || !K || !V) return fail(JOLT_EINVAL, "null argument");
+  int rc;
+  if ((rc = check_layout(L)) || (rc = check_options(o))) return rc;
+  if (!(budget > 0)) return fail(JOLT_EINVAL, "byte budget must be positive");
+  cudaStream_t st = (cudaStream_t)stream;
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
+  const double raw = 2.0 * 2.0 * (double)L->n_layers * L->n_kv_heads * L->seq_len * kD;
+  const int nc = 2 * L->n_groups;
+  const bool exact = o->token_mode == JOLT_TOKEN_EXACT;
+  if (exact && L->seq_len > 1024) return fail(JOLT_EUNSUPPORTED, "exact token spectra are built for T <= 1024 (got %d)", L->seq_len);
+  const int q_cap = o->q_cap > 0 ? o->q_cap : cap_policy(L->seq_len, raw / budget);
+  std::vector<jolt_cell_plan> probe(nc);
+  std::vector<CellDesc> cells;
+  for (int i = 0; i < nc; ++i) {
+    const int m = (L->group_start[i / 2 + 1] - L->group_start[i / 2]) * L->n_kv_heads;
+    const int lim = std::min(L->seq_len, m * kD);
+    probe[i] = {exact ? lim : std::min(q_cap, lim), kD, 0};
+  }
+  make_cells(L, K, V, probe.data(), o->oversample, cells);
+  if (exact) for (auto &c : cells) c.k = c.r_t;
+  const int mode = exact ? FM_EXACT : FM_RANDOMIZED;
+  const size_t esz = L->dtype == JOLT_F16 ? 2 : 4;
+  const size_t span = layout_span_elems(L) * esz;
+  const bool fast = g_fast.load() != 0;
+  std::vector<CellWork> ws(nc);
+  void *ws_base = nullptr;
+  int *d_status = nullptr;
+  char *stage_K = nullptr, *stage_V = nullptr;
+  for (int pass = 0; pass < 2; ++pass) {
+    Bump b;
+    b.base = (char *)ws_base;
+    d_status = b.take<int>(4 * (size_t)nc);
+    if (L->mem_space == JOLT_MEM_HOST) { stage_K = b.take<char>(span); stage_V = b.take<char>(span); }
+    for (int i = 0; i < nc; ++i) {
+      ws[i].c = cells[i]; ws[i].active = true; ws[i].status = d_status ? d_status + 4 * i : nullptr;
+      ws[i].lam = nullptr; ws[i].sigma = nullptr;
+      carve(b, ws[i], mode, false);
+    }
+    fast_carve(b, ws, fast);
+    if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) return rc;
+  }
+  if (L->mem_space == JOLT_MEM_HOST)
+    for (int i = 0; i < nc; ++i) {
+      const char *hb = (const char *)(i % 2 == 0 ? K : V);
+      ws[i].c.X = (i % 2 == 0 ? stage_K : stage_V) + ((const char *)ws[i].c.X - hb);
+    }
+  Program P;
+  build_factor_program(P, ws, mode, true, o->power_iters, o->seed, fast);
+  void *d_tab = nullptr;
+  if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
+  g_timer.begin(st);
+  CU(cudaMemsetAsync(d_status, 0, sizeof(int) * 4 * nc, st));
+  if (L->mem_space == JOLT_MEM_HOST) {
+    CU(cudaMemcpyAsync(stage_K, K, span, cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(stage_V, V, span, cudaMemcpyHostToDevice, st));
+  }
+  if ((rc = run_program(P, (char *)d_tab, st))) return rc;
+  std::vector<int> hstat(4 * nc);
+  std::vector<float> lam((size_t)nc * kD);
+  std::vector<std::vector<float>> sig(nc);
+  CU(cudaMemcpyAsync(hstat.data(), d_status, sizeof(int) * 4 * nc, cudaMemcpyDeviceToHost, st));
+  for (int i = 0; i < nc; ++i) {
+    sig[i].resize(ws[i].n_sigma);
+    CU(cudaMemcpyAsync(lam.data() + (size_t)i * kD, ws[i].lam, sizeof(float) * kD, cudaMemcpyDeviceToHost, st));
+    CU(cudaMemcpyAsync(sig[i].data(), ws[i].sigma, sizeof(float) * ws[i].n_sigma, cudaMemcpyDeviceToHost, st));
+  }
+  CU(cudaStreamSynchronize(st));
+  g_timer.finish();
+  if ((rc = status_to_code(hstat))) return rc;
+  // spectra -> allocator inputs (tail-mass accounting of Sec. 5 for the randomized probe)
+  std::vector<double> lam3((size_t)nc * kD), s2all, total(nc);
+  std::vector<int64_t> off(nc);
+  std::vector<int32_t> len(nc), mm(nc), rtmax(nc);
+  for (int i = 0; i < nc; ++i) {
+    double tot = 0;
+    for (int j = 0; j < kD; ++j) { lam3[(size_t)i * kD + j] = lam[(size_t)i * kD + j]; tot += lam[(size_t)i * kD + j]; }
+    total[i] = tot;
+    off[i] = (int64_t)s2all.size();
+    const int keep = exact ? (int)sig[i].size() : std::min((int)sig[i].size(), cells[i].r_t);
+    double acc = 0;
+    for (int j = 0; j < keep; ++j) { const double v = (double)sig[i][j] * sig[i][j]; s2all.push_back(v); acc += v; }
+    if (!exact) s2all.push_back(std::max(0.0, tot - acc));
+    len[i] = keep + (exact ? 0 : 1);
+    mm[i] = cells[i].m;
+    rtmax[i] = cells[i].r_t;
+  }
+  return jolt_allocate(nc, mm.data(), L->seq_len, kD, lam3.data(), s2all.data(), off.data(), len.data(), total.data(),
+                       rtmax.data(), budget, o, out, achieved);
+}
+
+// ------------------------------------------------------------------ misc exports
+extern "C" int jolt_sketch_host(uint64_t seed, int32_t cell, int32_t stream_id, int64_t n_rows, int32_t n_cols, float *out) {
+  if (!out || n_rows < 0 || n_cols < 0) return fail(JOLT_EINVAL, "bad argument");
+  const uint64_t base = stream_base(seed, cell, stream_id);
+  for (int64_t i = 0; i < n_rows * n_cols; ++i) out[i] = (float)gaussian_from_u64(mix64(base + (uint64_t)i));
+  return JOLT_OK;
+}
+extern "C" int jolt_signs_host(uint64_t seed, int32_t cell, float out[128]) {
+  if (!out) return fail(JOLT_EINVAL, "null argument");
+  const uint64_t base = stream_base(seed, cell, STREAM_SIGNS);
+  const uint64_t w[2] = {mix64(base + 0), mix64(base + 1)};
+  for (int f = 0; f < 128; ++f) out[f] = ((w[f / 64] >> (f % 64)) & 1) ? -1.f : 1.f;
+  return JOLT_OK;
+}
+extern "C" int jolt_release_workspace(void) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return JOLT_OK; }
+  std::lock_guard<std::mutex> lk(g_ws_mu);
+  cudaDeviceSynchronize();
+  if (g_ws[dev].base) { cudaFree(g_ws[dev].base); g_ws[dev] = Workspace(); }
+  if (g_tab[dev].base) { cudaFree(g_tab[dev].base); g_tab[dev] = Workspace(); }
+  return JOLT_OK;
+}
+extern "C" int64_t jolt_launch_count(void) { return g_launches.load(); }
+extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled ? 1 : 0); }
+extern "C" int jolt_last_stage_ms(float *out, int32_t cap, int32_t *n) {
+  if (!out || !n) return fail(JOLT_EINVAL, "null argument");
+  *n = std::min<int>(cap, kNumStages);
+  for (int i = 0; i < *n; ++i) out[i] = g_timer.ms[i];
+  return JOLT_OK;
+}
+extern "C" const char *jolt_stage_name(int32_t i) { return (i >= 0 && i < kNumStages) ? kStageNames[i] : ""; }
+extern "C" const char *jolt_strerror(int s) {
+  switch (s) {
+    case JOLT_OK: return "ok";
+    case JOLT_EINVAL: return "invalid argument";
+    case JOLT_EUNSUPPORTED: return "not supported by this build";
+    case JOLT_EBUDGET: return "byte budget below the cheapest allocation";
+    case JOLT_ENUMERIC: return "numerical failure";
+    case JOLT_ENOMEM: return "out of memory";
+    case JOLT_ECUDA: return "CUDA error";
+    case JOLT_ETIMEOUT: return "bounded device wait ran out";
+    default: return "unknown status";
+  }
+}
+extern "C" const char *jolt_last_error(void) { return g_err.c_str(); }

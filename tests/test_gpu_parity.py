@@ -1,0 +1,253 @@
+"""GPU-vs-oracle parity through the C ABI (run with -m gpu on a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import __graft_entry__ as entry
+from oracle import jolt_oracle as O
+from tests.helpers import cell_view, code_mismatch, oracle_cache, projector_distance
+
+pytestmark = pytest.mark.gpu
+
+REL_RECON = 1e-3       # ||X^_gpu - X^_oracle||_F / ||X^_oracle||_F
+REL_ERR = 0.02         # per-tensor reconstruction error within 2 % of the oracle's
+PROJ = 1e-3            # || U U^T - U0 U0^T ||_F
+CODE_FRAC = 1e-3       # fraction of codes allowed to differ (by exactly 1)
+
+
+@pytest.fixture(scope="module")
+def B():
+    entry.build()
+    import paper_2607_12550_b200 as pkg
+    return pkg.load()
+
+
+@pytest.fixture(scope="module")
+def synth():
+    from paper_2607_12550_b200 import synth as s
+    return s
+
+
+def _np(t):
+    return t.detach().cpu().numpy()
+
+
+def _roundtrip(B, K, V, gs, plans, opts, factors=None):
+    h = B.jolt_compress(K, V, gs, plans, opts, factors=factors)
+    Ko, Vo = torch.empty_like(K), torch.empty_like(V)
+    B.jolt_decompress(h, Ko, Vo, gs)
+    torch.cuda.synchronize()
+    return h, Ko, Vo
+
+
+def _check_recon(Knp, Vnp, Ko, Vo, gs, ocells, tag=""):
+    for c, oc in enumerate(ocells):
+        X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
+        Xg = cell_view(_np(Ko), _np(Vo), gs, c).astype(np.float64)
+        Xo = O.decompress_cell(oc)
+        rel = np.linalg.norm(Xg - Xo) / np.linalg.norm(Xo)
+        eg, eo = O.rel_frobenius(X, Xg), O.rel_frobenius(X, Xo)
+        assert rel <= REL_RECON, (tag, c, rel)
+        assert abs(eg - eo) <= REL_ERR * eo + 1e-7, (tag, c, eg, eo)
+
+
+def _stored_codes(B, h, c, bits):
+    words = h.component(c, 3)
+    return O.unpack_codes(words.reshape(-1, 4 * bits), bits, 128), words.reshape(-1, 4 * bits)
+
+
+# --------------------------------------------------------------------------- rotated quantiser alone (rank-0 mode)
+@pytest.mark.parametrize("bits", [1, 2, 3, 4, 8])
+@pytest.mark.parametrize("dtype", [torch.float16, torch.float32])
+def test_rank0_codes_scales_and_packing(B, bits, dtype):
+    g = torch.Generator().manual_seed(100 + bits)
+    L, nh, T = 3, 2, 384          # ragged: 3 layers in groups of 2 + 1
+    K = (torch.randn(L, nh, T, 128, generator=g) * torch.exp(torch.randn(L, nh, T, 1, generator=g))).to(dtype)
+    V = torch.randn(L, nh, T, 128, generator=g).to(dtype)
+    V[..., 7] *= 30.0
+    V[1, 0, 5] = 0.0              # an all-zero row: zero step, mid codes
+    gs = [0, 2, 3]
+    plans = [(0, 0, bits)] * 4
+    opts = B.default_options(seed=42)
+    h, Ko, Vo = _roundtrip(B, K.cuda(), V.cuda(), gs, plans, opts)
+    Knp, Vnp = _np(K), _np(V)
+    oc = oracle_cache(Knp, Vnp, gs, plans, seed=42, token_mode="randomized",
+                      out_dtype="f16" if dtype == torch.float16 else "f32")
+    assert h.bytes() == sum(O.stored_bytes(o.m, o.T, 128, 0, 0, bits) for o in oc)
+    for c, o in enumerate(oc):
+        codes, words = _stored_codes(B, h, c, bits)
+        ref = o.ideal["codes"].reshape(-1, 128)
+        frac, mx = code_mismatch(codes, ref)
+        assert frac <= CODE_FRAC and mx <= 1, (c, frac, mx)
+        # packing is bit-exact: the oracle's packer applied to the library's codes gives the library's words
+        assert np.array_equal(O.pack_codes(codes, bits), words)
+        sc = h.component(c, 4).reshape(-1, 4)
+        sref = o.scales.reshape(-1, 4)
+        assert (sc.view(np.uint16) != sref.view(np.uint16)).mean() <= CODE_FRAC
+    _check_recon(Knp, Vnp, Ko, Vo, gs, oc, f"rank0 b{bits}")
+    h.free()
+
+
+# --------------------------------------------------------------------------- residual against injected factors
+@pytest.mark.parametrize("bits", [2, 4])
+def test_injected_factors_codes_match(B, synth, bits):
+    cfg = synth.CacheConfig("t", 2, 2, 2, 256, n_terms=20, seed=21)
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2]
+    plans = [(16, 32, bits), (24, 128, bits)]
+    Knp, Vnp = _np(K), _np(V)
+    UT, UF = [], []
+    for c, (rt, rf, _) in enumerate(plans):
+        o = O.compress_cell(cell_view(Knp, Vnp, gs, c), rt, rf, 0, token_mode="exact")
+        UT.append(o.UT16.astype(np.float32)); UF.append(o.UF16.astype(np.float32))
+    opts = B.default_options(seed=3)
+    h, Ko, Vo = _roundtrip(B, K, V, gs, plans, opts, factors=(UT, UF))
+    oc = oracle_cache(Knp, Vnp, gs, plans, seed=3, token_mode="exact", factors=(UT, UF))
+    for c, o in enumerate(oc):
+        assert np.array_equal(h.component(c, 1).astype(np.float32).reshape(o.UT16.shape), o.UT16.astype(np.float32))
+        G = h.component(c, 0).astype(np.float64).reshape(o.Gs16.shape) * 2.0 ** int(h.component(c, 5)[0])
+        Go = o.Gs16 * 2.0 ** o.e
+        assert np.linalg.norm(G - Go) <= 1e-3 * np.linalg.norm(Go)
+        codes, words = _stored_codes(B, h, c, bits)
+        frac, mx = code_mismatch(codes, o.ideal["codes"].reshape(-1, 128))
+        assert frac <= 5e-3 and mx <= 1, (c, frac, mx)   # core rounding differences move a few thresholds
+        assert np.array_equal(O.pack_codes(codes, bits), words)
+    _check_recon(Knp, Vnp, Ko, Vo, gs, oc, "injected")
+    h.free()
+
+
+# --------------------------------------------------------------------------- config 0: tiny single group, fp32
+@pytest.mark.parametrize("token_mode", ["randomized", "exact"])
+def test_config0(B, synth, token_mode):
+    cfg = synth.CONFIGS["c0"]
+    K, V = synth.make_cache(cfg, device="cuda")
+    assert K.dtype == torch.float32 and tuple(K.shape) == (1, 8, 512, 128)
+    gs = [0, 1]
+    plans = [(64, 64, 2), (64, 64, 2)]
+    opts = B.default_options(seed=0, oversample=10, power_iters=1,
+                             token_mode=B.TOKEN_EXACT if token_mode == "exact" else B.TOKEN_RANDOMIZED)
+    h, Ko, Vo = _roundtrip(B, K, V, gs, plans, opts)
+    Knp, Vnp = _np(K), _np(V)
+    oc = oracle_cache(Knp, Vnp, gs, plans, seed=0, token_mode=token_mode, out_dtype="f32")
+    _check_recon(Knp, Vnp, Ko, Vo, gs, oc, "c0 " + token_mode)
+    for c, o in enumerate(oc):
+        X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
+        UF = h.component(c, 2).astype(np.float64).reshape(128, 64)
+        UT = h.component(c, 1).astype(np.float64).reshape(512, 64)
+        lam = o.ideal["lam"]
+        gap_f = (lam[63] - lam[64]) / lam[0]
+        assert gap_f > 1e-4
+        assert projector_distance(UF, o.UF16) <= PROJ, (c, "U_F")
+        sig = o.ideal["sigma"]
+        gap_t = (sig[63] - sig[64]) / sig[0]
+        if gap_t > 1e-2:
+            assert projector_distance(UT, o.UT16) <= PROJ, (c, "U_T", gap_t)
+        else:
+            # gapless spectrum at r_t (keys with amplified noise channels): the subspace is not unique to
+            # tolerance; compare the energy the two token factors capture instead
+            Y = np.einsum("htf,fs->hts", X, o.ideal["U_F"])
+            A = O.token_unfold(Y)
+            eg, eo = np.linalg.norm(UT.T @ A) ** 2, np.linalg.norm(o.UT16.T @ A) ** 2
+            assert abs(eg - eo) <= 1e-4 * eo, (c, eg, eo, gap_t)
+        # stored singular values / eigenvalues
+        ks = len(h.component(c, 6))
+        assert np.allclose(h.component(c, 6)[:64], sig[:64], rtol=1e-4)
+        assert np.allclose(h.component(c, 7), lam, rtol=1e-4, atol=1e-5 * lam[0])
+    h.free()
+
+
+# --------------------------------------------------------------------------- fp16 multi-group cache, several tiles
+@pytest.mark.parametrize("bits_k,bits_v", [(4, 8), (0, 3), (1, 2)])
+def test_small_gqa_cache(B, synth, bits_k, bits_v):
+    cfg = synth.CacheConfig("t", 4, 2, 4, 640, n_terms=40, seed=33)     # T = 5 tiles of 128, m = 8
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2, 4]
+    plans = [(48, 128, bits_k), (40, 112, bits_v), (32, 96, bits_k), (56, 128, bits_v)]
+    opts = B.default_options(seed=77, power_iters=2)
+    h, Ko, Vo = _roundtrip(B, K, V, gs, plans, opts)
+    Knp, Vnp = _np(K), _np(V)
+    oc = oracle_cache(Knp, Vnp, gs, plans, seed=77, token_mode="randomized", power_iters=2)
+    assert h.bytes() == sum(O.stored_bytes(o.m, o.T, 128, o.r_t, o.r_f, o.bits) for o in oc)
+    _check_recon(Knp, Vnp, Ko, Vo, gs, oc, "small gqa")
+    for c, o in enumerate(oc):
+        UT = h.component(c, 1).astype(np.float64).reshape(o.UT16.shape)
+        sig = o.ideal["sigma"]
+        rt = o.r_t
+        if (sig[rt - 1] - sig[rt]) / sig[0] > 1e-2:
+            assert projector_distance(UT, o.UT16) <= PROJ, c
+    h.free()
+
+
+def test_strided_layout_and_host_memory(B, synth):
+    cfg = synth.CacheConfig("t", 2, 1, 2, 256, n_terms=16, seed=5)
+    K, V = synth.make_cache(cfg, device="cpu")
+    gs = [0, 1, 2]
+    plans = [(16, 64, 4)] * 4
+    opts = B.default_options(seed=1)
+    # device tensors with padded token stride
+    Kp = torch.zeros(2, 2, 256, 160, dtype=torch.float16, device="cuda")[..., :128]
+    Vp = torch.zeros(2, 2, 256, 160, dtype=torch.float16, device="cuda")[..., :128]
+    Kp.copy_(K); Vp.copy_(V)
+    h1, Ko1, Vo1 = _roundtrip(B, Kp, Vp, gs, plans, opts)
+    # host tensors: the library stages the copies
+    Kh, Vh = K.pin_memory(), V.pin_memory()
+    h2 = B.jolt_compress(Kh, Vh, gs, plans, opts)
+    Ko2, Vo2 = torch.empty_like(Kh), torch.empty_like(Vh)
+    B.jolt_decompress(h2, Ko2, Vo2, gs)
+    assert torch.equal(Ko1.cpu(), Ko2) and torch.equal(Vo1.cpu(), Vo2)
+    oc = oracle_cache(_np(K), _np(V), gs, plans, seed=1, token_mode="randomized")
+    _check_recon(_np(K), _np(V), Ko2, Vo2, gs, oc, "host")
+    h1.free(); h2.free()
+
+
+def test_exact_low_rank_input_and_rank_deficient_sketch(B):
+    # exactly rank-(6, 9) input with sketch width 6 + 10 > rank: dead pivots in CholeskyQR must deflate
+    rng = np.random.default_rng(0)
+    G = rng.standard_normal((4, 6, 9)); UT = np.linalg.qr(rng.standard_normal((256, 6)))[0]
+    UF = np.linalg.qr(rng.standard_normal((128, 9)))[0]
+    X = np.einsum("hrs,tr,fs->htf", G, UT, UF) * 8
+    K = torch.tensor(X, dtype=torch.float32).reshape(2, 2, 256, 128).cuda()
+    V = K.clone()
+    gs = [0, 2]
+    plans = [(6, 9, 0), (6, 9, 4)]
+    opts = B.default_options(seed=4, power_iters=1)
+    h, Ko, Vo = _roundtrip(B, K, V, gs, plans, opts)
+    Xk = _np(Ko).reshape(4, 256, 128).astype(np.float64)
+    Xv = _np(Vo).reshape(4, 256, 128).astype(np.float64)
+    Xin = _np(K).reshape(4, 256, 128).astype(np.float64)
+    assert O.rel_frobenius(Xin, Xk) < 2e-3          # fp16 storage of factors and core only
+    assert O.rel_frobenius(Xin, Xv) < 2e-4          # residual absorbs the storage rounding
+    h.free()
+
+
+def test_plan_spectra_and_allocation(B, synth):
+    cfg = synth.CacheConfig("t", 4, 2, 2, 512, n_terms=48, seed=8)      # m = 4, T = 512
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2, 4]
+    raw = 2 * K.numel() * 2
+    opts = B.default_options(seed=6, power_iters=1)
+    plans, ach = B.jolt_plan(K, V, gs, raw / 2.0, opts)
+    assert ach <= raw / 2.0
+    # oracle: same probe (seeded), same dual
+    Knp, Vnp = _np(K), _np(V)
+    q_cap = O.cap_policy(512, 2.0)
+    eps2 = O.eps2_table([0, 2, 4, 8])
+    cells, trips = [], []
+    for c in range(4):
+        X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
+        lam, s2, tot = O.plan_spectra(X, q_cap, seed=6, cell=c, power_iters=1)
+        rt_grid, rf_grid = list(range(16, q_cap + 1, 16)), list(range(16, 129, 16))
+        tau = O.tau_table(lam, s2, tot, rt_grid, rf_grid)
+        e, s, t = O.cell_options(4, 512, 128, tau, rt_grid, rf_grid, [0, 2, 4, 8], eps2)
+        cells.append((e, s)); trips.append(t)
+    ch, cost, lam_star, ok = O.dual_allocate(cells, raw / 2.0)
+    ref = [trips[c][i] for c, i in enumerate(ch)]
+    # fp32 spectra can flip near-ties; the achieved error of the two plans must agree closely
+    e_ref = sum(cells[c][0][ch[c]] for c in range(4))
+    e_got = sum(cells[c][0][trips[c].index(tuple(plans[c]))] for c in range(4))
+    assert abs(e_got - e_ref) <= 1e-3 * e_ref + 1e-9, (plans, ref)
+    assert sum(p == r for p, r in zip(plans, ref)) >= 3, (plans, ref)
+    # and the planned cache really compresses to the planned size
+    h = B.jolt_compress(K, V, gs, plans, opts)
+    assert h.bytes() == ach
+    h.free()
