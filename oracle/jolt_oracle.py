@@ -261,6 +261,19 @@ def token_factor_randomized(A, r_t: int, Omega, power_iters: int):
     return Q @ Ut[:, :r_t], s, Q, Ut, B
 
 
+def projected_sketch(seed: int, cell: int, U_F, m: int, k: int, stream: int = STREAM_SKETCH):
+    """Test matrix of the range finder, Omega in R^{(m r_f) x k}.
+
+    The Gaussian is drawn in the ORIGINAL feature coordinates, Omega' in R^{(m d) x k} (row h*d + f),
+    and carried into the coordinates of the projected tensor: Omega_h = U_F^T Omega'_h.  U_F has
+    orthonormal columns, so Omega is again i.i.d. Gaussian; and A Omega = sum_h X_h (U_F U_F^T) Omega'_h
+    depends on U_F only through its projector, i.e. not on the sign or ordering the eigen-solver
+    happened to give the feature basis."""
+    d = U_F.shape[0]
+    Op = gaussian_sketch(seed, cell, m * d, k, stream=stream).reshape(m, d, k)
+    return np.einsum("fs,hfk->hsk", U_F, Op, optimize=True).reshape(m * U_F.shape[1], k)
+
+
 def sketch_width(r_t: int, oversample: int, T: int, N: int):
     return min(r_t + oversample, T, N)
 
@@ -340,7 +353,7 @@ def compress_cell(X, r_t: int, r_f: int, bits: int, *, seed: int = 0, cell: int 
                 U_T, sig = token_factor_exact(A, r_t)
             elif token_mode == "randomized":
                 k = sketch_width(r_t, oversample, T, N)
-                Omega = gaussian_sketch(seed, cell, N, k)
+                Omega = projected_sketch(seed, cell, U_F, m, k)
                 U_T, sig, _, _, _ = token_factor_randomized(A, r_t, Omega, power_iters)
             else:
                 raise ValueError(token_mode)
@@ -524,7 +537,7 @@ def plan_spectra(X, q_cap: int, *, seed: int = 0, cell: int = 0, oversample: int
         s = np.linalg.svd(A, compute_uv=False)
         return lam, s ** 2, total
     k = sketch_width(q_cap, oversample, T, A.shape[1])
-    Omega = gaussian_sketch(seed, cell, A.shape[1], k, stream=STREAM_PROBE)
+    Omega = projected_sketch(seed, cell, np.eye(d), m, k, stream=STREAM_PROBE)
     _, s, _, _, _ = token_factor_randomized(A, q_cap, Omega, power_iters)
     spec = tail_mass_spectrum(s[:q_cap], total)
     return lam, spec ** 2, total

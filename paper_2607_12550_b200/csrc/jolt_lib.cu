@@ -305,7 +305,7 @@ struct CellWork {      // device scratch of one cell
   bool active = false;       // has a backbone to compute
   double *gram_part = nullptr, *C = nullptr, *Cv = nullptr, *Cw = nullptr;
   float *UF32 = nullptr, *lam = nullptr;
-  float *omega = nullptr, *W = nullptr, *S = nullptr, *S2 = nullptr, *Zp = nullptr, *Z = nullptr, *Z2 = nullptr;
+  float *omega = nullptr, *PF = nullptr, *W = nullptr, *S = nullptr, *S2 = nullptr, *Zp = nullptr, *Z = nullptr, *Z2 = nullptr;
   double *Gs = nullptr, *Linv = nullptr; float *LinvT = nullptr;
   double *BBt = nullptr, *BBv = nullptr, *BBw = nullptr;
   float *Ut = nullptr, *sigma = nullptr;
@@ -336,7 +336,8 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
       w.C = b.take<double>(kD * kD); w.Cv = b.take<double>(kD * kD); w.Cw = b.take<double>(kD);
     }
     if (mode == FM_RANDOMIZED) {
-      w.omega = b.take<float>(N * k);
+      w.omega = b.take<float>((size_t)c.m * kD * k);
+      w.PF = b.take<float>(kD * kD);
       w.W = b.take<float>((size_t)c.m * kD * k);
       w.S = b.take<float>(T * k); w.S2 = b.take<float>(T * k);
       w.Z = b.take<float>(N * k); w.Z2 = b.take<float>(N * k);
@@ -380,22 +381,34 @@ void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side)
   }
 }
 
-// W_h = U_F R_h for every head (R = Omega or Z, N x k row blocks of r_f), then S = sum_h X_h W_h.
+// S = sum_h X_h W_h.  First sketch: W_h = (U_F U_F^T) Omega'_h with the Gaussian Omega' drawn in the
+// original feature coordinates (W_h = Omega'_h when r_f = d).  Power iteration: W_h = U_F Z_h.
 void add_sketch(Program &P, int stage, std::vector<CellWork> &ws, bool from_omega) {
-  std::vector<GemmTask> g1, g2;
+  std::vector<GemmTask> g0, g1, g2;
   for (auto &w : ws) {
     if (!w.active) continue;
     const CellDesc &c = w.c;
-    const float *R = from_omega ? w.omega : w.Z;
-    for (int h = 0; h < c.m; ++h)
-      g1.push_back(mk(w.UF32, DT_F32, c.r_f, 1, R + (size_t)h * c.r_f * c.k, DT_F32, c.k, 1,
-                      w.W + (size_t)h * kD * c.k, DT_F32, c.k, kD, c.k, c.r_f));
-    GemmTask t = mk(c.X, c.dtype, c.st, 1, w.W, DT_F32, c.k, 1, w.S, DT_F32, c.k, c.T, c.k, kD);
+    const float *Wsrc = w.W;
+    if (from_omega) {
+      if (c.r_f == kD) Wsrc = w.omega;
+      else {
+        g0.push_back(mk(w.UF32, DT_F32, c.r_f, 1, w.UF32, DT_F32, 1, c.r_f, w.PF, DT_F32, kD, kD, kD, c.r_f));
+        for (int h = 0; h < c.m; ++h)
+          g1.push_back(mk(w.PF, DT_F32, kD, 1, w.omega + (size_t)h * kD * c.k, DT_F32, c.k, 1,
+                          w.W + (size_t)h * kD * c.k, DT_F32, c.k, kD, c.k, kD));
+      }
+    } else {
+      for (int h = 0; h < c.m; ++h)
+        g1.push_back(mk(w.UF32, DT_F32, c.r_f, 1, w.Z + (size_t)h * c.r_f * c.k, DT_F32, c.k, 1,
+                        w.W + (size_t)h * kD * c.k, DT_F32, c.k, kD, c.k, c.r_f));
+    }
+    GemmTask t = mk(c.X, c.dtype, c.st, 1, Wsrc, DT_F32, c.k, 1, w.S, DT_F32, c.k, c.T, c.k, kD);
     t.nseg = c.m; t.seg_inner = c.n_heads;
     t.a_so = c.sl; t.a_si = c.sh;
     t.b_so = (long long)c.n_heads * kD * c.k; t.b_si = (long long)kD * c.k;
     g2.push_back(t);
   }
+  add_gemm(P, stage, g0, false);
   add_gemm(P, stage, g1, false);
   add_gemm(P, stage, g2, false);
 }
@@ -426,7 +439,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
   const int na = (int)act.size();
   if (mode == FM_RANDOMIZED) {
     std::vector<CellDesc> cd; std::vector<float *> om; std::vector<long long> cnt;
-    for (int i : act) { cd.push_back(ws[i].c); om.push_back(ws[i].omega); cnt.push_back((long long)ws[i].c.N * ws[i].c.k); }
+    for (int i : act) { cd.push_back(ws[i].c); om.push_back(ws[i].omega); cnt.push_back((long long)ws[i].c.m * kD * ws[i].c.k); }
     const size_t o1 = P.push(cd), o2 = P.push(om), o3 = P.push(cnt);
     const int sid = probe ? STREAM_PROBE : STREAM_SKETCH;
     P.add(ST_SKGEN, [=](char *dev, cudaStream_t s) {
