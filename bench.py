@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of the JoLT hot path on B200: one step = compress + decompress of one whole synthetic KV cache.
+
+Workload (N = 1): the GQA-shaped cache of the headline metric (32 layers in groups of 4, 8 KV heads,
+T = 4096, d_h = 128, fp16, budget 2x, randomized token factor, q = 1), ranks and bits from jolt_plan.
+Prints ONE JSON line.  `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "KV compress+decompress GB/s of fp16 cache (2x budget)"
+UNIT = "GB/s"
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm": d["hbm_gbs"], "tensor": d["bf16_tflops"], "tensor_sustained": d.get("bf16_tflops_sustained"),
+                "source": "measured"}
+    return {"hbm": 6650.0, "tensor": 1590.0, "tensor_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    Q = "index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown," \
+        "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+        sm = sorted(int(r[1]) for r in self.rows if len(r) >= 9 and r[1].isdigit())
+        mx = [int(r[2]) for r in self.rows if len(r) >= 9 and r[2].isdigit()]
+        reasons = set()
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cell_work(m, T, d, r_t, r_f, bits, k, q, in_bytes_per_elt):
+    """Algorithmic flops / bytes of one cell (split-precision passes do not count)."""
+    M = m * T * d
+    X = M * in_bytes_per_elt
+    out = 2 * (m * r_t * r_f + T * r_t + d * r_f) + bits * M // 8 + (2 * M // 32 if bits else 0)
+    w = {}
+    w["gram"] = (2 * M * d, X)
+    w["sketch"] = (2 * M * k, X)
+    w["power"] = (4 * M * k * q, 2 * q * X)
+    w["project"] = (2 * M * k, X)
+    w["residual_quant"] = (2 * M * r_t, X + out)
+    w["compress"] = (2 * M * d + 2 * M * k * (2 + 2 * q) + 2 * M * r_t, (4 + 2 * q) * X + out)
+    w["compress_strict_bytes"] = X + out
+    w["decompress"] = (2 * M * r_t + 2 * m * r_t * r_f * d, 2 * M + out)
+    return w
+
+
+def roof_time(flops, nbytes, pk):
+    return max(flops / (pk["tensor"] * 1e12), nbytes / (pk["hbm"] * 1e9))
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on a bounded sample of the same workload (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import torch
+    from oracle import jolt_oracle as O
+    from paper_2607_12550_b200 import synth
+    cfg = synth.CONFIGS["c1"]
+    # sample: the K and the V cell of group 0, with plans typical of the 2x allocation
+    plans = {0: (128, 128, 4), 1: (112, 128, 8)}
+    cells = {w: synth.make_cell(cfg, 0, w).to(torch.float16).numpy() for w in (0, 1)}
+    cell_bytes = cells[0].size * 2
+    n_cells_total = 2 * cfg.n_groups
+
+    def step():
+        tc = td = 0.0
+        for w, X in cells.items():
+            t0 = time.perf_counter()
+            oc = O.compress_cell(X, *plans[w], seed=cfg.seed, cell=w, token_mode="randomized", power_iters=1)
+            t1 = time.perf_counter()
+            O.decompress_cell(oc)
+            t2 = time.perf_counter()
+            tc += t1 - t0
+            td += t2 - t1
+        return tc, td
+
+    for _ in range(args.warmup_ref):
+        step()
+    tcs, tds = [], []
+    for _ in range(args.steps):
+        a, b = step()
+        tcs.append(a); tds.append(b)
+    tc, td = sum(tcs) / len(tcs), sum(tds) / len(tds)
+    sample_bytes = 2 * cell_bytes
+    value = sample_bytes / (tc + td) / 1e9
+    cores = os.cpu_count()
+    try:
+        cores = torch.get_num_threads()
+    except Exception:
+        pass
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup_ref, "ms_per_step": (tc + td) * 1e3 * n_cells_total / 2, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "c1: GQA 32 layers / 4 per group, 8 KV heads, T=4096, d=128, fp16, 2x budget",
+                       "sample": "2 of 16 cells (group 0: K at (128,128,4), V at (112,128,8)); ms_per_step scaled to 16 cells"},
+            "compress_gbs": sample_bytes / tc / 1e9, "decompress_gbs": sample_bytes / td / 1e9,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": "group 0 K and V cells (2 of 16), numpy fp64"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="jolt", choices=["jolt", "reference"])
+    ap.add_argument("--workload", default="c1")
+    ap.add_argument("--groups", type=int, default=0, help="limit the number of layer groups (profiling captures)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--portable", action="store_true", help="portable SIMT kernels only")
+    args = ap.parse_args()
+    args.warmup_ref = min(args.warmup, 1)
+    if args.impl == "reference":
+        args.steps = min(args.steps, 3)
+        return run_reference(args)
+
+    import numpy as np
+    import torch
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2607_12550_b200 as pkg
+    B = pkg.load()
+    synth = pkg.synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if args.portable:
+        B.set_fast_path(False)
+    W = max(args.warmup, 3)
+    pk = peaks()
+
+    cfg = synth.CONFIGS[args.workload]
+    ng = args.groups or cfg.n_groups
+    # weak scaling: every rank compresses its own sequence (seed + rank); no data-path collective
+    K, V = synth.make_cache(cfg, seq=rank, device=f"cuda:{local}", n_groups=ng)
+    gs = [g * cfg.layers_per_group for g in range(ng + 1)]
+    cache_bytes = 2 * K.numel() * 2
+    opts = B.default_options(seed=cfg.seed + rank, power_iters=cfg.power_iters)
+    t0 = time.perf_counter()
+    plans, planned_bytes = B.jolt_plan(K, V, gs, cache_bytes / cfg.ratio, opts)
+    torch.cuda.synchronize()
+    plan_ms = (time.perf_counter() - t0) * 1e3
+    Ko, Vo = torch.empty_like(K), torch.empty_like(V)
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    stage_acc = {}
+
+    def step(record=None):
+        e0, e1, e2 = ev(), ev(), ev()
+        e0.record()
+        h = B.jolt_compress(K, V, gs, plans, opts)
+        e1.record()
+        st_c = B.stage_ms()
+        B.jolt_decompress(h, Ko, Vo, gs)
+        e2.record()
+        torch.cuda.synchronize()
+        st_d = B.stage_ms()
+        h.free()
+        if record is not None:
+            record.append((e0.elapsed_time(e1), e1.elapsed_time(e2)))
+            for k_, v_ in list(st_c.items()) + list(st_d.items()):
+                stage_acc[k_] = stage_acc.get(k_, 0.0) + v_
+        return h
+
+    for _ in range(W):
+        step()
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    n0 = B.launch_count()
+    rec = []
+    for _ in range(args.steps):
+        step(rec)
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    launches = B.launch_count() - n0
+    clocks = sampler.stop() if rank == 0 else None
+    tc = sum(r[0] for r in rec) / len(rec)
+    td = sum(r[1] for r in rec) / len(rec)
+    # decompress stage timing (device events inside the library need a sync, done in step())
+    if dist:
+        t = torch.tensor([tc, td], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        tc, td = t.tolist()
+    ms = tc + td
+
+    # accuracy of the benchmarked configuration (mean relative Frobenius error over cells)
+    errs = []
+    for c in range(2 * ng):
+        g, w = divmod(c, 2)
+        a = (K, V)[w][gs[g]:gs[g + 1]].float()
+        b_ = (Ko, Vo)[w][gs[g]:gs[g + 1]].float()
+        errs.append(float((a - b_).norm() / a.norm()))
+    rel_k = sum(errs[0::2]) / ng
+    rel_v = sum(errs[1::2]) / ng
+
+    # end to end through the public API with host buffers (pinned), copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        Kh, Vh = K.cpu().pin_memory(), V.cpu().pin_memory()
+        Koh, Voh = torch.empty_like(Kh).pin_memory(), torch.empty_like(Vh).pin_memory()
+
+        def step_host():
+            h = B.jolt_compress(Kh, Vh, gs, plans, opts)
+            B.jolt_decompress(h, Koh, Voh, gs)
+            h.free()
+        for _ in range(2):
+            step_host()
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        t0 = time.perf_counter()
+        n_e2e = max(2, min(args.steps, 5))
+        for _ in range(n_e2e):
+            step_host()
+        torch.cuda.synchronize()
+        te = (time.perf_counter() - t0) / n_e2e
+        if dist:
+            t = torch.tensor([te], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            te = float(t.item())
+        e2e = {"value": world * cache_bytes / te / 1e9, "unit": UNIT, "h2d_bytes_per_step": cache_bytes,
+               "d2h_bytes_per_step": cache_bytes, "ms_per_step": te * 1e3}
+        del Kh, Vh, Koh, Voh
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+
+    # roofline bookkeeping
+    q = cfg.power_iters
+    tot = {}
+    for c, (rt, rf, b) in enumerate(plans):
+        kk = min(rt + 10, cfg.seq_len, cfg.m * rf)
+        w = cell_work(cfg.m, cfg.seq_len, cfg.head_dim, rt, rf, b, kk, q, 2)
+        for name, val in w.items():
+            if isinstance(val, tuple):
+                f0, b0 = tot.get(name, (0, 0))
+                tot[name] = (f0 + val[0], b0 + val[1])
+            else:
+                tot[name] = tot.get(name, 0) + val
+    t_roof_c = sum(roof_time(*cell_work(cfg.m, cfg.seq_len, cfg.head_dim, rt, rf, b, min(rt + 10, cfg.seq_len, cfg.m * rf), q, 2)["compress"], pk)
+                   for rt, rf, b in plans)
+    t_roof_d = sum(roof_time(*cell_work(cfg.m, cfg.seq_len, cfg.head_dim, rt, rf, b, min(rt + 10, cfg.seq_len, cfg.m * rf), q, 2)["decompress"], pk)
+                   for rt, rf, b in plans)
+    stages = {k_: v_ / len(rec) for k_, v_ in stage_acc.items()}
+    # dominant kernel = the decode pass (the headline HBM-bound kernel); its duration is the decompress call
+    fd, bd = tot["decompress"]
+    dec_bound = "hbm" if bd / (pk["hbm"] * 1e9) >= fd / (pk["tensor"] * 1e12) else "tensor"
+    if dec_bound == "hbm":
+        ach = bd / (td * 1e-3) / 1e9
+        roofline = {"kernel": "decompress pass", "bound": "hbm", "achieved": ach, "peak": pk["hbm"], "unit": "GB/s",
+                    "frac": ach / pk["hbm"], "traffic": None, "peak_source": pk["source"]}
+    else:
+        ach = fd / (td * 1e-3) / 1e12
+        roofline = {"kernel": "decompress pass", "bound": "tensor", "achieved": ach, "peak": pk["tensor"], "unit": "TFLOP/s",
+                    "frac": ach / pk["tensor"], "traffic": None, "peak_source": pk["source"]}
+
+    line = {"metric": METRIC, "value": world * cache_bytes / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f16 operands, f32 accumulate (f64 small solvers)", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: {ng * cfg.layers_per_group} layers / {cfg.layers_per_group} per group, "
+                                   f"{cfg.n_kv_heads} KV heads, T={cfg.seq_len}, d=128, fp16, budget {cfg.ratio}x, randomized q={q}",
+                       "cache_bytes": cache_bytes, "compressed_bytes": planned_bytes, "achieved_ratio": cache_bytes / planned_bytes,
+                       "plan": plans, "l2": "inputs (537 MB) exceed L2; no flush"},
+            "compress_ms": tc, "decompress_ms": td, "plan_ms": plan_ms,
+            "compress_gbs": world * cache_bytes / (tc * 1e-3) / 1e9, "decompress_gbs": world * cache_bytes / (td * 1e-3) / 1e9,
+            "compress_roofline_frac": t_roof_c * 1e3 / tc, "decompress_roofline_frac": t_roof_d * 1e3 / td,
+            "compress_roofline_ms": t_roof_c * 1e3, "decompress_roofline_ms": t_roof_d * 1e3,
+            "rel_frobenius_error": {"K": rel_k, "V": rel_v},
+            "stages_ms": stages, "roofline": roofline, "gpu_launches": launches, "clocks": clocks, "e2e": e2e}
+
+    if not args.no_cpu_baseline and world == 1:
+        from oracle import jolt_oracle as O
+        t0 = time.perf_counter()
+        sample = {}
+        for w_ in (0, 1):
+            X = (K, V)[w_][gs[0]:gs[1]].reshape(cfg.m, cfg.seq_len, 128).cpu().numpy()
+            a = time.perf_counter()
+            oc = O.compress_cell(X, *plans[w_], seed=cfg.seed, cell=w_, token_mode="randomized", power_iters=q)
+            b_ = time.perf_counter()
+            O.decompress_cell(oc)
+            c_ = time.perf_counter()
+            sample[w_] = (b_ - a, c_ - b_)
+        sc = sum(v[0] for v in sample.values()); sd = sum(v[1] for v in sample.values())
+        sb = 2 * cfg.m * cfg.seq_len * 128 * 2
+        line["cpu_baseline"] = {"value": sb / (sc + sd) / 1e9, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                                "sample": "cells 0 and 1 (group 0, K and V) of the same cache and plan, numpy fp64",
+                                "compress_gbs": sb / sc / 1e9, "decompress_gbs": sb / sd / 1e9}
+    print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -54,6 +54,7 @@ struct StageTimer {
   void begin(cudaStream_t s) { init(); n = 0; for (auto &m : ms) m = 0.f; cudaEventRecord(ev[0], s); }
   void mark(int stage, cudaStream_t s) { if (n < kNumStages) { order[n] = stage; ++n; cudaEventRecord(ev[n], s); } }
   void finish() {
+    for (auto &m : ms) m = 0.f;
     for (int i = 0; i < n; ++i) { float t = 0; if (cudaEventElapsedTime(&t, ev[i], ev[i + 1]) == cudaSuccess) ms[order[i]] += t; }
   }
 };
@@ -1169,6 +1170,7 @@ extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled 
 extern "C" int jolt_last_stage_ms(float *out, int32_t cap, int32_t *n) {
   if (!out || !n) return fail(JOLT_EINVAL, "null argument");
   *n = std::min<int>(cap, kNumStages);
+  if (g_timer.have) g_timer.finish();
   for (int i = 0; i < *n; ++i) out[i] = g_timer.ms[i];
   return JOLT_OK;
 }
