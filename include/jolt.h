@@ -109,6 +109,25 @@ int jolt_compress_with_factors(const jolt_layout *layout, const void *dK, const 
 int jolt_decompress(const jolt_handle *h, const jolt_layout *out_layout, void *dK_out, void *dV_out,
                     void *stream);
 
+/* jolt_decompress_static -- the paper has no counterpart; this is a deployment variant of jolt_decompress
+ * for callers that cannot allocate device memory while decoding (a serving process that has given all free
+ * memory to its own pool, a thread for which a driver allocation would stall the context, a host whose
+ * allocator policy forbids cudaMalloc after start-up).  It calls no cudaMalloc / cudaFree and no allocating
+ * library routine: all scratch (projected cores, the fp32 backbone buffer, status words, kernel argument
+ * tables) lives in one fixed 16 MiB device array that is part of the library image, so every GPU that loads
+ * the library holds those 16 MiB until the process exits.
+ *   - Arguments and result as jolt_decompress, device destinations only (JOLT_MEM_HOST -> JOLT_EUNSUPPORTED).
+ *   - A cache whose decode scratch (about 4 bytes per cache element of cells with a backbone, plus
+ *     2*m*r_t*128 bytes per such cell) exceeds 16 MiB is rejected with JOLT_EINVAL and a message that names
+ *     both sizes; nothing is launched.
+ *   - The first call on a device looks up the device address of the array (one cudaGetSymbolAddress with
+ *     that device current); make that first call before any stream capture.
+ *   - Every call shares the one array and finds the previous call's contents in it; the call clears what must
+ *     start at zero.  Two calls that overlap on the GPU (different streams, or different threads) race on
+ *     the array: issue them on one stream, or serialise them yourself. */
+int jolt_decompress_static(const jolt_handle *h, const jolt_layout *out_layout, void *dK_out, void *dV_out,
+                           void *stream);
+
 /* Release a handle and all buffers it owns.  NULL is accepted. */
 int jolt_free(jolt_handle *h);
 

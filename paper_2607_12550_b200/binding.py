@@ -54,6 +54,7 @@ lib.jolt_compress_with_factors.argtypes = [C.POINTER(Layout), _vp, _vp, C.POINTE
                                            C.POINTER(_vp), C.POINTER(_vp), _vp, C.POINTER(_vp)]
 lib.jolt_decompress.argtypes = [_vp, C.POINTER(Layout), _vp, _vp, _vp]
 lib.jolt_free.argtypes = [_vp]
+lib.jolt_decompress_static.argtypes = [_vp, C.POINTER(Layout), _vp, _vp, _vp]
 lib.jolt_compressed_bytes.argtypes = [_vp, C.POINTER(C.c_int64)]
 lib.jolt_get_component.argtypes = [_vp, C.c_int32, C.c_int32, _vp, C.c_int64, C.POINTER(C.c_int64)]
 lib.jolt_allocate.argtypes = [C.c_int32, C.POINTER(C.c_int32), C.c_int32, C.c_int32, C.POINTER(C.c_double),
@@ -208,6 +209,12 @@ def jolt_compress(K, V, group_start, plans, opts: Options | None = None, stream=
 def jolt_decompress(handle: Handle, K_out, V_out, group_start, stream=None):
     lay = make_layout(K_out, group_start)
     _check(lib.jolt_decompress(handle.ptr, C.byref(lay), K_out.data_ptr(), V_out.data_ptr(), _stream_ptr(stream)))
+
+
+def jolt_decompress_static(handle: Handle, K_out, V_out, group_start, stream=None):
+    """Decode without any device allocation (fixed 16 MiB scratch inside the library); see include/jolt.h."""
+    lay = make_layout(K_out, group_start)
+    _check(lib.jolt_decompress_static(handle.ptr, C.byref(lay), K_out.data_ptr(), V_out.data_ptr(), _stream_ptr(stream)))
 
 
 def jolt_free(handle: Handle):

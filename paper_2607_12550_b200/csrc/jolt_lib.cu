@@ -1189,3 +1189,5 @@ extern "C" const char *jolt_strerror(int s) {
   }
 }
 extern "C" const char *jolt_last_error(void) { return g_err.c_str(); }
+
+#include "decode_static.cuh"
