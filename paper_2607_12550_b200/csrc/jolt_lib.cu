@@ -12,6 +12,7 @@
 #include <string>
 #include <vector>
 
+#include <cuda.h>
 #include "allocator.h"
 #include "common.cuh"
 #include "rowquant.cuh"
@@ -174,6 +175,8 @@ struct CellStore {
   float *sigma = nullptr;  // k (or T for the exact path)
   float *lam = nullptr;    // 128
   int n_sigma = 0;
+  bool tc_ok = false;      // tensor maps below are valid
+  alignas(64) CUtensorMap tmUT, tmUF, tmG;
 };
 
 struct jolt_handle {
@@ -236,7 +239,7 @@ struct Program {
   struct Step { int stage; std::function<void(char *, cudaStream_t)> run; };
   std::vector<Step> steps;
   template <typename T> size_t push(const std::vector<T> &v) {
-    size_t off = (host.size() + 15) & ~(size_t)15;
+    size_t off = (host.size() + 127) & ~(size_t)127;
     host.resize(off + v.size() * sizeof(T));
     if (!v.empty()) memcpy(host.data() + off, v.data(), v.size() * sizeof(T));
     return off;
@@ -747,7 +750,6 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
       carve(b, w, mode, true);
       if (pass == 1 && !w.n_sigma) w.n_sigma = H->cells[i].n_sigma;
     }
-    fast_carve(b, ws, fast);
     if (pass == 0) {
       ws_bytes = b.off + 256;
       if ((rc = ws_reserve(dev, ws_bytes, &ws_base))) { free_blob(); return rc; }
@@ -767,7 +769,6 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   Program P;
   build_factor_program(P, ws, mode, false, o->power_iters, o->seed, fast);
   std::vector<StoreJob> sj;
-  std::vector<BackboneRef> br;
   for (int i = 0; i < nc; ++i) {
     const CellDesc &c = cells[i];
     const CellStore &cs = H->cells[i];
@@ -777,7 +778,6 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     j.G16 = cs.G16; j.UT16 = cs.UT16; j.UF16 = cs.UF16; j.e = cs.e;
     j.nG = (long long)c.m * c.r_t * c.r_f; j.nUT = (long long)c.T * c.r_t; j.nUF = (long long)kD * c.r_f; j.round_inputs = 0;
     sj.push_back(j);
-    br.push_back({ws[i].c, cs.G16, cs.UT16, cs.UF16, cs.e, ws[i].P16, ws[i].Xt});
   }
   if (!sj.empty()) {
     const size_t off = P.push(sj);
@@ -787,27 +787,58 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
       store_factors_kernel<<<dim3(64, n), 256, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
     });
   }
-  std::vector<RowJob> rj(nc);
-  long long rows = 0;
-  bool any_bits = false;
+  // residual / rotate / quantise / pack: tensor-core kernel where the cell fits it, portable kernels otherwise
+  std::vector<char> use_tc(nc, 0);
+  int tc_heads = 0;
+  const bool x_tma_ok = L->dtype == JOLT_F16 && L->stride_token * 2 % 16 == 0 && L->stride_head * 2 % 16 == 0 &&
+                        L->stride_layer * 2 % 16 == 0;
   for (int i = 0; i < nc; ++i) {
-    RowJob &j = rj[i];
-    memset(&j, 0, sizeof j);
-    j.c = ws[i].c; j.Xt = cells[i].r_t > 0 ? ws[i].Xt : nullptr;
-    j.words = H->cells[i].words; j.scales = H->cells[i].scales; j.status = d_status + 4 * i; j.row0 = rows;
-    rows += (long long)cells[i].m * cells[i].T;
-    any_bits |= cells[i].bits > 0;
-  }
-  if (!fast_residual(P, ws, br, rj, H.get(), o->seed, fast)) {
-    add_backbone(P, ST_BACK, br);
-    if (any_bits) {
-      const size_t off = P.push(rj);
-      const uint64_t seed = o->seed;
-      P.add(ST_RQ, [=](char *dev_t, cudaStream_t s) {
-        residual_quant_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, s>>>((const RowJob *)(dev_t + off), nc, rows, seed);
-        LAUNCHED();
-      });
+    CellStore &cs = H->cells[i];
+    if (fast && encode_store_maps(cs) && x_tma_ok && cells[i].bits > 0 && ((uintptr_t)cells[i].X % 16 == 0)) {
+      use_tc[i] = 1;
+      tc_heads += cells[i].m;
     }
+  }
+  std::vector<tc::BBCell> bbc;
+  std::vector<BackboneRef> br_port;
+  std::vector<RowJob> rj;
+  long long rows = 0;
+  int tpi = 1, iph = 1;
+  bb_split(tc_heads, L->seq_len / 128, tpi, iph);
+  for (int i = 0; i < nc; ++i) {
+    const CellDesc &c = cells[i];
+    const CellStore &cs = H->cells[i];
+    if (use_tc[i]) {
+      tc::BBCell b;
+      fill_bb_common(b, cs, d_status + 4 * i);
+      b.tiles_per_item = tpi; b.items_per_head = iph;
+      const int g = i / 2;
+      const int Lg = L->group_start[g + 1] - L->group_start[g];
+      const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)c.T, (uint64_t)c.n_heads, (uint64_t)Lg};
+      const uint64_t str[3] = {(uint64_t)c.st * 2, (uint64_t)c.sh * 2, (uint64_t)c.sl * 2};
+      const uint32_t box[4] = {64, 128, 1, 1};
+      if (!make_tmap_f16(&b.tmX, c.X, 4, dims, str, box)) { use_tc[i] = 0; }
+      else { bbc.push_back(b); continue; }
+    }
+    if (c.bits == 0) continue;
+    if (c.r_t > 0) br_port.push_back({ws[i].c, cs.G16, cs.UT16, cs.UF16, cs.e, ws[i].P16, ws[i].Xt});
+    RowJob j;
+    memset(&j, 0, sizeof j);
+    j.c = ws[i].c; j.Xt = c.r_t > 0 ? ws[i].Xt : nullptr;
+    j.words = cs.words; j.scales = cs.scales; j.status = d_status + 4 * i; j.row0 = rows;
+    rows += (long long)c.m * c.T;
+    rj.push_back(j);
+  }
+  add_backbone_tc<true>(P, ST_RQ, bbc, o->seed);
+  add_backbone(P, ST_BACK, br_port);
+  if (!rj.empty()) {
+    const size_t off = P.push(rj);
+    const uint64_t seed = o->seed;
+    const int nj = (int)rj.size();
+    P.add(ST_RQ, [=](char *dev_t, cudaStream_t s) {
+      residual_quant_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, s>>>((const RowJob *)(dev_t + off), nj, rows, seed);
+      LAUNCHED();
+    });
   }
   void *d_tab = nullptr;
   if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) { free_blob(); return rc; }
@@ -872,6 +903,10 @@ extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void 
   const size_t span = layout_span_elems(L) * esz;
   const bool fast = g_fast.load() != 0;
   std::vector<CellWork> ws(nc);
+  std::vector<char> use_tc(nc, 0);
+  int tc_heads = 0;
+  for (int i = 0; i < nc; ++i)
+    if (fast && H->cells[i].tc_ok) { use_tc[i] = 1; tc_heads += H->cells[i].c.m; }
   void *ws_base = nullptr;
   char *stage_K = nullptr, *stage_V = nullptr;
   int *d_status = nullptr;
@@ -884,37 +919,52 @@ extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void 
       ws[i].c = H->cells[i].c;
       ws[i].active = false;
       ws[i].status = d_status ? d_status + 4 * i : nullptr;
-      carve(b, ws[i], FM_INJECTED, !fast_decode_ok(ws[i].c, L, fast));
+      carve(b, ws[i], FM_INJECTED, !use_tc[i]);
     }
-    fast_carve_decode(b, ws, fast);
     if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) return rc;
   }
   char *Kd = L->mem_space == JOLT_MEM_HOST ? stage_K : (char *)Kout;
   char *Vd = L->mem_space == JOLT_MEM_HOST ? stage_V : (char *)Vout;
   Program P;
   std::vector<BackboneRef> br;
-  std::vector<RowJob> rj(nc);
+  std::vector<RowJob> rj;
+  std::vector<tc::BBCell> bbc;
   long long rows = 0;
+  int tpi = 1, iph = 1;
+  bb_split(tc_heads, L->seq_len / 128, tpi, iph);
   for (int i = 0; i < nc; ++i) {
     const CellStore &cs = H->cells[i];
     const CellDesc &c = cs.c;
+    const int g = i / 2;
+    char *obase = (i % 2 == 0 ? Kd : Vd) + (size_t)L->group_start[g] * L->stride_layer * esz;
+    if (use_tc[i]) {
+      tc::BBCell b;
+      fill_bb_common(b, cs, d_status + 4 * i);
+      b.tiles_per_item = tpi; b.items_per_head = iph;
+      b.out = obase; b.out_dtype = L->dtype == JOLT_F16 ? DT_F16 : DT_F32;
+      b.osl = L->stride_layer; b.osh = L->stride_head; b.ost = L->stride_token;
+      bbc.push_back(b);
+      continue;
+    }
     if (c.r_t > 0) br.push_back({c, cs.G16, cs.UT16, cs.UF16, cs.e, ws[i].P16, ws[i].Xt});
-    RowJob &j = rj[i];
+    RowJob j;
     memset(&j, 0, sizeof j);
     j.c = c; j.Xt = c.r_t > 0 ? ws[i].Xt : nullptr; j.words = cs.words; j.scales = cs.scales; j.status = d_status + 4 * i;
-    const int g = i / 2;
-    j.out = (i % 2 == 0 ? Kd : Vd) + (size_t)L->group_start[g] * L->stride_layer * esz;
+    j.out = obase;
     j.out_dtype = L->dtype == JOLT_F16 ? DT_F16 : DT_F32;
     j.osl = L->stride_layer; j.osh = L->stride_head; j.ost = L->stride_token;
     j.row0 = rows;
     rows += (long long)c.m * c.T;
+    rj.push_back(j);
   }
-  if (!fast_decode(P, ws, br, rj, H, L, fast)) {
-    add_backbone(P, ST_DBACK, br);
+  add_backbone_tc<false>(P, ST_DROWS, bbc, H->seed);
+  add_backbone(P, ST_DBACK, br);
+  if (!rj.empty()) {
     const size_t off = P.push(rj);
     const uint64_t seed = H->seed;
+    const int nj = (int)rj.size();
     P.add(ST_DROWS, [=](char *dev_t, cudaStream_t s) {
-      dequant_add_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, s>>>((const RowJob *)(dev_t + off), nc, rows, seed);
+      dequant_add_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, s>>>((const RowJob *)(dev_t + off), nj, rows, seed);
       LAUNCHED();
     });
   }
@@ -1090,7 +1140,6 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
       ws[i].lam = nullptr; ws[i].sigma = nullptr;
       carve(b, ws[i], mode, false);
     }
-    fast_carve(b, ws, fast);
     if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) return rc;
   }
   if (L->mem_space == JOLT_MEM_HOST)
