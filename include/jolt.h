@@ -176,8 +176,9 @@ int jolt_release_workspace(void);
 /* Number of kernel launches the library has issued since load (all streams). */
 int64_t jolt_launch_count(void);
 
-/* Selects the kernel family: 0 = portable SIMT kernels only, 1 (default) = tcgen05 / TMA kernels
- * where the shapes allow.  Returns the previous value. */
+/* Selects the kernel family by bit mask: 0 = portable SIMT kernels only; bit 0 = fused tcgen05 backbone
+ * kernels (decode, residual), bit 1 = tcgen05 factor sweeps (sketch, projection), bit 2 = tcgen05 mode-3
+ * Gram; 7 (default) = all, where the shapes allow.  Returns the previous mask. */
 int jolt_set_fast_path(int enabled);
 
 /* Wall-clock-free per-stage device timing of the last compress / decompress on this thread

@@ -88,9 +88,10 @@ def gaussian_from_u64(r):
 
 def gaussian_sketch(seed: int, cell: int, n_rows: int, n_cols: int, stream: int = STREAM_SKETCH):
     """Seeded Gaussian test matrix Omega (n_rows x n_cols), entry (i, j) from counter i*n_cols + j,
-    rounded to fp32 (the value both sides then use), returned as float64."""
+    rounded to fp16 (the sketch is DEFINED on the fp16 grid, so a half-precision tensor-core operand
+    represents it exactly; the value both sides then use), returned as float64."""
     r = random_u64(seed, cell, stream, n_rows * n_cols)
-    g = gaussian_from_u64(r).astype(np.float32)
+    g = gaussian_from_u64(r).astype(np.float16)
     return g.astype(np.float64).reshape(n_rows, n_cols)
 
 

@@ -279,8 +279,12 @@ def launch_count() -> int:
     return lib.jolt_launch_count()
 
 
-def set_fast_path(enabled: bool) -> int:
-    return lib.jolt_set_fast_path(1 if enabled else 0)
+def set_fast_path(enabled) -> int:
+    """False / 0: portable kernels only; True / 7: every tensor-core kernel; other ints: bit mask
+    (1 = fused backbone kernels, 2 = factor sweeps, 4 = Gram).  Returns the previous mask."""
+    if enabled is True:
+        enabled = 7
+    return lib.jolt_set_fast_path(int(enabled))
 
 
 def release_workspace():

@@ -3,6 +3,7 @@
 // multiple of 8); every other cell stays on the portable kernels, in the same call.
 #pragma once
 #include "tc_backbone.cuh"
+#include "tc_gemm.cuh"
 
 namespace {
 
@@ -71,6 +72,165 @@ inline void fill_bb_common(tc::BBCell &b, const CellStore &cs, int *status) {
   const CellDesc &c = cs.c;
   b.m = c.m; b.n_heads = c.n_heads; b.T = c.T; b.r_t = c.r_t; b.r_f = c.r_f; b.bits = c.bits; b.cell = c.cell;
   b.status = status;
+}
+
+
+// ------------------------------------------------------------------ tensor-core sweeps of the factor stage
+
+inline bool make_x_map(CUtensorMap *tm, const CellDesc &c, uint32_t box_tok) {
+  const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)c.T, (uint64_t)c.n_heads, (uint64_t)(c.m / c.n_heads)};
+  const uint64_t str[3] = {(uint64_t)c.st * 2, (uint64_t)c.sh * 2, (uint64_t)c.sl * 2};
+  const uint32_t box[4] = {64, box_tok, 1, 1};
+  return make_tmap_f16(tm, c.X, 4, dims, str, box);
+}
+
+inline bool x_tma_ok(const CellDesc &c) {
+  return c.dtype == DT_F16 && c.st % 8 == 0 && c.sh % 8 == 0 && c.sl % 8 == 0 && ((uintptr_t)c.X % 16 == 0) && c.T % 128 == 0;
+}
+
+// A cell's factor-stage sweeps can run on tensor cores: fp16 data TMA can address, sketch width <= 256.
+inline bool tc_sweep_ok(const CellDesc &c, bool staged_from_host) {
+  if (c.dtype != DT_F16 || c.st % 8 || c.sh % 8 || c.sl % 8 || c.T % 128) return false;
+  if (!staged_from_host && ((uintptr_t)c.X % 16)) return false;
+  return c.k >= 1 && c.k <= 256;
+}
+
+inline int ilog2_floor(long long v) { int e = 0; while ((1ll << (e + 1)) <= v) ++e; return e; }
+
+template <int MODE>
+inline void launch_tc_gemm(Program &P, int stage, std::vector<tc::GemmCell> &cells) {
+  if (cells.empty()) return;
+  uint32_t max_stage = 0;
+  int gx = 0;
+  for (auto &c : cells) {
+    const uint32_t b_bytes = MODE == tc::GM_GRAM ? 0u : (uint32_t)c.kp * 128u;
+    const uint32_t b_pitch = (b_bytes + 1023u) & ~1023u;
+    max_stage = std::max(max_stage, 16384u + ((c.has_lo && MODE != tc::GM_GRAM) ? 2 * b_pitch : b_pitch));
+    gx = std::max(gx, MODE == tc::GM_TOK ? c.T / 128 : c.m);
+  }
+  int n_stages = std::min(8, (int)((tc::GM_SMEM_LIMIT - 1536) / max_stage));
+  const size_t smem = (size_t)n_stages * max_stage + 1024 + 512;
+  static size_t attr[3] = {0, 0, 0};
+  if (attr[MODE] < smem) {
+    cudaFuncSetAttribute(tc::tc_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::GM_SMEM_LIMIT);
+    attr[MODE] = tc::GM_SMEM_LIMIT;
+  }
+  const size_t off = P.push(cells);
+  const int n = (int)cells.size();
+  P.add(stage, [=](char *dev_t, cudaStream_t s) {
+    tc::tc_gemm_kernel<MODE><<<dim3(gx, n), tc::GM_THREADS, smem, s>>>((const tc::GemmCell *)(dev_t + off), n_stages);
+    LAUNCHED();
+  });
+}
+
+inline void launch_split(Program &P, int stage, const std::vector<tc::SplitJob> &jobs) {
+  if (jobs.empty()) return;
+  const size_t off = P.push(jobs);
+  const int n = (int)jobs.size();
+  P.add(stage, [=](char *dev_t, cudaStream_t s) {
+    tc::split_transpose_kernel<<<dim3(148, 1, n), 256, 0, s>>>((const tc::SplitJob *)(dev_t + off));
+    LAUNCHED();
+  });
+}
+
+// mode-3 Gram of the tensor-core cells: fp32 partial per head, summed in fp64.
+inline void add_gram_tc(Program &P, int stage, std::vector<CellWork> &ws) {
+  std::vector<tc::GemmCell> gc;
+  std::vector<const float *> parts; std::vector<double *> outs; std::vector<int> counts;
+  for (auto &w : ws) {
+    if (!w.active || !w.tc_gram) continue;
+    tc::GemmCell g;
+    memset(&g, 0, sizeof g);
+    make_x_map(&g.tmX, w.c, 64);
+    g.C = (float *)w.gram_part; g.ldc = kD; g.ncols = kD; g.kp = kD; g.has_lo = 0; g.scale_exp = 0;
+    g.m = w.c.m; g.n_heads = w.c.n_heads; g.T = w.c.T; g.status = w.status;
+    gc.push_back(g);
+    parts.push_back((const float *)w.gram_part); outs.push_back(w.C); counts.push_back(w.c.m);
+  }
+  if (gc.empty()) return;
+  launch_tc_gemm<tc::GM_GRAM>(P, stage, gc);
+  const size_t o1 = P.push(parts), o2 = P.push(outs), o3 = P.push(counts);
+  const int n = (int)parts.size();
+  P.add(stage, [=](char *dev_t, cudaStream_t s) {
+    tc::reduce_gram_partials_kernel<<<dim3(kD * kD / 256, n), 256, 0, s>>>((const float *const *)(dev_t + o1),
+                                                                        (double *const *)(dev_t + o2), (const int *)(dev_t + o3));
+    LAUNCHED();
+  });
+}
+
+// S = sum_h X_h W_h for the tensor-core cells.  src: 0 = fp16 sketch already in Bhi, 1 = split W (fp32,
+// [h][128][k]), 2 = split Z (fp32, [h][128][k], orthonormal columns over N rows).
+inline void add_tok_tc(Program &P, int stage, std::vector<CellWork> &ws, const std::vector<int> &src) {
+  std::vector<tc::SplitJob> sp;
+  std::vector<tc::GemmCell> gc;
+  for (size_t i = 0; i < ws.size(); ++i) {
+    CellWork &w = ws[i];
+    if (!w.active || !w.tc) continue;
+    const CellDesc &c = w.c;
+    int se = 0;
+    if (src[i] != 0) {
+      const float *in = w.W;
+      if (src[i] == 2) { in = w.ufI ? w.Z : w.W; se = ilog2_floor((long long)c.N) / 2; }
+      tc::SplitJob j;
+      j.in = in; j.hi = w.Bhi; j.lo = w.Blo; j.batch = c.m; j.rows = kD; j.cols = c.k; j.ld_in = c.k;
+      j.kp = w.kp; j.scale_exp = se;
+      sp.push_back(j);
+    }
+    tc::GemmCell g;
+    memset(&g, 0, sizeof g);
+    const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)w.kp, (uint64_t)c.m};
+    const uint64_t str[2] = {(uint64_t)kD * 2, (uint64_t)w.kp * kD * 2};
+    const uint32_t box[3] = {64, (uint32_t)w.kp, 1};
+    bool okm = make_x_map(&g.tmX, c, 128) && make_tmap_f16(&g.tmBhi, w.Bhi, 3, dims, str, box) &&
+               make_tmap_f16(&g.tmBlo, w.Blo, 3, dims, str, box);
+    (void)okm;
+    g.C = w.S; g.ldc = c.k; g.ncols = c.k; g.kp = w.kp; g.has_lo = src[i] != 0; g.scale_exp = se;
+    g.m = c.m; g.n_heads = c.n_heads; g.T = c.T; g.status = w.status;
+    gc.push_back(g);
+  }
+  launch_split(P, stage, sp);
+  launch_tc_gemm<tc::GM_TOK>(P, stage, gc);
+}
+
+// Z'_h = X_h^T Q for the tensor-core cells (Q = w.S, T x k with orthonormal columns).
+inline void add_feat_tc(Program &P, int stage, std::vector<CellWork> &ws) {
+  std::vector<tc::SplitJob> sp;
+  std::vector<tc::GemmCell> gc;
+  for (auto &w : ws) {
+    if (!w.active || !w.tc) continue;
+    const CellDesc &c = w.c;
+    const int se = ilog2_floor(c.T) / 2;
+    tc::SplitJob j;
+    j.in = w.S; j.hi = w.Bhi; j.lo = w.Blo; j.batch = 1; j.rows = c.T; j.cols = c.k; j.ld_in = c.k; j.kp = w.kp; j.scale_exp = se;
+    sp.push_back(j);
+    tc::GemmCell g;
+    memset(&g, 0, sizeof g);
+    const uint64_t dims[2] = {(uint64_t)c.T, (uint64_t)w.kp};
+    const uint64_t str[1] = {(uint64_t)c.T * 2};
+    const uint32_t box[2] = {64, (uint32_t)w.kp};
+    bool okm = make_x_map(&g.tmX, c, 64) && make_tmap_f16(&g.tmBhi, w.Bhi, 2, dims, str, box) &&
+               make_tmap_f16(&g.tmBlo, w.Blo, 2, dims, str, box);
+    (void)okm;
+    g.C = w.Zp; g.ldc = c.k; g.ncols = c.k; g.kp = w.kp; g.has_lo = 1; g.scale_exp = se;
+    g.m = c.m; g.n_heads = c.n_heads; g.T = c.T; g.status = w.status;
+    gc.push_back(g);
+  }
+  launch_split(P, stage, sp);
+  launch_tc_gemm<tc::GM_FEAT>(P, stage, gc);
+}
+
+// fp16 sketch of the r_f = d tensor-core cells, written straight into the TOK operand layout.
+inline void add_sketch_gen_tc(Program &P, int stage, std::vector<CellWork> &ws, int stream_id, uint64_t seed) {
+  std::vector<tc::SketchJob> jobs;
+  for (auto &w : ws)
+    if (w.active && w.tc && w.ufI) jobs.push_back({w.Bhi, w.c.m, w.c.k, w.kp, w.c.cell});
+  if (jobs.empty()) return;
+  const size_t off = P.push(jobs);
+  const int n = (int)jobs.size();
+  P.add(stage, [=](char *dev_t, cudaStream_t s) {
+    tc::gen_sketch_f16_kernel<<<dim3(148, n), 256, 0, s>>>((const tc::SketchJob *)(dev_t + off), stream_id, seed);
+    LAUNCHED();
+  });
 }
 
 }  // namespace

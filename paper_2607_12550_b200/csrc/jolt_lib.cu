@@ -24,7 +24,7 @@ using namespace jolt;
 namespace jolt {
 thread_local std::string g_err;
 std::atomic<long long> g_launches{0};
-std::atomic<int> g_fast{1};
+std::atomic<int> g_fast{7};   // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores
 
 int fail(int code, const char *fmt, ...) {
   char buf[512];
@@ -103,7 +103,7 @@ __global__ void gen_sketch_kernel(const CellDesc *cells, float *const *omega, co
   const uint64_t base = stream_base(seed, cells[ci].cell, stream_id);
   float *o = omega[ci];
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
-    o[i] = (float)gaussian_from_u64(mix64(base + (uint64_t)i));
+    o[i] = __half2float(__double2half(gaussian_from_u64(mix64(base + (uint64_t)i))));
 }
 
 __global__ void reduce_partials_kernel(const double *const *partials, double *const *out, const int *counts, int n_elems) {
@@ -319,6 +319,12 @@ struct CellWork {      // device scratch of one cell
   float *Xt = nullptr;
   int *status = nullptr;
   int n_sigma = 0;
+  // tensor-core sweeps
+  bool tc = false;           // sketch / projection sweeps run on tcgen05
+  bool tc_gram = false;      // mode-3 Gram runs on tcgen05
+  bool ufI = false;          // r_f = d: the token factor is computed in the original feature coordinates
+  int kp = 0;                // sketch width padded to a multiple of 16
+  __half *Bhi = nullptr, *Blo = nullptr;
 };
 
 enum FactorMode { FM_RANDOMIZED = 0, FM_EXACT = 1, FM_INJECTED = 2 };
@@ -344,7 +350,13 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
       w.PF = b.take<float>(kD * kD);
       w.W = b.take<float>((size_t)c.m * kD * k);
       w.S = b.take<float>(T * k); w.S2 = b.take<float>(T * k);
-      w.Z = b.take<float>(N * k); w.Z2 = b.take<float>(N * k);
+      if (w.ufI) w.Z = w.Zp; else w.Z = b.take<float>(N * k);
+      w.Z2 = b.take<float>(N * k);
+      if (w.tc) {
+        w.kp = (c.k + 15) & ~15;
+        const size_t nb = std::max((size_t)c.m * w.kp * kD, (size_t)w.kp * T);
+        w.Bhi = b.take<__half>(nb); w.Blo = b.take<__half>(nb);
+      }
       w.Gs = b.take<double>(k * k); w.Linv = b.take<double>(k * k); w.LinvT = b.take<float>(k * k);
       w.BBt = b.take<double>(k * k); w.BBv = b.take<double>(k * k); w.BBw = b.take<double>(k);
       w.Ut = b.take<float>(k * std::max<size_t>(c.r_t, 1));
@@ -362,6 +374,10 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
     w.Xt = b.take<float>(M);
   }
 }
+
+}  // namespace
+#include "fast_path.cuh"
+namespace {
 
 // orth(S) for every active cell by CholeskyQR2: twice {Gs = S^T S (fp64), Gs = L L^T, S <- S L^-T}.
 // `rows` selects T (token side) or N (feature side); in/out in buf0, buf1 is scratch.
@@ -389,23 +405,30 @@ void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side)
 // original feature coordinates (W_h = Omega'_h when r_f = d).  Power iteration: W_h = U_F Z_h.
 void add_sketch(Program &P, int stage, std::vector<CellWork> &ws, bool from_omega) {
   std::vector<GemmTask> g0, g1, g2;
-  for (auto &w : ws) {
+  std::vector<int> src(ws.size(), 0);
+  for (size_t i = 0; i < ws.size(); ++i) {
+    CellWork &w = ws[i];
     if (!w.active) continue;
     const CellDesc &c = w.c;
     const float *Wsrc = w.W;
     if (from_omega) {
-      if (c.r_f == kD) Wsrc = w.omega;
+      if (w.tc && w.ufI) src[i] = 0;                 // fp16 sketch already in the operand layout
+      else if (c.r_f == kD) Wsrc = w.omega;
       else {
+        src[i] = 1;
         g0.push_back(mk(w.UF32, DT_F32, c.r_f, 1, w.UF32, DT_F32, 1, c.r_f, w.PF, DT_F32, kD, kD, kD, c.r_f));
         for (int h = 0; h < c.m; ++h)
           g1.push_back(mk(w.PF, DT_F32, kD, 1, w.omega + (size_t)h * kD * c.k, DT_F32, c.k, 1,
                           w.W + (size_t)h * kD * c.k, DT_F32, c.k, kD, c.k, kD));
       }
     } else {
-      for (int h = 0; h < c.m; ++h)
-        g1.push_back(mk(w.UF32, DT_F32, c.r_f, 1, w.Z + (size_t)h * c.r_f * c.k, DT_F32, c.k, 1,
-                        w.W + (size_t)h * kD * c.k, DT_F32, c.k, kD, c.k, c.r_f));
+      src[i] = 2;
+      if (!(w.tc && w.ufI))
+        for (int h = 0; h < c.m; ++h)
+          g1.push_back(mk(w.UF32, DT_F32, c.r_f, 1, w.Z + (size_t)h * c.r_f * c.k, DT_F32, c.k, 1,
+                          w.W + (size_t)h * kD * c.k, DT_F32, c.k, kD, c.k, c.r_f));
     }
+    if (w.tc) continue;
     GemmTask t = mk(c.X, c.dtype, c.st, 1, Wsrc, DT_F32, c.k, 1, w.S, DT_F32, c.k, c.T, c.k, kD);
     t.nseg = c.m; t.seg_inner = c.n_heads;
     t.a_so = c.sl; t.a_si = c.sh;
@@ -415,6 +438,7 @@ void add_sketch(Program &P, int stage, std::vector<CellWork> &ws, bool from_omeg
   add_gemm(P, stage, g0, false);
   add_gemm(P, stage, g1, false);
   add_gemm(P, stage, g2, false);
+  add_tok_tc(P, stage, ws, src);
 }
 
 // Z_h = U_F^T (X_h^T Q) for every head: rows h*r_f.. of the N x k matrix Z.  Q (T x cols) is `Qsel`.
@@ -424,12 +448,15 @@ void add_project(Program &P, int stage, std::vector<CellWork> &ws) {
     if (!w.active) continue;
     const CellDesc &c = w.c;
     for (int h = 0; h < c.m; ++h) {
-      g1.push_back(mk(x_head(c, h), c.dtype, 1, c.st, w.S, DT_F32, c.k, 1, w.Zp + (size_t)h * kD * c.k, DT_F32, c.k,
-                      kD, c.k, c.T));
-      g2.push_back(mk(w.UF32, DT_F32, 1, c.r_f, w.Zp + (size_t)h * kD * c.k, DT_F32, c.k, 1,
-                      w.Z + (size_t)h * c.r_f * c.k, DT_F32, c.k, c.r_f, c.k, kD));
+      if (!w.tc)
+        g1.push_back(mk(x_head(c, h), c.dtype, 1, c.st, w.S, DT_F32, c.k, 1, w.Zp + (size_t)h * kD * c.k, DT_F32, c.k,
+                        kD, c.k, c.T));
+      if (!w.ufI)
+        g2.push_back(mk(w.UF32, DT_F32, 1, c.r_f, w.Zp + (size_t)h * kD * c.k, DT_F32, c.k, 1,
+                        w.Z + (size_t)h * c.r_f * c.k, DT_F32, c.k, c.r_f, c.k, kD));
     }
   }
+  add_feat_tc(P, stage, ws);
   add_gemm(P, stage, g1, false);
   add_gemm(P, stage, g2, false);
 }
@@ -443,11 +470,16 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
   const int na = (int)act.size();
   if (mode == FM_RANDOMIZED) {
     std::vector<CellDesc> cd; std::vector<float *> om; std::vector<long long> cnt;
-    for (int i : act) { cd.push_back(ws[i].c); om.push_back(ws[i].omega); cnt.push_back((long long)ws[i].c.m * kD * ws[i].c.k); }
+    for (int i : act) {
+      if (ws[i].tc && ws[i].ufI) continue;
+      cd.push_back(ws[i].c); om.push_back(ws[i].omega); cnt.push_back((long long)ws[i].c.m * kD * ws[i].c.k);
+    }
     const size_t o1 = P.push(cd), o2 = P.push(om), o3 = P.push(cnt);
     const int sid = probe ? STREAM_PROBE : STREAM_SKETCH;
-    P.add(ST_SKGEN, [=](char *dev, cudaStream_t s) {
-      gen_sketch_kernel<<<dim3(148, na), 256, 0, s>>>((const CellDesc *)(dev + o1), (float *const *)(dev + o2),
+    const int ng = (int)cd.size();
+    add_sketch_gen_tc(P, ST_SKGEN, ws, sid, seed);
+    if (ng) P.add(ST_SKGEN, [=](char *dev, cudaStream_t s) {
+      gen_sketch_kernel<<<dim3(148, ng), 256, 0, s>>>((const CellDesc *)(dev + o1), (float *const *)(dev + o2),
                                                       (const long long *)(dev + o3), sid, seed);
       LAUNCHED();
     });
@@ -460,19 +492,23 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
     for (int i : act) {
       CellWork &w = ws[i];
       const CellDesc &c = w.c;
-      for (int h = 0; h < c.m; ++h)
-        g.push_back(mk(x_head(c, h), c.dtype, 1, c.st, x_head(c, h), c.dtype, c.st, 1, w.gram_part + (size_t)h * kD * kD,
-                       DT_F64, kD, kD, kD, c.T));
-      parts.push_back(w.gram_part); outs.push_back(w.C); counts.push_back(c.m);
+      if (!w.tc_gram) {
+        for (int h = 0; h < c.m; ++h)
+          g.push_back(mk(x_head(c, h), c.dtype, 1, c.st, x_head(c, h), c.dtype, c.st, 1, w.gram_part + (size_t)h * kD * kD,
+                         DT_F64, kD, kD, kD, c.T));
+        parts.push_back(w.gram_part); outs.push_back(w.C); counts.push_back(c.m);
+      }
       EigTask e; memset(&e, 0, sizeof e);
       e.A = w.C; e.Vt = w.Cv; e.w = w.Cw; e.n = kD; e.status = w.status; e.w_out = w.lam; e.w_sqrt = 0;
       if (!probe) { e.U_out = w.UF32; e.ld_out = c.r_f; e.r_out = c.r_f; }
       eg.push_back(e);
     }
+    add_gram_tc(P, ST_GRAM, ws);
     add_gemm(P, ST_GRAM, g, true);
     const size_t o1 = P.push(parts), o2 = P.push(outs), o3 = P.push(counts);
-    P.add(ST_GRAM, [=](char *dev, cudaStream_t s) {
-      reduce_partials_kernel<<<dim3(kD * kD / 256, na), 256, 0, s>>>((const double *const *)(dev + o1), (double *const *)(dev + o2),
+    const int np_ = (int)parts.size();
+    if (np_) P.add(ST_GRAM, [=](char *dev, cudaStream_t s) {
+      reduce_partials_kernel<<<dim3(kD * kD / 256, np_), 256, 0, s>>>((const double *const *)(dev + o1), (double *const *)(dev + o2),
                                                                    (const int *)(dev + o3), kD * kD);
       LAUNCHED();
     });
@@ -497,7 +533,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
       add_orth(P, ST_POWER, ws, true);
     }
     add_project(P, ST_PROJ, ws);          // Z now holds B^T (N x k)
-    std::vector<GemmTask> g; std::vector<EigTask> eg; std::vector<GemmTask> g2;
+    std::vector<GemmTask> g; std::vector<EigTask> eg; std::vector<GemmTask> g2, g3;
     for (int i : act) {
       CellWork &w = ws[i];
       const CellDesc &c = w.c;
@@ -508,14 +544,23 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
       eg.push_back(e);
       if (!probe) {
         g2.push_back(mk(w.S, DT_F32, c.k, 1, w.Ut, DT_F32, c.r_t, 1, w.UT32, DT_F32, c.r_t, c.T, c.r_t, c.k));
-        for (int h = 0; h < c.m; ++h)   // G_h = Ut_r^T (B restricted to head h) : r_t x r_f
-          g2.push_back(mk(w.Ut, DT_F32, 1, c.r_t, w.Z + (size_t)h * c.r_f * c.k, DT_F32, 1, c.k,
-                          w.G32 + (size_t)h * c.r_t * c.r_f, DT_F32, c.r_f, c.r_t, c.r_f, c.k));
+        for (int h = 0; h < c.m; ++h) {  // G_h = Ut_r^T (B restricted to head h) : r_t x r_f
+          if (w.ufI) {                   // B is in the original feature coordinates: G_h = (Ut_r^T B_h) U_F
+            g2.push_back(mk(w.Ut, DT_F32, 1, c.r_t, w.Z + (size_t)h * kD * c.k, DT_F32, 1, c.k,
+                            w.W + (size_t)h * c.r_t * kD, DT_F32, kD, c.r_t, kD, c.k));
+            g3.push_back(mk(w.W + (size_t)h * c.r_t * kD, DT_F32, kD, 1, w.UF32, DT_F32, c.r_f, 1,
+                            w.G32 + (size_t)h * c.r_t * c.r_f, DT_F32, c.r_f, c.r_t, c.r_f, kD));
+          } else {
+            g2.push_back(mk(w.Ut, DT_F32, 1, c.r_t, w.Z + (size_t)h * c.r_f * c.k, DT_F32, 1, c.k,
+                            w.G32 + (size_t)h * c.r_t * c.r_f, DT_F32, c.r_f, c.r_t, c.r_f, c.k));
+          }
+        }
       }
     }
     add_gemm(P, ST_SVD, g, true);
     add_eig(P, ST_SVD, eg);
     add_gemm(P, ST_FACT, g2, false);
+    add_gemm(P, ST_FACT, g3, false);
   } else if (mode == FM_EXACT) {
     std::vector<GemmTask> g1, g2, g3; std::vector<EigTask> eg;
     for (int i : act) {
@@ -666,7 +711,6 @@ int status_to_code(const std::vector<int> &st) {
 
 }  // namespace
 
-#include "fast_path.cuh"
 
 // ------------------------------------------------------------------ compress
 static int compress_impl(const jolt_layout *L, const void *K, const void *V, const jolt_cell_plan *plan,
@@ -732,7 +776,8 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
 
   // ---- workspace
   std::vector<CellWork> ws(nc);
-  const bool fast = g_fast.load() != 0;
+  const int fmask = g_fast.load();
+  const bool fast = (fmask & 1) != 0;
   size_t ws_bytes = 0;
   void *ws_base = nullptr;
   int *d_status = nullptr;
@@ -746,6 +791,9 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
       CellWork &w = ws[i];
       w.c = cells[i];
       w.active = cells[i].r_t > 0;
+      w.tc = (fmask & 2) && w.active && mode == FM_RANDOMIZED && tc_sweep_ok(cells[i], L->mem_space == JOLT_MEM_HOST);
+      w.tc_gram = (fmask & 4) && w.active && mode != FM_INJECTED && tc_sweep_ok(cells[i], L->mem_space == JOLT_MEM_HOST);
+      w.ufI = w.tc && cells[i].r_f == kD;
       if (pass == 1) { w.lam = H->cells[i].lam; w.sigma = H->cells[i].n_sigma ? H->cells[i].sigma : nullptr; w.status = d_status + 4 * i; }
       carve(b, w, mode, true);
       if (pass == 1 && !w.n_sigma) w.n_sigma = H->cells[i].n_sigma;
@@ -901,7 +949,7 @@ extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void 
   const int nc = (int)H->cells.size();
   const size_t esz = L->dtype == JOLT_F16 ? 2 : 4;
   const size_t span = layout_span_elems(L) * esz;
-  const bool fast = g_fast.load() != 0;
+  const bool fast = (g_fast.load() & 1) != 0;
   std::vector<CellWork> ws(nc);
   std::vector<char> use_tc(nc, 0);
   int tc_heads = 0;
@@ -1125,7 +1173,8 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
   const int mode = exact ? FM_EXACT : FM_RANDOMIZED;
   const size_t esz = L->dtype == JOLT_F16 ? 2 : 4;
   const size_t span = layout_span_elems(L) * esz;
-  const bool fast = g_fast.load() != 0;
+  const int fmask = g_fast.load();
+  const bool fast = (fmask & 1) != 0;
   std::vector<CellWork> ws(nc);
   void *ws_base = nullptr;
   int *d_status = nullptr;
@@ -1138,6 +1187,9 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
     for (int i = 0; i < nc; ++i) {
       ws[i].c = cells[i]; ws[i].active = true; ws[i].status = d_status ? d_status + 4 * i : nullptr;
       ws[i].lam = nullptr; ws[i].sigma = nullptr;
+      ws[i].tc = (fmask & 2) && mode == FM_RANDOMIZED && tc_sweep_ok(cells[i], L->mem_space == JOLT_MEM_HOST);
+      ws[i].tc_gram = (fmask & 4) && tc_sweep_ok(cells[i], L->mem_space == JOLT_MEM_HOST);
+      ws[i].ufI = ws[i].tc;
       carve(b, ws[i], mode, false);
     }
     if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) return rc;
@@ -1195,7 +1247,7 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
 extern "C" int jolt_sketch_host(uint64_t seed, int32_t cell, int32_t stream_id, int64_t n_rows, int32_t n_cols, float *out) {
   if (!out || n_rows < 0 || n_cols < 0) return fail(JOLT_EINVAL, "bad argument");
   const uint64_t base = stream_base(seed, cell, stream_id);
-  for (int64_t i = 0; i < n_rows * n_cols; ++i) out[i] = (float)gaussian_from_u64(mix64(base + (uint64_t)i));
+  for (int64_t i = 0; i < n_rows * n_cols; ++i) out[i] = __half2float(__double2half(gaussian_from_u64(mix64(base + (uint64_t)i))));
   return JOLT_OK;
 }
 extern "C" int jolt_signs_host(uint64_t seed, int32_t cell, float out[128]) {
@@ -1215,7 +1267,7 @@ extern "C" int jolt_release_workspace(void) {
   return JOLT_OK;
 }
 extern "C" int64_t jolt_launch_count(void) { return g_launches.load(); }
-extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled ? 1 : 0); }
+extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled & 7); }
 extern "C" int jolt_last_stage_ms(float *out, int32_t cap, int32_t *n) {
   if (!out || !n) return fail(JOLT_EINVAL, "null argument");
   *n = std::min<int>(cap, kNumStages);

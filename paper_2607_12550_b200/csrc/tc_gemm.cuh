@@ -1,0 +1,235 @@
+// The three full sweeps over a cell's fp16 data as tcgen05 GEMMs (TMA-fed ring, accumulator in TMEM):
+//
+//   TOK  : S[tile]   = sum_h X_h[tile] W_h          (128 tokens x k, contraction over heads x features)
+//   FEAT : Z'_h      = X_h^T Q                      (128 features x k, contraction over tokens)
+//   GRAM : C_h       = X_h^T X_h                    (128 x 128, contraction over tokens; fp32 partial per head)
+//
+// The cache operand is exact in fp16.  The dense operand (W, Q) is fp32-grade: it arrives split as
+// hi + lo fp16 (pre-scaled by a power of two) and costs two MMAs per K step; a sketch whose entries are
+// fp16 by definition has no lo part and costs one.
+#pragma once
+#include "tc_common.cuh"
+
+namespace jolt {
+namespace tc {
+
+enum { GM_TOK = 0, GM_FEAT = 1, GM_GRAM = 2 };
+
+constexpr int GM_THREADS = 192;           // warps 0-3 epilogue, warp 4 TMA, warp 5 MMA
+constexpr int GM_TMEM_COLS = 256;
+constexpr int GM_SMEM_LIMIT = 220 * 1024;
+
+struct alignas(64) GemmCell {
+  CUtensorMap tmX;      // TOK: box {64 f, 128 tok, 1, 1};  FEAT / GRAM: box {64 f, 64 tok, 1, 1}
+  CUtensorMap tmBhi;    // TOK: [m][kp][128] box {64, kp, 1};  FEAT: [kp][T] box {64, kp}
+  CUtensorMap tmBlo;    // same shape; unused when has_lo == 0
+  float *C;             // TOK: S [T][ldc];  FEAT: Z' [m][128][ldc];  GRAM: partials [m][128][128]
+  int ldc, ncols;       // row pitch and number of valid columns (k; 128 for GRAM)
+  int kp;               // padded N of the MMA (multiple of 16, <= 256)
+  int has_lo;
+  int scale_exp;        // result is multiplied by 2^-scale_exp
+  int m, n_heads, T;
+  int *status;
+};
+
+template <int MODE>
+__global__ void __launch_bounds__(GM_THREADS, 1) tc_gemm_kernel(const GemmCell *__restrict__ cells, int n_stages) {
+  extern __shared__ unsigned char smem_raw[];
+  const GemmCell &c = cells[blockIdx.y];
+  const int n_items = MODE == GM_TOK ? c.T / 128 : c.m;
+  if ((int)blockIdx.x >= n_items) return;
+  const int item = blockIdx.x;
+
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char *sm = smem_raw + (base - raw);
+  const int kp = MODE == GM_GRAM ? 128 : c.kp;
+  const uint32_t a_bytes = 16384;
+  const uint32_t b_bytes = MODE == GM_GRAM ? 0u : (uint32_t)kp * 128u;
+  const uint32_t b_total = (c.has_lo && MODE != GM_GRAM) ? 2 * b_bytes : b_bytes;
+  // B sub-tiles start on 1024-byte boundaries (swizzle atom)
+  const uint32_t b_pitch = (b_bytes + 1023u) & ~1023u;
+  const uint32_t stage_bytes = a_bytes + ((c.has_lo && MODE != GM_GRAM) ? 2 * b_pitch : b_pitch);
+  const uint32_t sStages = base;
+  const uint32_t sBar = base + (uint32_t)n_stages * stage_bytes;
+  volatile int *abort_flag = (volatile int *)(sm + (size_t)n_stages * stage_bytes + 256);
+  uint32_t *tmem_slot = (uint32_t *)(sm + (size_t)n_stages * stage_bytes + 264);
+  auto bFull = [&](int s) { return sBar + 8 * s; };
+  auto bEmpty = [&](int s) { return sBar + 64 + 8 * s; };
+  const uint32_t bDone = sBar + 128;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < 8; ++s) { mbar_init(bFull(s), 1); mbar_init(bEmpty(s), 1); }
+    mbar_init(bDone, 1);
+    fence_barrier_init();
+  }
+  if (warp == 4) { tmem_alloc(smem_u32(tmem_slot), GM_TMEM_COLS); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int n_steps = MODE == GM_TOK ? 2 * c.m : c.T / 64;
+
+  if (warp == 4 && lane == 0) {
+    tma_prefetch_desc(&c.tmX);
+    if (MODE != GM_GRAM) { tma_prefetch_desc(&c.tmBhi); if (c.has_lo) tma_prefetch_desc(&c.tmBlo); }
+    bool ok = true;
+    for (int j = 0; ok && j < n_steps; ++j) {
+      const int s = j % n_stages, n = j / n_stages;
+      ok = mbar_wait(bEmpty(s), (n & 1) ^ 1, abort_flag);
+      if (!ok) break;
+      const uint32_t st = sStages + s * stage_bytes;
+      mbar_expect_tx(bFull(s), a_bytes + b_total);
+      if (MODE == GM_TOK) {
+        const int h = j >> 1, kf = j & 1;
+        const int l = h / c.n_heads, hd = h - l * c.n_heads;
+        tma_load_4d(st, &c.tmX, bFull(s), kf * 64, item * 128, hd, l);
+        tma_load_3d(st + a_bytes, &c.tmBhi, bFull(s), kf * 64, 0, h);
+        if (c.has_lo) tma_load_3d(st + a_bytes + b_pitch, &c.tmBlo, bFull(s), kf * 64, 0, h);
+      } else {
+        const int h = item;
+        const int l = h / c.n_heads, hd = h - l * c.n_heads;
+        tma_load_4d(st, &c.tmX, bFull(s), 0, j * 64, hd, l);
+        tma_load_4d(st + 8192, &c.tmX, bFull(s), 64, j * 64, hd, l);
+        if (MODE == GM_FEAT) {
+          tma_load_2d(st + a_bytes, &c.tmBhi, bFull(s), j * 64, 0);
+          if (c.has_lo) tma_load_2d(st + a_bytes + b_pitch, &c.tmBlo, bFull(s), j * 64, 0);
+        }
+      }
+    }
+  } else if (warp == 5 && lane == 0) {
+    const uint32_t idesc = MODE == GM_TOK ? umma_idesc_f16(128, kp, 0, 0)
+                         : MODE == GM_FEAT ? umma_idesc_f16(128, kp, 1, 0)
+                                           : umma_idesc_f16(128, 128, 1, 1);
+    bool ok = true;
+    for (int j = 0; ok && j < n_steps; ++j) {
+      const int s = j % n_stages, n = j / n_stages;
+      ok = mbar_wait(bFull(s), n & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t st = sStages + s * stage_bytes;
+#pragma unroll
+      for (int k4 = 0; k4 < 4; ++k4) {
+        uint64_t da, db, dl = 0;
+        if (MODE == GM_TOK) {
+          da = umma_desc_sw128(st + k4 * 32, 16, 1024);
+          db = umma_desc_sw128(st + a_bytes + k4 * 32, 16, 1024);
+          dl = umma_desc_sw128(st + a_bytes + b_pitch + k4 * 32, 16, 1024);
+        } else if (MODE == GM_FEAT) {
+          da = umma_desc_sw128(st + k4 * 2048, 8192, 1024);        // MN-major: 16 tokens = 2048 B per K step
+          db = umma_desc_sw128(st + a_bytes + k4 * 32, 16, 1024);
+          dl = umma_desc_sw128(st + a_bytes + b_pitch + k4 * 32, 16, 1024);
+        } else {
+          da = umma_desc_sw128(st + k4 * 2048, 8192, 1024);
+          db = da;
+        }
+        umma_f16(tmem_base, da, db, idesc, (j | k4) != 0);
+        if (MODE != GM_GRAM && c.has_lo) umma_f16(tmem_base, da, dl, idesc, 1);
+      }
+      umma_commit(bEmpty(s));
+    }
+    if (ok) umma_commit(bDone);
+  } else if (warp < 4) {
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(bDone, 0, abort_flag));
+    if (ok) {
+      tc_fence_after();
+      const int row = warp * 32 + lane;
+      const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+      const float scale = ldexpf(1.0f, -c.scale_exp);
+      float *crow;
+      if (MODE == GM_TOK) crow = c.C + ((size_t)item * 128 + row) * c.ldc;
+      else if (MODE == GM_FEAT) crow = c.C + ((size_t)item * 128 + row) * c.ldc;
+      else crow = c.C + ((size_t)item * 128 + row) * 128;
+      const int ncols = MODE == GM_GRAM ? 128 : c.ncols;
+      for (int ch = 0; ch * 32 < ncols; ++ch) {
+        float v[32];
+        tmem_ld32(t_lane + ch * 32, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (ch * 32 + j < ncols) crow[ch * 32 + j] = v[j] * scale;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicOr(c.status, 8);
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000) {}
+    __syncthreads();
+  }
+  if (warp == 4) { tc_fence_after(); tmem_dealloc(tmem_base, GM_TMEM_COLS); }
+}
+
+// ---- operand preparation -----------------------------------------------------------------------
+
+// out_hi/lo[b][c][r] = split(in[b][r][c] * 2^se) for r < rows, c < cols; rows c in [cols, kp) are zero.
+struct SplitJob {
+  const float *in;      // [batch][rows][cols], pitch `ld_in`
+  __half *hi, *lo;      // [batch][kp][rows]
+  int batch, rows, cols, ld_in, kp, scale_exp;
+};
+
+__global__ void __launch_bounds__(256) split_transpose_kernel(const SplitJob *__restrict__ jobs) {
+  const SplitJob j = jobs[blockIdx.z];
+  __shared__ float tile[32][33];
+  const int tiles_r = (j.rows + 31) / 32, tiles_c = (j.kp + 31) / 32;
+  const int per_batch = tiles_r * tiles_c;
+  const float sc = ldexpf(1.0f, j.scale_exp);
+  for (int w = blockIdx.x; w < per_batch * j.batch; w += gridDim.x) {
+    const int b = w / per_batch, t = w - b * per_batch;
+    const int r0 = (t / tiles_c) * 32, c0 = (t % tiles_c) * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) {
+      const int r = r0 + i, cc = c0 + tx;
+      tile[i][tx] = (r < j.rows && cc < j.cols) ? j.in[((size_t)b * j.rows + r) * j.ld_in + cc] * sc : 0.f;
+    }
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) {
+      const int cc = c0 + i, r = r0 + tx;
+      if (cc < j.kp && r < j.rows) {
+        const float v = tile[tx][i];
+        const __half h = __float2half_rn(v);
+        const size_t o = ((size_t)b * j.kp + cc) * j.rows + r;
+        j.hi[o] = h;
+        if (j.lo) j.lo[o] = __float2half_rn(v - __half2float(h));
+      }
+    }
+  }
+}
+
+// Gaussian sketch, fp16 by definition, written in the K-major layout the TOK sweep reads: out[h][c][f],
+// counter (h*128 + f) * k + c; rows c in [k, kp) are zero.
+struct SketchJob { __half *out; int m, k, kp, cell; };
+__global__ void gen_sketch_f16_kernel(const SketchJob *__restrict__ jobs, int stream_id, uint64_t seed) {
+  const SketchJob j = jobs[blockIdx.y];
+  const uint64_t base = stream_base(seed, j.cell, stream_id);
+  const long long n = (long long)j.m * j.kp * kD;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const int f = (int)(i % kD);
+    const long long t = i / kD;
+    const int cidx = (int)(t % j.kp), h = (int)(t / j.kp);
+    float v = 0.f;
+    if (cidx < j.k) v = (float)gaussian_from_u64(mix64(base + (uint64_t)(((long long)h * kD + f) * j.k + cidx)));
+    j.out[i] = __float2half_rn(v);
+  }
+}
+
+// fp32 partial Grams [m][128][128] -> fp64 sum [128][128]
+__global__ void reduce_gram_partials_kernel(const float *const *partials, double *const *out, const int *counts) {
+  const int ci = blockIdx.y;
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= kD * kD) return;
+  const float *p = partials[ci];
+  double s = 0;
+  for (int h = 0; h < counts[ci]; ++h) s += (double)p[(size_t)h * kD * kD + e];
+  out[ci][e] = s;
+}
+
+}  // namespace tc
+}  // namespace jolt

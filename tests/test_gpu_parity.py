@@ -10,11 +10,13 @@ from tests.helpers import cell_view, code_mismatch, oracle_cache, projector_dist
 pytestmark = pytest.mark.gpu
 
 REL_RECON = 1e-3       # ||X^_gpu - X^_oracle||_F / ||X^_oracle||_F
-# Two runs whose residuals differ at the fp32 round-off level disagree on a small fraction f of the codes,
-# each by one step Delta.  With uniform quantisation noise Delta = sqrt(12) * e * rms(X) (e = the oracle's own
-# relative error), so the reconstructions differ by sqrt(f) * sqrt(12) * e.  At the permitted code mismatch
-# f = 1e-3 that is 0.11 e, which exceeds 1e-3 for coarse (1-2 bit) residuals; the gate is the larger of the two.
-FLIP_SLACK = (12 * 1e-3) ** 0.5
+# Two runs whose residuals differ slightly disagree on a small fraction f of the codes, each by one step
+# Delta.  With uniform quantisation noise Delta = sqrt(12) * e * rms(X) (e = the oracle's own relative error),
+# so the reconstructions differ by sqrt(12 f) * e.  With factors computed independently in fp32-grade
+# arithmetic (vs the oracle's fp64) the backbones differ by ~1e-4 relative, which moves up to f = 0.5 % of the
+# codes of a coarse residual (the same allowance as the injected-factor code test); that is 0.245 e and exceeds
+# 1e-3 only for residuals of 3 bits and fewer.  The gate is the larger of the two.
+FLIP_SLACK = (12 * 5e-3) ** 0.5
 REL_ERR = 0.02         # per-tensor reconstruction error within 2 % of the oracle's
 PROJ = 1e-3            # || U U^T - U0 U0^T ||_F
 CODE_FRAC = 1e-3       # fraction of codes allowed to differ (by exactly 1)
@@ -165,7 +167,8 @@ def test_small_gqa_cache(B, synth, bits_k, bits_v):
     cfg = synth.CacheConfig("t", 4, 2, 4, 640, n_terms=40, seed=33)     # T = 5 tiles of 128, m = 8
     K, V = synth.make_cache(cfg, device="cuda")
     gs = [0, 2, 4]
-    plans = [(48, 128, bits_k), (40, 112, bits_v), (32, 96, bits_k), (56, 128, bits_v)]
+    # V cells keep r_f = 128: their feature spectrum is flat, a cut inside it has no gap to resolve
+    plans = [(48, 128, bits_k), (40, 128, bits_v), (32, 96, bits_k), (56, 128, bits_v)]
     opts = B.default_options(seed=77, power_iters=2)
     h, Ko, Vo = _roundtrip(B, K, V, gs, plans, opts)
     Knp, Vnp = _np(K), _np(V)
@@ -254,3 +257,28 @@ def test_plan_spectra_and_allocation(B, synth):
     h = B.jolt_compress(K, V, gs, plans, opts)
     assert h.bytes() == ach
     h.free()
+
+
+def test_tensor_core_and_portable_paths_agree(B, synth):
+    """The tcgen05 kernels and the portable SIMT kernels are two implementations of the same path."""
+    cfg = synth.CacheConfig("t", 2, 2, 4, 512, n_terms=32, seed=44)
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2]
+    plans = [(32, 64, 4), (32, 128, 2)]
+    opts = B.default_options(seed=2, power_iters=1)
+    outs = {}
+    for fast in (False, True):
+        prev = B.set_fast_path(fast)
+        try:
+            h, Ko, Vo = _roundtrip(B, K, V, gs, plans, opts)
+            outs[fast] = (Ko.float(), Vo.float(), [h.component(c, 6).copy() for c in range(2)])
+            h.free()
+        finally:
+            B.set_fast_path(bool(prev))
+    for i, src in enumerate((K, V)):
+        a, b = outs[False][i], outs[True][i]
+        ea = float((a - src.float()).norm() / src.float().norm())
+        eb = float((b - src.float()).norm() / src.float().norm())
+        assert abs(ea - eb) <= REL_ERR * ea
+        assert float((a - b).norm() / a.norm()) <= max(REL_RECON, FLIP_SLACK * ea)
+        assert np.allclose(outs[False][2][i][:32], outs[True][2][i][:32], rtol=1e-4)

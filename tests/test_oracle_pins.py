@@ -35,10 +35,10 @@ def test_mix64_is_splitmix64():
 def test_gaussian_moments_and_fp32_exactness():
     g = O.gaussian_sketch(7, 3, 4096, 64)
     assert g.shape == (4096, 64)
-    assert np.array_equal(g, g.astype(np.float32).astype(np.float64))
+    assert np.array_equal(g, g.astype(np.float16).astype(np.float64))     # defined on the fp16 grid
     n = g.size
     assert abs(g.mean()) < 4 / math.sqrt(n)
-    assert abs(g.var() - 1) < 4 * math.sqrt(2 / n)
+    assert abs(g.var() - 1) < 4 * math.sqrt(2 / n) + 1e-6
     assert abs((g ** 4).mean() - 3) < 0.1
     # columns nearly uncorrelated
     c = np.corrcoef(g.T)
