@@ -346,7 +346,12 @@ def compress_cell(X, r_t: int, r_f: int, bits: int, *, seed: int = 0, cell: int 
             lam = None
             sig = None
         else:
-            U_F, lam = feature_factor(X, r_f)
+            if r_f == d:
+                # no feature truncation: the mode-3 factor of an untruncated mode is any orthogonal
+                # basis of R^d; the identity is taken (as for the pinned head and layer modes)
+                U_F, lam = np.eye(d), None
+            else:
+                U_F, lam = feature_factor(X, r_f)
             Y = np.einsum("htf,fs->hts", X, U_F, optimize=True)
             A = token_unfold(Y)
             N = A.shape[1]

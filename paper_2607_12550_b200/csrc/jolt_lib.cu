@@ -6,6 +6,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <chrono>
 #include <functional>
 #include <memory>
 #include <mutex>
@@ -24,6 +25,7 @@ using namespace jolt;
 namespace jolt {
 thread_local std::string g_err;
 std::atomic<long long> g_launches{0};
+std::atomic<int> g_eig_smem{1};
 std::atomic<int> g_fast{7};   // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores
 
 int fail(int code, const char *fmt, ...) {
@@ -277,15 +279,46 @@ void add_gemm(Program &P, int stage, const std::vector<GemmTask> &tasks, bool f6
 
 void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks) {
   if (tasks.empty()) return;
-  int mn = 0;
-  for (auto &t : tasks) mn = std::max(mn, t.n);
-  const size_t off = P.push(tasks);
-  const int n = (int)tasks.size();
-  const size_t shm = (size_t)(2 * ((mn + 1) / 2) + 32) * sizeof(double);
-  P.add(stage, [=](char *dev, cudaStream_t s) {
-    jacobi_eig_kernel<<<n, kEigThreads, shm, s>>>((const EigTask *)(dev + off));
-    LAUNCHED();
-  });
+  // problems that fit one CTA's shared memory take the resident kernel, the rest the global-memory one
+  std::vector<EigTask> small64, small32, big;
+  for (auto &t : tasks) {
+    if (!g_eig_smem.load() || t.n > kEigSmemMaxN) big.push_back(t);
+    else if (eig_smem_bytes(t.n, 8) <= kSmemOptIn - 1024) small64.push_back(t);   // fp64 eigenvector accumulator fits
+    else if (eig_smem_bytes(t.n, 4) <= kSmemOptIn - 1024) small32.push_back(t);
+    else big.push_back(t);
+  }
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaFuncSetAttribute(jacobi_eig_smem_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemOptIn - 1024));
+    cudaFuncSetAttribute(jacobi_eig_smem_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemOptIn - 1024));
+    attr_done = true;
+  }
+  for (int pass = 0; pass < 2; ++pass) {
+    const std::vector<EigTask> &small = pass == 0 ? small64 : small32;
+    if (small.empty()) continue;
+    int mn = 0;
+    for (auto &t : small) mn = std::max(mn, t.n);
+    const size_t shm = eig_smem_bytes(mn, pass == 0 ? 8 : 4);
+    const size_t off = P.push(small);
+    const int n = (int)small.size();
+    const bool dbl = pass == 0;
+    P.add(stage, [=](char *dev, cudaStream_t s) {
+      if (dbl) jacobi_eig_smem_kernel<double><<<n, kEigThreads, shm, s>>>((const EigTask *)(dev + off));
+      else jacobi_eig_smem_kernel<float><<<n, kEigThreads, shm, s>>>((const EigTask *)(dev + off));
+      LAUNCHED();
+    });
+  }
+  if (!big.empty()) {
+    int mn = 0;
+    for (auto &t : big) mn = std::max(mn, t.n);
+    const size_t off = P.push(big);
+    const int n = (int)big.size();
+    const size_t shm = (size_t)(2 * ((mn + 1) / 2) + 32) * sizeof(double);
+    P.add(stage, [=](char *dev, cudaStream_t s) {
+      jacobi_eig_kernel<<<n, kEigThreads, shm, s>>>((const EigTask *)(dev + off));
+      LAUNCHED();
+    });
+  }
 }
 
 void add_chol(Program &P, int stage, const std::vector<CholTask> &tasks) {
@@ -311,6 +344,7 @@ struct CellWork {      // device scratch of one cell
   float *UF32 = nullptr, *lam = nullptr;
   float *omega = nullptr, *PF = nullptr, *W = nullptr, *S = nullptr, *S2 = nullptr, *Zp = nullptr, *Z = nullptr, *Z2 = nullptr;
   double *Gs = nullptr, *Linv = nullptr; float *LinvT = nullptr;
+  double *gpart = nullptr; float *LT32 = nullptr, *invd = nullptr;
   double *BBt = nullptr, *BBv = nullptr, *BBw = nullptr;
   float *Ut = nullptr, *sigma = nullptr;
   float *UT32 = nullptr, *G32 = nullptr;
@@ -322,12 +356,14 @@ struct CellWork {      // device scratch of one cell
   // tensor-core sweeps
   bool tc = false;           // sketch / projection sweeps run on tcgen05
   bool tc_gram = false;      // mode-3 Gram runs on tcgen05
-  bool ufI = false;          // r_f = d: the token factor is computed in the original feature coordinates
+  bool ufI = false;          // r_f = d: U_F = I, the token factor is computed in the original feature coordinates
+  bool skip_feat = false;    // no mode-3 Gram / eigen-solve needed
   int kp = 0;                // sketch width padded to a multiple of 16
   __half *Bhi = nullptr, *Blo = nullptr;
 };
 
 enum FactorMode { FM_RANDOMIZED = 0, FM_EXACT = 1, FM_INJECTED = 2 };
+constexpr int kGramChunks = 32;   // row chunks of a tall Gram (fp64 partial per chunk, summed in order)
 
 // Scratch layout of one cell; run with b.base == nullptr to size it.
 void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
@@ -358,6 +394,7 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
         w.Bhi = b.take<__half>(nb); w.Blo = b.take<__half>(nb);
       }
       w.Gs = b.take<double>(k * k); w.Linv = b.take<double>(k * k); w.LinvT = b.take<float>(k * k);
+      w.gpart = b.take<double>(kGramChunks * k * k); w.LT32 = b.take<float>(k * (k + 4)); w.invd = b.take<float>(k + 4);
       w.BBt = b.take<double>(k * k); w.BBv = b.take<double>(k * k); w.BBw = b.take<double>(k);
       w.Ut = b.take<float>(k * std::max<size_t>(c.r_t, 1));
       if (!(real && w.sigma)) w.sigma = b.take<float>(k);
@@ -379,25 +416,79 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
 #include "fast_path.cuh"
 namespace {
 
+// G = M^T M (k x k, fp64) of tall fp32 matrices, split over row chunks so that the grid fills the GPU;
+// the partials are summed in a fixed order.
+struct TallGram { const float *M; int rows, k; double *part, *out; };
+void add_tall_gram(Program &P, int stage, const std::vector<TallGram> &jobs) {
+  std::vector<GemmTask> g;
+  std::vector<ReduceJob> rj;
+  for (auto &j : jobs) {
+    int chunk = std::max(256, (j.rows + kGramChunks - 1) / kGramChunks);
+    chunk = (chunk + 15) & ~15;
+    int n = 0;
+    for (int r0 = 0; r0 < j.rows; r0 += chunk, ++n) {
+      const float *m0 = j.M + (size_t)r0 * j.k;
+      g.push_back(mk(m0, DT_F32, 1, j.k, m0, DT_F32, j.k, 1, j.part + (size_t)n * j.k * j.k, DT_F64, j.k, j.k, j.k,
+                     std::min(chunk, j.rows - r0)));
+    }
+    rj.push_back({j.part, j.out, n, j.k * j.k});
+  }
+  add_gemm(P, stage, g, true);
+  if (rj.empty()) return;
+  const size_t off = P.push(rj);
+  const int n = (int)rj.size();
+  P.add(stage, [=](char *dev, cudaStream_t s) {
+    reduce_partials_var_kernel<<<dim3(32, n), 256, 0, s>>>((const ReduceJob *)(dev + off));
+    LAUNCHED();
+  });
+}
+
 // orth(S) for every active cell by CholeskyQR2: twice {Gs = S^T S (fp64), Gs = L L^T, S <- S L^-T}.
-// `rows` selects T (token side) or N (feature side); in/out in buf0, buf1 is scratch.
+// token_side selects S (T rows) or Z (N rows); the result is left in the source buffer.
 void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side) {
   for (int pass = 0; pass < 2; ++pass) {
-    std::vector<GemmTask> g1, g2;
+    std::vector<TallGram> tg;
+    std::vector<GemmTask> g2;
     std::vector<CholTask> ch;
+    std::vector<CholSmemTask> chs;
+    std::vector<TrsmJob> tj;
+    int max_k = 0;
     for (auto &w : ws) {
       if (!w.active) continue;
       const int k = w.c.k, rows = token_side ? w.c.T : w.c.N;
       float *src = token_side ? (pass == 0 ? w.S : w.S2) : (pass == 0 ? w.Z : w.Z2);
       float *dst = token_side ? (pass == 0 ? w.S2 : w.S) : (pass == 0 ? w.Z2 : w.Z);
-      g1.push_back(mk(src, DT_F32, 1, k, src, DT_F32, k, 1, w.Gs, DT_F64, k, k, k, rows));
-      CholTask c; c.G = w.Gs; c.Linv = w.Linv; c.LinvT32 = w.LinvT; c.n = k; c.status = w.status;
-      ch.push_back(c);
-      g2.push_back(mk(src, DT_F32, k, 1, w.LinvT, DT_F32, k, 1, dst, DT_F32, k, rows, k, k));
+      tg.push_back({src, rows, k, w.gpart, w.Gs});
+      if (k <= kCholSmemMaxN) {
+        chs.push_back({w.Gs, w.LT32, w.invd, k, w.status});
+        tj.push_back({src, dst, rows, k, w.LT32, w.invd});
+        max_k = std::max(max_k, k);
+      } else {
+        CholTask c; c.G = w.Gs; c.Linv = w.Linv; c.LinvT32 = w.LinvT; c.n = k; c.status = w.status;
+        ch.push_back(c);
+        g2.push_back(mk(src, DT_F32, k, 1, w.LinvT, DT_F32, k, 1, dst, DT_F32, k, rows, k, k));
+      }
     }
-    add_gemm(P, stage, g1, true);
+    add_tall_gram(P, stage, tg);
     add_chol(P, stage, ch);
     add_gemm(P, stage, g2, false);
+    if (!chs.empty()) {
+      static bool attr_done = false;
+      if (!attr_done) {
+        cudaFuncSetAttribute(cholesky_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)chol_smem_bytes(kCholSmemMaxN));
+        cudaFuncSetAttribute(trsm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)trsm_smem_bytes(kCholSmemMaxN));
+        attr_done = true;
+      }
+      const size_t o1 = P.push(chs), o2 = P.push(tj);
+      const int n = (int)chs.size();
+      int max_rows = 0;
+      for (auto &t : tj) max_rows = std::max(max_rows, t.rows);
+      const size_t sh1 = chol_smem_bytes(max_k), sh2 = trsm_smem_bytes(max_k);
+      P.add(stage, [=](char *dev, cudaStream_t s) {
+        cholesky_smem_kernel<<<n, 1024, sh1, s>>>((const CholSmemTask *)(dev + o1)); LAUNCHED();
+        trsm_rows_kernel<<<dim3((max_rows + 127) / 128, n), 128, sh2, s>>>((const TrsmJob *)(dev + o2)); LAUNCHED();
+      });
+    }
   }
 }
 
@@ -413,7 +504,7 @@ void add_sketch(Program &P, int stage, std::vector<CellWork> &ws, bool from_omeg
     const float *Wsrc = w.W;
     if (from_omega) {
       if (w.tc && w.ufI) src[i] = 0;                 // fp16 sketch already in the operand layout
-      else if (c.r_f == kD) Wsrc = w.omega;
+      else if (w.ufI) Wsrc = w.omega;
       else {
         src[i] = 1;
         g0.push_back(mk(w.UF32, DT_F32, c.r_f, 1, w.UF32, DT_F32, 1, c.r_f, w.PF, DT_F32, kD, kD, kD, c.r_f));
@@ -423,7 +514,8 @@ void add_sketch(Program &P, int stage, std::vector<CellWork> &ws, bool from_omeg
       }
     } else {
       src[i] = 2;
-      if (!(w.tc && w.ufI))
+      if (w.ufI) Wsrc = w.Z;
+      else
         for (int h = 0; h < c.m; ++h)
           g1.push_back(mk(w.UF32, DT_F32, c.r_f, 1, w.Z + (size_t)h * c.r_f * c.k, DT_F32, c.k, 1,
                           w.W + (size_t)h * kD * c.k, DT_F32, c.k, kD, c.k, c.r_f));
@@ -489,9 +581,12 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
     std::vector<GemmTask> g;
     std::vector<const double *> parts; std::vector<double *> outs; std::vector<int> counts;
     std::vector<EigTask> eg;
+    std::vector<float *> idU; std::vector<int> idLd;
     for (int i : act) {
       CellWork &w = ws[i];
       const CellDesc &c = w.c;
+      if (w.ufI) { idU.push_back(w.UF32); idLd.push_back(c.r_f); }
+      if (w.ufI && !probe) { w.tc_gram = false; w.skip_feat = true; continue; }   // r_f = d: U_F = I, no Gram, no eigen-solve
       if (!w.tc_gram) {
         for (int h = 0; h < c.m; ++h)
           g.push_back(mk(x_head(c, h), c.dtype, 1, c.st, x_head(c, h), c.dtype, c.st, 1, w.gram_part + (size_t)h * kD * kD,
@@ -513,12 +608,11 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
       LAUNCHED();
     });
     add_eig(P, ST_EIGF, eg);
-    if (probe) {
-      std::vector<float *> us; std::vector<int> lds;
-      for (int i : act) { us.push_back(ws[i].UF32); lds.push_back(ws[i].c.r_f); }
-      const size_t p1 = P.push(us), p2 = P.push(lds);
+    if (!idU.empty()) {
+      const size_t p1 = P.push(idU), p2 = P.push(idLd);
+      const int nid = (int)idU.size();
       P.add(ST_EIGF, [=](char *dev, cudaStream_t s) {
-        set_identity_kernel<<<dim3(kD * kD / 256, na), 256, 0, s>>>((float *const *)(dev + p1), (const int *)(dev + p2));
+        set_identity_kernel<<<dim3(kD * kD / 256, nid), 256, 0, s>>>((float *const *)(dev + p1), (const int *)(dev + p2));
         LAUNCHED();
       });
     }
@@ -533,11 +627,11 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
       add_orth(P, ST_POWER, ws, true);
     }
     add_project(P, ST_PROJ, ws);          // Z now holds B^T (N x k)
-    std::vector<GemmTask> g; std::vector<EigTask> eg; std::vector<GemmTask> g2, g3;
+    std::vector<TallGram> tgb; std::vector<EigTask> eg; std::vector<GemmTask> g2, g3;
     for (int i : act) {
       CellWork &w = ws[i];
       const CellDesc &c = w.c;
-      g.push_back(mk(w.Z, DT_F32, 1, c.k, w.Z, DT_F32, c.k, 1, w.BBt, DT_F64, c.k, c.k, c.k, c.N));
+      tgb.push_back({w.Z, c.N, c.k, w.gpart, w.BBt});
       EigTask e; memset(&e, 0, sizeof e);
       e.A = w.BBt; e.Vt = w.BBv; e.w = w.BBw; e.n = c.k; e.status = w.status; e.w_out = w.sigma; e.w_sqrt = 1;
       if (!probe) { e.U_out = w.Ut; e.ld_out = c.r_t; e.r_out = c.r_t; }
@@ -545,11 +639,9 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
       if (!probe) {
         g2.push_back(mk(w.S, DT_F32, c.k, 1, w.Ut, DT_F32, c.r_t, 1, w.UT32, DT_F32, c.r_t, c.T, c.r_t, c.k));
         for (int h = 0; h < c.m; ++h) {  // G_h = Ut_r^T (B restricted to head h) : r_t x r_f
-          if (w.ufI) {                   // B is in the original feature coordinates: G_h = (Ut_r^T B_h) U_F
+          if (w.ufI) {                   // U_F = I: B is already in the stored feature coordinates
             g2.push_back(mk(w.Ut, DT_F32, 1, c.r_t, w.Z + (size_t)h * kD * c.k, DT_F32, 1, c.k,
-                            w.W + (size_t)h * c.r_t * kD, DT_F32, kD, c.r_t, kD, c.k));
-            g3.push_back(mk(w.W + (size_t)h * c.r_t * kD, DT_F32, kD, 1, w.UF32, DT_F32, c.r_f, 1,
-                            w.G32 + (size_t)h * c.r_t * c.r_f, DT_F32, c.r_f, c.r_t, c.r_f, kD));
+                            w.G32 + (size_t)h * c.r_t * kD, DT_F32, kD, c.r_t, kD, c.k));
           } else {
             g2.push_back(mk(w.Ut, DT_F32, 1, c.r_t, w.Z + (size_t)h * c.r_f * c.k, DT_F32, 1, c.k,
                             w.G32 + (size_t)h * c.r_t * c.r_f, DT_F32, c.r_f, c.r_t, c.r_f, c.k));
@@ -557,7 +649,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
         }
       }
     }
-    add_gemm(P, ST_SVD, g, true);
+    add_tall_gram(P, ST_SVD, tgb);
     add_eig(P, ST_SVD, eg);
     add_gemm(P, ST_FACT, g2, false);
     add_gemm(P, ST_FACT, g3, false);
@@ -719,6 +811,9 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   if (out) *out = nullptr;
   if (!out || !plan || !K || !V) return fail(JOLT_EINVAL, "null argument");
   int rc;
+  const bool dbg = getenv("JOLT_DEBUG_TIMING") != nullptr;
+  auto t_start = std::chrono::steady_clock::now();
+  auto lap = [&](const char *what) { if (dbg) { auto n = std::chrono::steady_clock::now(); fprintf(stderr, "[jolt] %s: %.3f ms\n", what, std::chrono::duration<double, std::milli>(n - t_start).count()); t_start = n; } };
   if ((rc = check_layout(L)) || (rc = check_options(o))) return rc;
   const bool injected = inUT != nullptr || inUF != nullptr;
   if (injected && (!inUT || !inUF)) return fail(JOLT_EINVAL, "both factor arrays are needed");
@@ -773,6 +868,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     }
   }
   auto free_blob = [&]() { cudaFreeAsync(H->blob, st); H->blob = nullptr; };
+  lap("validate+blob");
 
   // ---- workspace
   std::vector<CellWork> ws(nc);
@@ -793,7 +889,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
       w.active = cells[i].r_t > 0;
       w.tc = (fmask & 2) && w.active && mode == FM_RANDOMIZED && tc_sweep_ok(cells[i], L->mem_space == JOLT_MEM_HOST);
       w.tc_gram = (fmask & 4) && w.active && mode != FM_INJECTED && tc_sweep_ok(cells[i], L->mem_space == JOLT_MEM_HOST);
-      w.ufI = w.tc && cells[i].r_f == kD;
+      w.ufI = w.active && cells[i].r_f == kD;
       if (pass == 1) { w.lam = H->cells[i].lam; w.sigma = H->cells[i].n_sigma ? H->cells[i].sigma : nullptr; w.status = d_status + 4 * i; }
       carve(b, w, mode, true);
       if (pass == 1 && !w.n_sigma) w.n_sigma = H->cells[i].n_sigma;
@@ -813,9 +909,11 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     }
   }
 
+  lap("workspace");
   // ---- program
   Program P;
   build_factor_program(P, ws, mode, false, o->power_iters, o->seed, fast);
+  lap("factor program");
   std::vector<StoreJob> sj;
   for (int i = 0; i < nc; ++i) {
     const CellDesc &c = cells[i];
@@ -890,10 +988,13 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   }
   void *d_tab = nullptr;
   if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) { free_blob(); return rc; }
+  lap("residual program");
 
   // ---- run
   g_timer.begin(st);
   cudaError_t ce = cudaMemsetAsync(d_status, 0, sizeof(int) * 4 * nc, st);
+  for (int i = 0; i < nc && ce == cudaSuccess; ++i)
+    if (cells[i].r_t == 0 || cells[i].r_f == kD || injected) ce = cudaMemsetAsync(H->cells[i].lam, 0, sizeof(float) * kD, st);
   if (ce == cudaSuccess && L->mem_space == JOLT_MEM_HOST) {
     ce = cudaMemcpyAsync(stage_K, K, span, cudaMemcpyHostToDevice, st);
     if (ce == cudaSuccess) ce = cudaMemcpyAsync(stage_V, V, span, cudaMemcpyHostToDevice, st);
@@ -911,11 +1012,13 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   }
   if (ce != cudaSuccess) { free_blob(); return fail(JOLT_ECUDA, "staging copy: %s", cudaGetErrorString(ce)); }
   if ((rc = run_program(P, (char *)d_tab, st))) { free_blob(); return rc; }
+  lap("launches");
   std::vector<int> hstat(4 * nc);
   ce = cudaMemcpyAsync(hstat.data(), d_status, sizeof(int) * 4 * nc, cudaMemcpyDeviceToHost, st);
   if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
   if (ce != cudaSuccess) { cudaGetLastError(); free_blob(); return fail(JOLT_ECUDA, "compress: %s", cudaGetErrorString(ce)); }
   g_timer.finish();
+  lap("sync");
   if ((rc = status_to_code(hstat))) { free_blob(); return rc; }
   *out = H.release();
   return JOLT_OK;
@@ -1189,7 +1292,7 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
       ws[i].lam = nullptr; ws[i].sigma = nullptr;
       ws[i].tc = (fmask & 2) && mode == FM_RANDOMIZED && tc_sweep_ok(cells[i], L->mem_space == JOLT_MEM_HOST);
       ws[i].tc_gram = (fmask & 4) && tc_sweep_ok(cells[i], L->mem_space == JOLT_MEM_HOST);
-      ws[i].ufI = ws[i].tc;
+      ws[i].ufI = true;
       carve(b, ws[i], mode, false);
     }
     if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) return rc;

@@ -139,6 +139,167 @@ __global__ void __launch_bounds__(kEigThreads) jacobi_eig_kernel(const EigTask *
   }
 }
 
+// Shared-memory variant for n <= kEigSmemMaxN: the symmetric matrix lives as a packed lower triangle in
+// fp64, the eigenvector accumulator as fp32 rows.  One round = rotation parameters for n/2 disjoint pairs,
+// then ONE fused update: every 2x2 block A[{p_a,q_a}][{p_b,q_b}] (a <= b) becomes J_a^T blk J_b, and rows
+// p, q of V^T rotate.  Two barriers per round, no global traffic.
+constexpr int kEigSmemMaxN = 168;
+constexpr size_t kSmemOptIn = 232448;    // 227 KB of dynamic shared memory per CTA
+
+__host__ __device__ inline size_t eig_smem_bytes(int n, size_t vsize) {
+  const int np = (n + 1) / 2;
+  size_t b = (size_t)n * (n + 1) / 2 * sizeof(double);       // packed A
+  b += (size_t)np * 2 * sizeof(double);                       // c, s
+  b += 40 * sizeof(double);                                   // reduction scratch
+  b += (size_t)n * n * vsize;                                 // V^T
+  b += (size_t)np * 2 * sizeof(int) + (size_t)n * sizeof(int) + 64;
+  return b;
+}
+
+__device__ __forceinline__ int tri_idx(int i, int j) { return i >= j ? i * (i + 1) / 2 + j : j * (j + 1) / 2 + i; }
+
+template <typename VT>
+__global__ void __launch_bounds__(kEigThreads, 1) jacobi_eig_smem_kernel(const EigTask *__restrict__ tasks) {
+  const EigTask t = tasks[blockIdx.x];
+  const int n = t.n;
+  if (n <= 0) return;
+  extern __shared__ double shd[];
+  const int ne = (n + 1) & ~1, np = ne / 2;
+  const int ntri = n * (n + 1) / 2;
+  double *A = shd;
+  double *cs_c = A + ntri, *cs_s = cs_c + np, *red = cs_s + np;
+  VT *Vt = (VT *)(red + 40);
+  int *pp = (int *)(Vt + (size_t)n * n), *qq = pp + np, *rk = qq + np;
+  __shared__ double s_total, s_off;
+  const int tid = threadIdx.x, nt = blockDim.x;
+
+  double loc = 0;
+  for (int e = tid; e < n * n; e += nt) {
+    const int i = e / n, j = e - i * n;
+    const double v = t.A[e];
+    loc += v * v;
+    if (j <= i) A[i * (i + 1) / 2 + j] = (i == j) ? v : 0.5 * (v + t.A[(size_t)j * n + i]);
+    Vt[e] = (i == j) ? VT(1) : VT(0);
+  }
+  for (int o = 16; o; o >>= 1) loc += __shfl_xor_sync(0xffffffffu, loc, o);
+  if ((tid & 31) == 0) red[tid >> 5] = loc;
+  __syncthreads();
+  if (tid == 0) { double s = 0; for (int i = 0; i < nt / 32; ++i) s += red[i]; s_total = s; }
+  __syncthreads();
+  const double total = s_total;
+  bool converged = (total == 0.0);
+  // static work assignment (the same every round): up to 4 pair-blocks (a <= b) per thread, one column of
+  // V^T per thread with a fixed stride over the pairs
+  const int nblk = np * (np + 1) / 2;
+  int blk_ab[4];
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int w = tid + u * nt;
+    blk_ab[u] = -1;
+    if (w < nblk) {
+      int b = (int)((sqrtf(8.0f * w + 1.0f) - 1.0f) * 0.5f);
+      while ((b + 1) * (b + 2) / 2 <= w) ++b;
+      while (b * (b + 1) / 2 > w) --b;
+      blk_ab[u] = (b << 16) | (w - b * (b + 1) / 2);
+    }
+  }
+  const int vcols = nt / n;                 // thread groups over the pairs
+  const int vj = tid % n, vi0 = tid / n;    // this thread's column and first pair
+  for (int sweep = 0; sweep < kEigMaxSweeps && !converged; ++sweep) {
+    for (int r = 0; r < ne - 1; ++r) {
+      for (int i = tid; i < np; i += nt) {
+        int p, q; rr_pair(r, i, ne, p, q);
+        double c = 1.0, s = 0.0;
+        if (q < n) {
+          const double apq = A[q * (q + 1) / 2 + p];
+          const double app = A[p * (p + 1) / 2 + p], aqq = A[q * (q + 1) / 2 + q];
+          if (fabs(apq) > 1e-300 && fabs(apq) > 1e-17 * sqrt(fabs(app * aqq))) {
+            const double tau = (aqq - app) / (2.0 * apq);
+            const double tt = (tau >= 0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
+            c = rsqrt(1.0 + tt * tt);
+            s = tt * c;
+          }
+        } else { q = -1; }
+        pp[i] = p; qq[i] = q; cs_c[i] = c; cs_s[i] = s;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (blk_ab[u] < 0) continue;
+        const int b = blk_ab[u] >> 16, a = blk_ab[u] & 0xffff;
+        const int pa = pp[a], qa = qq[a], pb = pp[b], qb = qq[b];
+        const double ca = cs_c[a], sa = cs_s[a], cb = cs_c[b], sb = cs_s[b];
+        if (a == b) {
+          if (qa < 0 || sa == 0.0) continue;
+          const int ipp = pa * (pa + 1) / 2 + pa, iqq = qa * (qa + 1) / 2 + qa, ipq = qa * (qa + 1) / 2 + pa;
+          const double app = A[ipp], aqq = A[iqq], apq = A[ipq];
+          A[ipp] = ca * ca * app - 2.0 * ca * sa * apq + sa * sa * aqq;
+          A[iqq] = sa * sa * app + 2.0 * ca * sa * apq + ca * ca * aqq;
+          A[ipq] = 0.0;
+          continue;
+        }
+        if (sa == 0.0 && sb == 0.0) continue;
+        const int i_pp = tri_idx(pa, pb);
+        double x_pp = A[i_pp], x_pq = 0, x_qp = 0, x_qq = 0;
+        int i_pq = -1, i_qp = -1, i_qq = -1;
+        if (qb >= 0) { i_pq = tri_idx(pa, qb); x_pq = A[i_pq]; }
+        if (qa >= 0) { i_qp = tri_idx(qa, pb); x_qp = A[i_qp]; }
+        if (qa >= 0 && qb >= 0) { i_qq = tri_idx(qa, qb); x_qq = A[i_qq]; }
+        const double r_pp = ca * x_pp - sa * x_qp, r_pq = ca * x_pq - sa * x_qq;
+        const double r_qp = sa * x_pp + ca * x_qp, r_qq = sa * x_pq + ca * x_qq;
+        A[i_pp] = cb * r_pp - sb * r_pq;
+        if (i_pq >= 0) A[i_pq] = sb * r_pp + cb * r_pq;
+        if (i_qp >= 0) A[i_qp] = cb * r_qp - sb * r_qq;
+        if (i_qq >= 0) A[i_qq] = sb * r_qp + cb * r_qq;
+      }
+      if (vi0 < vcols) {
+        for (int i = vi0; i < np; i += vcols) {
+          const int q = qq[i];
+          const VT s = (VT)cs_s[i];
+          if (q < 0 || s == VT(0)) continue;
+          const int p = pp[i];
+          const VT c = (VT)cs_c[i];
+          const VT vp = Vt[p * n + vj], vq = Vt[q * n + vj];
+          Vt[p * n + vj] = c * vp - s * vq;
+          Vt[q * n + vj] = s * vp + c * vq;
+        }
+      }
+      __syncthreads();
+    }
+    double off = 0;
+    for (int e = tid; e < ntri; e += nt) {
+      int i = (int)((sqrtf(8.0f * e + 1.0f) - 1.0f) * 0.5f);
+      while ((i + 1) * (i + 2) / 2 <= e) ++i;
+      while (i * (i + 1) / 2 > e) --i;
+      if (e - i * (i + 1) / 2 != i) { const double v = A[e]; off += v * v; }   // skip the diagonal (no cancellation)
+    }
+    for (int o = 16; o; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
+    if ((tid & 31) == 0) red[tid >> 5] = off;
+    __syncthreads();
+    if (tid == 0) { double s = 0; for (int i = 0; i < nt / 32; ++i) s += red[i]; s_off = 2.0 * s; }
+    __syncthreads();
+    converged = (s_off <= 1e-24 * total);
+    __syncthreads();
+  }
+  if (!converged && tid == 0 && t.status) atomicOr(t.status, 1);
+  for (int i = tid; i < n; i += nt) t.w[i] = A[i * (i + 1) / 2 + i];
+  __syncthreads();
+  for (int i = tid; i < n; i += nt) {
+    const double wi = t.w[i];
+    int rank = 0;
+    for (int j = 0; j < n; ++j) { const double wj = t.w[j]; rank += (wj > wi) || (wj == wi && j < i); }
+    if (t.w_out) { const double v = wi > 0 ? wi : 0.0; t.w_out[rank] = (float)(t.w_sqrt ? sqrt(v) : v); }
+    rk[i] = rank;
+  }
+  __syncthreads();
+  if (t.U_out)
+    for (int it = tid; it < n * n; it += nt) {
+      const int j = it / n, i = it - j * n;
+      const int rank = rk[i];
+      if (rank < t.r_out) t.U_out[(size_t)j * t.ld_out + rank] = (float)Vt[i * n + j];
+    }
+}
+
 struct CholTask {
   double *G;        // n x n symmetric positive semi-definite (lower part used); overwritten by L
   double *Linv;     // n x n out: inverse of L (lower), rows of dead pivots zero
@@ -197,6 +358,115 @@ __global__ void __launch_bounds__(1024) cholesky_inv_kernel(const CholTask *__re
       t.LinvT32[it] = (float)t.Linv[(size_t)j * n + c];
     }
   if (tid == 0 && t.status) { int any = 0; for (int i = 0; i < n; ++i) any |= dead[i]; if (any) atomicOr(t.status, 2); }
+}
+
+
+// ---- CholeskyQR pieces resident in shared memory (n <= kCholSmemMaxN) -----------------------------------
+// cholesky_smem_kernel: G = L L^T in fp64 (dead pivots deflated as in cholesky_inv_kernel); writes
+// LT[l][j] = L[j][l] (fp32, pitch kp = n rounded up to 4, zero above the diagonal of L) and invd[j] = 1 / L[j][j]
+// (0 for a dead pivot).  trsm_rows_kernel then solves  dst_row * L^T = src_row  for 128 rows per CTA.
+constexpr int kCholSmemMaxN = 168;
+
+struct CholSmemTask { const double *G; float *LT; float *invd; int n; int *status; };
+
+__global__ void __launch_bounds__(1024, 1) cholesky_smem_kernel(const CholSmemTask *__restrict__ tasks) {
+  const CholSmemTask t = tasks[blockIdx.x];
+  const int n = t.n;
+  if (n <= 0) return;
+  extern __shared__ double shd[];
+  const int ld = n + 1;
+  double *A = shd;                       // n x (n+1)
+  double *diag0 = A + (size_t)n * ld;    // n
+  int *dead = (int *)(diag0 + n);        // n
+  __shared__ double s_piv;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  for (int e = tid; e < n * n; e += nt) { const int i = e / n, j = e - i * n; A[i * ld + j] = t.G[e]; }
+  __syncthreads();
+  for (int i = tid; i < n; i += nt) { diag0[i] = A[i * ld + i]; dead[i] = 0; }
+  __syncthreads();
+  for (int j = 0; j < n; ++j) {
+    if (tid == 0) {
+      const double a = A[j * ld + j];
+      if (!(a > 1e-10 * diag0[j]) || !(diag0[j] > 0)) { dead[j] = 1; s_piv = 0.0; A[j * ld + j] = 1.0; }
+      else { s_piv = sqrt(a); A[j * ld + j] = s_piv; }
+    }
+    __syncthreads();
+    const double piv = s_piv;
+    const double ipiv = piv > 0 ? 1.0 / piv : 0.0;
+    for (int i = j + 1 + tid; i < n; i += nt) A[i * ld + j] *= ipiv;
+    __syncthreads();
+    if (piv > 0) {
+      const int rem = n - j - 1;
+      for (int it = tid; it < rem * rem; it += nt) {
+        const int ii = it / rem, ll = it - ii * rem;
+        if (ll <= ii) { const int i = j + 1 + ii, l = j + 1 + ll; A[i * ld + l] -= A[i * ld + j] * A[l * ld + j]; }
+      }
+    }
+    __syncthreads();
+  }
+  const int kp = (n + 3) & ~3;
+  for (int e = tid; e < n * kp; e += nt) {
+    const int l = e / kp, j = e - l * kp;
+    t.LT[e] = (j < n && j >= l) ? (float)A[j * ld + l] : 0.f;
+  }
+  for (int j = tid; j < n; j += nt) t.invd[j] = dead[j] ? 0.f : (float)(1.0 / A[j * ld + j]);
+  if (tid == 0 && t.status) { int any = 0; for (int i = 0; i < n; ++i) any |= dead[i]; if (any) atomicOr(t.status, 2); }
+}
+
+inline size_t chol_smem_bytes(int n) { return ((size_t)n * (n + 1) + n) * sizeof(double) + (size_t)n * sizeof(int) + 64; }
+
+struct TrsmJob { const float *src; float *dst; int rows, k; const float *LT; const float *invd; };
+
+inline size_t trsm_smem_bytes(int k) { const int kp = (k + 3) & ~3; return ((size_t)k * kp + (size_t)kp * 129 + kp) * sizeof(float) + 64; }
+
+__global__ void __launch_bounds__(128) trsm_rows_kernel(const TrsmJob *__restrict__ jobs) {
+  const TrsmJob t = jobs[blockIdx.y];
+  const int r0 = blockIdx.x * 128;
+  if (r0 >= t.rows) return;
+  const int k = t.k, kp = (k + 3) & ~3;
+  extern __shared__ float shf[];
+  float *LT = shf;                       // k x kp
+  float *sp = LT + (size_t)k * kp;       // kp x 129  (feature j, row r)
+  float *invd = sp + (size_t)kp * 129;   // kp
+  const int tid = threadIdx.x;
+  const int nrows = min(128, t.rows - r0);
+  for (int e = tid; e < k * kp; e += 128) LT[e] = t.LT[e];
+  for (int j = tid; j < kp; j += 128) invd[j] = j < k ? t.invd[j] : 0.f;
+  const float *src = t.src + (size_t)r0 * k;
+  for (int e = tid; e < nrows * k; e += 128) { const int r = e / k, j = e - r * k; sp[j * 129 + r] = src[e]; }
+  for (int e = tid; e < (kp - k) * 129; e += 128) sp[k * 129 + e] = 0.f;
+  __syncthreads();
+  if (tid < nrows) {
+    const int r = tid;
+    for (int jb = 0; jb < kp; jb += 4) {
+      float a0 = sp[(jb + 0) * 129 + r], a1 = sp[(jb + 1) * 129 + r], a2 = sp[(jb + 2) * 129 + r], a3 = sp[(jb + 3) * 129 + r];
+      for (int l = 0; l < jb; ++l) {
+        const float x = sp[l * 129 + r];
+        const float4 L4 = *(const float4 *)&LT[l * kp + jb];
+        a0 = fmaf(-x, L4.x, a0); a1 = fmaf(-x, L4.y, a1); a2 = fmaf(-x, L4.z, a2); a3 = fmaf(-x, L4.w, a3);
+      }
+      a0 *= invd[jb];
+      a1 = fmaf(-a0, LT[(jb + 0) * kp + jb + 1], a1); a1 *= invd[jb + 1];
+      a2 = fmaf(-a0, LT[(jb + 0) * kp + jb + 2], a2); a2 = fmaf(-a1, LT[(jb + 1) * kp + jb + 2], a2); a2 *= invd[jb + 2];
+      a3 = fmaf(-a0, LT[(jb + 0) * kp + jb + 3], a3); a3 = fmaf(-a1, LT[(jb + 1) * kp + jb + 3], a3);
+      a3 = fmaf(-a2, LT[(jb + 2) * kp + jb + 3], a3); a3 *= invd[jb + 3];
+      sp[(jb + 0) * 129 + r] = a0; sp[(jb + 1) * 129 + r] = a1; sp[(jb + 2) * 129 + r] = a2; sp[(jb + 3) * 129 + r] = a3;
+    }
+  }
+  __syncthreads();
+  float *dst = t.dst + (size_t)r0 * k;
+  for (int e = tid; e < nrows * k; e += 128) { const int r = e / k, j = e - r * k; dst[e] = sp[j * 129 + r]; }
+}
+
+// sum of fp64 partials with a per-job element count
+struct ReduceJob { const double *parts; double *out; int count, n_elems; };
+__global__ void reduce_partials_var_kernel(const ReduceJob *__restrict__ jobs) {
+  const ReduceJob j = jobs[blockIdx.y];
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < j.n_elems; e += gridDim.x * blockDim.x) {
+    double s = 0;
+    for (int h = 0; h < j.count; ++h) s += j.parts[(size_t)h * j.n_elems + e];
+    j.out[e] = s;
+  }
 }
 
 }  // namespace jolt
