@@ -237,8 +237,10 @@ def main():
         dist.barrier()
     launches = B.launch_count() - n0
     clocks = sampler.stop() if rank == 0 else None
-    tc = sum(r[0] for r in rec) / len(rec)
-    td = sum(r[1] for r in rec) / len(rec)
+    tc_all = sorted(r[0] for r in rec)
+    td_all = sorted(r[1] for r in rec)
+    tc = sum(tc_all) / len(rec)
+    td = sum(td_all) / len(rec)
     # decompress stage timing (device events inside the library need a sync, done in step())
     if dist:
         t = torch.tensor([tc, td], device="cuda", dtype=torch.float64)
@@ -327,6 +329,8 @@ def main():
                        "cache_bytes": cache_bytes, "compressed_bytes": planned_bytes, "achieved_ratio": cache_bytes / planned_bytes,
                        "plan": plans, "l2": "inputs (537 MB) exceed L2; no flush"},
             "compress_ms": tc, "decompress_ms": td, "plan_ms": plan_ms,
+            "compress_ms_min_med_max": [tc_all[0], tc_all[len(tc_all) // 2], tc_all[-1]],
+            "decompress_ms_min_med_max": [td_all[0], td_all[len(td_all) // 2], td_all[-1]],
             "compress_gbs": world * cache_bytes / (tc * 1e-3) / 1e9, "decompress_gbs": world * cache_bytes / (td * 1e-3) / 1e9,
             "compress_roofline_frac": t_roof_c * 1e3 / tc, "decompress_roofline_frac": t_roof_d * 1e3 / td,
             "compress_roofline_ms": t_roof_c * 1e3, "decompress_roofline_ms": t_roof_d * 1e3,

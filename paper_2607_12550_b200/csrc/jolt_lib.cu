@@ -19,6 +19,7 @@
 #include "rowquant.cuh"
 #include "simt_gemm.cuh"
 #include "small_solvers.cuh"
+#include "block_jacobi.cuh"
 
 using namespace jolt;
 
@@ -281,11 +282,49 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks) {
   if (tasks.empty()) return;
   // problems that fit one CTA's shared memory take the resident kernel, the rest the global-memory one
   std::vector<EigTask> small64, small32, big;
+  std::vector<BJTask> bj;
   for (auto &t : tasks) {
+    if (t.bjA && t.n > 32 && g_eig_smem.load() != 2) {
+      BJTask b; memset(&b, 0, sizeof b);
+      b.A_in = t.A; b.A = t.bjA; b.V = t.bjV; b.J = t.bjJ; b.off = t.bjOff; b.done = t.bjDone;
+      b.n = t.n; b.nbe = (((t.n + kBJBlock - 1) / kBJBlock) + 1) & ~1; b.nP = b.nbe * kBJBlock;
+      b.w = t.w; b.U_out = t.U_out; b.ld_out = t.ld_out; b.r_out = t.r_out; b.w_out = t.w_out; b.w_sqrt = t.w_sqrt; b.status = t.status;
+      bj.push_back(b);
+      continue;
+    }
     if (!g_eig_smem.load() || t.n > kEigSmemMaxN) big.push_back(t);
     else if (eig_smem_bytes(t.n, 8) <= kSmemOptIn - 1024) small64.push_back(t);   // fp64 eigenvector accumulator fits
     else if (eig_smem_bytes(t.n, 4) <= kSmemOptIn - 1024) small32.push_back(t);
     else big.push_back(t);
+  }
+  if (!bj.empty()) {
+    int max_nbe = 0, max_nP = 0;
+    for (auto &b : bj) { max_nbe = std::max(max_nbe, b.nbe); max_nP = std::max(max_nP, b.nP); }
+    const size_t off = P.push(bj);
+    const int n = (int)bj.size();
+    std::vector<BJTask> copy = bj;
+    P.add(stage, [=](char *dev, cudaStream_t s) {
+      const BJTask *d = (const BJTask *)(dev + off);
+      for (auto &b : copy) { cudaMemsetAsync(b.off, 0, 3 * sizeof(double), s); cudaMemsetAsync(b.done, 0, sizeof(int), s); }
+      bj_init_kernel<<<dim3(64, n), 256, 0, s>>>(d); LAUNCHED();
+      const int np = max_nbe / 2;
+      const int gx = np * np + np * (max_nP / 32);
+      const int max_sweeps = max_nbe > 12 ? 2 * kBJMaxSweeps : kBJMaxSweeps;   // larger problems take a few more sweeps
+      for (int sw = 0; sw < max_sweeps; ++sw) {
+        for (int r = 0; r < max_nbe - 1; ++r) {
+          bj_solve_kernel<<<dim3(np, n), 256, 0, s>>>(d, r); LAUNCHED();
+          bj_apply_kernel<<<dim3(gx, n), 256, 0, s>>>(d, r); LAUNCHED();
+        }
+        bj_check_kernel<<<dim3(32, n), 256, 0, s>>>(d, 0); LAUNCHED();
+        bj_check_kernel<<<dim3(1, n), 32, 0, s>>>(d, 1); LAUNCHED();
+      }
+      bj_finish_kernel<<<n, 256, 0, s>>>(d); LAUNCHED();
+      if (getenv("JOLT_DEBUG_EIG")) {
+        cudaStreamSynchronize(s);
+        for (auto &b : copy) { double o[3]; int dn; cudaMemcpy(o, b.off, 24, cudaMemcpyDeviceToHost); cudaMemcpy(&dn, b.done, 4, cudaMemcpyDeviceToHost);
+          fprintf(stderr, "[jolt] bj n=%d nbe=%d last_off=%g total=%g done=%d\n", b.n, b.nbe, o[2], o[1], dn); }
+      }
+    });
   }
   static bool attr_done = false;
   if (!attr_done) {
@@ -345,6 +384,7 @@ struct CellWork {      // device scratch of one cell
   float *omega = nullptr, *PF = nullptr, *W = nullptr, *S = nullptr, *S2 = nullptr, *Zp = nullptr, *Z = nullptr, *Z2 = nullptr;
   double *Gs = nullptr, *Linv = nullptr; float *LinvT = nullptr;
   double *gpart = nullptr; float *LT32 = nullptr, *invd = nullptr;
+  double *bjA = nullptr, *bjV = nullptr, *bjJ = nullptr, *bjOff = nullptr; int *bjDone = nullptr;
   double *BBt = nullptr, *BBv = nullptr, *BBw = nullptr;
   float *Ut = nullptr, *sigma = nullptr;
   float *UT32 = nullptr, *G32 = nullptr;
@@ -378,6 +418,12 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
     w.G32 = b.take<float>((size_t)c.m * c.r_t * c.r_f);
     w.Zp = b.take<float>((size_t)c.m * kD * std::max<size_t>(k, c.r_t));
     if (mode != FM_INJECTED) {
+      {
+        const size_t nmax = std::max<size_t>(kD, mode == FM_EXACT ? T : k);
+        const size_t nbe = (((nmax + kBJBlock - 1) / kBJBlock) + 1) & ~(size_t)1, nP = nbe * kBJBlock;
+        w.bjA = b.take<double>(nP * nP); w.bjV = b.take<double>(nP * nP); w.bjJ = b.take<double>(nbe / 2 * 1024);
+        w.bjOff = b.take<double>(4); w.bjDone = b.take<int>(1);
+      }
       w.gram_part = b.take<double>((size_t)c.m * kD * kD);
       w.C = b.take<double>(kD * kD); w.Cv = b.take<double>(kD * kD); w.Cw = b.take<double>(kD);
     }
@@ -445,7 +491,7 @@ void add_tall_gram(Program &P, int stage, const std::vector<TallGram> &jobs) {
 
 // orth(S) for every active cell by CholeskyQR2: twice {Gs = S^T S (fp64), Gs = L L^T, S <- S L^-T}.
 // token_side selects S (T rows) or Z (N rows); the result is left in the source buffer.
-void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side) {
+void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side, int passes) {
   for (int pass = 0; pass < 2; ++pass) {
     std::vector<TallGram> tg;
     std::vector<GemmTask> g2;
@@ -458,12 +504,16 @@ void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side)
       const int k = w.c.k, rows = token_side ? w.c.T : w.c.N;
       float *src = token_side ? (pass == 0 ? w.S : w.S2) : (pass == 0 ? w.Z : w.Z2);
       float *dst = token_side ? (pass == 0 ? w.S2 : w.S) : (pass == 0 ? w.Z2 : w.Z);
-      tg.push_back({src, rows, k, w.gpart, w.Gs});
       if (k <= kCholSmemMaxN) {
+        // resident path: the triangular solve works in place, so one pass is possible
+        if (pass >= passes) continue;
+        float *buf = token_side ? w.S : w.Z;
+        tg.push_back({buf, rows, k, w.gpart, w.Gs});
         chs.push_back({w.Gs, w.LT32, w.invd, k, w.status});
-        tj.push_back({src, dst, rows, k, w.LT32, w.invd});
+        tj.push_back({buf, buf, rows, k, w.LT32, w.invd});
         max_k = std::max(max_k, k);
       } else {
+        tg.push_back({src, rows, k, w.gpart, w.Gs});
         CholTask c; c.G = w.Gs; c.Linv = w.Linv; c.LinvT32 = w.LinvT; c.n = k; c.status = w.status;
         ch.push_back(c);
         g2.push_back(mk(src, DT_F32, k, 1, w.LinvT, DT_F32, k, 1, dst, DT_F32, k, rows, k, k));
@@ -594,6 +644,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
         parts.push_back(w.gram_part); outs.push_back(w.C); counts.push_back(c.m);
       }
       EigTask e; memset(&e, 0, sizeof e);
+      e.bjA = w.bjA; e.bjV = w.bjV; e.bjJ = w.bjJ; e.bjOff = w.bjOff; e.bjDone = w.bjDone;
       e.A = w.C; e.Vt = w.Cv; e.w = w.Cw; e.n = kD; e.status = w.status; e.w_out = w.lam; e.w_sqrt = 0;
       if (!probe) { e.U_out = w.UF32; e.ld_out = c.r_f; e.r_out = c.r_f; }
       eg.push_back(e);
@@ -618,13 +669,15 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
     }
   }
   if (mode == FM_RANDOMIZED) {
+    // only the range of the intermediate bases matters (one Cholesky-QR pass keeps them well conditioned);
+    // the final basis is orthonormalised twice
     add_sketch(P, ST_SKETCH, ws, true);
-    add_orth(P, ST_ORTH, ws, true);
+    add_orth(P, ST_ORTH, ws, true, power_iters == 0 ? 2 : 1);
     for (int it = 0; it < power_iters; ++it) {
       add_project(P, ST_POWER, ws);
-      add_orth(P, ST_POWER, ws, false);
+      add_orth(P, ST_POWER, ws, false, 1);
       add_sketch(P, ST_POWER, ws, false);
-      add_orth(P, ST_POWER, ws, true);
+      add_orth(P, ST_POWER, ws, true, it + 1 == power_iters ? 2 : 1);
     }
     add_project(P, ST_PROJ, ws);          // Z now holds B^T (N x k)
     std::vector<TallGram> tgb; std::vector<EigTask> eg; std::vector<GemmTask> g2, g3;
@@ -633,6 +686,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
       const CellDesc &c = w.c;
       tgb.push_back({w.Z, c.N, c.k, w.gpart, w.BBt});
       EigTask e; memset(&e, 0, sizeof e);
+      e.bjA = w.bjA; e.bjV = w.bjV; e.bjJ = w.bjJ; e.bjOff = w.bjOff; e.bjDone = w.bjDone;
       e.A = w.BBt; e.Vt = w.BBv; e.w = w.BBw; e.n = c.k; e.status = w.status; e.w_out = w.sigma; e.w_sqrt = 1;
       if (!probe) { e.U_out = w.Ut; e.ld_out = c.r_t; e.r_out = c.r_t; }
       eg.push_back(e);
@@ -665,6 +719,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
       t.nseg = c.m; t.seg_inner = c.m; t.a_si = (long long)c.T * c.r_f; t.b_si = (long long)c.T * c.r_f;
       g2.push_back(t);
       EigTask e; memset(&e, 0, sizeof e);
+      e.bjA = w.bjA; e.bjV = w.bjV; e.bjJ = w.bjJ; e.bjOff = w.bjOff; e.bjDone = w.bjDone;
       e.A = w.Gt; e.Vt = w.Gtv; e.w = w.Gtw; e.n = c.T; e.status = w.status; e.w_out = w.sigma; e.w_sqrt = 1;
       if (!probe) { e.U_out = w.UT32; e.ld_out = c.r_t; e.r_out = c.r_t; }
       eg.push_back(e);

@@ -17,10 +17,26 @@ struct EigTask {
   int w_sqrt;       // 1: write sqrt(max(w,0)) instead (singular values)
   int n;
   int *status;      // set to 1 if not converged
+  // optional scratch of the multi-launch block solver (null: single-CTA kernels)
+  double *bjA, *bjV, *bjJ, *bjOff; int *bjDone;
 };
 
 constexpr int kEigThreads = 1024;
 constexpr int kEigMaxSweeps = 40;
+
+// Jacobi rotation that annihilates apq, without divisions: with d = (aqq - app)/2 and h = hypot(d, apq),
+// cos 2t = |d|/h, so c = sqrt((1 + |d|/h)/2) and s = sgn(d) apq / (2 h c); two reciprocal square roots.
+__device__ __forceinline__ void jacobi_cs(double app, double aqq, double apq, double &c, double &s) {
+  c = 1.0; s = 0.0;
+  const double d = 0.5 * (aqq - app);
+  const double u = d * d + apq * apq;
+  if (!(fabs(apq) > 1e-17 * sqrt(fabs(app * aqq))) || !(u > 1e-280)) return;
+  const double rh = rsqrt(u);
+  const double x = 0.5 + 0.5 * fabs(d) * rh;
+  const double rc = rsqrt(x);
+  c = x * rc;
+  s = (d >= 0 ? 0.5 : -0.5) * apq * rh * rc;
+}
 
 __device__ __forceinline__ void rr_pair(int r, int i, int ne, int &p, int &q) {
   // circle method on ne (even) players: round r in [0, ne-1), slot i in [0, ne/2)
@@ -213,12 +229,7 @@ __global__ void __launch_bounds__(kEigThreads, 1) jacobi_eig_smem_kernel(const E
         if (q < n) {
           const double apq = A[q * (q + 1) / 2 + p];
           const double app = A[p * (p + 1) / 2 + p], aqq = A[q * (q + 1) / 2 + q];
-          if (fabs(apq) > 1e-300 && fabs(apq) > 1e-17 * sqrt(fabs(app * aqq))) {
-            const double tau = (aqq - app) / (2.0 * apq);
-            const double tt = (tau >= 0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
-            c = rsqrt(1.0 + tt * tt);
-            s = tt * c;
-          }
+          jacobi_cs(app, aqq, apq, c, s);
         } else { q = -1; }
         pp[i] = p; qq[i] = q; cs_c[i] = c; cs_s[i] = s;
       }
@@ -396,10 +407,11 @@ __global__ void __launch_bounds__(1024, 1) cholesky_smem_kernel(const CholSmemTa
     for (int i = j + 1 + tid; i < n; i += nt) A[i * ld + j] *= ipiv;
     __syncthreads();
     if (piv > 0) {
-      const int rem = n - j - 1;
-      for (int it = tid; it < rem * rem; it += nt) {
-        const int ii = it / rem, ll = it - ii * rem;
-        if (ll <= ii) { const int i = j + 1 + ii, l = j + 1 + ll; A[i * ld + l] -= A[i * ld + j] * A[l * ld + j]; }
+      // trailing update, lower triangle, 32 x 32 thread tiles (no integer division)
+      const int tx = tid & 31, ty = tid >> 5;
+      for (int i = j + 1 + ty; i < n; i += 32) {
+        const double lij = A[i * ld + j];
+        for (int l = j + 1 + tx; l <= i; l += 32) A[i * ld + l] -= lij * A[l * ld + j];
       }
     }
     __syncthreads();
