@@ -20,7 +20,7 @@ struct BJTask {
   double *A;            // nP x nP work matrix
   double *V;            // nP x nP, column i = eigenvector i on exit
   double *J;            // (nbe/2) x 32 x 32 rotations of the current round
-  double *off;          // [3]: off-diagonal mass (accumulator), total mass, last measured off-diagonal mass
+  double *off;          // [4]: off-diagonal mass (accumulator), total mass, last measured off-diagonal mass, sweeps run
   int *done;            // [1]
   int n, nP, nbe;       // size, padded size (16 * nbe), even number of blocks
   double *w;            // nP scratch (eigenvalues)
@@ -45,7 +45,7 @@ __global__ void bj_init_kernel(const BJTask *__restrict__ tasks) {
 }
 
 // One cyclic sweep of 2x2 rotations on the 32 x 32 principal submatrix of block pair `blockIdx.x`.
-__global__ void __launch_bounds__(256) bj_solve_kernel(const BJTask *__restrict__ tasks, int round) {
+__global__ void __launch_bounds__(256) bj_solve_kernel(const BJTask *__restrict__ tasks, int round, int cross_only) {
   const BJTask t = tasks[blockIdx.y];
   if (*t.done || (int)blockIdx.x >= t.nbe / 2) return;
   int I, Jb;
@@ -61,12 +61,16 @@ __global__ void __launch_bounds__(256) bj_solve_kernel(const BJTask *__restrict_
     Jm[i][j] = (i == j) ? 1.0 : 0.0;
   }
   __syncthreads();
-  for (int r = 0; r < 31; ++r) {
+  // The first round of a sweep rotates every pair of the 32 indices (31 inner rounds), which also covers
+  // the pairs inside each 16-block once per sweep; the other rounds rotate the 16 x 16 cross pairs only.
+  const int n_inner = cross_only ? 16 : 31;
+  for (int r = 0; r < n_inner; ++r) {
     if (tid < 16) {
-      int p, q; rr_pair(r, tid, 32, p, q);
+      int p, q;
+      if (cross_only) { p = tid; q = 16 + ((tid + r) & 15); } else rr_pair(r, tid, 32, p, q);
       double c = 1.0, s = 0.0;
       const double apq = S[p][q], app = S[p][p], aqq = S[q][q];
-      jacobi_cs(app, aqq, apq, c, s);
+      jacobi_cs_fast(app, aqq, apq, c, s);
       pp[tid] = p; qq[tid] = q; cs_c[tid] = c; cs_s[tid] = s;
     }
     __syncthreads();
@@ -101,14 +105,20 @@ __global__ void __launch_bounds__(256) bj_apply_kernel(const BJTask *__restrict_
   const BJTask t = tasks[blockIdx.y];
   if (*t.done) return;
   const int np = t.nbe / 2, nP = t.nP;
-  const int n_ablk = np * np, n_vblk = np * (nP / 32);
+  const int n_ablk = np * (np + 1) / 2, n_vblk = np * (nP / 32);       // A is symmetric: blocks a <= b only
   if ((int)blockIdx.x >= n_ablk + n_vblk) return;
   __shared__ double Ja[32][33], Jb[32][33], X[32][33], Y[32][33];
   __shared__ int ra[32], rb[32];
   const int tid = threadIdx.x;
   const bool is_a = (int)blockIdx.x < n_ablk;
   int a, b;
-  if (is_a) { a = blockIdx.x / np; b = blockIdx.x - a * np; }
+  if (is_a) {
+    const int w = blockIdx.x;
+    b = (int)((sqrtf(8.0f * w + 1.0f) - 1.0f) * 0.5f);
+    while ((b + 1) * (b + 2) / 2 <= w) ++b;
+    while (b * (b + 1) / 2 > w) --b;
+    a = w - b * (b + 1) / 2;
+  }
   else { const int v = blockIdx.x - n_ablk; a = v / (nP / 32); b = v - a * (nP / 32); }
   if (tid < 32) {
     int I, J2; rr_pair(round, a, t.nbe, I, J2);
@@ -145,7 +155,10 @@ __global__ void __launch_bounds__(256) bj_apply_kernel(const BJTask *__restrict_
       for (int u = 0; u < 4; ++u) o[u] += Y[i0 + u][k] * x;
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) t.A[(size_t)ra[i0 + u] * nP + rb[j]] = o[u];
+    for (int u = 0; u < 4; ++u) {
+      t.A[(size_t)ra[i0 + u] * nP + rb[j]] = o[u];
+      if (a != b) t.A[(size_t)rb[j] * nP + ra[i0 + u]] = o[u];      // mirrored block
+    }
   } else {
     double o[4] = {0, 0, 0, 0};
     for (int k = 0; k < 32; ++k) {
@@ -170,10 +183,11 @@ __global__ void bj_check_kernel(const BJTask *__restrict__ tasks, int phase) {
     for (int o = 16; o; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
     if ((threadIdx.x & 31) == 0 && off != 0.0) atomicAdd(&t.off[0], off);
   } else if (blockIdx.x == 0 && threadIdx.x == 0) {
-    // relative off-diagonal norm 3e-11: above the round-off floor of the 32-term block products (~1e-13 per
-    // entry), far below the fp32 grade of what is read out
-    if (t.off[0] <= 1e-21 * t.off[1]) *t.done = 1;
+    // relative off-diagonal norm 3e-10: above the round-off floor of the 32-term block products on a
+    // rank-deficient matrix (measured 5e-11), far below the fp32 grade of what is read out
+    if (t.off[0] <= 1e-19 * t.off[1]) *t.done = 1;
     t.off[2] = t.off[0];
+    t.off[3] += 1.0;      // sweeps run
     t.off[0] = 0.0;
   }
 }

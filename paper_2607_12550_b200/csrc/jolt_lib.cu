@@ -305,14 +305,14 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks) {
     std::vector<BJTask> copy = bj;
     P.add(stage, [=](char *dev, cudaStream_t s) {
       const BJTask *d = (const BJTask *)(dev + off);
-      for (auto &b : copy) { cudaMemsetAsync(b.off, 0, 3 * sizeof(double), s); cudaMemsetAsync(b.done, 0, sizeof(int), s); }
+      for (auto &b : copy) { cudaMemsetAsync(b.off, 0, 4 * sizeof(double), s); cudaMemsetAsync(b.done, 0, sizeof(int), s); }
       bj_init_kernel<<<dim3(64, n), 256, 0, s>>>(d); LAUNCHED();
       const int np = max_nbe / 2;
-      const int gx = np * np + np * (max_nP / 32);
+      const int gx = np * (np + 1) / 2 + np * (max_nP / 32);
       const int max_sweeps = max_nbe > 12 ? 2 * kBJMaxSweeps : kBJMaxSweeps;   // larger problems take a few more sweeps
       for (int sw = 0; sw < max_sweeps; ++sw) {
         for (int r = 0; r < max_nbe - 1; ++r) {
-          bj_solve_kernel<<<dim3(np, n), 256, 0, s>>>(d, r); LAUNCHED();
+          bj_solve_kernel<<<dim3(np, n), 256, 0, s>>>(d, r, r > 0 ? 1 : 0); LAUNCHED();
           bj_apply_kernel<<<dim3(gx, n), 256, 0, s>>>(d, r); LAUNCHED();
         }
         bj_check_kernel<<<dim3(32, n), 256, 0, s>>>(d, 0); LAUNCHED();
@@ -321,8 +321,8 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks) {
       bj_finish_kernel<<<n, 256, 0, s>>>(d); LAUNCHED();
       if (getenv("JOLT_DEBUG_EIG")) {
         cudaStreamSynchronize(s);
-        for (auto &b : copy) { double o[3]; int dn; cudaMemcpy(o, b.off, 24, cudaMemcpyDeviceToHost); cudaMemcpy(&dn, b.done, 4, cudaMemcpyDeviceToHost);
-          fprintf(stderr, "[jolt] bj n=%d nbe=%d last_off=%g total=%g done=%d\n", b.n, b.nbe, o[2], o[1], dn); }
+        for (auto &b : copy) { double o[4]; int dn; cudaMemcpy(o, b.off, 32, cudaMemcpyDeviceToHost); cudaMemcpy(&dn, b.done, 4, cudaMemcpyDeviceToHost);
+          fprintf(stderr, "[jolt] bj n=%d nbe=%d last_off=%g total=%g done=%d sweeps=%g\n", b.n, b.nbe, o[2], o[1], dn, o[3]); }
       }
     });
   }
@@ -468,16 +468,37 @@ struct TallGram { const float *M; int rows, k; double *part, *out; };
 void add_tall_gram(Program &P, int stage, const std::vector<TallGram> &jobs) {
   std::vector<GemmTask> g;
   std::vector<ReduceJob> rj;
+  std::vector<TallGramJob> fastj[3];        // register-tiled kernel for k <= 48 / 96 / 144
+  int fast_chunks[3] = {0, 0, 0};
   for (auto &j : jobs) {
-    int chunk = std::max(256, (j.rows + kGramChunks - 1) / kGramChunks);
+    int chunk = std::max(128, (j.rows + kGramChunks - 1) / kGramChunks);
     chunk = (chunk + 15) & ~15;
-    int n = 0;
-    for (int r0 = 0; r0 < j.rows; r0 += chunk, ++n) {
-      const float *m0 = j.M + (size_t)r0 * j.k;
-      g.push_back(mk(m0, DT_F32, 1, j.k, m0, DT_F32, j.k, 1, j.part + (size_t)n * j.k * j.k, DT_F64, j.k, j.k, j.k,
-                     std::min(chunk, j.rows - r0)));
+    const int n = (j.rows + chunk - 1) / chunk;
+    if (j.k <= 144) {
+      const int cls = j.k <= 48 ? 0 : (j.k <= 96 ? 1 : 2);
+      fastj[cls].push_back({j.M, j.rows, j.k, chunk, j.part});
+      fast_chunks[cls] = std::max(fast_chunks[cls], n);
+    } else {
+      int c = 0;
+      for (int r0 = 0; r0 < j.rows; r0 += chunk, ++c) {
+        const float *m0 = j.M + (size_t)r0 * j.k;
+        g.push_back(mk(m0, DT_F32, 1, j.k, m0, DT_F32, j.k, 1, j.part + (size_t)c * j.k * j.k, DT_F64, j.k, j.k, j.k,
+                       std::min(chunk, j.rows - r0)));
+      }
     }
     rj.push_back({j.part, j.out, n, j.k * j.k});
+  }
+  for (int cls = 0; cls < 3; ++cls) {
+    if (fastj[cls].empty()) continue;
+    const size_t off = P.push(fastj[cls]);
+    const int n = (int)fastj[cls].size(), nch = fast_chunks[cls];
+    P.add(stage, [=](char *dev, cudaStream_t s) {
+      const TallGramJob *d = (const TallGramJob *)(dev + off);
+      if (cls == 0) tall_gram_kernel<3><<<dim3(nch, n), 256, 0, s>>>(d);
+      else if (cls == 1) tall_gram_kernel<6><<<dim3(nch, n), 256, 0, s>>>(d);
+      else tall_gram_kernel<9><<<dim3(nch, n), 256, 0, s>>>(d);
+      LAUNCHED();
+    });
   }
   add_gemm(P, stage, g, true);
   if (rj.empty()) return;

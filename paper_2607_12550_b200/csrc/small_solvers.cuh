@@ -38,6 +38,28 @@ __device__ __forceinline__ void jacobi_cs(double app, double aqq, double apq, do
   s = (d >= 0 ? 0.5 : -0.5) * apq * rh * rc;
 }
 
+// Same rotation with the angle evaluated in fp32 (hardware rsqrt) and the pair (c, s) then renormalised
+// in fp64: the rotation is orthogonal to 1e-15, its angle is good to ~1e-7, which leaves a residual
+// apq' ~ 1e-7 apq for the next sweep instead of an exact zero.
+__device__ __forceinline__ void jacobi_cs_fast(double app, double aqq, double apq, double &c, double &s) {
+  c = 1.0; s = 0.0;
+  const double d = 0.5 * (aqq - app);
+  if (!(apq * apq > 1e-34 * fabs(app * aqq))) return;
+  const double mx = fmax(fabs(d), fabs(apq));
+  if (!(mx > 1e-290) || !(mx < 1e290)) return;
+  // scale by a power of two near 1/mx (exponent arithmetic only)
+  const int ex = ((__double2hiint(mx) >> 20) & 0x7ff) - 1023;
+  const double sc = __hiloint2double((1023 - ex) << 20, 0);
+  const float df = (float)(d * sc), af = (float)(apq * sc);
+  const float rh = rsqrtf(df * df + af * af);
+  const float x = 0.5f + 0.5f * fabsf(df) * rh;
+  const float rc = rsqrtf(x);
+  double cc = (double)(x * rc), ss = (double)((df >= 0.f ? 0.5f : -0.5f) * af * rh * rc);
+  const double e = fma(cc, cc, fma(ss, ss, -1.0));
+  const double corr = fma(e, fma(e, 0.375, -0.5), 1.0);
+  c = cc * corr; s = ss * corr;
+}
+
 __device__ __forceinline__ void rr_pair(int r, int i, int ne, int &p, int &q) {
   // circle method on ne (even) players: round r in [0, ne-1), slot i in [0, ne/2)
   const int md = ne - 1;
@@ -478,6 +500,58 @@ __global__ void reduce_partials_var_kernel(const ReduceJob *__restrict__ jobs) {
     double s = 0;
     for (int h = 0; h < j.count; ++h) s += j.parts[(size_t)h * j.n_elems + e];
     j.out[e] = s;
+  }
+}
+
+
+// ---- G = M^T M for a tall fp32 matrix, fp64 accumulation, one partial per row chunk ---------------------
+// Each of the 16 x 16 threads owns a TI x TI register tile of the k x k result (k <= 16 TI), rows stream
+// through shared memory 16 at a time (converted to fp64 once, on the way in).
+struct TallGramJob { const float *M; int rows, k, chunk; double *part; };
+
+template <int TI>
+__global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__restrict__ jobs) {
+  const TallGramJob t = jobs[blockIdx.y];
+  const int r_begin = blockIdx.x * t.chunk;
+  if (r_begin >= t.rows) return;
+  const int r_end = min(t.rows, r_begin + t.chunk);
+  constexpr int W = 16 * TI;
+  __shared__ double Ms[16][W + 2];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  double acc[TI][TI];
+#pragma unroll
+  for (int i = 0; i < TI; ++i)
+#pragma unroll
+    for (int j = 0; j < TI; ++j) acc[i][j] = 0.0;
+  for (int r0 = r_begin; r0 < r_end; r0 += 16) {
+    const int nr = min(16, r_end - r0);
+    for (int e = tid; e < 16 * W; e += 256) {
+      const int r = e / W, c = e - r * W;
+      Ms[r][c] = (r < nr && c < t.k) ? (double)t.M[(size_t)(r0 + r) * t.k + c] : 0.0;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int r = 0; r < 16; ++r) {
+      double a[TI], b[TI];
+#pragma unroll
+      for (int i = 0; i < TI; ++i) { a[i] = Ms[r][ty + 16 * i]; b[i] = Ms[r][tx + 16 * i]; }
+#pragma unroll
+      for (int i = 0; i < TI; ++i)
+#pragma unroll
+        for (int j = 0; j < TI; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  double *out = t.part + (size_t)blockIdx.x * t.k * t.k;
+#pragma unroll
+  for (int i = 0; i < TI; ++i) {
+    const int row = ty + 16 * i;
+    if (row >= t.k) continue;
+#pragma unroll
+    for (int j = 0; j < TI; ++j) {
+      const int col = tx + 16 * j;
+      if (col < t.k) out[(size_t)row * t.k + col] = acc[i][j];
+    }
   }
 }
 
