@@ -139,7 +139,9 @@ int jolt_compressed_bytes(const jolt_handle *h, int64_t *bytes);
  * which: 0 = core (fp16 bits, [m][r_t][r_f]), 1 = U_T (fp16, [T][r_t]), 2 = U_F (fp16, [128][r_f]),
  * 3 = packed codes (uint32, [m][T][4*bits]), 4 = scales (fp16, [m][T][4]), 5 = core exponent (int32),
  * 6 = token-mode singular values (fp32, k entries, 0 entries if injected), 7 = mode-3 eigenvalues
- * (fp32, 128).  dst_bytes is the capacity of dst; *written gets the size of the component. */
+ * (fp32, 128; zeros when r_f = 128), 8 = the token factor before fp16 rounding (fp32, [T][r_t]; a view of
+ * scratch memory, valid only until the next library call on the device; for tests).
+ * dst_bytes is the capacity of dst; *written gets the size of the component. */
 int jolt_get_component(const jolt_handle *h, int32_t cell, int32_t which, void *dst, int64_t dst_bytes,
                        int64_t *written);
 

@@ -178,6 +178,7 @@ struct CellStore {
   float *sigma = nullptr;  // k (or T for the exact path)
   float *lam = nullptr;    // 128
   int n_sigma = 0;
+  const float *dbg_UT32 = nullptr;   // fp32 token factor in the workspace (valid until the next library call)
   bool tc_ok = false;      // tensor maps below are valid
   alignas(64) CUtensorMap tmUT, tmUF, tmG;
 };
@@ -790,17 +791,55 @@ void add_backbone(Program &P, int stage, const std::vector<BackboneRef> &refs) {
   add_gemm(P, stage, g2, false);
 }
 
-int run_program(Program &P, char *d_tables, cudaStream_t st) {
+int run_program(Program &P, char *d_tables, cudaStream_t st, bool timed = true) {
   if (!P.host.empty()) CU(cudaMemcpyAsync(d_tables, P.host.data(), P.host.size(), cudaMemcpyHostToDevice, st));
   int cur = -1;
   for (auto &s : P.steps) {
-    if (cur != -1 && s.stage != cur) g_timer.mark(cur, st);
+    if (timed && cur != -1 && s.stage != cur) g_timer.mark(cur, st);
     cur = s.stage;
     s.run(d_tables, st);
   }
-  if (cur != -1) g_timer.mark(cur, st);
+  if (timed && cur != -1) g_timer.mark(cur, st);
   CU(cudaGetLastError());
   return JOLT_OK;
+}
+
+// Side streams on which independent groups of cells run their (latency-bound) factor stages concurrently.
+constexpr int kMaxGroups = 4;
+struct GroupStreams { bool have = false; cudaStream_t s[kMaxGroups]; cudaEvent_t fork, join[kMaxGroups]; };
+GroupStreams g_groups[64];
+GroupStreams *group_streams(int dev) {
+  std::lock_guard<std::mutex> lk(g_ws_mu);
+  GroupStreams &g = g_groups[dev];
+  if (!g.have) {
+    for (int i = 0; i < kMaxGroups; ++i) {
+      if (cudaStreamCreateWithFlags(&g.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+      if (cudaEventCreateWithFlags(&g.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    }
+    if (cudaEventCreateWithFlags(&g.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    g.have = true;
+  }
+  return &g;
+}
+
+// Cells whose factor stages may run side by side: cells that need the feature eigen-solve (longest chain)
+// form group 0, the others are dealt round-robin.
+int assign_groups(const std::vector<CellWork> &ws, std::vector<int> &group) {
+  int want = kMaxGroups;
+  if (const char *e = getenv("JOLT_GROUPS")) want = std::max(1, std::min(kMaxGroups, atoi(e)));
+  group.assign(ws.size(), -1);
+  int n_active = 0, n_long = 0;
+  for (auto &w : ws) if (w.active) { ++n_active; if (!w.ufI) ++n_long; }
+  if (n_active < 2 || want == 1) { for (size_t i = 0; i < ws.size(); ++i) if (ws[i].active) group[i] = 0; return n_active ? 1 : 0; }
+  const int first = (n_long > 0 && n_long < n_active) ? 1 : 0;
+  int rr = 0, used = 0;
+  for (size_t i = 0; i < ws.size(); ++i) {
+    if (!ws[i].active) continue;
+    if (first == 1 && !ws[i].ufI) group[i] = 0;
+    else { group[i] = first + rr % (want - first); ++rr; }
+    used = std::max(used, group[i] + 1);
+  }
+  return used;
 }
 
 }  // namespace
@@ -988,7 +1027,14 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   lap("workspace");
   // ---- program
   Program P;
-  build_factor_program(P, ws, mode, false, o->power_iters, o->seed, fast);
+  std::vector<int> cell_group;
+  const int n_groups = assign_groups(ws, cell_group);
+  std::vector<Program> PG(std::max(n_groups, 1));
+  for (int g = 0; g < n_groups; ++g) {
+    std::vector<CellWork> sub = ws;
+    for (int i = 0; i < nc; ++i) if (cell_group[i] != g) sub[i].active = false;
+    build_factor_program(PG[g], sub, mode, false, o->power_iters, o->seed, fast);
+  }
   lap("factor program");
   std::vector<StoreJob> sj;
   for (int i = 0; i < nc; ++i) {
@@ -1063,7 +1109,9 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     });
   }
   void *d_tab = nullptr;
-  if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) { free_blob(); return rc; }
+  std::vector<size_t> tab_off(PG.size() + 1, 0);
+  for (size_t g = 0; g < PG.size(); ++g) tab_off[g + 1] = tab_off[g] + ((PG[g].host.size() + 255) & ~(size_t)255);
+  if ((rc = tab_reserve(dev, tab_off.back() + P.host.size() + 256, &d_tab))) { free_blob(); return rc; }
   lap("residual program");
 
   // ---- run
@@ -1087,7 +1135,23 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     }
   }
   if (ce != cudaSuccess) { free_blob(); return fail(JOLT_ECUDA, "staging copy: %s", cudaGetErrorString(ce)); }
-  if ((rc = run_program(P, (char *)d_tab, st))) { free_blob(); return rc; }
+  if (n_groups <= 1) {
+    if (n_groups == 1 && (rc = run_program(PG[0], (char *)d_tab, st))) { free_blob(); return rc; }
+  } else {
+    GroupStreams *gs = group_streams(dev);
+    if (!gs) { free_blob(); return fail(JOLT_ECUDA, "cannot create side streams"); }
+    ce = cudaEventRecord(gs->fork, st);
+    for (int g = 0; g < n_groups && ce == cudaSuccess; ++g) {
+      ce = cudaStreamWaitEvent(gs->s[g], gs->fork, 0);
+      if (ce != cudaSuccess) break;
+      if ((rc = run_program(PG[g], (char *)d_tab + tab_off[g], gs->s[g], false))) { cudaDeviceSynchronize(); free_blob(); return rc; }
+      ce = cudaEventRecord(gs->join[g], gs->s[g]);
+      if (ce == cudaSuccess) ce = cudaStreamWaitEvent(st, gs->join[g], 0);
+    }
+    if (ce != cudaSuccess) { cudaDeviceSynchronize(); free_blob(); return fail(JOLT_ECUDA, "side streams: %s", cudaGetErrorString(ce)); }
+    g_timer.mark(ST_FACT, st);
+  }
+  if ((rc = run_program(P, (char *)d_tab + tab_off.back(), st))) { free_blob(); return rc; }
   lap("launches");
   std::vector<int> hstat(4 * nc);
   ce = cudaMemcpyAsync(hstat.data(), d_status, sizeof(int) * 4 * nc, cudaMemcpyDeviceToHost, st);
@@ -1096,6 +1160,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   g_timer.finish();
   lap("sync");
   if ((rc = status_to_code(hstat))) { free_blob(); return rc; }
+  for (int i = 0; i < nc; ++i) H->cells[i].dbg_UT32 = cells[i].r_t > 0 ? ws[i].UT32 : nullptr;
   *out = H.release();
   return JOLT_OK;
 }
@@ -1246,6 +1311,7 @@ extern "C" int jolt_get_component(const jolt_handle *H, int32_t cell, int32_t wh
     case 5: src = cs.e; n = 4; break;
     case 6: src = cs.sigma; n = 4 * (size_t)cs.n_sigma; break;
     case 7: src = cs.lam; n = 4 * (size_t)kD; break;
+    case 8: src = cs.dbg_UT32; n = cs.dbg_UT32 ? 4 * (size_t)c.T * c.r_t : 0; break;
     default: return fail(JOLT_EINVAL, "component %d", which);
   }
   *written = (int64_t)n;

@@ -10,13 +10,22 @@ from tests.helpers import cell_view, code_mismatch, oracle_cache, projector_dist
 pytestmark = pytest.mark.gpu
 
 REL_RECON = 1e-3       # ||X^_gpu - X^_oracle||_F / ||X^_oracle||_F
-# Two runs whose residuals differ slightly disagree on a small fraction f of the codes, each by one step
-# Delta.  With uniform quantisation noise Delta = sqrt(12) * e * rms(X) (e = the oracle's own relative error),
-# so the reconstructions differ by sqrt(12 f) * e.  With factors computed independently in fp32-grade
-# arithmetic (vs the oracle's fp64) the backbones differ by ~1e-4 relative, which moves up to f = 0.5 % of the
-# codes of a coarse residual (the same allowance as the injected-factor code test); that is 0.245 e and exceeds
-# 1e-3 only for residuals of 3 bits and fewer.  The gate is the larger of the two.
-FLIP_SLACK = (12 * 5e-3) ** 0.5
+# End-to-end reconstructions (factors computed independently on each side).  Factors that agree to fp32
+# grade (1e-5) still round to DIFFERENT fp16 neighbours on a large share of their entries, so the two stored
+# backbones differ by the fp16 rounding noise itself, d ~ 4e-4 of rms(X) (three rounded quantities, two
+# independent copies).  The closed-loop residual absorbs that, but a shifted residual lands in another bin for a
+# fraction f ~ d / Delta of the entries, Delta = sqrt(12) * e * rms(X) being the step at the oracle's own
+# relative error e; each flip moves one entry by Delta, so the reconstructions separate by
+# sqrt(f) * Delta = sqrt(d * sqrt(12) * e) ~ 0.04 sqrt(e).  The gate is the larger of 1e-3 and that.  With
+# IDENTICAL stored factors (test_injected_factors_codes_match) the strict 1e-3 applies.
+FLIP_COEF = 0.04
+
+
+def recon_gate(e):
+    return max(REL_RECON, FLIP_COEF * e ** 0.5)
+
+
+FLIP_SLACK = None   # superseded by recon_gate
 REL_ERR = 0.02         # per-tensor reconstruction error within 2 % of the oracle's
 PROJ = 1e-3            # || U U^T - U0 U0^T ||_F
 CODE_FRAC = 1e-3       # fraction of codes allowed to differ (by exactly 1)
@@ -41,6 +50,9 @@ def _np(t):
 
 def _roundtrip(B, K, V, gs, plans, opts, factors=None):
     h = B.jolt_compress(K, V, gs, plans, opts, factors=factors)
+    # the fp32 token factors are a view of scratch memory: read them before the next library call
+    h.UT32 = [h.component(c, 8).astype(np.float64) if plans[c][0] > 0 and factors is None else None
+              for c in range(len(plans))]
     Ko, Vo = torch.empty_like(K), torch.empty_like(V)
     B.jolt_decompress(h, Ko, Vo, gs)
     torch.cuda.synchronize()
@@ -54,7 +66,7 @@ def _check_recon(Knp, Vnp, Ko, Vo, gs, ocells, tag=""):
         Xo = O.decompress_cell(oc)
         rel = np.linalg.norm(Xg - Xo) / np.linalg.norm(Xo)
         eg, eo = O.rel_frobenius(X, Xg), O.rel_frobenius(X, Xo)
-        assert rel <= max(REL_RECON, FLIP_SLACK * eo), (tag, c, rel, eo)
+        assert rel <= recon_gate(eo), (tag, c, rel, eo)
         assert abs(eg - eo) <= REL_ERR * eo + 1e-7, (tag, c, eg, eo)
 
 
@@ -140,19 +152,20 @@ def test_config0(B, synth, token_mode):
     for c, o in enumerate(oc):
         X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
         UF = h.component(c, 2).astype(np.float64).reshape(128, 64)
-        UT = h.component(c, 1).astype(np.float64).reshape(512, 64)
+        UT = h.UT32[c].reshape(512, 64)      # token factor before fp16 storage
+        UTo = o.ideal["U_T"]
         lam = o.ideal["lam"]
         assert projector_distance(UF, o.UF16) <= PROJ, (c, "U_F")
         sig = o.ideal["sigma"]
         gap_t = (sig[63] - sig[64]) / sig[0]
         if gap_t > 1e-2:
-            assert projector_distance(UT, o.UT16) <= PROJ, (c, "U_T", gap_t)
+            assert projector_distance(UT, UTo) <= PROJ, (c, "U_T", gap_t)
         else:
             # gapless spectrum at r_t (keys with amplified noise channels): the subspace is not unique to
             # tolerance; compare the energy the two token factors capture instead
             Y = np.einsum("htf,fs->hts", X, o.ideal["U_F"])
             A = O.token_unfold(Y)
-            eg, eo = np.linalg.norm(UT.T @ A) ** 2, np.linalg.norm(o.UT16.T @ A) ** 2
+            eg, eo = np.linalg.norm(UT.T @ A) ** 2, np.linalg.norm(UTo.T @ A) ** 2
             assert abs(eg - eo) <= 1e-4 * eo, (c, eg, eo, gap_t)
         # stored singular values / eigenvalues
         ks = len(h.component(c, 6))
@@ -176,11 +189,12 @@ def test_small_gqa_cache(B, synth, bits_k, bits_v):
     assert h.bytes() == sum(O.stored_bytes(o.m, o.T, 128, o.r_t, o.r_f, o.bits) for o in oc)
     _check_recon(Knp, Vnp, Ko, Vo, gs, oc, "small gqa")
     for c, o in enumerate(oc):
-        UT = h.component(c, 1).astype(np.float64).reshape(o.UT16.shape)
+        UT = h.UT32[c].reshape(o.UT16.shape)   # before fp16 storage
         sig = o.ideal["sigma"]
         rt = o.r_t
         if (sig[rt - 1] - sig[rt]) / sig[0] > 1e-2:
-            assert projector_distance(UT, o.UT16) <= PROJ, c
+            assert projector_distance(UT, o.ideal["U_T"]) <= PROJ, c
+        assert np.linalg.norm(UT.T @ UT - np.eye(rt)) <= 1e-4
     h.free()
 
 
@@ -280,5 +294,5 @@ def test_tensor_core_and_portable_paths_agree(B, synth):
         ea = float((a - src.float()).norm() / src.float().norm())
         eb = float((b - src.float()).norm() / src.float().norm())
         assert abs(ea - eb) <= REL_ERR * ea
-        assert float((a - b).norm() / a.norm()) <= max(REL_RECON, FLIP_SLACK * ea)
+        assert float((a - b).norm() / a.norm()) <= recon_gate(ea)
         assert np.allclose(outs[False][2][i][:32], outs[True][2][i][:32], rtol=1e-4)
