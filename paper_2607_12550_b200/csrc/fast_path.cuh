@@ -3,6 +3,7 @@
 // multiple of 8); every other cell stays on the portable kernels, in the same call.
 #pragma once
 #include "tc_backbone.cuh"
+#include "tc_decode.cuh"
 #include "tc_gemm.cuh"
 
 namespace {
@@ -61,6 +62,23 @@ inline void add_backbone_tc(Program &P, int stage, const std::vector<tc::BBCell>
   const int n = (int)cells.size();
   P.add(stage, [=](char *dev_t, cudaStream_t s) {
     tc::backbone_kernel<RESIDUAL><<<dim3(gx, n), tc::BB_THREADS, tc::BB_SMEM_BYTES, s>>>((const tc::BBCell *)(dev_t + off), seed);
+    LAUNCHED();
+  });
+}
+
+inline void add_decode_tc(Program &P, int stage, const std::vector<tc::BBCell> &cells, uint64_t seed) {
+  if (cells.empty()) return;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaFuncSetAttribute(tc::decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::DEC_SMEM_BYTES);
+    attr_done = true;
+  }
+  int gx = 0;
+  for (auto &c : cells) gx = std::max(gx, c.m * c.items_per_head);
+  const size_t off = P.push(cells);
+  const int n = (int)cells.size();
+  P.add(stage, [=](char *dev_t, cudaStream_t s) {
+    tc::decode_kernel<<<dim3(gx, n), tc::DEC_THREADS, tc::DEC_SMEM_BYTES, s>>>((const tc::BBCell *)(dev_t + off), seed);
     LAUNCHED();
   });
 }

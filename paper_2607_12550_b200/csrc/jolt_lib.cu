@@ -27,6 +27,7 @@ namespace jolt {
 thread_local std::string g_err;
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_eig_smem{1};
+long long *g_dbg_stamps = nullptr;   // device buffer for kernel cycle stamps (profiling aid)
 std::atomic<int> g_fast{7};   // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores
 
 int fail(int code, const char *fmt, ...) {
@@ -1235,6 +1236,15 @@ extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void 
       b.tiles_per_item = tpi; b.items_per_head = iph;
       b.out = obase; b.out_dtype = L->dtype == JOLT_F16 ? DT_F16 : DT_F32;
       b.osl = L->stride_layer; b.osh = L->stride_head; b.ost = L->stride_token;
+      b.tma_out = 0;
+      b.dbg = g_dbg_stamps;
+      if (L->dtype == JOLT_F16 && L->stride_token % 8 == 0 && L->stride_head % 8 == 0 && L->stride_layer % 8 == 0 &&
+          ((uintptr_t)obase % 16 == 0)) {
+        const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)c.T, (uint64_t)c.n_heads, (uint64_t)(c.m / c.n_heads)};
+        const uint64_t str[3] = {(uint64_t)L->stride_token * 2, (uint64_t)L->stride_head * 2, (uint64_t)L->stride_layer * 2};
+        const uint32_t box[4] = {64, 128, 1, 1};
+        if (make_tmap_f16(&b.tmOut, obase, 4, dims, str, box)) b.tma_out = 1;
+      }
       bbc.push_back(b);
       continue;
     }
@@ -1249,7 +1259,7 @@ extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void 
     rows += (long long)c.m * c.T;
     rj.push_back(j);
   }
-  add_backbone_tc<false>(P, ST_DROWS, bbc, H->seed);
+  add_decode_tc(P, ST_DROWS, bbc, H->seed);
   add_backbone(P, ST_DBACK, br);
   if (!rj.empty()) {
     const size_t off = P.push(rj);
@@ -1510,6 +1520,16 @@ extern "C" int jolt_release_workspace(void) {
   if (g_ws[dev].base) { cudaFree(g_ws[dev].base); g_ws[dev] = Workspace(); }
   if (g_tab[dev].base) { cudaFree(g_tab[dev].base); g_tab[dev] = Workspace(); }
   return JOLT_OK;
+}
+extern "C" int jolt_debug_stamps(long long *host_out, int n) {
+  // n > 0 and host_out == nullptr: (re)allocate and zero a device stamp buffer of n entries; host_out != nullptr: read it back
+  if (!host_out) {
+    if (g_dbg_stamps) { cudaFree(g_dbg_stamps); g_dbg_stamps = nullptr; }
+    if (n > 0) { if (cudaMalloc(&g_dbg_stamps, sizeof(long long) * n) != cudaSuccess) return JOLT_ENOMEM; cudaMemset(g_dbg_stamps, 0, sizeof(long long) * n); }
+    return JOLT_OK;
+  }
+  if (!g_dbg_stamps) return JOLT_EINVAL;
+  return cudaMemcpy(host_out, g_dbg_stamps, sizeof(long long) * n, cudaMemcpyDeviceToHost) == cudaSuccess ? JOLT_OK : JOLT_ECUDA;
 }
 extern "C" int64_t jolt_launch_count(void) { return g_launches.load(); }
 extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled & 7); }

@@ -28,6 +28,9 @@ struct alignas(64) BBCell {
   CUtensorMap tmUF;     // fp16 [128][r_f]         dims {r_f, 128},     box {64, 128}
   CUtensorMap tmG;      // fp16 [m*r_t][r_f]       dims {r_f, m*r_t},   box {64, r_t}
   CUtensorMap tmX;      // fp16 [L][n_h][T][128]   dims {128, T, n_h, L}, box {64, 128, 1, 1}   (RESIDUAL)
+  CUtensorMap tmOut;    // same shape over the output tensor (DECODE, fp16 destinations TMA can address)
+  int tma_out;
+  long long *dbg;       // optional: cycle stamps of CTA 0 (profiling aid), 8 per tile per warpgroup
   uint32_t *words;      // [m][T][4*bits]
   __half *scales;       // [m][T][4]
   const int *e;         // core exponent
@@ -99,12 +102,12 @@ __global__ void __launch_bounds__(BB_THREADS, 1) backbone_kernel(const BBCell *_
   const uint32_t sX = sBig + 4 * BB_STAGE_BYTES;       // RESIDUAL: two X tiles behind a 4-stage ring
   // barrier slots (8 bytes each)
   const uint32_t bSetup = sBar + 0, bPdone = sBar + 8, bPready = sBar + 16;
-  auto bFull = [&](int s) { return sBar + 24 + 8 * s; };
-  auto bEmpty = [&](int s) { return sBar + 24 + 64 + 8 * s; };
-  auto bTfull = [&](int b) { return sBar + 152 + 8 * b; };
-  auto bTempty = [&](int b) { return sBar + 168 + 8 * b; };
-  auto bXfull = [&](int b) { return sBar + 184 + 8 * b; };
-  auto bXempty = [&](int b) { return sBar + 200 + 8 * b; };
+  auto bFull = [=](int s) { return sBar + 24 + 8 * s; };
+  auto bEmpty = [=](int s) { return sBar + 24 + 64 + 8 * s; };
+  auto bTfull = [=](int b) { return sBar + 152 + 8 * b; };
+  auto bTempty = [=](int b) { return sBar + 168 + 8 * b; };
+  auto bXfull = [=](int b) { return sBar + 184 + 8 * b; };
+  auto bXempty = [=](int b) { return sBar + 200 + 8 * b; };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = warp >> 2;

@@ -1,0 +1,370 @@
+// Fused decompress pass (paper Sec. 4 "decoding simply inverts the rotation", Sec. 7): for a (cell, head,
+// run of 128-token tiles)
+//
+//     X^[tile] = 2^e ( U_T[tile] P_h  +  R^[tile] (H S) )
+//
+// as ONE tcgen05 accumulation per tile: the backbone (K = r_t) and the inverse rotation of the dequantised
+// residual (K = 128, B operand = the +-1 Hadamard matrix with the sign flips folded in, exact in fp16) go into
+// the same TMEM accumulator.  The epilogue threads only unpack codes into a half-precision operand tile
+// (pre-scaled by Delta / sqrt(128) * 2^-e) and, after the MMA, scale, convert and store their row: no
+// Hadamard butterflies on the CUDA cores.  P_h^T = fp16(U_F G_h^T) is formed once per CTA as in the residual
+// kernel.  Rounding the dequantised residual to fp16 before the rotation costs 2^-11 of the residual, i.e.
+// ~1e-5 of the cache entries, far below the fp16 rounding of the output itself.
+#pragma once
+#include "tc_backbone.cuh"
+
+namespace jolt {
+namespace tc {
+
+constexpr int DEC_THREADS = 384;
+constexpr int DEC_P_BYTES = 65536, DEC_H_BYTES = 32768, DEC_BIG_BYTES = 131072;
+constexpr int DEC_NS = 4;
+constexpr int DEC_SMEM_BYTES = DEC_P_BYTES + DEC_H_BYTES + DEC_BIG_BYTES + 1024 + 512;
+
+template <int BITS>
+struct DecCodes { uint32_t words[BITS > 0 ? 4 * BITS : 1]; uint2 sc; };
+
+template <int BITS>
+__device__ __forceinline__ void dec_load_codes(const BBCell &c, long long row, DecCodes<BITS> &d) {
+  if constexpr (BITS > 0) {
+    const uint4 *wp = (const uint4 *)(c.words + row * (4 * BITS));
+#pragma unroll
+    for (int i = 0; i < BITS; ++i) { const uint4 v = __ldg(wp + i); d.words[4 * i] = v.x; d.words[4 * i + 1] = v.y; d.words[4 * i + 2] = v.z; d.words[4 * i + 3] = v.w; }
+    d.sc = __ldg((const uint2 *)(c.scales + row * 4));
+  }
+}
+
+// codes -> fp16 operand row (pre-scaled), written into the warpgroup's swizzled K-major tile
+template <int BITS>
+__device__ __forceinline__ void dec_unpack_row(const DecCodes<BITS> &d, float pre, unsigned char *rbuf, int rit) {
+  constexpr float off = 0.5f - (float)(1 << (BITS > 0 ? BITS - 1 : 0));
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  const __half *sc = (const __half *)&d.sc;
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    const float dq = __half2float(sc[g]) * pre;
+    unsigned char *rowp = rbuf + (g >> 1) * 16384 + rit * 128;
+#pragma unroll
+    for (int ck = 0; ck < 4; ++ck) {
+      uint4 pk;
+      __half2 *hp = (__half2 *)&pk;
+#pragma unroll
+      for (int e2 = 0; e2 < 4; ++e2) {
+        float v2[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          // code j of the group sits at bits [j*BITS, j*BITS + BITS) of its BITS little-endian words
+          const int j = ck * 8 + e2 * 2 + u;
+          const int bit = j * BITS, w = bit >> 5, sh = bit & 31;
+          uint32_t q = d.words[g * BITS + w] >> sh;
+          if (sh + BITS > 32) q |= d.words[g * BITS + w + 1] << (32 - sh);
+          v2[u] = ((float)(q & mask) + off) * dq;
+        }
+        hp[e2] = __floats2half2_rn(v2[0], v2[1]);
+      }
+      const int chunk = (g & 1) * 4 + ck;
+      *(uint4 *)(rowp + ((chunk ^ (rit & 7)) << 4)) = pk;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_store_4d(const void *tmap, uint32_t src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+               ::"l"(tmap), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+struct DecCtx {
+  uint32_t bTfull, bTempty, bRready, t_acc, s_obuf;
+  unsigned char *rbuf, *obuf;
+  bool sep_out;
+  volatile int *abort_flag;
+  int wg, rit, h, tile0, n_tiles, l, hd;
+  float scale, pre;
+};
+
+// The per-tile loop of one epilogue warpgroup (tiles wg, wg+2, ...).
+template <int BITS>
+__device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) {
+  DecCodes<BITS> cur, nxt;
+  bool ok = true;
+  const bool tma_out = c.tma_out != 0;
+  if (x.wg < x.n_tiles) dec_load_codes<BITS>(c, (long long)x.h * c.T + (x.tile0 + x.wg) * 128 + x.rit, cur);
+  const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;
+  for (int i = x.wg; ok && i < x.n_tiles; i += 2) {
+    const int tt = x.tile0 + i, nb = i >> 1;
+    const int token = tt * 128 + x.rit;
+    long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;
+    if (dbg) dbg[0] = clock64();
+    if (tma_out && !x.sep_out) {   // shared buffer: the previous store must have read it before the operand is written
+      if (x.rit == 0) tma_store_wait_read();
+      named_bar_sync(1 + x.wg, 128);
+    }
+    if (dbg) dbg[1] = clock64();
+    if constexpr (BITS > 0) {
+      dec_unpack_row<BITS>(cur, x.pre, x.rbuf, x.rit);
+      fence_proxy_async();
+      mbar_arrive(x.bRready);
+      if (dbg) dbg[2] = clock64();
+      if (i + 2 < x.n_tiles) dec_load_codes<BITS>(c, (long long)x.h * c.T + (tt + 2) * 128 + x.rit, nxt);   // in flight during the MMA
+    }
+    ok = __all_sync(0xffffffffu, mbar_wait(x.bTfull, nb & 1, x.abort_flag));
+    if (!ok) break;
+    if (dbg) dbg[3] = clock64();
+    tc_fence_after();
+    const long long off = (long long)x.l * c.osl + (long long)x.hd * c.osh + (long long)token * c.ost;
+    if (tma_out && x.sep_out) {    // own staging buffer: only now must the previous tile's store have drained
+      if (x.rit == 0) tma_store_wait_read();
+      named_bar_sync(1 + x.wg, 128);
+    }
+    float va[2][32];
+    tmem_ld32(x.t_acc, va[0]);
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch) {
+      tmem_wait_ld();
+      if (ch + 1 < 4) tmem_ld32(x.t_acc + (ch + 1) * 32, va[(ch + 1) & 1]);     // next chunk in flight during the conversion
+      else { tc_fence_before(); mbar_arrive(x.bTempty); if (dbg) dbg[4] = clock64(); }
+      const float *v = va[ch & 1];
+      if (c.out_dtype == DT_F16) {
+        uint4 o[4];
+#pragma unroll
+        for (int k8 = 0; k8 < 4; ++k8) {
+          __half2 *hp = (__half2 *)&o[k8];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) hp[j] = __floats2half2_rn(v[k8 * 8 + 2 * j] * x.scale, v[k8 * 8 + 2 * j + 1] * x.scale);
+        }
+        if (tma_out) {      // stage the row, same swizzled layout as a loaded X tile
+          unsigned char *rowp = x.obuf + (ch >> 1) * 16384 + x.rit * 128;
+#pragma unroll
+          for (int k8 = 0; k8 < 4; ++k8) *(uint4 *)(rowp + ((((ch & 1) * 4 + k8) ^ (x.rit & 7)) << 4)) = o[k8];
+        } else {
+          uint4 *p = (uint4 *)((__half *)c.out + off + ch * 32);
+#pragma unroll
+          for (int k8 = 0; k8 < 4; ++k8) p[k8] = o[k8];
+        }
+      } else {
+        float4 *p = (float4 *)((float *)c.out + off + ch * 32);
+#pragma unroll
+        for (int k4 = 0; k4 < 8; ++k4)
+          p[k4] = make_float4(v[4 * k4] * x.scale, v[4 * k4 + 1] * x.scale, v[4 * k4 + 2] * x.scale, v[4 * k4 + 3] * x.scale);
+      }
+    }
+    if (dbg) dbg[5] = clock64();
+    if (tma_out) {
+      fence_proxy_async();
+      named_bar_sync(1 + x.wg, 128);
+      if (dbg) dbg[6] = clock64();
+      if (x.rit == 0) {
+        tma_store_4d(&c.tmOut, x.s_obuf, 0, tt * 128, x.hd, x.l);
+        tma_store_4d(&c.tmOut, x.s_obuf + 16384, 64, tt * 128, x.hd, x.l);
+        tma_store_commit();
+      }
+    }
+    if (dbg) dbg[7] = clock64();
+    if constexpr (BITS > 0) cur = nxt;
+  }
+  if (tma_out && x.rit == 0) tma_store_wait_all();
+  return ok;
+}
+
+__global__ void __launch_bounds__(DEC_THREADS, 1) decode_kernel(const BBCell *__restrict__ cells, uint64_t seed) {
+  extern __shared__ unsigned char smem_raw[];
+  const BBCell &c = cells[blockIdx.y];
+  const int items = c.m * c.items_per_head;
+  if ((int)blockIdx.x >= items) return;
+  const int h = blockIdx.x / c.items_per_head;
+  const int item = blockIdx.x - h * c.items_per_head;
+  const int tile0 = item * c.tiles_per_item;
+  const int n_tiles = min(c.tiles_per_item, c.T / 128 - tile0);
+  if (n_tiles <= 0) return;
+
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char *sm = smem_raw + (base - raw);
+  const uint32_t sP = base, sH = base + DEC_P_BYTES, sBig = sH + DEC_H_BYTES;
+  const uint32_t sRing = sBig, sR = sBig + DEC_NS * BB_STAGE_BYTES;
+  const uint32_t sBar = sBig + DEC_BIG_BYTES;
+  unsigned char *smH = sm + DEC_P_BYTES, *smR = sm + DEC_P_BYTES + DEC_H_BYTES + DEC_NS * BB_STAGE_BYTES;
+  volatile int *abort_flag = (volatile int *)(sm + DEC_P_BYTES + DEC_H_BYTES + DEC_BIG_BYTES + 256);
+  uint32_t *tmem_slot = (uint32_t *)(sm + DEC_P_BYTES + DEC_H_BYTES + DEC_BIG_BYTES + 264);
+  const uint32_t bSetup = sBar + 0, bPdone = sBar + 8, bPready = sBar + 16;
+  auto bFull = [=](int s) { return sBar + 24 + 8 * s; };
+  auto bEmpty = [=](int s) { return sBar + 56 + 8 * s; };
+  auto bTfull = [=](int b) { return sBar + 88 + 8 * b; };
+  auto bTempty = [=](int b) { return sBar + 104 + 8 * b; };
+  auto bRready = [=](int b) { return sBar + 120 + 8 * b; };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int wg = warp >> 2;
+  const int nkt = (c.r_t + 63) / 64, nkf = (c.r_f + 63) / 64;
+  const bool has_res = c.bits > 0;
+  // r_t <= 128 leaves half of the P region and half of the ring free: each warpgroup then stages its output in a
+  // buffer of its own, so a tile's unpack never waits for the previous tile's TMA store to drain
+  const bool sep_out = nkt <= 2;
+  const int ns = sep_out ? 2 : DEC_NS;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    mbar_init(bSetup, 1); mbar_init(bPdone, 1); mbar_init(bPready, 256);
+    for (int s = 0; s < DEC_NS; ++s) { mbar_init(bFull(s), 1); mbar_init(bEmpty(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bTfull(b), 1); mbar_init(bTempty(b), 128); mbar_init(bRready(b), 128); }
+    fence_barrier_init();
+  }
+  if (warp == 8) { tmem_alloc(smem_u32(tmem_slot), BB_TMEM_COLS); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (wg == 2) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    if (warp == 8 && lane == 0) {
+      // ---------------- TMA producer
+      tma_prefetch_desc(&c.tmUT); tma_prefetch_desc(&c.tmUF); tma_prefetch_desc(&c.tmG);
+      mbar_expect_tx(bSetup, (uint32_t)nkf * (16384u + (uint32_t)c.r_t * 128u));
+      for (int kb = 0; kb < nkf; ++kb) {
+        tma_load_2d(sBig + kb * 16384, &c.tmUF, bSetup, kb * 64, 0);
+        tma_load_2d(sBig + 32768 + kb * 32768, &c.tmG, bSetup, kb * 64, h * c.r_t);
+      }
+      bool ok = mbar_wait(bPdone, 0, abort_flag);
+      int cnt = 0;
+      for (int i = 0; ok && i < n_tiles; ++i) {
+        const int tt = tile0 + i;
+        for (int kb = 0; kb < nkt; ++kb, ++cnt) {
+          const int s = cnt % ns, n = cnt / ns;
+          ok = mbar_wait(bEmpty(s), (n & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(bFull(s), BB_STAGE_BYTES);
+          tma_load_2d(sRing + s * BB_STAGE_BYTES, &c.tmUT, bFull(s), kb * 64, tt * 128);
+        }
+      }
+    } else if (warp == 9 && lane == 0) {
+      // ---------------- MMA issuer (one thread, tiles in order: the ring's phase parities stay unambiguous)
+      bool ok = mbar_wait(bSetup, 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        const uint32_t idescP = umma_idesc_f16(128, c.r_t, 0, 0);
+        for (int kb = 0; kb < nkf; ++kb)
+          for (int k4 = 0; k4 < 4; ++k4)
+            umma_f16(tmem_base, umma_desc_sw128(sBig + kb * 16384 + k4 * 32, 16, 1024),
+                     umma_desc_sw128(sBig + 32768 + kb * 32768 + k4 * 32, 16, 1024), idescP, (kb | k4) != 0);
+        umma_commit(bPdone);
+        ok = mbar_wait(bPready, 0, abort_flag);
+      }
+      if (ok) {
+        tc_fence_after();
+        const uint32_t idesc = umma_idesc_f16(128, 128, 0, 0);
+        int cnt = 0;
+        for (int i = 0; ok && i < n_tiles; ++i) {
+          const int b = i & 1, nb = i >> 1;
+          ok = mbar_wait(bTempty(b), (nb & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          for (int kb = 0; kb < nkt; ++kb, ++cnt) {
+            const int s = cnt % ns, n = cnt / ns;
+            ok = mbar_wait(bFull(s), n & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            for (int k4 = 0; k4 < 4; ++k4)
+              umma_f16(tmem_base + b * 128, umma_desc_sw128(sRing + s * BB_STAGE_BYTES + k4 * 32, 16, 1024),
+                       umma_desc_sw128(sP + kb * 16384 + k4 * 32, 16, 1024), idesc, (kb | k4) != 0);
+            umma_commit(bEmpty(s));
+          }
+          if (!ok) break;
+          if (has_res) {
+            ok = mbar_wait(bRready(b), nb & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            for (int kb = 0; kb < 2; ++kb)
+              for (int k4 = 0; k4 < 4; ++k4)
+                umma_f16(tmem_base + b * 128, umma_desc_sw128(sR + b * 32768 + kb * 16384 + k4 * 32, 16, 1024),
+                         umma_desc_sw128(sH + kb * 16384 + k4 * 32, 16, 1024), idesc, 1);
+          }
+          umma_commit(bTfull(b));
+        }
+      }
+    }
+  } else {
+    // ---------------- epilogue warpgroups
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    const int q = warp & 3;
+    const int rit = q * 32 + lane;                 // row in tile
+    const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
+    {  // B operand of the inverse rotation: Hs[f][f'] = s_f * (-1)^popcount(f & f'), fp16, K-major, swizzled
+      uint32_t sw[4];
+      cell_sign_words(seed, c.cell, sw);
+      const int et = wg * 128 + rit;               // 256 threads, 2048 16-byte chunks
+      for (int ci = et; ci < 2048; ci += 256) {
+        const int f = ci >> 4, chunk = ci & 15;
+        const uint32_t sgn = (sw[f >> 5] >> (f & 31)) & 1u;
+        uint4 pk;
+        uint32_t *pw = (uint32_t *)&pk;
+#pragma unroll
+        for (int e2 = 0; e2 < 4; ++e2) {
+          const int fp = chunk * 8 + e2 * 2;
+          const uint32_t n0 = (__popc(f & fp) & 1u) ^ sgn, n1 = (__popc(f & (fp + 1)) & 1u) ^ sgn;
+          pw[e2] = (0x3C00u | (n0 << 15)) | ((0x3C00u | (n1 << 15)) << 16);      // +-1.0 in fp16
+        }
+        *(uint4 *)(smH + (chunk >> 3) * 16384 + f * 128 + (((chunk & 7) ^ (f & 7)) << 4)) = pk;
+      }
+    }
+    bool ok = __all_sync(0xffffffffu, mbar_wait(bPdone, 0, abort_flag));
+    if (ok) {
+      tc_fence_after();
+      for (int ch = wg; ch < 2 * nkt; ch += 2) {
+        float v[32];
+        tmem_ld32(t_lane + ch * 32, v);
+        tmem_wait_ld();
+        unsigned char *rowp = sm + (ch >> 1) * 16384 + rit * 128;
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          uint4 pk;
+          __half2 *hp = (__half2 *)&pk;
+#pragma unroll
+          for (int e2 = 0; e2 < 4; ++e2) {
+            const int col = ch * 32 + jj * 8 + e2 * 2;
+            hp[e2] = __floats2half2_rn(col < c.r_t ? v[jj * 8 + e2 * 2] : 0.f, col + 1 < c.r_t ? v[jj * 8 + e2 * 2 + 1] : 0.f);
+          }
+          *(uint4 *)(rowp + ((((ch & 1) * 4 + jj) ^ (rit & 7)) << 4)) = pk;
+        }
+      }
+      fence_proxy_async();
+      tc_fence_before();
+      mbar_arrive(bPready);
+    }
+    const int ex = ok ? *c.e : 0;
+    const float scale = ldexpf(1.0f, ex);
+    const float pre = ldexpf(kInvSqrtD, -ex);        // residual operand is kept in the accumulator's units
+    if (ok) {
+      DecCtx x;
+      x.bTfull = bTfull(wg); x.bTempty = bTempty(wg); x.bRready = bRready(wg);
+      x.t_acc = t_lane + wg * 128; x.rbuf = smR + wg * 32768; x.sep_out = sep_out;
+      if (sep_out) { x.s_obuf = wg == 0 ? sP + 32768 : sRing + 32768; x.obuf = wg == 0 ? sm + 32768 : sm + DEC_P_BYTES + DEC_H_BYTES + 32768; }
+      else { x.s_obuf = sR + wg * 32768; x.obuf = x.rbuf; }
+      x.abort_flag = abort_flag; x.wg = wg; x.rit = rit; x.h = h; x.tile0 = tile0; x.n_tiles = n_tiles;
+      x.l = h / c.n_heads; x.hd = h - x.l * c.n_heads; x.scale = scale; x.pre = pre;
+      switch (c.bits) {
+        case 0: dec_tile_loop<0>(c, x); break;
+        case 1: dec_tile_loop<1>(c, x); break;
+        case 2: dec_tile_loop<2>(c, x); break;
+        case 3: dec_tile_loop<3>(c, x); break;
+        case 4: dec_tile_loop<4>(c, x); break;
+        default: dec_tile_loop<8>(c, x); break;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicOr(c.status, 8);
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000) {}
+    __syncthreads();
+  }
+  if (warp == 8) { tc_fence_after(); tmem_dealloc(tmem_base, BB_TMEM_COLS); }
+}
+
+}  // namespace tc
+}  // namespace jolt

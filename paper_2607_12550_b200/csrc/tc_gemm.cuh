@@ -54,8 +54,8 @@ __global__ void __launch_bounds__(GM_THREADS, 1) tc_gemm_kernel(const GemmCell *
   const uint32_t sBar = base + (uint32_t)n_stages * stage_bytes;
   volatile int *abort_flag = (volatile int *)(sm + (size_t)n_stages * stage_bytes + 256);
   uint32_t *tmem_slot = (uint32_t *)(sm + (size_t)n_stages * stage_bytes + 264);
-  auto bFull = [&](int s) { return sBar + 8 * s; };
-  auto bEmpty = [&](int s) { return sBar + 64 + 8 * s; };
+  auto bFull = [=](int s) { return sBar + 8 * s; };
+  auto bEmpty = [=](int s) { return sBar + 64 + 8 * s; };
   const uint32_t bDone = sBar + 128;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
