@@ -42,7 +42,7 @@ class ClockSampler:
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
                                           "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
@@ -150,7 +150,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="jolt", choices=["jolt", "reference"])
     ap.add_argument("--workload", default="c1")
@@ -309,17 +309,24 @@ def main():
     t_roof_d = sum(roof_time(*cell_work(cfg.m, cfg.seq_len, cfg.head_dim, rt, rf, b, min(rt + 10, cfg.seq_len, cfg.m * rf), q, 2)["decompress"], pk)
                    for rt, rf, b in plans)
     stages = {k_: v_ / len(rec) for k_, v_ in stage_acc.items()}
-    # dominant kernel = the decode pass (the headline HBM-bound kernel); its duration is the decompress call
+    # roofline of the dominant kernel of the headline (decompress) call: decode_kernel is the only kernel of
+    # jolt_decompress; its duration is the library's own CUDA-event stage timer on the launching stream
     fd, bd = tot["decompress"]
+    t_dec = stages.get("decode_rows", td)
     dec_bound = "hbm" if bd / (pk["hbm"] * 1e9) >= fd / (pk["tensor"] * 1e12) else "tensor"
+    # DRAM traffic of one launch: ncu capture of the first 2 groups (profiles/decode_kernel_config1_2groups.md:
+    # 60.4 MB read + 78.5 MB written for 4 of the 16 cells), scaled by the cells of this run
+    traffic = (60.438e6 + 78.455e6) * (2 * ng) / 4 if cfg.name == "c1" else None
     if dec_bound == "hbm":
-        ach = bd / (td * 1e-3) / 1e9
-        roofline = {"kernel": "decompress pass", "bound": "hbm", "achieved": ach, "peak": pk["hbm"], "unit": "GB/s",
-                    "frac": ach / pk["hbm"], "traffic": None, "peak_source": pk["source"]}
+        ach = bd / (t_dec * 1e-3) / 1e9
+        roofline = {"kernel": "tc::decode_kernel", "bound": "hbm", "achieved": ach, "peak": pk["hbm"], "unit": "GB/s",
+                    "frac": ach / pk["hbm"], "traffic": traffic, "algorithmic_bytes": bd, "kernel_ms": t_dec,
+                    "peak_source": pk["source"] + " (MEASURED_PEAKS.json hbm_gbs)"}
     else:
-        ach = fd / (td * 1e-3) / 1e12
-        roofline = {"kernel": "decompress pass", "bound": "tensor", "achieved": ach, "peak": pk["tensor"], "unit": "TFLOP/s",
-                    "frac": ach / pk["tensor"], "traffic": None, "peak_source": pk["source"]}
+        ach = fd / (t_dec * 1e-3) / 1e12
+        roofline = {"kernel": "tc::decode_kernel", "bound": "tensor", "achieved": ach, "peak": pk["tensor"], "unit": "TFLOP/s",
+                    "frac": ach / pk["tensor"], "traffic": traffic, "algorithmic_flops": fd, "kernel_ms": t_dec,
+                    "peak_source": pk["source"] + " (MEASURED_PEAKS.json bf16_tflops, burst)"}
 
     line = {"metric": METRIC, "value": world * cache_bytes / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
