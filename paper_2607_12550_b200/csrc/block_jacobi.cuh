@@ -13,7 +13,7 @@
 namespace jolt {
 
 constexpr int kBJBlock = 16;
-constexpr int kBJMaxSweeps = 12;
+constexpr int kBJMaxSweeps = 10;
 
 struct BJTask {
   const double *A_in;   // n x n symmetric input (untouched)
@@ -22,6 +22,7 @@ struct BJTask {
   double *J;            // (nbe/2) x 32 x 32 rotations of the current round
   double *off;          // [4]: off-diagonal mass (accumulator), total mass, last measured off-diagonal mass, sweeps run
   int *done;            // [1]
+  unsigned *ticket;     // [1] block counter of the check kernel
   int n, nP, nbe;       // size, padded size (16 * nbe), even number of blocks
   double *w;            // nP scratch (eigenvalues)
   float *U_out; int ld_out, r_out; float *w_out; int w_sqrt;
@@ -171,24 +172,37 @@ __global__ void __launch_bounds__(256) bj_apply_kernel(const BJTask *__restrict_
   }
 }
 
-__global__ void bj_check_kernel(const BJTask *__restrict__ tasks, int phase) {
+// Off-diagonal mass after a sweep; the last block to finish (ticket counter) compares it with the total mass,
+// raises `done` and resets the accumulators: one launch per sweep.
+__global__ void bj_check_kernel(const BJTask *__restrict__ tasks) {
   const BJTask t = tasks[blockIdx.y];
   if (*t.done) return;
-  if (phase == 0) {
-    double off = 0;
-    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < t.nP * t.nP; e += gridDim.x * blockDim.x) {
-      const int i = e / t.nP, j = e - i * t.nP;
-      if (i != j) { const double v = t.A[e]; off += v * v; }
+  double off = 0;
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < t.nP * t.nP; e += gridDim.x * blockDim.x) {
+    const int i = e / t.nP, j = e - i * t.nP;
+    if (i != j) { const double v = t.A[e]; off += v * v; }
+  }
+  for (int o = 16; o; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
+  __shared__ double red[8];
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = off;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0;
+    for (int i = 0; i < (int)blockDim.x / 32; ++i) s += red[i];
+    if (s != 0.0) atomicAdd(&t.off[0], s);
+    __threadfence();
+    const unsigned ticket = atomicAdd(t.ticket, 1u);
+    if (ticket == gridDim.x - 1) {           // every block's contribution is in
+      __threadfence();
+      const double total_off = atomicAdd(&t.off[0], 0.0);
+      // relative off-diagonal norm 3e-10: above the round-off floor of the 32-term block products on a
+      // rank-deficient matrix (measured 5e-11), far below the fp32 grade of what is read out
+      if (total_off <= 1e-19 * t.off[1]) *t.done = 1;
+      t.off[2] = total_off;
+      t.off[3] += 1.0;
+      t.off[0] = 0.0;
+      *t.ticket = 0u;
     }
-    for (int o = 16; o; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
-    if ((threadIdx.x & 31) == 0 && off != 0.0) atomicAdd(&t.off[0], off);
-  } else if (blockIdx.x == 0 && threadIdx.x == 0) {
-    // relative off-diagonal norm 3e-10: above the round-off floor of the 32-term block products on a
-    // rank-deficient matrix (measured 5e-11), far below the fp32 grade of what is read out
-    if (t.off[0] <= 1e-19 * t.off[1]) *t.done = 1;
-    t.off[2] = t.off[0];
-    t.off[3] += 1.0;      // sweeps run
-    t.off[0] = 0.0;
   }
 }
 
@@ -196,7 +210,9 @@ __global__ void __launch_bounds__(256) bj_finish_kernel(const BJTask *__restrict
   const BJTask t = tasks[blockIdx.x];
   const int n = t.n, nP = t.nP, tid = threadIdx.x, nt = blockDim.x;
   __shared__ int rk[2048];
-  if (tid == 0 && !*t.done && t.status) atomicOr(t.status, 1);
+  // not converged to the tight threshold after the last sweep: still accepted when the off-diagonal norm is below
+  // 1e-7 of the matrix norm (fp32 grade); flagged otherwise
+  if (tid == 0 && !*t.done && t.status && !(t.off[2] <= 1e-14 * t.off[1])) atomicOr(t.status, 1);
   for (int i = tid; i < n; i += nt) t.w[i] = t.A[(size_t)i * nP + i];
   __syncthreads();
   for (int i = tid; i < n; i += nt) {

@@ -280,7 +280,7 @@ void add_gemm(Program &P, int stage, const std::vector<GemmTask> &tasks, bool f6
   });
 }
 
-void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks) {
+void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sweeps) {
   if (tasks.empty()) return;
   // problems that fit one CTA's shared memory take the resident kernel, the rest the global-memory one
   std::vector<EigTask> small64, small32, big;
@@ -288,7 +288,7 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks) {
   for (auto &t : tasks) {
     if (t.bjA && t.n > 32 && g_eig_smem.load() != 2) {
       BJTask b; memset(&b, 0, sizeof b);
-      b.A_in = t.A; b.A = t.bjA; b.V = t.bjV; b.J = t.bjJ; b.off = t.bjOff; b.done = t.bjDone;
+      b.A_in = t.A; b.A = t.bjA; b.V = t.bjV; b.J = t.bjJ; b.off = t.bjOff; b.done = t.bjDone; b.ticket = (unsigned *)(t.bjDone + 1);
       b.n = t.n; b.nbe = (((t.n + kBJBlock - 1) / kBJBlock) + 1) & ~1; b.nP = b.nbe * kBJBlock;
       b.w = t.w; b.U_out = t.U_out; b.ld_out = t.ld_out; b.r_out = t.r_out; b.w_out = t.w_out; b.w_sqrt = t.w_sqrt; b.status = t.status;
       bj.push_back(b);
@@ -307,18 +307,17 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks) {
     std::vector<BJTask> copy = bj;
     P.add(stage, [=](char *dev, cudaStream_t s) {
       const BJTask *d = (const BJTask *)(dev + off);
-      for (auto &b : copy) { cudaMemsetAsync(b.off, 0, 4 * sizeof(double), s); cudaMemsetAsync(b.done, 0, sizeof(int), s); }
+      for (auto &b : copy) { cudaMemsetAsync(b.off, 0, 4 * sizeof(double), s); cudaMemsetAsync(b.done, 0, 2 * sizeof(int), s); }
       bj_init_kernel<<<dim3(64, n), 256, 0, s>>>(d); LAUNCHED();
       const int np = max_nbe / 2;
       const int gx = np * (np + 1) / 2 + np * (max_nP / 32);
-      const int max_sweeps = max_nbe > 12 ? 2 * kBJMaxSweeps : kBJMaxSweeps;   // larger problems take a few more sweeps
+      const int max_sweeps = bj_sweeps;
       for (int sw = 0; sw < max_sweeps; ++sw) {
         for (int r = 0; r < max_nbe - 1; ++r) {
           bj_solve_kernel<<<dim3(np, n), 256, 0, s>>>(d, r, r > 0 ? 1 : 0); LAUNCHED();
           bj_apply_kernel<<<dim3(gx, n), 256, 0, s>>>(d, r); LAUNCHED();
         }
-        bj_check_kernel<<<dim3(32, n), 256, 0, s>>>(d, 0); LAUNCHED();
-        bj_check_kernel<<<dim3(1, n), 32, 0, s>>>(d, 1); LAUNCHED();
+        bj_check_kernel<<<dim3(16, n), 256, 0, s>>>(d); LAUNCHED();
       }
       bj_finish_kernel<<<n, 256, 0, s>>>(d); LAUNCHED();
       if (getenv("JOLT_DEBUG_EIG")) {
@@ -424,7 +423,7 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
         const size_t nmax = std::max<size_t>(kD, mode == FM_EXACT ? T : k);
         const size_t nbe = (((nmax + kBJBlock - 1) / kBJBlock) + 1) & ~(size_t)1, nP = nbe * kBJBlock;
         w.bjA = b.take<double>(nP * nP); w.bjV = b.take<double>(nP * nP); w.bjJ = b.take<double>(nbe / 2 * 1024);
-        w.bjOff = b.take<double>(4); w.bjDone = b.take<int>(1);
+        w.bjOff = b.take<double>(4); w.bjDone = b.take<int>(2);
       }
       w.gram_part = b.take<double>((size_t)c.m * kD * kD);
       w.C = b.take<double>(kD * kD); w.Cv = b.take<double>(kD * kD); w.Cw = b.take<double>(kD);
@@ -681,7 +680,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
                                                                    (const int *)(dev + o3), kD * kD);
       LAUNCHED();
     });
-    add_eig(P, ST_EIGF, eg);
+    add_eig(P, ST_EIGF, eg, 14);        // Grams of caches with outlier channels span 1e6 in eigenvalue: slow to converge
     if (!idU.empty()) {
       const size_t p1 = P.push(idU), p2 = P.push(idLd);
       const int nid = (int)idU.size();
@@ -727,7 +726,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
       }
     }
     add_tall_gram(P, ST_SVD, tgb);
-    add_eig(P, ST_SVD, eg);
+    add_eig(P, ST_SVD, eg, 9);          // k x k, 6-7 sweeps observed
     add_gemm(P, ST_FACT, g2, false);
     add_gemm(P, ST_FACT, g3, false);
   } else if (mode == FM_EXACT) {
@@ -752,7 +751,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
     }
     add_gemm(P, ST_SKETCH, g1, false);
     add_gemm(P, ST_SKETCH, g2, true);
-    add_eig(P, ST_SVD, eg);
+    add_eig(P, ST_SVD, eg, 24);         // T x T
     add_gemm(P, ST_FACT, g3, false);
   } else if (mode == FM_INJECTED) {
     // core from given factors: Zp_h = X_h^T U_T (128 x r_t), G_h = Zp_h^T U_F (r_t x r_f)
@@ -978,6 +977,13 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
       stored += cell_bytes(c.m, c.T, kD, c.r_t, c.r_f, c.bits, true);
     }
     if (pass == 0) {
+      static bool pool_set[64] = {};
+      if (!pool_set[dev]) {      // keep freed blobs in the stream-ordered pool instead of returning them to the driver
+        cudaMemPool_t pool; unsigned long long thr = ~0ull;
+        if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &thr);
+        cudaGetLastError();
+        pool_set[dev] = true;
+      }
       H->blob_bytes = b.off + 256;
       H->stored_bytes = stored;
       if (cudaMallocAsync(&H->blob, H->blob_bytes, st) != cudaSuccess) { cudaGetLastError(); return fail(JOLT_ENOMEM, "compressed cache of %zu bytes", H->blob_bytes); }
@@ -1144,8 +1150,17 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     ce = cudaEventRecord(gs->fork, st);
     for (int g = 0; g < n_groups && ce == cudaSuccess; ++g) {
       ce = cudaStreamWaitEvent(gs->s[g], gs->fork, 0);
-      if (ce != cudaSuccess) break;
-      if ((rc = run_program(PG[g], (char *)d_tab + tab_off[g], gs->s[g], false))) { cudaDeviceSynchronize(); free_blob(); return rc; }
+      if (ce == cudaSuccess && !PG[g].host.empty())
+        ce = cudaMemcpyAsync((char *)d_tab + tab_off[g], PG[g].host.data(), PG[g].host.size(), cudaMemcpyHostToDevice, gs->s[g]);
+    }
+    // enqueue the groups' steps round-robin, so every side stream has work from the start
+    size_t max_steps = 0;
+    for (int g = 0; g < n_groups; ++g) max_steps = std::max(max_steps, PG[g].steps.size());
+    for (size_t si = 0; si < max_steps && ce == cudaSuccess; ++si)
+      for (int g = 0; g < n_groups; ++g)
+        if (si < PG[g].steps.size()) PG[g].steps[si].run((char *)d_tab + tab_off[g], gs->s[g]);
+    if (ce == cudaSuccess) ce = cudaGetLastError();
+    for (int g = 0; g < n_groups && ce == cudaSuccess; ++g) {
       ce = cudaEventRecord(gs->join[g], gs->s[g]);
       if (ce == cudaSuccess) ce = cudaStreamWaitEvent(st, gs->join[g], 0);
     }
