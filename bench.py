@@ -72,6 +72,27 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def shard_of_rank(rank: int, world: int, base_seed: int):
+    """Weak scaling: cells (and whole sequences) are independent, so rank r compresses its own sequence
+    (generator seed base_seed + r) and no collective touches the data path."""
+    return {"seq": rank, "seed": base_seed + rank}
+
+
+def max_over_ranks(dist, values, device):
+    """Element-wise maximum of per-rank timings (the job is as slow as its slowest rank)."""
+    import torch
+    if dist is None:
+        return list(values)
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_throughput(world: int, bytes_per_rank: int, ms: float) -> float:
+    """Whole-job GB/s: every rank processed bytes_per_rank in ms (max over ranks)."""
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9
+
+
 def cell_work(m, T, d, r_t, r_f, bits, k, q, in_bytes_per_elt):
     """Algorithmic flops / bytes of one cell (split-precision passes do not count)."""
     M = m * T * d
@@ -190,10 +211,11 @@ def main():
     cfg = synth.CONFIGS[args.workload]
     ng = args.groups or cfg.n_groups
     # weak scaling: every rank compresses its own sequence (seed + rank); no data-path collective
-    K, V = synth.make_cache(cfg, seq=rank, device=f"cuda:{local}", n_groups=ng)
+    shard = shard_of_rank(rank, world, cfg.seed)
+    K, V = synth.make_cache(cfg, seq=shard["seq"], device=f"cuda:{local}", n_groups=ng)
     gs = [g * cfg.layers_per_group for g in range(ng + 1)]
     cache_bytes = 2 * K.numel() * 2
-    opts = B.default_options(seed=cfg.seed + rank, power_iters=cfg.power_iters)
+    opts = B.default_options(seed=shard["seed"], power_iters=cfg.power_iters)
     t0 = time.perf_counter()
     plans, planned_bytes = B.jolt_plan(K, V, gs, cache_bytes / cfg.ratio, opts)
     torch.cuda.synchronize()
@@ -242,10 +264,7 @@ def main():
     tc = sum(tc_all) / len(rec)
     td = sum(td_all) / len(rec)
     # decompress stage timing (device events inside the library need a sync, done in step())
-    if dist:
-        t = torch.tensor([tc, td], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        tc, td = t.tolist()
+    tc, td = max_over_ranks(dist, [tc, td], "cuda")
     ms = tc + td
 
     # accuracy of the benchmarked configuration (mean relative Frobenius error over cells)
@@ -279,11 +298,8 @@ def main():
             step_host()
         torch.cuda.synchronize()
         te = (time.perf_counter() - t0) / n_e2e
-        if dist:
-            t = torch.tensor([te], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            te = float(t.item())
-        e2e = {"value": world * cache_bytes / te / 1e9, "unit": UNIT, "h2d_bytes_per_step": cache_bytes,
+        te = max_over_ranks(dist, [te], "cuda")[0]
+        e2e = {"value": job_throughput(world, cache_bytes, te * 1e3), "unit": UNIT, "h2d_bytes_per_step": cache_bytes,
                "d2h_bytes_per_step": cache_bytes, "ms_per_step": te * 1e3}
         del Kh, Vh, Koh, Voh
 
@@ -328,7 +344,7 @@ def main():
                     "frac": ach / pk["tensor"], "traffic": traffic, "algorithmic_flops": fd, "kernel_ms": t_dec,
                     "peak_source": pk["source"] + " (MEASURED_PEAKS.json bf16_tflops, burst)"}
 
-    line = {"metric": METRIC, "value": world * cache_bytes / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+    line = {"metric": METRIC, "value": job_throughput(world, cache_bytes, ms), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f16 operands, f32 accumulate (f64 small solvers)", "data": "synthetic",
             "config": {"workload": f"{cfg.name}: {ng * cfg.layers_per_group} layers / {cfg.layers_per_group} per group, "

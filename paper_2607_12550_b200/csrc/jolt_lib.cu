@@ -933,12 +933,12 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   const bool injected = inUT != nullptr || inUF != nullptr;
   if (injected && (!inUT || !inUF)) return fail(JOLT_EINVAL, "both factor arrays are needed");
   cudaStream_t st = (cudaStream_t)stream;
-  int dev = 0;
-  CU(cudaGetDevice(&dev));
   const int mode = injected ? FM_INJECTED : (o->token_mode == JOLT_TOKEN_EXACT ? FM_EXACT : FM_RANDOMIZED);
   std::vector<CellDesc> cells;
   make_cells(L, K, V, plan, o->oversample, cells);
-  if ((rc = check_plan(cells, plan))) return rc;
+  if ((rc = check_plan(cells, plan))) return rc;       // all argument checks come before the first CUDA call
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
   if (mode == FM_EXACT) {
     for (auto &c : cells) {
       if (c.r_t > 0 && c.T > 1024) return fail(JOLT_EUNSUPPORTED, "exact token factor is built for T <= 1024 (got %d)", c.T);

@@ -144,3 +144,28 @@ def test_budget_below_minimum_reports_ebudget_and_cheapest_plan(B):
     assert st == B.EBUDGET
     assert got == [(16, 16, 0)] * 2
     assert ach == 2 * B.cell_bytes(4, 256, 128, 16, 16, 0)
+
+
+def test_plan_validation_needs_no_gpu(B):
+    K, V = _cpu_cache(L=2, nh=2, T=128)
+    opts = B.default_options()
+    gs = [0, 2]
+    bad_plans = [
+        [(0, 0, 0), (16, 16, 4)],          # a cell that stores nothing
+        [(16, 16, 5), (16, 16, 4)],        # unsupported bit width
+        [(16, 0, 4), (16, 16, 4)],         # r_f out of range
+        [(16, 129, 4), (16, 16, 4)],
+        [(129, 128, 4), (16, 16, 4)],      # r_t > T
+        [(65, 16, 4), (16, 16, 4)],        # r_t > m * r_f  (m = 4)
+        [(-1, 16, 4), (16, 16, 4)],
+    ]
+    for plans in bad_plans:
+        with pytest.raises(B.JoltError) as e:
+            B.jolt_compress(K, V, gs, plans, opts)
+        assert e.value.status == B.EINVAL, plans
+    with pytest.raises(B.JoltError) as e:
+        B.jolt_compress(K, V, gs, [(16, 16, 4)] * 2, B.default_options(power_iters=9))
+    assert e.value.status == B.EINVAL
+    with pytest.raises(B.JoltError) as e:
+        B.jolt_plan(K, V, gs, -5.0, opts)
+    assert e.value.status == B.EINVAL

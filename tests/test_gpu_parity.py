@@ -296,3 +296,25 @@ def test_tensor_core_and_portable_paths_agree(B, synth):
         assert abs(ea - eb) <= REL_ERR * ea
         assert float((a - b).norm() / a.norm()) <= recon_gate(ea)
         assert np.allclose(outs[False][2][i][:32], outs[True][2][i][:32], rtol=1e-4)
+
+
+def test_degenerate_inputs(B):
+    """All-zero cache, a constant cache and the largest legal token rank."""
+    gs = [0, 1]
+    opts = B.default_options(seed=3)
+    Z = torch.zeros(1, 2, 128, 128, dtype=torch.float16, device="cuda")
+    h, Ko, Vo = _roundtrip(B, Z, Z.clone(), gs, [(0, 0, 4), (16, 128, 2)], opts)
+    assert float(Ko.abs().max()) == 0.0 and float(Vo.abs().max()) == 0.0
+    codes = O.unpack_codes(h.component(0, 3).reshape(-1, 16), 4, 128)
+    assert np.all(codes == 8)                       # zero step -> mid code
+    h.free()
+    Cst = torch.full((1, 2, 128, 128), 3.0, dtype=torch.float16, device="cuda")
+    h, Ko, Vo = _roundtrip(B, Cst, Cst.clone(), gs, [(16, 128, 0), (16, 128, 4)], opts)
+    assert float((Ko.float() - 3.0).abs().max()) < 5e-3 and float((Vo.float() - 3.0).abs().max()) < 5e-3
+    h.free()
+    # r_t = T = 128 (full token rank, m * r_f = 256): the backbone alone reproduces the input up to fp16 storage
+    g = torch.Generator().manual_seed(5)
+    X = torch.randn(1, 2, 128, 128, generator=g).to(torch.float16).cuda()
+    h, Ko, Vo = _roundtrip(B, X, X.clone(), gs, [(128, 128, 0), (128, 128, 0)], B.default_options(seed=3, oversample=0))
+    assert float((Ko.float() - X.float()).norm() / X.float().norm()) < 2e-3
+    h.free()
