@@ -16,10 +16,23 @@
 namespace jolt {
 namespace tc {
 
-constexpr int DEC_THREADS = 384;
-constexpr int DEC_P_BYTES = 65536, DEC_H_BYTES = 32768, DEC_BIG_BYTES = 131072;
-constexpr int DEC_NS = 4;
-constexpr int DEC_SMEM_BYTES = DEC_P_BYTES + DEC_H_BYTES + DEC_BIG_BYTES + 1024 + 512;
+// Two variants.  NWG = 2 epilogue warpgroups: any r_t <= 256 (P region 64 KB, 4-stage ring, and for r_t <= 128
+// a staging buffer per warpgroup).  NWG = 4: r_t <= 128 only (P region 32 KB, 2-stage ring, four operand /
+// staging tiles), twice the tiles in flight per SM.  Both use 224 KB of shared memory and one CTA per SM.
+constexpr int DEC_H_BYTES = 32768;
+template <int NWG> struct DecLayout {
+  static constexpr int THREADS = (NWG + 1) * 128;
+  static constexpr int P_BYTES = NWG == 4 ? 32768 : 65536;
+  static constexpr int NS = NWG == 4 ? 2 : 4;                       // ring stages allocated
+  static constexpr int BIG_BYTES = NS * 16384 + NWG * 32768;        // ring + operand tiles (set-up operands first)
+  static constexpr int SMEM_BYTES = P_BYTES + DEC_H_BYTES + BIG_BYTES + 1024 + 512;
+  static constexpr int TMEM_COLS = NWG == 4 ? 512 : 256;
+  // NWG = 2 moves registers from the producer warpgroup to the epilogue ones; NWG = 4 runs every thread at the
+  // launch allocation (96): 20 warps leave no slack in the register file for a blocking re-partition
+  static constexpr bool REPARTITION = NWG == 2;
+  static constexpr int EPI_REGS = 216;
+  static constexpr int PROD_REGS = 56;
+};
 
 template <int BITS>
 struct DecCodes { uint32_t words[BITS > 0 ? 4 * BITS : 1]; uint2 sc; };
@@ -81,7 +94,7 @@ struct DecCtx {
   unsigned char *rbuf, *obuf;
   bool sep_out;
   volatile int *abort_flag;
-  int wg, rit, h, tile0, n_tiles, l, hd;
+  int wg, nwg, rit, h, tile0, n_tiles, l, hd;
   float scale, pre;
 };
 
@@ -93,8 +106,8 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
   const bool tma_out = c.tma_out != 0;
   if (x.wg < x.n_tiles) dec_load_codes<BITS>(c, (long long)x.h * c.T + (x.tile0 + x.wg) * 128 + x.rit, cur);
   const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;
-  for (int i = x.wg; ok && i < x.n_tiles; i += 2) {
-    const int tt = x.tile0 + i, nb = i >> 1;
+  for (int i = x.wg; i < x.n_tiles; i += x.nwg) {
+    const int tt = x.tile0 + i, nb = i / x.nwg;
     const int token = tt * 128 + x.rit;
     long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;
     if (dbg) dbg[0] = clock64();
@@ -104,14 +117,15 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
     }
     if (dbg) dbg[1] = clock64();
     if constexpr (BITS > 0) {
-      dec_unpack_row<BITS>(cur, x.pre, x.rbuf, x.rit);
+      if (ok) dec_unpack_row<BITS>(cur, x.pre, x.rbuf, x.rit);
       fence_proxy_async();
       mbar_arrive(x.bRready);
       if (dbg) dbg[2] = clock64();
-      if (i + 2 < x.n_tiles) dec_load_codes<BITS>(c, (long long)x.h * c.T + (tt + 2) * 128 + x.rit, nxt);   // in flight during the MMA
+      if (i + x.nwg < x.n_tiles) dec_load_codes<BITS>(c, (long long)x.h * c.T + (tt + x.nwg) * 128 + x.rit, nxt);   // in flight during the MMA
     }
-    ok = __all_sync(0xffffffffu, mbar_wait(x.bTfull, nb & 1, x.abort_flag));
-    if (!ok) break;
+    // after a timed-out wait the warp keeps walking the loop (so the warpgroup's named barriers stay in
+    // lockstep) but touches neither TMEM nor the barriers' data again
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(x.bTfull, nb & 1, x.abort_flag));
     if (dbg) dbg[3] = clock64();
     tc_fence_after();
     const long long off = (long long)x.l * c.osl + (long long)x.hd * c.osh + (long long)token * c.ost;
@@ -120,9 +134,10 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
       named_bar_sync(1 + x.wg, 128);
     }
     float va[2][32];
-    tmem_ld32(x.t_acc, va[0]);
+    if (ok) tmem_ld32(x.t_acc, va[0]);
 #pragma unroll
     for (int ch = 0; ch < 4; ++ch) {
+      if (!ok) break;
       tmem_wait_ld();
       if (ch + 1 < 4) tmem_ld32(x.t_acc + (ch + 1) * 32, va[(ch + 1) & 1]);     // next chunk in flight during the conversion
       else { tc_fence_before(); mbar_arrive(x.bTempty); if (dbg) dbg[4] = clock64(); }
@@ -156,7 +171,7 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
       fence_proxy_async();
       named_bar_sync(1 + x.wg, 128);
       if (dbg) dbg[6] = clock64();
-      if (x.rit == 0) {
+      if (x.rit == 0 && ok) {
         tma_store_4d(&c.tmOut, x.s_obuf, 0, tt * 128, x.hd, x.l);
         tma_store_4d(&c.tmOut, x.s_obuf + 16384, 64, tt * 128, x.hd, x.l);
         tma_store_commit();
@@ -169,7 +184,10 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
   return ok;
 }
 
-__global__ void __launch_bounds__(DEC_THREADS, 1) decode_kernel(const BBCell *__restrict__ cells, uint64_t seed) {
+template <int NWG>
+__global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(const BBCell *__restrict__ cells, uint64_t seed) {
+  using LY = DecLayout<NWG>;
+  constexpr int DEC_P_BYTES = LY::P_BYTES, DEC_BIG_BYTES = LY::BIG_BYTES, DEC_NS = LY::NS;
   extern __shared__ unsigned char smem_raw[];
   const BBCell &c = cells[blockIdx.y];
   const int items = c.m * c.items_per_head;
@@ -193,8 +211,8 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_kernel(const BBCell *__
   auto bFull = [=](int s) { return sBar + 24 + 8 * s; };
   auto bEmpty = [=](int s) { return sBar + 56 + 8 * s; };
   auto bTfull = [=](int b) { return sBar + 88 + 8 * b; };
-  auto bTempty = [=](int b) { return sBar + 104 + 8 * b; };
-  auto bRready = [=](int b) { return sBar + 120 + 8 * b; };
+  auto bTempty = [=](int b) { return sBar + 120 + 8 * b; };
+  auto bRready = [=](int b) { return sBar + 152 + 8 * b; };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = warp >> 2;
@@ -202,25 +220,25 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_kernel(const BBCell *__
   const bool has_res = c.bits > 0;
   // r_t <= 128 leaves half of the P region and half of the ring free: each warpgroup then stages its output in a
   // buffer of its own, so a tile's unpack never waits for the previous tile's TMA store to drain
-  const bool sep_out = nkt <= 2;
-  const int ns = sep_out ? 2 : DEC_NS;
+  const bool sep_out = NWG == 2 && nkt <= 2;
+  const int ns = (NWG == 4 || sep_out) ? 2 : DEC_NS;
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
-    mbar_init(bSetup, 1); mbar_init(bPdone, 1); mbar_init(bPready, 256);
+    mbar_init(bSetup, 1); mbar_init(bPdone, 1); mbar_init(bPready, NWG * 128);
     for (int s = 0; s < DEC_NS; ++s) { mbar_init(bFull(s), 1); mbar_init(bEmpty(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bTfull(b), 1); mbar_init(bTempty(b), 128); mbar_init(bRready(b), 128); }
+    for (int b = 0; b < NWG; ++b) { mbar_init(bTfull(b), 1); mbar_init(bTempty(b), 128); mbar_init(bRready(b), 128); }
     fence_barrier_init();
   }
-  if (warp == 8) { tmem_alloc(smem_u32(tmem_slot), BB_TMEM_COLS); tmem_relinquish(); }
+  if (warp == NWG * 4) { tmem_alloc(smem_u32(tmem_slot), LY::TMEM_COLS); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (wg == 2) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-    if (warp == 8 && lane == 0) {
+  if (wg == NWG) {
+    if constexpr (LY::REPARTITION) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(LY::PROD_REGS));
+    if (warp == NWG * 4 && lane == 0) {
       // ---------------- TMA producer
       tma_prefetch_desc(&c.tmUT); tma_prefetch_desc(&c.tmUF); tma_prefetch_desc(&c.tmG);
       mbar_expect_tx(bSetup, (uint32_t)nkf * (16384u + (uint32_t)c.r_t * 128u));
@@ -240,7 +258,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_kernel(const BBCell *__
           tma_load_2d(sRing + s * BB_STAGE_BYTES, &c.tmUT, bFull(s), kb * 64, tt * 128);
         }
       }
-    } else if (warp == 9 && lane == 0) {
+    } else if (warp == NWG * 4 + 1 && lane == 0) {
       // ---------------- MMA issuer (one thread, tiles in order: the ring's phase parities stay unambiguous)
       bool ok = mbar_wait(bSetup, 0, abort_flag);
       if (ok) {
@@ -258,7 +276,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_kernel(const BBCell *__
         const uint32_t idesc = umma_idesc_f16(128, 128, 0, 0);
         int cnt = 0;
         for (int i = 0; ok && i < n_tiles; ++i) {
-          const int b = i & 1, nb = i >> 1;
+          const int b = i % NWG, nb = i / NWG;
           ok = mbar_wait(bTempty(b), (nb & 1) ^ 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
@@ -288,15 +306,15 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_kernel(const BBCell *__
     }
   } else {
     // ---------------- epilogue warpgroups
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    if constexpr (LY::REPARTITION) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(LY::EPI_REGS));
     const int q = warp & 3;
     const int rit = q * 32 + lane;                 // row in tile
     const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
     {  // B operand of the inverse rotation: Hs[f][f'] = s_f * (-1)^popcount(f & f'), fp16, K-major, swizzled
       uint32_t sw[4];
       cell_sign_words(seed, c.cell, sw);
-      const int et = wg * 128 + rit;               // 256 threads, 2048 16-byte chunks
-      for (int ci = et; ci < 2048; ci += 256) {
+      const int et = wg * 128 + rit;               // 2048 16-byte chunks over all epilogue threads
+      for (int ci = et; ci < 2048; ci += NWG * 128) {
         const int f = ci >> 4, chunk = ci & 15;
         const uint32_t sgn = (sw[f >> 5] >> (f & 31)) & 1u;
         uint4 pk;
@@ -313,7 +331,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_kernel(const BBCell *__
     bool ok = __all_sync(0xffffffffu, mbar_wait(bPdone, 0, abort_flag));
     if (ok) {
       tc_fence_after();
-      for (int ch = wg; ch < 2 * nkt; ch += 2) {
+      for (int ch = wg; ch < 2 * nkt; ch += NWG) {
         float v[32];
         tmem_ld32(t_lane + ch * 32, v);
         tmem_wait_ld();
@@ -343,7 +361,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_kernel(const BBCell *__
       x.t_acc = t_lane + wg * 128; x.rbuf = smR + wg * 32768; x.sep_out = sep_out;
       if (sep_out) { x.s_obuf = wg == 0 ? sP + 32768 : sRing + 32768; x.obuf = wg == 0 ? sm + 32768 : sm + DEC_P_BYTES + DEC_H_BYTES + 32768; }
       else { x.s_obuf = sR + wg * 32768; x.obuf = x.rbuf; }
-      x.abort_flag = abort_flag; x.wg = wg; x.rit = rit; x.h = h; x.tile0 = tile0; x.n_tiles = n_tiles;
+      x.abort_flag = abort_flag; x.wg = wg; x.nwg = NWG; x.rit = rit; x.h = h; x.tile0 = tile0; x.n_tiles = n_tiles;
       x.l = h / c.n_heads; x.hd = h - x.l * c.n_heads; x.scale = scale; x.pre = pre;
       switch (c.bits) {
         case 0: dec_tile_loop<0>(c, x); break;
@@ -363,7 +381,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_kernel(const BBCell *__
     while (clock64() - t0 < 2000000) {}
     __syncthreads();
   }
-  if (warp == 8) { tc_fence_after(); tmem_dealloc(tmem_base, BB_TMEM_COLS); }
+  if (warp == NWG * 4) { tc_fence_after(); tmem_dealloc(tmem_base, LY::TMEM_COLS); }
 }
 
 }  // namespace tc
