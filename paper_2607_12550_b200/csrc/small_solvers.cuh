@@ -403,6 +403,9 @@ constexpr int kCholSmemMaxN = 168;
 struct CholSmemTask { const double *G; float *LT; float *invd; int n; int *status; };
 
 __global__ void __launch_bounds__(1024, 1) cholesky_smem_kernel(const CholSmemTask *__restrict__ tasks) {
+  // Left-looking Cholesky by panels of 8 columns: (1) the panel minus the contribution of the finished
+  // columns, one dot product per entry; (2) the 8 x 8 diagonal block, one warp, reciprocal square roots instead
+  // of divisions; (3) the rows below it, one thread per row.  Three barriers per panel.
   const CholSmemTask t = tasks[blockIdx.x];
   const int n = t.n;
   if (n <= 0) return;
@@ -411,29 +414,59 @@ __global__ void __launch_bounds__(1024, 1) cholesky_smem_kernel(const CholSmemTa
   double *A = shd;                       // n x (n+1)
   double *diag0 = A + (size_t)n * ld;    // n
   int *dead = (int *)(diag0 + n);        // n
-  __shared__ double s_piv;
+  __shared__ double ipiv[8];
   const int tid = threadIdx.x, nt = blockDim.x;
   for (int e = tid; e < n * n; e += nt) { const int i = e / n, j = e - i * n; A[i * ld + j] = t.G[e]; }
   __syncthreads();
   for (int i = tid; i < n; i += nt) { diag0[i] = A[i * ld + i]; dead[i] = 0; }
   __syncthreads();
-  for (int j = 0; j < n; ++j) {
-    if (tid == 0) {
-      const double a = A[j * ld + j];
-      if (!(a > 1e-10 * diag0[j]) || !(diag0[j] > 0)) { dead[j] = 1; s_piv = 0.0; A[j * ld + j] = 1.0; }
-      else { s_piv = sqrt(a); A[j * ld + j] = s_piv; }
+  for (int j0 = 0; j0 < n; j0 += 8) {
+    const int w = min(8, n - j0);
+    // (1) panel update
+    for (int e = tid; e < (n - j0) * 8; e += nt) {
+      const int i = j0 + (e >> 3), c = e & 7;
+      if (c < w && i >= j0 + c) {
+        const double *ri = A + i * ld, *rc = A + (j0 + c) * ld;
+        double acc = ri[j0 + c];
+        for (int l = 0; l < j0; ++l) acc = fma(-ri[l], rc[l], acc);
+        A[i * ld + j0 + c] = acc;
+      }
     }
     __syncthreads();
-    const double piv = s_piv;
-    const double ipiv = piv > 0 ? 1.0 / piv : 0.0;
-    for (int i = j + 1 + tid; i < n; i += nt) A[i * ld + j] *= ipiv;
+    // (2) diagonal block, warp 0: lane r owns row j0 + r of the block
+    if (tid < 32) {
+      const int r = tid;
+      for (int c = 0; c < w; ++c) {
+        double rs = 0.0;
+        if (r == c) {
+          const double d = A[(j0 + c) * ld + j0 + c];
+          const bool bad = !(d > 1e-10 * diag0[j0 + c]) || !(diag0[j0 + c] > 0);
+          if (bad) { dead[j0 + c] = 1; A[(j0 + c) * ld + j0 + c] = 1.0; rs = 0.0; }
+          else { rs = rsqrt(d); A[(j0 + c) * ld + j0 + c] = d * rs; }
+          ipiv[c] = rs;
+        }
+        rs = __shfl_sync(0xffffffffu, rs, c);
+        __syncwarp();
+        if (r > c && r < w) {
+          const double v = A[(j0 + r) * ld + j0 + c] * rs;      // column c of the block is final
+          A[(j0 + r) * ld + j0 + c] = v;
+        }
+        __syncwarp();
+        // right-looking inside the block: remaining columns of row r lose the contribution of column c
+        if (r > c && r < w)
+          for (int cc = c + 1; cc <= r; ++cc) A[(j0 + r) * ld + j0 + cc] -= A[(j0 + r) * ld + j0 + c] * A[(j0 + cc) * ld + j0 + c];
+        __syncwarp();
+      }
+    }
     __syncthreads();
-    if (piv > 0) {
-      // trailing update, lower triangle, 32 x 32 thread tiles (no integer division)
-      const int tx = tid & 31, ty = tid >> 5;
-      for (int i = j + 1 + ty; i < n; i += 32) {
-        const double lij = A[i * ld + j];
-        for (int l = j + 1 + tx; l <= i; l += 32) A[i * ld + l] -= lij * A[l * ld + j];
+    // (3) rows below the block
+    for (int i = j0 + w + tid; i < n; i += nt) {
+      double *ri = A + i * ld + j0;
+      for (int c = 0; c < w; ++c) {
+        double acc = ri[c];
+        const double *rc = A + (j0 + c) * ld + j0;
+        for (int l = 0; l < c; ++l) acc = fma(-ri[l], rc[l], acc);
+        ri[c] = acc * ipiv[c];
       }
     }
     __syncthreads();
