@@ -263,22 +263,33 @@ GemmTask mk(const void *A, int ta, long long a_rs, long long a_cs, const void *B
   return t;
 }
 
-void add_gemm(Program &P, int stage, const std::vector<GemmTask> &tasks, bool f64) {
-  if (tasks.empty()) return;
-  int mM = 0, mN = 0;
-  for (auto &t : tasks) { mM = std::max(mM, t.M); mN = std::max(mN, t.N); }
-  if (mM == 0 || mN == 0) return;
-  const size_t off = P.push(tasks);
-  const int n = (int)tasks.size();
-  P.add(stage, [=](char *dev, cudaStream_t s) {
-    const GemmTask *d = (const GemmTask *)(dev + off);
-    for (int z0 = 0; z0 < n; z0 += 32768) {
-      dim3 grid((mN + 63) / 64, (mM + 63) / 64, std::min(32768, n - z0));
-      if (f64) simt_gemm_kernel<double><<<grid, 256, 0, s>>>(d + z0);
-      else simt_gemm_kernel<float><<<grid, 256, 0, s>>>(d + z0);
-      LAUNCHED();
-    }
-  });
+void add_gemm(Program &P, int stage, const std::vector<GemmTask> &all_tasks, bool f64) {
+  if (all_tasks.empty()) return;
+  // one launch per tile-count class: a grid sized for the largest task would start mostly empty CTAs for the rest
+  std::vector<std::pair<long long, std::vector<GemmTask>>> buckets;
+  for (auto &t : all_tasks) {
+    if (t.M <= 0 || t.N <= 0) continue;
+    const long long key = ((long long)((t.M + 63) / 64) << 32) | (long long)((t.N + 63) / 64);
+    size_t b = 0;
+    for (; b < buckets.size(); ++b) if (buckets[b].first == key) break;
+    if (b == buckets.size()) buckets.push_back({key, {}});
+    buckets[b].second.push_back(t);
+  }
+  for (auto &bk : buckets) {
+    const std::vector<GemmTask> &tasks = bk.second;
+    const int tm = (int)(bk.first >> 32), tn = (int)(bk.first & 0xffffffff);
+    const size_t off = P.push(tasks);
+    const int n = (int)tasks.size();
+    P.add(stage, [=](char *dev, cudaStream_t s) {
+      const GemmTask *d = (const GemmTask *)(dev + off);
+      for (int z0 = 0; z0 < n; z0 += 32768) {
+        dim3 grid(tn, tm, std::min(32768, n - z0));
+        if (f64) simt_gemm_kernel<double><<<grid, 256, 0, s>>>(d + z0);
+        else simt_gemm_kernel<float><<<grid, 256, 0, s>>>(d + z0);
+        LAUNCHED();
+      }
+    });
+  }
 }
 
 void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sweeps) {
@@ -496,9 +507,9 @@ void add_tall_gram(Program &P, int stage, const std::vector<TallGram> &jobs) {
     const int n = (int)fastj[cls].size(), nch = fast_chunks[cls];
     P.add(stage, [=](char *dev, cudaStream_t s) {
       const TallGramJob *d = (const TallGramJob *)(dev + off);
-      if (cls == 0) tall_gram_kernel<3><<<dim3(nch, n), 256, 0, s>>>(d);
-      else if (cls == 1) tall_gram_kernel<6><<<dim3(nch, n), 256, 0, s>>>(d);
-      else tall_gram_kernel<9><<<dim3(nch, n), 256, 0, s>>>(d);
+      if (cls == 0) tall_gram_kernel<3><<<dim3(nch, n), 160, 0, s>>>(d);
+      else if (cls == 1) tall_gram_kernel<6><<<dim3(nch, n), 160, 0, s>>>(d);
+      else tall_gram_kernel<9><<<dim3(nch, n), 160, 0, s>>>(d);
       LAUNCHED();
     });
   }
@@ -549,17 +560,21 @@ void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side,
       static bool attr_done = false;
       if (!attr_done) {
         cudaFuncSetAttribute(cholesky_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)chol_smem_bytes(kCholSmemMaxN));
-        cudaFuncSetAttribute(trsm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)trsm_smem_bytes(kCholSmemMaxN));
+        cudaFuncSetAttribute(trsm_rows_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)trsm_smem_bytes(kCholSmemMaxN, 128));
+        cudaFuncSetAttribute(trsm_rows_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemOptIn - 1024));
         attr_done = true;
       }
       const size_t o1 = P.push(chs), o2 = P.push(tj);
       const int n = (int)chs.size();
       int max_rows = 0;
       for (auto &t : tj) max_rows = std::max(max_rows, t.rows);
-      const size_t sh1 = chol_smem_bytes(max_k), sh2 = trsm_smem_bytes(max_k);
+      const bool wide = trsm_smem_bytes(max_k, 256) <= kSmemOptIn - 1024;
+      const size_t sh1 = chol_smem_bytes(max_k), sh2 = trsm_smem_bytes(max_k, wide ? 256 : 128);
       P.add(stage, [=](char *dev, cudaStream_t s) {
         cholesky_smem_kernel<<<n, 1024, sh1, s>>>((const CholSmemTask *)(dev + o1)); LAUNCHED();
-        trsm_rows_kernel<<<dim3((max_rows + 127) / 128, n), 128, sh2, s>>>((const TrsmJob *)(dev + o2)); LAUNCHED();
+        if (wide) trsm_rows_kernel<256><<<dim3((max_rows + 255) / 256, n), 256, sh2, s>>>((const TrsmJob *)(dev + o2));
+        else trsm_rows_kernel<128><<<dim3((max_rows + 127) / 128, n), 128, sh2, s>>>((const TrsmJob *)(dev + o2));
+        LAUNCHED();
       });
     }
   }

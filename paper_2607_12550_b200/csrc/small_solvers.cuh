@@ -484,31 +484,34 @@ inline size_t chol_smem_bytes(int n) { return ((size_t)n * (n + 1) + n) * sizeof
 
 struct TrsmJob { const float *src; float *dst; int rows, k; const float *LT; const float *invd; };
 
-inline size_t trsm_smem_bytes(int k) { const int kp = (k + 3) & ~3; return ((size_t)k * kp + (size_t)kp * 129 + kp) * sizeof(float) + 64; }
+inline size_t trsm_smem_bytes(int k, int rb) { const int kp = (k + 3) & ~3; return ((size_t)k * kp + (size_t)kp * (rb + 1) + kp) * sizeof(float) + 64; }
 
-__global__ void __launch_bounds__(128) trsm_rows_kernel(const TrsmJob *__restrict__ jobs) {
+// RB rows (= threads) per CTA: 256 when the tile fits shared memory, else 128
+template <int RB>
+__global__ void __launch_bounds__(RB) trsm_rows_kernel(const TrsmJob *__restrict__ jobs) {
   const TrsmJob t = jobs[blockIdx.y];
-  const int r0 = blockIdx.x * 128;
+  const int r0 = blockIdx.x * RB;
   if (r0 >= t.rows) return;
   const int k = t.k, kp = (k + 3) & ~3;
+  constexpr int PITCH = RB + 1;
   extern __shared__ float shf[];
   float *LT = shf;                       // k x kp
-  float *sp = LT + (size_t)k * kp;       // kp x 129  (feature j, row r)
-  float *invd = sp + (size_t)kp * 129;   // kp
+  float *sp = LT + (size_t)k * kp;       // kp x PITCH  (feature j, row r)
+  float *invd = sp + (size_t)kp * PITCH; // kp
   const int tid = threadIdx.x;
-  const int nrows = min(128, t.rows - r0);
-  for (int e = tid; e < k * kp; e += 128) LT[e] = t.LT[e];
-  for (int j = tid; j < kp; j += 128) invd[j] = j < k ? t.invd[j] : 0.f;
+  const int nrows = min(RB, t.rows - r0);
+  for (int e = tid; e < k * kp; e += RB) LT[e] = t.LT[e];
+  for (int j = tid; j < kp; j += RB) invd[j] = j < k ? t.invd[j] : 0.f;
   const float *src = t.src + (size_t)r0 * k;
-  for (int e = tid; e < nrows * k; e += 128) { const int r = e / k, j = e - r * k; sp[j * 129 + r] = src[e]; }
-  for (int e = tid; e < (kp - k) * 129; e += 128) sp[k * 129 + e] = 0.f;
+  for (int e = tid; e < nrows * k; e += RB) { const int r = e / k, j = e - r * k; sp[j * PITCH + r] = src[e]; }
+  for (int e = tid; e < (kp - k) * PITCH; e += RB) sp[k * PITCH + e] = 0.f;
   __syncthreads();
   if (tid < nrows) {
     const int r = tid;
     for (int jb = 0; jb < kp; jb += 4) {
-      float a0 = sp[(jb + 0) * 129 + r], a1 = sp[(jb + 1) * 129 + r], a2 = sp[(jb + 2) * 129 + r], a3 = sp[(jb + 3) * 129 + r];
+      float a0 = sp[(jb + 0) * PITCH + r], a1 = sp[(jb + 1) * PITCH + r], a2 = sp[(jb + 2) * PITCH + r], a3 = sp[(jb + 3) * PITCH + r];
       for (int l = 0; l < jb; ++l) {
-        const float x = sp[l * 129 + r];
+        const float x = sp[l * PITCH + r];
         const float4 L4 = *(const float4 *)&LT[l * kp + jb];
         a0 = fmaf(-x, L4.x, a0); a1 = fmaf(-x, L4.y, a1); a2 = fmaf(-x, L4.z, a2); a3 = fmaf(-x, L4.w, a3);
       }
@@ -517,12 +520,12 @@ __global__ void __launch_bounds__(128) trsm_rows_kernel(const TrsmJob *__restric
       a2 = fmaf(-a0, LT[(jb + 0) * kp + jb + 2], a2); a2 = fmaf(-a1, LT[(jb + 1) * kp + jb + 2], a2); a2 *= invd[jb + 2];
       a3 = fmaf(-a0, LT[(jb + 0) * kp + jb + 3], a3); a3 = fmaf(-a1, LT[(jb + 1) * kp + jb + 3], a3);
       a3 = fmaf(-a2, LT[(jb + 2) * kp + jb + 3], a3); a3 *= invd[jb + 3];
-      sp[(jb + 0) * 129 + r] = a0; sp[(jb + 1) * 129 + r] = a1; sp[(jb + 2) * 129 + r] = a2; sp[(jb + 3) * 129 + r] = a3;
+      sp[(jb + 0) * PITCH + r] = a0; sp[(jb + 1) * PITCH + r] = a1; sp[(jb + 2) * PITCH + r] = a2; sp[(jb + 3) * PITCH + r] = a3;
     }
   }
   __syncthreads();
   float *dst = t.dst + (size_t)r0 * k;
-  for (int e = tid; e < nrows * k; e += 128) { const int r = e / k, j = e - r * k; dst[e] = sp[j * 129 + r]; }
+  for (int e = tid; e < nrows * k; e += RB) { const int r = e / k, j = e - r * k; dst[e] = sp[j * PITCH + r]; }
 }
 
 // sum of fp64 partials with a per-job element count
@@ -543,14 +546,22 @@ __global__ void reduce_partials_var_kernel(const ReduceJob *__restrict__ jobs) {
 struct TallGramJob { const float *M; int rows, k, chunk; double *part; };
 
 template <int TI>
-__global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__restrict__ jobs) {
+__global__ void __launch_bounds__(160, 1) tall_gram_kernel(const TallGramJob *__restrict__ jobs) {
+  // G is symmetric: of the 16 x 16 thread tiles only the 136 with ty <= tx are computed (threads 0..135, packed so
+  // that no warp carries idle lanes for the skipped half); the mirror image is written at the end.
   const TallGramJob t = jobs[blockIdx.y];
   const int r_begin = blockIdx.x * t.chunk;
   if (r_begin >= t.rows) return;
   const int r_end = min(t.rows, r_begin + t.chunk);
   constexpr int W = 16 * TI;
   __shared__ double Ms[16][W + 2];
-  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int tid = threadIdx.x;
+  // unrank tid -> (ty, tx), ty <= tx:  tid = tx (tx + 1) / 2 + ty
+  int tx = (int)((sqrtf(8.0f * tid + 1.0f) - 1.0f) * 0.5f);
+  while ((tx + 1) * (tx + 2) / 2 <= tid) ++tx;
+  while (tx * (tx + 1) / 2 > tid) --tx;
+  const int ty = tid - tx * (tx + 1) / 2;
+  const bool active = tid < 136;
   double acc[TI][TI];
 #pragma unroll
   for (int i = 0; i < TI; ++i)
@@ -558,23 +569,26 @@ __global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__
     for (int j = 0; j < TI; ++j) acc[i][j] = 0.0;
   for (int r0 = r_begin; r0 < r_end; r0 += 16) {
     const int nr = min(16, r_end - r0);
-    for (int e = tid; e < 16 * W; e += 256) {
+    for (int e = tid; e < 16 * W; e += 160) {
       const int r = e / W, c = e - r * W;
       Ms[r][c] = (r < nr && c < t.k) ? (double)t.M[(size_t)(r0 + r) * t.k + c] : 0.0;
     }
     __syncthreads();
+    if (active) {
 #pragma unroll 4
-    for (int r = 0; r < 16; ++r) {
-      double a[TI], b[TI];
+      for (int r = 0; r < 16; ++r) {
+        double a[TI], b[TI];
 #pragma unroll
-      for (int i = 0; i < TI; ++i) { a[i] = Ms[r][ty + 16 * i]; b[i] = Ms[r][tx + 16 * i]; }
+        for (int i = 0; i < TI; ++i) { a[i] = Ms[r][ty + 16 * i]; b[i] = Ms[r][tx + 16 * i]; }
 #pragma unroll
-      for (int i = 0; i < TI; ++i)
+        for (int i = 0; i < TI; ++i)
 #pragma unroll
-        for (int j = 0; j < TI; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+          for (int j = 0; j < TI; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+      }
     }
     __syncthreads();
   }
+  if (!active) return;
   double *out = t.part + (size_t)blockIdx.x * t.k * t.k;
 #pragma unroll
   for (int i = 0; i < TI; ++i) {
@@ -583,7 +597,9 @@ __global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__
 #pragma unroll
     for (int j = 0; j < TI; ++j) {
       const int col = tx + 16 * j;
-      if (col < t.k) out[(size_t)row * t.k + col] = acc[i][j];
+      if (col >= t.k) continue;
+      out[(size_t)row * t.k + col] = acc[i][j];
+      if (ty != tx) out[(size_t)col * t.k + row] = acc[i][j];     // (col, row) belongs to the skipped tile (tx, ty)
     }
   }
 }
