@@ -2,11 +2,11 @@
 //
 // The n x n matrix (fp64, padded to a multiple of 32) is cut into 16-wide index blocks.  A round pairs
 // the blocks up (round-robin); for every pair one CTA runs one cyclic Jacobi sweep on the 32 x 32
-// principal submatrix and records the accumulated rotation J (solve kernel); then every 32 x 32 block of
-// A becomes J_a^T blk J_b and every row slab of V is multiplied by J_a (apply kernel).  Rounds are separate
-// launches, so nothing ever waits inside a kernel; all matrices of a call share the launches.  After each
-// sweep a small kernel measures the off-diagonal mass and raises a per-matrix `done` flag that turns the
-// remaining launches into no-ops.
+// principal submatrix and records the accumulated rotation J; then every 32 x 32 block of A becomes
+// J_a^T blk J_b and every row slab of V is multiplied by J_a.  Rounds are separate launches, so nothing
+// ever waits inside a kernel; all matrices of a call share the launches.  The apply half of every launch
+// measures the off-diagonal mass and raises a per-matrix `done` flag that turns the remaining launches
+// into no-ops.
 #pragma once
 #include "small_solvers.cuh"
 
@@ -17,12 +17,12 @@ constexpr int kBJMaxSweeps = 10;
 
 struct BJTask {
   const double *A_in;   // n x n symmetric input (untouched)
-  double *A;            // nP x nP work matrix
+  double *A;            // two nP x nP work matrices (ping-pong between rounds)
   double *V;            // nP x nP, column i = eigenvector i on exit
-  double *J;            // (nbe/2) x 32 x 32 rotations of the current round
-  double *off;          // [4]: off-diagonal mass (accumulator), total mass, last measured off-diagonal mass, sweeps run
-  int *done;            // [1]
-  unsigned *ticket;     // [1] block counter of the check kernel
+  double *J;            // two sets of (nbe/2) x 32 x 32 rotations (current round, next round)
+  double *off;          // [4]: off-diagonal mass (accumulator), total mass, last measured off-diagonal mass, rounds run
+  int *done;            // [4]: see bj_round_kernel
+  unsigned *ticket;     // = done + 1, counter of finished A blocks
   int n, nP, nbe;       // size, padded size (16 * nbe), even number of blocks
   double *w;            // nP scratch (eigenvalues)
   float *U_out; int ld_out, r_out; float *w_out; int w_sqrt;
@@ -45,175 +45,247 @@ __global__ void bj_init_kernel(const BJTask *__restrict__ tasks) {
   if ((threadIdx.x & 31) == 0 && tot != 0.0) atomicAdd(&t.off[1], tot);
 }
 
-// One cyclic sweep of 2x2 rotations on the 32 x 32 principal submatrix of block pair `blockIdx.x`.
-__global__ void __launch_bounds__(256) bj_solve_kernel(const BJTask *__restrict__ tasks, int round, int cross_only) {
-  const BJTask t = tasks[blockIdx.y];
-  if (*t.done || (int)blockIdx.x >= t.nbe / 2) return;
-  int I, Jb;
-  rr_pair(round, blockIdx.x, t.nbe, I, Jb);
-  __shared__ double S[32][33], Jm[32][33];
-  __shared__ double cs_c[16], cs_s[16];
-  __shared__ int pp[16], qq[16];
-  const int tid = threadIdx.x, nP = t.nP;
-  for (int e = tid; e < 1024; e += 256) {
-    const int i = e >> 5, j = e & 31;
-    const int gi = (i < 16 ? I * 16 + i : Jb * 16 + i - 16), gj = (j < 16 ? I * 16 + j : Jb * 16 + j - 16);
-    S[i][j] = t.A[(size_t)gi * nP + gj];
-    Jm[i][j] = (i == j) ? 1.0 : 0.0;
+// One launch per round.  Step s applies the rotations of round s-1 (A: buffer (s-1)&1 -> buffer s&1, V in place)
+// and, in other CTAs of the same launch, already solves round s: a solve CTA recomputes the three 32 x 32 blocks
+// its new pair needs from the old buffer and the old rotations instead of waiting for the apply CTAs, so the
+// two halves never depend on one another inside a launch.  The apply CTAs also sum the off-diagonal mass of
+// what they write; the last of them to finish compares it with the total mass and raises `done`.
+//   done[0] = 1 + step at which convergence was seen (0: not yet), done[1] = ticket, done[2] = final A buffer
+constexpr int kBJTile = 32 * 33;          // padded 32 x 32 fp64 tile
+
+// Programmatic dependent launch: the next round's grid may be scheduled while this one still runs; it does its
+// index arithmetic and then blocks in pdl_wait() until this grid has completed and its writes are visible.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ void bj_pair_rows(int round, int pair, int nbe, int lane, int *dst) {
+  int I, J2; rr_pair(round, pair, nbe, I, J2);
+  dst[lane] = lane < 16 ? I * 16 + lane : J2 * 16 + lane - 16;
+}
+
+__global__ void __launch_bounds__(256) bj_round_kernel(const BJTask *__restrict__ tasks, int step, int n_steps, int gx_apply) {
+  const BJTask t = tasks[blockIdx.y];      // the task table is uploaded before the chain starts
+  // Apply CTAs let the next grid go at once; solve CTAs, the longest, only a few inner rounds before they end,
+  // so the next grid's CTAs do not sit on the SMs (and in the way of other streams' kernels) for a whole round.
+  if ((int)blockIdx.x < gx_apply || step >= n_steps) pdl_launch_dependents();
+  const int nbe = t.nbe, np = nbe / 2, nP = t.nP, R = nbe - 1;
+  const int r_prev = (step + R - 1) % R, r_next = step % R;
+  const size_t asz = (size_t)nP * nP, jsz = (size_t)np * 1024;
+  const int ib = step ? ((step - 1) & 1) : 0, ob = step & 1;
+  const double *Ain = t.A + ib * asz, *Jin = t.J + ib * jsz;
+  double *Aout = t.A + ob * asz, *Jout = t.J + ob * jsz;
+  __shared__ __align__(16) double sm[5840];
+  __shared__ int ra[32], rb[32];
+  __shared__ double red[8];
+  __shared__ int s_ab[4];
+  const int tid = threadIdx.x;
+
+  if ((int)blockIdx.x < gx_apply) {
+    // ---- apply: A block (a, b) <- J_a^T blk J_b (a <= b, mirrored), or V slab (row chunk, pair a) <- slab J_a
+    if (step == 0) return;
+    const int n_ablk = np * (np + 1) / 2, n_vblk = np * (nP / 32);
+    if ((int)blockIdx.x >= n_ablk + n_vblk) return;
+    double (*Ja)[33] = (double (*)[33])sm, (*Jb)[33] = (double (*)[33])(sm + kBJTile);
+    double (*X)[33] = (double (*)[33])(sm + 2 * kBJTile), (*Y)[33] = (double (*)[33])(sm + 3 * kBJTile);
+    const bool is_a = (int)blockIdx.x < n_ablk;
+    int a, b;
+    if (is_a) {
+      const int w = blockIdx.x;
+      b = (int)((sqrtf(8.0f * w + 1.0f) - 1.0f) * 0.5f);
+      while ((b + 1) * (b + 2) / 2 <= w) ++b;
+      while (b * (b + 1) / 2 > w) --b;
+      a = w - b * (b + 1) / 2;
+    }
+    else { const int v = blockIdx.x - n_ablk; a = v / (nP / 32); b = v - a * (nP / 32); }
+    if (tid < 32) {
+      bj_pair_rows(r_prev, a, nbe, tid, ra);
+      if (is_a) bj_pair_rows(r_prev, b, nbe, tid, rb);
+      else rb[tid] = b * 32 + tid;       // V: plain row chunk
+    }
+    __syncthreads();
+    pdl_wait();
+    { const int dn = *(volatile int *)t.done; if (dn != 0 && dn <= step) return; }   // converged in an earlier launch
+    for (int e = tid; e < 1024; e += 256) {
+      const int i = e >> 5, j = e & 31;
+      Ja[i][j] = Jin[(size_t)a * 1024 + e];
+      if (is_a) { Jb[i][j] = Jin[(size_t)b * 1024 + e]; X[i][j] = Ain[(size_t)ra[i] * nP + rb[j]]; }
+      else X[i][j] = t.V[(size_t)rb[i] * nP + ra[j]];      // rows = chunk, cols = pair indices
+    }
+    __syncthreads();
+    const int i0 = (tid >> 5) * 4, j = tid & 31;
+    if (is_a) {
+      double acc[4] = {0, 0, 0, 0};                        // Y = J_a^T X
+      for (int k = 0; k < 32; ++k) {
+        const double x = X[k][j];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) acc[u] += Ja[k][i0 + u] * x;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) Y[i0 + u][j] = acc[u];
+      __syncthreads();
+      double o[4] = {0, 0, 0, 0};                          // out = Y J_b
+      for (int k = 0; k < 32; ++k) {
+        const double x = Jb[k][j];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) o[u] += Y[i0 + u][k] * x;
+      }
+      double mass = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        Aout[(size_t)ra[i0 + u] * nP + rb[j]] = o[u];
+        if (a != b) Aout[(size_t)rb[j] * nP + ra[i0 + u]] = o[u];      // mirrored block
+        if (a != b || i0 + u != j) mass += o[u] * o[u];
+      }
+      if (a != b) mass *= 2.0;
+      for (int o2 = 16; o2; o2 >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, o2);
+      if ((tid & 31) == 0) red[tid >> 5] = mass;
+      __syncthreads();
+      if (tid == 0) {
+        double sum = 0;
+        for (int i = 0; i < 8; ++i) sum += red[i];
+        if (sum != 0.0) atomicAdd(&t.off[0], sum);
+        __threadfence();
+        const unsigned ticket = atomicAdd(t.ticket, 1u);
+        if (ticket == (unsigned)n_ablk - 1) {           // every A block of this step is in
+          __threadfence();
+          const double total_off = atomicAdd(&t.off[0], 0.0);
+          // relative off-diagonal norm 3e-10: above the round-off floor of the 32-term block products on a
+          // rank-deficient matrix (measured 5e-11), far below the fp32 grade of what is read out
+          if (total_off <= 1e-19 * t.off[1]) { t.done[2] = ob; __threadfence(); *(volatile int *)t.done = step + 1; }
+          t.off[2] = total_off;
+          t.off[3] += 1.0;
+          t.off[0] = 0.0;
+          *t.ticket = 0u;
+        }
+      }
+    } else {
+      double o[4] = {0, 0, 0, 0};
+      for (int k = 0; k < 32; ++k) {
+        const double x = Ja[k][j];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) o[u] += X[i0 + u][k] * x;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) t.V[(size_t)rb[i0 + u] * nP + ra[j]] = o[u];
+    }
+    return;
+  }
+
+  // ---- solve round r_next on the matrix as it will be after this step's apply
+  if (step >= n_steps) return;
+  const int x = blockIdx.x - gx_apply;
+  if (x >= np) return;
+  double *S0 = sm, *Jm0 = sm + kBJTile, *S1 = sm + 2 * kBJTile, *Jm1 = sm + 3 * kBJTile;
+  int I, Jn;
+  rr_pair(r_next, x, nbe, I, Jn);
+  if (step == 0) {
+    pdl_wait();
+    for (int e = tid; e < 1024; e += 256) {
+      const int i = e >> 5, j = e & 31;
+      const int gi = (i < 16 ? I * 16 + i : Jn * 16 + i - 16), gj = (j < 16 ? I * 16 + j : Jn * 16 + j - 16);
+      S0[i * 33 + j] = Ain[(size_t)gi * nP + gj];
+      Jm0[i * 33 + j] = (i == j) ? 1.0 : 0.0;
+    }
+  } else {
+    // pairs a, b of the previous round that held blocks I and Jn, and at which half (0 / 16)
+    double *Xaa = sm, *Xab = sm + kBJTile, *Xbb = sm + 2 * kBJTile;
+    double *Jas = sm + 3 * kBJTile, *Jbs = Jas + 32 * 17;            // selected 16 columns of J_a, J_b
+    double *Y1 = Jbs + 32 * 17, *Y2 = Y1 + 16 * 33, *Y3 = Y2 + 16 * 33;
+    if (tid < np) {
+      int p, q; rr_pair(r_prev, tid, nbe, p, q);
+      if (p == I) { s_ab[0] = tid; s_ab[1] = 0; }
+      if (q == I) { s_ab[0] = tid; s_ab[1] = 16; }
+      if (p == Jn) { s_ab[2] = tid; s_ab[3] = 0; }
+      if (q == Jn) { s_ab[2] = tid; s_ab[3] = 16; }
+    }
+    __syncthreads();
+    const int a = s_ab[0], la = s_ab[1], b = s_ab[2], lb = s_ab[3];
+    if (tid < 32) bj_pair_rows(r_prev, a, nbe, tid, ra);
+    else if (tid < 64) bj_pair_rows(r_prev, b, nbe, tid - 32, rb);
+    __syncthreads();
+    pdl_wait();
+    { const int dn = *(volatile int *)t.done; if (dn != 0 && dn <= step) return; }
+    for (int e = tid; e < 1024; e += 256) {
+      const int i = e >> 5, j = e & 31;
+      Xaa[i * 33 + j] = Ain[(size_t)ra[i] * nP + ra[j]];
+      Xab[i * 33 + j] = Ain[(size_t)ra[i] * nP + rb[j]];
+      Xbb[i * 33 + j] = Ain[(size_t)rb[i] * nP + rb[j]];
+    }
+    for (int e = tid; e < 512; e += 256) {
+      const int k = e >> 4, c = e & 15;
+      Jas[k * 17 + c] = Jin[(size_t)a * 1024 + k * 32 + la + c];
+      Jbs[k * 17 + c] = Jin[(size_t)b * 1024 + k * 32 + lb + c];
+    }
+    __syncthreads();
+    {  // Y1 = Jas^T Xaa, Y2 = Jas^T Xab, Y3 = Jbs^T Xbb   (16 x 32 each)
+      const int j = tid & 31, c0 = (tid >> 5) * 2;
+      double y[6] = {0, 0, 0, 0, 0, 0};
+      for (int k = 0; k < 32; ++k) {
+        const double xa = Xaa[k * 33 + j], xb = Xab[k * 33 + j], xc = Xbb[k * 33 + j];
+        const double ja0 = Jas[k * 17 + c0], ja1 = Jas[k * 17 + c0 + 1], jb0 = Jbs[k * 17 + c0], jb1 = Jbs[k * 17 + c0 + 1];
+        y[0] += ja0 * xa; y[1] += ja1 * xa; y[2] += ja0 * xb; y[3] += ja1 * xb; y[4] += jb0 * xc; y[5] += jb1 * xc;
+      }
+      Y1[c0 * 33 + j] = y[0]; Y1[(c0 + 1) * 33 + j] = y[1];
+      Y2[c0 * 33 + j] = y[2]; Y2[(c0 + 1) * 33 + j] = y[3];
+      Y3[c0 * 33 + j] = y[4]; Y3[(c0 + 1) * 33 + j] = y[5];
+    }
+    __syncthreads();
+    {  // S = [Y1 Jas, Y2 Jbs; ., Y3 Jbs]; the X tiles are dead, S0 and Jm0 take their place
+      const int c = tid >> 4, d = tid & 15;
+      double sii = 0, sij = 0, sjj = 0;
+      for (int k = 0; k < 32; ++k) {
+        const double ja = Jas[k * 17 + d], jb = Jbs[k * 17 + d];
+        sii += Y1[c * 33 + k] * ja; sij += Y2[c * 33 + k] * jb; sjj += Y3[c * 33 + k] * jb;
+      }
+      S0[c * 33 + d] = sii; S0[c * 33 + 16 + d] = sij; S0[(16 + d) * 33 + c] = sij; S0[(16 + c) * 33 + 16 + d] = sjj;
+      for (int e = tid; e < 1024; e += 256) Jm0[(e >> 5) * 33 + (e & 31)] = ((e >> 5) == (e & 31)) ? 1.0 : 0.0;
+    }
   }
   __syncthreads();
   // The first round of a sweep rotates every pair of the 32 indices (31 inner rounds), which also covers
   // the pairs inside each 16-block once per sweep; the other rounds rotate the 16 x 16 cross pairs only.
+  // Every thread owns one 2 x 2 pair-block (pair a rows, pair b columns) and derives both rotations itself;
+  // S and the accumulated J ping-pong between two buffers, so an inner round needs one barrier.
+  const bool cross_only = r_next > 0;
   const int n_inner = cross_only ? 16 : 31;
+  const int a = tid >> 4, b = tid & 15;
+  double *Sc = S0, *Sn = S1, *Jc = Jm0, *Jx = Jm1;
   for (int r = 0; r < n_inner; ++r) {
-    if (tid < 16) {
-      int p, q;
-      if (cross_only) { p = tid; q = 16 + ((tid + r) & 15); } else rr_pair(r, tid, 32, p, q);
-      double c = 1.0, s = 0.0;
-      const double apq = S[p][q], app = S[p][p], aqq = S[q][q];
-      jacobi_cs_fast(app, aqq, apq, c, s);
-      pp[tid] = p; qq[tid] = q; cs_c[tid] = c; cs_s[tid] = s;
+    if (r == n_inner - 4) pdl_launch_dependents();
+    int pa, qa, pb, qb;
+    if (cross_only) { pa = a; qa = 16 + ((a + r) & 15); pb = b; qb = 16 + ((b + r) & 15); }
+    else { rr_pair(r, a, 32, pa, qa); rr_pair(r, b, 32, pb, qb); }
+    double ca, sa, cb, sb;
+    jacobi_cs_fast(Sc[pa * 33 + pa], Sc[qa * 33 + qa], Sc[pa * 33 + qa], ca, sa);
+    jacobi_cs_fast(Sc[pb * 33 + pb], Sc[qb * 33 + qb], Sc[pb * 33 + qb], cb, sb);
+    const double x_pp = Sc[pa * 33 + pb], x_pq = Sc[pa * 33 + qb], x_qp = Sc[qa * 33 + pb], x_qq = Sc[qa * 33 + qb];
+    const double r_pp = ca * x_pp - sa * x_qp, r_pq = ca * x_pq - sa * x_qq;
+    const double r_qp = sa * x_pp + ca * x_qp, r_qq = sa * x_pq + ca * x_qq;
+    Sn[pa * 33 + pb] = cb * r_pp - sb * r_pq; Sn[pa * 33 + qb] = sb * r_pp + cb * r_pq;
+    Sn[qa * 33 + pb] = cb * r_qp - sb * r_qq; Sn[qa * 33 + qb] = sb * r_qp + cb * r_qq;
+#pragma unroll
+    for (int u = 0; u < 32; u += 16) {       // J <- J Rot: columns pa, qa, rows b and b + 16
+      const int row = b + u;
+      const double vp = Jc[row * 33 + pa], vq = Jc[row * 33 + qa];
+      Jx[row * 33 + pa] = ca * vp - sa * vq;
+      Jx[row * 33 + qa] = sa * vp + ca * vq;
     }
     __syncthreads();
-    {  // 16 x 16 pair-blocks, one per thread
-      const int a = tid >> 4, b = tid & 15;
-      const int pa = pp[a], qa = qq[a], pb = pp[b], qb = qq[b];
-      const double ca = cs_c[a], sa = cs_s[a], cb = cs_c[b], sb = cs_s[b];
-      const double x_pp = S[pa][pb], x_pq = S[pa][qb], x_qp = S[qa][pb], x_qq = S[qa][qb];
-      const double r_pp = ca * x_pp - sa * x_qp, r_pq = ca * x_pq - sa * x_qq;
-      const double r_qp = sa * x_pp + ca * x_qp, r_qq = sa * x_pq + ca * x_qq;
-      S[pa][pb] = cb * r_pp - sb * r_pq; S[pa][qb] = sb * r_pp + cb * r_pq;
-      S[qa][pb] = cb * r_qp - sb * r_qq; S[qa][qb] = sb * r_qp + cb * r_qq;
-      // Jm <- Jm * Jrot : columns p, q of pair (tid >> 5 ... ) two items per thread
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const int it = tid + u * 256, pr = it >> 5, row = it & 31;
-        const int p = pp[pr], q = qq[pr];
-        const double c = cs_c[pr], s = cs_s[pr];
-        const double vp = Jm[row][p], vq = Jm[row][q];
-        Jm[row][p] = c * vp - s * vq;
-        Jm[row][q] = s * vp + c * vq;
-      }
-    }
-    __syncthreads();
+    double *tmp = Sc; Sc = Sn; Sn = tmp;
+    tmp = Jc; Jc = Jx; Jx = tmp;
   }
-  double *Jo = t.J + (size_t)blockIdx.x * 1024;
-  for (int e = tid; e < 1024; e += 256) Jo[e] = Jm[e >> 5][e & 31];
+  for (int e = tid; e < 1024; e += 256) Jout[(size_t)x * 1024 + e] = Jc[(e >> 5) * 33 + (e & 31)];
 }
 
-// blockIdx.x < np*np : A block (a, b) <- J_a^T blk J_b ;  otherwise V slab (a, row chunk) <- slab J_a
-__global__ void __launch_bounds__(256) bj_apply_kernel(const BJTask *__restrict__ tasks, int round) {
-  const BJTask t = tasks[blockIdx.y];
-  if (*t.done) return;
-  const int np = t.nbe / 2, nP = t.nP;
-  const int n_ablk = np * (np + 1) / 2, n_vblk = np * (nP / 32);       // A is symmetric: blocks a <= b only
-  if ((int)blockIdx.x >= n_ablk + n_vblk) return;
-  __shared__ double Ja[32][33], Jb[32][33], X[32][33], Y[32][33];
-  __shared__ int ra[32], rb[32];
-  const int tid = threadIdx.x;
-  const bool is_a = (int)blockIdx.x < n_ablk;
-  int a, b;
-  if (is_a) {
-    const int w = blockIdx.x;
-    b = (int)((sqrtf(8.0f * w + 1.0f) - 1.0f) * 0.5f);
-    while ((b + 1) * (b + 2) / 2 <= w) ++b;
-    while (b * (b + 1) / 2 > w) --b;
-    a = w - b * (b + 1) / 2;
-  }
-  else { const int v = blockIdx.x - n_ablk; a = v / (nP / 32); b = v - a * (nP / 32); }
-  if (tid < 32) {
-    int I, J2; rr_pair(round, a, t.nbe, I, J2);
-    ra[tid] = tid < 16 ? I * 16 + tid : J2 * 16 + tid - 16;
-    if (is_a) { rr_pair(round, b, t.nbe, I, J2); rb[tid] = tid < 16 ? I * 16 + tid : J2 * 16 + tid - 16; }
-    else rb[tid] = b * 32 + tid;       // V: plain row chunk
-  }
-  __syncthreads();
-  const double *Jga = t.J + (size_t)a * 1024;
-  for (int e = tid; e < 1024; e += 256) {
-    const int i = e >> 5, j = e & 31;
-    Ja[i][j] = Jga[e];
-    if (is_a) { Jb[i][j] = t.J[(size_t)b * 1024 + e]; X[i][j] = t.A[(size_t)ra[i] * nP + rb[j]]; }
-    else X[i][j] = t.V[(size_t)rb[i] * nP + ra[j]];      // rows = chunk, cols = pair indices
-  }
-  __syncthreads();
-  const int i0 = (tid >> 5) * 4, j = tid & 31;
-  if (is_a) {
-    // Y = J_a^T X
-    double acc[4] = {0, 0, 0, 0};
-    for (int k = 0; k < 32; ++k) {
-      const double x = X[k][j];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) acc[u] += Ja[k][i0 + u] * x;
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) Y[i0 + u][j] = acc[u];
-    __syncthreads();
-    // out = Y J_b
-    double o[4] = {0, 0, 0, 0};
-    for (int k = 0; k < 32; ++k) {
-      const double x = Jb[k][j];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) o[u] += Y[i0 + u][k] * x;
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      t.A[(size_t)ra[i0 + u] * nP + rb[j]] = o[u];
-      if (a != b) t.A[(size_t)rb[j] * nP + ra[i0 + u]] = o[u];      // mirrored block
-    }
-  } else {
-    double o[4] = {0, 0, 0, 0};
-    for (int k = 0; k < 32; ++k) {
-      const double x = Ja[k][j];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) o[u] += X[i0 + u][k] * x;
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) t.V[(size_t)rb[i0 + u] * nP + ra[j]] = o[u];
-  }
-}
-
-// Off-diagonal mass after a sweep; the last block to finish (ticket counter) compares it with the total mass,
-// raises `done` and resets the accumulators: one launch per sweep.
-__global__ void bj_check_kernel(const BJTask *__restrict__ tasks) {
-  const BJTask t = tasks[blockIdx.y];
-  if (*t.done) return;
-  double off = 0;
-  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < t.nP * t.nP; e += gridDim.x * blockDim.x) {
-    const int i = e / t.nP, j = e - i * t.nP;
-    if (i != j) { const double v = t.A[e]; off += v * v; }
-  }
-  for (int o = 16; o; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
-  __shared__ double red[8];
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = off;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double s = 0;
-    for (int i = 0; i < (int)blockDim.x / 32; ++i) s += red[i];
-    if (s != 0.0) atomicAdd(&t.off[0], s);
-    __threadfence();
-    const unsigned ticket = atomicAdd(t.ticket, 1u);
-    if (ticket == gridDim.x - 1) {           // every block's contribution is in
-      __threadfence();
-      const double total_off = atomicAdd(&t.off[0], 0.0);
-      // relative off-diagonal norm 3e-10: above the round-off floor of the 32-term block products on a
-      // rank-deficient matrix (measured 5e-11), far below the fp32 grade of what is read out
-      if (total_off <= 1e-19 * t.off[1]) *t.done = 1;
-      t.off[2] = total_off;
-      t.off[3] += 1.0;
-      t.off[0] = 0.0;
-      *t.ticket = 0u;
-    }
-  }
-}
-
-__global__ void __launch_bounds__(256) bj_finish_kernel(const BJTask *__restrict__ tasks) {
+__global__ void __launch_bounds__(256) bj_finish_kernel(const BJTask *__restrict__ tasks, int last_buf) {
   const BJTask t = tasks[blockIdx.x];
   const int n = t.n, nP = t.nP, tid = threadIdx.x, nt = blockDim.x;
+  const double *Af = t.A + (size_t)(*t.done ? t.done[2] : last_buf) * nP * nP;
   __shared__ int rk[2048];
   // not converged to the tight threshold after the last sweep: still accepted when the off-diagonal norm is below
   // 1e-7 of the matrix norm (fp32 grade); flagged otherwise
   if (tid == 0 && !*t.done && t.status && !(t.off[2] <= 1e-14 * t.off[1])) atomicOr(t.status, 1);
-  for (int i = tid; i < n; i += nt) t.w[i] = t.A[(size_t)i * nP + i];
+  for (int i = tid; i < n; i += nt) t.w[i] = Af[(size_t)i * nP + i];
   __syncthreads();
   for (int i = tid; i < n; i += nt) {
     const double wi = t.w[i];

@@ -319,23 +319,20 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
     std::vector<BJTask> copy = bj;
     P.add(stage, [=](char *dev, cudaStream_t s) {
       const BJTask *d = (const BJTask *)(dev + off);
-      for (auto &b : copy) { cudaMemsetAsync(b.off, 0, 4 * sizeof(double), s); cudaMemsetAsync(b.done, 0, 2 * sizeof(int), s); }
+      for (auto &b : copy) { cudaMemsetAsync(b.off, 0, 4 * sizeof(double), s); cudaMemsetAsync(b.done, 0, 4 * sizeof(int), s); }
       bj_init_kernel<<<dim3(64, n), 256, 0, s>>>(d); LAUNCHED();
       const int np = max_nbe / 2;
       const int gx = np * (np + 1) / 2 + np * (max_nP / 32);
-      const int max_sweeps = bj_sweeps;
-      for (int sw = 0; sw < max_sweeps; ++sw) {
-        for (int r = 0; r < max_nbe - 1; ++r) {
-          bj_solve_kernel<<<dim3(np, n), 256, 0, s>>>(d, r, r > 0 ? 1 : 0); LAUNCHED();
-          bj_apply_kernel<<<dim3(gx, n), 256, 0, s>>>(d, r); LAUNCHED();
-        }
-        bj_check_kernel<<<dim3(16, n), 256, 0, s>>>(d); LAUNCHED();
-      }
-      bj_finish_kernel<<<n, 256, 0, s>>>(d); LAUNCHED();
+      const int n_steps = bj_sweeps * (max_nbe - 1);
+      cudaLaunchAttribute pdl; pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization; pdl.val.programmaticStreamSerializationAllowed = 1;
+      cudaLaunchConfig_t cfg; memset(&cfg, 0, sizeof cfg);
+      cfg.gridDim = dim3(gx + np, n); cfg.blockDim = dim3(256); cfg.stream = s; cfg.attrs = &pdl; cfg.numAttrs = 1;
+      for (int step = 0; step <= n_steps; ++step) { cudaLaunchKernelEx(&cfg, bj_round_kernel, d, step, n_steps, gx); LAUNCHED(); }
+      bj_finish_kernel<<<n, 256, 0, s>>>(d, n_steps & 1); LAUNCHED();
       if (getenv("JOLT_DEBUG_EIG")) {
         cudaStreamSynchronize(s);
         for (auto &b : copy) { double o[4]; int dn; cudaMemcpy(o, b.off, 32, cudaMemcpyDeviceToHost); cudaMemcpy(&dn, b.done, 4, cudaMemcpyDeviceToHost);
-          fprintf(stderr, "[jolt] bj n=%d nbe=%d last_off=%g total=%g done=%d sweeps=%g\n", b.n, b.nbe, o[2], o[1], dn, o[3]); }
+          fprintf(stderr, "[jolt] bj n=%d nbe=%d last_off=%g total=%g done=%d rounds=%g\n", b.n, b.nbe, o[2], o[1], dn, o[3]); }
       }
     });
   }
@@ -434,8 +431,8 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
       {
         const size_t nmax = std::max<size_t>(kD, mode == FM_EXACT ? T : k);
         const size_t nbe = (((nmax + kBJBlock - 1) / kBJBlock) + 1) & ~(size_t)1, nP = nbe * kBJBlock;
-        w.bjA = b.take<double>(nP * nP); w.bjV = b.take<double>(nP * nP); w.bjJ = b.take<double>(nbe / 2 * 1024);
-        w.bjOff = b.take<double>(4); w.bjDone = b.take<int>(2);
+        w.bjA = b.take<double>(2 * nP * nP); w.bjV = b.take<double>(nP * nP); w.bjJ = b.take<double>(2 * (nbe / 2) * 1024);
+        w.bjOff = b.take<double>(4); w.bjDone = b.take<int>(4);
       }
       w.gram_part = b.take<double>((size_t)c.m * kD * kD);
       w.C = b.take<double>(kD * kD); w.Cv = b.take<double>(kD * kD); w.Cw = b.take<double>(kD);
@@ -507,9 +504,9 @@ void add_tall_gram(Program &P, int stage, const std::vector<TallGram> &jobs) {
     const int n = (int)fastj[cls].size(), nch = fast_chunks[cls];
     P.add(stage, [=](char *dev, cudaStream_t s) {
       const TallGramJob *d = (const TallGramJob *)(dev + off);
-      if (cls == 0) tall_gram_kernel<3><<<dim3(nch, n), 160, 0, s>>>(d);
-      else if (cls == 1) tall_gram_kernel<6><<<dim3(nch, n), 160, 0, s>>>(d);
-      else tall_gram_kernel<9><<<dim3(nch, n), 160, 0, s>>>(d);
+      if (cls == 0) tall_gram_kernel<3><<<dim3(nch, n), 256, 0, s>>>(d);
+      else if (cls == 1) tall_gram_kernel<6><<<dim3(nch, n), 256, 0, s>>>(d);
+      else tall_gram_kernel<9><<<dim3(nch, n), 256, 0, s>>>(d);
       LAUNCHED();
     });
   }

@@ -546,22 +546,14 @@ __global__ void reduce_partials_var_kernel(const ReduceJob *__restrict__ jobs) {
 struct TallGramJob { const float *M; int rows, k, chunk; double *part; };
 
 template <int TI>
-__global__ void __launch_bounds__(160, 1) tall_gram_kernel(const TallGramJob *__restrict__ jobs) {
-  // G is symmetric: of the 16 x 16 thread tiles only the 136 with ty <= tx are computed (threads 0..135, packed so
-  // that no warp carries idle lanes for the skipped half); the mirror image is written at the end.
+__global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__restrict__ jobs) {
   const TallGramJob t = jobs[blockIdx.y];
   const int r_begin = blockIdx.x * t.chunk;
   if (r_begin >= t.rows) return;
   const int r_end = min(t.rows, r_begin + t.chunk);
   constexpr int W = 16 * TI;
   __shared__ double Ms[16][W + 2];
-  const int tid = threadIdx.x;
-  // unrank tid -> (ty, tx), ty <= tx:  tid = tx (tx + 1) / 2 + ty
-  int tx = (int)((sqrtf(8.0f * tid + 1.0f) - 1.0f) * 0.5f);
-  while ((tx + 1) * (tx + 2) / 2 <= tid) ++tx;
-  while (tx * (tx + 1) / 2 > tid) --tx;
-  const int ty = tid - tx * (tx + 1) / 2;
-  const bool active = tid < 136;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   double acc[TI][TI];
 #pragma unroll
   for (int i = 0; i < TI; ++i)
@@ -569,26 +561,23 @@ __global__ void __launch_bounds__(160, 1) tall_gram_kernel(const TallGramJob *__
     for (int j = 0; j < TI; ++j) acc[i][j] = 0.0;
   for (int r0 = r_begin; r0 < r_end; r0 += 16) {
     const int nr = min(16, r_end - r0);
-    for (int e = tid; e < 16 * W; e += 160) {
+    for (int e = tid; e < 16 * W; e += 256) {
       const int r = e / W, c = e - r * W;
       Ms[r][c] = (r < nr && c < t.k) ? (double)t.M[(size_t)(r0 + r) * t.k + c] : 0.0;
     }
     __syncthreads();
-    if (active) {
 #pragma unroll 4
-      for (int r = 0; r < 16; ++r) {
-        double a[TI], b[TI];
+    for (int r = 0; r < 16; ++r) {
+      double a[TI], b[TI];
 #pragma unroll
-        for (int i = 0; i < TI; ++i) { a[i] = Ms[r][ty + 16 * i]; b[i] = Ms[r][tx + 16 * i]; }
+      for (int i = 0; i < TI; ++i) { a[i] = Ms[r][ty + 16 * i]; b[i] = Ms[r][tx + 16 * i]; }
 #pragma unroll
-        for (int i = 0; i < TI; ++i)
+      for (int i = 0; i < TI; ++i)
 #pragma unroll
-          for (int j = 0; j < TI; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
-      }
+        for (int j = 0; j < TI; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
     }
     __syncthreads();
   }
-  if (!active) return;
   double *out = t.part + (size_t)blockIdx.x * t.k * t.k;
 #pragma unroll
   for (int i = 0; i < TI; ++i) {
@@ -597,9 +586,7 @@ __global__ void __launch_bounds__(160, 1) tall_gram_kernel(const TallGramJob *__
 #pragma unroll
     for (int j = 0; j < TI; ++j) {
       const int col = tx + 16 * j;
-      if (col >= t.k) continue;
-      out[(size_t)row * t.k + col] = acc[i][j];
-      if (ty != tx) out[(size_t)col * t.k + row] = acc[i][j];     // (col, row) belongs to the skipped tile (tx, ty)
+      if (col < t.k) out[(size_t)row * t.k + col] = acc[i][j];
     }
   }
 }
