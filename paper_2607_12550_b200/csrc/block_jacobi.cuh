@@ -63,7 +63,67 @@ __device__ __forceinline__ void bj_pair_rows(int round, int pair, int nbe, int l
   dst[lane] = lane < 16 ? I * 16 + lane : J2 * 16 + lane - 16;
 }
 
-__global__ void __launch_bounds__(256) bj_round_kernel(const BJTask *__restrict__ tasks, int step, int n_steps, int gx_apply) {
+constexpr int kBJThreads = 288;           // 8 working warps + the warp that accumulates J
+
+__device__ __forceinline__ void bj_bar(int id, int nthreads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory"); }
+
+// pair `i` of inner round `r`: cross pairs (one index from each 16-block) or the circle method on all 32 indices
+template <bool CROSS>
+__device__ __forceinline__ void bj_inner_pair(int r, int i, int &p, int &q) {
+  if (CROSS) { p = i; q = 16 + ((i + r) & 15); }
+  else rr_pair(r, i, 32, p, q);
+}
+
+template <bool CROSS>
+__device__ __forceinline__ void bj_inner(double *S, double2 (*cs_buf)[16], double *Jo, int tid) {
+  constexpr int NR = CROSS ? 16 : 31;
+  if (tid >= 256) {
+    const int lane = tid & 31;
+    double Jr[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) Jr[j] = (j == lane) ? 1.0 : 0.0;
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+      if (r == NR - 4) pdl_launch_dependents();
+      bj_bar(2, kBJThreads);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        int p, q; bj_inner_pair<CROSS>(r, i, p, q);
+        const double2 cs = cs_buf[r & 1][i];
+        const double vp = Jr[p], vq = Jr[q];
+        Jr[p] = cs.x * vp - cs.y * vq;
+        Jr[q] = cs.y * vp + cs.x * vq;
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 32; ++j) Jo[lane * 32 + j] = Jr[j];
+    return;
+  }
+  const int a = tid >> 4, b = tid & 15;
+  for (int r = 0; r < NR; ++r) {
+    if (r == NR - 4) pdl_launch_dependents();
+    if (tid < 16) {
+      int p, q; bj_inner_pair<CROSS>(r, tid, p, q);
+      double c, s;
+      jacobi_cs_fast(S[p * 33 + p], S[q * 33 + q], S[p * 33 + q], c, s);
+      cs_buf[r & 1][tid] = make_double2(c, s);
+    }
+    bj_bar(2, kBJThreads);
+    int pa, qa, pb, qb;
+    bj_inner_pair<CROSS>(r, a, pa, qa);
+    bj_inner_pair<CROSS>(r, b, pb, qb);
+    const double2 ra = cs_buf[r & 1][a], rb = cs_buf[r & 1][b];
+    const double ca = ra.x, sa = ra.y, cb = rb.x, sb = rb.y;
+    const double x_pp = S[pa * 33 + pb], x_pq = S[pa * 33 + qb], x_qp = S[qa * 33 + pb], x_qq = S[qa * 33 + qb];
+    const double r_pp = ca * x_pp - sa * x_qp, r_pq = ca * x_pq - sa * x_qq;
+    const double r_qp = sa * x_pp + ca * x_qp, r_qq = sa * x_pq + ca * x_qq;
+    S[pa * 33 + pb] = cb * r_pp - sb * r_pq; S[pa * 33 + qb] = sb * r_pp + cb * r_pq;
+    S[qa * 33 + pb] = cb * r_qp - sb * r_qq; S[qa * 33 + qb] = sb * r_qp + cb * r_qq;
+    bj_bar(1, 256);
+  }
+}
+
+__global__ void __launch_bounds__(kBJThreads) bj_round_kernel(const BJTask *__restrict__ tasks, int step, int n_steps, int gx_apply) {
   const BJTask t = tasks[blockIdx.y];      // the task table is uploaded before the chain starts
   // Apply CTAs let the next grid go at once; solve CTAs, the longest, only a few inner rounds before they end,
   // so the next grid's CTAs do not sit on the SMs (and in the way of other streams' kernels) for a whole round.
@@ -78,11 +138,12 @@ __global__ void __launch_bounds__(256) bj_round_kernel(const BJTask *__restrict_
   __shared__ int ra[32], rb[32];
   __shared__ double red[8];
   __shared__ int s_ab[4];
+  __shared__ double2 cs_buf[2][16];
   const int tid = threadIdx.x;
 
   if ((int)blockIdx.x < gx_apply) {
     // ---- apply: A block (a, b) <- J_a^T blk J_b (a <= b, mirrored), or V slab (row chunk, pair a) <- slab J_a
-    if (step == 0) return;
+    if (step == 0 || tid >= 256) return;          // the ninth warp only works in solve CTAs
     const int n_ablk = np * (np + 1) / 2, n_vblk = np * (nP / 32);
     if ((int)blockIdx.x >= n_ablk + n_vblk) return;
     double (*Ja)[33] = (double (*)[33])sm, (*Jb)[33] = (double (*)[33])(sm + kBJTile);
@@ -102,7 +163,7 @@ __global__ void __launch_bounds__(256) bj_round_kernel(const BJTask *__restrict_
       if (is_a) bj_pair_rows(r_prev, b, nbe, tid, rb);
       else rb[tid] = b * 32 + tid;       // V: plain row chunk
     }
-    __syncthreads();
+    bj_bar(1, 256);
     pdl_wait();
     { const int dn = *(volatile int *)t.done; if (dn != 0 && dn <= step) return; }   // converged in an earlier launch
     for (int e = tid; e < 1024; e += 256) {
@@ -111,7 +172,7 @@ __global__ void __launch_bounds__(256) bj_round_kernel(const BJTask *__restrict_
       if (is_a) { Jb[i][j] = Jin[(size_t)b * 1024 + e]; X[i][j] = Ain[(size_t)ra[i] * nP + rb[j]]; }
       else X[i][j] = t.V[(size_t)rb[i] * nP + ra[j]];      // rows = chunk, cols = pair indices
     }
-    __syncthreads();
+    bj_bar(1, 256);
     const int i0 = (tid >> 5) * 4, j = tid & 31;
     if (is_a) {
       double acc[4] = {0, 0, 0, 0};                        // Y = J_a^T X
@@ -122,7 +183,7 @@ __global__ void __launch_bounds__(256) bj_round_kernel(const BJTask *__restrict_
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) Y[i0 + u][j] = acc[u];
-      __syncthreads();
+      bj_bar(1, 256);
       double o[4] = {0, 0, 0, 0};                          // out = Y J_b
       for (int k = 0; k < 32; ++k) {
         const double x = Jb[k][j];
@@ -139,7 +200,7 @@ __global__ void __launch_bounds__(256) bj_round_kernel(const BJTask *__restrict_
       if (a != b) mass *= 2.0;
       for (int o2 = 16; o2; o2 >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, o2);
       if ((tid & 31) == 0) red[tid >> 5] = mass;
-      __syncthreads();
+      bj_bar(1, 256);
       if (tid == 0) {
         double sum = 0;
         for (int i = 0; i < 8; ++i) sum += red[i];
@@ -175,22 +236,15 @@ __global__ void __launch_bounds__(256) bj_round_kernel(const BJTask *__restrict_
   if (step >= n_steps) return;
   const int x = blockIdx.x - gx_apply;
   if (x >= np) return;
-  double *S0 = sm, *Jm0 = sm + kBJTile, *S1 = sm + 2 * kBJTile, *Jm1 = sm + 3 * kBJTile;
+  const int warp = tid >> 5;
+  double *S = sm;                                   // 32 x 33, overlays the first X tile once that is dead
   int I, Jn;
   rr_pair(r_next, x, nbe, I, Jn);
-  if (step == 0) {
-    pdl_wait();
-    for (int e = tid; e < 1024; e += 256) {
-      const int i = e >> 5, j = e & 31;
-      const int gi = (i < 16 ? I * 16 + i : Jn * 16 + i - 16), gj = (j < 16 ? I * 16 + j : Jn * 16 + j - 16);
-      S0[i * 33 + j] = Ain[(size_t)gi * nP + gj];
-      Jm0[i * 33 + j] = (i == j) ? 1.0 : 0.0;
-    }
-  } else {
+  double *Xaa = sm, *Xab = sm + kBJTile, *Xbb = sm + 2 * kBJTile;
+  double *Jas = sm + 3 * kBJTile, *Jbs = Jas + 32 * 17;            // selected 16 columns of J_a, J_b
+  double *Y1 = Jbs + 32 * 17, *Y2 = Y1 + 16 * 33, *Y3 = Y2 + 16 * 33;
+  if (step > 0 && warp < 8) {
     // pairs a, b of the previous round that held blocks I and Jn, and at which half (0 / 16)
-    double *Xaa = sm, *Xab = sm + kBJTile, *Xbb = sm + 2 * kBJTile;
-    double *Jas = sm + 3 * kBJTile, *Jbs = Jas + 32 * 17;            // selected 16 columns of J_a, J_b
-    double *Y1 = Jbs + 32 * 17, *Y2 = Y1 + 16 * 33, *Y3 = Y2 + 16 * 33;
     if (tid < np) {
       int p, q; rr_pair(r_prev, tid, nbe, p, q);
       if (p == I) { s_ab[0] = tid; s_ab[1] = 0; }
@@ -198,83 +252,66 @@ __global__ void __launch_bounds__(256) bj_round_kernel(const BJTask *__restrict_
       if (p == Jn) { s_ab[2] = tid; s_ab[3] = 0; }
       if (q == Jn) { s_ab[2] = tid; s_ab[3] = 16; }
     }
-    __syncthreads();
-    const int a = s_ab[0], la = s_ab[1], b = s_ab[2], lb = s_ab[3];
-    if (tid < 32) bj_pair_rows(r_prev, a, nbe, tid, ra);
-    else if (tid < 64) bj_pair_rows(r_prev, b, nbe, tid - 32, rb);
-    __syncthreads();
-    pdl_wait();
-    { const int dn = *(volatile int *)t.done; if (dn != 0 && dn <= step) return; }
-    for (int e = tid; e < 1024; e += 256) {
-      const int i = e >> 5, j = e & 31;
-      Xaa[i * 33 + j] = Ain[(size_t)ra[i] * nP + ra[j]];
-      Xab[i * 33 + j] = Ain[(size_t)ra[i] * nP + rb[j]];
-      Xbb[i * 33 + j] = Ain[(size_t)rb[i] * nP + rb[j]];
-    }
-    for (int e = tid; e < 512; e += 256) {
-      const int k = e >> 4, c = e & 15;
-      Jas[k * 17 + c] = Jin[(size_t)a * 1024 + k * 32 + la + c];
-      Jbs[k * 17 + c] = Jin[(size_t)b * 1024 + k * 32 + lb + c];
-    }
-    __syncthreads();
-    {  // Y1 = Jas^T Xaa, Y2 = Jas^T Xab, Y3 = Jbs^T Xbb   (16 x 32 each)
-      const int j = tid & 31, c0 = (tid >> 5) * 2;
-      double y[6] = {0, 0, 0, 0, 0, 0};
-      for (int k = 0; k < 32; ++k) {
-        const double xa = Xaa[k * 33 + j], xb = Xab[k * 33 + j], xc = Xbb[k * 33 + j];
-        const double ja0 = Jas[k * 17 + c0], ja1 = Jas[k * 17 + c0 + 1], jb0 = Jbs[k * 17 + c0], jb1 = Jbs[k * 17 + c0 + 1];
-        y[0] += ja0 * xa; y[1] += ja1 * xa; y[2] += ja0 * xb; y[3] += ja1 * xb; y[4] += jb0 * xc; y[5] += jb1 * xc;
+    bj_bar(1, 256);
+    if (tid < 32) bj_pair_rows(r_prev, s_ab[0], nbe, tid, ra);
+    else if (tid < 64) bj_pair_rows(r_prev, s_ab[2], nbe, tid - 32, rb);
+    bj_bar(1, 256);
+  }
+  pdl_wait();
+  { const int dn = *(volatile int *)t.done; if (dn != 0 && dn <= step) return; }   // converged in an earlier launch
+  if (warp < 8) {
+    if (step == 0) {
+      for (int e = tid; e < 1024; e += 256) {
+        const int i = e >> 5, j = e & 31;
+        const int gi = (i < 16 ? I * 16 + i : Jn * 16 + i - 16), gj = (j < 16 ? I * 16 + j : Jn * 16 + j - 16);
+        S[i * 33 + j] = Ain[(size_t)gi * nP + gj];
       }
-      Y1[c0 * 33 + j] = y[0]; Y1[(c0 + 1) * 33 + j] = y[1];
-      Y2[c0 * 33 + j] = y[2]; Y2[(c0 + 1) * 33 + j] = y[3];
-      Y3[c0 * 33 + j] = y[4]; Y3[(c0 + 1) * 33 + j] = y[5];
-    }
-    __syncthreads();
-    {  // S = [Y1 Jas, Y2 Jbs; ., Y3 Jbs]; the X tiles are dead, S0 and Jm0 take their place
-      const int c = tid >> 4, d = tid & 15;
-      double sii = 0, sij = 0, sjj = 0;
-      for (int k = 0; k < 32; ++k) {
-        const double ja = Jas[k * 17 + d], jb = Jbs[k * 17 + d];
-        sii += Y1[c * 33 + k] * ja; sij += Y2[c * 33 + k] * jb; sjj += Y3[c * 33 + k] * jb;
+    } else {
+      const int a = s_ab[0], la = s_ab[1], b = s_ab[2], lb = s_ab[3];
+      for (int e = tid; e < 1024; e += 256) {
+        const int i = e >> 5, j = e & 31;
+        Xaa[i * 33 + j] = Ain[(size_t)ra[i] * nP + ra[j]];
+        Xab[i * 33 + j] = Ain[(size_t)ra[i] * nP + rb[j]];
+        Xbb[i * 33 + j] = Ain[(size_t)rb[i] * nP + rb[j]];
       }
-      S0[c * 33 + d] = sii; S0[c * 33 + 16 + d] = sij; S0[(16 + d) * 33 + c] = sij; S0[(16 + c) * 33 + 16 + d] = sjj;
-      for (int e = tid; e < 1024; e += 256) Jm0[(e >> 5) * 33 + (e & 31)] = ((e >> 5) == (e & 31)) ? 1.0 : 0.0;
+      for (int e = tid; e < 512; e += 256) {
+        const int k = e >> 4, c = e & 15;
+        Jas[k * 17 + c] = Jin[(size_t)a * 1024 + k * 32 + la + c];
+        Jbs[k * 17 + c] = Jin[(size_t)b * 1024 + k * 32 + lb + c];
+      }
+      bj_bar(1, 256);
+      {  // Y1 = Jas^T Xaa, Y2 = Jas^T Xab, Y3 = Jbs^T Xbb   (16 x 32 each)
+        const int j = tid & 31, c0 = (tid >> 5) * 2;
+        double y[6] = {0, 0, 0, 0, 0, 0};
+        for (int k = 0; k < 32; ++k) {
+          const double xa = Xaa[k * 33 + j], xb = Xab[k * 33 + j], xc = Xbb[k * 33 + j];
+          const double ja0 = Jas[k * 17 + c0], ja1 = Jas[k * 17 + c0 + 1], jb0 = Jbs[k * 17 + c0], jb1 = Jbs[k * 17 + c0 + 1];
+          y[0] += ja0 * xa; y[1] += ja1 * xa; y[2] += ja0 * xb; y[3] += ja1 * xb; y[4] += jb0 * xc; y[5] += jb1 * xc;
+        }
+        Y1[c0 * 33 + j] = y[0]; Y1[(c0 + 1) * 33 + j] = y[1];
+        Y2[c0 * 33 + j] = y[2]; Y2[(c0 + 1) * 33 + j] = y[3];
+        Y3[c0 * 33 + j] = y[4]; Y3[(c0 + 1) * 33 + j] = y[5];
+      }
+      bj_bar(1, 256);
+      {  // S = [Y1 Jas, Y2 Jbs; ., Y3 Jbs]; the X tiles are dead, S takes the place of the first
+        const int c = tid >> 4, d = tid & 15;
+        double sii = 0, sij = 0, sjj = 0;
+        for (int k = 0; k < 32; ++k) {
+          const double ja = Jas[k * 17 + d], jb = Jbs[k * 17 + d];
+          sii += Y1[c * 33 + k] * ja; sij += Y2[c * 33 + k] * jb; sjj += Y3[c * 33 + k] * jb;
+        }
+        S[c * 33 + d] = sii; S[c * 33 + 16 + d] = sij; S[(16 + d) * 33 + c] = sij; S[(16 + c) * 33 + 16 + d] = sjj;
+      }
     }
   }
   __syncthreads();
   // The first round of a sweep rotates every pair of the 32 indices (31 inner rounds), which also covers
   // the pairs inside each 16-block once per sweep; the other rounds rotate the 16 x 16 cross pairs only.
-  // Every thread owns one 2 x 2 pair-block (pair a rows, pair b columns) and derives both rotations itself;
-  // S and the accumulated J ping-pong between two buffers, so an inner round needs one barrier.
-  const bool cross_only = r_next > 0;
-  const int n_inner = cross_only ? 16 : 31;
-  const int a = tid >> 4, b = tid & 15;
-  double *Sc = S0, *Sn = S1, *Jc = Jm0, *Jx = Jm1;
-  for (int r = 0; r < n_inner; ++r) {
-    if (r == n_inner - 4) pdl_launch_dependents();
-    int pa, qa, pb, qb;
-    if (cross_only) { pa = a; qa = 16 + ((a + r) & 15); pb = b; qb = 16 + ((b + r) & 15); }
-    else { rr_pair(r, a, 32, pa, qa); rr_pair(r, b, 32, pb, qb); }
-    double ca, sa, cb, sb;
-    jacobi_cs_fast(Sc[pa * 33 + pa], Sc[qa * 33 + qa], Sc[pa * 33 + qa], ca, sa);
-    jacobi_cs_fast(Sc[pb * 33 + pb], Sc[qb * 33 + qb], Sc[pb * 33 + qb], cb, sb);
-    const double x_pp = Sc[pa * 33 + pb], x_pq = Sc[pa * 33 + qb], x_qp = Sc[qa * 33 + pb], x_qq = Sc[qa * 33 + qb];
-    const double r_pp = ca * x_pp - sa * x_qp, r_pq = ca * x_pq - sa * x_qq;
-    const double r_qp = sa * x_pp + ca * x_qp, r_qq = sa * x_pq + ca * x_qq;
-    Sn[pa * 33 + pb] = cb * r_pp - sb * r_pq; Sn[pa * 33 + qb] = sb * r_pp + cb * r_pq;
-    Sn[qa * 33 + pb] = cb * r_qp - sb * r_qq; Sn[qa * 33 + qb] = sb * r_qp + cb * r_qq;
-#pragma unroll
-    for (int u = 0; u < 32; u += 16) {       // J <- J Rot: columns pa, qa, rows b and b + 16
-      const int row = b + u;
-      const double vp = Jc[row * 33 + pa], vq = Jc[row * 33 + qa];
-      Jx[row * 33 + pa] = ca * vp - sa * vq;
-      Jx[row * 33 + qa] = sa * vp + ca * vq;
-    }
-    __syncthreads();
-    double *tmp = Sc; Sc = Sn; Sn = tmp;
-    tmp = Jc; Jc = Jx; Jx = tmp;
-  }
-  for (int e = tid; e < 1024; e += 256) Jout[(size_t)x * 1024 + e] = Jc[(e >> 5) * 33 + (e & 31)];
+  // An inner round: 16 threads derive the 16 rotations from the pivots (barrier A), then each of 256 threads
+  // updates its own 2 x 2 pair-block of S in place (barrier B).  The ninth warp keeps the accumulated rotation
+  // J in registers, one row per lane, and applies each round's rotations as they are published.
+  if (r_next > 0) bj_inner<true>(S, cs_buf, Jout + (size_t)x * 1024, tid);
+  else bj_inner<false>(S, cs_buf, Jout + (size_t)x * 1024, tid);
 }
 
 __global__ void __launch_bounds__(256) bj_finish_kernel(const BJTask *__restrict__ tasks, int last_buf) {

@@ -326,7 +326,7 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
       const int n_steps = bj_sweeps * (max_nbe - 1);
       cudaLaunchAttribute pdl; pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization; pdl.val.programmaticStreamSerializationAllowed = 1;
       cudaLaunchConfig_t cfg; memset(&cfg, 0, sizeof cfg);
-      cfg.gridDim = dim3(gx + np, n); cfg.blockDim = dim3(256); cfg.stream = s; cfg.attrs = &pdl; cfg.numAttrs = 1;
+      cfg.gridDim = dim3(gx + np, n); cfg.blockDim = dim3(kBJThreads); cfg.stream = s; cfg.attrs = &pdl; cfg.numAttrs = 1;
       for (int step = 0; step <= n_steps; ++step) { cudaLaunchKernelEx(&cfg, bj_round_kernel, d, step, n_steps, gx); LAUNCHED(); }
       bj_finish_kernel<<<n, 256, 0, s>>>(d, n_steps & 1); LAUNCHED();
       if (getenv("JOLT_DEBUG_EIG")) {
@@ -568,7 +568,7 @@ void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side,
       const bool wide = trsm_smem_bytes(max_k, 256) <= kSmemOptIn - 1024;
       const size_t sh1 = chol_smem_bytes(max_k), sh2 = trsm_smem_bytes(max_k, wide ? 256 : 128);
       P.add(stage, [=](char *dev, cudaStream_t s) {
-        cholesky_smem_kernel<<<n, 1024, sh1, s>>>((const CholSmemTask *)(dev + o1)); LAUNCHED();
+        cholesky_smem_kernel<<<n, 512, sh1, s>>>((const CholSmemTask *)(dev + o1)); LAUNCHED();
         if (wide) trsm_rows_kernel<256><<<dim3((max_rows + 255) / 256, n), 256, sh2, s>>>((const TrsmJob *)(dev + o2));
         else trsm_rows_kernel<128><<<dim3((max_rows + 127) / 128, n), 128, sh2, s>>>((const TrsmJob *)(dev + o2));
         LAUNCHED();
@@ -818,7 +818,8 @@ int run_program(Program &P, char *d_tables, cudaStream_t st, bool timed = true) 
 }
 
 // Side streams on which independent groups of cells run their (latency-bound) factor stages concurrently.
-constexpr int kMaxGroups = 4;
+constexpr int kMaxGroups = 8;
+constexpr int kDefaultGroups = 4;
 struct GroupStreams { bool have = false; cudaStream_t s[kMaxGroups]; cudaEvent_t fork, join[kMaxGroups]; };
 GroupStreams g_groups[64];
 GroupStreams *group_streams(int dev) {
@@ -835,21 +836,24 @@ GroupStreams *group_streams(int dev) {
   return &g;
 }
 
-// Cells whose factor stages may run side by side: cells that need the feature eigen-solve (longest chain)
-// form group 0, the others are dealt round-robin.
+// Cells whose factor stages may run side by side.  Cells that need the feature eigen-solve (the longest chain)
+// and the others never share a group.
 int assign_groups(const std::vector<CellWork> &ws, std::vector<int> &group) {
-  int want = kMaxGroups;
+  int want = kDefaultGroups;
   if (const char *e = getenv("JOLT_GROUPS")) want = std::max(1, std::min(kMaxGroups, atoi(e)));
   group.assign(ws.size(), -1);
   int n_active = 0, n_long = 0;
   for (auto &w : ws) if (w.active) { ++n_active; if (!w.ufI) ++n_long; }
   if (n_active < 2 || want == 1) { for (size_t i = 0; i < ws.size(); ++i) if (ws[i].active) group[i] = 0; return n_active ? 1 : 0; }
-  const int first = (n_long > 0 && n_long < n_active) ? 1 : 0;
-  int rr = 0, used = 0;
+  // long cells share the first groups, short cells the rest, each in proportion to their number
+  int g_long = 0;
+  if (n_long > 0 && n_long < n_active) g_long = std::max(1, std::min(want - 1, (want * n_long + n_active / 2) / n_active));
+  else if (n_long == n_active) g_long = want;
+  int rl = 0, rs = 0, used = 0;
   for (size_t i = 0; i < ws.size(); ++i) {
     if (!ws[i].active) continue;
-    if (first == 1 && !ws[i].ufI) group[i] = 0;
-    else { group[i] = first + rr % (want - first); ++rr; }
+    if (!ws[i].ufI && g_long > 0) { group[i] = rl % g_long; ++rl; }
+    else { group[i] = g_long % want + rs % std::max(1, want - g_long % want); ++rs; }
     used = std::max(used, group[i] + 1);
   }
   return used;
@@ -1169,9 +1173,29 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     // enqueue the groups' steps round-robin, so every side stream has work from the start
     size_t max_steps = 0;
     for (int g = 0; g < n_groups; ++g) max_steps = std::max(max_steps, PG[g].steps.size());
+    const bool tl = getenv("JOLT_DEBUG_TIMELINE") != nullptr;      // per-group stage boundaries, printed after the call
+    struct TL { int g, stage; cudaEvent_t ev; };
+    std::vector<TL> tls;
+    cudaEvent_t tl0 = nullptr;
+    if (tl) { cudaEventCreate(&tl0); cudaEventRecord(tl0, st); }
     for (size_t si = 0; si < max_steps && ce == cudaSuccess; ++si)
       for (int g = 0; g < n_groups; ++g)
-        if (si < PG[g].steps.size()) PG[g].steps[si].run((char *)d_tab + tab_off[g], gs->s[g]);
+        if (si < PG[g].steps.size()) {
+          PG[g].steps[si].run((char *)d_tab + tab_off[g], gs->s[g]);
+          if (tl && (si + 1 == PG[g].steps.size() || PG[g].steps[si + 1].stage != PG[g].steps[si].stage)) {
+            TL t{g, PG[g].steps[si].stage, nullptr}; cudaEventCreate(&t.ev); cudaEventRecord(t.ev, gs->s[g]); tls.push_back(t);
+          }
+        }
+    if (tl) {
+      cudaDeviceSynchronize();
+      for (int g = 0; g < n_groups; ++g) {
+        fprintf(stderr, "[jolt] group %d:", g);
+        for (auto &t : tls) if (t.g == g) { float ms = 0; cudaEventElapsedTime(&ms, tl0, t.ev); fprintf(stderr, " %s@%.2f", kStageNames[t.stage], ms); }
+        fprintf(stderr, "\n");
+      }
+      for (auto &t : tls) cudaEventDestroy(t.ev);
+      cudaEventDestroy(tl0);
+    }
     if (ce == cudaSuccess) ce = cudaGetLastError();
     for (int g = 0; g < n_groups && ce == cudaSuccess; ++g) {
       ce = cudaEventRecord(gs->join[g], gs->s[g]);

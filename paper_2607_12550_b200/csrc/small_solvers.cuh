@@ -400,12 +400,25 @@ __global__ void __launch_bounds__(1024) cholesky_inv_kernel(const CholTask *__re
 // (0 for a dead pivot).  trsm_rows_kernel then solves  dst_row * L^T = src_row  for 128 rows per CTA.
 constexpr int kCholSmemMaxN = 168;
 
+// 1 / sqrt(d) for d > 0: single-precision seed and two Newton steps in fp64 (full accuracy), the library routine
+// outside the single-precision range
+__device__ __forceinline__ double rsqrt_pos(double d) {
+  if (!(d > 1e-30 && d < 1e30)) return rsqrt(d);
+  const double h = 0.5 * d;
+  double y = (double)rsqrtf((float)d);
+  y = y * fma(-h * y, y, 1.5);
+  y = y * fma(-h * y, y, 1.5);
+  return y;
+}
+
+
 struct CholSmemTask { const double *G; float *LT; float *invd; int n; int *status; };
 
-__global__ void __launch_bounds__(1024, 1) cholesky_smem_kernel(const CholSmemTask *__restrict__ tasks) {
-  // Left-looking Cholesky by panels of 8 columns: (1) the panel minus the contribution of the finished
-  // columns, one dot product per entry; (2) the 8 x 8 diagonal block, one warp, reciprocal square roots instead
-  // of divisions; (3) the rows below it, one thread per row.  Three barriers per panel.
+__global__ void __launch_bounds__(512, 1) cholesky_smem_kernel(const CholSmemTask *__restrict__ tasks) {
+  // Left-looking Cholesky by panels of 8 columns.  (1) The panel loses the contribution of the finished columns,
+  // one dot product per entry on four independent accumulators.  (2) Warp 0 factors the 8 x 8 diagonal block in
+  // registers (shuffles, reciprocal square roots instead of divisions).  (3) The rows below are solved against the
+  // block, one thread per row.  Three barriers per panel.
   const CholSmemTask t = tasks[blockIdx.x];
   const int n = t.n;
   if (n <= 0) return;
@@ -414,59 +427,85 @@ __global__ void __launch_bounds__(1024, 1) cholesky_smem_kernel(const CholSmemTa
   double *A = shd;                       // n x (n+1)
   double *diag0 = A + (size_t)n * ld;    // n
   int *dead = (int *)(diag0 + n);        // n
+  __shared__ double blk[8][9];           // the factored diagonal block
   __shared__ double ipiv[8];
   const int tid = threadIdx.x, nt = blockDim.x;
-  for (int e = tid; e < n * n; e += nt) { const int i = e / n, j = e - i * n; A[i * ld + j] = t.G[e]; }
+  for (int e0 = tid; e0 < n * n; e0 += nt * 8) {
+    double v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { const int e = e0 + u * nt; v[u] = e < n * n ? t.G[e] : 0.0; }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { const int e = e0 + u * nt; if (e < n * n) { const int i = e / n, j = e - i * n; A[i * ld + j] = v[u]; } }
+  }
   __syncthreads();
   for (int i = tid; i < n; i += nt) { diag0[i] = A[i * ld + i]; dead[i] = 0; }
   __syncthreads();
   for (int j0 = 0; j0 < n; j0 += 8) {
     const int w = min(8, n - j0);
-    // (1) panel update
+    // (1) panel minus the contribution of the finished columns (lower part of the diagonal block included)
     for (int e = tid; e < (n - j0) * 8; e += nt) {
       const int i = j0 + (e >> 3), c = e & 7;
-      if (c < w && i >= j0 + c) {
-        const double *ri = A + i * ld, *rc = A + (j0 + c) * ld;
-        double acc = ri[j0 + c];
-        for (int l = 0; l < j0; ++l) acc = fma(-ri[l], rc[l], acc);
-        A[i * ld + j0 + c] = acc;
+      if (c >= w || j0 + c > i) continue;
+      const double *ri = A + i * ld, *rc = A + (j0 + c) * ld;
+      double a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+      int l = 0;
+      for (; l + 4 <= j0; l += 4) {
+        a0 = fma(ri[l], rc[l], a0); a1 = fma(ri[l + 1], rc[l + 1], a1);
+        a2 = fma(ri[l + 2], rc[l + 2], a2); a3 = fma(ri[l + 3], rc[l + 3], a3);
       }
+      for (; l < j0; ++l) a0 = fma(ri[l], rc[l], a0);
+      A[i * ld + j0 + c] -= (a0 + a1) + (a2 + a3);
     }
     __syncthreads();
-    // (2) diagonal block, warp 0: lane r owns row j0 + r of the block
+    // (2) the 8 x 8 diagonal block in the registers of warp 0: lane r holds row r
     if (tid < 32) {
-      const int r = tid;
-      for (int c = 0; c < w; ++c) {
-        double rs = 0.0;
-        if (r == c) {
-          const double d = A[(j0 + c) * ld + j0 + c];
-          const bool bad = !(d > 1e-10 * diag0[j0 + c]) || !(diag0[j0 + c] > 0);
-          if (bad) { dead[j0 + c] = 1; A[(j0 + c) * ld + j0 + c] = 1.0; rs = 0.0; }
-          else { rs = rsqrt(d); A[(j0 + c) * ld + j0 + c] = d * rs; }
-          ipiv[c] = rs;
+      const int r = tid & 7, i = j0 + r;
+      double row[8], piv[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) row[c] = (r < w && c <= r) ? A[i * ld + j0 + c] : 0.0;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        piv[c] = 0.0;
+        if (c < w) {
+          const double d = __shfl_sync(0xffffffffu, row[c], c);
+          const double dg = diag0[j0 + c];
+          const bool bad = !(d > 1e-10 * dg) || !(dg > 0);
+          const double rs = bad ? 0.0 : rsqrt_pos(d);
+          if (r == c) row[c] = bad ? 1.0 : d * rs; else row[c] *= rs;
+          if (tid == c && bad) dead[j0 + c] = 1;
+          piv[c] = rs;
+#pragma unroll
+          for (int cc = c + 1; cc < 8; ++cc) {
+            const double lcc = __shfl_sync(0xffffffffu, row[c], cc);     // L[cc][c]
+            if (r >= cc) row[cc] = fma(-row[c], lcc, row[cc]);
+          }
         }
-        rs = __shfl_sync(0xffffffffu, rs, c);
-        __syncwarp();
-        if (r > c && r < w) {
-          const double v = A[(j0 + r) * ld + j0 + c] * rs;      // column c of the block is final
-          A[(j0 + r) * ld + j0 + c] = v;
-        }
-        __syncwarp();
-        // right-looking inside the block: remaining columns of row r lose the contribution of column c
-        if (r > c && r < w)
-          for (int cc = c + 1; cc <= r; ++cc) A[(j0 + r) * ld + j0 + cc] -= A[(j0 + r) * ld + j0 + c] * A[(j0 + cc) * ld + j0 + c];
-        __syncwarp();
+      }
+      if (tid < w) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) if (c <= r) { A[i * ld + j0 + c] = row[c]; blk[r][c] = row[c]; }
+      }
+      if (tid == 0) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) ipiv[c] = piv[c];
       }
     }
     __syncthreads();
-    // (3) rows below the block
+    // (3) rows below the block: x_c = (p_c - sum_{l<c} x_l L[c][l]) / L[c][c]
     for (int i = j0 + w + tid; i < n; i += nt) {
       double *ri = A + i * ld + j0;
-      for (int c = 0; c < w; ++c) {
-        double acc = ri[c];
-        const double *rc = A + (j0 + c) * ld + j0;
-        for (int l = 0; l < c; ++l) acc = fma(-ri[l], rc[l], acc);
-        ri[c] = acc * ipiv[c];
+      double x[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) x[c] = c < w ? ri[c] : 0.0;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        if (c < w) {
+          double acc = x[c];
+#pragma unroll
+          for (int l = 0; l < c; ++l) acc = fma(-x[l], blk[c][l], acc);
+          x[c] = acc * ipiv[c];
+          ri[c] = x[c];
+        }
       }
     }
     __syncthreads();
@@ -500,20 +539,67 @@ __global__ void __launch_bounds__(RB) trsm_rows_kernel(const TrsmJob *__restrict
   float *invd = sp + (size_t)kp * PITCH; // kp
   const int tid = threadIdx.x;
   const int nrows = min(RB, t.rows - r0);
-  for (int e = tid; e < k * kp; e += RB) LT[e] = t.LT[e];
+  // staging loops read eight elements into registers before the first shared-memory store, so that the global
+  // loads of a trip are in flight together
+  {
+    const float4 *g4 = (const float4 *)t.LT;
+    float4 *s4 = (float4 *)LT;
+    const int n4 = k * kp / 4;
+    for (int e0 = tid; e0 < n4; e0 += RB * 4) {
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { const int e = e0 + u * RB; if (e < n4) v[u] = g4[e]; }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { const int e = e0 + u * RB; if (e < n4) s4[e] = v[u]; }
+    }
+  }
   for (int j = tid; j < kp; j += RB) invd[j] = j < k ? t.invd[j] : 0.f;
   const float *src = t.src + (size_t)r0 * k;
-  for (int e = tid; e < nrows * k; e += RB) { const int r = e / k, j = e - r * k; sp[j * PITCH + r] = src[e]; }
+  const int tot = nrows * k;
+  if ((((size_t)r0 * k) & 3) == 0) {          // the row block starts on a 16-byte boundary: vector loads
+    const float4 *src4 = (const float4 *)src;
+    const int tot4 = tot >> 2;
+    for (int e0 = tid; e0 < tot4; e0 += RB * 8) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const int e = e0 + u * RB; if (e < tot4) v[u] = src4[e]; }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = e0 + u * RB;
+        if (e < tot4) {
+          int r = (4 * e) / k, j = 4 * e - r * k;
+          const float vv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+          for (int c = 0; c < 4; ++c) { sp[j * PITCH + r] = vv[c]; if (++j == k) { j = 0; ++r; } }
+        }
+      }
+    }
+    for (int e = (tot4 << 2) + tid; e < tot; e += RB) { const int r = e / k, j = e - r * k; sp[j * PITCH + r] = src[e]; }
+  } else {
+    for (int e0 = tid; e0 < tot; e0 += RB * 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const int e = e0 + u * RB; v[u] = e < tot ? src[e] : 0.f; }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const int e = e0 + u * RB; if (e < tot) { const int r = e / k, j = e - r * k; sp[j * PITCH + r] = v[u]; } }
+    }
+  }
   for (int e = tid; e < (kp - k) * PITCH; e += RB) sp[k * PITCH + e] = 0.f;
   __syncthreads();
   if (tid < nrows) {
     const int r = tid;
     for (int jb = 0; jb < kp; jb += 4) {
       float a0 = sp[(jb + 0) * PITCH + r], a1 = sp[(jb + 1) * PITCH + r], a2 = sp[(jb + 2) * PITCH + r], a3 = sp[(jb + 3) * PITCH + r];
-      for (int l = 0; l < jb; ++l) {
-        const float x = sp[l * PITCH + r];
-        const float4 L4 = *(const float4 *)&LT[l * kp + jb];
-        a0 = fmaf(-x, L4.x, a0); a1 = fmaf(-x, L4.y, a1); a2 = fmaf(-x, L4.z, a2); a3 = fmaf(-x, L4.w, a3);
+      // jb is a multiple of 4: four finished columns per trip, all loads of a trip issued before its 16 FMAs
+#pragma unroll 2
+      for (int l = 0; l < jb; l += 4) {
+        float x[4]; float4 L4[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { x[u] = sp[(l + u) * PITCH + r]; L4[u] = *(const float4 *)&LT[(l + u) * kp + jb]; }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          a0 = fmaf(-x[u], L4[u].x, a0); a1 = fmaf(-x[u], L4[u].y, a1); a2 = fmaf(-x[u], L4[u].z, a2); a3 = fmaf(-x[u], L4[u].w, a3);
+        }
       }
       a0 *= invd[jb];
       a1 = fmaf(-a0, LT[(jb + 0) * kp + jb + 1], a1); a1 *= invd[jb + 1];
