@@ -176,6 +176,9 @@ def main():
     ap.add_argument("--impl", default="jolt", choices=["jolt", "reference"])
     ap.add_argument("--workload", default="c1")
     ap.add_argument("--groups", type=int, default=0, help="limit the number of layer groups (profiling captures)")
+    ap.add_argument("--token-mode", default="randomized", choices=["randomized", "exact"],
+                    help="token-mode solver; exact at T > 1024 is the converged block iteration")
+    ap.add_argument("--ratio", type=float, default=0.0, help="compression ratio of the byte budget (default: the workload's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--portable", action="store_true", help="portable SIMT kernels only")
@@ -215,9 +218,11 @@ def main():
     K, V = synth.make_cache(cfg, seq=shard["seq"], device=f"cuda:{local}", n_groups=ng)
     gs = [g * cfg.layers_per_group for g in range(ng + 1)]
     cache_bytes = 2 * K.numel() * 2
-    opts = B.default_options(seed=shard["seed"], power_iters=cfg.power_iters)
+    ratio = args.ratio or cfg.ratio
+    opts = B.default_options(seed=shard["seed"], power_iters=cfg.power_iters,
+                             token_mode=B.TOKEN_EXACT if args.token_mode == "exact" else B.TOKEN_RANDOMIZED)
     t0 = time.perf_counter()
-    plans, planned_bytes = B.jolt_plan(K, V, gs, cache_bytes / cfg.ratio, opts)
+    plans, planned_bytes = B.jolt_plan(K, V, gs, cache_bytes / ratio, opts)
     torch.cuda.synchronize()
     plan_ms = (time.perf_counter() - t0) * 1e3
     Ko, Vo = torch.empty_like(K), torch.empty_like(V)
@@ -348,9 +353,10 @@ def main():
             "steps": args.steps, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f16 operands, f32 accumulate (f64 small solvers)", "data": "synthetic",
             "config": {"workload": f"{cfg.name}: {ng * cfg.layers_per_group} layers / {cfg.layers_per_group} per group, "
-                                   f"{cfg.n_kv_heads} KV heads, T={cfg.seq_len}, d=128, fp16, budget {cfg.ratio}x, randomized q={q}",
+                                   f"{cfg.n_kv_heads} KV heads, T={cfg.seq_len}, d=128, fp16, budget {ratio}x, "
+                                   + (f"randomized q={q}" if args.token_mode == "randomized" else "exact (converged block iteration)"),
                        "cache_bytes": cache_bytes, "compressed_bytes": planned_bytes, "achieved_ratio": cache_bytes / planned_bytes,
-                       "plan": plans, "l2": "inputs (537 MB) exceed L2; no flush"},
+                       "plan": plans, "l2": f"inputs ({cache_bytes / 1e6:.0f} MB) exceed L2; no flush"},
             "compress_ms": tc, "decompress_ms": td, "plan_ms": plan_ms,
             "compress_ms_min_med_max": [tc_all[0], tc_all[len(tc_all) // 2], tc_all[-1]],
             "decompress_ms_min_med_max": [td_all[0], td_all[len(td_all) // 2], td_all[-1]],

@@ -57,7 +57,7 @@ typedef struct { int32_t r_t, r_f, bits; } jolt_cell_plan;
 
 /* Options of the token-mode solver (paper Sec. 5) and of the allocator's grid (paper Sec. 4, Eq. (3)). */
 typedef struct {
-  int32_t token_mode;               /* JOLT_TOKEN_EXACT | JOLT_TOKEN_RANDOMIZED                          */
+  int32_t token_mode;               /* JOLT_TOKEN_EXACT | JOLT_TOKEN_RANDOMIZED (see below)               */
   int32_t oversample;               /* p: sketch width k = min(r_t + p, T, m*r_f); default 10             */
   int32_t power_iters;              /* q >= 0 power iterations of the range finder                        */
   int32_t quant_group;              /* must be 32                                                         */
@@ -71,6 +71,12 @@ typedef struct {
   int32_t count_scale_bytes;        /* 1 (default): the fp16 group scales count toward the budget         */
 } jolt_options;
 
+/* JOLT_TOKEN_EXACT (the exact token-mode SVD that Sec. 5 replaces): up to T = 1024 the T x T Gram of the
+ * projected unfolding is diagonalised in fp64.  Beyond that the dominant r_t subspace is computed by block
+ * subspace iteration on the unfolding (block r_t + max(p, 32), max(q, 8) iterations, Rayleigh-Ritz), and the
+ * residual || A V - U S ||_F / || U S ||_F, V = A^T U S^-1, of the result is stored with the cell (component 9);
+ * a residual above 5e-4 fails the call with JOLT_ENUMERIC.  jolt_plan in exact mode at T > 1024 probes the
+ * top q_cap singular values the same way and accounts the tail mass like the randomized probe. */
 typedef struct jolt_handle jolt_handle;
 
 /* Fill *o with the defaults listed above (randomized token mode, p = 10, q = 1, seed 0). */
@@ -140,7 +146,8 @@ int jolt_compressed_bytes(const jolt_handle *h, int64_t *bytes);
  * 3 = packed codes (uint32, [m][T][4*bits]), 4 = scales (fp16, [m][T][4]), 5 = core exponent (int32),
  * 6 = token-mode singular values (fp32, k entries, 0 entries if injected), 7 = mode-3 eigenvalues
  * (fp32, 128; zeros when r_f = 128), 8 = the token factor before fp16 rounding (fp32, [T][r_t]; a view of
- * scratch memory, valid only until the next library call on the device; for tests).
+ * scratch memory, valid only until the next library call on the device; for tests), 9 = residual of the
+ * converged-subspace check (fp32, one value; 0 bytes unless the handle was made in exact mode at T > 1024).
  * dst_bytes is the capacity of dst; *written gets the size of the component. */
 int jolt_get_component(const jolt_handle *h, int32_t cell, int32_t which, void *dst, int64_t dst_bytes,
                        int64_t *written);

@@ -176,7 +176,7 @@ class Handle:
         return b.value
 
     _DT = {0: np.float16, 1: np.float16, 2: np.float16, 3: np.uint32, 4: np.float16, 5: np.int32, 6: np.float32,
-           7: np.float32, 8: np.float32}
+           7: np.float32, 8: np.float32, 9: np.float32}
 
     def component(self, cell: int, which: int) -> np.ndarray:
         n = C.c_int64(0)

@@ -194,6 +194,7 @@ struct jolt_handle {
   size_t blob_bytes = 0;
   uint64_t seed = 0;
   int64_t stored_bytes = 0;
+  bool subspace = false;     // token factors came from the converged block iteration (exact mode, large T)
 };
 
 // ------------------------------------------------------------------ validation
@@ -402,6 +403,7 @@ struct CellWork {      // device scratch of one cell
   __half *P16 = nullptr;
   float *Xt = nullptr;
   int *status = nullptr;
+  float *rho = nullptr;      // where the residual of the converged-subspace check goes (exact mode at large T)
   int n_sigma = 0;
   // tensor-core sweeps
   bool tc = false;           // sketch / projection sweeps run on tcgen05
@@ -638,8 +640,59 @@ void add_project(Program &P, int stage, std::vector<CellWork> &ws) {
   add_gemm(P, stage, g2, false);
 }
 
+// ---- exact token factor at sizes where the T x T eigen-solve is out of reach (Sec. 5 calls the exact token SVD
+// the dominant cost): block subspace iteration, i.e. the range finder with a wider block and enough power
+// iterations to converge, followed by Rayleigh-Ritz (the small SVD).  The residual || A V - U Sigma ||_F /
+// || U Sigma ||_F, V = A^T U Sigma^-1, of the returned factor is measured with two more sweeps and stored with
+// the cell (V has unit columns, which is what the fp16 operand split of the sweeps is scaled for).
+constexpr int kSubspaceOversample = 32;
+constexpr int kSubspaceIters = 8;
+constexpr float kSubspaceTol = 5e-4f;
+constexpr int kExactEigMaxT = 1024;        // largest T for which the T x T Gram is diagonalised directly
+
+struct ResidJob { float *S; const float *UT; const float *sigma; int T, k, r_t; float *rho; int *status; float *Z; int N; };
+
+__global__ void pad_copy_kernel(const ResidJob *__restrict__ jobs) {      // S (T x k) <- [U_T | 0]
+  const ResidJob j = jobs[blockIdx.y];
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < (long long)j.T * j.k; e += (long long)gridDim.x * blockDim.x) {
+    const int t = (int)(e / j.k), c = (int)(e - (long long)t * j.k);
+    j.S[e] = c < j.r_t ? j.UT[(size_t)t * j.r_t + c] : 0.f;
+  }
+}
+
+__global__ void scale_columns_kernel(const ResidJob *__restrict__ jobs) {  // Z (N x k) <- Z Sigma^-1 on the first r_t columns
+  const ResidJob j = jobs[blockIdx.y];
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < (long long)j.N * j.k; e += (long long)gridDim.x * blockDim.x) {
+    const int c = (int)(e % j.k);
+    const float sg = c < j.r_t ? j.sigma[c] : 0.f;
+    j.Z[e] = sg > 0.f ? j.Z[e] / sg : 0.f;
+  }
+}
+
+__global__ void __launch_bounds__(1024) subspace_residual_kernel(const ResidJob *__restrict__ jobs) {   // S holds A V
+  const ResidJob j = jobs[blockIdx.x];
+  double num = 0, den = 0;
+  for (long long e = threadIdx.x; e < (long long)j.T * j.r_t; e += blockDim.x) {
+    const int t = (int)(e / j.r_t), c = (int)(e - (long long)t * j.r_t);
+    const double u = (double)j.sigma[c] * j.UT[e], d = (double)j.S[(size_t)t * j.k + c] - u;
+    num += d * d; den += u * u;
+  }
+  __shared__ double rn[32], rd[32];
+  for (int o = 16; o; o >>= 1) { num += __shfl_xor_sync(0xffffffffu, num, o); den += __shfl_xor_sync(0xffffffffu, den, o); }
+  if ((threadIdx.x & 31) == 0) { rn[threadIdx.x >> 5] = num; rd[threadIdx.x >> 5] = den; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    num = 0; den = 0;
+    for (int i = 0; i < (int)blockDim.x / 32; ++i) { num += rn[i]; den += rd[i]; }
+    const float rho = den > 0 ? (float)sqrt(num / den) : 0.f;
+    if (j.rho) *j.rho = rho;
+    if (!(rho <= kSubspaceTol) && j.status) atomicOr(j.status, 16);
+  }
+}
+
 // Stages that produce U_F (fp32), U_T (fp32) and the core (fp32) of every active cell.
-void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool probe, int power_iters, uint64_t seed, bool fast) {
+void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool probe, int power_iters, uint64_t seed, bool fast,
+                          bool check_subspace = false) {
   (void)fast;
   std::vector<int> act;
   for (size_t i = 0; i < ws.size(); ++i) if (ws[i].active) act.push_back((int)i);
@@ -742,6 +795,20 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
     add_eig(P, ST_SVD, eg, 9);          // k x k, 6-7 sweeps observed
     add_gemm(P, ST_FACT, g2, false);
     add_gemm(P, ST_FACT, g3, false);
+    if (check_subspace && !probe) {
+      std::vector<ResidJob> rj;
+      for (int i : act) {
+        CellWork &w = ws[i];
+        rj.push_back({w.S, w.UT32, w.sigma, w.c.T, w.c.k, w.c.r_t, w.rho, w.status, w.Z, w.c.N});
+      }
+      const size_t off = P.push(rj);
+      const int n = (int)rj.size();
+      P.add(ST_FACT, [=](char *dev, cudaStream_t s) { pad_copy_kernel<<<dim3(64, n), 256, 0, s>>>((const ResidJob *)(dev + off)); LAUNCHED(); });
+      add_project(P, ST_FACT, ws);
+      P.add(ST_FACT, [=](char *dev, cudaStream_t s) { scale_columns_kernel<<<dim3(64, n), 256, 0, s>>>((const ResidJob *)(dev + off)); LAUNCHED(); });
+      add_sketch(P, ST_FACT, ws, false);
+      P.add(ST_FACT, [=](char *dev, cudaStream_t s) { subspace_residual_kernel<<<n, 1024, 0, s>>>((const ResidJob *)(dev + off)); LAUNCHED(); });
+    }
   } else if (mode == FM_EXACT) {
     std::vector<GemmTask> g1, g2, g3; std::vector<EigTask> eg;
     for (int i : act) {
@@ -929,6 +996,7 @@ int status_to_code(const std::vector<int> &st) {
     if (st[i] & 1) return fail(JOLT_ENUMERIC, "cell %zu: eigen-solver did not converge", i / 4);
     if (st[i] & 4) return fail(JOLT_ENUMERIC, "cell %zu: quantisation step is not finite in fp16", i / 4);
     if (st[i] & 8) return fail(JOLT_ETIMEOUT, "cell %zu: a bounded device-side wait ran out", i / 4);
+    if (st[i] & 16) return fail(JOLT_ENUMERIC, "cell %zu: the exact token subspace did not converge in %d block iterations (use the randomized mode)", i / 4, kSubspaceIters);
   }
   return JOLT_OK;
 }
@@ -950,17 +1018,18 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   const bool injected = inUT != nullptr || inUF != nullptr;
   if (injected && (!inUT || !inUF)) return fail(JOLT_EINVAL, "both factor arrays are needed");
   cudaStream_t st = (cudaStream_t)stream;
-  const int mode = injected ? FM_INJECTED : (o->token_mode == JOLT_TOKEN_EXACT ? FM_EXACT : FM_RANDOMIZED);
+  // exact mode: direct T x T eigen-solve up to kExactEigMaxT tokens, converged block subspace iteration beyond
+  const bool subspace = !injected && o->token_mode == JOLT_TOKEN_EXACT && L->seq_len > kExactEigMaxT;
+  const int mode = injected ? FM_INJECTED : (o->token_mode == JOLT_TOKEN_EXACT && !subspace ? FM_EXACT : FM_RANDOMIZED);
+  const int oversample = subspace ? std::max(o->oversample, kSubspaceOversample) : o->oversample;
+  const int power_iters = subspace ? std::max(o->power_iters, kSubspaceIters) : o->power_iters;
   std::vector<CellDesc> cells;
-  make_cells(L, K, V, plan, o->oversample, cells);
+  make_cells(L, K, V, plan, oversample, cells);
   if ((rc = check_plan(cells, plan))) return rc;       // all argument checks come before the first CUDA call
   int dev = 0;
   CU(cudaGetDevice(&dev));
   if (mode == FM_EXACT) {
-    for (auto &c : cells) {
-      if (c.r_t > 0 && c.T > 1024) return fail(JOLT_EUNSUPPORTED, "exact token factor is built for T <= 1024 (got %d)", c.T);
-      c.k = c.r_t;
-    }
+    for (auto &c : cells) c.k = c.r_t;
   }
   if (injected) for (auto &c : cells) c.k = c.r_t;
   const int nc = (int)cells.size();
@@ -972,6 +1041,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   H->device = dev; H->n_layers = L->n_layers; H->n_kv_heads = L->n_kv_heads; H->T = L->seq_len; H->n_groups = L->n_groups;
   H->group_start.assign(L->group_start, L->group_start + L->n_groups + 1);
   H->seed = o->seed;
+  H->subspace = subspace;
   H->cells.resize(nc);
   for (int pass = 0; pass < 2; ++pass) {
     Bump b;
@@ -1029,7 +1099,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
       w.tc = (fmask & 2) && w.active && mode == FM_RANDOMIZED && tc_sweep_ok(cells[i], L->mem_space == JOLT_MEM_HOST);
       w.tc_gram = (fmask & 4) && w.active && mode != FM_INJECTED && tc_sweep_ok(cells[i], L->mem_space == JOLT_MEM_HOST);
       w.ufI = w.active && cells[i].r_f == kD;
-      if (pass == 1) { w.lam = H->cells[i].lam; w.sigma = H->cells[i].n_sigma ? H->cells[i].sigma : nullptr; w.status = d_status + 4 * i; }
+      if (pass == 1) { w.lam = H->cells[i].lam; w.sigma = H->cells[i].n_sigma ? H->cells[i].sigma : nullptr; w.status = d_status + 4 * i; w.rho = (float *)(H->cells[i].e + 1); }
       carve(b, w, mode, true);
       if (pass == 1 && !w.n_sigma) w.n_sigma = H->cells[i].n_sigma;
     }
@@ -1057,7 +1127,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   for (int g = 0; g < n_groups; ++g) {
     std::vector<CellWork> sub = ws;
     for (int i = 0; i < nc; ++i) if (cell_group[i] != g) sub[i].active = false;
-    build_factor_program(PG[g], sub, mode, false, o->power_iters, o->seed, fast);
+    build_factor_program(PG[g], sub, mode, false, power_iters, o->seed, fast, subspace);
   }
   lap("factor program");
   std::vector<StoreJob> sj;
@@ -1141,6 +1211,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   // ---- run
   g_timer.begin(st);
   cudaError_t ce = cudaMemsetAsync(d_status, 0, sizeof(int) * 4 * nc, st);
+  if (subspace) for (int i = 0; i < nc && ce == cudaSuccess; ++i) ce = cudaMemsetAsync(H->cells[i].e, 0, 4 * sizeof(int), st);
   for (int i = 0; i < nc && ce == cudaSuccess; ++i)
     if (cells[i].r_t == 0 || cells[i].r_f == kD || injected) ce = cudaMemsetAsync(H->cells[i].lam, 0, sizeof(float) * kD, st);
   if (ce == cudaSuccess && L->mem_space == JOLT_MEM_HOST) {
@@ -1374,6 +1445,7 @@ extern "C" int jolt_get_component(const jolt_handle *H, int32_t cell, int32_t wh
     case 6: src = cs.sigma; n = 4 * (size_t)cs.n_sigma; break;
     case 7: src = cs.lam; n = 4 * (size_t)kD; break;
     case 8: src = cs.dbg_UT32; n = cs.dbg_UT32 ? 4 * (size_t)c.T * c.r_t : 0; break;
+    case 9: src = cs.e + 1; n = (H->subspace && c.r_t > 0) ? 4 : 0; break;   // residual of the converged-subspace check
     default: return fail(JOLT_EINVAL, "component %d", which);
   }
   *written = (int64_t)n;
@@ -1465,8 +1537,12 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
   CU(cudaGetDevice(&dev));
   const double raw = 2.0 * 2.0 * (double)L->n_layers * L->n_kv_heads * L->seq_len * kD;
   const int nc = 2 * L->n_groups;
-  const bool exact = o->token_mode == JOLT_TOKEN_EXACT;
-  if (exact && L->seq_len > 1024) return fail(JOLT_EUNSUPPORTED, "exact token spectra are built for T <= 1024 (got %d)", L->seq_len);
+  // exact spectra come from the T x T eigen-solve up to kExactEigMaxT tokens; beyond, the probe is the converged
+  // block iteration at the cap with the tail-mass accounting of the randomized probe
+  const bool subspace = o->token_mode == JOLT_TOKEN_EXACT && L->seq_len > kExactEigMaxT;
+  const bool exact = o->token_mode == JOLT_TOKEN_EXACT && !subspace;
+  const int oversample = subspace ? std::max(o->oversample, kSubspaceOversample) : o->oversample;
+  const int power_iters = subspace ? std::max(o->power_iters, kSubspaceIters) : o->power_iters;
   const int q_cap = o->q_cap > 0 ? o->q_cap : cap_policy(L->seq_len, raw / budget);
   std::vector<jolt_cell_plan> probe(nc);
   std::vector<CellDesc> cells;
@@ -1475,7 +1551,7 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
     const int lim = std::min(L->seq_len, m * kD);
     probe[i] = {exact ? lim : std::min(q_cap, lim), kD, 0};
   }
-  make_cells(L, K, V, probe.data(), o->oversample, cells);
+  make_cells(L, K, V, probe.data(), oversample, cells);
   if (exact) for (auto &c : cells) c.k = c.r_t;
   const int mode = exact ? FM_EXACT : FM_RANDOMIZED;
   const size_t esz = L->dtype == JOLT_F16 ? 2 : 4;
@@ -1507,7 +1583,7 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
       ws[i].c.X = (i % 2 == 0 ? stage_K : stage_V) + ((const char *)ws[i].c.X - hb);
     }
   Program P;
-  build_factor_program(P, ws, mode, true, o->power_iters, o->seed, fast);
+  build_factor_program(P, ws, mode, true, power_iters, o->seed, fast);
   void *d_tab = nullptr;
   if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
   g_timer.begin(st);

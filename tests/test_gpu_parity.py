@@ -174,6 +174,57 @@ def test_config0(B, synth, token_mode):
     h.free()
 
 
+# --------------------------------------------------------------------------- exact mode beyond the direct eigen-solve
+def test_exact_mode_large_T_converged_subspace(B, synth):
+    # T = 2048 > 1024: the library's exact mode runs block subspace iteration to convergence; the oracle
+    # diagonalises the Gram of the smaller side.  Same dominant subspace wherever the spectrum has a gap.
+    cfg = synth.CacheConfig("t", 4, 2, 2, 2048, n_terms=24, seed=5)      # m = 4, N = 512
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2, 4]
+    plans = [(24, 96, 4), (24, 128, 4), (16, 128, 2), (32, 128, 8)]
+    opts = B.default_options(seed=9, token_mode=B.TOKEN_EXACT)
+    h, Ko, Vo = _roundtrip(B, K, V, gs, plans, opts)
+    Knp, Vnp = _np(K), _np(V)
+    oc = oracle_cache(Knp, Vnp, gs, plans, seed=9, token_mode="exact")
+    _check_recon(Knp, Vnp, Ko, Vo, gs, oc, "exact T=2048")
+    for c, o in enumerate(oc):
+        rt = o.r_t
+        rho = float(h.component(c, 9)[0])
+        assert 0.0 <= rho <= 5e-4, (c, rho)
+        UT = h.UT32[c].reshape(o.UT16.shape)
+        sig = o.ideal["sigma"]
+        ns = min(rt, cfg.n_terms)          # beyond the signal rank the spectrum is the flat noise floor: no gap for a
+        sg = h.component(c, 6)             # block method to converge on, Ritz values there are lower bounds
+        assert np.allclose(sg[:ns], sig[:ns], rtol=1e-4), c
+        assert np.all(sg[ns:rt] <= sig[ns:rt] * (1 + 1e-4)) and np.allclose(sg[ns:rt], sig[ns:rt], rtol=2e-2), c
+        if (sig[rt - 1] - sig[rt]) / sig[0] > 1e-2:
+            assert projector_distance(UT, o.ideal["U_T"]) <= PROJ, (c, "U_T")
+        else:
+            X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
+            A = O.token_unfold(np.einsum("htf,fs->hts", X, o.ideal["U_F"]))
+            eg, eo = np.linalg.norm(UT.T @ A) ** 2, np.linalg.norm(o.ideal["U_T"].T @ A) ** 2
+            assert abs(eg - eo) <= 1e-4 * eo, (c, eg, eo)
+    h.free()
+    # the plan probe in exact mode at this T: spectra agree with the oracle's on the values the dual uses
+    budget = 0.5 * 2 * K.numel() * 2
+    plan_g, _ = B.jolt_plan(K, V, gs, budget, opts)
+    assert len(plan_g) == 4 and all(p[0] > 0 for p in plan_g)
+
+
+def test_exact_mode_large_T_reports_a_gapless_spectrum(B):
+    # white noise has no gap for a block method to converge on: the measured residual fails the call with a
+    # numerical-failure status instead of handing back an unconverged "exact" factor
+    g = torch.Generator().manual_seed(3)
+    K = torch.randn(2, 2, 2048, 128, generator=g).to(torch.float16).cuda()
+    V = torch.randn(2, 2, 2048, 128, generator=g).to(torch.float16).cuda()
+    with pytest.raises(B.JoltError) as e:
+        B.jolt_compress(K, V, [0, 2], [(32, 128, 4), (32, 128, 4)], B.default_options(seed=1, token_mode=B.TOKEN_EXACT))
+    assert e.value.status == B.ENUMERIC
+    # the randomized mode takes the same input
+    h = B.jolt_compress(K, V, [0, 2], [(32, 128, 4), (32, 128, 4)], B.default_options(seed=1))
+    h.free()
+
+
 # --------------------------------------------------------------------------- fp16 multi-group cache, several tiles
 @pytest.mark.parametrize("bits_k,bits_v", [(4, 8), (0, 3), (1, 2)])
 def test_small_gqa_cache(B, synth, bits_k, bits_v):
