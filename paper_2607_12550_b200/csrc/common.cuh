@@ -51,4 +51,9 @@ __device__ __forceinline__ long long cell_row_offset(const CellDesc &c, int h, i
   return (long long)l * c.sl + (long long)hd * c.sh + (long long)t * c.st;
 }
 
+// Longest token range one tensor-core accumulator contracts over (see tc_gemm.cuh); longer sequences are cut
+// into segments whose partial results are added in fp64.
+constexpr int kTokSegment = 4096;
+inline int tok_segments(int T) { return (T + kTokSegment - 1) / kTokSegment; }
+
 }  // namespace jolt

@@ -116,11 +116,21 @@ inline bool x_tma_ok(const CellDesc &c) {
   return c.dtype == DT_F16 && c.st % 8 == 0 && c.sh % 8 == 0 && c.sl % 8 == 0 && ((uintptr_t)c.X % 16 == 0) && c.T % 128 == 0;
 }
 
-// A cell's factor-stage sweeps can run on tensor cores: fp16 data TMA can address, sketch width <= 256.
+// A cell's factor-stage sweeps can run on tensor cores: fp16 data TMA can address.  One MMA takes N <= 256
+// columns; wider sketches are swept in column chunks (one more read of X per chunk).
+constexpr int kTcMaxSketch = 768;
 inline bool tc_sweep_ok(const CellDesc &c, bool staged_from_host) {
   if (c.dtype != DT_F16 || c.st % 8 || c.sh % 8 || c.sl % 8 || c.T % 128) return false;
   if (!staged_from_host && ((uintptr_t)c.X % 16)) return false;
-  return c.k >= 1 && c.k <= 256;
+  return c.k >= 1 && c.k <= kTcMaxSketch;
+}
+
+// column chunks of a padded sketch width: equal multiples of 16, each <= 256
+inline void sketch_chunks(int kp, std::vector<std::pair<int, int>> &out) {
+  const int n = (kp + 255) / 256;
+  const int w = (((kp + n - 1) / n) + 15) & ~15;
+  out.clear();
+  for (int c0 = 0; c0 < kp; c0 += w) out.push_back({c0, std::min(w, kp - c0)});
 }
 
 inline int ilog2_floor(long long v) { int e = 0; while ((1ll << (e + 1)) <= v) ++e; return e; }
@@ -170,10 +180,15 @@ inline void add_gram_tc(Program &P, int stage, std::vector<CellWork> &ws) {
     tc::GemmCell g;
     memset(&g, 0, sizeof g);
     make_x_map(&g.tmX, w.c, 64);
-    g.C = (float *)w.gram_part; g.ldc = kD; g.ncols = kD; g.kp = kD; g.has_lo = 0; g.scale_exp = 0;
+    g.ldc = kD; g.ncols = kD; g.kp = kD; g.has_lo = 0; g.scale_exp = 0;
     g.m = w.c.m; g.n_heads = w.c.n_heads; g.T = w.c.T; g.status = w.status;
-    gc.push_back(g);
-    parts.push_back((const float *)w.gram_part); outs.push_back(w.C); counts.push_back(w.c.m);
+    const int nseg = tok_segments(w.c.T);
+    for (int sg = 0; sg < nseg; ++sg) {
+      g.C = (float *)w.gram_part + (size_t)sg * w.c.m * kD * kD;
+      g.t0 = sg * kTokSegment; g.n_tok = std::min(kTokSegment, w.c.T - g.t0);
+      gc.push_back(g);
+    }
+    parts.push_back((const float *)w.gram_part); outs.push_back(w.C); counts.push_back(w.c.m * nseg);
   }
   if (gc.empty()) return;
   launch_tc_gemm<tc::GM_GRAM>(P, stage, gc);
@@ -204,17 +219,23 @@ inline void add_tok_tc(Program &P, int stage, std::vector<CellWork> &ws, const s
       j.kp = w.kp; j.scale_exp = se;
       sp.push_back(j);
     }
-    tc::GemmCell g;
-    memset(&g, 0, sizeof g);
-    const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)w.kp, (uint64_t)c.m};
-    const uint64_t str[2] = {(uint64_t)kD * 2, (uint64_t)w.kp * kD * 2};
-    const uint32_t box[3] = {64, (uint32_t)w.kp, 1};
-    bool okm = make_x_map(&g.tmX, c, 128) && make_tmap_f16(&g.tmBhi, w.Bhi, 3, dims, str, box) &&
-               make_tmap_f16(&g.tmBlo, w.Blo, 3, dims, str, box);
-    (void)okm;
-    g.C = w.S; g.ldc = c.k; g.ncols = c.k; g.kp = w.kp; g.has_lo = src[i] != 0; g.scale_exp = se;
-    g.m = c.m; g.n_heads = c.n_heads; g.T = c.T; g.status = w.status;
-    gc.push_back(g);
+    std::vector<std::pair<int, int>> ch;
+    sketch_chunks(w.kp, ch);
+    for (auto &cc : ch) {
+      const int c0 = cc.first, kc = cc.second;
+      if (c0 >= c.k) break;
+      tc::GemmCell g;
+      memset(&g, 0, sizeof g);
+      const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)kc, (uint64_t)c.m};
+      const uint64_t str[2] = {(uint64_t)kD * 2, (uint64_t)w.kp * kD * 2};
+      const uint32_t box[3] = {64, (uint32_t)kc, 1};
+      bool okm = make_x_map(&g.tmX, c, 128) && make_tmap_f16(&g.tmBhi, w.Bhi + (size_t)c0 * kD, 3, dims, str, box) &&
+                 make_tmap_f16(&g.tmBlo, w.Blo + (size_t)c0 * kD, 3, dims, str, box);
+      (void)okm;
+      g.C = w.S + c0; g.ldc = c.k; g.ncols = std::min(kc, c.k - c0); g.kp = kc; g.has_lo = src[i] != 0; g.scale_exp = se;
+      g.m = c.m; g.n_heads = c.n_heads; g.T = c.T; g.status = w.status;
+      gc.push_back(g);
+    }
   }
   launch_split(P, stage, sp);
   launch_tc_gemm<tc::GM_TOK>(P, stage, gc);
@@ -224,6 +245,7 @@ inline void add_tok_tc(Program &P, int stage, std::vector<CellWork> &ws, const s
 inline void add_feat_tc(Program &P, int stage, std::vector<CellWork> &ws) {
   std::vector<tc::SplitJob> sp;
   std::vector<tc::GemmCell> gc;
+  std::vector<tc::SumJob> sums;
   for (auto &w : ws) {
     if (!w.active || !w.tc) continue;
     const CellDesc &c = w.c;
@@ -231,20 +253,40 @@ inline void add_feat_tc(Program &P, int stage, std::vector<CellWork> &ws) {
     tc::SplitJob j;
     j.in = w.S; j.hi = w.Bhi; j.lo = w.Blo; j.batch = 1; j.rows = c.T; j.cols = c.k; j.ld_in = c.k; j.kp = w.kp; j.scale_exp = se;
     sp.push_back(j);
-    tc::GemmCell g;
-    memset(&g, 0, sizeof g);
-    const uint64_t dims[2] = {(uint64_t)c.T, (uint64_t)w.kp};
-    const uint64_t str[1] = {(uint64_t)c.T * 2};
-    const uint32_t box[2] = {64, (uint32_t)w.kp};
-    bool okm = make_x_map(&g.tmX, c, 64) && make_tmap_f16(&g.tmBhi, w.Bhi, 2, dims, str, box) &&
-               make_tmap_f16(&g.tmBlo, w.Blo, 2, dims, str, box);
-    (void)okm;
-    g.C = w.Zp; g.ldc = c.k; g.ncols = c.k; g.kp = w.kp; g.has_lo = 1; g.scale_exp = se;
-    g.m = c.m; g.n_heads = c.n_heads; g.T = c.T; g.status = w.status;
-    gc.push_back(g);
+    std::vector<std::pair<int, int>> ch;
+    sketch_chunks(w.kp, ch);
+    for (auto &cc : ch) {
+      const int c0 = cc.first, kc = cc.second;
+      if (c0 >= c.k) break;
+      tc::GemmCell g;
+      memset(&g, 0, sizeof g);
+      const uint64_t dims[2] = {(uint64_t)c.T, (uint64_t)kc};
+      const uint64_t str[1] = {(uint64_t)c.T * 2};
+      const uint32_t box[2] = {64, (uint32_t)kc};
+      bool okm = make_x_map(&g.tmX, c, 64) && make_tmap_f16(&g.tmBhi, w.Bhi + (size_t)c0 * c.T, 2, dims, str, box) &&
+                 make_tmap_f16(&g.tmBlo, w.Blo + (size_t)c0 * c.T, 2, dims, str, box);
+      (void)okm;
+      g.ldc = c.k; g.ncols = std::min(kc, c.k - c0); g.kp = kc; g.has_lo = 1; g.scale_exp = se;
+      g.m = c.m; g.n_heads = c.n_heads; g.T = c.T; g.status = w.status;
+      const int nseg = tok_segments(c.T);
+      for (int sg = 0; sg < nseg; ++sg) {
+        g.C = (nseg > 1 ? w.Zpart + (size_t)sg * c.m * kD * c.k : w.Zp) + c0;
+        g.t0 = sg * kTokSegment; g.n_tok = std::min(kTokSegment, c.T - g.t0);
+        gc.push_back(g);
+      }
+    }
+    if (tok_segments(c.T) > 1) sums.push_back({w.Zpart, w.Zp, (long long)c.m * kD * c.k, (long long)c.m * kD * c.k, tok_segments(c.T)});
   }
   launch_split(P, stage, sp);
   launch_tc_gemm<tc::GM_FEAT>(P, stage, gc);
+  if (!sums.empty()) {
+    const size_t off = P.push(sums);
+    const int n = (int)sums.size();
+    P.add(stage, [=](char *dev_t, cudaStream_t s) {
+      tc::sum_partials_f32_kernel<<<dim3(296, n), 256, 0, s>>>((const tc::SumJob *)(dev_t + off));
+      LAUNCHED();
+    });
+  }
 }
 
 // fp16 sketch of the r_f = d tensor-core cells, written straight into the TOK operand layout.

@@ -400,6 +400,7 @@ struct CellWork {      // device scratch of one cell
   float *Ut = nullptr, *sigma = nullptr;
   float *UT32 = nullptr, *G32 = nullptr;
   float *Y = nullptr; double *Gt = nullptr, *Gtv = nullptr, *Gtw = nullptr;
+  float *Zpart = nullptr;    // per-token-segment partials of the projection sweep (T > 4096 on tensor cores)
   __half *P16 = nullptr;
   float *Xt = nullptr;
   int *status = nullptr;
@@ -436,7 +437,7 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
         w.bjA = b.take<double>(2 * nP * nP); w.bjV = b.take<double>(nP * nP); w.bjJ = b.take<double>(2 * (nbe / 2) * 1024);
         w.bjOff = b.take<double>(4); w.bjDone = b.take<int>(4);
       }
-      w.gram_part = b.take<double>((size_t)c.m * kD * kD);
+      w.gram_part = b.take<double>((size_t)c.m * kD * kD * std::max(1, (tok_segments(c.T) + 1) / 2));
       w.C = b.take<double>(kD * kD); w.Cv = b.take<double>(kD * kD); w.Cw = b.take<double>(kD);
     }
     if (mode == FM_RANDOMIZED) {
@@ -450,8 +451,9 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
         w.kp = (c.k + 15) & ~15;
         const size_t nb = std::max((size_t)c.m * w.kp * kD, (size_t)w.kp * T);
         w.Bhi = b.take<__half>(nb); w.Blo = b.take<__half>(nb);
+        if (tok_segments(c.T) > 1) w.Zpart = b.take<float>((size_t)tok_segments(c.T) * c.m * kD * k);
       }
-      w.Gs = b.take<double>(k * k); w.Linv = b.take<double>(k * k); w.LinvT = b.take<float>(k * k);
+      w.Gs = b.take<double>(k * k); w.Linv = b.take<double>(k * (k + 1)); w.LinvT = b.take<float>(k * k);
       w.gpart = b.take<double>(kGramChunks * k * k); w.LT32 = b.take<float>(k * (k + 4)); w.invd = b.take<float>(k + 4);
       w.BBt = b.take<double>(k * k); w.BBv = b.take<double>(k * k); w.BBw = b.take<double>(k);
       w.Ut = b.take<float>(k * std::max<size_t>(c.r_t, 1));
@@ -480,24 +482,18 @@ struct TallGram { const float *M; int rows, k; double *part, *out; };
 void add_tall_gram(Program &P, int stage, const std::vector<TallGram> &jobs) {
   std::vector<GemmTask> g;
   std::vector<ReduceJob> rj;
-  std::vector<TallGramJob> fastj[3];        // register-tiled kernel for k <= 48 / 96 / 144
+  std::vector<TallGramJob> fastj[3];        // register-tiled kernel, column blocks of width <= 48 / 96 / 144
   int fast_chunks[3] = {0, 0, 0};
   for (auto &j : jobs) {
     int chunk = std::max(128, (j.rows + kGramChunks - 1) / kGramChunks);
     chunk = (chunk + 15) & ~15;
     const int n = (j.rows + chunk - 1) / chunk;
-    if (j.k <= 144) {
-      const int cls = j.k <= 48 ? 0 : (j.k <= 96 ? 1 : 2);
-      fastj[cls].push_back({j.M, j.rows, j.k, chunk, j.part});
-      fast_chunks[cls] = std::max(fast_chunks[cls], n);
-    } else {
-      int c = 0;
-      for (int r0 = 0; r0 < j.rows; r0 += chunk, ++c) {
-        const float *m0 = j.M + (size_t)r0 * j.k;
-        g.push_back(mk(m0, DT_F32, 1, j.k, m0, DT_F32, j.k, 1, j.part + (size_t)c * j.k * j.k, DT_F64, j.k, j.k, j.k,
-                       std::min(chunk, j.rows - r0)));
-      }
-    }
+    const int nb = (j.k + 143) / 144, bw = (j.k + nb - 1) / nb;          // column blocks of at most 144
+    const int cls = bw <= 48 ? 0 : (bw <= 96 ? 1 : 2);
+    for (int bi = 0; bi < nb; ++bi)
+      for (int bj = 0; bj <= bi; ++bj)
+        fastj[cls].push_back({j.M, j.rows, j.k, chunk, j.part, bi * bw, std::min(bw, j.k - bi * bw), bj * bw, std::min(bw, j.k - bj * bw)});
+    fast_chunks[cls] = std::max(fast_chunks[cls], n);
     rj.push_back({j.part, j.out, n, j.k * j.k});
   }
   for (int cls = 0; cls < 3; ++cls) {
@@ -526,53 +522,47 @@ void add_tall_gram(Program &P, int stage, const std::vector<TallGram> &jobs) {
 // token_side selects S (T rows) or Z (N rows); the result is left in the source buffer.
 void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side, int passes) {
   for (int pass = 0; pass < 2; ++pass) {
+    // cls 0: Cholesky work matrix and L^T resident in shared memory (k <= kCholSmemMaxN); cls 1: both in global memory
     std::vector<TallGram> tg;
-    std::vector<GemmTask> g2;
-    std::vector<CholTask> ch;
-    std::vector<CholSmemTask> chs;
-    std::vector<TrsmJob> tj;
-    int max_k = 0;
+    std::vector<CholSmemTask> chs[2];
+    std::vector<TrsmJob> tj[2];
+    int max_k[2] = {0, 0};
+    if (pass >= passes) continue;          // the triangular solve works in place, so one pass is possible
     for (auto &w : ws) {
       if (!w.active) continue;
       const int k = w.c.k, rows = token_side ? w.c.T : w.c.N;
-      float *src = token_side ? (pass == 0 ? w.S : w.S2) : (pass == 0 ? w.Z : w.Z2);
-      float *dst = token_side ? (pass == 0 ? w.S2 : w.S) : (pass == 0 ? w.Z2 : w.Z);
-      if (k <= kCholSmemMaxN) {
-        // resident path: the triangular solve works in place, so one pass is possible
-        if (pass >= passes) continue;
-        float *buf = token_side ? w.S : w.Z;
-        tg.push_back({buf, rows, k, w.gpart, w.Gs});
-        chs.push_back({w.Gs, w.LT32, w.invd, k, w.status});
-        tj.push_back({buf, buf, rows, k, w.LT32, w.invd});
-        max_k = std::max(max_k, k);
-      } else {
-        tg.push_back({src, rows, k, w.gpart, w.Gs});
-        CholTask c; c.G = w.Gs; c.Linv = w.Linv; c.LinvT32 = w.LinvT; c.n = k; c.status = w.status;
-        ch.push_back(c);
-        g2.push_back(mk(src, DT_F32, k, 1, w.LinvT, DT_F32, k, 1, dst, DT_F32, k, rows, k, k));
-      }
+      const int cls = k <= kCholSmemMaxN ? 0 : 1;
+      float *buf = token_side ? w.S : w.Z;
+      tg.push_back({buf, rows, k, w.gpart, w.Gs});
+      chs[cls].push_back({w.Gs, w.LT32, w.invd, k, w.status, w.Linv});
+      tj[cls].push_back({buf, buf, rows, k, w.LT32, w.invd});
+      max_k[cls] = std::max(max_k[cls], k);
     }
     add_tall_gram(P, stage, tg);
-    add_chol(P, stage, ch);
-    add_gemm(P, stage, g2, false);
-    if (!chs.empty()) {
-      static bool attr_done = false;
-      if (!attr_done) {
-        cudaFuncSetAttribute(cholesky_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)chol_smem_bytes(kCholSmemMaxN));
-        cudaFuncSetAttribute(trsm_rows_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)trsm_smem_bytes(kCholSmemMaxN, 128));
-        cudaFuncSetAttribute(trsm_rows_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemOptIn - 1024));
-        attr_done = true;
-      }
-      const size_t o1 = P.push(chs), o2 = P.push(tj);
-      const int n = (int)chs.size();
+    static bool attr_done = false;
+    if (!attr_done) {
+      cudaFuncSetAttribute(cholesky_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)chol_smem_bytes(kCholSmemMaxN));
+      cudaFuncSetAttribute(trsm_rows_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemOptIn - 1024));
+      cudaFuncSetAttribute(trsm_rows_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemOptIn - 1024));
+      cudaFuncSetAttribute(trsm_rows_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemOptIn - 1024));
+      attr_done = true;
+    }
+    for (int cls = 0; cls < 2; ++cls) {
+      if (chs[cls].empty()) continue;
+      const size_t o1 = P.push(chs[cls]), o2 = P.push(tj[cls]);
+      const int n = (int)chs[cls].size(), glob = cls;
       int max_rows = 0;
-      for (auto &t : tj) max_rows = std::max(max_rows, t.rows);
-      const bool wide = trsm_smem_bytes(max_k, 256) <= kSmemOptIn - 1024;
-      const size_t sh1 = chol_smem_bytes(max_k), sh2 = trsm_smem_bytes(max_k, wide ? 256 : 128);
+      for (auto &t : tj[cls]) max_rows = std::max(max_rows, t.rows);
+      int rb = 256;
+      while (rb > 64 && trsm_smem_bytes(max_k[cls], rb, glob) > kSmemOptIn - 1024) rb >>= 1;
+      const size_t sh1 = chol_smem_bytes(max_k[cls], glob), sh2 = trsm_smem_bytes(max_k[cls], rb, glob);
       P.add(stage, [=](char *dev, cudaStream_t s) {
-        cholesky_smem_kernel<<<n, 512, sh1, s>>>((const CholSmemTask *)(dev + o1)); LAUNCHED();
-        if (wide) trsm_rows_kernel<256><<<dim3((max_rows + 255) / 256, n), 256, sh2, s>>>((const TrsmJob *)(dev + o2));
-        else trsm_rows_kernel<128><<<dim3((max_rows + 127) / 128, n), 128, sh2, s>>>((const TrsmJob *)(dev + o2));
+        cholesky_smem_kernel<<<n, 512, sh1, s>>>((const CholSmemTask *)(dev + o1), glob); LAUNCHED();
+        const dim3 grid((max_rows + rb - 1) / rb, n);
+        const TrsmJob *jobs = (const TrsmJob *)(dev + o2);
+        if (rb == 256) trsm_rows_kernel<256><<<grid, 256, sh2, s>>>(jobs, glob);
+        else if (rb == 128) trsm_rows_kernel<128><<<grid, 128, sh2, s>>>(jobs, glob);
+        else trsm_rows_kernel<64><<<grid, 64, sh2, s>>>(jobs, glob);
         LAUNCHED();
       });
     }

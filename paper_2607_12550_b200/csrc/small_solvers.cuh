@@ -412,9 +412,9 @@ __device__ __forceinline__ double rsqrt_pos(double d) {
 }
 
 
-struct CholSmemTask { const double *G; float *LT; float *invd; int n; int *status; };
+struct CholSmemTask { const double *G; float *LT; float *invd; int n; int *status; double *work; };
 
-__global__ void __launch_bounds__(512, 1) cholesky_smem_kernel(const CholSmemTask *__restrict__ tasks) {
+__global__ void __launch_bounds__(512, 1) cholesky_smem_kernel(const CholSmemTask *__restrict__ tasks, int in_global) {
   // Left-looking Cholesky by panels of 8 columns.  (1) The panel loses the contribution of the finished columns,
   // one dot product per entry on four independent accumulators.  (2) Warp 0 factors the 8 x 8 diagonal block in
   // registers (shuffles, reciprocal square roots instead of divisions).  (3) The rows below are solved against the
@@ -424,9 +424,11 @@ __global__ void __launch_bounds__(512, 1) cholesky_smem_kernel(const CholSmemTas
   if (n <= 0) return;
   extern __shared__ double shd[];
   const int ld = n + 1;
-  double *A = shd;                       // n x (n+1)
-  double *diag0 = A + (size_t)n * ld;    // n
-  int *dead = (int *)(diag0 + n);        // n
+  // the work matrix lives in shared memory when it fits (n <= kCholSmemMaxN), else in a global buffer that the
+  // CTA reads through L1 (all its threads sit on one SM, so their writes are seen after a barrier)
+  double *A = in_global ? t.work : shd;                         // n x (n+1)
+  double *diag0 = in_global ? shd : shd + (size_t)n * ld;       // n
+  int *dead = (int *)(diag0 + n);                               // n
   __shared__ double blk[8][9];           // the factored diagonal block
   __shared__ double ipiv[8];
   const int tid = threadIdx.x, nt = blockDim.x;
@@ -519,31 +521,39 @@ __global__ void __launch_bounds__(512, 1) cholesky_smem_kernel(const CholSmemTas
   if (tid == 0 && t.status) { int any = 0; for (int i = 0; i < n; ++i) any |= dead[i]; if (any) atomicOr(t.status, 2); }
 }
 
-inline size_t chol_smem_bytes(int n) { return ((size_t)n * (n + 1) + n) * sizeof(double) + (size_t)n * sizeof(int) + 64; }
+inline size_t chol_smem_bytes(int n, bool in_global = false) {
+  return ((in_global ? 0 : (size_t)n * (n + 1)) + n) * sizeof(double) + (size_t)n * sizeof(int) + 64;
+}
 
 struct TrsmJob { const float *src; float *dst; int rows, k; const float *LT; const float *invd; };
 
-inline size_t trsm_smem_bytes(int k, int rb) { const int kp = (k + 3) & ~3; return ((size_t)k * kp + (size_t)kp * (rb + 1) + kp) * sizeof(float) + 64; }
+inline size_t trsm_smem_bytes(int k, int rb, bool lt_global = false) {
+  const int kp = (k + 3) & ~3;
+  return ((lt_global ? 0 : (size_t)k * kp) + (size_t)kp * (rb + 1) + kp) * sizeof(float) + 64;
+}
 
 // RB rows (= threads) per CTA: 256 when the tile fits shared memory, else 128
 template <int RB>
-__global__ void __launch_bounds__(RB) trsm_rows_kernel(const TrsmJob *__restrict__ jobs) {
+__global__ void __launch_bounds__(RB) trsm_rows_kernel(const TrsmJob *__restrict__ jobs, int lt_global) {
   const TrsmJob t = jobs[blockIdx.y];
   const int r0 = blockIdx.x * RB;
   if (r0 >= t.rows) return;
   const int k = t.k, kp = (k + 3) & ~3;
   constexpr int PITCH = RB + 1;
   extern __shared__ float shf[];
-  float *LT = shf;                       // k x kp
-  float *sp = LT + (size_t)k * kp;       // kp x PITCH  (feature j, row r)
-  float *invd = sp + (size_t)kp * PITCH; // kp
+  // L^T stays in global memory (read through L1, every lane of a warp reads the same entries) when it does not fit
+  // beside the row tile
+  float *LTs = shf;                                              // k x kp
+  float *sp = lt_global ? shf : shf + (size_t)k * kp;            // kp x PITCH  (feature j, row r)
+  float *invd = sp + (size_t)kp * PITCH;                         // kp
+  const float *__restrict__ LT = lt_global ? t.LT : LTs;
   const int tid = threadIdx.x;
   const int nrows = min(RB, t.rows - r0);
   // staging loops read eight elements into registers before the first shared-memory store, so that the global
   // loads of a trip are in flight together
-  {
+  if (!lt_global) {
     const float4 *g4 = (const float4 *)t.LT;
-    float4 *s4 = (float4 *)LT;
+    float4 *s4 = (float4 *)LTs;
     const int n4 = k * kp / 4;
     for (int e0 = tid; e0 < n4; e0 += RB * 4) {
       float4 v[4];
@@ -629,7 +639,9 @@ __global__ void reduce_partials_var_kernel(const ReduceJob *__restrict__ jobs) {
 // ---- G = M^T M for a tall fp32 matrix, fp64 accumulation, one partial per row chunk ---------------------
 // Each of the 16 x 16 threads owns a TI x TI register tile of the k x k result (k <= 16 TI), rows stream
 // through shared memory 16 at a time (converted to fp64 once, on the way in).
-struct TallGramJob { const float *M; int rows, k, chunk; double *part; };
+// One job = one block (columns [ca, ca+wa) x [cb, cb+wb)) of the k x k Gram; k <= 16 TI takes a single block,
+// wider matrices the lower-triangular blocks, whose results are also written mirrored.
+struct TallGramJob { const float *M; int rows, k, chunk; double *part; int ca, wa, cb, wb; };
 
 template <int TI>
 __global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__restrict__ jobs) {
@@ -638,7 +650,8 @@ __global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__
   if (r_begin >= t.rows) return;
   const int r_end = min(t.rows, r_begin + t.chunk);
   constexpr int W = 16 * TI;
-  __shared__ double Ms[16][W + 2];
+  __shared__ double Ma[16][W + 2], Mb[16][W + 2];
+  const bool same = t.ca == t.cb;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   double acc[TI][TI];
 #pragma unroll
@@ -649,14 +662,17 @@ __global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__
     const int nr = min(16, r_end - r0);
     for (int e = tid; e < 16 * W; e += 256) {
       const int r = e / W, c = e - r * W;
-      Ms[r][c] = (r < nr && c < t.k) ? (double)t.M[(size_t)(r0 + r) * t.k + c] : 0.0;
+      const float *row = t.M + (size_t)(r0 + r) * t.k;
+      Ma[r][c] = (r < nr && c < t.wa) ? (double)row[t.ca + c] : 0.0;
+      if (!same) Mb[r][c] = (r < nr && c < t.wb) ? (double)row[t.cb + c] : 0.0;
     }
     __syncthreads();
+    const double (*B)[W + 2] = same ? Ma : Mb;
 #pragma unroll 4
     for (int r = 0; r < 16; ++r) {
       double a[TI], b[TI];
 #pragma unroll
-      for (int i = 0; i < TI; ++i) { a[i] = Ms[r][ty + 16 * i]; b[i] = Ms[r][tx + 16 * i]; }
+      for (int i = 0; i < TI; ++i) { a[i] = Ma[r][ty + 16 * i]; b[i] = B[r][tx + 16 * i]; }
 #pragma unroll
       for (int i = 0; i < TI; ++i)
 #pragma unroll
@@ -668,11 +684,13 @@ __global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__
 #pragma unroll
   for (int i = 0; i < TI; ++i) {
     const int row = ty + 16 * i;
-    if (row >= t.k) continue;
+    if (row >= t.wa) continue;
 #pragma unroll
     for (int j = 0; j < TI; ++j) {
       const int col = tx + 16 * j;
-      if (col < t.k) out[(size_t)row * t.k + col] = acc[i][j];
+      if (col >= t.wb) continue;
+      out[(size_t)(t.ca + row) * t.k + t.cb + col] = acc[i][j];
+      if (!same) out[(size_t)(t.cb + col) * t.k + t.ca + row] = acc[i][j];
     }
   }
 }

@@ -7,6 +7,10 @@
 // The cache operand is exact in fp16.  The dense operand (W, Q) is fp32-grade: it arrives split as
 // hi + lo fp16 (pre-scaled by a power of two) and costs two MMAs per K step; a sketch whose entries are
 // fp16 by definition has no lo part and costs one.
+//
+// The fp32 accumulation of tcgen05.mma truncates: a same-sign chain loses about 2^-24 per K step, 2e-5 after
+// 4096 tokens.  Contractions over tokens (FEAT, GRAM) are therefore cut into segments of at most kTokSegment
+// tokens, each its own accumulator, and the partial results are added in fp64.
 #pragma once
 #include "tc_common.cuh"
 
@@ -29,6 +33,7 @@ struct alignas(64) GemmCell {
   int has_lo;
   int scale_exp;        // result is multiplied by 2^-scale_exp
   int m, n_heads, T;
+  int t0, n_tok;        // FEAT / GRAM: the token range this launch item contracts over (a multiple of 64)
   int *status;
 };
 
@@ -71,7 +76,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1) tc_gemm_kernel(const GemmCell *
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int n_steps = MODE == GM_TOK ? 2 * c.m : c.T / 64;
+  const int n_steps = MODE == GM_TOK ? 2 * c.m : c.n_tok / 64;
 
   if (warp == 4 && lane == 0) {
     tma_prefetch_desc(&c.tmX);
@@ -92,11 +97,12 @@ __global__ void __launch_bounds__(GM_THREADS, 1) tc_gemm_kernel(const GemmCell *
       } else {
         const int h = item;
         const int l = h / c.n_heads, hd = h - l * c.n_heads;
-        tma_load_4d(st, &c.tmX, bFull(s), 0, j * 64, hd, l);
-        tma_load_4d(st + 8192, &c.tmX, bFull(s), 64, j * 64, hd, l);
+        const int tok = c.t0 + j * 64;
+        tma_load_4d(st, &c.tmX, bFull(s), 0, tok, hd, l);
+        tma_load_4d(st + 8192, &c.tmX, bFull(s), 64, tok, hd, l);
         if (MODE == GM_FEAT) {
-          tma_load_2d(st + a_bytes, &c.tmBhi, bFull(s), j * 64, 0);
-          if (c.has_lo) tma_load_2d(st + a_bytes + b_pitch, &c.tmBlo, bFull(s), j * 64, 0);
+          tma_load_2d(st + a_bytes, &c.tmBhi, bFull(s), tok, 0);
+          if (c.has_lo) tma_load_2d(st + a_bytes + b_pitch, &c.tmBlo, bFull(s), tok, 0);
         }
       }
     }
@@ -229,6 +235,17 @@ __global__ void reduce_gram_partials_kernel(const float *const *partials, double
   double s = 0;
   for (int h = 0; h < counts[ci]; ++h) s += (double)p[(size_t)h * kD * kD + e];
   out[ci][e] = s;
+}
+
+// out[e] = sum of `count` fp32 partials `stride` elements apart, added in fp64 in a fixed order
+struct SumJob { const float *part; float *out; long long n, stride; int count; };
+__global__ void sum_partials_f32_kernel(const SumJob *__restrict__ jobs) {
+  const SumJob j = jobs[blockIdx.y];
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < j.n; e += (long long)gridDim.x * blockDim.x) {
+    double s = 0;
+    for (int p = 0; p < j.count; ++p) s += (double)j.part[(size_t)p * j.stride + e];
+    j.out[e] = (float)s;
+  }
 }
 
 }  // namespace tc
