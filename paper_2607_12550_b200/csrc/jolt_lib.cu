@@ -371,15 +371,6 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
   }
 }
 
-void add_chol(Program &P, int stage, const std::vector<CholTask> &tasks) {
-  if (tasks.empty()) return;
-  const size_t off = P.push(tasks);
-  const int n = (int)tasks.size();
-  P.add(stage, [=](char *dev, cudaStream_t s) {
-    cholesky_inv_kernel<<<n, 1024, 0, s>>>((const CholTask *)(dev + off));
-    LAUNCHED();
-  });
-}
 
 inline const void *x_head(const CellDesc &c, int h) {
   const int l = h / c.n_heads, hd = h % c.n_heads;
@@ -392,8 +383,8 @@ struct CellWork {      // device scratch of one cell
   bool active = false;       // has a backbone to compute
   double *gram_part = nullptr, *C = nullptr, *Cv = nullptr, *Cw = nullptr;
   float *UF32 = nullptr, *lam = nullptr;
-  float *omega = nullptr, *PF = nullptr, *W = nullptr, *S = nullptr, *S2 = nullptr, *Zp = nullptr, *Z = nullptr, *Z2 = nullptr;
-  double *Gs = nullptr, *Linv = nullptr; float *LinvT = nullptr;
+  float *omega = nullptr, *PF = nullptr, *W = nullptr, *S = nullptr, *Zp = nullptr, *Z = nullptr;
+  double *Gs = nullptr, *Lwork = nullptr;      // Gram of the basis, Cholesky work matrix (k x (k+1)) for k > kCholSmemMaxN
   double *gpart = nullptr; float *LT32 = nullptr, *invd = nullptr;
   double *bjA = nullptr, *bjV = nullptr, *bjJ = nullptr, *bjOff = nullptr; int *bjDone = nullptr;
   double *BBt = nullptr, *BBv = nullptr, *BBw = nullptr;
@@ -444,16 +435,15 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
       w.omega = b.take<float>((size_t)c.m * kD * k);
       w.PF = b.take<float>(kD * kD);
       w.W = b.take<float>((size_t)c.m * kD * k);
-      w.S = b.take<float>(T * k); w.S2 = b.take<float>(T * k);
+      w.S = b.take<float>(T * k);
       if (w.ufI) w.Z = w.Zp; else w.Z = b.take<float>(N * k);
-      w.Z2 = b.take<float>(N * k);
       if (w.tc) {
         w.kp = (c.k + 15) & ~15;
         const size_t nb = std::max((size_t)c.m * w.kp * kD, (size_t)w.kp * T);
         w.Bhi = b.take<__half>(nb); w.Blo = b.take<__half>(nb);
         if (tok_segments(c.T) > 1) w.Zpart = b.take<float>((size_t)tok_segments(c.T) * c.m * kD * k);
       }
-      w.Gs = b.take<double>(k * k); w.Linv = b.take<double>(k * (k + 1)); w.LinvT = b.take<float>(k * k);
+      w.Gs = b.take<double>(k * k); w.Lwork = k > (size_t)kCholSmemMaxN ? b.take<double>(k * (k + 1)) : nullptr;
       w.gpart = b.take<double>(kGramChunks * k * k); w.LT32 = b.take<float>(k * (k + 4)); w.invd = b.take<float>(k + 4);
       w.BBt = b.take<double>(k * k); w.BBv = b.take<double>(k * k); w.BBw = b.take<double>(k);
       w.Ut = b.take<float>(k * std::max<size_t>(c.r_t, 1));
@@ -480,9 +470,8 @@ namespace {
 // the partials are summed in a fixed order.
 struct TallGram { const float *M; int rows, k; double *part, *out; };
 void add_tall_gram(Program &P, int stage, const std::vector<TallGram> &jobs) {
-  std::vector<GemmTask> g;
   std::vector<ReduceJob> rj;
-  std::vector<TallGramJob> fastj[3];        // register-tiled kernel, column blocks of width <= 48 / 96 / 144
+  std::vector<TallGramJob> fastj[6];        // register-tiled kernel, column blocks of width <= 48 / 96 / 144; +3: off-diagonal blocks
   int fast_chunks[3] = {0, 0, 0};
   for (auto &j : jobs) {
     int chunk = std::max(128, (j.rows + kGramChunks - 1) / kGramChunks);
@@ -492,23 +481,24 @@ void add_tall_gram(Program &P, int stage, const std::vector<TallGram> &jobs) {
     const int cls = bw <= 48 ? 0 : (bw <= 96 ? 1 : 2);
     for (int bi = 0; bi < nb; ++bi)
       for (int bj = 0; bj <= bi; ++bj)
-        fastj[cls].push_back({j.M, j.rows, j.k, chunk, j.part, bi * bw, std::min(bw, j.k - bi * bw), bj * bw, std::min(bw, j.k - bj * bw)});
+        fastj[cls + (bi == bj ? 0 : 3)].push_back({j.M, j.rows, j.k, chunk, j.part, bi * bw, std::min(bw, j.k - bi * bw), bj * bw, std::min(bw, j.k - bj * bw)});
     fast_chunks[cls] = std::max(fast_chunks[cls], n);
     rj.push_back({j.part, j.out, n, j.k * j.k});
   }
-  for (int cls = 0; cls < 3; ++cls) {
-    if (fastj[cls].empty()) continue;
-    const size_t off = P.push(fastj[cls]);
-    const int n = (int)fastj[cls].size(), nch = fast_chunks[cls];
+  for (int q = 0; q < 6; ++q) {
+    if (fastj[q].empty()) continue;
+    const size_t off = P.push(fastj[q]);
+    const int n = (int)fastj[q].size(), cls = q % 3, nch = fast_chunks[cls];
+    const bool diag = q < 3;
     P.add(stage, [=](char *dev, cudaStream_t s) {
       const TallGramJob *d = (const TallGramJob *)(dev + off);
-      if (cls == 0) tall_gram_kernel<3><<<dim3(nch, n), 256, 0, s>>>(d);
-      else if (cls == 1) tall_gram_kernel<6><<<dim3(nch, n), 256, 0, s>>>(d);
-      else tall_gram_kernel<9><<<dim3(nch, n), 256, 0, s>>>(d);
+      const dim3 grid(nch, n);
+      if (cls == 0) { if (diag) tall_gram_kernel<3, true><<<grid, 256, 0, s>>>(d); else tall_gram_kernel<3, false><<<grid, 256, 0, s>>>(d); }
+      else if (cls == 1) { if (diag) tall_gram_kernel<6, true><<<grid, 256, 0, s>>>(d); else tall_gram_kernel<6, false><<<grid, 256, 0, s>>>(d); }
+      else { if (diag) tall_gram_kernel<9, true><<<grid, 256, 0, s>>>(d); else tall_gram_kernel<9, false><<<grid, 256, 0, s>>>(d); }
       LAUNCHED();
     });
   }
-  add_gemm(P, stage, g, true);
   if (rj.empty()) return;
   const size_t off = P.push(rj);
   const int n = (int)rj.size();
@@ -534,7 +524,7 @@ void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side,
       const int cls = k <= kCholSmemMaxN ? 0 : 1;
       float *buf = token_side ? w.S : w.Z;
       tg.push_back({buf, rows, k, w.gpart, w.Gs});
-      chs[cls].push_back({w.Gs, w.LT32, w.invd, k, w.status, w.Linv});
+      chs[cls].push_back({w.Gs, w.LT32, w.invd, k, w.status, w.Lwork});
       tj[cls].push_back({buf, buf, rows, k, w.LT32, w.invd});
       max_k[cls] = std::max(max_k[cls], k);
     }

@@ -1,7 +1,6 @@
-// Batched small dense solvers in fp64, one CTA per problem: symmetric eigen-decomposition by
-// parallel two-sided Jacobi (round-robin ordering), Cholesky with dead-pivot deflation and the
-// inverse of the triangular factor (the pieces of CholeskyQR2).  Problems live in global memory
-// (L2-resident: n <= 522 in the randomized path).
+// Batched small dense solvers: symmetric eigen-decomposition by parallel two-sided Jacobi in fp64 (round-robin
+// ordering, one CTA per problem; the multi-CTA block version is in block_jacobi.cuh) and the pieces of
+// CholeskyQR2: tall Gram (fp64), Cholesky with dead-pivot deflation (fp64), row-wise triangular solve (fp32).
 #pragma once
 #include "common.cuh"
 
@@ -333,69 +332,10 @@ __global__ void __launch_bounds__(kEigThreads, 1) jacobi_eig_smem_kernel(const E
     }
 }
 
-struct CholTask {
-  double *G;        // n x n symmetric positive semi-definite (lower part used); overwritten by L
-  double *Linv;     // n x n out: inverse of L (lower), rows of dead pivots zero
-  float *LinvT32;   // optional n x n out, row-major: (L^-1)^T in fp32 (entry [c][j] = Linv[j][c])
-  int n;
-  int *status;      // bit 1 set if a pivot was deflated (rank deficiency; not an error)
-};
-
-__global__ void __launch_bounds__(1024) cholesky_inv_kernel(const CholTask *__restrict__ tasks) {
-  const CholTask t = tasks[blockIdx.x];
-  const int n = t.n;
-  if (n <= 0) return;
-  double *G = t.G;
-  const int tid = threadIdx.x, nt = blockDim.x;
-  __shared__ int dead[2048];
-  __shared__ double s_piv;
-  __shared__ double diag0[2048];
-  for (int i = tid; i < n; i += nt) { diag0[i] = G[(size_t)i * n + i]; dead[i] = 0; }
-  __syncthreads();
-  for (int j = 0; j < n; ++j) {
-    if (tid == 0) {
-      const double a = G[(size_t)j * n + j];
-      if (!(a > 1e-10 * diag0[j]) || !(diag0[j] > 0)) { dead[j] = 1; s_piv = 0.0; G[(size_t)j * n + j] = 1.0; }
-      else { s_piv = sqrt(a); G[(size_t)j * n + j] = s_piv; }
-    }
-    __syncthreads();
-    const double piv = s_piv;
-    for (int i = j + 1 + tid; i < n; i += nt)
-      G[(size_t)i * n + j] = (piv > 0) ? G[(size_t)i * n + j] / piv : 0.0;
-    __syncthreads();
-    if (piv > 0) {
-      const int rem = n - j - 1;
-      for (int it = tid; it < rem * rem; it += nt) {
-        const int i = j + 1 + it / rem, l = j + 1 + it % rem;
-        if (l <= i) G[(size_t)i * n + l] -= G[(size_t)i * n + j] * G[(size_t)l * n + j];
-      }
-    }
-    __syncthreads();
-  }
-  // Linv by forward substitution, one thread per column c: solve L x = e_c
-  for (int c = tid; c < n; c += nt) {
-    for (int i = 0; i < n; ++i) {
-      double v = 0.0;
-      if (i >= c && !dead[i] && !dead[c]) {
-        double acc = (i == c) ? 1.0 : 0.0;
-        for (int l = c; l < i; ++l) acc -= G[(size_t)i * n + l] * t.Linv[(size_t)l * n + c];
-        v = acc / G[(size_t)i * n + i];
-      }
-      t.Linv[(size_t)i * n + c] = v;
-    }
-  }
-  __syncthreads();
-  if (t.LinvT32)
-    for (int it = tid; it < n * n; it += nt) {
-      const int c = it / n, j = it - c * n;
-      t.LinvT32[it] = (float)t.Linv[(size_t)j * n + c];
-    }
-  if (tid == 0 && t.status) { int any = 0; for (int i = 0; i < n; ++i) any |= dead[i]; if (any) atomicOr(t.status, 2); }
-}
-
-
-// ---- CholeskyQR pieces resident in shared memory (n <= kCholSmemMaxN) -----------------------------------
-// cholesky_smem_kernel: G = L L^T in fp64 (dead pivots deflated as in cholesky_inv_kernel); writes
+// ---- CholeskyQR pieces ------------------------------------------------------------------------------------
+// cholesky_smem_kernel: G = L L^T in fp64.  A pivot that is not above 1e-10 of its original diagonal entry is
+// deflated (the column of L is zeroed, the diagonal set to 1, status bit 2): rank-deficient sketches lose the
+// dependent directions instead of dividing by rounding noise.  Writes
 // LT[l][j] = L[j][l] (fp32, pitch kp = n rounded up to 4, zero above the diagonal of L) and invd[j] = 1 / L[j][j]
 // (0 for a dead pivot).  trsm_rows_kernel then solves  dst_row * L^T = src_row  for 128 rows per CTA.
 constexpr int kCholSmemMaxN = 168;
@@ -643,15 +583,15 @@ __global__ void reduce_partials_var_kernel(const ReduceJob *__restrict__ jobs) {
 // wider matrices the lower-triangular blocks, whose results are also written mirrored.
 struct TallGramJob { const float *M; int rows, k, chunk; double *part; int ca, wa, cb, wb; };
 
-template <int TI>
+template <int TI, bool SAME>      // SAME: diagonal block (ca == cb), one staged tile serves both operands
 __global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__restrict__ jobs) {
   const TallGramJob t = jobs[blockIdx.y];
   const int r_begin = blockIdx.x * t.chunk;
   if (r_begin >= t.rows) return;
   const int r_end = min(t.rows, r_begin + t.chunk);
   constexpr int W = 16 * TI;
-  __shared__ double Ma[16][W + 2], Mb[16][W + 2];
-  const bool same = t.ca == t.cb;
+  __shared__ double Ma[16][W + 2], Mb[SAME ? 1 : 16][W + 2];
+  constexpr bool same = SAME;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   double acc[TI][TI];
 #pragma unroll
@@ -667,12 +607,11 @@ __global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__
       if (!same) Mb[r][c] = (r < nr && c < t.wb) ? (double)row[t.cb + c] : 0.0;
     }
     __syncthreads();
-    const double (*B)[W + 2] = same ? Ma : Mb;
 #pragma unroll 4
     for (int r = 0; r < 16; ++r) {
       double a[TI], b[TI];
 #pragma unroll
-      for (int i = 0; i < TI; ++i) { a[i] = Ma[r][ty + 16 * i]; b[i] = B[r][tx + 16 * i]; }
+      for (int i = 0; i < TI; ++i) { a[i] = Ma[r][ty + 16 * i]; b[i] = same ? Ma[r][tx + 16 * i] : Mb[r][tx + 16 * i]; }
 #pragma unroll
       for (int i = 0; i < TI; ++i)
 #pragma unroll
