@@ -1301,8 +1301,11 @@ extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void 
   std::vector<CellWork> ws(nc);
   std::vector<char> use_tc(nc, 0);
   int tc_heads = 0;
+  // the tensor-core kernel stores 16-byte vectors: the output tensors must start on a 16-byte boundary (strides are
+  // multiples of 8 elements by check_layout); staged host outputs always do
+  const bool out_al16 = L->mem_space == JOLT_MEM_HOST || (((uintptr_t)Kout | (uintptr_t)Vout) % 16 == 0);
   for (int i = 0; i < nc; ++i)
-    if (fast && H->cells[i].tc_ok) { use_tc[i] = 1; tc_heads += H->cells[i].c.m; }
+    if (fast && out_al16 && H->cells[i].tc_ok) { use_tc[i] = 1; tc_heads += H->cells[i].c.m; }
   void *ws_base = nullptr;
   char *stage_K = nullptr, *stage_V = nullptr;
   int *d_status = nullptr;

@@ -98,6 +98,11 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr, uint32_t
   d |= (uint64_t)2 << 61;    // SWIZZLE_128B
   return d;
 }
+// The k-th 16-element (32-byte) K slice of a K-major swizzled tile: the start-address field counts 16-byte units,
+// so the slice's descriptor is the tile's plus 2k.  Building descriptors once and stepping them keeps the single
+// MMA-issuing thread ahead of the tensor pipe (a full rebuild per MMA costs it ~100 cycles, more than the MMA).
+__device__ __forceinline__ uint64_t umma_desc_kslice(uint64_t tile_desc, int k) { return tile_desc + (uint64_t)(2 * k); }
+
 // Instruction descriptor: fp16 A and B, fp32 D, M x N tile, per-operand major (0 = K-major, 1 = MN-major).
 __host__ __device__ constexpr uint32_t umma_idesc_f16(int M, int N, int a_mn_major, int b_mn_major) {
   return (1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |

@@ -16,9 +16,12 @@
 namespace jolt {
 namespace tc {
 
-// Two variants.  NWG = 2 epilogue warpgroups: any r_t <= 256 (P region 64 KB, 4-stage ring, and for r_t <= 128
-// a staging buffer per warpgroup).  NWG = 4: r_t <= 128 only (P region 32 KB, 2-stage ring, four operand /
-// staging tiles), twice the tiles in flight per SM.  Both use 224 KB of shared memory and one CTA per SM.
+// Two variants.  NWG = 2 epilogue warpgroups: any r_t <= 256 (P region 64 KB, 4-stage ring, one operand tile and
+// one accumulator per warpgroup).  For r_t <= 128 half of the P region is free and extends the ring to six stages
+// (three U_T tiles in flight), and each warpgroup owns TWO accumulators: the MMA thread issues the backbone of a
+// tile two tiles before its rotation, so backbones wait in TMEM instead of U_T tiles waiting in shared memory, and
+// a warpgroup only waits for the eight rotation MMAs of its tile.  NWG = 4: r_t <= 128 only (P region 32 KB,
+// 2-stage ring, four operand / staging tiles).  Both use 224 KB of shared memory, one CTA per SM.
 constexpr int DEC_H_BYTES = 32768;
 template <int NWG> struct DecLayout {
   static constexpr int THREADS = (NWG + 1) * 128;
@@ -26,7 +29,7 @@ template <int NWG> struct DecLayout {
   static constexpr int NS = NWG == 4 ? 2 : 4;                       // ring stages allocated
   static constexpr int BIG_BYTES = NS * 16384 + NWG * 32768;        // ring + operand tiles (set-up operands first)
   static constexpr int SMEM_BYTES = P_BYTES + DEC_H_BYTES + BIG_BYTES + 1024 + 512;
-  static constexpr int TMEM_COLS = NWG == 4 ? 512 : 256;
+  static constexpr int TMEM_COLS = 512;     // NWG = 2 keeps two accumulators per warpgroup when r_t <= 128
   // NWG = 2 moves registers from the producer warpgroup to the epilogue ones; NWG = 4 runs every thread at the
   // launch allocation (96): 20 warps leave no slack in the register file for a blocking re-partition
   static constexpr bool REPARTITION = NWG == 2;
@@ -47,16 +50,53 @@ __device__ __forceinline__ void dec_load_codes(const BBCell &c, long long row, D
   }
 }
 
+// Code j of a 32-code group as the bit pattern of the float 2^23 + code (the code dropped into the low mantissa
+// byte of 0x4B000000 by one byte permute): adding -(2^23 + 2^(BITS-1)) gives code - 2^(BITS-1) exactly, without an
+// integer conversion, and one FMA with dq and dq/2 the dequantised value (code - 2^(BITS-1) + 1/2) dq, rounded once.  W = the group's BITS words, code j at bits [j*BITS, j*BITS + BITS).
+template <int BITS>
+struct DecGroupBytes {      // per-group byte lanes from which every code is one PRMT away
+  uint32_t t[BITS == 8 ? 8 : (BITS == 4 ? 8 : (BITS == 2 ? 8 : (BITS == 1 ? 8 : 1)))];
+  __device__ __forceinline__ void load(const uint32_t *W) {
+    if constexpr (BITS == 8) {
+#pragma unroll
+      for (int w = 0; w < 8; ++w) t[w] = W[w];
+    } else if constexpr (BITS == 4) {       // t[2w] even nibbles, t[2w+1] odd nibbles of word w
+#pragma unroll
+      for (int w = 0; w < 4; ++w) { t[2 * w] = W[w] & 0x0F0F0F0Fu; t[2 * w + 1] = (W[w] >> 4) & 0x0F0F0F0Fu; }
+    } else if constexpr (BITS == 2) {       // t[4w + k]: fields k, k+4, k+8, k+12 of word w
+#pragma unroll
+      for (int w = 0; w < 2; ++w)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) t[4 * w + k] = (W[w] >> (2 * k)) & 0x03030303u;
+    } else if constexpr (BITS == 1) {       // t[k]: bits k, k+8, k+16, k+24
+#pragma unroll
+      for (int k = 0; k < 8; ++k) t[k] = (W[0] >> k) & 0x01010101u;
+    }
+  }
+  __device__ __forceinline__ float value(int j) const {     // j is a compile-time constant after unrolling
+    uint32_t src; int byte;
+    if constexpr (BITS == 8) { src = t[j >> 2]; byte = j & 3; }
+    else if constexpr (BITS == 4) { src = t[2 * (j >> 3) + (j & 1)]; byte = (j & 7) >> 1; }
+    else if constexpr (BITS == 2) { src = t[4 * (j >> 4) + (j & 3)]; byte = (j & 15) >> 2; }
+    else { src = t[j & 7]; byte = j >> 3; }
+    return __uint_as_float(__byte_perm(src, 0x4B000000u, 0x7650u + (uint32_t)byte));
+  }
+};
+
 // codes -> fp16 operand row (pre-scaled), written into the warpgroup's swizzled K-major tile
 template <int BITS>
 __device__ __forceinline__ void dec_unpack_row(const DecCodes<BITS> &d, float pre, unsigned char *rbuf, int rit) {
   constexpr float off = 0.5f - (float)(1 << (BITS > 0 ? BITS - 1 : 0));
   constexpr uint32_t mask = (1u << BITS) - 1u;
+  constexpr bool kFast = BITS == 8 || BITS == 4 || BITS == 2 || BITS == 1;
+  constexpr float c0 = -(8388608.0f + (float)(1 << (BITS > 0 ? BITS - 1 : 0)));
   const __half *sc = (const __half *)&d.sc;
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
-    const float dq = __half2float(sc[g]) * pre;
+    const float dq = __half2float(sc[g]) * pre, hdq = 0.5f * dq;
     unsigned char *rowp = rbuf + (g >> 1) * 16384 + rit * 128;
+    DecGroupBytes<kFast ? BITS : 8> gb;
+    if constexpr (kFast) gb.load(&d.words[g * BITS]);
 #pragma unroll
     for (int ck = 0; ck < 4; ++ck) {
       uint4 pk;
@@ -66,12 +106,16 @@ __device__ __forceinline__ void dec_unpack_row(const DecCodes<BITS> &d, float pr
         float v2[2];
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
-          // code j of the group sits at bits [j*BITS, j*BITS + BITS) of its BITS little-endian words
           const int j = ck * 8 + e2 * 2 + u;
-          const int bit = j * BITS, w = bit >> 5, sh = bit & 31;
-          uint32_t q = d.words[g * BITS + w] >> sh;
-          if (sh + BITS > 32) q |= d.words[g * BITS + w + 1] << (32 - sh);
-          v2[u] = ((float)(q & mask) + off) * dq;
+          if constexpr (kFast) {
+            v2[u] = fmaf(gb.value(j) + c0, dq, hdq);
+          } else {
+            // code j of the group sits at bits [j*BITS, j*BITS + BITS) of its BITS little-endian words
+            const int bit = j * BITS, w = bit >> 5, sh = bit & 31;
+            uint32_t q = d.words[g * BITS + w] >> sh;
+            if (sh + BITS > 32) q |= d.words[g * BITS + w + 1] << (32 - sh);
+            v2[u] = ((float)(q & mask) + off) * dq;
+          }
         }
         hp[e2] = __floats2half2_rn(v2[0], v2[1]);
       }
@@ -184,6 +228,92 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
   return ok;
 }
 
+// Per-tile loop of one of TWO epilogue warpgroups with two accumulators each (tiles wg, wg+2, ...; local index n,
+// accumulator n & 1; barriers and TMEM columns of accumulator 1 sit 16 bytes / 256 columns after accumulator 0).
+//   unpack the tile's codes into the warpgroup's operand tile, wait for the tile's MMAs, read the accumulator,
+//   convert; the fp16 rows go through the warp's OWN 32 rows of the operand tile (which the MMA has just consumed)
+//   and leave as fully coalesced 16-byte stores, two 256-byte rows per warp instruction.  A warp only ever touches
+//   its own rows outside the MMA, so the loop needs no barrier between warps and no asynchronous store to wait for.
+template <int BITS>
+__device__ __forceinline__ bool dec_tile_loop_acc4(const BBCell &c, const DecCtx &x) {
+  DecCodes<BITS> cur;
+  bool ok = true;
+  const long long row0 = (long long)x.h * c.T + x.tile0 * 128 + x.rit;
+  if (x.wg < x.n_tiles) dec_load_codes<BITS>(c, row0 + x.wg * 128, cur);
+  const int lane = x.rit & 31, wrow0 = x.rit & ~31;       // this warp's rows of the tile: wrow0 .. wrow0 + 31
+  unsigned char *obuf = x.rbuf;
+  int n = 0;
+  const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;
+  for (int i = x.wg; i < x.n_tiles; i += 2, ++n) {
+    const int acc = n & 1, ph = n >> 1;
+    const int tt = x.tile0 + i, token = tt * 128 + x.rit;
+    long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;
+    if (dbg) dbg[0] = clock64();
+    if constexpr (BITS > 0) {
+      if (ok) dec_unpack_row<BITS>(cur, x.pre, obuf, x.rit);
+      fence_proxy_async();
+      mbar_arrive(x.bRready + 16 * acc);
+      if (i + 2 < x.n_tiles) dec_load_codes<BITS>(c, row0 + (i + 2) * 128, cur);      // in flight during the MMA and the epilogue
+    }
+    if (dbg) dbg[2] = clock64();
+    // after a timed-out wait the warp keeps walking the loop but touches neither TMEM nor the barriers' data again
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(x.bTfull + 16 * acc, ph & 1, x.abort_flag));
+    if (dbg) dbg[3] = clock64();
+    tc_fence_after();
+    const long long off = (long long)x.l * c.osl + (long long)x.hd * c.osh + (long long)token * c.ost;
+    const uint32_t t_acc = x.t_acc + acc * 256;
+    // the whole accumulator row in one go: four loads in flight, one wait
+    float va[4][32];
+    if (ok) {
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) tmem_ld32(t_acc + ch * 32, va[ch]);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(x.bTempty + 16 * acc);
+    }
+    if (dbg) dbg[4] = clock64();
+    if (ok) {
+      if (c.out_dtype == DT_F16) {
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          const float *v = va[ch];
+          unsigned char *rowp = obuf + (ch >> 1) * 16384 + x.rit * 128;
+#pragma unroll
+          for (int k8 = 0; k8 < 4; ++k8) {
+            uint4 o;
+            __half2 *hp = (__half2 *)&o;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) hp[j] = __floats2half2_rn(v[k8 * 8 + 2 * j] * x.scale, v[k8 * 8 + 2 * j + 1] * x.scale);
+            *(uint4 *)(rowp + ((((ch & 1) * 4 + k8) ^ (x.rit & 7)) << 4)) = o;
+          }
+        }
+        __syncwarp();
+        if (dbg) dbg[5] = clock64();
+        // read back: lane l takes 16-byte chunk l & 15 of rows 2 it + (l >> 4); a row is 256 contiguous bytes of output
+        const int q16 = lane & 15;
+        __half *obase = (__half *)c.out + (long long)x.l * c.osl + (long long)x.hd * c.osh;
+#pragma unroll 4
+        for (int it = 0; it < 16; ++it) {
+          const int r = wrow0 + 2 * it + (lane >> 4);
+          const uint4 o = *(const uint4 *)(obuf + (q16 >> 3) * 16384 + r * 128 + (((q16 & 7) ^ (r & 7)) << 4));
+          *(uint4 *)(obase + (long long)(tt * 128 + r) * c.ost + q16 * 8) = o;
+        }
+        __syncwarp();
+      } else {
+        float4 *p = (float4 *)((float *)c.out + off);
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch)
+#pragma unroll
+          for (int k4 = 0; k4 < 8; ++k4)
+            p[ch * 8 + k4] = make_float4(va[ch][4 * k4] * x.scale, va[ch][4 * k4 + 1] * x.scale, va[ch][4 * k4 + 2] * x.scale,
+                                         va[ch][4 * k4 + 3] * x.scale);
+      }
+    }
+    if (dbg) dbg[7] = clock64();
+  }
+  return ok;
+}
+
 template <int NWG>
 __global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(const BBCell *__restrict__ cells, uint64_t seed) {
   using LY = DecLayout<NWG>;
@@ -208,26 +338,30 @@ __global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(cons
   volatile int *abort_flag = (volatile int *)(sm + DEC_P_BYTES + DEC_H_BYTES + DEC_BIG_BYTES + 256);
   uint32_t *tmem_slot = (uint32_t *)(sm + DEC_P_BYTES + DEC_H_BYTES + DEC_BIG_BYTES + 264);
   const uint32_t bSetup = sBar + 0, bPdone = sBar + 8, bPready = sBar + 16;
-  auto bFull = [=](int s) { return sBar + 24 + 8 * s; };
-  auto bEmpty = [=](int s) { return sBar + 56 + 8 * s; };
-  auto bTfull = [=](int b) { return sBar + 88 + 8 * b; };
-  auto bTempty = [=](int b) { return sBar + 120 + 8 * b; };
-  auto bRready = [=](int b) { return sBar + 152 + 8 * b; };
+  auto bFull = [=](int s) { return sBar + 24 + 8 * s; };          // up to 6 ring stages
+  auto bEmpty = [=](int s) { return sBar + 72 + 8 * s; };
+  auto bTfull = [=](int b) { return sBar + 120 + 8 * b; };        // up to 4 accumulators
+  auto bTempty = [=](int b) { return sBar + 152 + 8 * b; };
+  auto bRready = [=](int b) { return sBar + 184 + 8 * b; };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = warp >> 2;
+  long long *kdbg = (c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ? c.dbg + 16 * 8 : nullptr;
+  if (kdbg) kdbg[0] = clock64();
   const int nkt = (c.r_t + 63) / 64, nkf = (c.r_f + 63) / 64;
   const bool has_res = c.bits > 0;
   // r_t <= 128 leaves half of the P region and half of the ring free: each warpgroup then stages its output in a
   // buffer of its own, so a tile's unpack never waits for the previous tile's TMA store to drain
-  const bool sep_out = NWG == 2 && nkt <= 2;
-  const int ns = (NWG == 4 || sep_out) ? 2 : DEC_NS;
+  // r_t <= 128 with two warpgroups: four accumulators and a six-stage ring (see the top of the file)
+  const bool acc4 = NWG == 2 && nkt <= 2;
+  const int ns = NWG == 4 ? 2 : (acc4 ? 6 : DEC_NS);
+  auto sStage = [=](int s) { return s < 4 ? sRing + (uint32_t)s * BB_STAGE_BYTES : sP + 32768u + (uint32_t)(s - 4) * BB_STAGE_BYTES; };
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
     mbar_init(bSetup, 1); mbar_init(bPdone, 1); mbar_init(bPready, NWG * 128);
-    for (int s = 0; s < DEC_NS; ++s) { mbar_init(bFull(s), 1); mbar_init(bEmpty(s), 1); }
-    for (int b = 0; b < NWG; ++b) { mbar_init(bTfull(b), 1); mbar_init(bTempty(b), 128); mbar_init(bRready(b), 128); }
+    for (int s = 0; s < 6; ++s) { mbar_init(bFull(s), 1); mbar_init(bEmpty(s), 1); }
+    for (int b = 0; b < 4; ++b) { mbar_init(bTfull(b), 1); mbar_init(bTempty(b), 128); mbar_init(bRready(b), 128); }
     fence_barrier_init();
   }
   if (warp == NWG * 4) { tmem_alloc(smem_u32(tmem_slot), LY::TMEM_COLS); tmem_relinquish(); }
@@ -255,7 +389,7 @@ __global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(cons
           ok = mbar_wait(bEmpty(s), (n & 1) ^ 1, abort_flag);
           if (!ok) break;
           mbar_expect_tx(bFull(s), BB_STAGE_BYTES);
-          tma_load_2d(sRing + s * BB_STAGE_BYTES, &c.tmUT, bFull(s), kb * 64, tt * 128);
+          tma_load_2d(sStage(s), &c.tmUT, bFull(s), kb * 64, tt * 128);
         }
       }
     } else if (warp == NWG * 4 + 1 && lane == 0) {
@@ -264,43 +398,67 @@ __global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(cons
       if (ok) {
         tc_fence_after();
         const uint32_t idescP = umma_idesc_f16(128, c.r_t, 0, 0);
-        for (int kb = 0; kb < nkf; ++kb)
-          for (int k4 = 0; k4 < 4; ++k4)
-            umma_f16(tmem_base, umma_desc_sw128(sBig + kb * 16384 + k4 * 32, 16, 1024),
-                     umma_desc_sw128(sBig + 32768 + kb * 32768 + k4 * 32, 16, 1024), idescP, (kb | k4) != 0);
+        for (int kb = 0; kb < nkf; ++kb) {
+          const uint64_t da = umma_desc_sw128(sBig + kb * 16384, 16, 1024), db = umma_desc_sw128(sBig + 32768 + kb * 32768, 16, 1024);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4) umma_f16(tmem_base, umma_desc_kslice(da, k4), umma_desc_kslice(db, k4), idescP, (kb | k4) != 0);
+        }
         umma_commit(bPdone);
         ok = mbar_wait(bPready, 0, abort_flag);
       }
       if (ok) {
         tc_fence_after();
         const uint32_t idesc = umma_idesc_f16(128, 128, 0, 0);
+        // With four accumulators the backbone MMAs run `lead` tiles ahead of the rotation MMAs: a ring stage is
+        // released (and the next U_T tile requested) that much earlier, so the load latency hides behind the
+        // tiles whose backbone already waits in TMEM.  MMAs on one accumulator are still issued in order.
+        const int lead = acc4 ? 2 : 0;
+        // tile descriptors built once; per MMA only the K-slice step remains
+        const uint64_t dP0 = umma_desc_sw128(sP, 16, 1024), dH0 = umma_desc_sw128(sH, 16, 1024);
+        const uint64_t dS0 = umma_desc_sw128(sRing, 16, 1024), dS4 = umma_desc_sw128(sP + 32768, 16, 1024);
+        const uint64_t dR0 = umma_desc_sw128(sR, 16, 1024);
+        constexpr uint64_t kStep16K = 16384 >> 4, kStep32K = 32768 >> 4;      // address-field steps
         int cnt = 0;
-        for (int i = 0; ok && i < n_tiles; ++i) {
-          const int b = i % NWG, nb = i / NWG;
-          ok = mbar_wait(bTempty(b), (nb & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          for (int kb = 0; kb < nkt; ++kb, ++cnt) {
-            const int s = cnt % ns, n = cnt / ns;
-            ok = mbar_wait(bFull(s), n & 1, abort_flag);
+        for (int j = 0; ok && j < n_tiles + lead; ++j) {
+          if (j < n_tiles) {
+            // accumulator / barrier index b and how often it has been used (nb)
+            const int wgi = j % NWG, ni = j / NWG;
+            const int b = acc4 ? wgi + 2 * (ni & 1) : wgi, nb = acc4 ? ni >> 1 : ni;
+            ok = mbar_wait(bTempty(b), (nb & 1) ^ 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            for (int k4 = 0; k4 < 4; ++k4)
-              umma_f16(tmem_base + b * 128, umma_desc_sw128(sRing + s * BB_STAGE_BYTES + k4 * 32, 16, 1024),
-                       umma_desc_sw128(sP + kb * 16384 + k4 * 32, 16, 1024), idesc, (kb | k4) != 0);
-            umma_commit(bEmpty(s));
-          }
-          if (!ok) break;
-          if (has_res) {
-            ok = mbar_wait(bRready(b), nb & 1, abort_flag);
+            const uint32_t tacc = tmem_base + b * 128;
+            for (int kb = 0; kb < nkt; ++kb, ++cnt) {
+              const int s = cnt % ns, n = cnt / ns;
+              ok = mbar_wait(bFull(s), n & 1, abort_flag);
+              if (!ok) break;
+              tc_fence_after();
+              const uint64_t da = s < 4 ? dS0 + (uint64_t)s * kStep16K : dS4 + (uint64_t)(s - 4) * kStep16K;
+              const uint64_t db = dP0 + (uint64_t)kb * kStep16K;
+#pragma unroll
+              for (int k4 = 0; k4 < 4; ++k4) umma_f16(tacc, umma_desc_kslice(da, k4), umma_desc_kslice(db, k4), idesc, (kb | k4) != 0);
+              umma_commit(bEmpty(s));
+            }
             if (!ok) break;
-            tc_fence_after();
-            for (int kb = 0; kb < 2; ++kb)
-              for (int k4 = 0; k4 < 4; ++k4)
-                umma_f16(tmem_base + b * 128, umma_desc_sw128(sR + b * 32768 + kb * 16384 + k4 * 32, 16, 1024),
-                         umma_desc_sw128(sH + kb * 16384 + k4 * 32, 16, 1024), idesc, 1);
           }
-          umma_commit(bTfull(b));
+          if (j >= lead) {
+            const int t = j - lead;
+            const int wgi = t % NWG, ni = t / NWG;
+            const int b = acc4 ? wgi + 2 * (ni & 1) : wgi, nb = acc4 ? ni >> 1 : ni;
+            if (has_res) {
+              ok = mbar_wait(bRready(b), nb & 1, abort_flag);
+              if (!ok) break;
+              tc_fence_after();
+              const uint32_t tacc = tmem_base + b * 128;
+              const uint64_t dR = dR0 + (uint64_t)wgi * kStep32K;
+#pragma unroll
+              for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+                for (int k4 = 0; k4 < 4; ++k4)
+                  umma_f16(tacc, umma_desc_kslice(dR + kb * kStep16K, k4), umma_desc_kslice(dH0 + kb * kStep16K, k4), idesc, 1);
+            }
+            umma_commit(bTfull(b));
+          }
         }
       }
     }
@@ -328,7 +486,9 @@ __global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(cons
         *(uint4 *)(smH + (chunk >> 3) * 16384 + f * 128 + (((chunk & 7) ^ (f & 7)) << 4)) = pk;
       }
     }
+    if (kdbg) kdbg[1] = clock64();
     bool ok = __all_sync(0xffffffffu, mbar_wait(bPdone, 0, abort_flag));
+    if (kdbg) kdbg[2] = clock64();
     if (ok) {
       tc_fence_after();
       for (int ch = wg; ch < 2 * nkt; ch += NWG) {
@@ -352,29 +512,42 @@ __global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(cons
       tc_fence_before();
       mbar_arrive(bPready);
     }
+    if (kdbg) kdbg[3] = clock64();
     const int ex = ok ? *c.e : 0;
     const float scale = ldexpf(1.0f, ex);
     const float pre = ldexpf(kInvSqrtD, -ex);        // residual operand is kept in the accumulator's units
     if (ok) {
       DecCtx x;
       x.bTfull = bTfull(wg); x.bTempty = bTempty(wg); x.bRready = bRready(wg);
-      x.t_acc = t_lane + wg * 128; x.rbuf = smR + wg * 32768; x.sep_out = sep_out;
-      if (sep_out) { x.s_obuf = wg == 0 ? sP + 32768 : sRing + 32768; x.obuf = wg == 0 ? sm + 32768 : sm + DEC_P_BYTES + DEC_H_BYTES + 32768; }
-      else { x.s_obuf = sR + wg * 32768; x.obuf = x.rbuf; }
+      x.t_acc = t_lane + wg * 128; x.rbuf = smR + wg * 32768; x.sep_out = false;
+      x.s_obuf = sR + wg * 32768; x.obuf = x.rbuf;
       x.abort_flag = abort_flag; x.wg = wg; x.nwg = NWG; x.rit = rit; x.h = h; x.tile0 = tile0; x.n_tiles = n_tiles;
       x.l = h / c.n_heads; x.hd = h - x.l * c.n_heads; x.scale = scale; x.pre = pre;
-      switch (c.bits) {
-        case 0: dec_tile_loop<0>(c, x); break;
-        case 1: dec_tile_loop<1>(c, x); break;
-        case 2: dec_tile_loop<2>(c, x); break;
-        case 3: dec_tile_loop<3>(c, x); break;
-        case 4: dec_tile_loop<4>(c, x); break;
-        default: dec_tile_loop<8>(c, x); break;
+      if (acc4) {
+        switch (c.bits) {
+          case 0: dec_tile_loop_acc4<0>(c, x); break;
+          case 1: dec_tile_loop_acc4<1>(c, x); break;
+          case 2: dec_tile_loop_acc4<2>(c, x); break;
+          case 3: dec_tile_loop_acc4<3>(c, x); break;
+          case 4: dec_tile_loop_acc4<4>(c, x); break;
+          default: dec_tile_loop_acc4<8>(c, x); break;
+        }
+      } else {
+        switch (c.bits) {
+          case 0: dec_tile_loop<0>(c, x); break;
+          case 1: dec_tile_loop<1>(c, x); break;
+          case 2: dec_tile_loop<2>(c, x); break;
+          case 3: dec_tile_loop<3>(c, x); break;
+          case 4: dec_tile_loop<4>(c, x); break;
+          default: dec_tile_loop<8>(c, x); break;
+        }
       }
     }
   }
+  if (kdbg) kdbg[4] = clock64();
   tc_fence_before();
   __syncthreads();
+  if (kdbg) kdbg[5] = clock64();
   if (*abort_flag) {
     if (threadIdx.x == 0) atomicOr(c.status, 8);
     const long long t0 = clock64();
