@@ -66,13 +66,12 @@ inline void add_backbone_tc(Program &P, int stage, const std::vector<tc::BBCell>
   });
 }
 
-template <int NWG>
-inline void launch_decode(Program &P, int stage, const std::vector<tc::BBCell> &cells, uint64_t seed) {
+inline void add_decode_tc(Program &P, int stage, const std::vector<tc::BBCell> &cells, uint64_t seed) {
   if (cells.empty()) return;
-  using LY = tc::DecLayout<NWG>;
+  using LY = tc::DecLayout;
   static bool attr_done = false;
   if (!attr_done) {
-    cudaFuncSetAttribute(tc::decode_kernel<NWG>, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
+    cudaFuncSetAttribute(tc::decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
     attr_done = true;
   }
   int gx = 0;
@@ -80,17 +79,9 @@ inline void launch_decode(Program &P, int stage, const std::vector<tc::BBCell> &
   const size_t off = P.push(cells);
   const int n = (int)cells.size();
   P.add(stage, [=](char *dev_t, cudaStream_t s) {
-    tc::decode_kernel<NWG><<<dim3(gx, n), LY::THREADS, LY::SMEM_BYTES, s>>>((const tc::BBCell *)(dev_t + off), seed);
+    tc::decode_kernel<<<dim3(gx, n), LY::THREADS, LY::SMEM_BYTES, s>>>((const tc::BBCell *)(dev_t + off), seed);
     LAUNCHED();
   });
-}
-
-// cells with r_t <= 128 take the four-warpgroup variant, the others the two-warpgroup one
-inline void add_decode_tc(Program &P, int stage, const std::vector<tc::BBCell> &cells, uint64_t seed) {
-  std::vector<tc::BBCell> c4, c2;
-  for (auto &c : cells) (c.r_t <= 128 && g_dec_nwg.load() == 4 ? c4 : c2).push_back(c);
-  launch_decode<4>(P, stage, c4, seed);
-  launch_decode<2>(P, stage, c2, seed);
 }
 
 inline void fill_bb_common(tc::BBCell &b, const CellStore &cs, int *status) {

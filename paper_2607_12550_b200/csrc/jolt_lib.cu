@@ -27,7 +27,6 @@ namespace jolt {
 thread_local std::string g_err;
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_eig_smem{1};
-std::atomic<int> g_dec_nwg{2};      // 4: decode cells with r_t <= 128 on the four-warpgroup kernel (measured: no faster)
 long long *g_dbg_stamps = nullptr;   // device buffer for kernel cycle stamps (profiling aid)
 std::atomic<int> g_fast{7};   // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores
 

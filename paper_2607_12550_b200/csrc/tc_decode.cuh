@@ -16,23 +16,23 @@
 namespace jolt {
 namespace tc {
 
-// Two variants.  NWG = 2 epilogue warpgroups: any r_t <= 256 (P region 64 KB, 4-stage ring, one operand tile and
-// one accumulator per warpgroup).  For r_t <= 128 half of the P region is free and extends the ring to six stages
-// (three U_T tiles in flight), and each warpgroup owns TWO accumulators: the MMA thread issues the backbone of a
-// tile two tiles before its rotation, so backbones wait in TMEM instead of U_T tiles waiting in shared memory, and
-// a warpgroup only waits for the eight rotation MMAs of its tile.  NWG = 4: r_t <= 128 only (P region 32 KB,
-// 2-stage ring, four operand / staging tiles).  Both use 224 KB of shared memory, one CTA per SM.
+// Two epilogue warpgroups, a producer warpgroup (TMA thread, MMA thread), 224 KB of shared memory, one CTA per SM.
+// Any r_t <= 256: P region 64 KB, 4-stage U_T ring, one operand tile and one accumulator per warpgroup.  For
+// r_t <= 128 half of the P region is free and extends the ring to six stages (three U_T tiles in flight), and each
+// warpgroup owns TWO accumulators: the MMA thread issues the backbone of a tile two tiles before its rotation, so
+// backbones wait in TMEM instead of U_T tiles waiting in shared memory, and a warpgroup only waits for the eight
+// rotation MMAs of its tile.
 constexpr int DEC_H_BYTES = 32768;
-template <int NWG> struct DecLayout {
-  static constexpr int THREADS = (NWG + 1) * 128;
-  static constexpr int P_BYTES = NWG == 4 ? 32768 : 65536;
-  static constexpr int NS = NWG == 4 ? 2 : 4;                       // ring stages allocated
-  static constexpr int BIG_BYTES = NS * 16384 + NWG * 32768;        // ring + operand tiles (set-up operands first)
+constexpr int DEC_NWG = 2;
+struct DecLayout {
+  static constexpr int THREADS = (DEC_NWG + 1) * 128;
+  static constexpr int P_BYTES = 65536;
+  static constexpr int NS = 4;                                          // ring stages in the ring region proper
+  static constexpr int BIG_BYTES = NS * 16384 + DEC_NWG * 32768;        // ring + operand tiles (set-up operands first)
   static constexpr int SMEM_BYTES = P_BYTES + DEC_H_BYTES + BIG_BYTES + 1024 + 512;
-  static constexpr int TMEM_COLS = 512;     // NWG = 2 keeps two accumulators per warpgroup when r_t <= 128
-  // NWG = 2 moves registers from the producer warpgroup to the epilogue ones; NWG = 4 runs every thread at the
-  // launch allocation (96): 20 warps leave no slack in the register file for a blocking re-partition
-  static constexpr bool REPARTITION = NWG == 2;
+  static constexpr int TMEM_COLS = 512;     // two accumulators per warpgroup when r_t <= 128
+  // registers move from the producer warpgroup to the epilogue ones (12 warps: the register file has the slack a
+  // blocking re-partition needs)
   static constexpr int EPI_REGS = 216;
   static constexpr int PROD_REGS = 56;
 };
@@ -136,13 +136,12 @@ __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bu
 struct DecCtx {
   uint32_t bTfull, bTempty, bRready, t_acc, s_obuf;
   unsigned char *rbuf, *obuf;
-  bool sep_out;
   volatile int *abort_flag;
   int wg, nwg, rit, h, tile0, n_tiles, l, hd;
   float scale, pre;
 };
 
-// The per-tile loop of one epilogue warpgroup (tiles wg, wg+2, ...).
+// The per-tile loop of one epilogue warpgroup (tiles wg, wg+2, ...) with one accumulator per warpgroup (r_t > 128).
 template <int BITS>
 __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) {
   DecCodes<BITS> cur, nxt;
@@ -155,7 +154,7 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
     const int token = tt * 128 + x.rit;
     long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;
     if (dbg) dbg[0] = clock64();
-    if (tma_out && !x.sep_out) {   // shared buffer: the previous store must have read it before the operand is written
+    if (tma_out) {   // the operand tile doubles as staging buffer: the previous store must have read it first
       if (x.rit == 0) tma_store_wait_read();
       named_bar_sync(1 + x.wg, 128);
     }
@@ -173,10 +172,6 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
     if (dbg) dbg[3] = clock64();
     tc_fence_after();
     const long long off = (long long)x.l * c.osl + (long long)x.hd * c.osh + (long long)token * c.ost;
-    if (tma_out && x.sep_out) {    // own staging buffer: only now must the previous tile's store have drained
-      if (x.rit == 0) tma_store_wait_read();
-      named_bar_sync(1 + x.wg, 128);
-    }
     float va[2][32];
     if (ok) tmem_ld32(x.t_acc, va[0]);
 #pragma unroll
@@ -314,9 +309,9 @@ __device__ __forceinline__ bool dec_tile_loop_acc4(const BBCell &c, const DecCtx
   return ok;
 }
 
-template <int NWG>
-__global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(const BBCell *__restrict__ cells, uint64_t seed) {
-  using LY = DecLayout<NWG>;
+__global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBCell *__restrict__ cells, uint64_t seed) {
+  using LY = DecLayout;
+  constexpr int NWG = DEC_NWG;
   constexpr int DEC_P_BYTES = LY::P_BYTES, DEC_BIG_BYTES = LY::BIG_BYTES, DEC_NS = LY::NS;
   extern __shared__ unsigned char smem_raw[];
   const BBCell &c = cells[blockIdx.y];
@@ -353,8 +348,8 @@ __global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(cons
   // r_t <= 128 leaves half of the P region and half of the ring free: each warpgroup then stages its output in a
   // buffer of its own, so a tile's unpack never waits for the previous tile's TMA store to drain
   // r_t <= 128 with two warpgroups: four accumulators and a six-stage ring (see the top of the file)
-  const bool acc4 = NWG == 2 && nkt <= 2;
-  const int ns = NWG == 4 ? 2 : (acc4 ? 6 : DEC_NS);
+  const bool acc4 = nkt <= 2;
+  const int ns = acc4 ? 6 : DEC_NS;
   auto sStage = [=](int s) { return s < 4 ? sRing + (uint32_t)s * BB_STAGE_BYTES : sP + 32768u + (uint32_t)(s - 4) * BB_STAGE_BYTES; };
 
   if (threadIdx.x == 0) {
@@ -371,7 +366,7 @@ __global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(cons
   const uint32_t tmem_base = *tmem_slot;
 
   if (wg == NWG) {
-    if constexpr (LY::REPARTITION) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(LY::PROD_REGS));
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(LY::PROD_REGS));
     if (warp == NWG * 4 && lane == 0) {
       // ---------------- TMA producer
       tma_prefetch_desc(&c.tmUT); tma_prefetch_desc(&c.tmUF); tma_prefetch_desc(&c.tmG);
@@ -464,7 +459,7 @@ __global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(cons
     }
   } else {
     // ---------------- epilogue warpgroups
-    if constexpr (LY::REPARTITION) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(LY::EPI_REGS));
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(LY::EPI_REGS));
     const int q = warp & 3;
     const int rit = q * 32 + lane;                 // row in tile
     const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -519,7 +514,7 @@ __global__ void __launch_bounds__(DecLayout<NWG>::THREADS, 1) decode_kernel(cons
     if (ok) {
       DecCtx x;
       x.bTfull = bTfull(wg); x.bTempty = bTempty(wg); x.bRready = bRready(wg);
-      x.t_acc = t_lane + wg * 128; x.rbuf = smR + wg * 32768; x.sep_out = false;
+      x.t_acc = t_lane + wg * 128; x.rbuf = smR + wg * 32768;
       x.s_obuf = sR + wg * 32768; x.obuf = x.rbuf;
       x.abort_flag = abort_flag; x.wg = wg; x.nwg = NWG; x.rit = rit; x.h = h; x.tile0 = tile0; x.n_tiles = n_tiles;
       x.l = h / c.n_heads; x.hd = h - x.l * c.n_heads; x.scale = scale; x.pre = pre;
