@@ -1109,77 +1109,92 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     build_factor_program(PG[g], sub, mode, false, power_iters, o->seed, fast, subspace);
   }
   lap("factor program");
-  std::vector<StoreJob> sj;
-  for (int i = 0; i < nc; ++i) {
-    const CellDesc &c = cells[i];
-    const CellStore &cs = H->cells[i];
-    if (c.r_t == 0) continue;
-    StoreJob j;
-    j.G32 = ws[i].G32; j.UT32 = ws[i].UT32; j.UF32 = ws[i].UF32;
-    j.G16 = cs.G16; j.UT16 = cs.UT16; j.UF16 = cs.UF16; j.e = cs.e;
-    j.nG = (long long)c.m * c.r_t * c.r_f; j.nUT = (long long)c.T * c.r_t; j.nUF = (long long)kD * c.r_f; j.round_inputs = 0;
-    sj.push_back(j);
-  }
-  if (!sj.empty()) {
-    const size_t off = P.push(sj);
-    const int n = (int)sj.size();
-    P.add(ST_STORE, [=](char *dev_t, cudaStream_t s) {
-      core_exponent_kernel<<<n, 1024, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
-      store_factors_kernel<<<dim3(64, n), 256, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
-    });
-  }
-  // residual / rotate / quantise / pack: tensor-core kernel where the cell fits it, portable kernels otherwise
+  // fp16 storage of the factors and the residual / rotate / quantise / pack pass (tensor-core kernel where the cell
+  // fits it, portable kernels otherwise).  With several cell groups each group's program ends with the tail of its
+  // own cells, so only the last group's tail is left when the others have finished.
   std::vector<char> use_tc(nc, 0);
-  int tc_heads = 0;
   const bool x_tma_ok = L->dtype == JOLT_F16 && L->stride_token * 2 % 16 == 0 && L->stride_head * 2 % 16 == 0 &&
                         L->stride_layer * 2 % 16 == 0;
   for (int i = 0; i < nc; ++i) {
     CellStore &cs = H->cells[i];
-    if (fast && encode_store_maps(cs) && x_tma_ok && cells[i].bits > 0 && ((uintptr_t)cells[i].X % 16 == 0)) {
-      use_tc[i] = 1;
-      tc_heads += cells[i].m;
-    }
+    if (fast && encode_store_maps(cs) && x_tma_ok && cells[i].bits > 0 && ((uintptr_t)cells[i].X % 16 == 0)) use_tc[i] = 1;
   }
-  std::vector<tc::BBCell> bbc;
-  std::vector<BackboneRef> br_port;
-  std::vector<RowJob> rj;
-  long long rows = 0;
-  int tpi = 1, iph = 1;
-  bb_split(tc_heads, L->seq_len / 128, tpi, iph);
-  for (int i = 0; i < nc; ++i) {
-    const CellDesc &c = cells[i];
-    const CellStore &cs = H->cells[i];
-    if (use_tc[i]) {
-      tc::BBCell b;
-      fill_bb_common(b, cs, d_status + 4 * i);
-      b.tiles_per_item = tpi; b.items_per_head = iph;
-      const int g = i / 2;
-      const int Lg = L->group_start[g + 1] - L->group_start[g];
-      const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)c.T, (uint64_t)c.n_heads, (uint64_t)Lg};
-      const uint64_t str[3] = {(uint64_t)c.st * 2, (uint64_t)c.sh * 2, (uint64_t)c.sl * 2};
-      const uint32_t box[4] = {64, 128, 1, 1};
-      if (!make_tmap_f16(&b.tmX, c.X, 4, dims, str, box)) { use_tc[i] = 0; }
-      else { bbc.push_back(b); continue; }
+  auto build_tail = [&](Program &PP, const std::vector<int> &idx) {
+    std::vector<StoreJob> sj;
+    for (int i : idx) {
+      const CellDesc &c = cells[i];
+      const CellStore &cs = H->cells[i];
+      if (c.r_t == 0) continue;
+      StoreJob j;
+      j.G32 = ws[i].G32; j.UT32 = ws[i].UT32; j.UF32 = ws[i].UF32;
+      j.G16 = cs.G16; j.UT16 = cs.UT16; j.UF16 = cs.UF16; j.e = cs.e;
+      j.nG = (long long)c.m * c.r_t * c.r_f; j.nUT = (long long)c.T * c.r_t; j.nUF = (long long)kD * c.r_f; j.round_inputs = 0;
+      sj.push_back(j);
     }
-    if (c.bits == 0) continue;
-    if (c.r_t > 0) br_port.push_back({ws[i].c, cs.G16, cs.UT16, cs.UF16, cs.e, ws[i].P16, ws[i].Xt});
-    RowJob j;
-    memset(&j, 0, sizeof j);
-    j.c = ws[i].c; j.Xt = c.r_t > 0 ? ws[i].Xt : nullptr;
-    j.words = cs.words; j.scales = cs.scales; j.status = d_status + 4 * i; j.row0 = rows;
-    rows += (long long)c.m * c.T;
-    rj.push_back(j);
-  }
-  add_backbone_tc<true>(P, ST_RQ, bbc, o->seed);
-  add_backbone(P, ST_BACK, br_port);
-  if (!rj.empty()) {
-    const size_t off = P.push(rj);
-    const uint64_t seed = o->seed;
-    const int nj = (int)rj.size();
-    P.add(ST_RQ, [=](char *dev_t, cudaStream_t s) {
-      residual_quant_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, s>>>((const RowJob *)(dev_t + off), nj, rows, seed);
-      LAUNCHED();
-    });
+    if (!sj.empty()) {
+      const size_t off = PP.push(sj);
+      const int n = (int)sj.size();
+      PP.add(ST_STORE, [=](char *dev_t, cudaStream_t s) {
+        core_exponent_kernel<<<n, 1024, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
+        store_factors_kernel<<<dim3(64, n), 256, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
+      });
+    }
+    int tc_heads = 0;
+    for (int i : idx) if (use_tc[i]) tc_heads += cells[i].m;
+    std::vector<tc::BBCell> bbc;
+    std::vector<BackboneRef> br_port;
+    std::vector<RowJob> rj;
+    long long rows = 0;
+    int tpi = 1, iph = 1;
+    bb_split(tc_heads, L->seq_len / 128, tpi, iph);
+    for (int i : idx) {
+      const CellDesc &c = cells[i];
+      const CellStore &cs = H->cells[i];
+      if (use_tc[i]) {
+        tc::BBCell b;
+        fill_bb_common(b, cs, d_status + 4 * i);
+        b.tiles_per_item = tpi; b.items_per_head = iph;
+        const int g = i / 2;
+        const int Lg = L->group_start[g + 1] - L->group_start[g];
+        const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)c.T, (uint64_t)c.n_heads, (uint64_t)Lg};
+        const uint64_t str[3] = {(uint64_t)c.st * 2, (uint64_t)c.sh * 2, (uint64_t)c.sl * 2};
+        const uint32_t box[4] = {64, 128, 1, 1};
+        if (make_tmap_f16(&b.tmX, c.X, 4, dims, str, box)) { bbc.push_back(b); continue; }
+      }
+      if (c.bits == 0) continue;
+      if (c.r_t > 0) br_port.push_back({ws[i].c, cs.G16, cs.UT16, cs.UF16, cs.e, ws[i].P16, ws[i].Xt});
+      RowJob j;
+      memset(&j, 0, sizeof j);
+      j.c = ws[i].c; j.Xt = c.r_t > 0 ? ws[i].Xt : nullptr;
+      j.words = cs.words; j.scales = cs.scales; j.status = d_status + 4 * i; j.row0 = rows;
+      rows += (long long)c.m * c.T;
+      rj.push_back(j);
+    }
+    add_backbone_tc<true>(PP, ST_RQ, bbc, o->seed);
+    add_backbone(PP, ST_BACK, br_port);
+    if (!rj.empty()) {
+      const size_t off = PP.push(rj);
+      const uint64_t seed = o->seed;
+      const int nj = (int)rj.size();
+      PP.add(ST_RQ, [=](char *dev_t, cudaStream_t s) {
+        residual_quant_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, s>>>((const RowJob *)(dev_t + off), nj, rows, seed);
+        LAUNCHED();
+      });
+    }
+  };
+  if (n_groups > 1) {
+    std::vector<int> rest;
+    for (int g = 0; g < n_groups; ++g) {
+      std::vector<int> idx;
+      for (int i = 0; i < nc; ++i) if (cell_group[i] == g) idx.push_back(i);
+      build_tail(PG[g], idx);
+    }
+    for (int i = 0; i < nc; ++i) if (cell_group[i] < 0) rest.push_back(i);
+    build_tail(P, rest);
+  } else {
+    std::vector<int> all(nc);
+    for (int i = 0; i < nc; ++i) all[i] = i;
+    build_tail(P, all);
   }
   void *d_tab = nullptr;
   std::vector<size_t> tab_off(PG.size() + 1, 0);

@@ -598,15 +598,29 @@ __global__ void __launch_bounds__(256, 1) tall_gram_kernel(const TallGramJob *__
   for (int i = 0; i < TI; ++i)
 #pragma unroll
     for (int j = 0; j < TI; ++j) acc[i][j] = 0.0;
-  for (int r0 = r_begin; r0 < r_end; r0 += 16) {
+  // the 16 x W tile is TI elements per thread (and per operand); the next tile's elements are fetched into registers
+  // while the current one is being multiplied, so the global-load latency hides behind the 16 * TI * TI FMAs
+  float pa[TI], pb[TI];
+  auto fetch = [&](int r0) {
     const int nr = min(16, r_end - r0);
-    for (int e = tid; e < 16 * W; e += 256) {
-      const int r = e / W, c = e - r * W;
+#pragma unroll
+    for (int u = 0; u < TI; ++u) {
+      const int e = tid + u * 256, r = e / W, c = e - r * W;
       const float *row = t.M + (size_t)(r0 + r) * t.k;
-      Ma[r][c] = (r < nr && c < t.wa) ? (double)row[t.ca + c] : 0.0;
-      if (!same) Mb[r][c] = (r < nr && c < t.wb) ? (double)row[t.cb + c] : 0.0;
+      pa[u] = (r < nr && c < t.wa) ? row[t.ca + c] : 0.f;
+      if (!same) pb[u] = (r < nr && c < t.wb) ? row[t.cb + c] : 0.f;
+    }
+  };
+  if (r_begin < r_end) fetch(r_begin);
+  for (int r0 = r_begin; r0 < r_end; r0 += 16) {
+#pragma unroll
+    for (int u = 0; u < TI; ++u) {
+      const int e = tid + u * 256, r = e / W, c = e - r * W;
+      Ma[r][c] = (double)pa[u];
+      if (!same) Mb[r][c] = (double)pb[u];
     }
     __syncthreads();
+    if (r0 + 16 < r_end) fetch(r0 + 16);
 #pragma unroll 4
     for (int r = 0; r < 16; ++r) {
       double a[TI], b[TI];
