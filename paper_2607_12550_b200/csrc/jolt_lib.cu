@@ -265,19 +265,24 @@ GemmTask mk(const void *A, int ta, long long a_rs, long long a_cs, const void *B
 
 void add_gemm(Program &P, int stage, const std::vector<GemmTask> &all_tasks, bool f64) {
   if (all_tasks.empty()) return;
-  // one launch per tile-count class: a grid sized for the largest task would start mostly empty CTAs for the rest
-  std::vector<std::pair<long long, std::vector<GemmTask>>> buckets;
+  // one launch per tile-count class: a grid sized for the largest task would start mostly empty CTAs for the rest.
+  // Plain fp32 tasks take the register-tiled kernel (128 x 64 tiles), everything else the generic one (64 x 64).
+  struct Bucket { long long key; bool fast; std::vector<GemmTask> tasks; };
+  std::vector<Bucket> buckets;
   for (auto &t : all_tasks) {
     if (t.M <= 0 || t.N <= 0) continue;
-    const long long key = ((long long)((t.M + 63) / 64) << 32) | (long long)((t.N + 63) / 64);
+    const bool fastk = !f64 && sgemm_fast_ok(t);
+    const int bm = fastk ? 128 : 64;
+    const long long key = ((long long)((t.M + bm - 1) / bm) << 32) | (long long)((t.N + 63) / 64);
     size_t b = 0;
-    for (; b < buckets.size(); ++b) if (buckets[b].first == key) break;
-    if (b == buckets.size()) buckets.push_back({key, {}});
-    buckets[b].second.push_back(t);
+    for (; b < buckets.size(); ++b) if (buckets[b].key == key && buckets[b].fast == fastk) break;
+    if (b == buckets.size()) buckets.push_back({key, fastk, {}});
+    buckets[b].tasks.push_back(t);
   }
   for (auto &bk : buckets) {
-    const std::vector<GemmTask> &tasks = bk.second;
-    const int tm = (int)(bk.first >> 32), tn = (int)(bk.first & 0xffffffff);
+    const std::vector<GemmTask> &tasks = bk.tasks;
+    const int tm = (int)(bk.key >> 32), tn = (int)(bk.key & 0xffffffff);
+    const bool fastk = bk.fast;
     const size_t off = P.push(tasks);
     const int n = (int)tasks.size();
     P.add(stage, [=](char *dev, cudaStream_t s) {
@@ -285,6 +290,7 @@ void add_gemm(Program &P, int stage, const std::vector<GemmTask> &all_tasks, boo
       for (int z0 = 0; z0 < n; z0 += 32768) {
         dim3 grid(tn, tm, std::min(32768, n - z0));
         if (f64) simt_gemm_kernel<double><<<grid, 256, 0, s>>>(d + z0);
+        else if (fastk) simt_sgemm_kernel<<<grid, 256, 0, s>>>(d + z0);
         else simt_gemm_kernel<float><<<grid, 256, 0, s>>>(d + z0);
         LAUNCHED();
       }

@@ -106,4 +106,87 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const GemmTask *__restri
   }
 }
 
+// fp32 in, fp32 out, one K segment, no accumulate: 128 x 64 tiles, 8 x 4 results per thread read from shared memory
+// as 16-byte vectors, the next K slab fetched into registers while the current one is multiplied.
+inline bool sgemm_fast_ok(const GemmTask &t) {
+  return t.ta == DT_F32 && t.tb == DT_F32 && t.tc == DT_F32 && t.nseg == 1 && !t.accumulate && !t.alpha_exp;
+}
+
+__global__ void __launch_bounds__(256, 2) simt_sgemm_kernel(const GemmTask *__restrict__ tasks) {
+  constexpr int BM = 128, BN = 64, BK = 16;
+  const GemmTask t = tasks[blockIdx.z];
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  if (m0 >= t.M || n0 >= t.N) return;
+  __shared__ __align__(16) float As[BK][BM + 4];
+  __shared__ __align__(16) float Bs[BK][BN + 4];
+  const int tid = threadIdx.x;
+  const int tx = tid & 15, ty = tid >> 4;
+  const float *A = (const float *)t.A, *B = (const float *)t.B;
+  const bool a_kfast = (t.a_cs == 1), b_kfast = (t.b_rs == 1);
+  float acc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  float pa[8], pb[4];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int idx = tid + e * 256;
+      int i, kk;
+      if (a_kfast) { i = idx >> 4; kk = idx & 15; } else { kk = idx >> 7; i = idx & 127; }
+      pa[e] = (m0 + i < t.M && k0 + kk < t.K) ? A[(long long)(m0 + i) * t.a_rs + (long long)(k0 + kk) * t.a_cs] : 0.f;
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int idx = tid + e * 256;
+      int j, kb;
+      if (b_kfast) { j = idx >> 4; kb = idx & 15; } else { kb = idx >> 6; j = idx & 63; }
+      pb[e] = (n0 + j < t.N && k0 + kb < t.K) ? B[(long long)(k0 + kb) * t.b_rs + (long long)(n0 + j) * t.b_cs] : 0.f;
+    }
+  };
+  fetch(0);
+  for (int k0 = 0; k0 < t.K; k0 += BK) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int idx = tid + e * 256;
+      int i, kk;
+      if (a_kfast) { i = idx >> 4; kk = idx & 15; } else { kk = idx >> 7; i = idx & 127; }
+      As[kk][i] = pa[e];
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int idx = tid + e * 256;
+      int j, kb;
+      if (b_kfast) { j = idx >> 4; kb = idx & 15; } else { kb = idx >> 6; j = idx & 63; }
+      Bs[kb][j] = pb[e];
+    }
+    __syncthreads();
+    if (k0 + BK < t.K) fetch(k0 + BK);
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      const float4 a0 = *(const float4 *)&As[kk][ty * 8], a1 = *(const float4 *)&As[kk][ty * 8 + 4];
+      const float4 b4 = *(const float4 *)&Bs[kk][tx * 4];
+      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  float *C = (float *)t.C;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = m0 + ty * 8 + i;
+    if (r >= t.M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int c = n0 + tx * 4 + j;
+      if (c < t.N) C[(long long)r * t.c_rs + (long long)c * t.c_cs] = acc[i][j] * t.alpha;
+    }
+  }
+}
+
 }  // namespace jolt
