@@ -449,7 +449,7 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
         if (tok_segments(c.T) > 1) w.Zpart = b.take<float>((size_t)tok_segments(c.T) * c.m * kD * k);
       }
       w.Gs = b.take<double>(k * k); w.Lwork = k > (size_t)kCholSmemMaxN ? b.take<double>(k * (k + 1)) : nullptr;
-      w.gpart = b.take<double>(kGramChunks * k * k); w.LT32 = b.take<float>(k * (k + 4)); w.invd = b.take<float>(k + 4);
+      w.gpart = b.take<double>(kGramChunks * k * k); w.LT32 = b.take<float>(k * (k + 8)); w.invd = b.take<float>(k + 8);
       w.BBt = b.take<double>(k * k); w.BBv = b.take<double>(k * k); w.BBw = b.take<double>(k);
       w.Ut = b.take<float>(k * std::max<size_t>(c.r_t, 1));
       if (!(real && w.sigma)) w.sigma = b.take<float>(k);
@@ -555,9 +555,9 @@ void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side,
         cholesky_smem_kernel<<<n, 512, sh1, s>>>((const CholSmemTask *)(dev + o1), glob); LAUNCHED();
         const dim3 grid((max_rows + rb - 1) / rb, n);
         const TrsmJob *jobs = (const TrsmJob *)(dev + o2);
-        if (rb == 256) trsm_rows_kernel<256><<<grid, 256, sh2, s>>>(jobs, glob);
-        else if (rb == 128) trsm_rows_kernel<128><<<grid, 128, sh2, s>>>(jobs, glob);
-        else trsm_rows_kernel<64><<<grid, 64, sh2, s>>>(jobs, glob);
+        if (rb == 256) trsm_rows_kernel<256><<<grid, 128, sh2, s>>>(jobs, glob);
+        else if (rb == 128) trsm_rows_kernel<128><<<grid, 64, sh2, s>>>(jobs, glob);
+        else trsm_rows_kernel<64><<<grid, 32, sh2, s>>>(jobs, glob);
         LAUNCHED();
       });
     }

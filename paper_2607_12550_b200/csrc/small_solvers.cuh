@@ -336,7 +336,7 @@ __global__ void __launch_bounds__(kEigThreads, 1) jacobi_eig_smem_kernel(const E
 // cholesky_smem_kernel: G = L L^T in fp64.  A pivot that is not above 1e-10 of its original diagonal entry is
 // deflated (the column of L is zeroed, the diagonal set to 1, status bit 2): rank-deficient sketches lose the
 // dependent directions instead of dividing by rounding noise.  Writes
-// LT[l][j] = L[j][l] (fp32, pitch kp = n rounded up to 4, zero above the diagonal of L) and invd[j] = 1 / L[j][j]
+// LT[l][j] = L[j][l] (fp32, pitch kp = n rounded up to 8, zero above the diagonal of L) and invd[j] = 1 / L[j][j]
 // (0 for a dead pivot).  trsm_rows_kernel then solves  dst_row * L^T = src_row  for 128 rows per CTA.
 constexpr int kCholSmemMaxN = 168;
 
@@ -452,7 +452,7 @@ __global__ void __launch_bounds__(512, 1) cholesky_smem_kernel(const CholSmemTas
     }
     __syncthreads();
   }
-  const int kp = (n + 3) & ~3;
+  const int kp = (n + 7) & ~7;
   for (int e = tid; e < n * kp; e += nt) {
     const int l = e / kp, j = e - l * kp;
     t.LT[e] = (j < n && j >= l) ? (float)A[j * ld + l] : 0.f;
@@ -468,17 +468,19 @@ inline size_t chol_smem_bytes(int n, bool in_global = false) {
 struct TrsmJob { const float *src; float *dst; int rows, k; const float *LT; const float *invd; };
 
 inline size_t trsm_smem_bytes(int k, int rb, bool lt_global = false) {
-  const int kp = (k + 3) & ~3;
+  const int kp = (k + 7) & ~7;
   return ((lt_global ? 0 : (size_t)k * kp) + (size_t)kp * (rb + 1) + kp) * sizeof(float) + 64;
 }
 
-// RB rows (= threads) per CTA: 256 when the tile fits shared memory, else 128
+// RB rows per CTA (256 when the tile fits shared memory, else 128 or 64), RB / 2 threads: a thread solves two rows,
+// eight columns at a time, so that one pair of 16-byte loads of L^T feeds 16 FMAs.
 template <int RB>
-__global__ void __launch_bounds__(RB) trsm_rows_kernel(const TrsmJob *__restrict__ jobs, int lt_global) {
+__global__ void __launch_bounds__(RB / 2) trsm_rows_kernel(const TrsmJob *__restrict__ jobs, int lt_global) {
+  constexpr int NT = RB / 2;
   const TrsmJob t = jobs[blockIdx.y];
   const int r0 = blockIdx.x * RB;
   if (r0 >= t.rows) return;
-  const int k = t.k, kp = (k + 3) & ~3;
+  const int k = t.k, kp = (k + 7) & ~7;
   constexpr int PITCH = RB + 1;
   extern __shared__ float shf[];
   // L^T stays in global memory (read through L1, every lane of a warp reads the same entries) when it does not fit
@@ -489,33 +491,33 @@ __global__ void __launch_bounds__(RB) trsm_rows_kernel(const TrsmJob *__restrict
   const float *__restrict__ LT = lt_global ? t.LT : LTs;
   const int tid = threadIdx.x;
   const int nrows = min(RB, t.rows - r0);
-  // staging loops read eight elements into registers before the first shared-memory store, so that the global
+  // staging loops read several elements into registers before the first shared-memory store, so that the global
   // loads of a trip are in flight together
   if (!lt_global) {
     const float4 *g4 = (const float4 *)t.LT;
     float4 *s4 = (float4 *)LTs;
     const int n4 = k * kp / 4;
-    for (int e0 = tid; e0 < n4; e0 += RB * 4) {
+    for (int e0 = tid; e0 < n4; e0 += NT * 4) {
       float4 v[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) { const int e = e0 + u * RB; if (e < n4) v[u] = g4[e]; }
+      for (int u = 0; u < 4; ++u) { const int e = e0 + u * NT; if (e < n4) v[u] = g4[e]; }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) { const int e = e0 + u * RB; if (e < n4) s4[e] = v[u]; }
+      for (int u = 0; u < 4; ++u) { const int e = e0 + u * NT; if (e < n4) s4[e] = v[u]; }
     }
   }
-  for (int j = tid; j < kp; j += RB) invd[j] = j < k ? t.invd[j] : 0.f;
+  for (int j = tid; j < kp; j += NT) invd[j] = j < k ? t.invd[j] : 0.f;
   const float *src = t.src + (size_t)r0 * k;
   const int tot = nrows * k;
   if ((((size_t)r0 * k) & 3) == 0) {          // the row block starts on a 16-byte boundary: vector loads
     const float4 *src4 = (const float4 *)src;
     const int tot4 = tot >> 2;
-    for (int e0 = tid; e0 < tot4; e0 += RB * 8) {
+    for (int e0 = tid; e0 < tot4; e0 += NT * 8) {
       float4 v[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) { const int e = e0 + u * RB; if (e < tot4) v[u] = src4[e]; }
+      for (int u = 0; u < 8; ++u) { const int e = e0 + u * NT; if (e < tot4) v[u] = src4[e]; }
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
-        const int e = e0 + u * RB;
+        const int e = e0 + u * NT;
         if (e < tot4) {
           int r = (4 * e) / k, j = 4 * e - r * k;
           const float vv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
@@ -524,44 +526,54 @@ __global__ void __launch_bounds__(RB) trsm_rows_kernel(const TrsmJob *__restrict
         }
       }
     }
-    for (int e = (tot4 << 2) + tid; e < tot; e += RB) { const int r = e / k, j = e - r * k; sp[j * PITCH + r] = src[e]; }
+    for (int e = (tot4 << 2) + tid; e < tot; e += NT) { const int r = e / k, j = e - r * k; sp[j * PITCH + r] = src[e]; }
   } else {
-    for (int e0 = tid; e0 < tot; e0 += RB * 8) {
+    for (int e0 = tid; e0 < tot; e0 += NT * 8) {
       float v[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) { const int e = e0 + u * RB; v[u] = e < tot ? src[e] : 0.f; }
+      for (int u = 0; u < 8; ++u) { const int e = e0 + u * NT; v[u] = e < tot ? src[e] : 0.f; }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) { const int e = e0 + u * RB; if (e < tot) { const int r = e / k, j = e - r * k; sp[j * PITCH + r] = v[u]; } }
+      for (int u = 0; u < 8; ++u) { const int e = e0 + u * NT; if (e < tot) { const int r = e / k, j = e - r * k; sp[j * PITCH + r] = v[u]; } }
     }
   }
-  for (int e = tid; e < (kp - k) * PITCH; e += RB) sp[k * PITCH + e] = 0.f;
+  for (int e = tid; e < (kp - k) * PITCH; e += NT) sp[k * PITCH + e] = 0.f;
   __syncthreads();
   if (tid < nrows) {
-    const int r = tid;
-    for (int jb = 0; jb < kp; jb += 4) {
-      float a0 = sp[(jb + 0) * PITCH + r], a1 = sp[(jb + 1) * PITCH + r], a2 = sp[(jb + 2) * PITCH + r], a3 = sp[(jb + 3) * PITCH + r];
-      // jb is a multiple of 4: four finished columns per trip, all loads of a trip issued before its 16 FMAs
-#pragma unroll 2
-      for (int l = 0; l < jb; l += 4) {
-        float x[4]; float4 L4[4];
+    const int ra = tid, rb = tid + NT;            // row rb may lie beyond the ragged end: computed, never written out
+    for (int jb = 0; jb < kp; jb += 8) {
+      float a[8], b[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { x[u] = sp[(l + u) * PITCH + r]; L4[u] = *(const float4 *)&LT[(l + u) * kp + jb]; }
+      for (int c = 0; c < 8; ++c) { a[c] = sp[(jb + c) * PITCH + ra]; b[c] = sp[(jb + c) * PITCH + rb]; }
+      // jb is a multiple of 8: four finished columns per trip, all loads of a trip issued before its 64 FMAs
+      for (int l = 0; l < jb; l += 4) {
+        float xa[4], xb[4]; float4 L0[4], L1[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          a0 = fmaf(-x[u], L4[u].x, a0); a1 = fmaf(-x[u], L4[u].y, a1); a2 = fmaf(-x[u], L4[u].z, a2); a3 = fmaf(-x[u], L4[u].w, a3);
+          xa[u] = sp[(l + u) * PITCH + ra]; xb[u] = sp[(l + u) * PITCH + rb];
+          L0[u] = *(const float4 *)&LT[(l + u) * kp + jb]; L1[u] = *(const float4 *)&LT[(l + u) * kp + jb + 4];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float Lv[8] = {L0[u].x, L0[u].y, L0[u].z, L0[u].w, L1[u].x, L1[u].y, L1[u].z, L1[u].w};
+#pragma unroll
+          for (int c = 0; c < 8; ++c) { a[c] = fmaf(-xa[u], Lv[c], a[c]); b[c] = fmaf(-xb[u], Lv[c], b[c]); }
         }
       }
-      a0 *= invd[jb];
-      a1 = fmaf(-a0, LT[(jb + 0) * kp + jb + 1], a1); a1 *= invd[jb + 1];
-      a2 = fmaf(-a0, LT[(jb + 0) * kp + jb + 2], a2); a2 = fmaf(-a1, LT[(jb + 1) * kp + jb + 2], a2); a2 *= invd[jb + 2];
-      a3 = fmaf(-a0, LT[(jb + 0) * kp + jb + 3], a3); a3 = fmaf(-a1, LT[(jb + 1) * kp + jb + 3], a3);
-      a3 = fmaf(-a2, LT[(jb + 2) * kp + jb + 3], a3); a3 *= invd[jb + 3];
-      sp[(jb + 0) * PITCH + r] = a0; sp[(jb + 1) * PITCH + r] = a1; sp[(jb + 2) * PITCH + r] = a2; sp[(jb + 3) * PITCH + r] = a3;
+      // the 8 x 8 triangle of the block itself
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+#pragma unroll
+        for (int i = 0; i < c; ++i) { const float Lic = LT[(jb + i) * kp + jb + c]; a[c] = fmaf(-a[i], Lic, a[c]); b[c] = fmaf(-b[i], Lic, b[c]); }
+        const float d = invd[jb + c];
+        a[c] *= d; b[c] *= d;
+      }
+#pragma unroll
+      for (int c = 0; c < 8; ++c) { sp[(jb + c) * PITCH + ra] = a[c]; sp[(jb + c) * PITCH + rb] = b[c]; }
     }
   }
   __syncthreads();
   float *dst = t.dst + (size_t)r0 * k;
-  for (int e = tid; e < nrows * k; e += RB) { const int r = e / k, j = e - r * k; dst[e] = sp[j * PITCH + r]; }
+  for (int e = tid; e < nrows * k; e += NT) { const int r = e / k, j = e - r * k; dst[e] = sp[j * PITCH + r]; }
 }
 
 // sum of fp64 partials with a per-job element count
