@@ -52,9 +52,12 @@ __device__ __forceinline__ void quantize_pack_row(float (&r)[128], const uint32_
     int nb = 0, wi = 0;
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
-      float q = floorf(__fmul_rn(r[g * 32 + j], inv));
-      q = fminf(fmaxf(q, -half_levels), half_levels - 1.0f) + half_levels;
-      const uint32_t u = (delta == 0.f) ? (uint32_t)half_levels : (uint32_t)q;
+      // clamp(floor(v), -L, L-1) + L without a rounding or conversion instruction (both run on the quarter-rate
+      // pipe and bound this pass): clamp v to [-L, L - 1/2] first (same result: floor is monotone), then one
+      // round-toward-zero add of 2^23 + L leaves floor(v + L) in the low mantissa bits of a positive float
+      const float v = fminf(fmaxf(__fmul_rn(r[g * 32 + j], inv), -half_levels), half_levels - 0.5f);
+      const uint32_t code = __float_as_uint(__fadd_rz(v, 8388608.0f + half_levels)) & 0x1FFu;
+      const uint32_t u = (delta == 0.f) ? (uint32_t)half_levels : code;
       accw |= (uint64_t)u << nb;
       nb += BITS;
       if (nb >= 32) { words[g * BITS + wi] = (uint32_t)accw; accw >>= 32; nb -= 32; ++wi; }
