@@ -39,7 +39,9 @@ enum { JOLT_K = 0, JOLT_V = 1 };
 /* Shape and strides shared by the K and the V tensor (paper Sec. 4: "partition the L layers into G
  * contiguous groups").  Element (layer l, head n, token t, feature f) sits at
  * l*stride_layer + n*stride_head + t*stride_token + f (in elements; the feature stride is 1).
- * head_dim must be 128; seq_len a multiple of 128; stride_token a multiple of 8.
+ * head_dim must be 128; seq_len a multiple of 128; all strides multiples of 8 elements; device tensors must start on
+ * a 16-byte boundary (JOLT_EINVAL otherwise: the kernels use 16-byte vector accesses); host tensors are staged and
+ * may start anywhere.
  * group_start has n_groups + 1 ascending entries, group_start[0] = 0, group_start[n_groups] = n_layers. */
 typedef struct {
   int32_t n_layers, n_kv_heads, seq_len, head_dim;

@@ -36,7 +36,7 @@ int static_scratch_address(int dev, char **out) {
 extern "C" int jolt_decompress_static(const jolt_handle *H, const jolt_layout *L, void *Kout, void *Vout, void *stream) {
   if (!H || !Kout || !Vout) return fail(JOLT_EINVAL, "null argument");
   int rc;
-  if ((rc = check_layout(L))) return rc;
+  if ((rc = check_layout(L)) || (rc = check_device_alignment(L, Kout, Vout))) return rc;
   if (L->mem_space != JOLT_MEM_DEVICE) return fail(JOLT_EUNSUPPORTED, "the allocation-free decode writes device memory only");
   if (L->n_layers != H->n_layers || L->n_kv_heads != H->n_kv_heads || L->seq_len != H->T || L->n_groups != H->n_groups)
     return fail(JOLT_EINVAL, "output layout does not match the compressed cache");

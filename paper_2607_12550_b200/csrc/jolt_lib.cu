@@ -213,6 +213,13 @@ static int check_layout(const jolt_layout *L) {
   return JOLT_OK;
 }
 
+// Device tensors are read and written with 16-byte vector accesses (strides are multiples of 8 elements already).
+static int check_device_alignment(const jolt_layout *L, const void *a, const void *b) {
+  if (L->mem_space == JOLT_MEM_DEVICE && ((((uintptr_t)a) | ((uintptr_t)b)) & 15))
+    return fail(JOLT_EINVAL, "device tensors must start on a 16-byte boundary");
+  return JOLT_OK;
+}
+
 static size_t layout_span_elems(const jolt_layout *L) {
   return (size_t)(L->n_layers - 1) * L->stride_layer + (size_t)(L->n_kv_heads - 1) * L->stride_head +
          (size_t)(L->seq_len - 1) * L->stride_token + kD;
@@ -999,7 +1006,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   const bool dbg = getenv("JOLT_DEBUG_TIMING") != nullptr;
   auto t_start = std::chrono::steady_clock::now();
   auto lap = [&](const char *what) { if (dbg) { auto n = std::chrono::steady_clock::now(); fprintf(stderr, "[jolt] %s: %.3f ms\n", what, std::chrono::duration<double, std::milli>(n - t_start).count()); t_start = n; } };
-  if ((rc = check_layout(L)) || (rc = check_options(o))) return rc;
+  if ((rc = check_layout(L)) || (rc = check_options(o)) || (rc = check_device_alignment(L, K, V))) return rc;
   const bool injected = inUT != nullptr || inUF != nullptr;
   if (injected && (!inUT || !inUF)) return fail(JOLT_EINVAL, "both factor arrays are needed");
   cudaStream_t st = (cudaStream_t)stream;
@@ -1305,7 +1312,7 @@ extern "C" int jolt_compress_with_factors(const jolt_layout *L, const void *K, c
 extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void *Kout, void *Vout, void *stream) {
   if (!H || !Kout || !Vout) return fail(JOLT_EINVAL, "null argument");
   int rc;
-  if ((rc = check_layout(L))) return rc;
+  if ((rc = check_layout(L)) || (rc = check_device_alignment(L, Kout, Vout))) return rc;
   if (L->n_layers != H->n_layers || L->n_kv_heads != H->n_kv_heads || L->seq_len != H->T || L->n_groups != H->n_groups)
     return fail(JOLT_EINVAL, "output layout does not match the compressed cache");
   for (int g = 0; g <= L->n_groups; ++g)
@@ -1321,11 +1328,8 @@ extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void 
   std::vector<CellWork> ws(nc);
   std::vector<char> use_tc(nc, 0);
   int tc_heads = 0;
-  // the tensor-core kernel stores 16-byte vectors: the output tensors must start on a 16-byte boundary (strides are
-  // multiples of 8 elements by check_layout); staged host outputs always do
-  const bool out_al16 = L->mem_space == JOLT_MEM_HOST || (((uintptr_t)Kout | (uintptr_t)Vout) % 16 == 0);
   for (int i = 0; i < nc; ++i)
-    if (fast && out_al16 && H->cells[i].tc_ok) { use_tc[i] = 1; tc_heads += H->cells[i].c.m; }
+    if (fast && H->cells[i].tc_ok) { use_tc[i] = 1; tc_heads += H->cells[i].c.m; }
   void *ws_base = nullptr;
   char *stage_K = nullptr, *stage_V = nullptr;
   int *d_status = nullptr;
@@ -1533,7 +1537,7 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
                          jolt_cell_plan *out, double *achieved) {
   if (!out || !K || !V) return fail(JOLT_EINVAL, "null argument");
   int rc;
-  if ((rc = check_layout(L)) || (rc = check_options(o))) return rc;
+  if ((rc = check_layout(L)) || (rc = check_options(o)) || (rc = check_device_alignment(L, K, V))) return rc;
   if (!(budget > 0)) return fail(JOLT_EINVAL, "byte budget must be positive");
   cudaStream_t st = (cudaStream_t)stream;
   int dev = 0;

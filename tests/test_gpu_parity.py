@@ -225,6 +225,30 @@ def test_exact_mode_large_T_reports_a_gapless_spectrum(B):
     h.free()
 
 
+def test_misaligned_device_tensors_are_rejected(B):
+    # device tensors are read and written with 16-byte vector accesses: a base that is not 16-byte aligned is an
+    # argument error reported before any kernel is launched
+    g = torch.Generator().manual_seed(2)
+    flat = torch.randn(2 * 2 * 128 * 128 + 8, generator=g).to(torch.float16).cuda()
+    Kmis = flat[4:4 + 2 * 2 * 128 * 128].view(2, 2, 128, 128)          # base + 8 bytes
+    Kok = flat[8:8 + 2 * 2 * 128 * 128].view(2, 2, 128, 128)           # base + 16 bytes
+    assert Kmis.data_ptr() % 16 == 8 and Kok.data_ptr() % 16 == 0
+    V = torch.randn(2, 2, 128, 128, generator=g).to(torch.float16).cuda()
+    plans = [(16, 128, 4), (16, 128, 4)]
+    with pytest.raises(B.JoltError) as e:
+        B.jolt_compress(Kmis, V, [0, 2], plans, B.default_options(seed=1))
+    assert e.value.status == B.EINVAL
+    h = B.jolt_compress(Kok, V, [0, 2], plans, B.default_options(seed=1))
+    with pytest.raises(B.JoltError) as e:
+        B.jolt_decompress(h, Kmis, torch.empty_like(V), [0, 2])
+    assert e.value.status == B.EINVAL
+    Ko, Vo = torch.empty_like(V), torch.empty_like(V)
+    B.jolt_decompress(h, Ko, Vo, [0, 2])
+    torch.cuda.synchronize()
+    assert float((Ko.float() - Kok.float()).norm() / Kok.float().norm()) < 0.2
+    h.free()
+
+
 # --------------------------------------------------------------------------- fp16 multi-group cache, several tiles
 @pytest.mark.parametrize("bits_k,bits_v", [(4, 8), (0, 3), (1, 2)])
 def test_small_gqa_cache(B, synth, bits_k, bits_v):
