@@ -316,6 +316,8 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
       b.A_in = t.A; b.A = t.bjA; b.V = t.bjV; b.J = t.bjJ; b.off = t.bjOff; b.done = t.bjDone; b.ticket = (unsigned *)(t.bjDone + 1);
       b.n = t.n; b.nbe = (((t.n + kBJBlock - 1) / kBJBlock) + 1) & ~1; b.nP = b.nbe * kBJBlock;
       b.w = t.w; b.U_out = t.U_out; b.ld_out = t.ld_out; b.r_out = t.r_out; b.w_out = t.w_out; b.w_sqrt = t.w_sqrt; b.status = t.status;
+      b.tol = kBJTol;
+      if (const char *e = getenv("JOLT_BJ_TOL")) b.tol = atof(e);      // experiments only
       bj.push_back(b);
       continue;
     }
