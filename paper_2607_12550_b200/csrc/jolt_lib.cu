@@ -1391,6 +1391,10 @@ extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void 
     rows += (long long)c.m * c.T;
     rj.push_back(j);
   }
+  // the costliest cells (most residual bits, then largest r_t) first: the last wave of CTAs is then the cheapest one
+  std::stable_sort(bbc.begin(), bbc.end(), [](const tc::BBCell &x, const tc::BBCell &y) {
+    return x.bits != y.bits ? x.bits > y.bits : x.r_t > y.r_t;
+  });
   add_decode_tc(P, ST_DROWS, bbc, H->seed);
   add_backbone(P, ST_DBACK, br);
   if (!rj.empty()) {

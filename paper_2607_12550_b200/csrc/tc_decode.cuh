@@ -342,7 +342,7 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = warp >> 2;
   long long *kdbg = (c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ? c.dbg + 16 * 8 : nullptr;
-  if (kdbg) kdbg[0] = clock64();
+  if (kdbg) { kdbg[0] = clock64(); long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); kdbg[6] = gt; }
   const int nkt = (c.r_t + 63) / 64, nkf = (c.r_f + 63) / 64;
   const bool has_res = c.bits > 0;
   // r_t <= 128 leaves half of the P region and half of the ring free: each warpgroup then stages its output in a
@@ -542,7 +542,7 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
   if (kdbg) kdbg[4] = clock64();
   tc_fence_before();
   __syncthreads();
-  if (kdbg) kdbg[5] = clock64();
+  if (kdbg) { kdbg[5] = clock64(); long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); kdbg[7] = gt; }
   if (*abort_flag) {
     if (threadIdx.x == 0) atomicOr(c.status, 8);
     const long long t0 = clock64();
