@@ -38,10 +38,10 @@ struct DecLayout {
 };
 
 template <int BITS>
-struct DecCodes { uint32_t words[BITS > 0 ? 4 * BITS : 1]; uint2 sc; };
+struct DecCodesRow { uint32_t words[BITS > 0 ? 4 * BITS : 1]; uint2 sc; };
 
 template <int BITS>
-__device__ __forceinline__ void dec_load_codes(const BBCell &c, long long row, DecCodes<BITS> &d) {
+__device__ __forceinline__ void dec_load_codes_row(const BBCell &c, long long row, DecCodesRow<BITS> &d) {
   if constexpr (BITS > 0) {
     const uint4 *wp = (const uint4 *)(c.words + row * (4 * BITS));
 #pragma unroll
@@ -85,7 +85,7 @@ struct DecGroupBytes {      // per-group byte lanes from which every code is one
 
 // codes -> fp16 operand row (pre-scaled), written into the warpgroup's swizzled K-major tile
 template <int BITS>
-__device__ __forceinline__ void dec_unpack_row(const DecCodes<BITS> &d, float pre, unsigned char *rbuf, int rit) {
+__device__ __forceinline__ void dec_unpack_row_row(const DecCodesRow<BITS> &d, float pre, unsigned char *rbuf, int rit) {
   constexpr float off = 0.5f - (float)(1 << (BITS > 0 ? BITS - 1 : 0));
   constexpr uint32_t mask = (1u << BITS) - 1u;
   constexpr bool kFast = BITS == 8 || BITS == 4 || BITS == 2 || BITS == 1;
@@ -121,6 +121,93 @@ __device__ __forceinline__ void dec_unpack_row(const DecCodes<BITS> &d, float pr
       }
       const int chunk = (g & 1) * 4 + ck;
       *(uint4 *)(rowp + ((chunk ^ (rit & 7)) << 4)) = pk;
+    }
+  }
+}
+
+// ---- warp-cooperative code path (BITS in {1, 2, 4, 8}) --------------------------------------------------------
+// A row of codes is BITS 16-byte chunks.  Instead of every thread fetching its own row (32 rows, 32 half-used
+// sectors per load instruction), BITS neighbouring lanes fetch the BITS chunks of one row: a warp instruction then
+// reads 512 contiguous bytes, and after BITS instructions the warp holds the codes of its 32 rows.  Each lane
+// dequantises the 128 / BITS features of the chunks it holds and writes them into the operand tile itself.
+template <int BITS>
+struct DecCodes {
+  static constexpr bool kCoop = BITS == 8 || BITS == 4 || BITS == 2 || BITS == 1;
+  uint32_t words[BITS > 0 ? 4 * BITS : 1];     // coop: chunk of iteration `it` at words[4 it ..]; else the thread's row
+  alignas(8) __half sc[8];                     // coop: the scales those chunks need; else sc[0..3] = the row's scales
+};
+
+template <int BITS>
+__device__ __forceinline__ void dec_load_codes(const BBCell &c, long long row, DecCodes<BITS> &d) {
+  if constexpr (BITS == 0) return;
+  else if constexpr (!DecCodes<BITS>::kCoop) {
+    const uint4 *wp = (const uint4 *)(c.words + row * (4 * BITS));
+#pragma unroll
+    for (int i = 0; i < BITS; ++i) { const uint4 v = __ldg(wp + i); d.words[4 * i] = v.x; d.words[4 * i + 1] = v.y; d.words[4 * i + 2] = v.z; d.words[4 * i + 3] = v.w; }
+    *(uint2 *)d.sc = __ldg((const uint2 *)(c.scales + row * 4));
+  } else {
+    constexpr int RPI = 32 / BITS;                            // rows per load instruction
+    const int lane = threadIdx.x & 31;
+    const long long wrow = row - lane;                        // first row of this warp's 32-row slab
+    const int chunk = lane % BITS, rsub = lane / BITS;
+#pragma unroll
+    for (int it = 0; it < BITS; ++it) {
+      const long long r = wrow + it * RPI + rsub;
+      const uint4 v = __ldg((const uint4 *)(c.words + r * (4 * BITS)) + chunk);
+      d.words[4 * it] = v.x; d.words[4 * it + 1] = v.y; d.words[4 * it + 2] = v.z; d.words[4 * it + 3] = v.w;
+      const __half *sp = c.scales + r * 4;
+      if constexpr (BITS == 8) d.sc[it] = __ldg(sp + (chunk >> 1));
+      else if constexpr (BITS == 4) d.sc[it] = __ldg(sp + chunk);
+      else if constexpr (BITS == 2) *(uint32_t *)&d.sc[2 * it] = __ldg((const uint32_t *)(sp + 2 * chunk));
+      else *(uint2 *)&d.sc[0] = __ldg((const uint2 *)sp);
+    }
+  }
+}
+
+// codes -> fp16 operand values (pre-scaled), written into the warpgroup's swizzled K-major tile.  (code - 2^(BITS-1)
+// + 1/2) dq is formed as in dec_unpack_row_row: byte permute into 2^23 + code, one add, one FMA, rounded once.
+template <int BITS>
+__device__ __forceinline__ void dec_unpack_row(const DecCodes<BITS> &d, float pre, unsigned char *rbuf, int rit) {
+  if constexpr (BITS == 0) return;
+  else if constexpr (!DecCodes<BITS>::kCoop) {
+    DecCodesRow<BITS> r;
+#pragma unroll
+    for (int i = 0; i < 4 * BITS; ++i) r.words[i] = d.words[i];
+    r.sc = *(const uint2 *)d.sc;
+    dec_unpack_row_row<BITS>(r, pre, rbuf, rit);
+  } else {
+    constexpr int RPI = 32 / BITS, NV = 128 / BITS;           // rows per instruction, values per chunk
+    constexpr float c0 = -(8388608.0f + (float)(1 << (BITS - 1)));
+    const int lane = rit & 31, wrow0 = rit & ~31;
+    const int chunk = lane % BITS, rsub = lane / BITS;
+#pragma unroll
+    for (int it = 0; it < BITS; ++it) {
+      const int row = wrow0 + it * RPI + rsub;                // row of the tile this chunk belongs to
+      const uint32_t *W = &d.words[4 * it];
+      unsigned char *rowp = rbuf + row * 128;
+#pragma unroll
+      for (int v = 0; v < NV; v += 8) {
+        uint4 pk;
+        __half2 *hp = (__half2 *)&pk;
+#pragma unroll
+        for (int e2 = 0; e2 < 4; ++e2) {
+          float v2[2];
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int j = v + e2 * 2 + u;                     // value index within the chunk (compile-time)
+            uint32_t src; int byte, gi;
+            if constexpr (BITS == 8) { src = W[j >> 2]; byte = j & 3; gi = it; }
+            else if constexpr (BITS == 4) { src = (j & 1) ? ((W[j >> 3] >> 4) & 0x0F0F0F0Fu) : (W[j >> 3] & 0x0F0F0F0Fu); byte = (j & 7) >> 1; gi = it; }
+            else if constexpr (BITS == 2) { const int gg = j >> 5, jj = j & 31; src = (W[2 * gg + (jj >> 4)] >> (2 * (jj & 3))) & 0x03030303u; byte = (jj & 15) >> 2; gi = 2 * it + gg; }
+            else { const int gg = j >> 5, jj = j & 31; src = (W[gg] >> (jj & 7)) & 0x01010101u; byte = jj >> 3; gi = gg; }
+            const float dq = __half2float(d.sc[gi]) * pre;
+            v2[u] = fmaf(__uint_as_float(__byte_perm(src, 0x4B000000u, 0x7650u + (uint32_t)byte)) + c0, dq, 0.5f * dq);
+          }
+          hp[e2] = __floats2half2_rn(v2[0], v2[1]);
+        }
+        const int oc = chunk * (NV / 8) + (v >> 3);           // 16-byte chunk of the 256-byte operand row
+        *(uint4 *)(rowp + (oc >> 3) * 16384 + (((oc & 7) ^ (row & 7)) << 4)) = pk;
+      }
     }
   }
 }
