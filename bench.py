@@ -337,7 +337,7 @@ def main():
     dec_bound = "hbm" if bd / (pk["hbm"] * 1e9) >= fd / (pk["tensor"] * 1e12) else "tensor"
     # DRAM traffic of one launch: ncu capture of the first 2 groups (profiles/decode_kernel_config1_2groups.md:
     # 60.4 MB read + 78.5 MB written for 4 of the 16 cells), scaled by the cells of this run
-    traffic = (60.437e6 + 79.090e6) * (2 * ng) / 4 if cfg.name == "c1" else None
+    traffic = (60.440e6 + 78.180e6) * (2 * ng) / 4 if cfg.name == "c1" else None
     if dec_bound == "hbm":
         ach = bd / (t_dec * 1e-3) / 1e9
         roofline = {"kernel": "tc::decode_kernel", "bound": "hbm", "achieved": ach, "peak": pk["hbm"], "unit": "GB/s",
