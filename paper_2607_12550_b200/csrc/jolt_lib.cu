@@ -130,29 +130,41 @@ struct StoreJob {
   const float *G32; const float *UT32; const float *UF32;
   __half *G16, *UT16, *UF16;
   int *e;
+  float *pmax;        // kCoreMaxParts partial maxima of |G| (scratch)
   long long nG, nUT, nUF;
   int round_inputs;   // 1: UT32/UF32 are rounded to fp16 in place as well (injected factors)
 };
 
+// max |G| of a cell in kCoreMaxParts partial maxima (one CTA each); store_factors_kernel finishes the reduction
+constexpr int kCoreMaxParts = 32;
 __global__ void core_exponent_kernel(const StoreJob *jobs) {
-  const StoreJob j = jobs[blockIdx.x];
+  const StoreJob j = jobs[blockIdx.y];
   float mx = 0.f;
-  for (long long i = threadIdx.x; i < j.nG; i += blockDim.x) mx = fmaxf(mx, fabsf(j.G32[i]));
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < j.nG; i += (long long)gridDim.x * blockDim.x)
+    mx = fmaxf(mx, fabsf(j.G32[i]));
   for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
   __shared__ float red[32];
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
   __syncthreads();
   if (threadIdx.x == 0) {
     for (int i = 0; i < (int)blockDim.x / 32; ++i) mx = fmaxf(mx, red[i]);
-    int e = 0;
-    if (mx > 0.f && isfinite(mx)) e = ilogbf(mx) - kCoreTargetExp;
-    *j.e = e;
+    j.pmax[blockIdx.x] = mx;
   }
 }
 
 __global__ void store_factors_kernel(const StoreJob *jobs) {
   const StoreJob j = jobs[blockIdx.y];
-  const int e = *j.e;
+  __shared__ int s_e;
+  if (threadIdx.x == 0) {
+    float mx = 0.f;
+    for (int i = 0; i < kCoreMaxParts; ++i) mx = fmaxf(mx, j.pmax[i]);
+    int e = 0;
+    if (mx > 0.f && isfinite(mx)) e = ilogbf(mx) - kCoreTargetExp;
+    s_e = e;
+    if (blockIdx.x == 0) *j.e = e;
+  }
+  __syncthreads();
+  const int e = s_e;
   const long long stride = (long long)gridDim.x * blockDim.x;
   const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   for (long long i = i0; i < j.nG; i += stride) j.G16[i] = __float2half_rn(ldexpf(j.G32[i], -e));
@@ -409,6 +421,7 @@ struct CellWork {      // device scratch of one cell
   __half *P16 = nullptr;
   float *Xt = nullptr;
   int *status = nullptr;
+  float *pmax = nullptr;     // partial maxima of |G| for the core exponent
   float *rho = nullptr;      // where the residual of the converged-subspace check goes (exact mode at large T)
   int n_sigma = 0;
   // tensor-core sweeps
@@ -434,6 +447,7 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
     if (!(real && w.lam)) w.lam = b.take<float>(kD);
     w.UT32 = b.take<float>(T * c.r_t);
     w.G32 = b.take<float>((size_t)c.m * c.r_t * c.r_f);
+    w.pmax = b.take<float>(32);
     w.Zp = b.take<float>((size_t)c.m * kD * std::max<size_t>(k, c.r_t));
     if (mode != FM_INJECTED) {
       {
@@ -1142,7 +1156,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
       if (c.r_t == 0) continue;
       StoreJob j;
       j.G32 = ws[i].G32; j.UT32 = ws[i].UT32; j.UF32 = ws[i].UF32;
-      j.G16 = cs.G16; j.UT16 = cs.UT16; j.UF16 = cs.UF16; j.e = cs.e;
+      j.G16 = cs.G16; j.UT16 = cs.UT16; j.UF16 = cs.UF16; j.e = cs.e; j.pmax = ws[i].pmax;
       j.nG = (long long)c.m * c.r_t * c.r_f; j.nUT = (long long)c.T * c.r_t; j.nUF = (long long)kD * c.r_f; j.round_inputs = 0;
       sj.push_back(j);
     }
@@ -1150,7 +1164,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
       const size_t off = PP.push(sj);
       const int n = (int)sj.size();
       PP.add(ST_STORE, [=](char *dev_t, cudaStream_t s) {
-        core_exponent_kernel<<<n, 1024, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
+        core_exponent_kernel<<<dim3(kCoreMaxParts, n), 256, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
         store_factors_kernel<<<dim3(64, n), 256, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
       });
     }
