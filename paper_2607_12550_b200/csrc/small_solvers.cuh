@@ -357,7 +357,7 @@ struct CholSmemTask { const double *G; float *LT; float *invd; int n; int *statu
 __global__ void __launch_bounds__(512, 1) cholesky_smem_kernel(const CholSmemTask *__restrict__ tasks, int in_global) {
   // Left-looking Cholesky by panels of 8 columns.  (1) The panel loses the contribution of the finished columns,
   // one dot product per entry on four independent accumulators.  (2) Warp 0 factors the 8 x 8 diagonal block in
-  // registers (shuffles, reciprocal square roots instead of divisions).  (3) The rows below are solved against the
+  // registers (reciprocal square roots instead of divisions).  (3) The rows below are solved against the
   // block, one thread per row.  Three barriers per panel.
   const CholSmemTask t = tasks[blockIdx.x];
   const int n = t.n;
@@ -399,33 +399,40 @@ __global__ void __launch_bounds__(512, 1) cholesky_smem_kernel(const CholSmemTas
       A[i * ld + j0 + c] -= (a0 + a1) + (a2 + a3);
     }
     __syncthreads();
-    // (2) the 8 x 8 diagonal block in the registers of warp 0: lane r holds row r
+    // (2) the 8 x 8 diagonal block: every lane of warp 0 factors the whole block in its own registers (36 entries,
+    // broadcast loads, no shuffles on the dependent chain); lane r then writes row r back
     if (tid < 32) {
-      const int r = tid & 7, i = j0 + r;
-      double row[8], piv[8];
+      double L[8][8], piv[8];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) row[c] = (r < w && c <= r) ? A[i * ld + j0 + c] : 0.0;
+      for (int r = 0; r < 8; ++r)
+#pragma unroll
+        for (int c = 0; c <= r; ++c) L[r][c] = (r < w) ? A[(j0 + r) * ld + j0 + c] : (r == c ? 1.0 : 0.0);
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         piv[c] = 0.0;
         if (c < w) {
-          const double d = __shfl_sync(0xffffffffu, row[c], c);
-          const double dg = diag0[j0 + c];
+          const double d = L[c][c], dg = diag0[j0 + c];
           const bool bad = !(d > 1e-10 * dg) || !(dg > 0);
           const double rs = bad ? 0.0 : rsqrt_pos(d);
-          if (r == c) row[c] = bad ? 1.0 : d * rs; else row[c] *= rs;
-          if (tid == c && bad) dead[j0 + c] = 1;
+          L[c][c] = bad ? 1.0 : d * rs;
+          if (tid == 0 && bad) dead[j0 + c] = 1;
           piv[c] = rs;
 #pragma unroll
-          for (int cc = c + 1; cc < 8; ++cc) {
-            const double lcc = __shfl_sync(0xffffffffu, row[c], cc);     // L[cc][c]
-            if (r >= cc) row[cc] = fma(-row[c], lcc, row[cc]);
-          }
+          for (int r = c + 1; r < 8; ++r) L[r][c] *= rs;
+#pragma unroll
+          for (int cc = c + 1; cc < 8; ++cc)
+#pragma unroll
+            for (int r = cc; r < 8; ++r) L[r][cc] = fma(-L[r][c], L[cc][c], L[r][cc]);
         }
       }
+      const int r = tid & 7;
       if (tid < w) {
 #pragma unroll
-        for (int c = 0; c < 8; ++c) if (c <= r) { A[i * ld + j0 + c] = row[c]; blk[r][c] = row[c]; }
+        for (int rr = 0; rr < 8; ++rr)
+          if (rr == r) {
+#pragma unroll
+            for (int c = 0; c <= rr; ++c) { A[(j0 + rr) * ld + j0 + c] = L[rr][c]; blk[rr][c] = L[rr][c]; }
+          }
       }
       if (tid == 0) {
 #pragma unroll
