@@ -202,7 +202,10 @@ inline void add_tok_tc(Program &P, int stage, std::vector<CellWork> &ws, const s
     if (!w.active || !w.tc) continue;
     const CellDesc &c = w.c;
     int se = 0;
-    if (src[i] != 0) {
+    if (src[i] == 2 && w.ufI && w.split_ready == 2) {
+      se = ilog2_floor((long long)c.N) / 2;          // the triangular solve of orth(Z) has written the operand already
+      w.split_ready = 0;
+    } else if (src[i] != 0) {
       const float *in = w.W;
       if (src[i] == 2) { in = w.ufI ? w.Z : w.W; se = ilog2_floor((long long)c.N) / 2; }
       tc::SplitJob j;
@@ -241,9 +244,12 @@ inline void add_feat_tc(Program &P, int stage, std::vector<CellWork> &ws) {
     if (!w.active || !w.tc) continue;
     const CellDesc &c = w.c;
     const int se = ilog2_floor(c.T) / 2;
-    tc::SplitJob j;
-    j.in = w.S; j.hi = w.Bhi; j.lo = w.Blo; j.batch = 1; j.rows = c.T; j.cols = c.k; j.ld_in = c.k; j.kp = w.kp; j.scale_exp = se;
-    sp.push_back(j);
+    if (w.split_ready != 1) {      // else the triangular solve of orth(S) has written the operand already
+      tc::SplitJob j;
+      j.in = w.S; j.hi = w.Bhi; j.lo = w.Blo; j.batch = 1; j.rows = c.T; j.cols = c.k; j.ld_in = c.k; j.kp = w.kp; j.scale_exp = se;
+      sp.push_back(j);
+    }
+    w.split_ready = 0;
     std::vector<std::pair<int, int>> ch;
     sketch_chunks(w.kp, ch);
     for (auto &cc : ch) {

@@ -431,6 +431,7 @@ struct CellWork {      // device scratch of one cell
   bool skip_feat = false;    // no mode-3 Gram / eigen-solve needed
   int kp = 0;                // sketch width padded to a multiple of 16
   __half *Bhi = nullptr, *Blo = nullptr;
+  int split_ready = 0;       // 1 / 2: Bhi, Blo already hold the split of S / Z (written by the last triangular solve)
 };
 
 enum FactorMode { FM_RANDOMIZED = 0, FM_EXACT = 1, FM_INJECTED = 2 };
@@ -553,7 +554,15 @@ void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side,
       float *buf = token_side ? w.S : w.Z;
       tg.push_back({buf, rows, k, w.gpart, w.Gs});
       chs[cls].push_back({w.Gs, w.LT32, w.invd, k, w.status, w.Lwork});
-      tj[cls].push_back({buf, buf, rows, k, w.LT32, w.invd});
+      TrsmJob tjob{buf, buf, rows, k, w.LT32, w.invd, nullptr, nullptr, 0, 0, 0};
+      w.split_ready = 0;
+      if (w.tc && pass == passes - 1 && (token_side || w.ufI)) {
+        // the next sweep reads this basis as its dense operand: emit the hi + lo fp16 split here
+        tjob.hi = w.Bhi; tjob.lo = w.Blo; tjob.split_mode = token_side ? 1 : 2; tjob.kp16 = w.kp;
+        tjob.scale_exp = ilog2_floor(token_side ? (long long)w.c.T : (long long)w.c.N) / 2;
+        w.split_ready = tjob.split_mode;
+      }
+      tj[cls].push_back(tjob);
       max_k[cls] = std::max(max_k[cls], k);
     }
     add_tall_gram(P, stage, tg);

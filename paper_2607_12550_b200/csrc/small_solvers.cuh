@@ -472,7 +472,14 @@ inline size_t chol_smem_bytes(int n, bool in_global = false) {
   return ((in_global ? 0 : (size_t)n * (n + 1)) + n) * sizeof(double) + (size_t)n * sizeof(int) + 64;
 }
 
-struct TrsmJob { const float *src; float *dst; int rows, k; const float *LT; const float *invd; };
+// Optional second output: the solved rows again as the hi + lo fp16 operand of the next tensor-core sweep (scaled by
+// 2^scale_exp, zero-padded to kp16 columns), so that no separate split / transpose pass is needed.
+//   split_mode 1: [kp16][rows]           (token-side basis, operand of the projection sweep)
+//   split_mode 2: [rows / 128][kp16][128] (feature-side basis, rows = (head, feature), operand of the sketch sweep)
+struct TrsmJob {
+  const float *src; float *dst; int rows, k; const float *LT; const float *invd;
+  __half *hi, *lo; int split_mode, kp16, scale_exp;
+};
 
 inline size_t trsm_smem_bytes(int k, int rb, bool lt_global = false) {
   const int kp = (k + 7) & ~7;
@@ -581,6 +588,19 @@ __global__ void __launch_bounds__(RB / 2) trsm_rows_kernel(const TrsmJob *__rest
   __syncthreads();
   float *dst = t.dst + (size_t)r0 * k;
   for (int e = tid; e < nrows * k; e += NT) { const int r = e / k, j = e - r * k; dst[e] = sp[j * PITCH + r]; }
+  if (t.split_mode) {
+    const float sc = ldexpf(1.0f, t.scale_exp);
+    for (int e = tid; e < nrows * t.kp16; e += NT) {
+      const int j = e / nrows, r = e - j * nrows;          // r fastest: conflict-free reads, contiguous writes
+      const float v = j < k ? sp[j * PITCH + r] * sc : 0.f;
+      const __half h = __float2half_rn(v);
+      const int row = r0 + r;
+      const size_t o = t.split_mode == 1 ? (size_t)j * t.rows + row
+                                         : ((size_t)(row >> 7) * t.kp16 + j) * 128 + (row & 127);
+      t.hi[o] = h;
+      t.lo[o] = __float2half_rn(v - __half2float(h));
+    }
+  }
 }
 
 // sum of fp64 partials with a per-job element count
