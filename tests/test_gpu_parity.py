@@ -205,10 +205,28 @@ def test_exact_mode_large_T_converged_subspace(B, synth):
             eg, eo = np.linalg.norm(UT.T @ A) ** 2, np.linalg.norm(o.ideal["U_T"].T @ A) ** 2
             assert abs(eg - eo) <= 1e-4 * eo, (c, eg, eo)
     h.free()
-    # the plan probe in exact mode at this T: spectra agree with the oracle's on the values the dual uses
-    budget = 0.5 * 2 * K.numel() * 2
-    plan_g, _ = B.jolt_plan(K, V, gs, budget, opts)
-    assert len(plan_g) == 4 and all(p[0] > 0 for p in plan_g)
+    # the plan probe in exact mode at this T: the exact top q_cap singular values plus the tail mass (Sec. 5
+    # accounting), fed to the same dual, give the library's plan
+    raw = 2 * K.numel() * 2
+    plan_g, ach = B.jolt_plan(K, V, gs, raw / 2.0, opts)
+    assert ach <= raw / 2.0
+    q_cap = O.cap_policy(2048, 2.0)
+    eps2 = O.eps2_table([0, 2, 4, 8])
+    cells, trips = [], []
+    for c in range(4):
+        X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
+        lam, s2_all, tot = O.plan_spectra(X, q_cap, token_mode="exact")
+        s2 = O.tail_mass_spectrum(np.sqrt(s2_all[:q_cap]), tot) ** 2
+        rt_grid, rf_grid = list(range(16, q_cap + 1, 16)), list(range(16, 129, 16))
+        tau = O.tau_table(lam, s2, tot, rt_grid, rf_grid)
+        e, sz, t = O.cell_options(4, 2048, 128, tau, rt_grid, rf_grid, [0, 2, 4, 8], eps2)
+        cells.append((e, sz)); trips.append(t)
+    ch, cost, lam_star, ok = O.dual_allocate(cells, raw / 2.0)
+    ref = [trips[c][i] for c, i in enumerate(ch)]
+    e_ref = sum(cells[c][0][ch[c]] for c in range(4))
+    e_got = sum(cells[c][0][trips[c].index(tuple(plan_g[c]))] for c in range(4))
+    assert abs(e_got - e_ref) <= 1e-3 * e_ref + 1e-9, (plan_g, ref)
+    assert sum(p == r for p, r in zip(plan_g, ref)) >= 3, (plan_g, ref)
 
 
 def test_exact_mode_large_T_reports_a_gapless_spectrum(B):
