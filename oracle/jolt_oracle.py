@@ -18,6 +18,8 @@ Each function names the passage of the paper it follows:
 * Eq. (1)                            -> eq1_bytes, stored_bytes
 * Eq. (2)                            -> eps2_table, tau_table
 * Eq. (3), Eq. (4)                   -> dual_allocate
+* App. "RoPE pre vs. post on K" (keys are decomposed before the rotary embedding, which is
+  re-applied at decode time)        -> rope_rotate, decompress_cell_rope
 
 Pins (tests/test_oracle_*.py): full-rank exactness, exact low-rank recovery, orthonormality,
 energy split, ST-HOSVD sandwich bound, norm preservation and involution of the rotation,
@@ -400,6 +402,42 @@ def decompress_cell(c: CompressedCell):
     if c.out_dtype == "f16":
         return fp16_round(Xh)
     return Xh.astype(np.float32).astype(np.float64)
+
+
+# --------------------------------------------------------------------------------------
+# Rotary position embedding re-applied to decoded keys (App. "RoPE pre vs. post on K").
+# The paper names the operation only; the reading taken is the rotate-half form used by the
+# models it evaluates (Mistral, LLaMA): feature j pairs with feature j + d/2, angle
+# (pos0 + t) * base^(-2j/d).
+# --------------------------------------------------------------------------------------
+def rope_rotate(X, base: float = 10000.0, pos0: int = 0, inverse: bool = False):
+    """X: (..., T, d) -> same shape; token index is the second-to-last axis."""
+    X = np.asarray(X, dtype=np.float64)
+    T, d = X.shape[-2], X.shape[-1]
+    half = d // 2
+    j = np.arange(half, dtype=np.float64)
+    inv_freq = base ** (-2.0 * j / d)
+    ang = (pos0 + np.arange(T, dtype=np.float64))[:, None] * inv_freq[None, :]
+    c, s = np.cos(ang), np.sin(ang)
+    if inverse:
+        s = -s
+    a, b = X[..., :half], X[..., half:]
+    return np.concatenate([a * c - b * s, b * c + a * s], axis=-1)
+
+
+def decompress_cell_rope(c: "CompressedCell", base: float = 10000.0, pos0: int = 0):
+    """Decode a key cell and re-apply the rotary embedding before the single rounding to the output type."""
+    if c.r_t > 0:
+        Xh = stored_backbone(c.Gs16, c.e, c.UT16, c.UF16)
+    else:
+        Xh = np.zeros((c.m, c.T, c.d))
+    if c.bits > 0:
+        codes = unpack_codes(c.words, c.bits, c.d)
+        Xh = Xh + unrotate(dequantize_rows(codes, c.scales, c.bits, c.group), c.signs)
+    Xr = rope_rotate(Xh, base, pos0)
+    if c.out_dtype == "f16":
+        return fp16_round(Xr)
+    return Xr.astype(np.float32).astype(np.float64)
 
 
 def rel_frobenius(X, Xh):

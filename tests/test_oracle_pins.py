@@ -405,3 +405,33 @@ def test_dual_moves_bits_to_flat_spectrum_cell():
     assert ok and cost <= raw / 3
     bK, bV = trips[0][ch[0]][2], trips[1][ch[1]][2]
     assert bV >= bK
+
+
+# ----------------------------------------------------------------------------- rotary embedding at decode
+def test_rope_is_the_textbook_rotation():
+    # d = 4: pairs (0, 2) and (1, 3), frequencies 1 and base^(-1/2); written out by hand
+    x = np.array([[1.0, 2.0, 3.0, 4.0], [0.5, -1.0, 2.0, 0.25]])
+    y = O.rope_rotate(x, base=100.0, pos0=3)
+    for t in range(2):
+        p = 3 + t
+        for j, th in enumerate([1.0, 0.1]):
+            c, s = math.cos(p * th), math.sin(p * th)
+            assert abs(y[t, j] - (x[t, j] * c - x[t, j + 2] * s)) < 1e-14
+            assert abs(y[t, j + 2] - (x[t, j + 2] * c + x[t, j] * s)) < 1e-14
+
+
+def test_rope_invariants():
+    X = RNG.standard_normal((3, 40, 128))
+    Y = O.rope_rotate(X, base=10000.0, pos0=17)
+    # orthogonal per token: norms kept, inverse undoes it, position 0 is the identity
+    assert np.allclose(np.linalg.norm(Y, axis=-1), np.linalg.norm(X, axis=-1), rtol=1e-13)
+    assert np.allclose(O.rope_rotate(Y, 10000.0, 17, inverse=True), X, atol=1e-13)
+    assert np.allclose(O.rope_rotate(X[:, :1], 10000.0, 0), X[:, :1], atol=0)
+    # the defining property: <rope(q, m), rope(k, n)> depends on m - n only
+    q, k = RNG.standard_normal((1, 128)), RNG.standard_normal((1, 128))
+    def score(m, n):
+        return float(O.rope_rotate(q, 10000.0, m) @ O.rope_rotate(k, 10000.0, n).T)
+    assert abs(score(5, 2) - score(105, 102)) < 1e-10
+    assert abs(score(5, 2) - score(5, 3)) > 1e-6
+    # composition of shifts: rotating by a then by b is rotating by a + b
+    assert np.allclose(O.rope_rotate(O.rope_rotate(X[:, :1], 10000.0, 7), 10000.0, 5), O.rope_rotate(X[:, :1], 10000.0, 12), atol=1e-12)
