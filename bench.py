@@ -168,6 +168,17 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def torch_rope(x, base):
+    """Rotate-half rotary embedding of a [..., T, 128] tensor (accuracy bookkeeping of --rope only)."""
+    import torch
+    T = x.shape[-2]
+    inv = base ** (-torch.arange(64, device=x.device, dtype=torch.float64) / 64)
+    ang = torch.arange(T, device=x.device, dtype=torch.float64)[:, None] * inv[None, :]
+    c, s_ = ang.cos().float(), ang.sin().float()
+    a, b = x[..., :64], x[..., 64:]
+    return torch.cat([a * c - b * s_, b * c + a * s_], dim=-1)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -179,6 +190,8 @@ def main():
     ap.add_argument("--token-mode", default="randomized", choices=["randomized", "exact"],
                     help="token-mode solver; exact at T > 1024 is the converged block iteration")
     ap.add_argument("--ratio", type=float, default=0.0, help="compression ratio of the byte budget (default: the workload's)")
+    ap.add_argument("--rope", action="store_true",
+                    help="decode through jolt_decompress_rope (keys rotated at decode; not the headline workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--portable", action="store_true", help="portable SIMT kernels only")
@@ -236,7 +249,10 @@ def main():
         h = B.jolt_compress(K, V, gs, plans, opts)
         e1.record()
         st_c = B.stage_ms()
-        B.jolt_decompress(h, Ko, Vo, gs)
+        if args.rope:
+            B.jolt_decompress_rope(h, Ko, Vo, gs, base=10000.0, pos0=0)
+        else:
+            B.jolt_decompress(h, Ko, Vo, gs)
         e2.record()
         torch.cuda.synchronize()
         st_d = B.stage_ms()
@@ -278,6 +294,8 @@ def main():
         g, w = divmod(c, 2)
         a = (K, V)[w][gs[g]:gs[g + 1]].float()
         b_ = (Ko, Vo)[w][gs[g]:gs[g + 1]].float()
+        if args.rope and w == 0:
+            a = torch_rope(a, 10000.0)
         errs.append(float((a - b_).norm() / a.norm()))
     rel_k = sum(errs[0::2]) / ng
     rel_v = sum(errs[1::2]) / ng
@@ -356,7 +374,7 @@ def main():
                                    f"{cfg.n_kv_heads} KV heads, T={cfg.seq_len}, d=128, fp16, budget {ratio}x, "
                                    + (f"randomized q={q}" if args.token_mode == "randomized" else "exact (converged block iteration)"),
                        "cache_bytes": cache_bytes, "compressed_bytes": planned_bytes, "achieved_ratio": cache_bytes / planned_bytes,
-                       "plan": plans, "l2": f"inputs ({cache_bytes / 1e6:.0f} MB) exceed L2; no flush"},
+                       "rope_at_decode": bool(args.rope), "plan": plans, "l2": f"inputs ({cache_bytes / 1e6:.0f} MB) exceed L2; no flush"},
             "compress_ms": tc, "decompress_ms": td, "plan_ms": plan_ms,
             "compress_ms_min_med_max": [tc_all[0], tc_all[len(tc_all) // 2], tc_all[-1]],
             "decompress_ms_min_med_max": [td_all[0], td_all[len(td_all) // 2], td_all[-1]],

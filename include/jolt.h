@@ -117,6 +117,23 @@ int jolt_compress_with_factors(const jolt_layout *layout, const void *dK, const 
 int jolt_decompress(const jolt_handle *h, const jolt_layout *out_layout, void *dK_out, void *dV_out,
                     void *stream);
 
+/* jolt_decompress_rope -- paper App. "RoPE pre vs. post on K": keys are decomposed before the rotary
+ * position embedding, which is applied again when the cache is decoded.  The paper names the operation
+ * without a formula; this entry point takes the common rotate-half form on head_dim 128: for token t at
+ * position p = pos0 + t and feature j < 64, with angle p * base^(-j/64),
+ *     K_out[.., t, j]      = K^[.., t, j] cos - K^[.., t, j + 64] sin
+ *     K_out[.., t, j + 64] = K^[.., t, j + 64] cos + K^[.., t, j] sin
+ * where K^ is what jolt_decompress writes.  V is written as by jolt_decompress.  Angles are evaluated in
+ * fp64, the rotation in fp32; an fp16 destination is rounded once after decoding and once after the
+ * rotation.  rope: host pointer; 1 < base < 1e12, 0 <= pos0 <= 2^40 (JOLT_EINVAL otherwise).  All other
+ * arguments, the result and the error behaviour are those of jolt_decompress. */
+typedef struct {
+  double base;   /* frequency base (10000 in the original formulation) */
+  int64_t pos0;  /* position of token 0 of this cache */
+} jolt_rope;
+int jolt_decompress_rope(const jolt_handle *h, const jolt_layout *out_layout, void *dK_out, void *dV_out,
+                         const jolt_rope *rope, void *stream);
+
 /* jolt_decompress_static -- the paper has no counterpart; this is a deployment variant of jolt_decompress
  * for callers that cannot allocate device memory while decoding (a serving process that has given all free
  * memory to its own pool, a thread for which a driver allocation would stall the context, a host whose

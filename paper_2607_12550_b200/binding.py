@@ -54,6 +54,13 @@ lib.jolt_compress_with_factors.argtypes = [C.POINTER(Layout), _vp, _vp, C.POINTE
                                            C.POINTER(_vp), C.POINTER(_vp), _vp, C.POINTER(_vp)]
 lib.jolt_decompress.argtypes = [_vp, C.POINTER(Layout), _vp, _vp, _vp]
 lib.jolt_free.argtypes = [_vp]
+
+
+class Rope(C.Structure):
+    _fields_ = [("base", C.c_double), ("pos0", C.c_int64)]
+
+
+lib.jolt_decompress_rope.argtypes = [_vp, C.POINTER(Layout), _vp, _vp, C.POINTER(Rope), _vp]
 lib.jolt_decompress_static.argtypes = [_vp, C.POINTER(Layout), _vp, _vp, _vp]
 lib.jolt_compressed_bytes.argtypes = [_vp, C.POINTER(C.c_int64)]
 lib.jolt_get_component.argtypes = [_vp, C.c_int32, C.c_int32, _vp, C.c_int64, C.POINTER(C.c_int64)]
@@ -99,9 +106,13 @@ class _Keep:
     gs: object
 
 
-def make_layout(K: torch.Tensor, group_start: Sequence[int]) -> Layout:
-    """Layout of a [n_layers, n_kv_heads, T, 128] tensor (any strides with unit feature stride)."""
+def make_layout(K: torch.Tensor, group_start: Sequence[int], V: torch.Tensor | None = None) -> Layout:
+    """Layout of a [n_layers, n_kv_heads, T, 128] tensor (any strides with unit feature stride).
+
+    The C ABI describes K and V by ONE layout: when V is given it must match K in shape, strides, dtype and device."""
     assert K.dim() == 4 and K.stride(3) == 1
+    if V is not None and (V.shape != K.shape or V.stride() != K.stride() or V.dtype != K.dtype or V.device != K.device):
+        raise ValueError("K and V must share shape, strides, dtype and device (one jolt_layout describes both)")
     gs = (C.c_int32 * len(group_start))(*group_start)
     lay = Layout(K.shape[0], K.shape[1], K.shape[2], K.shape[3],
                  F16 if K.dtype == torch.float16 else F32,
@@ -145,7 +156,7 @@ def _plans(plans) -> C.Array:
 
 
 def jolt_plan(K, V, group_start, byte_budget: float, opts: Options | None = None, stream=None, allow_budget=False):
-    lay = make_layout(K, group_start)
+    lay = make_layout(K, group_start, V)
     opts = opts or default_options()
     out = (CellPlan * (2 * lay.n_groups))()
     ach = C.c_double(0)
@@ -188,7 +199,7 @@ class Handle:
 
 
 def jolt_compress(K, V, group_start, plans, opts: Options | None = None, stream=None, factors=None) -> Handle:
-    lay = make_layout(K, group_start)
+    lay = make_layout(K, group_start, V)
     opts = opts or default_options()
     arr = _plans(plans)
     h = C.c_void_p(None)
@@ -207,13 +218,21 @@ def jolt_compress(K, V, group_start, plans, opts: Options | None = None, stream=
 
 
 def jolt_decompress(handle: Handle, K_out, V_out, group_start, stream=None):
-    lay = make_layout(K_out, group_start)
+    lay = make_layout(K_out, group_start, V_out)
     _check(lib.jolt_decompress(handle.ptr, C.byref(lay), K_out.data_ptr(), V_out.data_ptr(), _stream_ptr(stream)))
+
+
+def jolt_decompress_rope(handle: Handle, K_out, V_out, group_start, base=10000.0, pos0=0, stream=None):
+    """Decode and re-apply the rotary embedding to the keys (rotate-half form); see include/jolt.h."""
+    lay = make_layout(K_out, group_start, V_out)
+    rope = Rope(float(base), int(pos0))
+    _check(lib.jolt_decompress_rope(handle.ptr, C.byref(lay), K_out.data_ptr(), V_out.data_ptr(), C.byref(rope),
+                                    _stream_ptr(stream)))
 
 
 def jolt_decompress_static(handle: Handle, K_out, V_out, group_start, stream=None):
     """Decode without any device allocation (fixed 16 MiB scratch inside the library); see include/jolt.h."""
-    lay = make_layout(K_out, group_start)
+    lay = make_layout(K_out, group_start, V_out)
     _check(lib.jolt_decompress_static(handle.ptr, C.byref(lay), K_out.data_ptr(), V_out.data_ptr(), _stream_ptr(stream)))
 
 

@@ -20,6 +20,7 @@
 #include "simt_gemm.cuh"
 #include "small_solvers.cuh"
 #include "block_jacobi.cuh"
+#include "rope.cuh"
 
 using namespace jolt;
 
@@ -43,7 +44,7 @@ int fail(int code, const char *fmt, ...) {
 // ------------------------------------------------------------------ stage timing
 static const char *kStageNames[] = {"stage_in", "sketch_gen", "gram", "eig_feat", "sketch", "orth", "power", "project",
                                     "small_svd", "factors", "store", "backbone", "residual_quant", "decode_backbone",
-                                    "decode_rows", "stage_out"};
+                                    "decode_rows", "rope", "stage_out"};
 constexpr int kNumStages = sizeof(kStageNames) / sizeof(kStageNames[0]);
 struct StageTimer {
   cudaEvent_t ev[kNumStages + 1];
@@ -65,7 +66,7 @@ struct StageTimer {
 };
 thread_local StageTimer g_timer;
 enum { ST_IN = 0, ST_SKGEN, ST_GRAM, ST_EIGF, ST_SKETCH, ST_ORTH, ST_POWER, ST_PROJ, ST_SVD, ST_FACT, ST_STORE, ST_BACK,
-       ST_RQ, ST_DBACK, ST_DROWS, ST_OUT };
+       ST_RQ, ST_DBACK, ST_DROWS, ST_ROPE, ST_OUT };
 
 // ------------------------------------------------------------------ workspace cache (per device)
 struct Workspace { void *base = nullptr; size_t cap = 0; };
@@ -1334,10 +1335,13 @@ extern "C" int jolt_compress_with_factors(const jolt_layout *L, const void *K, c
 }
 
 // ------------------------------------------------------------------ decompress
-extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void *Kout, void *Vout, void *stream) {
+static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kout, void *Vout, const jolt_rope *rope,
+                           void *stream) {
   if (!H || !Kout || !Vout) return fail(JOLT_EINVAL, "null argument");
   int rc;
   if ((rc = check_layout(L)) || (rc = check_device_alignment(L, Kout, Vout))) return rc;
+  if (rope && !(rope->base > 1.0 && rope->base < 1e12)) return fail(JOLT_EINVAL, "rotary base %g", rope->base);
+  if (rope && (rope->pos0 < 0 || rope->pos0 > ((int64_t)1 << 40))) return fail(JOLT_EINVAL, "rotary pos0 out of range");
   if (L->n_layers != H->n_layers || L->n_kv_heads != H->n_kv_heads || L->seq_len != H->T || L->n_groups != H->n_groups)
     return fail(JOLT_EINVAL, "output layout does not match the compressed cache");
   for (int g = 0; g <= L->n_groups; ++g)
@@ -1429,6 +1433,21 @@ extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void 
       LAUNCHED();
     });
   }
+  if (rope) {
+    // keys only, in place on the decoded tensor (the staging buffer when the destination is host memory)
+    RopeJob j;
+    j.K = Kd; j.dtype = L->dtype == JOLT_F16 ? DT_F16 : DT_F32;
+    j.n_rows = L->n_layers * L->n_kv_heads; j.n_heads = L->n_kv_heads; j.T = L->seq_len;
+    j.sl = L->stride_layer; j.sh = L->stride_head; j.st = L->stride_token;
+    j.base = rope->base; j.pos0 = rope->pos0;
+    const int gx = (L->seq_len + kRopeTokensPerCta - 1) / kRopeTokensPerCta;
+    // about 16 CTAs per SM in flight; every CTA still visits several rows with one set of sines
+    const int gy = std::max(1, std::min(j.n_rows, (16 * 148 + gx - 1) / gx));
+    P.add(ST_ROPE, [=](char *, cudaStream_t s) {
+      rope_rows_kernel<<<dim3(gx, gy), 256, 0, s>>>(j);
+      LAUNCHED();
+    });
+  }
   void *d_tab = nullptr;
   if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
   g_timer.begin(st);
@@ -1442,6 +1461,16 @@ extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void 
     g_timer.finish();
   }
   return JOLT_OK;
+}
+
+extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void *Kout, void *Vout, void *stream) {
+  return decompress_impl(H, L, Kout, Vout, nullptr, stream);
+}
+
+extern "C" int jolt_decompress_rope(const jolt_handle *H, const jolt_layout *L, void *Kout, void *Vout,
+                                    const jolt_rope *rope, void *stream) {
+  if (!rope) return fail(JOLT_EINVAL, "rotary parameters are null");
+  return decompress_impl(H, L, Kout, Vout, rope, stream);
 }
 
 extern "C" int jolt_free(jolt_handle *H) {

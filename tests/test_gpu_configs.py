@@ -36,6 +36,13 @@ def test_first_group_of_config(B, name):
     Ko, Vo = torch.empty_like(K), torch.empty_like(V)
     B.jolt_decompress(h, Ko, Vo, gs)
     torch.cuda.synchronize()
+    # the same cache decoded with the rotary embedding re-applied to the keys (values must not change)
+    Kr, Vr = torch.empty_like(K), torch.empty_like(V)
+    B.jolt_decompress_rope(h, Kr, Vr, gs, base=10000.0, pos0=1000)
+    torch.cuda.synchronize()
+    assert torch.equal(Vr, Vo)
+    Krnp = Kr.cpu().numpy()
+    del Kr, Vr
     Knp, Vnp = K.cpu().numpy(), V.cpu().numpy()
     Konp, Vonp = Ko.cpu().numpy(), Vo.cpu().numpy()
     for c in range(2):
@@ -48,6 +55,12 @@ def test_first_group_of_config(B, name):
         rel = np.linalg.norm(Xg - Xo) / np.linalg.norm(Xo)
         assert abs(eg - eo) <= REL_ERR * eo, (name, c, plans[c], eg, eo)
         assert rel <= recon_gate(eo), (name, c, plans[c], rel, eo)
+        if c == 0:
+            Xro = O.decompress_cell_rope(o, 10000.0, 1000)
+            Xrg = cell_view(Krnp, Vonp, gs, 0).astype(np.float64)
+            relr = np.linalg.norm(Xrg - Xro) / np.linalg.norm(Xro)
+            assert relr <= recon_gate(eo), (name, "rope", relr, eo)
+            del Xro, Xrg
         if rt > 0:
             # projectors are compared before fp16 storage: independently rounded fp16 copies of two factors
             # that agree to 1e-5 are already ~2e-3 apart
