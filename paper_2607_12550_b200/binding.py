@@ -299,10 +299,11 @@ def launch_count() -> int:
 
 
 def set_fast_path(enabled) -> int:
-    """False / 0: portable kernels only; True / 7: every tensor-core kernel; other ints: bit mask
-    (1 = fused backbone kernels, 2 = factor sweeps, 4 = Gram).  Returns the previous mask."""
+    """False / 0: portable kernels only; True / 15: every tensor-core kernel; other ints: bit mask
+    (1 = fused backbone kernels, 2 = factor sweeps, 4 = Gram, 8 = rotary embedding inside the decode kernel).
+    Returns the previous mask."""
     if enabled is True:
-        enabled = 7
+        enabled = 15
     return lib.jolt_set_fast_path(int(enabled))
 
 

@@ -29,7 +29,8 @@ thread_local std::string g_err;
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_eig_smem{1};
 long long *g_dbg_stamps = nullptr;   // device buffer for kernel cycle stamps (profiling aid)
-std::atomic<int> g_fast{7};   // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores
+std::atomic<int> g_fast{15};  // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores,
+                              // bit 3: rotary embedding inside the decode kernel
 
 int fail(int code, const char *fmt, ...) {
   char buf[512];
@@ -1359,6 +1360,12 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
   int tc_heads = 0;
   for (int i = 0; i < nc; ++i)
     if (fast && H->cells[i].tc_ok) { use_tc[i] = 1; tc_heads += H->cells[i].c.m; }
+  // key cells that the tensor-core decode kernel rotates in its epilogue (its r_t <= 128 form holds a whole row in registers)
+  std::vector<char> rope_fused(nc, 0);
+  int n_rope_fused = 0;
+  for (int i = 0; rope && i < nc; i += 2)
+    if (use_tc[i] && H->cells[i].c.r_t <= 128 && (g_fast.load() & 8)) { rope_fused[i] = 1; ++n_rope_fused; }
+  float2 *rope_tab = nullptr;
   void *ws_base = nullptr;
   char *stage_K = nullptr, *stage_V = nullptr;
   int *d_status = nullptr;
@@ -1367,6 +1374,7 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
     b.base = (char *)ws_base;
     d_status = b.take<int>(4 * (size_t)nc);
     if (L->mem_space == JOLT_MEM_HOST) { stage_K = b.take<char>(span); stage_V = b.take<char>(span); }
+    if (n_rope_fused) rope_tab = b.take<float2>((size_t)(kD / 2) * L->seq_len);
     for (int i = 0; i < nc; ++i) {
       ws[i].c = H->cells[i].c;
       ws[i].active = false;
@@ -1397,6 +1405,7 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
       b.osl = L->stride_layer; b.osh = L->stride_head; b.ost = L->stride_token;
       b.tma_out = 0;
       b.dbg = g_dbg_stamps;
+      b.rope = rope_fused[i] ? rope_tab : nullptr;
       if (L->dtype == JOLT_F16 && L->stride_token % 8 == 0 && L->stride_head % 8 == 0 && L->stride_layer % 8 == 0 &&
           ((uintptr_t)obase % 16 == 0)) {
         const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)c.T, (uint64_t)c.n_heads, (uint64_t)(c.m / c.n_heads)};
@@ -1422,6 +1431,15 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
   std::stable_sort(bbc.begin(), bbc.end(), [](const tc::BBCell &x, const tc::BBCell &y) {
     return x.bits != y.bits ? x.bits > y.bits : x.r_t > y.r_t;
   });
+  if (n_rope_fused) {
+    const int T = L->seq_len;
+    const double base = rope->base;
+    const long long pos0 = rope->pos0;
+    P.add(ST_ROPE, [=](char *, cudaStream_t s) {
+      rope_table_kernel<<<dim3((T + 255) / 256, kD / 2), 256, 0, s>>>(rope_tab, T, base, pos0);
+      LAUNCHED();
+    });
+  }
   add_decode_tc(P, ST_DROWS, bbc, H->seed);
   add_backbone(P, ST_DBACK, br);
   if (!rj.empty()) {
@@ -1433,11 +1451,14 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
       LAUNCHED();
     });
   }
-  if (rope) {
-    // keys only, in place on the decoded tensor (the staging buffer when the destination is host memory)
+  // key cells the decode kernel did not rotate itself: in place on the decoded tensor (the staging buffer when the
+  // destination is host memory), one launch per cell
+  for (int i = 0; rope && i < nc; i += 2) {
+    if (rope_fused[i]) continue;
+    const int g = i / 2;
     RopeJob j;
-    j.K = Kd; j.dtype = L->dtype == JOLT_F16 ? DT_F16 : DT_F32;
-    j.n_rows = L->n_layers * L->n_kv_heads; j.n_heads = L->n_kv_heads; j.T = L->seq_len;
+    j.K = Kd + (size_t)L->group_start[g] * L->stride_layer * esz; j.dtype = L->dtype == JOLT_F16 ? DT_F16 : DT_F32;
+    j.n_rows = (L->group_start[g + 1] - L->group_start[g]) * L->n_kv_heads; j.n_heads = L->n_kv_heads; j.T = L->seq_len;
     j.sl = L->stride_layer; j.sh = L->stride_head; j.st = L->stride_token;
     j.base = rope->base; j.pos0 = rope->pos0;
     const int gx = (L->seq_len + kRopeTokensPerCta - 1) / kRopeTokensPerCta;
@@ -1725,7 +1746,7 @@ extern "C" int jolt_debug_stamps(long long *host_out, int n) {
   return cudaMemcpy(host_out, g_dbg_stamps, sizeof(long long) * n, cudaMemcpyDeviceToHost) == cudaSuccess ? JOLT_OK : JOLT_ECUDA;
 }
 extern "C" int64_t jolt_launch_count(void) { return g_launches.load(); }
-extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled & 7); }
+extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled & 15); }
 extern "C" int jolt_last_stage_ms(float *out, int32_t cap, int32_t *n) {
   if (!out || !n) return fail(JOLT_EINVAL, "null argument");
   *n = std::min<int>(cap, kNumStages);

@@ -5,7 +5,10 @@
 // of token position p pairs with feature j + 64 and the pair turns by the angle p * base^(-j/64),
 //     y_j = x_j cos - x_{j+64} sin,     y_{j+64} = x_{j+64} cos + x_j sin,        p = pos0 + t.
 //
-// One pass over the key tensor in place, bound by HBM (one read and one write of every key).  A thread owns
+// Two forms.  Key cells whose decode runs on the tensor-core kernel with r_t <= 128 are rotated inside that kernel, on
+// the accumulator row in registers, from a (cos, sin) table that rope_table_kernel writes once per call.  All other key
+// cells take rope_rows_kernel afterwards:
+// one pass over the key tensor in place, bound by HBM (one read and one write of every key).  A thread owns
 // one token and eight features of each half; its eight (cos, sin) pairs are computed once in fp64 (the angle
 // reaches pos0 + T radians, far past what an fp32 argument resolves) and reused for every (layer, head) row the
 // thread visits, so the transcendental work is T * 64 * gridDim.y evaluations per call however many heads
@@ -34,6 +37,18 @@ __device__ __forceinline__ void rope_pair(float &a, float &b, float c, float s) 
   const float ya = __fmaf_rn(a, c, -__fmul_rn(b, s));
   const float yb = __fmaf_rn(b, c, __fmul_rn(a, s));
   a = ya; b = yb;
+}
+
+// (cos, sin) of every (feature pair, token) of a call, for the decode kernel's fused rotation: tab[j * T + t].
+__global__ void __launch_bounds__(256) rope_table_kernel(float2 *tab, int T, double base, long long pos0) {
+  const int t = blockIdx.x * 256 + threadIdx.x, j = blockIdx.y;
+  __shared__ double inv_freq;
+  if (threadIdx.x == 0) inv_freq = pow(base, -(double)j / (double)(kD / 2));
+  __syncthreads();
+  if (t >= T) return;
+  double s, c;
+  sincos((double)(pos0 + t) * inv_freq, &s, &c);
+  tab[(size_t)j * T + t] = make_float2((float)c, (float)s);
 }
 
 __global__ void __launch_bounds__(256) rope_rows_kernel(RopeJob j) {

@@ -40,6 +40,7 @@ struct alignas(64) BBCell {
   int m, n_heads, T, r_t, r_f, bits, cell;
   int tiles_per_item, items_per_head;
   int *status;
+  const float2 *rope;   // DECODE of key cells: (cos, sin) of feature pair j at token t in rope[j * T + t]; null = no rotation
 };
 
 template <int BITS>

@@ -396,6 +396,108 @@ __device__ __forceinline__ bool dec_tile_loop_acc4(const BBCell &c, const DecCtx
   return ok;
 }
 
+// The loop above for key cells of a decode that re-applies the rotary embedding: feature j pairs with j + 64 and the pair turns by
+//   the angle whose (cos, sin) sit in c.rope[j * T + token] (32 consecutive tokens per warp instruction, 256 contiguous
+//   bytes, L2-resident across heads).  The accumulator row is then read in two halves, features {0..31, 64..95} and
+//   {32..63, 96..127}; the table entries of the first half are requested BEFORE the wait for the tile's MMAs and those of
+//   the second half while the first is converted and staged, so no table latency is exposed.
+template <int BITS>
+__device__ __forceinline__ bool dec_tile_loop_acc4_rope(const BBCell &c, const DecCtx &x) {
+  DecCodes<BITS> cur;
+  bool ok = true;
+  const long long row0 = (long long)x.h * c.T + x.tile0 * 128 + x.rit;
+  if (x.wg < x.n_tiles) dec_load_codes<BITS>(c, row0 + x.wg * 128, cur);
+  const int lane = x.rit & 31, wrow0 = x.rit & ~31;       // this warp's rows of the tile: wrow0 .. wrow0 + 31
+  unsigned char *obuf = x.rbuf;
+  int n = 0;
+  const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;
+  for (int i = x.wg; i < x.n_tiles; i += 2, ++n) {
+    const int acc = n & 1, ph = n >> 1;
+    const int tt = x.tile0 + i, token = tt * 128 + x.rit;
+    long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;
+    if (dbg) dbg[0] = clock64();
+    if constexpr (BITS > 0) {
+      if (ok) dec_unpack_row<BITS>(cur, x.pre, obuf, x.rit);
+      fence_proxy_async();
+      mbar_arrive(x.bRready + 16 * acc);
+      if (i + 2 < x.n_tiles) dec_load_codes<BITS>(c, row0 + (i + 2) * 128, cur);      // in flight during the MMA and the epilogue
+    }
+    if (dbg) dbg[2] = clock64();
+    float2 tb[32];
+    const float2 *tp = nullptr;
+    {
+      tp = c.rope + token;
+#pragma unroll
+      for (int k = 0; k < 32; ++k) tb[k] = __ldg(tp + (size_t)k * c.T);
+    }
+    // after a timed-out wait the warp keeps walking the loop but touches neither TMEM nor the barriers' data again
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(x.bTfull + 16 * acc, ph & 1, x.abort_flag));
+    if (dbg) dbg[3] = clock64();
+    tc_fence_after();
+    const long long off = (long long)x.l * c.osl + (long long)x.hd * c.osh + (long long)token * c.ost;
+    const uint32_t t_acc = x.t_acc + acc * 256;
+    // one 32-feature chunk of the row: scaled, rounded and put into the warp's staging rows (fp16) or stored (fp32)
+    auto emit = [&](const float *v, int ch) {
+      if (c.out_dtype == DT_F16) {
+        unsigned char *rowp = obuf + (ch >> 1) * 16384 + x.rit * 128;
+#pragma unroll
+        for (int k8 = 0; k8 < 4; ++k8) {
+          uint4 o;
+          __half2 *hp = (__half2 *)&o;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) hp[j] = __floats2half2_rn(v[k8 * 8 + 2 * j] * x.scale, v[k8 * 8 + 2 * j + 1] * x.scale);
+          *(uint4 *)(rowp + ((((ch & 1) * 4 + k8) ^ (x.rit & 7)) << 4)) = o;
+        }
+      } else {
+        float4 *p = (float4 *)((float *)c.out + off);
+#pragma unroll
+        for (int k4 = 0; k4 < 8; ++k4)
+          p[ch * 8 + k4] = make_float4(v[4 * k4] * x.scale, v[4 * k4 + 1] * x.scale, v[4 * k4 + 2] * x.scale, v[4 * k4 + 3] * x.scale);
+      }
+    };
+    {
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        float lo[32], hi[32];
+        if (ok) {
+          tmem_ld32(t_acc + half * 32, lo);
+          tmem_ld32(t_acc + 64 + half * 32, hi);
+          tmem_wait_ld();
+          if (half == 1) { tc_fence_before(); mbar_arrive(x.bTempty + 16 * acc); }
+#pragma unroll
+          for (int k = 0; k < 32; ++k) {
+            const float a = lo[k], b = hi[k];
+            lo[k] = __fmaf_rn(a, tb[k].x, -__fmul_rn(b, tb[k].y));
+            hi[k] = __fmaf_rn(b, tb[k].x, __fmul_rn(a, tb[k].y));
+          }
+        }
+        if (half == 0) {
+#pragma unroll
+          for (int k = 0; k < 32; ++k) tb[k] = __ldg(tp + (size_t)(32 + k) * c.T);
+        }
+        if (ok) { emit(lo, half); emit(hi, 2 + half); }
+      }
+      if (dbg) dbg[4] = clock64();
+    }
+    if (ok && c.out_dtype == DT_F16) {
+      __syncwarp();
+      if (dbg) dbg[5] = clock64();
+      // read back: lane l takes 16-byte chunk l & 15 of rows 2 it + (l >> 4); a row is 256 contiguous bytes of output
+      const int q16 = lane & 15;
+      __half *obase = (__half *)c.out + (long long)x.l * c.osl + (long long)x.hd * c.osh;
+#pragma unroll 4
+      for (int it = 0; it < 16; ++it) {
+        const int r = wrow0 + 2 * it + (lane >> 4);
+        const uint4 o = *(const uint4 *)(obuf + (q16 >> 3) * 16384 + r * 128 + (((q16 & 7) ^ (r & 7)) << 4));
+        *(uint4 *)(obase + (long long)(tt * 128 + r) * c.ost + q16 * 8) = o;
+      }
+      __syncwarp();
+    }
+    if (dbg) dbg[7] = clock64();
+  }
+  return ok;
+}
+
 __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBCell *__restrict__ cells, uint64_t seed) {
   using LY = DecLayout;
   constexpr int NWG = DEC_NWG;
@@ -605,7 +707,16 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
       x.s_obuf = sR + wg * 32768; x.obuf = x.rbuf;
       x.abort_flag = abort_flag; x.wg = wg; x.nwg = NWG; x.rit = rit; x.h = h; x.tile0 = tile0; x.n_tiles = n_tiles;
       x.l = h / c.n_heads; x.hd = h - x.l * c.n_heads; x.scale = scale; x.pre = pre;
-      if (acc4) {
+      if (acc4 && c.rope) {
+        switch (c.bits) {
+          case 0: dec_tile_loop_acc4_rope<0>(c, x); break;
+          case 1: dec_tile_loop_acc4_rope<1>(c, x); break;
+          case 2: dec_tile_loop_acc4_rope<2>(c, x); break;
+          case 3: dec_tile_loop_acc4_rope<3>(c, x); break;
+          case 4: dec_tile_loop_acc4_rope<4>(c, x); break;
+          default: dec_tile_loop_acc4_rope<8>(c, x); break;
+        }
+      } else if (acc4) {
         switch (c.bits) {
           case 0: dec_tile_loop_acc4<0>(c, x); break;
           case 1: dec_tile_loop_acc4<1>(c, x); break;

@@ -414,14 +414,18 @@ def test_degenerate_inputs(B):
 
 
 # --------------------------------------------------------------------------- rotary embedding re-applied to decoded keys
+@pytest.mark.parametrize("fused", [True, False])
 @pytest.mark.parametrize("dtype", ["f16", "f32"])
-def test_rope_at_decode(B, synth, dtype):
+def test_rope_at_decode(B, synth, dtype, fused):
     # Injected factors, so both sides hold the same stored backbone.  Cell 0 (keys, backbone only) admits an
     # element-wise bound; cell 2 (keys, backbone + 4-bit residual) and the value cells take the usual gate.
-    cfg = synth.CacheConfig("t", 4, 2, 2, 384, n_terms=20, seed=33, dtype=dtype)
+    # fused: the rotation inside the tensor-core decode kernel; otherwise the separate in-place pass.
+    # Key cells 0 and 2 have tensor-core shapes; key cell 4 (r_t = 24) decodes on the portable kernels and is always
+    # rotated by the separate pass.
+    cfg = synth.CacheConfig("t", 6, 2, 2, 384, n_terms=20, seed=33, dtype=dtype)
     K, V = synth.make_cache(cfg, device="cuda")
-    gs = [0, 2, 4]
-    plans = [(16, 64, 0), (16, 128, 2), (24, 96, 4), (0, 0, 4)]
+    gs = [0, 2, 4, 6]
+    plans = [(16, 64, 0), (16, 128, 2), (32, 96, 4), (0, 0, 4), (24, 96, 4), (16, 64, 2)]
     Knp, Vnp = _np(K), _np(V)
     UT, UF = [], []
     for c, (rt, rf, _) in enumerate(plans):
@@ -435,14 +439,26 @@ def test_rope_at_decode(B, synth, dtype):
     oc = oracle_cache(Knp, Vnp, gs, plans, seed=3, token_mode="exact", factors=(UT, UF), out_dtype=dtype)
     base, pos0 = 5000.0, 123457
     # a destination with padded token and head strides, and a host destination
-    pad = torch.zeros(2, 4, 2, 384 + 8, 128 + 8, dtype=K.dtype, device="cuda")
+    pad = torch.zeros(2, 6, 2, 384 + 8, 128 + 8, dtype=K.dtype, device="cuda")
     Kr, Vr = pad[0, :, :, :384, :128], pad[1, :, :, :384, :128]
-    B.jolt_decompress_rope(h, Kr, Vr, gs, base=base, pos0=pos0)
     Kh, Vh = torch.empty(K.shape, dtype=K.dtype).pin_memory(), torch.empty(V.shape, dtype=V.dtype).pin_memory()
-    B.jolt_decompress_rope(h, Kh, Vh, gs, base=base, pos0=pos0)
     Vo = torch.empty_like(V)
-    B.jolt_decompress(h, torch.empty_like(K), Vo, gs)
-    torch.cuda.synchronize()
+    prev = B.set_fast_path(15 if fused else 7)
+    try:
+        n0 = B.launch_count()
+        B.jolt_decompress_rope(h, Kr, Vr, gs, base=base, pos0=pos0)
+        n_launch = B.launch_count() - n0
+        B.jolt_decompress_rope(h, Kh, Vh, gs, base=base, pos0=pos0)
+        n0 = B.launch_count()
+        B.jolt_decompress(h, torch.empty_like(K), Vo, gs)
+        n_plain = B.launch_count() - n0
+        torch.cuda.synchronize()
+        with pytest.raises(B.JoltError):
+            B.jolt_decompress_rope(h, Kr, Vr, gs, base=0.5, pos0=0)
+    finally:
+        B.set_fast_path(prev)
+    # on top of the plain decode -- fused: the table kernel and the pass over cell 4; separate: one pass per key cell
+    assert n_launch - n_plain == (2 if fused else 3), (n_launch, n_plain)
     assert torch.equal(Kr.cpu(), Kh) and torch.equal(Vr.cpu(), Vh) and torch.equal(Vr, Vo)
     assert float(pad[:, :, :, 384:].abs().max()) == 0.0 and float(pad[..., 128:].abs().max()) == 0.0
     Kg, Vg = _np(Kr), _np(Vr)
@@ -450,21 +466,21 @@ def test_rope_at_decode(B, synth, dtype):
         Xg = cell_view(Kg, Vg, gs, c).astype(np.float64)
         Xo = O.decompress_cell_rope(o, base, pos0) if c % 2 == 0 else O.decompress_cell(o)
         rel = np.linalg.norm(Xg - Xo) / np.linalg.norm(Xo)
-        assert rel <= REL_RECON, (c, rel)
-    # cell 0: no residual, hence no threshold decisions.  The fp16 destination is rounded after decoding and again
-    # after the rotation: each input of a pair carries half an ulp, the result another half.
+        # the gate of the plain decode (the rotation is orthogonal: same relative error)
+        eo = O.rel_frobenius(cell_view(Knp, Vnp, gs, c).astype(np.float64), O.decompress_cell(o))
+        assert rel <= recon_gate(eo), (c, rel, eo)
+    # cell 0: no residual, hence no threshold decisions.  The separate pass rounds an fp16 destination after decoding
+    # and again after the rotation (each input of a pair carries half an ulp, the result another half); the fused
+    # form rounds once.  An fp32 destination gets the same bound: the decode holds the projected core G U_F^T in fp16.
+    # The floor covers the library's fp32 accumulation of the backbone where the terms cancel.
     plain = O.decompress_cell(oc[0])
     mag = np.abs(plain[..., :64]) + np.abs(plain[..., 64:])
     mag = np.concatenate([mag, mag], axis=-1)
-    # (an fp32 destination gets the same bound: the library's decode holds the projected core G U_F^T in fp16)
     ulp = 2.0 ** -10
-    # (the floor covers the library's fp32 accumulation of the backbone where the terms cancel)
     floor = 1e-5 * np.abs(plain).max()
     err = np.abs(cell_view(Kg, Vg, gs, 0).astype(np.float64) - O.decompress_cell_rope(oc[0], base, pos0))
     assert np.all(err <= ulp * mag + floor), float((err - ulp * mag).max())
     # and the rotation undone by the oracle gives back the plain decode
     back = O.rope_rotate(cell_view(Kg, Vg, gs, 0).astype(np.float64), base, pos0, inverse=True)
     assert np.all(np.abs(back - plain) <= 1.5 * ulp * mag + 2 * floor)
-    with pytest.raises(Exception):
-        B.jolt_decompress_rope(h, Kr, Vr, gs, base=0.5, pos0=0)
     h.free()
