@@ -195,6 +195,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--portable", action="store_true", help="portable SIMT kernels only")
+    ap.add_argument("--fast-mask", type=int, default=-1, help="kernel family bit mask (jolt_set_fast_path); default: all")
     args = ap.parse_args()
     args.warmup_ref = min(args.warmup, 1)
     if args.impl == "reference":
@@ -221,6 +222,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     if args.portable:
         B.set_fast_path(False)
+    elif args.fast_mask >= 0:
+        B.set_fast_path(args.fast_mask)
     W = max(args.warmup, 3)
     pk = peaks()
 

@@ -123,9 +123,11 @@ int jolt_decompress(const jolt_handle *h, const jolt_layout *out_layout, void *d
  * position p = pos0 + t and feature j < 64, with angle p * base^(-j/64),
  *     K_out[.., t, j]      = K^[.., t, j] cos - K^[.., t, j + 64] sin
  *     K_out[.., t, j + 64] = K^[.., t, j + 64] cos + K^[.., t, j] sin
- * where K^ is what jolt_decompress writes.  V is written as by jolt_decompress.  Angles are evaluated in
- * fp64, the rotation in fp32; an fp16 destination is rounded once after decoding and once after the
- * rotation.  rope: host pointer; 1 < base < 1e12, 0 <= pos0 <= 2^40 (JOLT_EINVAL otherwise).  All other
+ * where K^ is the decoded key before it is rounded to the destination type.  V is written as by
+ * jolt_decompress.  Angles are evaluated in fp64, the rotation in fp32.  Key cells decoded by the tensor-core
+ * kernel with r_t <= 128 are rotated inside that kernel and rounded once; the other key cells are rotated by a
+ * separate in-place pass over the decoded tensor, so an fp16 destination is rounded after decoding and again
+ * after the rotation (jolt_set_fast_path bit 3 off sends every cell that way).  rope: host pointer; 1 < base < 1e12, 0 <= pos0 <= 2^40 (JOLT_EINVAL otherwise).  All other
  * arguments, the result and the error behaviour are those of jolt_decompress. */
 typedef struct {
   double base;   /* frequency base (10000 in the original formulation) */

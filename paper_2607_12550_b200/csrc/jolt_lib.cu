@@ -1452,13 +1452,15 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
     });
   }
   // key cells the decode kernel did not rotate itself: in place on the decoded tensor (the staging buffer when the
-  // destination is host memory), one launch per cell
-  for (int i = 0; rope && i < nc; i += 2) {
-    if (rope_fused[i]) continue;
-    const int g = i / 2;
+  // destination is host memory), one launch per run of consecutive layer groups
+  for (int g = 0; rope && g < L->n_groups;) {
+    if (rope_fused[2 * g]) { ++g; continue; }
+    int g1 = g + 1;
+    while (g1 < L->n_groups && !rope_fused[2 * g1]) ++g1;
     RopeJob j;
     j.K = Kd + (size_t)L->group_start[g] * L->stride_layer * esz; j.dtype = L->dtype == JOLT_F16 ? DT_F16 : DT_F32;
-    j.n_rows = (L->group_start[g + 1] - L->group_start[g]) * L->n_kv_heads; j.n_heads = L->n_kv_heads; j.T = L->seq_len;
+    j.n_rows = (L->group_start[g1] - L->group_start[g]) * L->n_kv_heads; j.n_heads = L->n_kv_heads; j.T = L->seq_len;
+    g = g1;
     j.sl = L->stride_layer; j.sh = L->stride_head; j.st = L->stride_token;
     j.base = rope->base; j.pos0 = rope->pos0;
     const int gx = (L->seq_len + kRopeTokensPerCta - 1) / kRopeTokensPerCta;
