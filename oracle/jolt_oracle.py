@@ -20,6 +20,8 @@ Each function names the passage of the paper it follows:
 * Eq. (3), Eq. (4)                   -> dual_allocate
 * App. "RoPE pre vs. post on K" (keys are decomposed before the rotary embedding, which is
   re-applied at decode time)        -> rope_rotate, decompress_cell_rope
+* Sec. 7 / closing discussion (attention directly on the factors, named as the route to decode
+  parity, no algorithm given)       -> decoded_unrounded, attend_cells (the plain definition)
 
 Pins (tests/test_oracle_*.py): full-rank exactness, exact low-rank recovery, orthonormality,
 energy split, ST-HOSVD sandwich bound, norm preservation and involution of the rotation,
@@ -438,6 +440,38 @@ def decompress_cell_rope(c: "CompressedCell", base: float = 10000.0, pos0: int =
     if c.out_dtype == "f16":
         return fp16_round(Xr)
     return Xr.astype(np.float32).astype(np.float64)
+
+
+# --------------------------------------------------------------------------------------
+# Attention on the compressed cache (Sec. 7 and the closing discussion name "a fused kernel that
+# runs attention directly on the factors, without materializing the cache" as the route to decode
+# parity and give no algorithm).  The oracle is the plain definition: single-step softmax attention
+# of given queries over the decoded, not yet rounded, keys and values of one layer group.
+# --------------------------------------------------------------------------------------
+
+
+def decoded_unrounded(c: "CompressedCell"):
+    """X^ of a cell before the rounding to the output type: stored backbone + un-rotated residual."""
+    if c.r_t > 0:
+        Xh = stored_backbone(c.Gs16, c.e, c.UT16, c.UF16)
+    else:
+        Xh = np.zeros((c.m, c.T, c.d))
+    if c.bits > 0:
+        codes = unpack_codes(c.words, c.bits, c.d)
+        Xh = Xh + unrotate(dequantize_rows(codes, c.scales, c.bits, c.group), c.signs)
+    return Xh
+
+
+def attend_cells(cK: "CompressedCell", cV: "CompressedCell", Q, scale: float):
+    """Q: [m, n_q, d] (n_q queries per merged head) -> O: [m, n_q, d],
+    O[h, i] = sum_t softmax_t(scale * <Q[h, i], K^[h, t]>) V^[h, t]."""
+    Q = np.asarray(Q, dtype=np.float64)
+    Kh, Vh = decoded_unrounded(cK), decoded_unrounded(cV)
+    S = scale * np.einsum("hif,htf->hit", Q, Kh)
+    S = S - S.max(axis=-1, keepdims=True)
+    P = np.exp(S)
+    P = P / P.sum(axis=-1, keepdims=True)
+    return np.einsum("hit,htf->hif", P, Vh)
 
 
 def rel_frobenius(X, Xh):

@@ -435,3 +435,71 @@ def test_rope_invariants():
     assert abs(score(5, 2) - score(5, 3)) > 1e-6
     # composition of shifts: rotating by a then by b is rotating by a + b
     assert np.allclose(O.rope_rotate(O.rope_rotate(X[:, :1], 10000.0, 7), 10000.0, 5), O.rope_rotate(X[:, :1], 10000.0, 12), atol=1e-12)
+
+
+# --------------------------------------------------------------------------- attention on the compressed cache
+def _attend_case(seed=5, m=2, T=24, n_q=3, bits_k=4, bits_v=2, r_t=8, r_f=64):
+    rng = np.random.default_rng(seed)
+    XK = rng.standard_normal((m, T, 128)) * np.exp(0.5 * rng.standard_normal((m, T, 1)))
+    XV = rng.standard_normal((m, T, 128))
+    cK = O.compress_cell(XK, r_t, r_f, bits_k, seed=1, cell=0, token_mode="exact")
+    cV = O.compress_cell(XV, r_t, 128, bits_v, seed=1, cell=1, token_mode="exact")
+    Q = rng.standard_normal((m, n_q, 128))
+    return cK, cV, Q
+
+
+def test_attend_matches_brute_force_loops():
+    import math
+    cK, cV, Q = _attend_case()
+    scale = 1.0 / math.sqrt(128)
+    Out = O.attend_cells(cK, cV, Q, scale)
+    Kh, Vh = O.decoded_unrounded(cK), O.decoded_unrounded(cV)
+    for h in range(cK.m):
+        for i in range(Q.shape[1]):
+            s = [scale * sum(float(Q[h, i, f]) * float(Kh[h, t, f]) for f in range(128)) for t in range(cK.T)]
+            mx = max(s)
+            w = [math.exp(v - mx) for v in s]
+            z = sum(w)
+            for f in range(0, 128, 17):
+                ref = sum(w[t] * float(Vh[h, t, f]) for t in range(cK.T)) / z
+                assert abs(Out[h, i, f] - ref) <= 1e-12 * max(1.0, abs(ref))
+
+
+def test_attend_limits():
+    cK, cV, Q = _attend_case(seed=6)
+    Vh, Kh = O.decoded_unrounded(cV), O.decoded_unrounded(cK)
+    # zero query: uniform weights, the output is the mean decoded value
+    assert np.allclose(O.attend_cells(cK, cV, np.zeros_like(Q), 0.3), Vh.mean(axis=1, keepdims=True).repeat(Q.shape[1], 1))
+    # zero scale: the same
+    assert np.allclose(O.attend_cells(cK, cV, Q, 0.0), Vh.mean(axis=1, keepdims=True).repeat(Q.shape[1], 1))
+    # very sharp softmax: the output is the decoded value at the best-scoring token
+    Out = O.attend_cells(cK, cV, Q, 1e4)
+    best = np.einsum("hif,htf->hit", Q, Kh).argmax(axis=-1)
+    for h in range(cK.m):
+        for i in range(Q.shape[1]):
+            assert np.allclose(Out[h, i], Vh[h, best[h, i]], atol=1e-9)
+    # the unrounded decode rounds to what decompress_cell returns
+    assert np.array_equal(O.fp16_round(Kh), O.decompress_cell(cK))
+
+
+def test_attend_scores_on_the_factors_identity():
+    # The identity behind attention on the factors: with P_h the stored projected core,
+    #   <q, K^[h, t]> = sum_k U_T[t, k] (P_h q)[k] 2^e  +  <H(s . q) / sqrt(d), r^'[h, t]>,
+    # and for the values  sum_t p_t V^[h, t] = 2^e (p^T U_T) P_h + s . H(sum_t p_t r^'[h, t]) / sqrt(d).
+    import math
+    cK, cV, Q = _attend_case(seed=7, bits_k=3, bits_v=4)
+    Kh, Vh = O.decoded_unrounded(cK), O.decoded_unrounded(cV)
+    PK = O.fp16_round(np.einsum("hrs,fs->hrf", cK.Gs16, cK.UF16))
+    rK = O.dequantize_rows(O.unpack_codes(cK.words, cK.bits, 128), cK.scales, cK.bits, cK.group)
+    S_fact = math.ldexp(1.0, cK.e) * np.einsum("tk,hik->hit", cK.UT16, np.einsum("hkf,hif->hik", PK, Q)) \
+        + np.einsum("hif,htf->hit", O.rotate(Q, cK.signs), rK)
+    S_def = np.einsum("hif,htf->hit", Q, Kh)
+    assert np.abs(S_fact - S_def).max() <= 1e-11 * np.abs(S_def).max()
+    rng = np.random.default_rng(0)
+    Pw = rng.random((cV.m, 2, cV.T))
+    PV = O.fp16_round(np.einsum("hrs,fs->hrf", cV.Gs16, cV.UF16))
+    rV = O.dequantize_rows(O.unpack_codes(cV.words, cV.bits, 128), cV.scales, cV.bits, cV.group)
+    O_fact = math.ldexp(1.0, cV.e) * np.einsum("hik,hkf->hif", np.einsum("hit,tk->hik", Pw, cV.UT16), PV) \
+        + O.unrotate(np.einsum("hit,htf->hif", Pw, rV), cV.signs)
+    O_def = np.einsum("hit,htf->hif", Pw, Vh)
+    assert np.abs(O_fact - O_def).max() <= 1e-11 * np.abs(O_def).max()
