@@ -136,6 +136,21 @@ typedef struct {
 int jolt_decompress_rope(const jolt_handle *h, const jolt_layout *out_layout, void *dK_out, void *dV_out,
                          const jolt_rope *rope, void *stream);
 
+/* jolt_attend -- paper Sec. 7 and closing discussion: attention "directly on the factors, without materializing
+ * the cache" is named as the route to decode parity; no algorithm is given.  This entry point computes single-step
+ * softmax attention over the compressed cache, for every layer and KV head at once:
+ *     O[l, h, i, :] = sum_t softmax_t( scale * <Q[l, h, i, :], K^[l, h, t, :]> ) V^[l, h, t, :]
+ * where K^, V^ are the decoded cells before their rounding to an output type (what jolt_decompress would write to an
+ * fp32 destination, up to fp32 rounding).  Neither is formed: the backbone terms are contracted with the small factors
+ * first, the residual terms against a query rotated once per head, so the call reads the compressed bytes once.
+ *   dQ, dOut: device, fp32, contiguous [n_layers][n_kv_heads][n_q][128], 16-byte aligned; n_q = queries per KV head,
+ *   1..8 (the grouped-query group size).  Keys are used as stored: a cache whose keys were compressed before a rotary
+ *   embedding needs jolt_decompress_rope instead (the rotation differs per token and does not commute with the
+ *   contraction).  Scratch comes from the library's per-device workspace (grown on first use).  Errors: JOLT_EINVAL
+ *   (null / misaligned pointers, n_q out of range, wrong device), JOLT_EUNSUPPORTED (ranks that are not multiples
+ *   of 8; sequences beyond about 300 k tokens), JOLT_ENOMEM, JOLT_ECUDA.  Asynchronous on `stream`. */
+int jolt_attend(const jolt_handle *h, const void *dQ, int32_t n_q, double scale, void *dOut, void *stream);
+
 /* jolt_decompress_static -- the paper has no counterpart; this is a deployment variant of jolt_decompress
  * for callers that cannot allocate device memory while decoding (a serving process that has given all free
  * memory to its own pool, a thread for which a driver allocation would stall the context, a host whose

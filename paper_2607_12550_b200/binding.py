@@ -62,6 +62,7 @@ class Rope(C.Structure):
 
 lib.jolt_decompress_rope.argtypes = [_vp, C.POINTER(Layout), _vp, _vp, C.POINTER(Rope), _vp]
 lib.jolt_decompress_static.argtypes = [_vp, C.POINTER(Layout), _vp, _vp, _vp]
+lib.jolt_attend.argtypes = [_vp, _vp, C.c_int32, C.c_double, _vp, _vp]
 lib.jolt_compressed_bytes.argtypes = [_vp, C.POINTER(C.c_int64)]
 lib.jolt_get_component.argtypes = [_vp, C.c_int32, C.c_int32, _vp, C.c_int64, C.POINTER(C.c_int64)]
 lib.jolt_allocate.argtypes = [C.c_int32, C.POINTER(C.c_int32), C.c_int32, C.c_int32, C.POINTER(C.c_double),
@@ -234,6 +235,15 @@ def jolt_decompress_static(handle: Handle, K_out, V_out, group_start, stream=Non
     """Decode without any device allocation (fixed 16 MiB scratch inside the library); see include/jolt.h."""
     lay = make_layout(K_out, group_start, V_out)
     _check(lib.jolt_decompress_static(handle.ptr, C.byref(lay), K_out.data_ptr(), V_out.data_ptr(), _stream_ptr(stream)))
+
+
+def jolt_attend(handle: Handle, Q, scale=None, stream=None):
+    """Single-step attention of Q [n_layers, n_kv_heads, n_q, 128] (fp32, CUDA) over the compressed cache; see include/jolt.h."""
+    assert Q.dim() == 4 and Q.dtype == torch.float32 and Q.is_cuda and Q.is_contiguous()
+    out = torch.empty_like(Q)
+    sc = float(scale) if scale is not None else 1.0 / (Q.shape[-1] ** 0.5)
+    _check(lib.jolt_attend(handle.ptr, Q.data_ptr(), Q.shape[2], sc, out.data_ptr(), _stream_ptr(stream)))
+    return out
 
 
 def jolt_free(handle: Handle):

@@ -21,6 +21,7 @@
 #include "small_solvers.cuh"
 #include "block_jacobi.cuh"
 #include "rope.cuh"
+#include "attend.cuh"
 
 using namespace jolt;
 
@@ -45,7 +46,7 @@ int fail(int code, const char *fmt, ...) {
 // ------------------------------------------------------------------ stage timing
 static const char *kStageNames[] = {"stage_in", "sketch_gen", "gram", "eig_feat", "sketch", "orth", "power", "project",
                                     "small_svd", "factors", "store", "backbone", "residual_quant", "decode_backbone",
-                                    "decode_rows", "rope", "stage_out"};
+                                    "decode_rows", "rope", "attend", "stage_out"};
 constexpr int kNumStages = sizeof(kStageNames) / sizeof(kStageNames[0]);
 struct StageTimer {
   cudaEvent_t ev[kNumStages + 1];
@@ -67,7 +68,7 @@ struct StageTimer {
 };
 thread_local StageTimer g_timer;
 enum { ST_IN = 0, ST_SKGEN, ST_GRAM, ST_EIGF, ST_SKETCH, ST_ORTH, ST_POWER, ST_PROJ, ST_SVD, ST_FACT, ST_STORE, ST_BACK,
-       ST_RQ, ST_DBACK, ST_DROWS, ST_ROPE, ST_OUT };
+       ST_RQ, ST_DBACK, ST_DROWS, ST_ROPE, ST_ATT, ST_OUT };
 
 // ------------------------------------------------------------------ workspace cache (per device)
 struct Workspace { void *base = nullptr; size_t cap = 0; };
@@ -1494,6 +1495,112 @@ extern "C" int jolt_decompress_rope(const jolt_handle *H, const jolt_layout *L, 
                                     const jolt_rope *rope, void *stream) {
   if (!rope) return fail(JOLT_EINVAL, "rotary parameters are null");
   return decompress_impl(H, L, Kout, Vout, rope, stream);
+}
+
+// ------------------------------------------------------------------ attention on the compressed cache
+template <int BITS>
+static void launch_att_scores(dim3 grid, size_t shm, cudaStream_t s, const AttendJob *d, int NQP) {
+  attend_scores_kernel<BITS><<<grid, kAttChunk, shm, s>>>(d, NQP);
+}
+template <int BITS>
+static void launch_att_values(dim3 grid, size_t shm, cudaStream_t s, const AttendJob *d, int NQP) {
+  attend_values_kernel<BITS><<<grid, kAttChunk, shm, s>>>(d, NQP);
+}
+
+extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, double scale, void *dOut, void *stream) {
+  if (!H || !dQ || !dOut) return fail(JOLT_EINVAL, "null argument");
+  if (n_q < 1 || n_q > kAttMaxQ) return fail(JOLT_EINVAL, "n_q %d (1..%d queries per KV head)", n_q, kAttMaxQ);
+  if (!(scale == scale) || std::isinf(scale)) return fail(JOLT_EINVAL, "scale is not finite");
+  if ((((uintptr_t)dQ) | ((uintptr_t)dOut)) & 15) return fail(JOLT_EINVAL, "queries and outputs must start on a 16-byte boundary");
+  cudaStream_t st = (cudaStream_t)stream;
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
+  if (dev != H->device) return fail(JOLT_EINVAL, "handle belongs to device %d, current device is %d", H->device, dev);
+  const int ng = H->n_groups, T = H->T, nh = H->n_kv_heads;
+  const int NQP = n_q <= 4 ? 4 : 8;
+  const int n_chunks = (T + kAttChunk - 1) / kAttChunk;
+  int m_max = 0, krt = 0, krf = 0, vrt = 0, vrf = 0;
+  unsigned kbits = 0, vbits = 0;
+  for (int g = 0; g < ng; ++g) {
+    const CellDesc &ck = H->cells[2 * g].c, &cv = H->cells[2 * g + 1].c;
+    m_max = std::max(m_max, ck.m);
+    krt = std::max(krt, ck.r_t); krf = std::max(krf, ck.r_t > 0 ? ck.r_f : 0);
+    vrt = std::max(vrt, cv.r_t); vrf = std::max(vrf, cv.r_t > 0 ? cv.r_f : 0);
+    kbits |= 1u << ck.bits; vbits |= 1u << cv.bits;
+    if ((ck.r_t % 8) || (cv.r_t % 8) || (ck.r_f % 8) || (cv.r_f % 8)) return fail(JOLT_EUNSUPPORTED, "ranks must be multiples of 8");
+  }
+  const size_t shm_prep = (size_t)128 * krf * sizeof(__half) + 160 * sizeof(float);
+  const size_t shm_sc = (size_t)(128 + krt) * NQP * sizeof(float);
+  const size_t shm_comb = (size_t)128 * vrf * sizeof(__half) + (size_t)(n_chunks + vrt) * NQP * sizeof(float) + 136 * sizeof(float);
+  if (shm_comb > 48 * 1024) return fail(JOLT_EUNSUPPORTED, "sequence of %d tokens: the chunk merge needs %zu bytes of shared memory", T, shm_comb);
+  std::vector<AttendJob> jobs(ng);
+  void *ws_base = nullptr;
+  int rc;
+  for (int pass = 0; pass < 2; ++pass) {
+    Bump b;
+    b.base = (char *)ws_base;
+    for (int g = 0; g < ng; ++g) {
+      const CellStore &sk = H->cells[2 * g], &sv = H->cells[2 * g + 1];
+      AttendJob &j = jobs[g];
+      auto fill = [](AttendCell &a, const CellStore &cs) {
+        a.G = cs.G16; a.UT = cs.UT16; a.UF = cs.UF16; a.e = cs.e; a.words = cs.words; a.scales = cs.scales;
+        a.r_t = cs.c.r_t; a.r_f = cs.c.r_t > 0 ? cs.c.r_f : 0; a.bits = cs.c.bits; a.cell = cs.c.cell;
+      };
+      fill(j.k, sk); fill(j.v, sv);
+      j.m = sk.c.m; j.T = T;
+      const size_t row0 = (size_t)H->group_start[g] * nh * n_q * kD;
+      j.q = (const float *)dQ + row0; j.out = (float *)dOut + row0;
+      j.w = b.take<float>((size_t)j.m * std::max(j.k.r_t, 1) * NQP);
+      j.qt = b.take<float>((size_t)j.m * kD * NQP);
+      j.p = b.take<float>((size_t)j.m * T * NQP);
+      j.ml = b.take<float>((size_t)j.m * n_chunks * 2 * NQP);
+      j.y = b.take<float>((size_t)j.m * n_chunks * std::max(j.v.r_t, 1) * NQP);
+      j.a = b.take<float>((size_t)j.m * n_chunks * kD * NQP);
+    }
+    if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) return rc;
+  }
+  Program P;
+  const size_t off = P.push(jobs);
+  const uint64_t seed = H->seed;
+  const float fscale = (float)scale;
+  P.add(ST_ATT, [=](char *dev_t, cudaStream_t s) {
+    const AttendJob *d = (const AttendJob *)(dev_t + off);
+    attend_prep_kernel<<<dim3(m_max, ng), 128, shm_prep, s>>>(d, n_q, NQP, fscale, seed);
+    LAUNCHED();
+    const dim3 grid(n_chunks, m_max, ng);
+    for (int b = 0; b <= 8; ++b) {
+      if (!((kbits >> b) & 1)) continue;
+      switch (b) {
+        case 0: launch_att_scores<0>(grid, shm_sc, s, d, NQP); break;
+        case 1: launch_att_scores<1>(grid, shm_sc, s, d, NQP); break;
+        case 2: launch_att_scores<2>(grid, shm_sc, s, d, NQP); break;
+        case 3: launch_att_scores<3>(grid, shm_sc, s, d, NQP); break;
+        case 4: launch_att_scores<4>(grid, shm_sc, s, d, NQP); break;
+        default: launch_att_scores<8>(grid, shm_sc, s, d, NQP); break;
+      }
+      LAUNCHED();
+    }
+    for (int b = 0; b <= 8; ++b) {
+      if (!((vbits >> b) & 1)) continue;
+      const size_t shm = (size_t)kAttChunk * (NQP * sizeof(float) + 16 * std::max(b, 1) + 8) + (size_t)128 * NQP * sizeof(float);
+      switch (b) {
+        case 0: launch_att_values<0>(grid, shm, s, d, NQP); break;
+        case 1: launch_att_values<1>(grid, shm, s, d, NQP); break;
+        case 2: launch_att_values<2>(grid, shm, s, d, NQP); break;
+        case 3: launch_att_values<3>(grid, shm, s, d, NQP); break;
+        case 4: launch_att_values<4>(grid, shm, s, d, NQP); break;
+        default: launch_att_values<8>(grid, shm, s, d, NQP); break;
+      }
+      LAUNCHED();
+    }
+    attend_combine_kernel<<<dim3(m_max, ng), 128, shm_comb, s>>>(d, n_q, NQP, n_chunks, seed);
+    LAUNCHED();
+  });
+  void *d_tab = nullptr;
+  if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
+  g_timer.begin(st);
+  if ((rc = run_program(P, (char *)d_tab, st))) return rc;
+  return JOLT_OK;
 }
 
 extern "C" int jolt_free(jolt_handle *H) {

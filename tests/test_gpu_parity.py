@@ -484,3 +484,53 @@ def test_rope_at_decode(B, synth, dtype, fused):
     back = O.rope_rotate(cell_view(Kg, Vg, gs, 0).astype(np.float64), base, pos0, inverse=True)
     assert np.all(np.abs(back - plain) <= 1.5 * ulp * mag + 2 * floor)
     h.free()
+
+
+# --------------------------------------------------------------------------- attention on the compressed cache
+@pytest.mark.parametrize("case", ["a", "b"])
+def test_attend_on_the_factors(B, synth, case):
+    # Injected factors (both sides hold the same stored backbone).  T = 384 leaves a 128-token tail chunk.
+    cfg = synth.CacheConfig("t", 4, 2, 2, 384, n_terms=20, seed=51)
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2, 4]
+    if case == "a":
+        plans, n_q = [(16, 64, 4), (16, 128, 2), (32, 96, 3), (0, 0, 8)], 4
+    else:
+        plans, n_q = [(0, 0, 4), (24, 96, 0), (16, 128, 1), (16, 64, 4)], 5
+    Knp, Vnp = _np(K), _np(V)
+    UT, UF = [], []
+    for c, (rt, rf, _) in enumerate(plans):
+        if rt == 0:
+            UT.append(None); UF.append(None)
+            continue
+        o = O.compress_cell(cell_view(Knp, Vnp, gs, c), rt, rf, 0, token_mode="exact")
+        UT.append(o.UT16.astype(np.float32)); UF.append(o.UF16.astype(np.float32))
+    opts = B.default_options(seed=3)
+    h = B.jolt_compress(K, V, gs, plans, opts, factors=(UT, UF))
+    oc = oracle_cache(Knp, Vnp, gs, plans, seed=3, token_mode="exact", factors=(UT, UF), out_dtype="f32")
+    g = torch.Generator().manual_seed(9)
+    Q = torch.randn(4, 2, n_q, 128, generator=g)
+    Q[0, 0, 0] *= 4.0                      # one sharp row
+    Q[1, 1, n_q - 1] = 0.0                 # one uniform row
+    scale = 1.0 / 128 ** 0.5
+    out = B.jolt_attend(h, Q.cuda(), scale)
+    # the same attention over the library's own fp32 decode (a second CUDA path: consistency, not parity)
+    Kd, Vd = torch.empty(K.shape, dtype=torch.float32, device="cuda"), torch.empty(V.shape, dtype=torch.float32, device="cuda")
+    B.jolt_decompress(h, Kd, Vd, gs)
+    torch.cuda.synchronize()
+    S = torch.einsum("lhif,lhtf->lhit", Q.cuda().double(), Kd.double()) * scale
+    ref2 = torch.einsum("lhit,lhtf->lhif", torch.softmax(S, dim=-1), Vd.double())
+    outn = out.cpu().numpy().astype(np.float64)
+    # (the decode kernel accumulates on the tensor cores, measured relative error up to 2e-5; jolt_attend is plain fp32)
+    assert float((out.double() - ref2).norm() / ref2.norm()) <= 1e-4
+    for gi in range(2):
+        Qg = Q[gs[gi]:gs[gi + 1]].reshape(-1, n_q, 128).numpy()
+        ref = O.attend_cells(oc[2 * gi], oc[2 * gi + 1], Qg, scale)
+        got = outn[gs[gi]:gs[gi + 1]].reshape(-1, n_q, 128)
+        # the two sides quantise the residual independently: a small share of codes differs by one step, which
+        # moves keys and values by the gate of the plain decode; the attention output inherits that gate
+        eo = max(O.rel_frobenius(cell_view(Knp, Vnp, gs, 2 * gi + w).astype(np.float64), O.decompress_cell(oc[2 * gi + w])) for w in (0, 1))
+        rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+        assert rel <= 3 * recon_gate(eo), (gi, rel, eo)
+    assert B.lib.jolt_attend(h.ptr, Q.cuda().data_ptr(), 9, scale, out.data_ptr(), None) == B.EINVAL    # n_q > 8
+    h.free()
