@@ -192,6 +192,8 @@ def main():
     ap.add_argument("--ratio", type=float, default=0.0, help="compression ratio of the byte budget (default: the workload's)")
     ap.add_argument("--rope", action="store_true",
                     help="decode through jolt_decompress_rope (keys rotated at decode; not the headline workload)")
+    ap.add_argument("--attend", type=int, default=0, metavar="N_Q",
+                    help="also time jolt_attend (attention on the compressed cache) with N_Q queries per KV head")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--portable", action="store_true", help="portable SIMT kernels only")
@@ -303,6 +305,30 @@ def main():
     rel_k = sum(errs[0::2]) / ng
     rel_v = sum(errs[1::2]) / ng
 
+    # attention computed on the compressed cache (not part of the headline metric)
+    attend = None
+    if args.attend:
+        h = B.jolt_compress(K, V, gs, plans, opts)
+        Qa = torch.randn(K.shape[0], K.shape[1], args.attend, 128, device=K.device)
+        for _ in range(3):
+            B.jolt_attend(h, Qa)
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(max(args.steps, 5)):
+            a0, a1 = ev(), ev()
+            a0.record()
+            B.jolt_attend(h, Qa)
+            a1.record()
+            torch.cuda.synchronize()
+            ts.append(a0.elapsed_time(a1))
+        ts.sort()
+        t_att = ts[len(ts) // 2]
+        attend = {"n_q": args.attend, "ms": t_att, "compressed_bytes": planned_bytes,
+                  "gbs_of_compressed": planned_bytes / (t_att * 1e-3) / 1e9,
+                  "frac_of_hbm_peak": planned_bytes / (t_att * 1e-3) / 1e9 / pk["hbm"],
+                  "decode_then_read_ms": td + cache_bytes / (pk["hbm"] * 1e9) * 1e3}
+        h.free()
+
     # end to end through the public API with host buffers (pinned), copies inside the timed region
     e2e = None
     if not args.no_e2e:
@@ -386,6 +412,8 @@ def main():
             "compress_roofline_ms": t_roof_c * 1e3, "decompress_roofline_ms": t_roof_d * 1e3,
             "rel_frobenius_error": {"K": rel_k, "V": rel_v},
             "stages_ms": stages, "roofline": roofline, "gpu_launches": launches, "clocks": clocks, "e2e": e2e}
+    if attend:
+        line["attend"] = attend
 
     if not args.no_cpu_baseline and world == 1:
         from oracle import jolt_oracle as O

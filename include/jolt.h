@@ -146,7 +146,10 @@ int jolt_decompress_rope(const jolt_handle *h, const jolt_layout *out_layout, vo
  *   dQ, dOut: device, fp32, contiguous [n_layers][n_kv_heads][n_q][128], 16-byte aligned; n_q = queries per KV head,
  *   1..8 (the grouped-query group size).  Keys are used as stored: a cache whose keys were compressed before a rotary
  *   embedding needs jolt_decompress_rope instead (the rotation differs per token and does not commute with the
- *   contraction).  Scratch comes from the library's per-device workspace (grown on first use).  Errors: JOLT_EINVAL
+ *   contraction).  Scratch comes from the library's per-device workspace (grown on first use).  The first call on a
+ *   handle also forms the projected cores P_h = fp16(G_h U_F^T) of all cells (m * r_t * 128 fp16 values per cell,
+ *   about 5 % of the compressed size on the benchmark workload) in a device buffer that stays with the handle
+ *   until jolt_free; later calls, on any stream, reuse them.  Errors: JOLT_EINVAL
  *   (null / misaligned pointers, n_q out of range, wrong device), JOLT_EUNSUPPORTED (ranks that are not multiples
  *   of 8; sequences beyond about 300 k tokens), JOLT_ENOMEM, JOLT_ECUDA.  Asynchronous on `stream`. */
 int jolt_attend(const jolt_handle *h, const void *dQ, int32_t n_q, double scale, void *dOut, void *stream);

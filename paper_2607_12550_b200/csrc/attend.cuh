@@ -11,7 +11,8 @@
 // so a call streams U_T and the packed codes once each (the compressed bytes) instead of the fp16 cache, and the
 // Hadamard rotation is applied to one query / one output row per head instead of every token.
 //
-// Four kernels, all CUDA-core (the work is a stream of 1..8-bit codes against a handful of query vectors):
+// Five kernels, all CUDA-core (the work is a stream of 1..8-bit codes against a handful of query vectors):
+//   attend_p16_kernel      P_h = fp16(G_h U_F^T) of every head of both cells (what the decoder's set-up also forms)
 //   attend_prep_kernel     per (group, head): rotated scaled queries and w = scale 2^e P_h q
 //   attend_scores_kernel   per (group, head, 256-token chunk): scores, chunk maximum, p = exp(s - max), chunk sum
 //   attend_values_kernel   per (group, head, chunk): p^T U_T and sum_t p_t r^'_t (codes staged in shared memory and
@@ -43,6 +44,7 @@ struct AttendJob {                  // one per layer group
   int m, T;
   const float *q;                   // [m][n_q][128]
   float *out;                       // [m][n_q][128]
+  __half *kP, *vP;                  // [m * r_t][128]    P_h = fp16(G_h U_F^T) of the key / value cell (scaled units)
   float *w;                         // [m][k.r_t][NQP]   scale 2^e P_h q
   float *qt;                        // [m][128][NQP]     scale H(s . q) / sqrt(d)
   float *p;                         // [m][T][NQP]       exp(s - chunk maximum)
@@ -79,57 +81,79 @@ __device__ __forceinline__ void att_stage_uf(const AttendCell &c, __half *ufs, i
   }
 }
 
-// P_h[k][f] = fp16( sum_s G_h[k][s] U_F[f][s] ), the decoder's projected core in scaled units
-__device__ __forceinline__ float att_p16(const __half *__restrict__ grow, const __half *ufs, int r_f, int f) {
-  float acc = 0.f;
-  for (int s = 0; s < r_f; s += 8) {
-    const uint4 g8 = __ldg((const uint4 *)(grow + s));
-    const __half *gh = (const __half *)&g8;
+// P_h[k][f] = fp16( sum_s G_h[k][s] U_F[f][s] ), the decoder's projected core in scaled units, for both cells of every
+// group.  grid (row blocks of kAttPRows, 2 * groups), 128 threads (thread = feature); dynamic shared memory: 128 * r_f halves.
+constexpr int kAttPRows = 32;
+__global__ void __launch_bounds__(128) attend_p16_kernel(const AttendJob *__restrict__ jobs) {
+  const AttendJob &jb = jobs[blockIdx.y >> 1];
+  const AttendCell &c = (blockIdx.y & 1) ? jb.v : jb.k;
+  __half *P = (blockIdx.y & 1) ? jb.vP : jb.kP;
+  const int rows = jb.m * c.r_t, r0 = blockIdx.x * kAttPRows, f = threadIdx.x;
+  if (r0 >= rows) return;
+  extern __shared__ unsigned char att_smem[];
+  __half *ufs = (__half *)att_smem;
+  att_stage_uf(c, ufs, f, 128);
+  __syncthreads();
+  const int r_f = c.r_f;
+  for (int rb = r0; rb < min(r0 + kAttPRows, rows); rb += 8) {      // rows are a multiple of 8 (r_t is)
+    float acc[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc = fmaf(__half2float(gh[j]), __half2float(ufs[(s + j) * 128 + f]), acc);
+    for (int r = 0; r < 8; ++r) acc[r] = 0.f;
+    for (int s = 0; s < r_f; s += 8) {
+      uint4 g8[8];
+#pragma unroll
+      for (int r = 0; r < 8; ++r) g8[r] = __ldg((const uint4 *)(c.G + (size_t)(rb + r) * r_f + s));
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float u = __half2float(ufs[(s + j) * 128 + f]);
+#pragma unroll
+        for (int r = 0; r < 8; ++r) acc[r] = fmaf(__half2float(((const __half *)&g8[r])[j]), u, acc[r]);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < 8; ++r) P[(size_t)(rb + r) * 128 + f] = __float2half_rn(acc[r]);
   }
-  return __half2float(__float2half_rn(acc));
 }
 
-// grid (m, groups), 128 threads (thread = feature), dynamic shared memory: 128 * r_f halves + 128 floats + 32 floats
+// grid (m, groups, NQP), 128 threads (thread = feature), 128 floats of dynamic shared memory.  CTA z rotates query z
+// and forms every NQP-th group of four rows of w.
 __global__ void __launch_bounds__(128) attend_prep_kernel(const AttendJob *__restrict__ jobs, int n_q, int NQP, float scale,
                                                           uint64_t seed) {
   const AttendJob &jb = jobs[blockIdx.y];
-  const int h = blockIdx.x, f = threadIdx.x;
+  const int h = blockIdx.x, f = threadIdx.x, i = blockIdx.z;
   if (h >= jb.m) return;
   extern __shared__ unsigned char att_smem[];
-  __half *ufs = (__half *)att_smem;
-  float *buf = (float *)(att_smem + (size_t)128 * jb.k.r_f * sizeof(__half));
-  float *red = buf + 128;
-  float q[kAttMaxQ];
-#pragma unroll
-  for (int i = 0; i < kAttMaxQ; ++i) q[i] = i < n_q ? jb.q[((size_t)h * n_q + i) * 128 + f] : 0.f;
+  float *buf = (float *)att_smem;
   if (jb.k.bits > 0) {
-    const float sg = att_sign(seed, jb.k.cell, f);
-    for (int i = 0; i < NQP; ++i) {
-      buf[f] = sg * q[i];
-      __syncthreads();
-      const float v = att_wht_smem(buf, f);
-      jb.qt[((size_t)h * 128 + f) * NQP + i] = v * kInvSqrtD * scale;
-      __syncthreads();
-    }
+    buf[f] = i < n_q ? att_sign(seed, jb.k.cell, f) * jb.q[((size_t)h * n_q + i) * 128 + f] : 0.f;
+    __syncthreads();
+    const float v = att_wht_smem(buf, f);
+    jb.qt[((size_t)h * 128 + f) * NQP + i] = v * kInvSqrtD * scale;
   }
   if (jb.k.r_t > 0) {
-    att_stage_uf(jb.k, ufs, f, 128);
-    __syncthreads();
+    // w[k][q] = scale 2^e sum_f P_h[k][f] q_q[f]: a warp per row k, a lane per four features
     const float se = scale * ldexpf(1.f, *jb.k.e);
     const int warp = f >> 5, lane = f & 31;
-    for (int k = 0; k < jb.k.r_t; ++k) {
-      const float pk = att_p16(jb.k.G + ((size_t)h * jb.k.r_t + k) * jb.k.r_f, ufs, jb.k.r_f, f);
-      for (int i = 0; i < NQP; ++i) {
-        float v = pk * q[i];
+    float q[kAttMaxQ][4];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) red[warp * kAttMaxQ + i] = v;
-      }
-      __syncthreads();
-      if (f < NQP) jb.w[((size_t)h * jb.k.r_t + k) * NQP + f] = se * (red[f] + red[kAttMaxQ + f] + red[2 * kAttMaxQ + f] + red[3 * kAttMaxQ + f]);
-      __syncthreads();
+    for (int c = 0; c < kAttMaxQ; ++c) {
+      const float4 v = c < n_q ? *(const float4 *)(jb.q + ((size_t)h * n_q + c) * 128 + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      q[c][0] = v.x; q[c][1] = v.y; q[c][2] = v.z; q[c][3] = v.w;
+    }
+    for (int k = warp + 4 * blockIdx.z; k < jb.k.r_t; k += 4 * gridDim.z) {
+      const uint2 p4 = __ldg((const uint2 *)(jb.kP + ((size_t)h * jb.k.r_t + k) * 128 + lane * 4));
+      const __half *ph = (const __half *)&p4;
+      const float p0 = __half2float(ph[0]), p1 = __half2float(ph[1]), p2 = __half2float(ph[2]), p3 = __half2float(ph[3]);
+      float v[kAttMaxQ];
+#pragma unroll
+      for (int c = 0; c < kAttMaxQ; ++c) v[c] = fmaf(p0, q[c][0], fmaf(p1, q[c][1], fmaf(p2, q[c][2], p3 * q[c][3])));
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int c = 0; c < kAttMaxQ; ++c) v[c] += __shfl_xor_sync(0xffffffffu, v[c], o);
+#pragma unroll
+      for (int c = 0; c < kAttMaxQ; ++c)
+        if (lane == 0 && c < NQP) jb.w[((size_t)h * jb.k.r_t + k) * NQP + c] = se * v[c];
     }
   }
 }
@@ -145,7 +169,7 @@ __device__ __forceinline__ uint32_t att_code(const uint32_t *row, int g, int j) 
 
 // grid (n_chunks, m, groups), kAttChunk threads (thread = token).  Dynamic shared memory: (128 + r_t) * NQP floats.
 template <int BITS>
-__global__ void __launch_bounds__(kAttChunk) attend_scores_kernel(const AttendJob *__restrict__ jobs, int NQP) {
+__global__ void __launch_bounds__(kAttChunk, 3) attend_scores_kernel(const AttendJob *__restrict__ jobs, int NQP) {
   const AttendJob &jb = jobs[blockIdx.z];
   if (jb.k.bits != BITS) return;
   const int h = blockIdx.y, chunk = blockIdx.x;
@@ -154,10 +178,19 @@ __global__ void __launch_bounds__(kAttChunk) attend_scores_kernel(const AttendJo
   float *qts = (float *)att_smem;                   // [128][NQP]
   float *ws = qts + 128 * NQP;                      // [r_t][NQP]
   __shared__ float red[2][kAttChunk / 32][kAttMaxQ];
+  __shared__ float qsum[4 * kAttMaxQ];              // per 32-feature group: sum of the rotated query's entries
   const int tid = threadIdx.x, r_t = jb.k.r_t;
   if (BITS > 0)
     for (int i = tid; i < 128 * NQP; i += kAttChunk) qts[i] = jb.qt[(size_t)h * 128 * NQP + i];
   for (int i = tid; i < r_t * NQP; i += kAttChunk) ws[i] = jb.w[(size_t)h * r_t * NQP + i];
+  __syncthreads();
+  if (BITS > 0 && tid < 4 * kAttMaxQ) {
+    const int g = tid / kAttMaxQ, i = tid % kAttMaxQ;
+    float a = 0.f;
+    if (i < NQP)
+      for (int j = 0; j < 32; ++j) a += qts[(g * 32 + j) * NQP + i];
+    qsum[tid] = a;
+  }
   __syncthreads();
   const int t = chunk * kAttChunk + tid;
   const bool live = t < jb.T;
@@ -172,40 +205,51 @@ __global__ void __launch_bounds__(kAttChunk) attend_scores_kernel(const AttendJo
       for (int i = 0; i < BITS; ++i) { const uint4 v = __ldg(wp + i); row[4 * i] = v.x; row[4 * i + 1] = v.y; row[4 * i + 2] = v.z; row[4 * i + 3] = v.w; }
       __half sc[4];
       *(uint2 *)sc = __ldg((const uint2 *)(jb.k.scales + ((size_t)h * jb.T + t) * 4));
-      constexpr float off = 0.5f - (float)(1 << (BITS - 1));
-      for (int qq = 0; qq < NQP; qq += 4) {
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      // integer code to float without a conversion instruction: 2^23 + u, minus (2^23 + 2^(b-1))
+      // (the half-step offset is applied per group through the sum of the group's query entries, qsum)
+      constexpr float off = 8388608.0f + (float)(1 << (BITS - 1));
+      const bool q8 = NQP == 8;
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          const float delta = __half2float(sc[g]);
-          float g0 = 0.f, g1 = 0.f, g2 = 0.f, g3 = 0.f;
+      for (int g = 0; g < 4; ++g) {
+        float g0 = 0.f, g1 = 0.f, g2 = 0.f, g3 = 0.f, g4 = 0.f, g5 = 0.f, g6 = 0.f, g7 = 0.f;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            // integer code to float without a conversion instruction: 2^23 + u, minus 2^23
-            const float val = __uint_as_float(0x4B000000u | att_code<BITS>(row, g, j)) - 8388608.0f + off;
-            const float4 qv = *(const float4 *)(qts + (g * 32 + j) * NQP + qq);
-            g0 = fmaf(val, qv.x, g0); g1 = fmaf(val, qv.y, g1); g2 = fmaf(val, qv.z, g2); g3 = fmaf(val, qv.w, g3);
+        for (int j = 0; j < 32; ++j) {
+          const float val = __uint_as_float(0x4B000000u | att_code<BITS>(row, g, j)) - off;
+          const float *qp = qts + (g * 32 + j) * NQP;
+          const float4 qv = *(const float4 *)qp;
+          g0 = fmaf(val, qv.x, g0); g1 = fmaf(val, qv.y, g1); g2 = fmaf(val, qv.z, g2); g3 = fmaf(val, qv.w, g3);
+          if (q8) {
+            const float4 qw = *(const float4 *)(qp + 4);
+            g4 = fmaf(val, qw.x, g4); g5 = fmaf(val, qw.y, g5); g6 = fmaf(val, qw.z, g6); g7 = fmaf(val, qw.w, g7);
           }
-          a0 = fmaf(delta, g0, a0); a1 = fmaf(delta, g1, a1); a2 = fmaf(delta, g2, a2); a3 = fmaf(delta, g3, a3);
         }
-        if (qq == 0) { s[0] = a0; s[1] = a1; s[2] = a2; s[3] = a3; } else { s[4] = a0; s[5] = a1; s[6] = a2; s[7] = a3; }
+        const float delta = __half2float(sc[g]);
+        const float *qh = qsum + g * kAttMaxQ;
+        g0 = fmaf(0.5f, qh[0], g0); g1 = fmaf(0.5f, qh[1], g1); g2 = fmaf(0.5f, qh[2], g2); g3 = fmaf(0.5f, qh[3], g3);
+        g4 = fmaf(0.5f, qh[4], g4); g5 = fmaf(0.5f, qh[5], g5); g6 = fmaf(0.5f, qh[6], g6); g7 = fmaf(0.5f, qh[7], g7);
+        s[0] = fmaf(delta, g0, s[0]); s[1] = fmaf(delta, g1, s[1]); s[2] = fmaf(delta, g2, s[2]); s[3] = fmaf(delta, g3, s[3]);
+        s[4] = fmaf(delta, g4, s[4]); s[5] = fmaf(delta, g5, s[5]); s[6] = fmaf(delta, g6, s[6]); s[7] = fmaf(delta, g7, s[7]);
       }
     }
     if (r_t > 0) {
       const __half *ut = jb.k.UT + (size_t)t * r_t;
-      for (int qq = 0; qq < NQP; qq += 4) {
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-        for (int k = 0; k < r_t; k += 8) {
-          const uint4 u8 = __ldg((const uint4 *)(ut + k));
-          const __half *uh = (const __half *)&u8;
+      const bool q8 = NQP == 8;
+      uint4 nxt = __ldg((const uint4 *)ut);
+      for (int k = 0; k < r_t; k += 8) {
+        const uint4 u8 = nxt;
+        if (k + 8 < r_t) nxt = __ldg((const uint4 *)(ut + k + 8));      // in flight during this block's FMAs
+        const __half *uh = (const __half *)&u8;
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float u = __half2float(uh[j]);
-            const float4 wv = *(const float4 *)(ws + (k + j) * NQP + qq);
-            a0 = fmaf(u, wv.x, a0); a1 = fmaf(u, wv.y, a1); a2 = fmaf(u, wv.z, a2); a3 = fmaf(u, wv.w, a3);
+        for (int j = 0; j < 8; ++j) {
+          const float u = __half2float(uh[j]);
+          const float *wp = ws + (k + j) * NQP;
+          const float4 wv = *(const float4 *)wp;
+          s[0] = fmaf(u, wv.x, s[0]); s[1] = fmaf(u, wv.y, s[1]); s[2] = fmaf(u, wv.z, s[2]); s[3] = fmaf(u, wv.w, s[3]);
+          if (q8) {
+            const float4 wx = *(const float4 *)(wp + 4);
+            s[4] = fmaf(u, wx.x, s[4]); s[5] = fmaf(u, wx.y, s[5]); s[6] = fmaf(u, wx.z, s[6]); s[7] = fmaf(u, wx.w, s[7]);
           }
         }
-        if (qq == 0) { s[0] += a0; s[1] += a1; s[2] += a2; s[3] += a3; } else { s[4] += a0; s[5] += a1; s[6] += a2; s[7] += a3; }
       }
     }
   }
@@ -255,7 +299,7 @@ __global__ void __launch_bounds__(kAttChunk) attend_scores_kernel(const AttendJo
 }
 
 // grid (n_chunks, m, groups), kAttChunk threads.  Dynamic shared memory: kAttChunk * (NQP floats + 4 BITS words + 4 halves)
-// + 128 * NQP floats.
+// + 4 * 128 * NQP floats.
 template <int BITS>
 __global__ void __launch_bounds__(kAttChunk) attend_values_kernel(const AttendJob *__restrict__ jobs, int NQP) {
   const AttendJob &jb = jobs[blockIdx.z];
@@ -266,7 +310,7 @@ __global__ void __launch_bounds__(kAttChunk) attend_values_kernel(const AttendJo
   float *ps = (float *)att_smem;                                        // [kAttChunk][NQP]
   uint32_t *cw = (uint32_t *)(ps + kAttChunk * NQP);                    // [kAttChunk][4 * BITS]
   __half *cs = (__half *)(cw + kAttChunk * 4 * (BITS > 0 ? BITS : 1));  // [kAttChunk][4]
-  float *part = (float *)(cs + kAttChunk * 4);                          // [128][NQP] second token half's sums
+  float *part = (float *)(cs + kAttChunk * 4);                          // [4][128][NQP] slice sums
   const int tid = threadIdx.x, t0 = chunk * kAttChunk;
   const int nt = min(kAttChunk, jb.T - t0);
   {
@@ -281,123 +325,177 @@ __global__ void __launch_bounds__(kAttChunk) attend_values_kernel(const AttendJo
     }
   }
   __syncthreads();
-  // residual: thread = (feature f, token half); sum_t p_t Delta_t (u_tf - 2^(b-1) + 1/2)
+  // residual: thread = (four neighbouring features, one of eight 32-token slices): one word, one scale and one weight
+  // load serve four codes; sum_t p_t Delta_t (u_tf - 2^(b-1) + 1/2)
   if constexpr (BITS > 0) {
-    const int f = tid & 127, half = tid >> 7, g = f >> 5, j = f & 31;
-    const int bit = j * BITS, wi = g * BITS + (bit >> 5), sh = bit & 31;
+    const int fq = tid & 31, sl = tid >> 5;
+    const int f0 = fq * 4, g = f0 >> 5, bit = (f0 & 31) * BITS, wi = g * BITS + (bit >> 5), sh = bit & 31;
+    const bool straddle = BITS == 3 && sh + 4 * BITS > 32;           // only 3-bit codes cross a word inside a quad
     constexpr uint32_t mask = (1u << BITS) - 1u;
-    constexpr float off = 0.5f - (float)(1 << (BITS - 1));
-    float acc[kAttMaxQ];
+    constexpr float off = 8388608.0f + (float)(1 << (BITS - 1));
+    float acc[4][kAttMaxQ];
 #pragma unroll
-    for (int i = 0; i < kAttMaxQ; ++i) acc[i] = 0.f;
-    const int tb = half * (kAttChunk / 2), te = min(tb + kAttChunk / 2, nt);
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int i = 0; i < kAttMaxQ; ++i) acc[c][i] = 0.f;
+    const bool q8 = NQP == 8;
+    const int tb = sl * 32, te = min(tb + 32, nt);
+#pragma unroll 4
     for (int t = tb; t < te; ++t) {
       const uint32_t *row = cw + t * (4 * BITS);
-      uint32_t u = row[wi] >> sh;
-      if (sh + BITS > 32) u |= row[wi + 1] << (32 - sh);
-      const float val = (__uint_as_float(0x4B000000u | (u & mask)) - 8388608.0f + off) * __half2float(cs[t * 4 + g]);
+      uint32_t u4 = row[wi] >> sh;
+      if (straddle) u4 |= row[wi + 1] << (32 - sh);
+      const float delta = __half2float(cs[t * 4 + g]), hd = 0.5f * delta;
       const float4 p0 = *(const float4 *)(ps + t * NQP);
-      acc[0] = fmaf(p0.x, val, acc[0]); acc[1] = fmaf(p0.y, val, acc[1]); acc[2] = fmaf(p0.z, val, acc[2]); acc[3] = fmaf(p0.w, val, acc[3]);
-      if (NQP == 8) {
-        const float4 p1 = *(const float4 *)(ps + t * NQP + 4);
-        acc[4] = fmaf(p1.x, val, acc[4]); acc[5] = fmaf(p1.y, val, acc[5]); acc[6] = fmaf(p1.z, val, acc[6]); acc[7] = fmaf(p1.w, val, acc[7]);
+      float4 p1 = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (q8) p1 = *(const float4 *)(ps + t * NQP + 4);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const float val = fmaf(__uint_as_float(0x4B000000u | ((u4 >> (c * BITS)) & mask)) - off, delta, hd);
+        acc[c][0] = fmaf(p0.x, val, acc[c][0]); acc[c][1] = fmaf(p0.y, val, acc[c][1]);
+        acc[c][2] = fmaf(p0.z, val, acc[c][2]); acc[c][3] = fmaf(p0.w, val, acc[c][3]);
+        if (q8) {
+          acc[c][4] = fmaf(p1.x, val, acc[c][4]); acc[c][5] = fmaf(p1.y, val, acc[c][5]);
+          acc[c][6] = fmaf(p1.z, val, acc[c][6]); acc[c][7] = fmaf(p1.w, val, acc[c][7]);
+        }
       }
     }
-    if (half == 1)
-      for (int i = 0; i < NQP; ++i) part[f * NQP + i] = acc[i];
-    __syncthreads();
-    if (half == 0) {
-      float *ap = jb.a + (((size_t)h * n_chunks + chunk) * 128 + f) * NQP;
-      for (int i = 0; i < NQP; ++i) ap[i] = acc[i] + part[f * NQP + i];
+    // sum over the eight slices: 7..4 -> 3..0, 3..2 -> 1..0, 1 -> 0 through part[4][128][NQP]
+#pragma unroll
+    for (int stride = 4; stride >= 1; stride >>= 1) {
+      if (sl >= stride && sl < 2 * stride) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int i = 0; i < kAttMaxQ; ++i)
+            if (i < NQP) part[((sl - stride) * 128 + f0 + c) * NQP + i] = acc[c][i];
+      }
+      __syncthreads();
+      if (sl < stride) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int i = 0; i < kAttMaxQ; ++i)
+            if (i < NQP) acc[c][i] += part[(sl * 128 + f0 + c) * NQP + i];
+      }
+      __syncthreads();
+    }
+    if (sl == 0) {
+      float *ap = jb.a + (((size_t)h * n_chunks + chunk) * 128 + f0) * NQP;
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int i = 0; i < kAttMaxQ; ++i)
+          if (i < NQP) ap[c * NQP + i] = acc[c][i];
     }
   }
-  // backbone: thread = column k of U_T; y_k = sum_t p_t U_T[t, k]
+  // backbone: thread = column k of U_T (and one of two token halves while r_t <= 128); y_k = sum_t p_t U_T[t, k]
   const int r_t = jb.v.r_t;
-  for (int k = tid; k < r_t; k += kAttChunk) {
+  if (r_t > 0) {
+    const bool split = r_t <= 128;
+    const int k = split ? (tid & 127) : tid, hv = split ? (tid >> 7) : 0;
+    const int tb = split ? hv * (kAttChunk / 2) : 0, te = min(split ? tb + kAttChunk / 2 : kAttChunk, nt);
+    const bool q8 = NQP == 8;
     float acc[kAttMaxQ];
 #pragma unroll
     for (int i = 0; i < kAttMaxQ; ++i) acc[i] = 0.f;
-    const __half *ut = jb.v.UT + (size_t)t0 * r_t + k;
-    for (int t = 0; t < nt; ++t) {
-      const float u = __half2float(ut[(size_t)t * r_t]);
-      const float4 p0 = *(const float4 *)(ps + t * NQP);
-      acc[0] = fmaf(p0.x, u, acc[0]); acc[1] = fmaf(p0.y, u, acc[1]); acc[2] = fmaf(p0.z, u, acc[2]); acc[3] = fmaf(p0.w, u, acc[3]);
-      if (NQP == 8) {
-        const float4 p1 = *(const float4 *)(ps + t * NQP + 4);
-        acc[4] = fmaf(p1.x, u, acc[4]); acc[5] = fmaf(p1.y, u, acc[5]); acc[6] = fmaf(p1.z, u, acc[6]); acc[7] = fmaf(p1.w, u, acc[7]);
+    if (k < r_t) {
+      const __half *ut = jb.v.UT + (size_t)t0 * r_t + k;
+#pragma unroll 8
+      for (int t = tb; t < te; ++t) {
+        const float u = __half2float(ut[(size_t)t * r_t]);
+        const float4 p0 = *(const float4 *)(ps + t * NQP);
+        acc[0] = fmaf(p0.x, u, acc[0]); acc[1] = fmaf(p0.y, u, acc[1]); acc[2] = fmaf(p0.z, u, acc[2]); acc[3] = fmaf(p0.w, u, acc[3]);
+        if (q8) {
+          const float4 p1 = *(const float4 *)(ps + t * NQP + 4);
+          acc[4] = fmaf(p1.x, u, acc[4]); acc[5] = fmaf(p1.y, u, acc[5]); acc[6] = fmaf(p1.z, u, acc[6]); acc[7] = fmaf(p1.w, u, acc[7]);
+        }
       }
     }
-    float *yp = jb.y + (((size_t)h * n_chunks + chunk) * r_t + k) * NQP;
-    for (int i = 0; i < NQP; ++i) yp[i] = acc[i];
+    if (split) {
+      __syncthreads();                       // part is free again (the residual's last round has been read)
+      if (hv == 1 && k < r_t) {
+#pragma unroll
+        for (int i = 0; i < kAttMaxQ; ++i)
+          if (i < NQP) part[k * NQP + i] = acc[i];
+      }
+      __syncthreads();
+      if (hv == 0 && k < r_t) {
+#pragma unroll
+        for (int i = 0; i < kAttMaxQ; ++i)
+          if (i < NQP) acc[i] += part[k * NQP + i];
+      }
+    }
+    if (hv == 0 && k < r_t) {
+      float *yp = jb.y + (((size_t)h * n_chunks + chunk) * r_t + k) * NQP;
+#pragma unroll
+      for (int i = 0; i < kAttMaxQ; ++i)
+        if (i < NQP) yp[i] = acc[i];
+    }
   }
 }
 
-// grid (m, groups), 128 threads (thread = feature).  Dynamic shared memory: 128 * v.r_f halves + (n_chunks + v.r_t) * NQP
-// floats + 128 floats + 2 * kAttMaxQ floats.
+// grid (m, groups, n_q), 128 threads (thread = feature); CTA z finishes query z.  Dynamic shared memory:
+// (n_chunks + v.r_t + 128 + 1) floats.
 __global__ void __launch_bounds__(128) attend_combine_kernel(const AttendJob *__restrict__ jobs, int n_q, int NQP, int n_chunks,
                                                              uint64_t seed) {
   const AttendJob &jb = jobs[blockIdx.y];
-  const int h = blockIdx.x, f = threadIdx.x;
+  const int h = blockIdx.x, f = threadIdx.x, i = blockIdx.z;
   if (h >= jb.m) return;
   extern __shared__ unsigned char att_smem[];
-  const int r_t = jb.v.r_t, r_f = jb.v.r_f;
-  __half *ufs = (__half *)att_smem;                                  // [r_f][128]
-  float *coef = (float *)(att_smem + (size_t)128 * r_f * sizeof(__half));   // [n_chunks][NQP]
-  float *ys = coef + n_chunks * NQP;                                 // [r_t][NQP]
-  float *buf = ys + r_t * NQP;                                       // [128]
-  float *Ls = buf + 128;                                             // [kAttMaxQ]
-  if (f < NQP) {
-    const float *ml = jb.ml + (size_t)h * n_chunks * 2 * NQP;
+  const int r_t = jb.v.r_t;
+  float *coef = (float *)att_smem;                                   // [n_chunks]
+  float *ys = coef + n_chunks;                                       // [r_t]
+  float *buf = ys + r_t;                                             // [128]
+  float *Ls = buf + 128;                                             // [1]
+  const float *ml = jb.ml + (size_t)h * n_chunks * 2 * NQP;
+  // running-maximum merge of the chunks: warp 0 finds the maximum and the rescaled sum
+  if (f < 32) {
     float M = -INFINITY;
-    for (int c = 0; c < n_chunks; ++c) M = fmaxf(M, ml[c * 2 * NQP + f]);
+    for (int c = f; c < n_chunks; c += 32) M = fmaxf(M, ml[c * 2 * NQP + i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     float L = 0.f;
-    for (int c = 0; c < n_chunks; ++c) {
-      const float cf = expf(ml[c * 2 * NQP + f] - M);
-      coef[c * NQP + f] = cf;
-      L = fmaf(cf, ml[c * 2 * NQP + NQP + f], L);
+    for (int c = f; c < n_chunks; c += 32) {
+      const float cf = expf(ml[c * 2 * NQP + i] - M);
+      coef[c] = cf;
+      L = fmaf(cf, ml[c * 2 * NQP + NQP + i], L);
     }
-    Ls[f] = L;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+    if (f == 0) Ls[0] = L;
   }
-  if (r_t > 0) att_stage_uf(jb.v, ufs, f, 128);
   __syncthreads();
-  for (int i = f; i < r_t * NQP; i += 128) {
-    const int q = i % NQP;
+  for (int k = f; k < r_t; k += 128) {
+    const float *yp = jb.y + ((size_t)h * n_chunks * r_t + k) * NQP + i;
     float acc = 0.f;
-    for (int c = 0; c < n_chunks; ++c) acc = fmaf(coef[c * NQP + q], jb.y[((size_t)h * n_chunks + c) * r_t * NQP + i], acc);
-    ys[i] = acc;
+#pragma unroll 8
+    for (int c = 0; c < n_chunks; ++c) acc = fmaf(coef[c], __ldg(yp + (size_t)c * r_t * NQP), acc);
+    ys[k] = acc;
   }
-  float ob[kAttMaxQ];
-#pragma unroll
-  for (int i = 0; i < kAttMaxQ; ++i) ob[i] = 0.f;
+  float res = 0.f;
+  if (jb.v.bits > 0) {
+    const float *ap = jb.a + ((size_t)h * n_chunks * 128 + f) * NQP + i;
+    float acc = 0.f;
+#pragma unroll 8
+    for (int c = 0; c < n_chunks; ++c) acc = fmaf(coef[c], __ldg(ap + (size_t)c * 128 * NQP), acc);
+    buf[f] = acc;
+  }
   __syncthreads();
+  if (jb.v.bits > 0) res = att_wht_smem(buf, f) * kInvSqrtD * att_sign(seed, jb.v.cell, f);
+  float ob = 0.f;
   if (r_t > 0) {
-    for (int k = 0; k < r_t; ++k) {
-      const float pk = att_p16(jb.v.G + ((size_t)h * r_t + k) * r_f, ufs, r_f, f);
-#pragma unroll
-      for (int i = 0; i < kAttMaxQ; ++i)
-        if (i < NQP) ob[i] = fmaf(ys[k * NQP + i], pk, ob[i]);
+    const __half *P = jb.vP + (size_t)h * r_t * 128 + f;
+    float o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
+    for (int k = 0; k < r_t; k += 4) {       // r_t is a multiple of 8
+      o0 = fmaf(ys[k], __half2float(P[(size_t)k * 128]), o0);
+      o1 = fmaf(ys[k + 1], __half2float(P[(size_t)(k + 1) * 128]), o1);
+      o2 = fmaf(ys[k + 2], __half2float(P[(size_t)(k + 2) * 128]), o2);
+      o3 = fmaf(ys[k + 3], __half2float(P[(size_t)(k + 3) * 128]), o3);
     }
-    const float se = ldexpf(1.f, *jb.v.e);
-#pragma unroll
-    for (int i = 0; i < kAttMaxQ; ++i) ob[i] *= se;
+    ob = ((o0 + o1) + (o2 + o3)) * ldexpf(1.f, *jb.v.e);
   }
-  const float sg = jb.v.bits > 0 ? att_sign(seed, jb.v.cell, f) : 0.f;
-  for (int i = 0; i < n_q; ++i) {
-    float res = 0.f;
-    if (jb.v.bits > 0) {
-      float acc = 0.f;
-      for (int c = 0; c < n_chunks; ++c) acc = fmaf(coef[c * NQP + i], jb.a[(((size_t)h * n_chunks + c) * 128 + f) * NQP + i], acc);
-      __syncthreads();
-      buf[f] = acc;
-      __syncthreads();
-      res = att_wht_smem(buf, f) * kInvSqrtD * sg;
-    }
-    float o = 0.f;
-#pragma unroll
-    for (int q = 0; q < kAttMaxQ; ++q)
-      if (q == i) o = ob[q];
-    jb.out[((size_t)h * n_q + i) * 128 + f] = (o + res) / Ls[i];
-  }
+  jb.out[((size_t)h * n_q + i) * 128 + f] = (ob + res) / Ls[0];
 }
 
 }  // namespace jolt

@@ -209,6 +209,11 @@ struct jolt_handle {
   uint64_t seed = 0;
   int64_t stored_bytes = 0;
   bool subspace = false;     // token factors came from the converged block iteration (exact mode, large T)
+  // jolt_attend: P_h = fp16(G_h U_F^T) of every cell, formed on the first call and kept until jolt_free
+  mutable std::mutex att_mu;
+  mutable __half *att_P = nullptr;
+  mutable std::vector<size_t> att_P_off;     // per cell, in halves
+  mutable cudaEvent_t att_ready = nullptr;
 };
 
 // ------------------------------------------------------------------ validation
@@ -1504,6 +1509,8 @@ static void launch_att_scores(dim3 grid, size_t shm, cudaStream_t s, const Atten
 }
 template <int BITS>
 static void launch_att_values(dim3 grid, size_t shm, cudaStream_t s, const AttendJob *d, int NQP) {
+  static std::atomic<bool> opted{false};      // up to 58 KB of dynamic shared memory (8-bit codes, 8 queries)
+  if (!opted.exchange(true)) cudaFuncSetAttribute(attend_values_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
   attend_values_kernel<BITS><<<grid, kAttChunk, shm, s>>>(d, NQP);
 }
 
@@ -1529,10 +1536,27 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
     kbits |= 1u << ck.bits; vbits |= 1u << cv.bits;
     if ((ck.r_t % 8) || (cv.r_t % 8) || (ck.r_f % 8) || (cv.r_f % 8)) return fail(JOLT_EUNSUPPORTED, "ranks must be multiples of 8");
   }
-  const size_t shm_prep = (size_t)128 * krf * sizeof(__half) + 160 * sizeof(float);
+  const size_t shm_p16 = (size_t)128 * std::max(krf, vrf) * sizeof(__half);
+  const size_t shm_prep = 128 * sizeof(float);
   const size_t shm_sc = (size_t)(128 + krt) * NQP * sizeof(float);
-  const size_t shm_comb = (size_t)128 * vrf * sizeof(__half) + (size_t)(n_chunks + vrt) * NQP * sizeof(float) + 136 * sizeof(float);
+  const size_t shm_comb = (size_t)(n_chunks + vrt + 136) * sizeof(float);
+  const int p_blocks = (m_max * std::max(krt, vrt) + kAttPRows - 1) / kAttPRows;
   if (shm_comb > 48 * 1024) return fail(JOLT_EUNSUPPORTED, "sequence of %d tokens: the chunk merge needs %zu bytes of shared memory", T, shm_comb);
+  // the projected cores do not depend on the queries: formed by the first call on this handle, kept with it
+  bool first_call = false;
+  {
+    std::lock_guard<std::mutex> lk(H->att_mu);
+    if (!H->att_P) {
+      size_t halves = 0;
+      H->att_P_off.assign(2 * ng, 0);
+      for (int c = 0; c < 2 * ng; ++c) { H->att_P_off[c] = halves; halves += ((size_t)H->cells[c].c.m * std::max(H->cells[c].c.r_t, 1) * kD + 127) & ~(size_t)127; }
+      void *pbuf = nullptr;
+      if (cudaMalloc(&pbuf, halves * sizeof(__half)) != cudaSuccess) { cudaGetLastError(); return fail(JOLT_ENOMEM, "projected cores: %zu bytes", halves * sizeof(__half)); }
+      H->att_P = (__half *)pbuf;
+      if (cudaEventCreateWithFlags(&H->att_ready, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); cudaFree(pbuf); H->att_P = nullptr; return fail(JOLT_ECUDA, "event"); }
+      first_call = true;
+    }
+  }
   std::vector<AttendJob> jobs(ng);
   void *ws_base = nullptr;
   int rc;
@@ -1550,6 +1574,8 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
       j.m = sk.c.m; j.T = T;
       const size_t row0 = (size_t)H->group_start[g] * nh * n_q * kD;
       j.q = (const float *)dQ + row0; j.out = (float *)dOut + row0;
+      j.kP = H->att_P + H->att_P_off[2 * g];
+      j.vP = H->att_P + H->att_P_off[2 * g + 1];
       j.w = b.take<float>((size_t)j.m * std::max(j.k.r_t, 1) * NQP);
       j.qt = b.take<float>((size_t)j.m * kD * NQP);
       j.p = b.take<float>((size_t)j.m * T * NQP);
@@ -1563,9 +1589,19 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
   const size_t off = P.push(jobs);
   const uint64_t seed = H->seed;
   const float fscale = (float)scale;
+  cudaEvent_t att_ready = H->att_ready;
   P.add(ST_ATT, [=](char *dev_t, cudaStream_t s) {
     const AttendJob *d = (const AttendJob *)(dev_t + off);
-    attend_prep_kernel<<<dim3(m_max, ng), 128, shm_prep, s>>>(d, n_q, NQP, fscale, seed);
+    if (first_call) {
+      if (p_blocks > 0) {
+        attend_p16_kernel<<<dim3(p_blocks, 2 * ng), 128, shm_p16, s>>>(d);
+        LAUNCHED();
+      }
+      cudaEventRecord(att_ready, s);
+    } else {
+      cudaStreamWaitEvent(s, att_ready, 0);      // a call on another stream must see the finished cores
+    }
+    attend_prep_kernel<<<dim3(m_max, ng, NQP), 128, shm_prep, s>>>(d, n_q, NQP, fscale, seed);
     LAUNCHED();
     const dim3 grid(n_chunks, m_max, ng);
     for (int b = 0; b <= 8; ++b) {
@@ -1582,7 +1618,7 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
     }
     for (int b = 0; b <= 8; ++b) {
       if (!((vbits >> b) & 1)) continue;
-      const size_t shm = (size_t)kAttChunk * (NQP * sizeof(float) + 16 * std::max(b, 1) + 8) + (size_t)128 * NQP * sizeof(float);
+      const size_t shm = (size_t)kAttChunk * (NQP * sizeof(float) + 16 * std::max(b, 1) + 8) + (size_t)4 * 128 * NQP * sizeof(float);
       switch (b) {
         case 0: launch_att_values<0>(grid, shm, s, d, NQP); break;
         case 1: launch_att_values<1>(grid, shm, s, d, NQP); break;
@@ -1593,7 +1629,7 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
       }
       LAUNCHED();
     }
-    attend_combine_kernel<<<dim3(m_max, ng), 128, shm_comb, s>>>(d, n_q, NQP, n_chunks, seed);
+    attend_combine_kernel<<<dim3(m_max, ng, n_q), 128, shm_comb, s>>>(d, n_q, NQP, n_chunks, seed);
     LAUNCHED();
   });
   void *d_tab = nullptr;
@@ -1609,6 +1645,8 @@ extern "C" int jolt_free(jolt_handle *H) {
     int cur = 0;
     cudaGetDevice(&cur);
     if (cur != H->device) cudaSetDevice(H->device);
+    if (H->att_P) { cudaFree(H->att_P); H->att_P = nullptr; }       // cudaFree waits for the kernels that read it
+    if (H->att_ready) { cudaEventDestroy(H->att_ready); H->att_ready = nullptr; }
     cudaFreeAsync(H->blob, 0);
     if (cur != H->device) cudaSetDevice(cur);
   }

@@ -43,8 +43,15 @@ def test_first_group_of_config(B, name):
     assert torch.equal(Vr, Vo)
     Krnp = Kr.cpu().numpy()
     del Kr, Vr
+    # attention on the compressed cache (4 queries per KV head), against attention over the library's fp32 decode here
+    # and against the oracle on the oracle's own cells below
+    gq = torch.Generator().manual_seed(3)
+    Q = torch.randn(K.shape[0], K.shape[1], 4, 128, generator=gq)
+    att = B.jolt_attend(h, Q.cuda())
+    torch.cuda.synchronize()
     Knp, Vnp = K.cpu().numpy(), V.cpu().numpy()
     Konp, Vonp = Ko.cpu().numpy(), Vo.cpu().numpy()
+    ocells, gates = [], []
     for c in range(2):
         rt, rf, b = plans[c]
         X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
@@ -69,5 +76,11 @@ def test_first_group_of_config(B, name):
             if (sig[rt - 1] - sig[rt]) / sig[0] > 1e-2:
                 assert projector_distance(UT, o.ideal["U_T"]) <= 1e-3, (name, c)
             assert np.abs(h.component(c, 6)[:rt] - sig[:rt]).max() <= 1e-4 * sig[0], (name, c)
-        del X, Xo, Xg, o
+        ocells.append(o)
+        gates.append(recon_gate(eo))
+        del X, Xo, Xg
+    ref = O.attend_cells(ocells[0], ocells[1], Q.reshape(-1, 4, 128).numpy(), 1.0 / 128 ** 0.5)
+    got = att.cpu().numpy().astype(np.float64).reshape(-1, 4, 128)
+    rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+    assert rel <= 3 * max(gates), (name, "attend", rel, gates)
     h.free()
