@@ -11,12 +11,15 @@
 // so a call streams U_T and the packed codes once each (the compressed bytes) instead of the fp16 cache, and the
 // Hadamard rotation is applied to one query / one output row per head instead of every token.
 //
-// Five kernels, all CUDA-core (the work is a stream of 1..8-bit codes against a handful of query vectors):
+// Seven kernels, all CUDA-core (the work is a stream of 1..8-bit codes against a handful of query vectors):
 //   attend_p16_kernel      P_h = fp16(G_h U_F^T) of every head of both cells (what the decoder's set-up also forms)
 //   attend_prep_kernel     per (group, head): rotated scaled queries and w = scale 2^e P_h q
-//   attend_scores_kernel   per (group, head, 256-token chunk): scores, chunk maximum, p = exp(s - max), chunk sum
-//   attend_values_kernel   per (group, head, chunk): p^T U_T and sum_t p_t r^'_t (codes staged in shared memory and
-//                          read feature-wise, so the token reduction stays inside a thread)
+//   attend_bscore_kernel   backbone scores U_T w of all heads of a cell as one dense product (U_T is shared by the heads)
+//   attend_scores_kernel   per (group, head, 256-token chunk): residual scores added, chunk maximum, p = exp(s - max),
+//                          chunk sum
+//   attend_values_kernel   per (group, head, chunk): sum_t p_t r^'_t (codes staged in shared memory and read
+//                          feature-wise, so the token reduction stays inside a thread)
+//   attend_bvalue_kernel   p^T U_T per chunk for all heads of a cell as one dense product
 //   attend_combine_kernel  per (group, head): merges the chunks (running-maximum rescaling), applies P_h of the
 //                          value cell and the inverse rotation, divides by the softmax denominator
 // Keys compressed before a rotary embedding cannot use the first identity (the rotation differs per token).
@@ -176,13 +179,11 @@ __global__ void __launch_bounds__(kAttChunk, 3) attend_scores_kernel(const Atten
   if (h >= jb.m || chunk * kAttChunk >= jb.T) return;
   extern __shared__ unsigned char att_smem[];
   float *qts = (float *)att_smem;                   // [128][NQP]
-  float *ws = qts + 128 * NQP;                      // [r_t][NQP]
   __shared__ float red[2][kAttChunk / 32][kAttMaxQ];
   __shared__ float qsum[4 * kAttMaxQ];              // per 32-feature group: sum of the rotated query's entries
   const int tid = threadIdx.x, r_t = jb.k.r_t;
   if (BITS > 0)
     for (int i = tid; i < 128 * NQP; i += kAttChunk) qts[i] = jb.qt[(size_t)h * 128 * NQP + i];
-  for (int i = tid; i < r_t * NQP; i += kAttChunk) ws[i] = jb.w[(size_t)h * r_t * NQP + i];
   __syncthreads();
   if (BITS > 0 && tid < 4 * kAttMaxQ) {
     const int g = tid / kAttMaxQ, i = tid % kAttMaxQ;
@@ -232,24 +233,13 @@ __global__ void __launch_bounds__(kAttChunk, 3) attend_scores_kernel(const Atten
       }
     }
     if (r_t > 0) {
-      const __half *ut = jb.k.UT + (size_t)t * r_t;
-      const bool q8 = NQP == 8;
-      uint4 nxt = __ldg((const uint4 *)ut);
-      for (int k = 0; k < r_t; k += 8) {
-        const uint4 u8 = nxt;
-        if (k + 8 < r_t) nxt = __ldg((const uint4 *)(ut + k + 8));      // in flight during this block's FMAs
-        const __half *uh = (const __half *)&u8;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float u = __half2float(uh[j]);
-          const float *wp = ws + (k + j) * NQP;
-          const float4 wv = *(const float4 *)wp;
-          s[0] = fmaf(u, wv.x, s[0]); s[1] = fmaf(u, wv.y, s[1]); s[2] = fmaf(u, wv.z, s[2]); s[3] = fmaf(u, wv.w, s[3]);
-          if (q8) {
-            const float4 wx = *(const float4 *)(wp + 4);
-            s[4] = fmaf(u, wx.x, s[4]); s[5] = fmaf(u, wx.y, s[5]); s[6] = fmaf(u, wx.z, s[6]); s[7] = fmaf(u, wx.w, s[7]);
-          }
-        }
+      // backbone scores of this token: written to the weight buffer by attend_bscore_kernel, replaced by the weights below
+      const float *sb = jb.p + ((size_t)h * jb.T + t) * NQP;
+      const float4 b0 = *(const float4 *)sb;
+      s[0] += b0.x; s[1] += b0.y; s[2] += b0.z; s[3] += b0.w;
+      if (NQP == 8) {
+        const float4 b1 = *(const float4 *)(sb + 4);
+        s[4] += b1.x; s[5] += b1.y; s[6] += b1.z; s[7] += b1.w;
       }
     }
   }
@@ -389,48 +379,129 @@ __global__ void __launch_bounds__(kAttChunk) attend_values_kernel(const AttendJo
           if (i < NQP) ap[c * NQP + i] = acc[c][i];
     }
   }
-  // backbone: thread = column k of U_T (and one of two token halves while r_t <= 128); y_k = sum_t p_t U_T[t, k]
-  const int r_t = jb.v.r_t;
-  if (r_t > 0) {
-    const bool split = r_t <= 128;
-    const int k = split ? (tid & 127) : tid, hv = split ? (tid >> 7) : 0;
-    const int tb = split ? hv * (kAttChunk / 2) : 0, te = min(split ? tb + kAttChunk / 2 : kAttChunk, nt);
-    const bool q8 = NQP == 8;
-    float acc[kAttMaxQ];
+}
+
+// The backbone terms are shared by all heads of a cell (one U_T per cell), so they are two small dense products over the
+// whole cell instead of a loop per head:  with n = (head, query),
+//   attend_bscore_kernel   S_b[t][n] = sum_k U_T[t][k] w[n][k]            written to the weight buffer p[h][t][i]
+//   attend_bvalue_kernel   y[chunk][n][k] = sum_{t in chunk} p[n][t] U_T[t][k]
+// Register-tiled CUDA-core products (0.13 GFLOP per cell each): U_T is read once per 128 columns n instead of once per head.
+
+// grid (ceil(T / 64), ceil(m NQP / 128), groups), 256 threads: 64 tokens x 128 columns, 4 x 8 per thread
+__global__ void __launch_bounds__(256) attend_bscore_kernel(const AttendJob *__restrict__ jobs, int NQP) {
+  const AttendJob &jb = jobs[blockIdx.z];
+  const int r_t = jb.k.r_t, N = jb.m * NQP, n0 = blockIdx.y * 128, t0 = blockIdx.x * 64;
+  if (r_t == 0 || n0 >= N || t0 >= jb.T) return;
+  __shared__ __align__(16) float As[16][64 + 4];
+  __shared__ __align__(16) float Bs[16][128];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  float acc[4][8];
 #pragma unroll
-    for (int i = 0; i < kAttMaxQ; ++i) acc[i] = 0.f;
-    if (k < r_t) {
-      const __half *ut = jb.v.UT + (size_t)t0 * r_t + k;
-#pragma unroll 8
-      for (int t = tb; t < te; ++t) {
-        const float u = __half2float(ut[(size_t)t * r_t]);
-        const float4 p0 = *(const float4 *)(ps + t * NQP);
-        acc[0] = fmaf(p0.x, u, acc[0]); acc[1] = fmaf(p0.y, u, acc[1]); acc[2] = fmaf(p0.z, u, acc[2]); acc[3] = fmaf(p0.w, u, acc[3]);
-        if (q8) {
-          const float4 p1 = *(const float4 *)(ps + t * NQP + 4);
-          acc[4] = fmaf(p1.x, u, acc[4]); acc[5] = fmaf(p1.y, u, acc[5]); acc[6] = fmaf(p1.z, u, acc[6]); acc[7] = fmaf(p1.w, u, acc[7]);
-        }
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 8; ++b) acc[a][b] = 0.f;
+  const int at = tid >> 2, akq = (tid & 3) * 4;          // A loader: token, first of four k
+  const int bk = tid >> 4, bn = (tid & 15) * 8;          // B loader: k, first of eight n
+  for (int k0 = 0; k0 < r_t; k0 += 16) {
+    {
+      uint2 u = make_uint2(0u, 0u);
+      if (t0 + at < jb.T && k0 + akq < r_t) u = __ldg((const uint2 *)(jb.k.UT + (size_t)(t0 + at) * r_t + k0 + akq));
+      const __half *uh = (const __half *)&u;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) As[akq + j][at] = __half2float(uh[j]);
+#pragma unroll
+      for (int q4 = 0; q4 < 2; ++q4) {
+        const int n = n0 + bn + q4 * 4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (n < N && k0 + bk < r_t) v = *(const float4 *)(jb.w + ((size_t)(n / NQP) * r_t + k0 + bk) * NQP + n % NQP);
+        *(float4 *)&Bs[bk][bn + q4 * 4] = v;
       }
     }
-    if (split) {
-      __syncthreads();                       // part is free again (the residual's last round has been read)
-      if (hv == 1 && k < r_t) {
+    __syncthreads();
 #pragma unroll
-        for (int i = 0; i < kAttMaxQ; ++i)
-          if (i < NQP) part[k * NQP + i] = acc[i];
-      }
-      __syncthreads();
-      if (hv == 0 && k < r_t) {
+    for (int kk = 0; kk < 16; ++kk) {
+      const float4 a4 = *(const float4 *)&As[kk][ty * 4];
+      const float4 b0 = *(const float4 *)&Bs[kk][tx * 8], b1 = *(const float4 *)&Bs[kk][tx * 8 + 4];
+      const float a[4] = {a4.x, a4.y, a4.z, a4.w};
+      const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
-        for (int i = 0; i < kAttMaxQ; ++i)
-          if (i < NQP) acc[i] += part[k * NQP + i];
-      }
+      for (int ia = 0; ia < 4; ++ia)
+#pragma unroll
+        for (int ib = 0; ib < 8; ++ib) acc[ia][ib] = fmaf(a[ia], b[ib], acc[ia][ib]);
     }
-    if (hv == 0 && k < r_t) {
-      float *yp = jb.y + (((size_t)h * n_chunks + chunk) * r_t + k) * NQP;
+    __syncthreads();
+  }
 #pragma unroll
-      for (int i = 0; i < kAttMaxQ; ++i)
-        if (i < NQP) yp[i] = acc[i];
+  for (int ia = 0; ia < 4; ++ia) {
+    const int t = t0 + ty * 4 + ia;
+    if (t >= jb.T) continue;
+#pragma unroll
+    for (int q4 = 0; q4 < 2; ++q4) {
+      const int n = n0 + tx * 8 + q4 * 4;
+      if (n < N)
+        *(float4 *)(jb.p + ((size_t)(n / NQP) * jb.T + t) * NQP + n % NQP) =
+            make_float4(acc[ia][q4 * 4], acc[ia][q4 * 4 + 1], acc[ia][q4 * 4 + 2], acc[ia][q4 * 4 + 3]);
+    }
+  }
+}
+
+// grid (n_chunks * KT, ceil(m NQP / 128), groups) with KT = ceil(max r_t / 64), 256 threads: 128 columns n x 64 columns k of
+// one 256-token chunk, 8 x 4 per thread
+__global__ void __launch_bounds__(256) attend_bvalue_kernel(const AttendJob *__restrict__ jobs, int NQP, int n_chunks, int KT) {
+  const AttendJob &jb = jobs[blockIdx.z];
+  const int r_t = jb.v.r_t, N = jb.m * NQP, n0 = blockIdx.y * 128;
+  const int chunk = blockIdx.x / KT, kb = (blockIdx.x % KT) * 64, t0 = chunk * kAttChunk;
+  if (r_t == 0 || n0 >= N || kb >= r_t || t0 >= jb.T) return;
+  __shared__ __align__(16) float Ps[16][128];
+  __shared__ __align__(16) float Us[16][64];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  float acc[8][4];
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+  const int lt = tid >> 4, ln = (tid & 15) * 8, lk = (tid & 15) * 4;      // loaders: token, first of eight n / four k
+  const int nt = min(kAttChunk, jb.T - t0);
+  for (int tt0 = 0; tt0 < nt; tt0 += 16) {
+    const int t = t0 + tt0 + lt;
+    const bool tok = tt0 + lt < nt;
+#pragma unroll
+    for (int q4 = 0; q4 < 2; ++q4) {
+      const int n = n0 + ln + q4 * 4;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (tok && n < N) v = *(const float4 *)(jb.p + ((size_t)(n / NQP) * jb.T + t) * NQP + n % NQP);
+      *(float4 *)&Ps[lt][ln + q4 * 4] = v;
+    }
+    {
+      uint2 u = make_uint2(0u, 0u);
+      if (tok && kb + lk < r_t) u = __ldg((const uint2 *)(jb.v.UT + (size_t)t * r_t + kb + lk));
+      const __half *uh = (const __half *)&u;
+      *(float4 *)&Us[lt][lk] = make_float4(__half2float(uh[0]), __half2float(uh[1]), __half2float(uh[2]), __half2float(uh[3]));
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+      const float4 a0 = *(const float4 *)&Ps[kk][ty * 8], a1 = *(const float4 *)&Ps[kk][ty * 8 + 4];
+      const float4 b4 = *(const float4 *)&Us[kk][tx * 4];
+      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int ia = 0; ia < 8; ++ia)
+#pragma unroll
+        for (int ib = 0; ib < 4; ++ib) acc[ia][ib] = fmaf(a[ia], b[ib], acc[ia][ib]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int ib = 0; ib < 4; ++ib) {
+    const int k = kb + tx * 4 + ib;
+    if (k >= r_t) continue;
+#pragma unroll
+    for (int q4 = 0; q4 < 2; ++q4) {
+      const int n = n0 + ty * 8 + q4 * 4;
+      if (n < N)
+        *(float4 *)(jb.y + (((size_t)(n / NQP) * n_chunks + chunk) * r_t + k) * NQP + n % NQP) =
+            make_float4(acc[q4 * 4][ib], acc[q4 * 4 + 1][ib], acc[q4 * 4 + 2][ib], acc[q4 * 4 + 3][ib]);
     }
   }
 }

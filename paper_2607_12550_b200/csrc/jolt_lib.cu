@@ -1538,7 +1538,7 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
   }
   const size_t shm_p16 = (size_t)128 * std::max(krf, vrf) * sizeof(__half);
   const size_t shm_prep = 128 * sizeof(float);
-  const size_t shm_sc = (size_t)(128 + krt) * NQP * sizeof(float);
+  const size_t shm_sc = (size_t)128 * NQP * sizeof(float);
   const size_t shm_comb = (size_t)(n_chunks + vrt + 136) * sizeof(float);
   const int p_blocks = (m_max * std::max(krt, vrt) + kAttPRows - 1) / kAttPRows;
   if (shm_comb > 48 * 1024) return fail(JOLT_EUNSUPPORTED, "sequence of %d tokens: the chunk merge needs %zu bytes of shared memory", T, shm_comb);
@@ -1604,6 +1604,11 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
     attend_prep_kernel<<<dim3(m_max, ng, NQP), 128, shm_prep, s>>>(d, n_q, NQP, fscale, seed);
     LAUNCHED();
     const dim3 grid(n_chunks, m_max, ng);
+    const int n_tiles = (m_max * NQP + 127) / 128;
+    if (krt > 0) {
+      attend_bscore_kernel<<<dim3((T + 63) / 64, n_tiles, ng), 256, 0, s>>>(d, NQP);
+      LAUNCHED();
+    }
     for (int b = 0; b <= 8; ++b) {
       if (!((kbits >> b) & 1)) continue;
       switch (b) {
@@ -1627,6 +1632,11 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
         case 4: launch_att_values<4>(grid, shm, s, d, NQP); break;
         default: launch_att_values<8>(grid, shm, s, d, NQP); break;
       }
+      LAUNCHED();
+    }
+    if (vrt > 0) {
+      const int KT = (vrt + 63) / 64;
+      attend_bvalue_kernel<<<dim3(n_chunks * KT, n_tiles, ng), 256, 0, s>>>(d, NQP, n_chunks, KT);
       LAUNCHED();
     }
     attend_combine_kernel<<<dim3(m_max, ng, n_q), 128, shm_comb, s>>>(d, n_q, NQP, n_chunks, seed);
