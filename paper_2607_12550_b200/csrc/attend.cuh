@@ -11,7 +11,8 @@
 // so a call streams U_T and the packed codes once each (the compressed bytes) instead of the fp16 cache, and the
 // Hadamard rotation is applied to one query / one output row per head instead of every token.
 //
-// Seven kernels, all CUDA-core (the work is a stream of 1..8-bit codes against a handful of query vectors):
+// Seven kernels; the code streams are CUDA-core work (1..8-bit codes against a handful of query vectors), the two
+// backbone products warp-level tensor-core MMAs:
 //   attend_p16_kernel      P_h = fp16(G_h U_F^T) of every head of both cells (what the decoder's set-up also forms)
 //   attend_prep_kernel     per (group, head): rotated scaled queries and w = scale 2^e P_h q
 //   attend_bscore_kernel   backbone scores U_T w of all heads of a cell as one dense product (U_T is shared by the heads)
@@ -385,125 +386,169 @@ __global__ void __launch_bounds__(kAttChunk) attend_values_kernel(const AttendJo
 // whole cell instead of a loop per head:  with n = (head, query),
 //   attend_bscore_kernel   S_b[t][n] = sum_k U_T[t][k] w[n][k]            written to the weight buffer p[h][t][i]
 //   attend_bvalue_kernel   y[chunk][n][k] = sum_{t in chunk} p[n][t] U_T[t][k]
-// Register-tiled CUDA-core products (0.13 GFLOP per cell each): U_T is read once per 128 columns n instead of once per head.
+// Both run on the tensor cores as warp-level m16n8k8 TF32 MMAs with fp32 accumulation: an fp16 entry of U_T is exact in
+// TF32, and the fp32 operand (w, p) enters as hi + lo (hi = the top 19 bits, lo = the remainder), which keeps about 21
+// bits of it.  0.13 GFLOP per cell each: too small to set up TMEM-resident tcgen05 tiles for.
+__device__ __forceinline__ void att_mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t att_tf32_hi(float x) { return __float_as_uint(x) & 0xFFFFE000u; }
+__device__ __forceinline__ uint32_t att_tf32_lo(float x) { return __float_as_uint(x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u)); }
+// half number c (0..7) of eight packed halves, as the bits of the equal float
+__device__ __forceinline__ uint32_t att_half_of(const uint4 &u, int c) {
+  const uint32_t w = (c & 4) ? ((c & 2) ? u.w : u.z) : ((c & 2) ? u.y : u.x);
+  return __float_as_uint(__half2float(__ushort_as_half((unsigned short)((c & 1) ? (w >> 16) : (w & 0xFFFFu)))));
+}
 
-// grid (ceil(T / 64), ceil(m NQP / 128), groups), 256 threads: 64 tokens x 128 columns, 4 x 8 per thread
-__global__ void __launch_bounds__(256) attend_bscore_kernel(const AttendJob *__restrict__ jobs, int NQP) {
+constexpr int kAttBPitch = 136;     // floats per staged operand row: 8 c + g addresses all 32 banks
+
+// grid (ceil(T / 64), ceil(m NQP / 128), groups), 128 threads: a warp owns 16 tokens x 128 columns n
+__global__ void __launch_bounds__(128) attend_bscore_kernel(const AttendJob *__restrict__ jobs, int NQP) {
   const AttendJob &jb = jobs[blockIdx.z];
   const int r_t = jb.k.r_t, N = jb.m * NQP, n0 = blockIdx.y * 128, t0 = blockIdx.x * 64;
   if (r_t == 0 || n0 >= N || t0 >= jb.T) return;
-  __shared__ __align__(16) float As[16][64 + 4];
-  __shared__ __align__(16) float Bs[16][128];
-  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  float acc[4][8];
+  __shared__ __align__(16) uint32_t Bh[32][kAttBPitch], Bl[32][kAttBPitch];       // w chunk, hi and lo, [k][n]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
+  float acc[16][4];
 #pragma unroll
-  for (int a = 0; a < 4; ++a)
+  for (int nt = 0; nt < 16; ++nt)
 #pragma unroll
-    for (int b = 0; b < 8; ++b) acc[a][b] = 0.f;
-  const int at = tid >> 2, akq = (tid & 3) * 4;          // A loader: token, first of four k
-  const int bk = tid >> 4, bn = (tid & 15) * 8;          // B loader: k, first of eight n
-  for (int k0 = 0; k0 < r_t; k0 += 16) {
-    {
-      uint2 u = make_uint2(0u, 0u);
-      if (t0 + at < jb.T && k0 + akq < r_t) u = __ldg((const uint2 *)(jb.k.UT + (size_t)(t0 + at) * r_t + k0 + akq));
-      const __half *uh = (const __half *)&u;
+    for (int j = 0; j < 4; ++j) acc[nt][j] = 0.f;
+  const int ta = min(t0 + warp * 16 + g, jb.T - 1), tb = min(t0 + warp * 16 + g + 8, jb.T - 1);   // rows past the end repeat the last
+  const __half *rowa = jb.k.UT + (size_t)ta * r_t, *rowb = jb.k.UT + (size_t)tb * r_t;
+  for (int k0 = 0; k0 < r_t; k0 += 32) {
+    __syncthreads();
+    for (int idx = tid; idx < 32 * 32; idx += 128) {
+      const int kk = idx >> 5, q4 = idx & 31, n = n0 + q4 * 4;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (n < N && k0 + kk < r_t) v = *(const float4 *)(jb.w + ((size_t)(n / NQP) * r_t + k0 + kk) * NQP + n % NQP);
+      *(uint4 *)&Bh[kk][q4 * 4] = make_uint4(att_tf32_hi(v.x), att_tf32_hi(v.y), att_tf32_hi(v.z), att_tf32_hi(v.w));
+      *(uint4 *)&Bl[kk][q4 * 4] = make_uint4(att_tf32_lo(v.x), att_tf32_lo(v.y), att_tf32_lo(v.z), att_tf32_lo(v.w));
+    }
+    __syncthreads();
 #pragma unroll
-      for (int j = 0; j < 4; ++j) As[akq + j][at] = __half2float(uh[j]);
+    for (int k8 = 0; k8 < 4; ++k8) {
+      if (k0 + k8 * 8 >= r_t) break;
+      const uint4 ua = __ldg((const uint4 *)(rowa + k0 + k8 * 8)), ub = __ldg((const uint4 *)(rowb + k0 + k8 * 8));
+      const uint32_t a[4] = {att_half_of(ua, c), att_half_of(ub, c), att_half_of(ua, c + 4), att_half_of(ub, c + 4)};
 #pragma unroll
-      for (int q4 = 0; q4 < 2; ++q4) {
-        const int n = n0 + bn + q4 * 4;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (n < N && k0 + bk < r_t) v = *(const float4 *)(jb.w + ((size_t)(n / NQP) * r_t + k0 + bk) * NQP + n % NQP);
-        *(float4 *)&Bs[bk][bn + q4 * 4] = v;
+      for (int nt = 0; nt < 16; ++nt) {
+        att_mma_tf32(acc[nt], a, Bh[k8 * 8 + c][nt * 8 + g], Bh[k8 * 8 + c + 4][nt * 8 + g]);
+        att_mma_tf32(acc[nt], a, Bl[k8 * 8 + c][nt * 8 + g], Bl[k8 * 8 + c + 4][nt * 8 + g]);
       }
     }
-    __syncthreads();
-#pragma unroll
-    for (int kk = 0; kk < 16; ++kk) {
-      const float4 a4 = *(const float4 *)&As[kk][ty * 4];
-      const float4 b0 = *(const float4 *)&Bs[kk][tx * 8], b1 = *(const float4 *)&Bs[kk][tx * 8 + 4];
-      const float a[4] = {a4.x, a4.y, a4.z, a4.w};
-      const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-      for (int ia = 0; ia < 4; ++ia)
-#pragma unroll
-        for (int ib = 0; ib < 8; ++ib) acc[ia][ib] = fmaf(a[ia], b[ib], acc[ia][ib]);
-    }
-    __syncthreads();
   }
+  const int t_lo = t0 + warp * 16 + g, t_hi = t_lo + 8;
 #pragma unroll
-  for (int ia = 0; ia < 4; ++ia) {
-    const int t = t0 + ty * 4 + ia;
-    if (t >= jb.T) continue;
-#pragma unroll
-    for (int q4 = 0; q4 < 2; ++q4) {
-      const int n = n0 + tx * 8 + q4 * 4;
-      if (n < N)
-        *(float4 *)(jb.p + ((size_t)(n / NQP) * jb.T + t) * NQP + n % NQP) =
-            make_float4(acc[ia][q4 * 4], acc[ia][q4 * 4 + 1], acc[ia][q4 * 4 + 2], acc[ia][q4 * 4 + 3]);
-    }
+  for (int nt = 0; nt < 16; ++nt) {
+    const int n = n0 + nt * 8 + 2 * c;
+    if (n >= N) continue;
+    const size_t col = (size_t)(n / NQP) * jb.T * NQP + n % NQP;
+    if (t_lo < jb.T) *(float2 *)(jb.p + col + (size_t)t_lo * NQP) = make_float2(acc[nt][0], acc[nt][1]);
+    if (t_hi < jb.T) *(float2 *)(jb.p + col + (size_t)t_hi * NQP) = make_float2(acc[nt][2], acc[nt][3]);
   }
 }
 
-// grid (n_chunks * KT, ceil(m NQP / 128), groups) with KT = ceil(max r_t / 64), 256 threads: 128 columns n x 64 columns k of
-// one 256-token chunk, 8 x 4 per thread
-__global__ void __launch_bounds__(256) attend_bvalue_kernel(const AttendJob *__restrict__ jobs, int NQP, int n_chunks, int KT) {
+__device__ __forceinline__ void att_mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// grid (n_chunks * KT, ceil(m NQP / 128), groups) with KT = ceil(max r_t / 64), 128 threads: 128 columns n x 64 columns k
+// of one 256-token chunk; a warp owns 32 n x 64 k.  m16n8k16 fp16 MMAs: U_T is fp16 as stored, a weight p in [0, 1]
+// enters as hi + lo fp16 (22 bits; the lo part of a tiny weight may be subnormal, an absolute error below 2^-25).
+__global__ void __launch_bounds__(128) attend_bvalue_kernel(const AttendJob *__restrict__ jobs, int NQP, int n_chunks, int KT) {
   const AttendJob &jb = jobs[blockIdx.z];
   const int r_t = jb.v.r_t, N = jb.m * NQP, n0 = blockIdx.y * 128;
   const int chunk = blockIdx.x / KT, kb = (blockIdx.x % KT) * 64, t0 = chunk * kAttChunk;
   if (r_t == 0 || n0 >= N || kb >= r_t || t0 >= jb.T) return;
-  __shared__ __align__(16) float Ps[16][128];
-  __shared__ __align__(16) float Us[16][64];
-  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  float acc[8][4];
+  // token pairs (2 tp, 2 tp + 1) packed as half2, low half = the even token
+  __shared__ __align__(16) uint32_t Ph[16][kAttBPitch], Pl[16][kAttBPitch];     // weights hi / lo, [tp][n]
+  __shared__ __align__(16) uint32_t Us[16][64 + 8];                             // U_T, [tp][k]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
+  float acc[2][8][4];
 #pragma unroll
-  for (int a = 0; a < 8; ++a)
+  for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
-  const int lt = tid >> 4, ln = (tid & 15) * 8, lk = (tid & 15) * 4;      // loaders: token, first of eight n / four k
-  const int nt = min(kAttChunk, jb.T - t0);
-  for (int tt0 = 0; tt0 < nt; tt0 += 16) {
-    const int t = t0 + tt0 + lt;
-    const bool tok = tt0 + lt < nt;
+    for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
-    for (int q4 = 0; q4 < 2; ++q4) {
-      const int n = n0 + ln + q4 * 4;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (tok && n < N) v = *(const float4 *)(jb.p + ((size_t)(n / NQP) * jb.T + t) * NQP + n % NQP);
-      *(float4 *)&Ps[lt][ln + q4 * 4] = v;
+      for (int j = 0; j < 4; ++j) acc[mt][nt][j] = 0.f;
+  const int nt_tok = min(kAttChunk, jb.T - t0);          // a multiple of 128
+  for (int tt0 = 0; tt0 < nt_tok; tt0 += 32) {
+    __syncthreads();
+    for (int idx = tid; idx < 16 * 32; idx += 128) {
+      const int tp = idx >> 5, q4 = idx & 31, n = n0 + q4 * 4;
+      float4 v0 = make_float4(0.f, 0.f, 0.f, 0.f), v1 = v0;
+      if (n < N) {
+        const float *src = jb.p + ((size_t)(n / NQP) * jb.T + t0 + tt0 + 2 * tp) * NQP + n % NQP;
+        v0 = *(const float4 *)src;
+        v1 = *(const float4 *)(src + NQP);
+      }
+      const float x0[4] = {v0.x, v0.y, v0.z, v0.w}, x1[4] = {v1.x, v1.y, v1.z, v1.w};
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const __half2 h2 = __floats2half2_rn(x0[j], x1[j]);
+        const float2 hf = __half22float2(h2);
+        const __half2 l2 = __floats2half2_rn(x0[j] - hf.x, x1[j] - hf.y);
+        hi[j] = *(const uint32_t *)&h2; lo[j] = *(const uint32_t *)&l2;
+      }
+      *(uint4 *)&Ph[tp][q4 * 4] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *(uint4 *)&Pl[tp][q4 * 4] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     }
-    {
-      uint2 u = make_uint2(0u, 0u);
-      if (tok && kb + lk < r_t) u = __ldg((const uint2 *)(jb.v.UT + (size_t)t * r_t + kb + lk));
-      const __half *uh = (const __half *)&u;
-      *(float4 *)&Us[lt][lk] = make_float4(__half2float(uh[0]), __half2float(uh[1]), __half2float(uh[2]), __half2float(uh[3]));
+    for (int idx = tid; idx < 16 * 8; idx += 128) {
+      const int tp = idx >> 3, k8 = (idx & 7) * 8;
+      uint4 u0 = make_uint4(0u, 0u, 0u, 0u), u1 = u0;
+      if (kb + k8 < r_t) {
+        const __half *src = jb.v.UT + (size_t)(t0 + tt0 + 2 * tp) * r_t + kb + k8;
+        u0 = __ldg((const uint4 *)src);
+        u1 = __ldg((const uint4 *)(src + r_t));
+      }
+      const uint32_t w0[4] = {u0.x, u0.y, u0.z, u0.w}, w1[4] = {u1.x, u1.y, u1.z, u1.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        Us[tp][k8 + 2 * j] = (w0[j] & 0xFFFFu) | (w1[j] << 16);
+        Us[tp][k8 + 2 * j + 1] = (w0[j] >> 16) | (w1[j] & 0xFFFF0000u);
+      }
     }
     __syncthreads();
 #pragma unroll
-    for (int kk = 0; kk < 16; ++kk) {
-      const float4 a0 = *(const float4 *)&Ps[kk][ty * 8], a1 = *(const float4 *)&Ps[kk][ty * 8 + 4];
-      const float4 b4 = *(const float4 *)&Us[kk][tx * 4];
-      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-      const float b[4] = {b4.x, b4.y, b4.z, b4.w};
+    for (int s16 = 0; s16 < 2; ++s16) {
+      uint32_t ah[2][4], al[2][4];
 #pragma unroll
-      for (int ia = 0; ia < 8; ++ia)
+      for (int mt = 0; mt < 2; ++mt) {
+        const int nr = warp * 32 + mt * 16 + g;
+        ah[mt][0] = Ph[s16 * 8 + c][nr]; ah[mt][1] = Ph[s16 * 8 + c][nr + 8]; ah[mt][2] = Ph[s16 * 8 + c + 4][nr]; ah[mt][3] = Ph[s16 * 8 + c + 4][nr + 8];
+        al[mt][0] = Pl[s16 * 8 + c][nr]; al[mt][1] = Pl[s16 * 8 + c][nr + 8]; al[mt][2] = Pl[s16 * 8 + c + 4][nr]; al[mt][3] = Pl[s16 * 8 + c + 4][nr + 8];
+      }
 #pragma unroll
-        for (int ib = 0; ib < 4; ++ib) acc[ia][ib] = fmaf(a[ia], b[ib], acc[ia][ib]);
-    }
-    __syncthreads();
-  }
+      for (int nt = 0; nt < 8; ++nt) {
+        const uint32_t b0 = Us[s16 * 8 + c][nt * 8 + g], b1 = Us[s16 * 8 + c + 4][nt * 8 + g];
 #pragma unroll
-  for (int ib = 0; ib < 4; ++ib) {
-    const int k = kb + tx * 4 + ib;
-    if (k >= r_t) continue;
-#pragma unroll
-    for (int q4 = 0; q4 < 2; ++q4) {
-      const int n = n0 + ty * 8 + q4 * 4;
-      if (n < N)
-        *(float4 *)(jb.y + (((size_t)(n / NQP) * n_chunks + chunk) * r_t + k) * NQP + n % NQP) =
-            make_float4(acc[q4 * 4][ib], acc[q4 * 4 + 1][ib], acc[q4 * 4 + 2][ib], acc[q4 * 4 + 3][ib]);
+        for (int mt = 0; mt < 2; ++mt) {
+          att_mma_f16(acc[mt][nt], ah[mt], b0, b1);
+          att_mma_f16(acc[mt][nt], al[mt], b0, b1);
+        }
+      }
     }
   }
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int n = n0 + warp * 32 + mt * 16 + g + half * 8;
+      if (n >= N) continue;
+      float *yr = jb.y + ((size_t)(n / NQP) * n_chunks + chunk) * r_t * NQP + n % NQP;
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+        const int k = kb + nt * 8 + 2 * c;
+        if (k < r_t) yr[(size_t)k * NQP] = acc[mt][nt][half * 2];
+        if (k + 1 < r_t) yr[(size_t)(k + 1) * NQP] = acc[mt][nt][half * 2 + 1];
+      }
+    }
 }
 
 // grid (m, groups, n_q), 128 threads (thread = feature); CTA z finishes query z.  Dynamic shared memory:
