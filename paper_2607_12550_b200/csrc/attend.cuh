@@ -404,46 +404,70 @@ __device__ __forceinline__ uint32_t att_half_of(const uint4 &u, int c) {
 
 constexpr int kAttBPitch = 136;     // floats per staged operand row: 8 c + g addresses all 32 banks
 
-// grid (ceil(T / 64), ceil(m NQP / 128), groups), 128 threads: a warp owns 16 tokens x 128 columns n
-__global__ void __launch_bounds__(128) attend_bscore_kernel(const AttendJob *__restrict__ jobs, int NQP) {
+// grid (ceil(T / 64), ceil(m NQP / 128), groups), 256 threads: warp w owns 16 tokens (w & 3) x 64 columns n (w >> 2).
+// The operands of the next 32-wide k chunk are requested into registers before the MMAs of the current one.
+__global__ void __launch_bounds__(256) attend_bscore_kernel(const AttendJob *__restrict__ jobs, int NQP) {
   const AttendJob &jb = jobs[blockIdx.z];
   const int r_t = jb.k.r_t, N = jb.m * NQP, n0 = blockIdx.y * 128, t0 = blockIdx.x * 64;
   if (r_t == 0 || n0 >= N || t0 >= jb.T) return;
   __shared__ __align__(16) uint32_t Bh[32][kAttBPitch], Bl[32][kAttBPitch];       // w chunk, hi and lo, [k][n]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
-  float acc[16][4];
+  const int wt = warp & 3, wn = warp >> 2;
+  float acc[8][4];
 #pragma unroll
-  for (int nt = 0; nt < 16; ++nt)
+  for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[nt][j] = 0.f;
-  const int ta = min(t0 + warp * 16 + g, jb.T - 1), tb = min(t0 + warp * 16 + g + 8, jb.T - 1);   // rows past the end repeat the last
+  const int ta = min(t0 + wt * 16 + g, jb.T - 1), tb = min(t0 + wt * 16 + g + 8, jb.T - 1);   // rows past the end repeat the last
   const __half *rowa = jb.k.UT + (size_t)ta * r_t, *rowb = jb.k.UT + (size_t)tb * r_t;
+  float4 breg[4];
+  uint4 areg[4][2];
+  auto load_chunk = [&](int k0) {
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      const int idx = tid + it * 256, kk = idx >> 5, q4 = idx & 31, n = n0 + q4 * 4;
+      breg[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (n < N && k0 + kk < r_t) breg[it] = *(const float4 *)(jb.w + ((size_t)(n / NQP) * r_t + k0 + kk) * NQP + n % NQP);
+    }
+#pragma unroll
+    for (int k8 = 0; k8 < 4; ++k8) {
+      areg[k8][0] = make_uint4(0u, 0u, 0u, 0u); areg[k8][1] = areg[k8][0];
+      if (k0 + k8 * 8 < r_t) {
+        areg[k8][0] = __ldg((const uint4 *)(rowa + k0 + k8 * 8));
+        areg[k8][1] = __ldg((const uint4 *)(rowb + k0 + k8 * 8));
+      }
+    }
+  };
+  load_chunk(0);
   for (int k0 = 0; k0 < r_t; k0 += 32) {
     __syncthreads();
-    for (int idx = tid; idx < 32 * 32; idx += 128) {
-      const int kk = idx >> 5, q4 = idx & 31, n = n0 + q4 * 4;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (n < N && k0 + kk < r_t) v = *(const float4 *)(jb.w + ((size_t)(n / NQP) * r_t + k0 + kk) * NQP + n % NQP);
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      const int idx = tid + it * 256, kk = idx >> 5, q4 = idx & 31;
+      const float4 v = breg[it];
       *(uint4 *)&Bh[kk][q4 * 4] = make_uint4(att_tf32_hi(v.x), att_tf32_hi(v.y), att_tf32_hi(v.z), att_tf32_hi(v.w));
       *(uint4 *)&Bl[kk][q4 * 4] = make_uint4(att_tf32_lo(v.x), att_tf32_lo(v.y), att_tf32_lo(v.z), att_tf32_lo(v.w));
     }
+    uint4 acur[4][2];
+#pragma unroll
+    for (int k8 = 0; k8 < 4; ++k8) { acur[k8][0] = areg[k8][0]; acur[k8][1] = areg[k8][1]; }
     __syncthreads();
+    if (k0 + 32 < r_t) load_chunk(k0 + 32);
 #pragma unroll
     for (int k8 = 0; k8 < 4; ++k8) {
-      if (k0 + k8 * 8 >= r_t) break;
-      const uint4 ua = __ldg((const uint4 *)(rowa + k0 + k8 * 8)), ub = __ldg((const uint4 *)(rowb + k0 + k8 * 8));
-      const uint32_t a[4] = {att_half_of(ua, c), att_half_of(ub, c), att_half_of(ua, c + 4), att_half_of(ub, c + 4)};
+      const uint32_t a[4] = {att_half_of(acur[k8][0], c), att_half_of(acur[k8][1], c), att_half_of(acur[k8][0], c + 4), att_half_of(acur[k8][1], c + 4)};
 #pragma unroll
-      for (int nt = 0; nt < 16; ++nt) {
-        att_mma_tf32(acc[nt], a, Bh[k8 * 8 + c][nt * 8 + g], Bh[k8 * 8 + c + 4][nt * 8 + g]);
-        att_mma_tf32(acc[nt], a, Bl[k8 * 8 + c][nt * 8 + g], Bl[k8 * 8 + c + 4][nt * 8 + g]);
+      for (int nt = 0; nt < 8; ++nt) {
+        const int col = wn * 64 + nt * 8 + g;
+        att_mma_tf32(acc[nt], a, Bh[k8 * 8 + c][col], Bh[k8 * 8 + c + 4][col]);
+        att_mma_tf32(acc[nt], a, Bl[k8 * 8 + c][col], Bl[k8 * 8 + c + 4][col]);
       }
     }
   }
-  const int t_lo = t0 + warp * 16 + g, t_hi = t_lo + 8;
+  const int t_lo = t0 + wt * 16 + g, t_hi = t_lo + 8;
 #pragma unroll
-  for (int nt = 0; nt < 16; ++nt) {
-    const int n = n0 + nt * 8 + 2 * c;
+  for (int nt = 0; nt < 8; ++nt) {
+    const int n = n0 + wn * 64 + nt * 8 + 2 * c;
     if (n >= N) continue;
     const size_t col = (size_t)(n / NQP) * jb.T * NQP + n % NQP;
     if (t_lo < jb.T) *(float2 *)(jb.p + col + (size_t)t_lo * NQP) = make_float2(acc[nt][0], acc[nt][1]);
@@ -457,10 +481,11 @@ __device__ __forceinline__ void att_mma_f16(float (&d)[4], const uint32_t (&a)[4
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// grid (n_chunks * KT, ceil(m NQP / 128), groups) with KT = ceil(max r_t / 64), 128 threads: 128 columns n x 64 columns k
-// of one 256-token chunk; a warp owns 32 n x 64 k.  m16n8k16 fp16 MMAs: U_T is fp16 as stored, a weight p in [0, 1]
-// enters as hi + lo fp16 (22 bits; the lo part of a tiny weight may be subnormal, an absolute error below 2^-25).
-__global__ void __launch_bounds__(128) attend_bvalue_kernel(const AttendJob *__restrict__ jobs, int NQP, int n_chunks, int KT) {
+// grid (n_chunks * KT, ceil(m NQP / 128), groups) with KT = ceil(max r_t / 64), 256 threads: 128 columns n x 64 columns k
+// of one 256-token chunk; warp w owns 16 n x 64 k.  m16n8k16 fp16 MMAs: U_T is fp16 as stored, a weight p in [0, 1]
+// enters as hi + lo fp16 (22 bits; the lo part of a tiny weight may be subnormal, an absolute error below 2^-25).  The
+// next 32 tokens' operands are requested into registers before the MMAs of the current 32.
+__global__ void __launch_bounds__(256) attend_bvalue_kernel(const AttendJob *__restrict__ jobs, int NQP, int n_chunks, int KT) {
   const AttendJob &jb = jobs[blockIdx.z];
   const int r_t = jb.v.r_t, N = jb.m * NQP, n0 = blockIdx.y * 128;
   const int chunk = blockIdx.x / KT, kb = (blockIdx.x % KT) * 64, t0 = chunk * kAttChunk;
@@ -469,24 +494,40 @@ __global__ void __launch_bounds__(128) attend_bvalue_kernel(const AttendJob *__r
   __shared__ __align__(16) uint32_t Ph[16][kAttBPitch], Pl[16][kAttBPitch];     // weights hi / lo, [tp][n]
   __shared__ __align__(16) uint32_t Us[16][64 + 8];                             // U_T, [tp][k]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
-  float acc[2][8][4];
+  float acc[8][4];
 #pragma unroll
-  for (int mt = 0; mt < 2; ++mt)
+  for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
-    for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) acc[mt][nt][j] = 0.f;
+    for (int j = 0; j < 4; ++j) acc[nt][j] = 0.f;
   const int nt_tok = min(kAttChunk, jb.T - t0);          // a multiple of 128
-  for (int tt0 = 0; tt0 < nt_tok; tt0 += 32) {
-    __syncthreads();
-    for (int idx = tid; idx < 16 * 32; idx += 128) {
-      const int tp = idx >> 5, q4 = idx & 31, n = n0 + q4 * 4;
-      float4 v0 = make_float4(0.f, 0.f, 0.f, 0.f), v1 = v0;
+  float4 preg[2][2];
+  uint4 ureg[2];
+  const int u_tp = (tid & 127) >> 3, u_k8 = (tid & 7) * 8;
+  auto load_step = [&](int tt0) {
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+      const int idx = tid + it * 256, tp = idx >> 5, q4 = idx & 31, n = n0 + q4 * 4;
+      preg[it][0] = make_float4(0.f, 0.f, 0.f, 0.f); preg[it][1] = preg[it][0];
       if (n < N) {
         const float *src = jb.p + ((size_t)(n / NQP) * jb.T + t0 + tt0 + 2 * tp) * NQP + n % NQP;
-        v0 = *(const float4 *)src;
-        v1 = *(const float4 *)(src + NQP);
+        preg[it][0] = *(const float4 *)src;
+        preg[it][1] = *(const float4 *)(src + NQP);
       }
+    }
+    ureg[0] = make_uint4(0u, 0u, 0u, 0u); ureg[1] = ureg[0];
+    if (tid < 128 && kb + u_k8 < r_t) {
+      const __half *src = jb.v.UT + (size_t)(t0 + tt0 + 2 * u_tp) * r_t + kb + u_k8;
+      ureg[0] = __ldg((const uint4 *)src);
+      ureg[1] = __ldg((const uint4 *)(src + r_t));
+    }
+  };
+  load_step(0);
+  for (int tt0 = 0; tt0 < nt_tok; tt0 += 32) {
+    __syncthreads();
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+      const int idx = tid + it * 256, tp = idx >> 5, q4 = idx & 31;
+      const float4 v0 = preg[it][0], v1 = preg[it][1];
       const float x0[4] = {v0.x, v0.y, v0.z, v0.w}, x1[4] = {v1.x, v1.y, v1.z, v1.w};
       uint32_t hi[4], lo[4];
 #pragma unroll
@@ -499,56 +540,41 @@ __global__ void __launch_bounds__(128) attend_bvalue_kernel(const AttendJob *__r
       *(uint4 *)&Ph[tp][q4 * 4] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
       *(uint4 *)&Pl[tp][q4 * 4] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     }
-    for (int idx = tid; idx < 16 * 8; idx += 128) {
-      const int tp = idx >> 3, k8 = (idx & 7) * 8;
-      uint4 u0 = make_uint4(0u, 0u, 0u, 0u), u1 = u0;
-      if (kb + k8 < r_t) {
-        const __half *src = jb.v.UT + (size_t)(t0 + tt0 + 2 * tp) * r_t + kb + k8;
-        u0 = __ldg((const uint4 *)src);
-        u1 = __ldg((const uint4 *)(src + r_t));
-      }
-      const uint32_t w0[4] = {u0.x, u0.y, u0.z, u0.w}, w1[4] = {u1.x, u1.y, u1.z, u1.w};
+    if (tid < 128) {
+      const uint32_t w0[4] = {ureg[0].x, ureg[0].y, ureg[0].z, ureg[0].w}, w1[4] = {ureg[1].x, ureg[1].y, ureg[1].z, ureg[1].w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        Us[tp][k8 + 2 * j] = (w0[j] & 0xFFFFu) | (w1[j] << 16);
-        Us[tp][k8 + 2 * j + 1] = (w0[j] >> 16) | (w1[j] & 0xFFFF0000u);
+        Us[u_tp][u_k8 + 2 * j] = (w0[j] & 0xFFFFu) | (w1[j] << 16);
+        Us[u_tp][u_k8 + 2 * j + 1] = (w0[j] >> 16) | (w1[j] & 0xFFFF0000u);
       }
     }
     __syncthreads();
+    if (tt0 + 32 < nt_tok) load_step(tt0 + 32);
 #pragma unroll
     for (int s16 = 0; s16 < 2; ++s16) {
-      uint32_t ah[2][4], al[2][4];
-#pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
-        const int nr = warp * 32 + mt * 16 + g;
-        ah[mt][0] = Ph[s16 * 8 + c][nr]; ah[mt][1] = Ph[s16 * 8 + c][nr + 8]; ah[mt][2] = Ph[s16 * 8 + c + 4][nr]; ah[mt][3] = Ph[s16 * 8 + c + 4][nr + 8];
-        al[mt][0] = Pl[s16 * 8 + c][nr]; al[mt][1] = Pl[s16 * 8 + c][nr + 8]; al[mt][2] = Pl[s16 * 8 + c + 4][nr]; al[mt][3] = Pl[s16 * 8 + c + 4][nr + 8];
-      }
+      const int nr = warp * 16 + g;
+      const uint32_t ah[4] = {Ph[s16 * 8 + c][nr], Ph[s16 * 8 + c][nr + 8], Ph[s16 * 8 + c + 4][nr], Ph[s16 * 8 + c + 4][nr + 8]};
+      const uint32_t al[4] = {Pl[s16 * 8 + c][nr], Pl[s16 * 8 + c][nr + 8], Pl[s16 * 8 + c + 4][nr], Pl[s16 * 8 + c + 4][nr + 8]};
 #pragma unroll
       for (int nt = 0; nt < 8; ++nt) {
         const uint32_t b0 = Us[s16 * 8 + c][nt * 8 + g], b1 = Us[s16 * 8 + c + 4][nt * 8 + g];
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-          att_mma_f16(acc[mt][nt], ah[mt], b0, b1);
-          att_mma_f16(acc[mt][nt], al[mt], b0, b1);
-        }
+        att_mma_f16(acc[nt], ah, b0, b1);
+        att_mma_f16(acc[nt], al, b0, b1);
       }
     }
   }
 #pragma unroll
-  for (int mt = 0; mt < 2; ++mt)
+  for (int half = 0; half < 2; ++half) {
+    const int n = n0 + warp * 16 + g + half * 8;
+    if (n >= N) continue;
+    float *yr = jb.y + ((size_t)(n / NQP) * n_chunks + chunk) * r_t * NQP + n % NQP;
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      const int n = n0 + warp * 32 + mt * 16 + g + half * 8;
-      if (n >= N) continue;
-      float *yr = jb.y + ((size_t)(n / NQP) * n_chunks + chunk) * r_t * NQP + n % NQP;
-#pragma unroll
-      for (int nt = 0; nt < 8; ++nt) {
-        const int k = kb + nt * 8 + 2 * c;
-        if (k < r_t) yr[(size_t)k * NQP] = acc[mt][nt][half * 2];
-        if (k + 1 < r_t) yr[(size_t)(k + 1) * NQP] = acc[mt][nt][half * 2 + 1];
-      }
+    for (int nt = 0; nt < 8; ++nt) {
+      const int k = kb + nt * 8 + 2 * c;
+      if (k < r_t) yr[(size_t)k * NQP] = acc[nt][half * 2];
+      if (k + 1 < r_t) yr[(size_t)(k + 1) * NQP] = acc[nt][half * 2 + 1];
     }
+  }
 }
 
 // grid (m, groups, n_q), 128 threads (thread = feature); CTA z finishes query z.  Dynamic shared memory:

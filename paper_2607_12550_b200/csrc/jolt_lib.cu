@@ -1606,7 +1606,7 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
     const dim3 grid(n_chunks, m_max, ng);
     const int n_tiles = (m_max * NQP + 127) / 128;
     if (krt > 0) {
-      attend_bscore_kernel<<<dim3((T + 63) / 64, n_tiles, ng), 128, 0, s>>>(d, NQP);
+      attend_bscore_kernel<<<dim3((T + 63) / 64, n_tiles, ng), 256, 0, s>>>(d, NQP);
       LAUNCHED();
     }
     for (int b = 0; b <= 8; ++b) {
@@ -1636,7 +1636,7 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
     }
     if (vrt > 0) {
       const int KT = (vrt + 63) / 64;
-      attend_bvalue_kernel<<<dim3(n_chunks * KT, n_tiles, ng), 128, 0, s>>>(d, NQP, n_chunks, KT);
+      attend_bvalue_kernel<<<dim3(n_chunks * KT, n_tiles, ng), 256, 0, s>>>(d, NQP, n_chunks, KT);
       LAUNCHED();
     }
     attend_combine_kernel<<<dim3(m_max, ng, n_q), 128, shm_comb, s>>>(d, n_q, NQP, n_chunks, seed);
