@@ -386,9 +386,10 @@ __global__ void __launch_bounds__(kAttChunk) attend_values_kernel(const AttendJo
 // whole cell instead of a loop per head:  with n = (head, query),
 //   attend_bscore_kernel   S_b[t][n] = sum_k U_T[t][k] w[n][k]            written to the weight buffer p[h][t][i]
 //   attend_bvalue_kernel   y[chunk][n][k] = sum_{t in chunk} p[n][t] U_T[t][k]
-// Both run on the tensor cores as warp-level m16n8k8 TF32 MMAs with fp32 accumulation: an fp16 entry of U_T is exact in
-// TF32, and the fp32 operand (w, p) enters as hi + lo (hi = the top 19 bits, lo = the remainder), which keeps about 21
-// bits of it.  0.13 GFLOP per cell each: too small to set up TMEM-resident tcgen05 tiles for.
+// Both run on the tensor cores as warp-level MMAs with fp32 accumulation, the fp32 operand entering as hi + lo:
+// the first as m16n8k8 TF32 (an fp16 entry of U_T is exact in TF32; w has no bounded range, hi = its top 19 bits, lo = the
+// remainder, about 21 bits kept), the second as m16n8k16 fp16 (p lies in [0, 1]).  0.13 GFLOP per cell each with
+// N = 128: too small to set up TMEM-resident tcgen05 tiles for.
 __device__ __forceinline__ void att_mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
