@@ -16,8 +16,9 @@
 //   attend_p16_kernel      P_h = fp16(G_h U_F^T) of every head of both cells (what the decoder's set-up also forms)
 //   attend_prep_kernel     per (group, head): rotated scaled queries and w = scale 2^e P_h q
 //   attend_bscore_kernel   backbone scores U_T w of all heads of a cell as one dense product (U_T is shared by the heads)
-//   attend_scores_kernel   per (group, head, 256-token chunk): residual scores added, chunk maximum, p = exp(s - max),
-//                          chunk sum
+//   attend_scores_mma_kernel / attend_scores_kernel   per (group, head, 256-token chunk): residual scores added (codes
+//                          times rotated query: warp-level fp16 MMAs for 1-, 2-, 4- and 8-bit codes, CUDA cores for 3-bit
+//                          codes and for cells without a residual), chunk maximum, p = exp(s - max), chunk sum
 //   attend_values_kernel   per (group, head, chunk): sum_t p_t r^'_t (codes staged in shared memory and read
 //                          feature-wise, so the token reduction stays inside a thread)
 //   attend_bvalue_kernel   p^T U_T per chunk for all heads of a cell as one dense product
@@ -51,6 +52,8 @@ struct AttendJob {                  // one per layer group
   __half *kP, *vP;                  // [m * r_t][128]    P_h = fp16(G_h U_F^T) of the key / value cell (scaled units)
   float *w;                         // [m][k.r_t][NQP]   scale 2^e P_h q
   float *qt;                        // [m][128][NQP]     scale H(s . q) / sqrt(d)
+  __half *qh, *ql;                  // [m][8][128]       the same, times 2^-E per (head, query), as hi + lo fp16 (MMA operand)
+  float *qe;                        // [m][8]            2^E
   float *p;                         // [m][T][NQP]       exp(s - chunk maximum)
   float *ml;                        // [m][n_chunks][2][NQP]  chunk maximum, chunk sum
   float *y;                         // [m][n_chunks][v.r_t][NQP]
@@ -131,8 +134,23 @@ __global__ void __launch_bounds__(128) attend_prep_kernel(const AttendJob *__res
   if (jb.k.bits > 0) {
     buf[f] = i < n_q ? att_sign(seed, jb.k.cell, f) * jb.q[((size_t)h * n_q + i) * 128 + f] : 0.f;
     __syncthreads();
-    const float v = att_wht_smem(buf, f);
-    jb.qt[((size_t)h * 128 + f) * NQP + i] = v * kInvSqrtD * scale;
+    const float v = att_wht_smem(buf, f) * kInvSqrtD * scale;
+    jb.qt[((size_t)h * 128 + f) * NQP + i] = v;
+    // the tensor-core form of the same row: scaled by a power of two so that hi + lo fp16 hold it (|entry| < 2^13)
+    __shared__ float wmax[4];
+    float mx = fabsf(v);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if ((f & 31) == 0) wmax[f >> 5] = mx;
+    __syncthreads();
+    mx = fmaxf(fmaxf(wmax[0], wmax[1]), fmaxf(wmax[2], wmax[3]));
+    int ex = 0;
+    if (mx > 0.f && mx < INFINITY) frexpf(mx, &ex);                  // mx < 2^ex
+    const float sv = ldexpf(v, 13 - ex);
+    const __half hi = __float2half_rn(sv);
+    jb.qh[((size_t)h * kAttMaxQ + i) * 128 + f] = hi;
+    jb.ql[((size_t)h * kAttMaxQ + i) * 128 + f] = __float2half_rn(sv - __half2float(hi));
+    if (f == 0) jb.qe[h * kAttMaxQ + i] = ldexpf(1.f, ex - 13);
   }
   if (jb.k.r_t > 0) {
     // w[k][q] = scale 2^e sum_f P_h[k][f] q_q[f]: a warp per row k, a lane per four features
@@ -284,6 +302,164 @@ __global__ void __launch_bounds__(kAttChunk, 3) attend_scores_kernel(const Atten
     float *ml = jb.ml + ((size_t)h * n_chunks + chunk) * 2 * NQP;
     float m_i = red[0][0][tid];
     for (int wq = 1; wq < kAttChunk / 32; ++wq) m_i = fmaxf(m_i, red[0][wq][tid]);
+    ml[tid] = m_i;
+    ml[NQP + tid] = l;
+  }
+}
+
+// warp-level m16n8k16 MMA, fp16 operands, fp32 accumulation
+__device__ __forceinline__ void att_mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// The score kernel for 1-, 2-, 4- and 8-bit codes with the code-times-query contraction on the tensor cores.
+// grid (n_chunks, m, groups), kAttChunk threads = 8 warps; a warp owns 32 tokens = two 16-row MMA tiles.  Every lane
+// still loads its own token's packed row and scales (as in the CUDA-core kernel); the m16n8k16 A fragments are built from
+// words handed over by warp shuffles (the lane of row g holds that row), a pair of codes expanding to the exact fp16
+// integers 2u + 1 - 2^b (so the mid-rise half step is part of the operand and the product is twice the wanted sum).
+// B = the rotated query as hi + lo fp16, 8 query columns, resident in registers for the whole CTA.  Per 32-feature
+// group the 16 x 8 partial product is scaled by Delta / 2 of its row.  No shared-memory traffic per code.
+__device__ __forceinline__ uint32_t att_pair_f16(uint32_t x, int bits) {
+  const uint32_t mask = (1u << bits) - 1u;
+  const uint32_t v = ((x & mask) << 1) | (((x >> bits) & mask) << 17) | 0x64016401u;        // half2(1024 + 2u + 1)
+  const __half2 off = __float2half2_rn(1024.f + (float)(1 << bits));
+  const __half2 r = __hsub2(*(const __half2 *)&v, off);
+  return *(const uint32_t *)&r;
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kAttChunk, 2) attend_scores_mma_kernel(const AttendJob *__restrict__ jobs, int NQP) {
+  static_assert(BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8, "codes that do not straddle words");
+  const AttendJob &jb = jobs[blockIdx.z];
+  if (jb.k.bits != BITS) return;
+  const int h = blockIdx.y, chunk = blockIdx.x, n_chunks = gridDim.x;
+  if (h >= jb.m || chunk * kAttChunk >= jb.T) return;
+  __shared__ float red[2][kAttChunk / 32][kAttMaxQ];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
+  const int t = chunk * kAttChunk + tid;                 // this lane's own token (row `lane` of the warp's 32)
+  const bool live = chunk * kAttChunk + warp * 32 < jb.T;      // T is a multiple of 128: a warp is all in or all out
+  // the lane's own packed row and scales
+  uint32_t row[4 * BITS];
+  uint2 scw = make_uint2(0u, 0u);
+  if (live) {
+    const uint4 *wp = (const uint4 *)(jb.k.words + ((size_t)h * jb.T + t) * (4 * BITS));
+#pragma unroll
+    for (int i = 0; i < BITS; ++i) { const uint4 v = __ldg(wp + i); row[4 * i] = v.x; row[4 * i + 1] = v.y; row[4 * i + 2] = v.z; row[4 * i + 3] = v.w; }
+    scw = __ldg((const uint2 *)(jb.k.scales + ((size_t)h * jb.T + t) * 4));
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4 * BITS; ++i) row[i] = 0u;
+  }
+  // B fragments of all eight k16 steps: query column g, features 16 s + 2c, +1 and + 8
+  uint32_t bh[8][2], bl[8][2];
+  {
+    const uint32_t *qh = (const uint32_t *)(jb.qh + ((size_t)h * kAttMaxQ + g) * 128);
+    const uint32_t *ql = (const uint32_t *)(jb.ql + ((size_t)h * kAttMaxQ + g) * 128);
+    const bool have = g < NQP;
+#pragma unroll
+    for (int s8 = 0; s8 < 8; ++s8) {
+      bh[s8][0] = have ? __ldg(qh + s8 * 8 + c) : 0u; bh[s8][1] = have ? __ldg(qh + s8 * 8 + c + 4) : 0u;
+      bl[s8][0] = have ? __ldg(ql + s8 * 8 + c) : 0u; bl[s8][1] = have ? __ldg(ql + s8 * 8 + c + 4) : 0u;
+    }
+  }
+  float sc[2][4];          // [tile][row g: queries 2c, 2c+1; row g + 8: queries 2c, 2c+1]
+#pragma unroll
+  for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) sc[tl][j] = 0.f;
+#pragma unroll
+  for (int tl = 0; tl < 2; ++tl) {
+    const int la = tl * 16 + g, lb = la + 8;           // lanes that hold rows g and g + 8 of this tile
+    const uint32_t sxa = __shfl_sync(0xffffffffu, scw.x, la), sya = __shfl_sync(0xffffffffu, scw.y, la);
+    const uint32_t sxb = __shfl_sync(0xffffffffu, scw.x, lb), syb = __shfl_sync(0xffffffffu, scw.y, lb);
+#pragma unroll
+    for (int gq = 0; gq < 4; ++gq) {
+      float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int s2 = 0; s2 < 2; ++s2) {
+        const int s8 = gq * 2 + s2;
+        uint32_t a[4];
+        if constexpr (BITS == 8) {            // 16 bits at bit 128 s2 + 16 c: word 4 s2 + (c >> 1), half c & 1; + 8 columns: two words on
+          const int w0 = gq * 8 + s2 * 4;
+          const uint32_t a00 = __shfl_sync(0xffffffffu, row[w0], la), a01 = __shfl_sync(0xffffffffu, row[w0 + 1], la);
+          const uint32_t a02 = __shfl_sync(0xffffffffu, row[w0 + 2], la), a03 = __shfl_sync(0xffffffffu, row[w0 + 3], la);
+          const uint32_t b00 = __shfl_sync(0xffffffffu, row[w0], lb), b01 = __shfl_sync(0xffffffffu, row[w0 + 1], lb);
+          const uint32_t b02 = __shfl_sync(0xffffffffu, row[w0 + 2], lb), b03 = __shfl_sync(0xffffffffu, row[w0 + 3], lb);
+          const int sh = 16 * (c & 1);
+          a[0] = att_pair_f16(((c & 2) ? a01 : a00) >> sh, 8); a[1] = att_pair_f16(((c & 2) ? b01 : b00) >> sh, 8);
+          a[2] = att_pair_f16(((c & 2) ? a03 : a02) >> sh, 8); a[3] = att_pair_f16(((c & 2) ? b03 : b02) >> sh, 8);
+        } else if constexpr (BITS == 4) {     // 8 bits at bit 64 s2 + 8 c: word 2 s2, byte c; + 8 columns: the next word
+          const int w0 = gq * 4 + s2 * 2;
+          const uint32_t a0 = __shfl_sync(0xffffffffu, row[w0], la), a1 = __shfl_sync(0xffffffffu, row[w0 + 1], la);
+          const uint32_t b0 = __shfl_sync(0xffffffffu, row[w0], lb), b1 = __shfl_sync(0xffffffffu, row[w0 + 1], lb);
+          a[0] = att_pair_f16(a0 >> (8 * c), 4); a[1] = att_pair_f16(b0 >> (8 * c), 4);
+          a[2] = att_pair_f16(a1 >> (8 * c), 4); a[3] = att_pair_f16(b1 >> (8 * c), 4);
+        } else if constexpr (BITS == 2) {     // 4 bits at bit 32 s2 + 4 c: word s2, nibble c; + 8 columns: 16 bits on
+          const int w0 = gq * 2 + s2;
+          const uint32_t a0 = __shfl_sync(0xffffffffu, row[w0], la), b0 = __shfl_sync(0xffffffffu, row[w0], lb);
+          a[0] = att_pair_f16(a0 >> (4 * c), 2); a[1] = att_pair_f16(b0 >> (4 * c), 2);
+          a[2] = att_pair_f16(a0 >> (4 * c + 16), 2); a[3] = att_pair_f16(b0 >> (4 * c + 16), 2);
+        } else {                              // 2 bits at bit 16 s2 + 2 c of the group's single word; + 8 columns: 8 bits on
+          const uint32_t a0 = __shfl_sync(0xffffffffu, row[gq], la), b0 = __shfl_sync(0xffffffffu, row[gq], lb);
+          a[0] = att_pair_f16(a0 >> (16 * s2 + 2 * c), 1); a[1] = att_pair_f16(b0 >> (16 * s2 + 2 * c), 1);
+          a[2] = att_pair_f16(a0 >> (16 * s2 + 2 * c + 8), 1); a[3] = att_pair_f16(b0 >> (16 * s2 + 2 * c + 8), 1);
+        }
+        att_mma_f16(d, a, bh[s8][0], bh[s8][1]);
+        att_mma_f16(d, a, bl[s8][0], bl[s8][1]);
+      }
+      // Delta / 2 of rows g and g + 8 for this group: half (gq & 1) of scale word gq >> 1
+      const uint32_t wa = (gq & 2) ? sya : sxa, wb = (gq & 2) ? syb : sxb;
+      const float da = 0.5f * __half2float(__ushort_as_half((unsigned short)((gq & 1) ? (wa >> 16) : (wa & 0xFFFFu))));
+      const float db = 0.5f * __half2float(__ushort_as_half((unsigned short)((gq & 1) ? (wb >> 16) : (wb & 0xFFFFu))));
+      sc[tl][0] = fmaf(da, d[0], sc[tl][0]); sc[tl][1] = fmaf(da, d[1], sc[tl][1]);
+      sc[tl][2] = fmaf(db, d[2], sc[tl][2]); sc[tl][3] = fmaf(db, d[3], sc[tl][3]);
+    }
+  }
+  // undo the query scaling, add the backbone scores; this lane: queries 2c, 2c + 1 of rows g, g + 8, 16 + g, 24 + g
+  const bool qok = 2 * c < NQP;
+  const float e0 = qok ? jb.qe[h * kAttMaxQ + 2 * c] : 0.f, e1 = qok ? jb.qe[h * kAttMaxQ + 2 * c + 1] : 0.f;
+  const int tw = chunk * kAttChunk + warp * 32;
+  float *prow[4];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) prow[r] = jb.p + ((size_t)h * jb.T + tw + (r >> 1) * 16 + (r & 1) * 8 + g) * NQP + 2 * c;
+  float sv[4][2];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    sv[r][0] = sc[r >> 1][(r & 1) * 2] * e0;
+    sv[r][1] = sc[r >> 1][(r & 1) * 2 + 1] * e1;
+    if (live && qok && jb.k.r_t > 0) { const float2 b = *(const float2 *)prow[r]; sv[r][0] += b.x; sv[r][1] += b.y; }
+  }
+  // chunk maximum and sum of exp(s - maximum), per query: over this lane's rows, the lanes of equal c, the warps
+  float m0 = -INFINITY, m1 = -INFINITY;
+  if (live) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) { m0 = fmaxf(m0, sv[r][0]); m1 = fmaxf(m1, sv[r][1]); }
+  }
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) { m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, o)); m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o)); }
+  if (g == 0) { red[0][warp][2 * c] = m0; red[0][warp][2 * c + 1] = m1; }
+  __syncthreads();
+  m0 = red[0][0][2 * c]; m1 = red[0][0][2 * c + 1];
+#pragma unroll
+  for (int wq = 1; wq < kAttChunk / 32; ++wq) { m0 = fmaxf(m0, red[0][wq][2 * c]); m1 = fmaxf(m1, red[0][wq][2 * c + 1]); }
+  float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const float p0 = live ? expf(sv[r][0] - m0) : 0.f, p1 = live ? expf(sv[r][1] - m1) : 0.f;
+    l0 += p0; l1 += p1;
+    if (live && qok) *(float2 *)prow[r] = make_float2(p0, p1);
+  }
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) { l0 += __shfl_xor_sync(0xffffffffu, l0, o); l1 += __shfl_xor_sync(0xffffffffu, l1, o); }
+  if (g == 0) { red[1][warp][2 * c] = l0; red[1][warp][2 * c + 1] = l1; }
+  __syncthreads();
+  if (tid < NQP) {
+    float l = 0.f, m_i = red[0][0][tid];
+    for (int wq = 0; wq < kAttChunk / 32; ++wq) l += red[1][wq][tid];
+    for (int wq = 1; wq < kAttChunk / 32; ++wq) m_i = fmaxf(m_i, red[0][wq][tid]);
+    float *ml = jb.ml + ((size_t)h * n_chunks + chunk) * 2 * NQP;
     ml[tid] = m_i;
     ml[NQP + tid] = l;
   }
@@ -474,12 +650,6 @@ __global__ void __launch_bounds__(256) attend_bscore_kernel(const AttendJob *__r
     if (t_lo < jb.T) *(float2 *)(jb.p + col + (size_t)t_lo * NQP) = make_float2(acc[nt][0], acc[nt][1]);
     if (t_hi < jb.T) *(float2 *)(jb.p + col + (size_t)t_hi * NQP) = make_float2(acc[nt][2], acc[nt][3]);
   }
-}
-
-__device__ __forceinline__ void att_mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
 // grid (n_chunks * KT, ceil(m NQP / 128), groups) with KT = ceil(max r_t / 64), 256 threads: 128 columns n x 64 columns k

@@ -1508,6 +1508,10 @@ static void launch_att_scores(dim3 grid, size_t shm, cudaStream_t s, const Atten
   attend_scores_kernel<BITS><<<grid, kAttChunk, shm, s>>>(d, NQP);
 }
 template <int BITS>
+static void launch_att_scores_mma(dim3 grid, cudaStream_t s, const AttendJob *d, int NQP) {
+  attend_scores_mma_kernel<BITS><<<grid, kAttChunk, 0, s>>>(d, NQP);
+}
+template <int BITS>
 static void launch_att_values(dim3 grid, size_t shm, cudaStream_t s, const AttendJob *d, int NQP) {
   static std::atomic<bool> opted{false};      // up to 58 KB of dynamic shared memory (8-bit codes, 8 queries)
   if (!opted.exchange(true)) cudaFuncSetAttribute(attend_values_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
@@ -1578,6 +1582,9 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
       j.vP = H->att_P + H->att_P_off[2 * g + 1];
       j.w = b.take<float>((size_t)j.m * std::max(j.k.r_t, 1) * NQP);
       j.qt = b.take<float>((size_t)j.m * kD * NQP);
+      j.qh = b.take<__half>((size_t)j.m * kAttMaxQ * kD);
+      j.ql = b.take<__half>((size_t)j.m * kAttMaxQ * kD);
+      j.qe = b.take<float>((size_t)j.m * kAttMaxQ);
       j.p = b.take<float>((size_t)j.m * T * NQP);
       j.ml = b.take<float>((size_t)j.m * n_chunks * 2 * NQP);
       j.y = b.take<float>((size_t)j.m * n_chunks * std::max(j.v.r_t, 1) * NQP);
@@ -1590,6 +1597,7 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
   const uint64_t seed = H->seed;
   const float fscale = (float)scale;
   cudaEvent_t att_ready = H->att_ready;
+  const bool mma = (g_fast.load() & 1) != 0;        // warp-MMA form of the score kernel (the CUDA-core form stays as the portable path)
   P.add(ST_ATT, [=](char *dev_t, cudaStream_t s) {
     const AttendJob *d = (const AttendJob *)(dev_t + off);
     if (first_call) {
@@ -1613,11 +1621,11 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
       if (!((kbits >> b) & 1)) continue;
       switch (b) {
         case 0: launch_att_scores<0>(grid, shm_sc, s, d, NQP); break;
-        case 1: launch_att_scores<1>(grid, shm_sc, s, d, NQP); break;
-        case 2: launch_att_scores<2>(grid, shm_sc, s, d, NQP); break;
+        case 1: if (mma) launch_att_scores_mma<1>(grid, s, d, NQP); else launch_att_scores<1>(grid, shm_sc, s, d, NQP); break;
+        case 2: if (mma) launch_att_scores_mma<2>(grid, s, d, NQP); else launch_att_scores<2>(grid, shm_sc, s, d, NQP); break;
         case 3: launch_att_scores<3>(grid, shm_sc, s, d, NQP); break;
-        case 4: launch_att_scores<4>(grid, shm_sc, s, d, NQP); break;
-        default: launch_att_scores<8>(grid, shm_sc, s, d, NQP); break;
+        case 4: if (mma) launch_att_scores_mma<4>(grid, s, d, NQP); else launch_att_scores<4>(grid, shm_sc, s, d, NQP); break;
+        default: if (mma) launch_att_scores_mma<8>(grid, s, d, NQP); else launch_att_scores<8>(grid, shm_sc, s, d, NQP); break;
       }
       LAUNCHED();
     }

@@ -487,7 +487,7 @@ def test_rope_at_decode(B, synth, dtype, fused):
 
 
 # --------------------------------------------------------------------------- attention on the compressed cache
-@pytest.mark.parametrize("case", ["a", "b"])
+@pytest.mark.parametrize("case", ["a", "b", "c"])
 def test_attend_on_the_factors(B, synth, case):
     # Injected factors (both sides hold the same stored backbone).  T = 384 leaves a 128-token tail chunk.
     cfg = synth.CacheConfig("t", 4, 2, 2, 384, n_terms=20, seed=51)
@@ -495,8 +495,10 @@ def test_attend_on_the_factors(B, synth, case):
     gs = [0, 2, 4]
     if case == "a":
         plans, n_q = [(16, 64, 4), (16, 128, 2), (32, 96, 3), (0, 0, 8)], 4
-    else:
+    elif case == "b":
         plans, n_q = [(0, 0, 4), (24, 96, 0), (16, 128, 1), (16, 64, 4)], 5
+    else:
+        plans, n_q = [(16, 64, 8), (16, 128, 4), (32, 96, 2), (0, 0, 8)], 8
     Knp, Vnp = _np(K), _np(V)
     UT, UF = [], []
     for c, (rt, rf, _) in enumerate(plans):
