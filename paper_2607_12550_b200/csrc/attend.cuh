@@ -315,12 +315,14 @@ __device__ __forceinline__ void att_mma_f16(float (&d)[4], const uint32_t (&a)[4
 }
 
 // The score kernel for 1-, 2-, 4- and 8-bit codes with the code-times-query contraction on the tensor cores.
-// grid (n_chunks, m, groups), kAttChunk threads = 8 warps; a warp owns 32 tokens = two 16-row MMA tiles.  Every lane
+// grid (ceil(n_chunks / 2), m, groups), kAttChunk threads = 8 warps; a CTA walks every gridDim.x-th chunk of its head, a
+// warp owns 32 tokens of the chunk = two 16-row MMA tiles.  Every lane
 // still loads its own token's packed row and scales (as in the CUDA-core kernel); the m16n8k16 A fragments are built from
 // words handed over by warp shuffles (the lane of row g holds that row), a pair of codes expanding to the exact fp16
 // integers 2u + 1 - 2^b (so the mid-rise half step is part of the operand and the product is twice the wanted sum).
-// B = the rotated query as hi + lo fp16, 8 query columns, resident in registers for the whole CTA.  Per 32-feature
-// group the 16 x 8 partial product is scaled by Delta / 2 of its row.  No shared-memory traffic per code.
+// B = the rotated query as hi + lo fp16, 8 query columns, staged once per CTA in shared memory (4 conflict-free word
+// reads per MMA pair).  Per 32-feature group the 16 x 8 partial product is scaled by Delta / 2 of its row.  Registers are
+// capped for three CTAs per SM: the kernel is bound by the latency of its row loads, not by any pipe.
 __device__ __forceinline__ uint32_t att_pair_f16(uint32_t x, int bits) {
   const uint32_t mask = (1u << bits) - 1u;
   const uint32_t v = ((x & mask) << 1) | (((x >> bits) & mask) << 17) | 0x64016401u;        // half2(1024 + 2u + 1)
@@ -330,40 +332,55 @@ __device__ __forceinline__ uint32_t att_pair_f16(uint32_t x, int bits) {
 }
 
 template <int BITS>
-__global__ void __launch_bounds__(kAttChunk, 2) attend_scores_mma_kernel(const AttendJob *__restrict__ jobs, int NQP) {
+__global__ void __launch_bounds__(kAttChunk, 3) attend_scores_mma_kernel(const AttendJob *__restrict__ jobs, int NQP, int n_chunks) {
   static_assert(BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8, "codes that do not straddle words");
   const AttendJob &jb = jobs[blockIdx.z];
   if (jb.k.bits != BITS) return;
-  const int h = blockIdx.y, chunk = blockIdx.x, n_chunks = gridDim.x;
-  if (h >= jb.m || chunk * kAttChunk >= jb.T) return;
+  const int h = blockIdx.y;
+  if (h >= jb.m || (int)blockIdx.x * kAttChunk >= jb.T) return;
   __shared__ float red[2][kAttChunk / 32][kAttMaxQ];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
-  const int t = chunk * kAttChunk + tid;                 // this lane's own token (row `lane` of the warp's 32)
-  const bool live = chunk * kAttChunk + warp * 32 < jb.T;      // T is a multiple of 128: a warp is all in or all out
-  // the lane's own packed row and scales
-  uint32_t row[4 * BITS];
-  uint2 scw = make_uint2(0u, 0u);
-  if (live) {
-    const uint4 *wp = (const uint4 *)(jb.k.words + ((size_t)h * jb.T + t) * (4 * BITS));
+  // the lane's own packed row and scales, requested one chunk ahead
+  uint32_t nrow[4 * BITS];
+  uint2 nsc = make_uint2(0u, 0u);
+  float2 nsb[4];                   // backbone scores of this lane's four (row, query pair) results
+  const bool qok = 2 * c < NQP;
+  auto fetch = [&](int chunk) {
+    const int t = chunk * kAttChunk + tid;
 #pragma unroll
-    for (int i = 0; i < BITS; ++i) { const uint4 v = __ldg(wp + i); row[4 * i] = v.x; row[4 * i + 1] = v.y; row[4 * i + 2] = v.z; row[4 * i + 3] = v.w; }
-    scw = __ldg((const uint2 *)(jb.k.scales + ((size_t)h * jb.T + t) * 4));
-  } else {
+    for (int r = 0; r < 4; ++r) nsb[r] = make_float2(0.f, 0.f);
+    if (chunk < n_chunks && chunk * kAttChunk + warp * 32 < jb.T) {
+      if (qok && jb.k.r_t > 0) {
 #pragma unroll
-    for (int i = 0; i < 4 * BITS; ++i) row[i] = 0u;
-  }
-  // B fragments of all eight k16 steps: query column g, features 16 s + 2c, +1 and + 8
-  uint32_t bh[8][2], bl[8][2];
-  {
-    const uint32_t *qh = (const uint32_t *)(jb.qh + ((size_t)h * kAttMaxQ + g) * 128);
-    const uint32_t *ql = (const uint32_t *)(jb.ql + ((size_t)h * kAttMaxQ + g) * 128);
-    const bool have = g < NQP;
+        for (int r = 0; r < 4; ++r)
+          nsb[r] = *(const float2 *)(jb.p + ((size_t)h * jb.T + chunk * kAttChunk + warp * 32 + (r >> 1) * 16 + (r & 1) * 8 + g) * NQP + 2 * c);
+      }
+      const uint4 *wp = (const uint4 *)(jb.k.words + ((size_t)h * jb.T + t) * (4 * BITS));
 #pragma unroll
-    for (int s8 = 0; s8 < 8; ++s8) {
-      bh[s8][0] = have ? __ldg(qh + s8 * 8 + c) : 0u; bh[s8][1] = have ? __ldg(qh + s8 * 8 + c + 4) : 0u;
-      bl[s8][0] = have ? __ldg(ql + s8 * 8 + c) : 0u; bl[s8][1] = have ? __ldg(ql + s8 * 8 + c + 4) : 0u;
+      for (int i = 0; i < BITS; ++i) { const uint4 v = __ldg(wp + i); nrow[4 * i] = v.x; nrow[4 * i + 1] = v.y; nrow[4 * i + 2] = v.z; nrow[4 * i + 3] = v.w; }
+      nsc = __ldg((const uint2 *)(jb.k.scales + ((size_t)h * jb.T + t) * 4));
     }
+  };
+  fetch(blockIdx.x);
+  // B operand (rotated query, hi and lo) of the head in shared memory: [query][feature pair], 68 words per row so that
+  // the fragment reads (query g, pair 8 s + c) touch 32 different banks
+  __shared__ uint32_t Bq[2][kAttMaxQ][68];
+  for (int i = tid; i < 2 * kAttMaxQ * 64; i += kAttChunk) {
+    const int hl = i >> 9, q = (i >> 6) & 7, w = i & 63;
+    const uint32_t *src = (const uint32_t *)((hl ? jb.ql : jb.qh) + ((size_t)h * kAttMaxQ + q) * 128);
+    Bq[hl][q][w] = q < NQP ? __ldg(src + w) : 0u;
   }
+  __syncthreads();
+  for (int chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+  const bool live = chunk * kAttChunk + warp * 32 < jb.T;      // T is a multiple of 128: a warp is all in or all out
+  uint32_t row[4 * BITS];
+#pragma unroll
+  for (int i = 0; i < 4 * BITS; ++i) row[i] = live ? nrow[i] : 0u;
+  const uint2 scw = nsc;
+  float2 sb[4];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) sb[r] = nsb[r];
+  fetch(chunk + gridDim.x);                              // in flight during this chunk's MMAs
   float sc[2][4];          // [tile][row g: queries 2c, 2c+1; row g + 8: queries 2c, 2c+1]
 #pragma unroll
   for (int tl = 0; tl < 2; ++tl)
@@ -406,8 +423,8 @@ __global__ void __launch_bounds__(kAttChunk, 2) attend_scores_mma_kernel(const A
           a[0] = att_pair_f16(a0 >> (16 * s2 + 2 * c), 1); a[1] = att_pair_f16(b0 >> (16 * s2 + 2 * c), 1);
           a[2] = att_pair_f16(a0 >> (16 * s2 + 2 * c + 8), 1); a[3] = att_pair_f16(b0 >> (16 * s2 + 2 * c + 8), 1);
         }
-        att_mma_f16(d, a, bh[s8][0], bh[s8][1]);
-        att_mma_f16(d, a, bl[s8][0], bl[s8][1]);
+        att_mma_f16(d, a, Bq[0][g][s8 * 8 + c], Bq[0][g][s8 * 8 + c + 4]);
+        att_mma_f16(d, a, Bq[1][g][s8 * 8 + c], Bq[1][g][s8 * 8 + c + 4]);
       }
       // Delta / 2 of rows g and g + 8 for this group: half (gq & 1) of scale word gq >> 1
       const uint32_t wa = (gq & 2) ? sya : sxa, wb = (gq & 2) ? syb : sxb;
@@ -418,7 +435,6 @@ __global__ void __launch_bounds__(kAttChunk, 2) attend_scores_mma_kernel(const A
     }
   }
   // undo the query scaling, add the backbone scores; this lane: queries 2c, 2c + 1 of rows g, g + 8, 16 + g, 24 + g
-  const bool qok = 2 * c < NQP;
   const float e0 = qok ? jb.qe[h * kAttMaxQ + 2 * c] : 0.f, e1 = qok ? jb.qe[h * kAttMaxQ + 2 * c + 1] : 0.f;
   const int tw = chunk * kAttChunk + warp * 32;
   float *prow[4];
@@ -429,7 +445,7 @@ __global__ void __launch_bounds__(kAttChunk, 2) attend_scores_mma_kernel(const A
   for (int r = 0; r < 4; ++r) {
     sv[r][0] = sc[r >> 1][(r & 1) * 2] * e0;
     sv[r][1] = sc[r >> 1][(r & 1) * 2 + 1] * e1;
-    if (live && qok && jb.k.r_t > 0) { const float2 b = *(const float2 *)prow[r]; sv[r][0] += b.x; sv[r][1] += b.y; }
+    sv[r][0] += sb[r].x; sv[r][1] += sb[r].y;
   }
   // chunk maximum and sum of exp(s - maximum), per query: over this lane's rows, the lanes of equal c, the warps
   float m0 = -INFINITY, m1 = -INFINITY;
@@ -462,6 +478,8 @@ __global__ void __launch_bounds__(kAttChunk, 2) attend_scores_mma_kernel(const A
     float *ml = jb.ml + ((size_t)h * n_chunks + chunk) * 2 * NQP;
     ml[tid] = m_i;
     ml[NQP + tid] = l;
+  }
+  __syncthreads();            // red is rewritten by the next chunk
   }
 }
 

@@ -1509,7 +1509,9 @@ static void launch_att_scores(dim3 grid, size_t shm, cudaStream_t s, const Atten
 }
 template <int BITS>
 static void launch_att_scores_mma(dim3 grid, cudaStream_t s, const AttendJob *d, int NQP) {
-  attend_scores_mma_kernel<BITS><<<grid, kAttChunk, 0, s>>>(d, NQP);
+  const int n_chunks = (int)grid.x;
+  grid.x = (grid.x + 1) / 2;                 // two chunks per CTA: the query operand is staged once, the second chunk's rows are prefetched
+  attend_scores_mma_kernel<BITS><<<grid, kAttChunk, 0, s>>>(d, NQP, n_chunks);
 }
 template <int BITS>
 static void launch_att_values(dim3 grid, size_t shm, cudaStream_t s, const AttendJob *d, int NQP) {
