@@ -483,96 +483,95 @@ __global__ void __launch_bounds__(kAttChunk, 3) attend_scores_mma_kernel(const A
   }
 }
 
-// grid (n_chunks, m, groups), kAttChunk threads.  Dynamic shared memory: kAttChunk * (NQP floats + 4 BITS words + 4 halves)
-// + 4 * 128 * NQP floats.
-template <int BITS>
-__global__ void __launch_bounds__(kAttChunk) attend_values_kernel(const AttendJob *__restrict__ jobs, int NQP) {
+// grid (n_chunks, m, groups), kAttChunk threads.  The chunk is staged in two halves of 128 tokens (codes, scales and
+// weights, coalesced), so that six CTAs fit an SM: the kernel lives on the number of warps that hide its staging
+// latency.  NQ = 4 or 8 query slots (compile time: the accumulators are the register budget).  Dynamic shared memory:
+// 128 * (NQ floats + 4 BITS words + 4 halves) + 4 * 128 * NQ floats.
+constexpr int kAttHalf = kAttChunk / 2;
+template <int BITS, int NQ>
+__global__ void __launch_bounds__(kAttChunk, NQ == 4 ? 6 : 4) attend_values_kernel(const AttendJob *__restrict__ jobs) {
   const AttendJob &jb = jobs[blockIdx.z];
-  if (jb.v.bits != BITS) return;
+  if (jb.v.bits != BITS || BITS == 0) return;
   const int h = blockIdx.y, chunk = blockIdx.x, n_chunks = gridDim.x;
   if (h >= jb.m || chunk * kAttChunk >= jb.T) return;
+  constexpr int NB = BITS > 0 ? BITS : 1;
   extern __shared__ unsigned char att_smem[];
-  float *ps = (float *)att_smem;                                        // [kAttChunk][NQP]
-  uint32_t *cw = (uint32_t *)(ps + kAttChunk * NQP);                    // [kAttChunk][4 * BITS]
-  __half *cs = (__half *)(cw + kAttChunk * 4 * (BITS > 0 ? BITS : 1));  // [kAttChunk][4]
-  float *part = (float *)(cs + kAttChunk * 4);                          // [4][128][NQP] slice sums
-  const int tid = threadIdx.x, t0 = chunk * kAttChunk;
-  const int nt = min(kAttChunk, jb.T - t0);
-  {
-    const float4 *src = (const float4 *)(jb.p + ((size_t)h * jb.T + t0) * NQP);
-    for (int i = tid; i < nt * NQP / 4; i += kAttChunk) ((float4 *)ps)[i] = src[i];
-    for (int i = nt * NQP / 4 + tid; i < kAttChunk * NQP / 4; i += kAttChunk) ((float4 *)ps)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if constexpr (BITS > 0) {
-      const uint4 *wsrc = (const uint4 *)(jb.v.words + ((size_t)h * jb.T + t0) * (4 * BITS));
-      for (int i = tid; i < nt * BITS; i += kAttChunk) ((uint4 *)cw)[i] = __ldg(wsrc + i);
+  float *ps = (float *)att_smem;                                        // [128][NQ]
+  uint32_t *cw = (uint32_t *)(ps + kAttHalf * NQ);                      // [128][4 * BITS]
+  __half *cs = (__half *)(cw + kAttHalf * 4 * NB);                      // [128][4]
+  float *part = (float *)(cs + kAttHalf * 4);                           // [4][128][NQ] slice sums
+  const int tid = threadIdx.x;
+  // residual: thread = (four neighbouring features, one of eight 16-token slices of the staged half): one word, one scale
+  // and one weight load serve four codes; sum_t p_t Delta_t (u_tf - 2^(b-1) + 1/2)
+  const int fq = tid & 31, sl = tid >> 5;
+  const int f0 = fq * 4, g = f0 >> 5, bit = (f0 & 31) * NB, wi = g * NB + (bit >> 5), sh = bit & 31;
+  const bool straddle = NB == 3 && sh + 4 * NB > 32;           // only 3-bit codes cross a word inside a quad
+  constexpr uint32_t mask = (1u << NB) - 1u;
+  constexpr float off = 8388608.0f + (float)(1 << (NB - 1));
+  float acc[4][NQ];
+#pragma unroll
+  for (int c = 0; c < 4; ++c)
+#pragma unroll
+    for (int i = 0; i < NQ; ++i) acc[c][i] = 0.f;
+  for (int hf = 0; hf < 2; ++hf) {
+    const int t0 = chunk * kAttChunk + hf * kAttHalf;
+    if (t0 >= jb.T) break;                              // T is a multiple of 128: a half is all in or all out
+    if (hf) __syncthreads();                            // the first half has been read
+    {
+      const float4 *src = (const float4 *)(jb.p + ((size_t)h * jb.T + t0) * NQ);
+      for (int i = tid; i < kAttHalf * NQ / 4; i += kAttChunk) ((float4 *)ps)[i] = src[i];
+      const uint4 *wsrc = (const uint4 *)(jb.v.words + ((size_t)h * jb.T + t0) * (4 * NB));
+      for (int i = tid; i < kAttHalf * NB; i += kAttChunk) ((uint4 *)cw)[i] = __ldg(wsrc + i);
       const uint2 *ssrc = (const uint2 *)(jb.v.scales + ((size_t)h * jb.T + t0) * 4);
-      for (int i = tid; i < nt; i += kAttChunk) ((uint2 *)cs)[i] = __ldg(ssrc + i);
+      for (int i = tid; i < kAttHalf; i += kAttChunk) ((uint2 *)cs)[i] = __ldg(ssrc + i);
     }
-  }
-  __syncthreads();
-  // residual: thread = (four neighbouring features, one of eight 32-token slices): one word, one scale and one weight
-  // load serve four codes; sum_t p_t Delta_t (u_tf - 2^(b-1) + 1/2)
-  if constexpr (BITS > 0) {
-    const int fq = tid & 31, sl = tid >> 5;
-    const int f0 = fq * 4, g = f0 >> 5, bit = (f0 & 31) * BITS, wi = g * BITS + (bit >> 5), sh = bit & 31;
-    const bool straddle = BITS == 3 && sh + 4 * BITS > 32;           // only 3-bit codes cross a word inside a quad
-    constexpr uint32_t mask = (1u << BITS) - 1u;
-    constexpr float off = 8388608.0f + (float)(1 << (BITS - 1));
-    float acc[4][kAttMaxQ];
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-#pragma unroll
-      for (int i = 0; i < kAttMaxQ; ++i) acc[c][i] = 0.f;
-    const bool q8 = NQP == 8;
-    const int tb = sl * 32, te = min(tb + 32, nt);
+    __syncthreads();
+    const int tb = sl * 16;
 #pragma unroll 4
-    for (int t = tb; t < te; ++t) {
-      const uint32_t *row = cw + t * (4 * BITS);
+    for (int t = tb; t < tb + 16; ++t) {
+      const uint32_t *row = cw + t * (4 * NB);
       uint32_t u4 = row[wi] >> sh;
       if (straddle) u4 |= row[wi + 1] << (32 - sh);
       const float delta = __half2float(cs[t * 4 + g]), hd = 0.5f * delta;
-      const float4 p0 = *(const float4 *)(ps + t * NQP);
-      float4 p1 = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (q8) p1 = *(const float4 *)(ps + t * NQP + 4);
+      float pv[NQ];
+#pragma unroll
+      for (int q4 = 0; q4 < NQ; q4 += 4) {
+        const float4 p4 = *(const float4 *)(ps + t * NQ + q4);
+        pv[q4] = p4.x; pv[q4 + 1] = p4.y; pv[q4 + 2] = p4.z; pv[q4 + 3] = p4.w;
+      }
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        const float val = fmaf(__uint_as_float(0x4B000000u | ((u4 >> (c * BITS)) & mask)) - off, delta, hd);
-        acc[c][0] = fmaf(p0.x, val, acc[c][0]); acc[c][1] = fmaf(p0.y, val, acc[c][1]);
-        acc[c][2] = fmaf(p0.z, val, acc[c][2]); acc[c][3] = fmaf(p0.w, val, acc[c][3]);
-        if (q8) {
-          acc[c][4] = fmaf(p1.x, val, acc[c][4]); acc[c][5] = fmaf(p1.y, val, acc[c][5]);
-          acc[c][6] = fmaf(p1.z, val, acc[c][6]); acc[c][7] = fmaf(p1.w, val, acc[c][7]);
-        }
+        // integer code to float without a conversion instruction: 2^23 + u, minus (2^23 + 2^(b-1)); then Delta (u - 2^(b-1) + 1/2)
+        const float val = fmaf(__uint_as_float(0x4B000000u | ((u4 >> (c * NB)) & mask)) - off, delta, hd);
+#pragma unroll
+        for (int i = 0; i < NQ; ++i) acc[c][i] = fmaf(pv[i], val, acc[c][i]);
       }
     }
-    // sum over the eight slices: 7..4 -> 3..0, 3..2 -> 1..0, 1 -> 0 through part[4][128][NQP]
+  }
+  // sum over the eight slices: 7..4 -> 3..0, 3..2 -> 1..0, 1 -> 0 through part[4][128][NQ]
 #pragma unroll
-    for (int stride = 4; stride >= 1; stride >>= 1) {
-      if (sl >= stride && sl < 2 * stride) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int i = 0; i < kAttMaxQ; ++i)
-            if (i < NQP) part[((sl - stride) * 128 + f0 + c) * NQP + i] = acc[c][i];
-      }
-      __syncthreads();
-      if (sl < stride) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int i = 0; i < kAttMaxQ; ++i)
-            if (i < NQP) acc[c][i] += part[(sl * 128 + f0 + c) * NQP + i];
-      }
-      __syncthreads();
-    }
-    if (sl == 0) {
-      float *ap = jb.a + (((size_t)h * n_chunks + chunk) * 128 + f0) * NQP;
+  for (int stride = 4; stride >= 1; stride >>= 1) {
+    if (sl >= stride && sl < 2 * stride) {
 #pragma unroll
       for (int c = 0; c < 4; ++c)
 #pragma unroll
-        for (int i = 0; i < kAttMaxQ; ++i)
-          if (i < NQP) ap[c * NQP + i] = acc[c][i];
+        for (int i = 0; i < NQ; ++i) part[((sl - stride) * 128 + f0 + c) * NQ + i] = acc[c][i];
     }
+    __syncthreads();
+    if (sl < stride) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int i = 0; i < NQ; ++i) acc[c][i] += part[(sl * 128 + f0 + c) * NQ + i];
+    }
+    __syncthreads();
+  }
+  if (sl == 0) {
+    float *ap = jb.a + (((size_t)h * n_chunks + chunk) * 128 + f0) * NQ;
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int i = 0; i < NQ; ++i) ap[c * NQ + i] = acc[c][i];
   }
 }
 

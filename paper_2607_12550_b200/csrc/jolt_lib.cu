@@ -1514,10 +1514,10 @@ static void launch_att_scores_mma(dim3 grid, cudaStream_t s, const AttendJob *d,
   attend_scores_mma_kernel<BITS><<<grid, kAttChunk, 0, s>>>(d, NQP, n_chunks);
 }
 template <int BITS>
-static void launch_att_values(dim3 grid, size_t shm, cudaStream_t s, const AttendJob *d, int NQP) {
-  static std::atomic<bool> opted{false};      // up to 58 KB of dynamic shared memory (8-bit codes, 8 queries)
-  if (!opted.exchange(true)) cudaFuncSetAttribute(attend_values_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-  attend_values_kernel<BITS><<<grid, kAttChunk, shm, s>>>(d, NQP);
+static void launch_att_values(dim3 grid, cudaStream_t s, const AttendJob *d, int NQP) {
+  const size_t shm = (size_t)kAttHalf * (NQP * sizeof(float) + 16 * BITS + 8) + (size_t)4 * 128 * NQP * sizeof(float);
+  if (NQP == 4) attend_values_kernel<BITS, 4><<<grid, kAttChunk, shm, s>>>(d);
+  else attend_values_kernel<BITS, 8><<<grid, kAttChunk, shm, s>>>(d);
 }
 
 extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, double scale, void *dOut, void *stream) {
@@ -1631,16 +1631,14 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
       }
       LAUNCHED();
     }
-    for (int b = 0; b <= 8; ++b) {
+    for (int b = 1; b <= 8; ++b) {                 // b = 0: no residual, nothing to stream
       if (!((vbits >> b) & 1)) continue;
-      const size_t shm = (size_t)kAttChunk * (NQP * sizeof(float) + 16 * std::max(b, 1) + 8) + (size_t)4 * 128 * NQP * sizeof(float);
       switch (b) {
-        case 0: launch_att_values<0>(grid, shm, s, d, NQP); break;
-        case 1: launch_att_values<1>(grid, shm, s, d, NQP); break;
-        case 2: launch_att_values<2>(grid, shm, s, d, NQP); break;
-        case 3: launch_att_values<3>(grid, shm, s, d, NQP); break;
-        case 4: launch_att_values<4>(grid, shm, s, d, NQP); break;
-        default: launch_att_values<8>(grid, shm, s, d, NQP); break;
+        case 1: launch_att_values<1>(grid, s, d, NQP); break;
+        case 2: launch_att_values<2>(grid, s, d, NQP); break;
+        case 3: launch_att_values<3>(grid, s, d, NQP); break;
+        case 4: launch_att_values<4>(grid, s, d, NQP); break;
+        default: launch_att_values<8>(grid, s, d, NQP); break;
       }
       LAUNCHED();
     }
