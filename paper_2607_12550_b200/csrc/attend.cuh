@@ -50,7 +50,8 @@ struct AttendJob {                  // one per layer group
   const float *q;                   // [m][n_q][128]
   float *out;                       // [m][n_q][128]
   __half *kP, *vP;                  // [m * r_t][128]    P_h = fp16(G_h U_F^T) of the key / value cell (scaled units)
-  float *w;                         // [m][k.r_t][NQP]   scale 2^e P_h q
+  __half *wh, *wl;                  // [m NQP][k.r_t]    P_h q times 2^-E_n per column n = (head, query), as hi + lo fp16
+  float *we;                        // [m NQP]           scale 2^e 2^E_n
   float *qt;                        // [m][128][NQP]     scale H(s . q) / sqrt(d)
   __half *qh, *ql;                  // [m][8][128]       the same, times 2^-E per (head, query), as hi + lo fp16 (MMA operand)
   float *qe;                        // [m][8]            2^E
@@ -153,14 +154,33 @@ __global__ void __launch_bounds__(128) attend_prep_kernel(const AttendJob *__res
     if (f == 0) jb.qe[h * kAttMaxQ + i] = ldexpf(1.f, ex - 13);
   }
   if (jb.k.r_t > 0) {
-    // w[k][q] = scale 2^e sum_f P_h[k][f] q_q[f]: a warp per row k, a lane per four features
+    // w[n][k] = sum_f P_h[k][f] q[f] for column n = (head, query): a warp per row k, a lane per four features.  Stored as
+    // hi + lo fp16 times 2^-E_n with 2^E_n > |q|_2: a row of P_h has norm below 2^14.52 (|G| 2^-e < 2^11, r_f <= 128, U_F
+    // orthonormal, fp16 rounding), so every scaled entry is below 2^14.52 in magnitude and fits fp16.
     const float se = scale * ldexpf(1.f, *jb.k.e);
     const int warp = f >> 5, lane = f & 31;
     float q[kAttMaxQ][4];
+    int ex[kAttMaxQ];
+    float inv[kAttMaxQ];
 #pragma unroll
     for (int c = 0; c < kAttMaxQ; ++c) {
       const float4 v = c < n_q ? *(const float4 *)(jb.q + ((size_t)h * n_q + c) * 128 + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
       q[c][0] = v.x; q[c][1] = v.y; q[c][2] = v.z; q[c][3] = v.w;
+      float sq = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, v.w * v.w)));
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      const float nrm = sqrtf(sq);
+      ex[c] = 0;
+      if (nrm > 0.f && nrm < INFINITY) frexpf(nrm, &ex[c]);              // |q|_2 < 2^ex
+      ++ex[c];                                                          // headroom for the rounding of the norm itself
+      inv[c] = ldexpf(1.f, -ex[c]);
+    }
+    if (blockIdx.z == 0 && f < NQP) {
+      int e_f = 0;
+#pragma unroll
+      for (int c = 0; c < kAttMaxQ; ++c)
+        if (c == f) e_f = ex[c];
+      jb.we[h * NQP + f] = se * ldexpf(1.f, e_f);
     }
     for (int k = warp + 4 * blockIdx.z; k < jb.k.r_t; k += 4 * gridDim.z) {
       const uint2 p4 = __ldg((const uint2 *)(jb.kP + ((size_t)h * jb.k.r_t + k) * 128 + lane * 4));
@@ -173,9 +193,16 @@ __global__ void __launch_bounds__(128) attend_prep_kernel(const AttendJob *__res
       for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
         for (int c = 0; c < kAttMaxQ; ++c) v[c] += __shfl_xor_sync(0xffffffffu, v[c], o);
+      // lane c stores column c (every lane holds all the sums)
+      float sv = 0.f;
 #pragma unroll
       for (int c = 0; c < kAttMaxQ; ++c)
-        if (lane == 0 && c < NQP) jb.w[((size_t)h * jb.k.r_t + k) * NQP + c] = se * v[c];
+        if (c == lane) sv = v[c] * inv[c];
+      if (lane < NQP) {
+        const __half hi = __float2half_rn(sv);
+        jb.wh[((size_t)h * NQP + lane) * jb.k.r_t + k] = hi;
+        jb.wl[((size_t)h * NQP + lane) * jb.k.r_t + k] = __float2half_rn(sv - __half2float(hi));
+      }
     }
   }
 }
@@ -579,32 +606,20 @@ __global__ void __launch_bounds__(kAttChunk, NQ == 4 ? 6 : 4) attend_values_kern
 // whole cell instead of a loop per head:  with n = (head, query),
 //   attend_bscore_kernel   S_b[t][n] = sum_k U_T[t][k] w[n][k]            written to the weight buffer p[h][t][i]
 //   attend_bvalue_kernel   y[chunk][n][k] = sum_{t in chunk} p[n][t] U_T[t][k]
-// Both run on the tensor cores as warp-level MMAs with fp32 accumulation, the fp32 operand entering as hi + lo:
-// the first as m16n8k8 TF32 (an fp16 entry of U_T is exact in TF32; w has no bounded range, hi = its top 19 bits, lo = the
-// remainder, about 21 bits kept), the second as m16n8k16 fp16 (p lies in [0, 1]).  0.13 GFLOP per cell each with
-// N = 128: too small to set up TMEM-resident tcgen05 tiles for.
-__device__ __forceinline__ void att_mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t att_tf32_hi(float x) { return __float_as_uint(x) & 0xFFFFE000u; }
-__device__ __forceinline__ uint32_t att_tf32_lo(float x) { return __float_as_uint(x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u)); }
-// half number c (0..7) of eight packed halves, as the bits of the equal float
-__device__ __forceinline__ uint32_t att_half_of(const uint4 &u, int c) {
-  const uint32_t w = (c & 4) ? ((c & 2) ? u.w : u.z) : ((c & 2) ? u.y : u.x);
-  return __float_as_uint(__half2float(__ushort_as_half((unsigned short)((c & 1) ? (w >> 16) : (w & 0xFFFFu)))));
-}
-
+// Both run on the tensor cores as warp-level m16n8k16 fp16 MMAs with fp32 accumulation: U_T is fp16 as stored, the
+// fp32 operand enters as hi + lo fp16 (22 bits) -- p lies in [0, 1]; w is scaled per column by a power of two bounded
+// through |q|_2 (see attend_prep_kernel).  0.13 GFLOP per cell each with N = 128: too small to set up TMEM-resident
+// tcgen05 tiles for.  (A TF32 m16n8k8 form of the first product ran at the CUDA-core FMA rate and was replaced.)
 constexpr int kAttBPitch = 136;     // floats per staged operand row: 8 c + g addresses all 32 banks
 
 // grid (ceil(T / 64), ceil(m NQP / 128), groups), 256 threads: warp w owns 16 tokens (w & 3) x 64 columns n (w >> 2).
-// The operands of the next 32-wide k chunk are requested into registers before the MMAs of the current one.
-__global__ void __launch_bounds__(256) attend_bscore_kernel(const AttendJob *__restrict__ jobs, int NQP) {
+// m16n8k16 fp16 MMAs: A = U_T as stored, B = the scaled w as hi + lo.  The operands of the next 32-wide k chunk are
+// requested into registers before the MMAs of the current one.
+__global__ void __launch_bounds__(256, 2) attend_bscore_kernel(const AttendJob *__restrict__ jobs, int NQP) {
   const AttendJob &jb = jobs[blockIdx.z];
   const int r_t = jb.k.r_t, N = jb.m * NQP, n0 = blockIdx.y * 128, t0 = blockIdx.x * 64;
   if (r_t == 0 || n0 >= N || t0 >= jb.T) return;
-  __shared__ __align__(16) uint32_t Bh[32][kAttBPitch], Bl[32][kAttBPitch];       // w chunk, hi and lo, [k][n]
+  __shared__ __align__(16) uint32_t Bh[16][kAttBPitch], Bl[16][kAttBPitch];       // w chunk as k pairs, hi and lo, [k / 2][n]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
   const int wt = warp & 3, wn = warp >> 2;
   float acc[8][4];
@@ -614,14 +629,15 @@ __global__ void __launch_bounds__(256) attend_bscore_kernel(const AttendJob *__r
     for (int j = 0; j < 4; ++j) acc[nt][j] = 0.f;
   const int ta = min(t0 + wt * 16 + g, jb.T - 1), tb = min(t0 + wt * 16 + g + 8, jb.T - 1);   // rows past the end repeat the last
   const __half *rowa = jb.k.UT + (size_t)ta * r_t, *rowb = jb.k.UT + (size_t)tb * r_t;
-  float4 breg[4];
+  // staging items of a chunk: (hi | lo, column n, block of eight k) -> 2 * 128 * 4 = 1024, four per thread
+  uint4 breg[4];
   uint4 areg[4][2];
   auto load_chunk = [&](int k0) {
 #pragma unroll
     for (int it = 0; it < 4; ++it) {
-      const int idx = tid + it * 256, kk = idx >> 5, q4 = idx & 31, n = n0 + q4 * 4;
-      breg[it] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (n < N && k0 + kk < r_t) breg[it] = *(const float4 *)(jb.w + ((size_t)(n / NQP) * r_t + k0 + kk) * NQP + n % NQP);
+      const int idx = tid + it * 256, hl = idx >> 9, nn = (idx >> 2) & 127, kb8 = (idx & 3) * 8, n = n0 + nn;
+      breg[it] = make_uint4(0u, 0u, 0u, 0u);
+      if (n < N && k0 + kb8 < r_t) breg[it] = *(const uint4 *)((hl ? jb.wl : jb.wh) + (size_t)n * r_t + k0 + kb8);
     }
 #pragma unroll
     for (int k8 = 0; k8 < 4; ++k8) {
@@ -632,15 +648,15 @@ __global__ void __launch_bounds__(256) attend_bscore_kernel(const AttendJob *__r
       }
     }
   };
+  auto word_of = [](const uint4 &u, int w) { return (w & 2) ? ((w & 1) ? u.w : u.z) : ((w & 1) ? u.y : u.x); };
   load_chunk(0);
   for (int k0 = 0; k0 < r_t; k0 += 32) {
     __syncthreads();
 #pragma unroll
     for (int it = 0; it < 4; ++it) {
-      const int idx = tid + it * 256, kk = idx >> 5, q4 = idx & 31;
-      const float4 v = breg[it];
-      *(uint4 *)&Bh[kk][q4 * 4] = make_uint4(att_tf32_hi(v.x), att_tf32_hi(v.y), att_tf32_hi(v.z), att_tf32_hi(v.w));
-      *(uint4 *)&Bl[kk][q4 * 4] = make_uint4(att_tf32_lo(v.x), att_tf32_lo(v.y), att_tf32_lo(v.z), att_tf32_lo(v.w));
+      const int idx = tid + it * 256, hl = idx >> 9, nn = (idx >> 2) & 127, kp0 = (idx & 3) * 4;
+      uint32_t (*dst)[kAttBPitch] = hl ? Bl : Bh;
+      dst[kp0][nn] = breg[it].x; dst[kp0 + 1][nn] = breg[it].y; dst[kp0 + 2][nn] = breg[it].z; dst[kp0 + 3][nn] = breg[it].w;
     }
     uint4 acur[4][2];
 #pragma unroll
@@ -648,13 +664,14 @@ __global__ void __launch_bounds__(256) attend_bscore_kernel(const AttendJob *__r
     __syncthreads();
     if (k0 + 32 < r_t) load_chunk(k0 + 32);
 #pragma unroll
-    for (int k8 = 0; k8 < 4; ++k8) {
-      const uint32_t a[4] = {att_half_of(acur[k8][0], c), att_half_of(acur[k8][1], c), att_half_of(acur[k8][0], c + 4), att_half_of(acur[k8][1], c + 4)};
+    for (int s16 = 0; s16 < 2; ++s16) {
+      // A: rows g, g + 8; k = 16 s16 + 2c, +1 (word c of the first eight halves) and + 8 (word c of the next eight)
+      const uint32_t a[4] = {word_of(acur[2 * s16][0], c), word_of(acur[2 * s16][1], c), word_of(acur[2 * s16 + 1][0], c), word_of(acur[2 * s16 + 1][1], c)};
 #pragma unroll
       for (int nt = 0; nt < 8; ++nt) {
         const int col = wn * 64 + nt * 8 + g;
-        att_mma_tf32(acc[nt], a, Bh[k8 * 8 + c][col], Bh[k8 * 8 + c + 4][col]);
-        att_mma_tf32(acc[nt], a, Bl[k8 * 8 + c][col], Bl[k8 * 8 + c + 4][col]);
+        att_mma_f16(acc[nt], a, Bh[s16 * 8 + c][col], Bh[s16 * 8 + c + 4][col]);
+        att_mma_f16(acc[nt], a, Bl[s16 * 8 + c][col], Bl[s16 * 8 + c + 4][col]);
       }
     }
   }
@@ -663,9 +680,10 @@ __global__ void __launch_bounds__(256) attend_bscore_kernel(const AttendJob *__r
   for (int nt = 0; nt < 8; ++nt) {
     const int n = n0 + wn * 64 + nt * 8 + 2 * c;
     if (n >= N) continue;
+    const float2 we = *(const float2 *)(jb.we + n);
     const size_t col = (size_t)(n / NQP) * jb.T * NQP + n % NQP;
-    if (t_lo < jb.T) *(float2 *)(jb.p + col + (size_t)t_lo * NQP) = make_float2(acc[nt][0], acc[nt][1]);
-    if (t_hi < jb.T) *(float2 *)(jb.p + col + (size_t)t_hi * NQP) = make_float2(acc[nt][2], acc[nt][3]);
+    if (t_lo < jb.T) *(float2 *)(jb.p + col + (size_t)t_lo * NQP) = make_float2(acc[nt][0] * we.x, acc[nt][1] * we.y);
+    if (t_hi < jb.T) *(float2 *)(jb.p + col + (size_t)t_hi * NQP) = make_float2(acc[nt][2] * we.x, acc[nt][3] * we.y);
   }
 }
 

@@ -1582,7 +1582,9 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
       j.q = (const float *)dQ + row0; j.out = (float *)dOut + row0;
       j.kP = H->att_P + H->att_P_off[2 * g];
       j.vP = H->att_P + H->att_P_off[2 * g + 1];
-      j.w = b.take<float>((size_t)j.m * std::max(j.k.r_t, 1) * NQP);
+      j.wh = b.take<__half>((size_t)j.m * NQP * std::max(j.k.r_t, 8));
+      j.wl = b.take<__half>((size_t)j.m * NQP * std::max(j.k.r_t, 8));
+      j.we = b.take<float>((size_t)j.m * NQP);
       j.qt = b.take<float>((size_t)j.m * kD * NQP);
       j.qh = b.take<__half>((size_t)j.m * kAttMaxQ * kD);
       j.ql = b.take<__half>((size_t)j.m * kAttMaxQ * kD);
