@@ -359,7 +359,7 @@ __device__ __forceinline__ uint32_t att_pair_f16(uint32_t x, int bits) {
 }
 
 template <int BITS>
-__global__ void __launch_bounds__(kAttChunk, 3) attend_scores_mma_kernel(const AttendJob *__restrict__ jobs, int NQP, int n_chunks) {
+__global__ void __launch_bounds__(kAttChunk, BITS == 8 ? 2 : 3) attend_scores_mma_kernel(const AttendJob *__restrict__ jobs, int NQP, int n_chunks) {
   static_assert(BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8, "codes that do not straddle words");
   const AttendJob &jb = jobs[blockIdx.z];
   if (jb.k.bits != BITS) return;
