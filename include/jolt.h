@@ -151,7 +151,9 @@ int jolt_decompress_rope(const jolt_handle *h, const jolt_layout *out_layout, vo
  *   about 5 % of the compressed size on the benchmark workload) in a device buffer that stays with the handle
  *   until jolt_free; later calls, on any stream, reuse them.  Errors: JOLT_EINVAL
  *   (null / misaligned pointers, n_q out of range, wrong device), JOLT_EUNSUPPORTED (ranks that are not multiples
- *   of 8; sequences beyond about 300 k tokens), JOLT_ENOMEM, JOLT_ECUDA.  Asynchronous on `stream`. */
+ *   of 8; sequences beyond about 3 million tokens), JOLT_ENOMEM, JOLT_ECUDA.  Asynchronous on `stream`.  Arithmetic:
+ *   fp32; the contractions that run on the tensor cores take their fp32 operand as hi + lo fp16 (about 22 bits) and
+ *   accumulate in fp32. */
 int jolt_attend(const jolt_handle *h, const void *dQ, int32_t n_q, double scale, void *dOut, void *stream);
 
 /* jolt_decompress_static -- the paper has no counterpart; this is a deployment variant of jolt_decompress

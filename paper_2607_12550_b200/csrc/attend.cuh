@@ -11,18 +11,19 @@
 // so a call streams U_T and the packed codes once each (the compressed bytes) instead of the fp16 cache, and the
 // Hadamard rotation is applied to one query / one output row per head instead of every token.
 //
-// Seven kernels; the code streams are CUDA-core work (1..8-bit codes against a handful of query vectors), the two
-// backbone products warp-level tensor-core MMAs:
-//   attend_p16_kernel      P_h = fp16(G_h U_F^T) of every head of both cells (what the decoder's set-up also forms)
-//   attend_prep_kernel     per (group, head): rotated scaled queries and w = scale 2^e P_h q
+// Kernels of a call (the contractions with a tensor-core shape are warp-level fp16 MMAs with fp32 accumulation, an fp32
+// operand entering as hi + lo fp16; the rest is CUDA-core fp32):
+//   attend_p16_kernel      P_h = fp16(G_h U_F^T) of every head of both cells (what the decoder's set-up also forms);
+//                          first call on a handle only
+//   attend_prep_kernel     per (group, head, query): rotated scaled query (fp32, and scaled hi + lo fp16), w = P_h q
 //   attend_bscore_kernel   backbone scores U_T w of all heads of a cell as one dense product (U_T is shared by the heads)
 //   attend_scores_mma_kernel / attend_scores_kernel   per (group, head, 256-token chunk): residual scores added (codes
-//                          times rotated query: warp-level fp16 MMAs for 1-, 2-, 4- and 8-bit codes, CUDA cores for 3-bit
-//                          codes and for cells without a residual), chunk maximum, p = exp(s - max), chunk sum
+//                          times rotated query: MMAs for 1-, 2-, 4- and 8-bit codes, CUDA cores for 3-bit codes and for
+//                          cells without a residual), chunk maximum, p = exp(s - max), chunk sum
 //   attend_values_kernel   per (group, head, chunk): sum_t p_t r^'_t (codes staged in shared memory and read
 //                          feature-wise, so the token reduction stays inside a thread)
 //   attend_bvalue_kernel   p^T U_T per chunk for all heads of a cell as one dense product
-//   attend_combine_kernel  per (group, head): merges the chunks (running-maximum rescaling), applies P_h of the
+//   attend_combine_kernel  per (group, head, query): merges the chunks (running-maximum rescaling), applies P_h of the
 //                          value cell and the inverse rotation, divides by the softmax denominator
 // Keys compressed before a rotary embedding cannot use the first identity (the rotation differs per token).
 #pragma once
