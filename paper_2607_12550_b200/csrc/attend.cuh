@@ -603,6 +603,122 @@ __global__ void __launch_bounds__(kAttChunk, NQ == 4 ? 6 : 4) attend_values_kern
   }
 }
 
+// The value-side code stream on the tensor cores, for 1-, 2-, 4- and 8-bit codes:
+//     a[f][i] = sum_t (2 u_tf + 1 - 2^b) * (Delta_t,g(f) p_t,i / 2)
+// is a product with M = features, N = queries, K = tokens.  Per 128-token half of the chunk the CTA expands the packed
+// codes to an fp16 tile E[t][f] in shared memory (exact integers; 16-byte pieces swizzled by the token index so that both
+// the row-wise writes and the transposed 8 x 8 fragment loads are conflict-free), writes the weights times the steps,
+// scaled by one power of two per half so that fp16 holds them, as hi + lo fp16 W[g][i][t], and then every warp owns 16
+// features: one transposed ldmatrix.x4 and two MMAs per 16 tokens.  No reduction between warps.
+// grid (n_chunks, m, groups), kAttChunk threads.  Dynamic shared memory: 32 KB + 4 * 2 * NQ * 136 halves.
+__device__ __forceinline__ void att_ldmatrix_x4_trans(uint32_t (&r)[4], const void *smem_row) {
+  const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_row);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+template <int BITS, int NQ>
+__global__ void __launch_bounds__(kAttChunk, 4) attend_values_mma_kernel(const AttendJob *__restrict__ jobs) {
+  static_assert(BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8, "codes that do not straddle words");
+  const AttendJob &jb = jobs[blockIdx.z];
+  if (jb.v.bits != BITS) return;
+  const int h = blockIdx.y, chunk = blockIdx.x, n_chunks = gridDim.x;
+  if (h >= jb.m || chunk * kAttChunk >= jb.T) return;
+  extern __shared__ unsigned char att_smem[];
+  typedef __half ERow[128];
+  typedef __half WBlk[2][NQ][kAttHalf + 8];
+  ERow *E = (ERow *)att_smem;                                   // [128 tokens][128 f], swizzled: piece j of row t sits at j ^ (t & 7)
+  WBlk *W = (WBlk *)(att_smem + sizeof(ERow) * kAttHalf);       // [group][hi | lo][query][token]
+  __shared__ float dmax[kAttChunk / 32];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
+  const int row = tid >> 1, hh = tid & 1;              // staging: token row of the half, feature half (groups 2 hh, 2 hh + 1)
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int hf = 0; hf < 2; ++hf) {
+    const int t0 = chunk * kAttChunk + hf * kAttHalf;
+    if (t0 >= jb.T) break;                             // T is a multiple of 128: a half is all in or all out
+    const size_t grow = (size_t)h * jb.T + t0 + row;
+    uint32_t wd[2 * BITS];
+    {
+      const uint32_t *wp = jb.v.words + grow * (4 * BITS) + hh * 2 * BITS;
+      if constexpr (BITS >= 2) {
+#pragma unroll
+        for (int i = 0; i < 2 * BITS / 4; ++i) { const uint4 v = __ldg((const uint4 *)wp + i); wd[4 * i] = v.x; wd[4 * i + 1] = v.y; wd[4 * i + 2] = v.z; wd[4 * i + 3] = v.w; }
+      } else {
+        const uint2 v = __ldg((const uint2 *)wp); wd[0] = v.x; wd[1] = v.y;
+      }
+    }
+    const uint32_t sc2 = __ldg((const uint32_t *)(jb.v.scales + grow * 4) + hh);       // steps of groups 2 hh, 2 hh + 1
+    const float d0 = __half2float(__ushort_as_half((unsigned short)(sc2 & 0xFFFFu))), d1 = __half2float(__ushort_as_half((unsigned short)(sc2 >> 16)));
+    float pv[NQ];
+#pragma unroll
+    for (int q4 = 0; q4 < NQ; q4 += 4) {
+      const float4 p4 = *(const float4 *)(jb.p + grow * NQ + q4);
+      pv[q4] = p4.x; pv[q4 + 1] = p4.y; pv[q4 + 2] = p4.z; pv[q4 + 3] = p4.w;
+    }
+    // one power of two per half so that step * weight / 2 fits fp16: largest step of the half -> below 2^14
+    float mx = fmaxf(d0, d1);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (hf) __syncthreads();                           // the previous half's tiles have been read
+    if (lane == 0) dmax[warp] = mx;
+    // codes -> E: group gl of this thread, 32 codes = 16 half2 words = four 16-byte pieces
+#pragma unroll
+    for (int gl = 0; gl < 2; ++gl) {
+#pragma unroll
+      for (int pc = 0; pc < 4; ++pc) {
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int pp = pc * 4 + j, bit = 2 * pp * BITS;             // pair pp of the group
+          o[j] = att_pair_f16(wd[gl * BITS + (bit >> 5)] >> (bit & 31), BITS);
+        }
+        const int piece = hh * 8 + gl * 4 + pc;
+        *(uint4 *)&E[row][((piece ^ (row & 7)) << 3)] = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+    }
+    __syncthreads();
+    mx = dmax[0];
+#pragma unroll
+    for (int wq = 1; wq < kAttChunk / 32; ++wq) mx = fmaxf(mx, dmax[wq]);
+    int ex = 0;
+    if (mx > 0.f && mx < INFINITY) frexpf(mx, &ex);                    // mx < 2^ex
+    const float up = ldexpf(0.5f, 14 - ex), down = ldexpf(1.f, ex - 14);
+#pragma unroll
+    for (int gl = 0; gl < 2; ++gl) {
+      const float ds = (gl ? d1 : d0) * up;
+#pragma unroll
+      for (int i = 0; i < NQ; ++i) {
+        const float x = ds * pv[i];
+        const __half hi = __float2half_rn(x);
+        W[hh * 2 + gl][0][i][row] = hi;
+        W[hh * 2 + gl][1][i][row] = __float2half_rn(x - __half2float(hi));
+      }
+    }
+    __syncthreads();
+    // warp = features 16 warp .. +15 (group warp >> 1); 8 steps of 16 tokens
+    float d[4] = {0.f, 0.f, 0.f, 0.f};
+    const int mi = lane >> 3, r8 = lane & 7, tb8 = mi >> 1, fb = mi & 1;
+    const bool have = g < NQ;                           // query columns beyond NQ are zero
+    const uint32_t *wh = (const uint32_t *)&W[warp >> 1][0][have ? g : 0][0], *wl = (const uint32_t *)&W[warp >> 1][1][have ? g : 0][0];
+#pragma unroll
+    for (int s16 = 0; s16 < kAttHalf / 16; ++s16) {
+      uint32_t a[4];
+      const int tr = s16 * 16 + tb8 * 8 + r8;
+      att_ldmatrix_x4_trans(a, &E[tr][(((2 * warp + fb) ^ (tr & 7)) << 3)]);
+      // ldmatrix order: (tokens 0-7, f 0-7), (tokens 0-7, f 8-15), (tokens 8-15, f 0-7), (tokens 8-15, f 8-15) = a0, a1, a2, a3
+      att_mma_f16(d, a, have ? wh[s16 * 8 + c] : 0u, have ? wh[s16 * 8 + c + 4] : 0u);
+      att_mma_f16(d, a, have ? wl[s16 * 8 + c] : 0u, have ? wl[s16 * 8 + c + 4] : 0u);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[j] = fmaf(d[j], down, acc[j]);
+  }
+  if (2 * c < NQ) {
+    float *ap = jb.a + (((size_t)h * n_chunks + chunk) * 128 + warp * 16 + g) * NQ + 2 * c;
+    *(float2 *)ap = make_float2(acc[0], acc[1]);
+    *(float2 *)(ap + 8 * NQ) = make_float2(acc[2], acc[3]);
+  }
+}
+
 // The backbone terms are shared by all heads of a cell (one U_T per cell), so they are two small dense products over the
 // whole cell instead of a loop per head:  with n = (head, query),
 //   attend_bscore_kernel   S_b[t][n] = sum_k U_T[t][k] w[n][k]            written to the weight buffer p[h][t][i]

@@ -1514,6 +1514,17 @@ static void launch_att_scores_mma(dim3 grid, cudaStream_t s, const AttendJob *d,
   attend_scores_mma_kernel<BITS><<<grid, kAttChunk, 0, s>>>(d, NQP, n_chunks);
 }
 template <int BITS>
+static void launch_att_values_mma(dim3 grid, cudaStream_t s, const AttendJob *d, int NQP) {
+  const size_t shm = (size_t)kAttHalf * 128 * sizeof(__half) + (size_t)4 * 2 * NQP * (kAttHalf + 8) * sizeof(__half);
+  static std::atomic<bool> opted{false};      // 49.4 KB with eight query slots
+  if (!opted.exchange(true)) {
+    cudaFuncSetAttribute(attend_values_mma_kernel<BITS, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    cudaFuncSetAttribute(attend_values_mma_kernel<BITS, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+  }
+  if (NQP == 4) attend_values_mma_kernel<BITS, 4><<<grid, kAttChunk, shm, s>>>(d);
+  else attend_values_mma_kernel<BITS, 8><<<grid, kAttChunk, shm, s>>>(d);
+}
+template <int BITS>
 static void launch_att_values(dim3 grid, cudaStream_t s, const AttendJob *d, int NQP) {
   const size_t shm = (size_t)kAttHalf * (NQP * sizeof(float) + 16 * BITS + 8) + (size_t)4 * 128 * NQP * sizeof(float);
   if (NQP == 4) attend_values_kernel<BITS, 4><<<grid, kAttChunk, shm, s>>>(d);
@@ -1602,6 +1613,7 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
   const float fscale = (float)scale;
   cudaEvent_t att_ready = H->att_ready;
   const bool mma = (g_fast.load() & 1) != 0;        // warp-MMA form of the score kernel (the CUDA-core form stays as the portable path)
+  const bool vmma = mma && !getenv("JOLT_ATT_VSIMT");
   P.add(ST_ATT, [=](char *dev_t, cudaStream_t s) {
     const AttendJob *d = (const AttendJob *)(dev_t + off);
     if (first_call) {
@@ -1636,11 +1648,11 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
     for (int b = 1; b <= 8; ++b) {                 // b = 0: no residual, nothing to stream
       if (!((vbits >> b) & 1)) continue;
       switch (b) {
-        case 1: launch_att_values<1>(grid, s, d, NQP); break;
-        case 2: launch_att_values<2>(grid, s, d, NQP); break;
+        case 1: if (vmma) launch_att_values_mma<1>(grid, s, d, NQP); else launch_att_values<1>(grid, s, d, NQP); break;
+        case 2: if (vmma) launch_att_values_mma<2>(grid, s, d, NQP); else launch_att_values<2>(grid, s, d, NQP); break;
         case 3: launch_att_values<3>(grid, s, d, NQP); break;
-        case 4: launch_att_values<4>(grid, s, d, NQP); break;
-        default: launch_att_values<8>(grid, s, d, NQP); break;
+        case 4: if (vmma) launch_att_values_mma<4>(grid, s, d, NQP); else launch_att_values<4>(grid, s, d, NQP); break;
+        default: if (vmma) launch_att_values_mma<8>(grid, s, d, NQP); else launch_att_values<8>(grid, s, d, NQP); break;
       }
       LAUNCHED();
     }
