@@ -1612,8 +1612,8 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
   const uint64_t seed = H->seed;
   const float fscale = (float)scale;
   cudaEvent_t att_ready = H->att_ready;
-  const bool mma = (g_fast.load() & 1) != 0;        // warp-MMA form of the score kernel (the CUDA-core form stays as the portable path)
-  const bool vmma = mma && !getenv("JOLT_ATT_VSIMT");
+  const bool mma = (g_fast.load() & 1) != 0;        // warp-MMA forms of the two code streams (the CUDA-core forms stay as the portable path)
+  const bool vmma = mma;
   P.add(ST_ATT, [=](char *dev_t, cudaStream_t s) {
     const AttendJob *d = (const AttendJob *)(dev_t + off);
     if (first_call) {

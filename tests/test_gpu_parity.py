@@ -516,6 +516,14 @@ def test_attend_on_the_factors(B, synth, case):
     Q[1, 1, n_q - 1] = 0.0                 # one uniform row
     scale = 1.0 / 128 ** 0.5
     out = B.jolt_attend(h, Q.cuda(), scale)
+    # the CUDA-core forms of the two code streams (fast-path bit 0 off) agree with the tensor-core forms
+    prev = B.set_fast_path(14)
+    try:
+        out_cc = B.jolt_attend(h, Q.cuda(), scale)
+        torch.cuda.synchronize()
+    finally:
+        B.set_fast_path(prev)
+    assert float((out_cc - out).norm() / out.norm()) <= 1e-5
     # the same attention over the library's own fp32 decode (a second CUDA path: consistency, not parity)
     Kd, Vd = torch.empty(K.shape, dtype=torch.float32, device="cuda"), torch.empty(V.shape, dtype=torch.float32, device="cuda")
     B.jolt_decompress(h, Kd, Vd, gs)
