@@ -637,14 +637,15 @@ __global__ void __launch_bounds__(kAttChunk, 4) attend_values_mma_kernel(const A
     const int t0 = chunk * kAttChunk + hf * kAttHalf;
     if (t0 >= jb.T) break;                             // T is a multiple of 128: a half is all in or all out
     const size_t grow = (size_t)h * jb.T + t0 + row;
-    uint32_t wd[2 * BITS];
+    // packed codes of the half: 128 * BITS pieces of 16 bytes, consecutive threads take consecutive pieces (coalesced)
+    constexpr int NIT = (kAttHalf * BITS + kAttChunk - 1) / kAttChunk;
+    uint4 cw[NIT];
     {
-      const uint32_t *wp = jb.v.words + grow * (4 * BITS) + hh * 2 * BITS;
-      if constexpr (BITS >= 2) {
+      const uint4 *src = (const uint4 *)(jb.v.words + ((size_t)h * jb.T + t0) * (4 * BITS));
 #pragma unroll
-        for (int i = 0; i < 2 * BITS / 4; ++i) { const uint4 v = __ldg((const uint4 *)wp + i); wd[4 * i] = v.x; wd[4 * i + 1] = v.y; wd[4 * i + 2] = v.z; wd[4 * i + 3] = v.w; }
-      } else {
-        const uint2 v = __ldg((const uint2 *)wp); wd[0] = v.x; wd[1] = v.y;
+      for (int it = 0; it < NIT; ++it) {
+        const int idx = tid + it * kAttChunk;
+        cw[it] = idx < kAttHalf * BITS ? __ldg(src + idx) : make_uint4(0u, 0u, 0u, 0u);
       }
     }
     const uint32_t sc2 = __ldg((const uint32_t *)(jb.v.scales + grow * 4) + hh);       // steps of groups 2 hh, 2 hh + 1
@@ -661,19 +662,24 @@ __global__ void __launch_bounds__(kAttChunk, 4) attend_values_mma_kernel(const A
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if (hf) __syncthreads();                           // the previous half's tiles have been read
     if (lane == 0) dmax[warp] = mx;
-    // codes -> E: group gl of this thread, 32 codes = 16 half2 words = four 16-byte pieces
+    // codes -> E: a 16-byte piece of a packed row holds 128 / BITS codes = 16 / BITS output pieces of eight fp16 values
 #pragma unroll
-    for (int gl = 0; gl < 2; ++gl) {
+    for (int it = 0; it < NIT; ++it) {
+      const int idx = tid + it * kAttChunk;
+      if (idx < kAttHalf * BITS) {
+        const int er = idx / BITS, seg = idx % BITS;
+        const uint32_t w4[4] = {cw[it].x, cw[it].y, cw[it].z, cw[it].w};
 #pragma unroll
-      for (int pc = 0; pc < 4; ++pc) {
-        uint32_t o[4];
+        for (int pc = 0; pc < 16 / BITS; ++pc) {
+          uint32_t o[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int pp = pc * 4 + j, bit = 2 * pp * BITS;             // pair pp of the group
-          o[j] = att_pair_f16(wd[gl * BITS + (bit >> 5)] >> (bit & 31), BITS);
+          for (int j = 0; j < 4; ++j) {
+            const int bit = 2 * (pc * 4 + j) * BITS;                  // pair pc * 4 + j of this piece of the row's bit string
+            o[j] = att_pair_f16(w4[bit >> 5] >> (bit & 31), BITS);
+          }
+          const int piece = seg * (16 / BITS) + pc;
+          *(uint4 *)&E[er][((piece ^ (er & 7)) << 3)] = make_uint4(o[0], o[1], o[2], o[3]);
         }
-        const int piece = hh * 8 + gl * 4 + pc;
-        *(uint4 *)&E[row][((piece ^ (row & 7)) << 3)] = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
     __syncthreads();
