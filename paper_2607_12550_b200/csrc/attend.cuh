@@ -20,8 +20,9 @@
 //   attend_scores_mma_kernel / attend_scores_kernel   per (group, head, 256-token chunk): residual scores added (codes
 //                          times rotated query: MMAs for 1-, 2-, 4- and 8-bit codes, CUDA cores for 3-bit codes and for
 //                          cells without a residual), chunk maximum, p = exp(s - max), chunk sum
-//   attend_values_kernel   per (group, head, chunk): sum_t p_t r^'_t (codes staged in shared memory and read
-//                          feature-wise, so the token reduction stays inside a thread)
+//   attend_values_mma_kernel / attend_values_kernel   per (group, head, chunk): sum_t p_t r^'_t (MMAs with M = features,
+//                          K = tokens over an fp16 tile of expanded codes for 1-, 2-, 4- and 8-bit codes; CUDA cores,
+//                          codes staged in shared memory and read feature-wise, for 3-bit codes)
 //   attend_bvalue_kernel   p^T U_T per chunk for all heads of a cell as one dense product
 //   attend_combine_kernel  per (group, head, query): merges the chunks (running-maximum rescaling), applies P_h of the
 //                          value cell and the inverse rotation, divides by the softmax denominator
