@@ -175,6 +175,19 @@ int jolt_attend(const jolt_handle *h, const void *dQ, int32_t n_q, double scale,
 int jolt_decompress_static(const jolt_handle *h, const jolt_layout *out_layout, void *dK_out, void *dV_out,
                            void *stream);
 
+/* Persistence of a compressed cache (paper Sec. 7: the footprint that shrinks is "the persistent state ... what matters
+ * for prompt-caching deployments that keep many cached prefixes resident"; no format is given).  jolt_serialize writes a
+ * self-describing image -- header, layer grouping, cell descriptors, then the stored arrays exactly as they sit in device
+ * memory -- into host memory; jolt_deserialize maps such an image back into a new handle on the current device, with
+ * which jolt_decompress / jolt_attend give bit-identical results.  The image is tied to this library version and to the
+ * host's byte order.  host_dst / host_src: host pointers (pinned memory makes the copy asynchronous up to the final
+ * synchronisation; both calls return after the copy has finished).  Errors: JOLT_EINVAL (null pointers, a buffer
+ * smaller than jolt_serialized_bytes, an image that is truncated or fails its consistency checks), JOLT_ENOMEM,
+ * JOLT_ECUDA; on error *out is NULL. */
+int jolt_serialized_bytes(const jolt_handle *h, int64_t *bytes);
+int jolt_serialize(const jolt_handle *h, void *host_dst, int64_t cap, void *stream);
+int jolt_deserialize(const void *host_src, int64_t bytes, void *stream, jolt_handle **out);
+
 /* Release a handle and all buffers it owns.  NULL is accepted. */
 int jolt_free(jolt_handle *h);
 

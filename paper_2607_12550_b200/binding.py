@@ -63,6 +63,9 @@ class Rope(C.Structure):
 lib.jolt_decompress_rope.argtypes = [_vp, C.POINTER(Layout), _vp, _vp, C.POINTER(Rope), _vp]
 lib.jolt_decompress_static.argtypes = [_vp, C.POINTER(Layout), _vp, _vp, _vp]
 lib.jolt_attend.argtypes = [_vp, _vp, C.c_int32, C.c_double, _vp, _vp]
+lib.jolt_serialized_bytes.argtypes = [_vp, C.POINTER(C.c_int64)]
+lib.jolt_serialize.argtypes = [_vp, _vp, C.c_int64, _vp]
+lib.jolt_deserialize.argtypes = [_vp, C.c_int64, _vp, C.POINTER(_vp)]
 lib.jolt_compressed_bytes.argtypes = [_vp, C.POINTER(C.c_int64)]
 lib.jolt_get_component.argtypes = [_vp, C.c_int32, C.c_int32, _vp, C.c_int64, C.POINTER(C.c_int64)]
 lib.jolt_allocate.argtypes = [C.c_int32, C.POINTER(C.c_int32), C.c_int32, C.c_int32, C.POINTER(C.c_double),
@@ -244,6 +247,23 @@ def jolt_attend(handle: Handle, Q, scale=None, stream=None):
     sc = float(scale) if scale is not None else 1.0 / (Q.shape[-1] ** 0.5)
     _check(lib.jolt_attend(handle.ptr, Q.data_ptr(), Q.shape[2], sc, out.data_ptr(), _stream_ptr(stream)))
     return out
+
+
+def jolt_serialize(handle: Handle, stream=None) -> np.ndarray:
+    """The compressed cache as a self-describing byte image (host numpy array); see include/jolt.h."""
+    n = C.c_int64(0)
+    _check(lib.jolt_serialized_bytes(handle.ptr, C.byref(n)))
+    buf = np.empty(n.value, dtype=np.uint8)
+    _check(lib.jolt_serialize(handle.ptr, buf.ctypes.data, n.value, _stream_ptr(stream)))
+    return buf
+
+
+def jolt_deserialize(image: np.ndarray, stream=None) -> Handle:
+    image = np.ascontiguousarray(image, dtype=np.uint8)
+    h = _vp()
+    _check(lib.jolt_deserialize(image.ctypes.data, image.size, _stream_ptr(stream), C.byref(h)))
+    hd = np.frombuffer(image[:48].tobytes(), dtype=np.int32)
+    return Handle(h.value, int(hd[8]))
 
 
 def jolt_free(handle: Handle):

@@ -1030,6 +1030,30 @@ int status_to_code(const std::vector<int> &st) {
 
 
 // ------------------------------------------------------------------ compress
+// Lays the stored arrays of every cell out in the handle's device buffer (cells[i].c and n_sigma must be set).  With a
+// null buffer only the size is computed.  The layout is a function of the cell descriptors alone, which is what lets a
+// serialised cache be mapped again.
+static size_t carve_handle_blob(jolt_handle &H) {
+  Bump b;
+  b.base = (char *)H.blob;
+  int64_t stored = 0;
+  for (auto &cs : H.cells) {
+    const CellDesc &c = cs.c;
+    const size_t M = (size_t)c.m * c.T * kD;
+    cs.e = b.take<int>(4);
+    cs.lam = b.take<float>(kD);
+    cs.sigma = b.take<float>(std::max(cs.n_sigma, 1));
+    cs.G16 = b.take<__half>((size_t)c.m * c.r_t * c.r_f);
+    cs.UT16 = b.take<__half>((size_t)c.T * c.r_t);
+    cs.UF16 = b.take<__half>((size_t)kD * c.r_f);
+    cs.words = b.take<uint32_t>(M / 32 * c.bits);
+    cs.scales = b.take<__half>(c.bits ? M / 32 : 0);
+    stored += cell_bytes(c.m, c.T, kD, c.r_t, c.r_f, c.bits, true);
+  }
+  H.stored_bytes = stored;
+  return b.off + 256;
+}
+
 static int compress_impl(const jolt_layout *L, const void *K, const void *V, const jolt_cell_plan *plan,
                          const jolt_options *o, const float *const *inUT, const float *const *inUF, void *stream,
                          jolt_handle **out) {
@@ -1068,26 +1092,12 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   H->seed = o->seed;
   H->subspace = subspace;
   H->cells.resize(nc);
+  for (int i = 0; i < nc; ++i) {
+    H->cells[i].c = cells[i]; H->cells[i].c.X = nullptr;
+    H->cells[i].n_sigma = cells[i].r_t > 0 && !injected ? (mode == FM_EXACT ? cells[i].T : cells[i].k) : 0;
+  }
   for (int pass = 0; pass < 2; ++pass) {
-    Bump b;
-    b.base = (char *)H->blob;
-    int64_t stored = 0;
-    for (int i = 0; i < nc; ++i) {
-      CellStore &cs = H->cells[i];
-      const CellDesc &c = cells[i];
-      cs.c = c; cs.c.X = nullptr;
-      const size_t M = (size_t)c.m * c.T * kD;
-      cs.e = b.take<int>(4);
-      cs.lam = b.take<float>(kD);
-      cs.n_sigma = c.r_t > 0 && !injected ? (mode == FM_EXACT ? c.T : c.k) : 0;
-      cs.sigma = b.take<float>(std::max(cs.n_sigma, 1));
-      cs.G16 = b.take<__half>((size_t)c.m * c.r_t * c.r_f);
-      cs.UT16 = b.take<__half>((size_t)c.T * c.r_t);
-      cs.UF16 = b.take<__half>((size_t)kD * c.r_f);
-      cs.words = b.take<uint32_t>(M / 32 * c.bits);
-      cs.scales = b.take<__half>(c.bits ? M / 32 : 0);
-      stored += cell_bytes(c.m, c.T, kD, c.r_t, c.r_f, c.bits, true);
-    }
+    const size_t bytes = carve_handle_blob(*H);
     if (pass == 0) {
       static bool pool_set[64] = {};
       if (!pool_set[dev]) {      // keep freed blobs in the stream-ordered pool instead of returning them to the driver
@@ -1096,8 +1106,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
         cudaGetLastError();
         pool_set[dev] = true;
       }
-      H->blob_bytes = b.off + 256;
-      H->stored_bytes = stored;
+      H->blob_bytes = bytes;
       if (cudaMallocAsync(&H->blob, H->blob_bytes, st) != cudaSuccess) { cudaGetLastError(); return fail(JOLT_ENOMEM, "compressed cache of %zu bytes", H->blob_bytes); }
     }
   }
@@ -1668,6 +1677,97 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
   if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
   g_timer.begin(st);
   if ((rc = run_program(P, (char *)d_tab, st))) return rc;
+  return JOLT_OK;
+}
+
+// ------------------------------------------------------------------ serialisation
+namespace {
+constexpr uint64_t kBlobMagic = 0x314C424F544C4F4Aull;      // "JOLTOBL1"
+struct BlobHeader {
+  uint64_t magic;
+  uint32_t version, head_dim;
+  int32_t n_layers, n_kv_heads, T, n_groups, n_cells, subspace;
+  uint64_t seed, blob_bytes;
+};
+struct BlobCell { CellDesc c; int32_t n_sigma, pad; };
+size_t blob_image_bytes(const jolt_handle *H) {
+  return sizeof(BlobHeader) + sizeof(int32_t) * (H->n_groups + 1) + sizeof(BlobCell) * H->cells.size() + H->blob_bytes;
+}
+}  // namespace
+
+extern "C" int jolt_serialized_bytes(const jolt_handle *H, int64_t *bytes) {
+  if (!H || !bytes) return fail(JOLT_EINVAL, "null argument");
+  *bytes = (int64_t)blob_image_bytes(H);
+  return JOLT_OK;
+}
+
+extern "C" int jolt_serialize(const jolt_handle *H, void *host_dst, int64_t cap, void *stream) {
+  if (!H || !host_dst) return fail(JOLT_EINVAL, "null argument");
+  const size_t need = blob_image_bytes(H);
+  if (cap < (int64_t)need) return fail(JOLT_EINVAL, "buffer of %lld bytes, %zu needed", (long long)cap, need);
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
+  if (dev != H->device) return fail(JOLT_EINVAL, "handle belongs to device %d, current device is %d", H->device, dev);
+  char *p = (char *)host_dst;
+  BlobHeader hd;
+  memset(&hd, 0, sizeof hd);
+  hd.magic = kBlobMagic; hd.version = 1; hd.head_dim = kD;
+  hd.n_layers = H->n_layers; hd.n_kv_heads = H->n_kv_heads; hd.T = H->T; hd.n_groups = H->n_groups;
+  hd.n_cells = (int32_t)H->cells.size(); hd.subspace = H->subspace ? 1 : 0; hd.seed = H->seed; hd.blob_bytes = H->blob_bytes;
+  memcpy(p, &hd, sizeof hd); p += sizeof hd;
+  memcpy(p, H->group_start.data(), sizeof(int32_t) * (H->n_groups + 1)); p += sizeof(int32_t) * (H->n_groups + 1);
+  for (auto &cs : H->cells) {
+    BlobCell bc;
+    memset(&bc, 0, sizeof bc);
+    bc.c = cs.c; bc.c.X = nullptr; bc.n_sigma = cs.n_sigma;
+    memcpy(p, &bc, sizeof bc); p += sizeof bc;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  CU(cudaMemcpyAsync(p, H->blob, H->blob_bytes, cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  return JOLT_OK;
+}
+
+extern "C" int jolt_deserialize(const void *host_src, int64_t bytes, void *stream, jolt_handle **out) {
+  if (out) *out = nullptr;
+  if (!host_src || !out) return fail(JOLT_EINVAL, "null argument");
+  const char *p = (const char *)host_src;
+  BlobHeader hd;
+  if (bytes < (int64_t)sizeof hd) return fail(JOLT_EINVAL, "image of %lld bytes is shorter than its header", (long long)bytes);
+  memcpy(&hd, p, sizeof hd); p += sizeof hd;
+  if (hd.magic != kBlobMagic || hd.version != 1 || hd.head_dim != (uint32_t)kD) return fail(JOLT_EINVAL, "not a compressed-cache image of this library version");
+  if (hd.n_groups <= 0 || hd.n_cells != 2 * hd.n_groups || hd.n_layers <= 0 || hd.n_kv_heads <= 0 || hd.T <= 0) return fail(JOLT_EINVAL, "corrupt image header");
+  const size_t need = sizeof hd + sizeof(int32_t) * (hd.n_groups + 1) + sizeof(BlobCell) * (size_t)hd.n_cells + hd.blob_bytes;
+  if ((size_t)bytes < need) return fail(JOLT_EINVAL, "image of %lld bytes, header asks for %zu", (long long)bytes, need);
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
+  std::unique_ptr<jolt_handle> H(new jolt_handle);
+  H->device = dev; H->n_layers = hd.n_layers; H->n_kv_heads = hd.n_kv_heads; H->T = hd.T; H->n_groups = hd.n_groups;
+  H->seed = hd.seed; H->subspace = hd.subspace != 0;
+  H->group_start.resize(hd.n_groups + 1);
+  memcpy(H->group_start.data(), p, sizeof(int32_t) * (hd.n_groups + 1)); p += sizeof(int32_t) * (hd.n_groups + 1);
+  if (H->group_start[0] != 0 || H->group_start[hd.n_groups] != hd.n_layers) return fail(JOLT_EINVAL, "corrupt layer grouping");
+  H->cells.resize(hd.n_cells);
+  for (int i = 0; i < hd.n_cells; ++i) {
+    BlobCell bc;
+    memcpy(&bc, p, sizeof bc); p += sizeof bc;
+    const CellDesc &c = bc.c;
+    const int g = i / 2;
+    if (c.T != hd.T || c.n_heads != hd.n_kv_heads || c.m != (H->group_start[g + 1] - H->group_start[g]) * hd.n_kv_heads || c.cell != i ||
+        c.r_t < 0 || c.r_t > c.T || c.r_f < 0 || c.r_f > kD || !bits_ok(c.bits) || bc.n_sigma < 0 || bc.n_sigma > c.T)
+      return fail(JOLT_EINVAL, "corrupt descriptor of cell %d", i);
+    H->cells[i].c = c; H->cells[i].c.X = nullptr; H->cells[i].n_sigma = bc.n_sigma;
+  }
+  if (carve_handle_blob(*H) != hd.blob_bytes) return fail(JOLT_EINVAL, "image payload size does not match its descriptors");
+  H->blob_bytes = hd.blob_bytes;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMallocAsync(&H->blob, H->blob_bytes, st) != cudaSuccess) { cudaGetLastError(); return fail(JOLT_ENOMEM, "compressed cache of %zu bytes", H->blob_bytes); }
+  carve_handle_blob(*H);
+  cudaError_t ce = cudaMemcpyAsync(H->blob, p, H->blob_bytes, cudaMemcpyHostToDevice, st);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+  if (ce != cudaSuccess) { cudaGetLastError(); cudaFreeAsync(H->blob, st); return fail(JOLT_ECUDA, "upload: %s", cudaGetErrorString(ce)); }
+  for (auto &cs : H->cells) encode_store_maps(cs);          // tensor maps point into the new buffer
+  *out = H.release();
   return JOLT_OK;
 }
 

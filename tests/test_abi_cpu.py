@@ -72,6 +72,19 @@ def test_argument_validation_needs_no_gpu(B):
     assert B.lib.jolt_decompress(None, ctypes.byref(lay), K.data_ptr(), V.data_ptr(), None) == B.EINVAL
 
 
+def test_image_checks_come_before_any_gpu_call(B):
+    import numpy as np
+    h = ctypes.c_void_p()
+    assert B.lib.jolt_deserialize(None, 0, None, ctypes.byref(h)) == B.EINVAL
+    junk = np.zeros(4096, dtype=np.uint8)
+    assert B.lib.jolt_deserialize(junk.ctypes.data, junk.size, None, ctypes.byref(h)) == B.EINVAL and not h.value
+    assert B.lib.jolt_deserialize(junk.ctypes.data, 8, None, ctypes.byref(h)) == B.EINVAL
+    n = ctypes.c_int64(0)
+    assert B.lib.jolt_serialized_bytes(None, ctypes.byref(n)) == B.EINVAL
+    assert B.lib.jolt_serialize(None, junk.ctypes.data, junk.size, None) == B.EINVAL
+    assert B.lib.jolt_attend(None, junk.ctypes.data, 4, 1.0, junk.ctypes.data, None) == B.EINVAL
+
+
 def test_byte_model_and_cap_policy_match_oracle(B):
     for (m, T, rt, rf, b) in [(32, 4096, 128, 128, 4), (8, 512, 64, 64, 2), (160, 4096, 48, 112, 0), (32, 8192, 16, 16, 8)]:
         assert B.cell_bytes(m, T, 128, rt, rf, b, True) == O.stored_bytes(m, T, 128, rt, rf, b)

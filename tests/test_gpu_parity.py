@@ -544,3 +544,43 @@ def test_attend_on_the_factors(B, synth, case):
         assert rel <= 3 * recon_gate(eo), (gi, rel, eo)
     assert B.lib.jolt_attend(h.ptr, Q.cuda().data_ptr(), 9, scale, out.data_ptr(), None) == B.EINVAL    # n_q > 8
     h.free()
+
+
+# --------------------------------------------------------------------------- persistence of a compressed cache
+def test_serialized_cache_round_trip_is_bit_exact(B, synth):
+    cfg = synth.CacheConfig("t", 4, 2, 2, 384, n_terms=20, seed=61)
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2, 4]
+    plans = [(32, 96, 4), (16, 128, 8), (0, 0, 2), (48, 64, 3)]
+    opts = B.default_options(seed=17)
+    h = B.jolt_compress(K, V, gs, plans, opts)
+    Ko, Vo = torch.empty_like(K), torch.empty_like(V)
+    B.jolt_decompress(h, Ko, Vo, gs)
+    g = torch.Generator().manual_seed(4)
+    Q = torch.randn(4, 2, 4, 128, generator=g).cuda()
+    att = B.jolt_attend(h, Q)
+    sig = [h.component(c, 6).copy() for c in range(4)]
+    nbytes = h.bytes()
+    image = B.jolt_serialize(h)
+    h.free()
+    # the image is position independent: a copy at another address, after the original is gone
+    h2 = B.jolt_deserialize(image.copy())
+    assert h2.bytes() == nbytes
+    Ko2, Vo2 = torch.empty_like(K), torch.empty_like(V)
+    B.jolt_decompress(h2, Ko2, Vo2, gs)
+    att2 = B.jolt_attend(h2, Q)
+    torch.cuda.synchronize()
+    assert torch.equal(Ko2, Ko) and torch.equal(Vo2, Vo) and torch.equal(att2, att)
+    for c in range(4):
+        assert np.array_equal(h2.component(c, 6), sig[c])
+    assert np.array_equal(B.jolt_serialize(h2), image)
+    # truncated and damaged images are refused
+    for bad in (image[: image.size // 2], np.concatenate([image[:8] ^ 1, image[8:]])):
+        with pytest.raises(B.JoltError) as e:
+            B.jolt_deserialize(bad)
+        assert e.value.status == B.EINVAL
+    worse = image.copy()
+    worse[56 + 12 + 12] ^= 0xFF          # the head count in the first cell descriptor
+    with pytest.raises(B.JoltError):
+        B.jolt_deserialize(worse)
+    h2.free()
