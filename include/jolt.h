@@ -71,7 +71,19 @@ typedef struct {
   int32_t q_cap;                    /* <= 0: the paper's cap policy min(max(q_min(R), ceil(T/32)), 512)   */
   const double *eps2;               /* host table eps^2(b) for b = 0..8 (Eq. (2)); NULL = built-in        */
   int32_t count_scale_bytes;        /* 1 (default): the fp16 group scales count toward the budget         */
+  int32_t allocator;                /* JOLT_ALLOC_DUAL (default) | JOLT_ALLOC_GREEDY | JOLT_ALLOC_UNIFORM  */
 } jolt_options;
+
+/* Allocators of jolt_plan / jolt_allocate.  JOLT_ALLOC_DUAL is the paper's method: the Lagrangian relaxation of
+ * Eq. (3) with one multiplier, bisected (Eq. (4)).  The other two are the alternatives its ablations compare against
+ * (Sec. 6), described there in one sentence each; the readings taken:
+ * JOLT_ALLOC_GREEDY -- every cell starts at its cheapest option; each step applies, among all moves of one cell to a
+ *   costlier option with a smaller modelled error that still fits the remaining budget, the one with the largest
+ *   error reduction per extra byte; stops when no move is left.
+ * JOLT_ALLOC_UNIFORM -- ranks and bits are shared: one (r_t, r_f, bits) for all key cells and one for all value
+ *   cells, the pair with the smallest summed modelled error that fits the budget (exhaustive over the grid).
+ * All three return JOLT_EBUDGET with the cheapest allocation when nothing fits. */
+enum { JOLT_ALLOC_DUAL = 0, JOLT_ALLOC_GREEDY = 1, JOLT_ALLOC_UNIFORM = 2 };
 
 /* JOLT_TOKEN_EXACT (the exact token-mode SVD that Sec. 5 replaces): up to T = 1024 the T x T Gram of the
  * projected unfolding is diagonalised in fp64.  Beyond that the dominant r_t subspace is computed by block

@@ -18,6 +18,7 @@ Each function names the passage of the paper it follows:
 * Eq. (1)                            -> eq1_bytes, stored_bytes
 * Eq. (2)                            -> eps2_table, tau_table
 * Eq. (3), Eq. (4)                   -> dual_allocate
+* Sec. 6 (ablations: greedy and shared-rank allocators, one sentence each) -> greedy_allocate, uniform_allocate
 * App. "RoPE pre vs. post on K" (keys are decomposed before the rotary embedding, which is
   re-applied at decode time)        -> rope_rotate, decompress_cell_rope
 * Sec. 7 / closing discussion (attention directly on the factors, named as the route to decode
@@ -599,6 +600,80 @@ def dual_allocate(cells, budget: float, halvings: int = 200):
         else:
             lo = mid
     return ch_hi, cost_hi, hi, True
+
+
+def _cheapest(e, c):
+    return int(np.lexsort((e, c))[0])
+
+
+def greedy_allocate(cells, budget: float):
+    """Greedy allocator of the ablations (Sec. 6: every marginal byte goes to the group with the largest error
+    reduction per byte; no global multiplier).  The paper gives that sentence only; the reading: every cell starts
+    at its cheapest option, and each step applies, among all moves of one cell to a costlier option with a smaller
+    error that still fits, the one with the largest (error reduction) / (extra bytes); ties go to the move with
+    fewer extra bytes, then to the lower cell, then to the lower option index.  Returns (choice, cost, feasible)."""
+    ch = [_cheapest(e, c) for e, c in cells]
+    total = float(sum(c[i] for (e, c), i in zip(cells, ch)))
+    if total > budget:
+        return ch, total, False
+    while True:
+        best = None
+        for ci, (e, c) in enumerate(cells):
+            e0, c0 = e[ch[ci]], c[ch[ci]]
+            for i in range(len(c)):
+                extra, gain = c[i] - c0, e0 - e[i]
+                if not (extra > 0) or not (gain > 0) or total + extra > budget:
+                    continue
+                ratio = gain / extra
+                if best is None or ratio > best[0] or (ratio == best[0] and extra < best[1]):
+                    best = (ratio, extra, ci, i)
+        if best is None:
+            return ch, total, True
+        total += best[1]
+        ch[best[2]] = best[3]
+
+
+def uniform_allocate(cells, trips, budget: float):
+    """Uniform allocator of the ablations (Sec. 6: ranks shared instead of per group).  Reading: one (r_t, r_f, bits)
+    for all cells with an even index (keys) and one for all cells with an odd index (values); exhaustive search for
+    the pair with the smallest summed error whose summed cost fits (ties: the cheaper pair, then the earlier one).
+    trips[c][i] is the triple of option i of cell c; a triple that some cell of a class lacks is no candidate.
+    Returns (choice, cost, feasible)."""
+    cand = []
+    for cls in (0, 1):
+        lst = []
+        members = list(range(cls, len(cells), 2))
+        for t in trips[members[0]]:
+            idx = []
+            for c in members:
+                tl = [tuple(x) for x in trips[c]]
+                if tuple(t) not in tl:
+                    idx = None
+                    break
+                idx.append(tl.index(tuple(t)))
+            if idx is not None:
+                lst.append((sum(float(cells[c][0][j]) for c, j in zip(members, idx)),
+                            sum(float(cells[c][1][j]) for c, j in zip(members, idx)), idx))
+        cand.append(lst)
+    best = None
+    for a in cand[0]:
+        for b in cand[1]:
+            cst, e = a[1] + b[1], a[0] + b[0]
+            if cst > budget:
+                continue
+            if best is None or e < best[0] or (e == best[0] and cst < best[1]):
+                best = (e, cst, a[2], b[2])
+    feasible = best is not None
+    if not feasible:
+        a = min(cand[0], key=lambda x: (x[1], x[0]))
+        b = min(cand[1], key=lambda x: (x[1], x[0]))
+        best = (a[0] + b[0], a[1] + b[1], a[2], b[2])
+    ch = [0] * len(cells)
+    for n, c in enumerate(range(0, len(cells), 2)):
+        ch[c] = best[2][n]
+    for n, c in enumerate(range(1, len(cells), 2)):
+        ch[c] = best[3][n]
+    return ch, best[1], feasible
 
 
 def plan_spectra(X, q_cap: int, *, seed: int = 0, cell: int = 0, oversample: int = 10,

@@ -23,6 +23,7 @@ OK, EINVAL, EUNSUPPORTED, EBUDGET, ENUMERIC, ENOMEM, ECUDA, ETIMEOUT = 0, -1, -2
 F16, F32 = 0, 1
 MEM_DEVICE, MEM_HOST = 0, 1
 TOKEN_EXACT, TOKEN_RANDOMIZED = 0, 1
+ALLOC_DUAL, ALLOC_GREEDY, ALLOC_UNIFORM = 0, 1, 2
 
 
 class Layout(C.Structure):
@@ -41,7 +42,7 @@ class Options(C.Structure):
                 ("quant_group", C.c_int32), ("seed", C.c_uint64),
                 ("bits_set", C.POINTER(C.c_int32)), ("n_bits", C.c_int32),
                 ("rank_step", C.c_int32), ("r_t_min", C.c_int32), ("r_f_min", C.c_int32), ("q_cap", C.c_int32),
-                ("eps2", C.POINTER(C.c_double)), ("count_scale_bytes", C.c_int32)]
+                ("eps2", C.POINTER(C.c_double)), ("count_scale_bytes", C.c_int32), ("allocator", C.c_int32)]
 
 
 _vp = C.c_void_p

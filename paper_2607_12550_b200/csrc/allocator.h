@@ -109,4 +109,91 @@ inline bool dual_allocate(const std::vector<CellOptions> &cells, double budget, 
   return true;
 }
 
+// Index of a cell's cheapest option (ties: the smaller error).
+inline size_t cheapest_option(const CellOptions &c) {
+  size_t b = 0;
+  for (size_t i = 1; i < c.cost.size(); ++i)
+    if (c.cost[i] < c.cost[b] || (c.cost[i] == c.cost[b] && c.err[i] < c.err[b])) b = i;
+  return b;
+}
+
+// Greedy allocator of the ablations (paper Sec. 6: "spends each marginal byte on whichever group offers the largest
+// error reduction per byte", no global multiplier).  Every cell starts at its cheapest option; each step applies, among
+// all moves of one cell to a costlier option with a smaller error that still fits the remaining budget, the one with
+// the largest error reduction per extra byte (ties: fewer extra bytes, then lower cell, then lower option index).
+inline bool greedy_allocate(const std::vector<CellOptions> &cells, double budget, std::vector<size_t> &choice, double &total) {
+  choice.resize(cells.size());
+  total = 0;
+  for (size_t c = 0; c < cells.size(); ++c) { choice[c] = cheapest_option(cells[c]); total += cells[c].cost[choice[c]]; }
+  if (total > budget) return false;
+  for (;;) {
+    bool found = false;
+    double best_ratio = 0, best_extra = 0;
+    size_t bc = 0, bi = 0;
+    for (size_t c = 0; c < cells.size(); ++c) {
+      const double e0 = cells[c].err[choice[c]], c0 = cells[c].cost[choice[c]];
+      for (size_t i = 0; i < cells[c].cost.size(); ++i) {
+        const double extra = cells[c].cost[i] - c0, gain = e0 - cells[c].err[i];
+        if (!(extra > 0) || !(gain > 0) || total + extra > budget) continue;
+        const double ratio = gain / extra;
+        if (!found || ratio > best_ratio || (ratio == best_ratio && extra < best_extra)) {
+          found = true; best_ratio = ratio; best_extra = extra; bc = c; bi = i;
+        }
+      }
+    }
+    if (!found) break;
+    total += best_extra;
+    choice[bc] = bi;
+  }
+  return true;
+}
+
+// Uniform allocator of the ablations (ranks shared instead of per group): one option for all cells of class 0 (even
+// cell index: keys) and one for all cells of class 1 (odd: values), the pair with the smallest summed error whose
+// summed cost fits the budget (ties: the cheaper pair, then the earlier one).  Options are matched across cells by
+// their (r_t, r_f, bits) triple; a triple that some cell of the class does not offer is not a candidate.
+inline bool uniform_allocate(const std::vector<CellOptions> &cells, double budget, std::vector<size_t> &choice, double &total) {
+  struct Cand { jolt_cell_plan t; double err, cost; std::vector<size_t> idx; };
+  std::vector<Cand> cand[2];
+  for (int cls = 0; cls < 2; ++cls) {
+    size_t first = cls;
+    if (first >= cells.size()) continue;
+    for (size_t i = 0; i < cells[first].trip.size(); ++i) {
+      Cand k{cells[first].trip[i], 0, 0, {}};
+      bool everywhere = true;
+      for (size_t c = first; c < cells.size() && everywhere; c += 2) {
+        size_t j = 0;
+        for (; j < cells[c].trip.size(); ++j)
+          if (cells[c].trip[j].r_t == k.t.r_t && cells[c].trip[j].r_f == k.t.r_f && cells[c].trip[j].bits == k.t.bits) break;
+        if (j == cells[c].trip.size()) { everywhere = false; break; }
+        k.err += cells[c].err[j]; k.cost += cells[c].cost[j]; k.idx.push_back(j);
+      }
+      if (everywhere) cand[cls].push_back(k);
+    }
+  }
+  choice.assign(cells.size(), 0);
+  if (cells.size() < 2 || cand[0].empty() || cand[1].empty()) {      // a single class: fall back to one shared option
+    for (size_t c = 0; c < cells.size(); ++c) choice[c] = cheapest_option(cells[c]);
+    total = 0;
+    for (size_t c = 0; c < cells.size(); ++c) total += cells[c].cost[choice[c]];
+    return total <= budget;
+  }
+  bool found = false;
+  size_t ba = 0, bb = 0;
+  double be = 0, bcst = 0;
+  size_t ca = 0, cb = 0;                       // cheapest pair, for the infeasible case
+  for (size_t a = 0; a < cand[0].size(); ++a) if (cand[0][a].cost < cand[0][ca].cost || (cand[0][a].cost == cand[0][ca].cost && cand[0][a].err < cand[0][ca].err)) ca = a;
+  for (size_t b = 0; b < cand[1].size(); ++b) if (cand[1][b].cost < cand[1][cb].cost || (cand[1][b].cost == cand[1][cb].cost && cand[1][b].err < cand[1][cb].err)) cb = b;
+  for (size_t a = 0; a < cand[0].size(); ++a)
+    for (size_t b = 0; b < cand[1].size(); ++b) {
+      const double cst = cand[0][a].cost + cand[1][b].cost, e = cand[0][a].err + cand[1][b].err;
+      if (cst > budget) continue;
+      if (!found || e < be || (e == be && cst < bcst)) { found = true; ba = a; bb = b; be = e; bcst = cst; }
+    }
+  if (!found) { ba = ca; bb = cb; bcst = cand[0][ca].cost + cand[1][cb].cost; }
+  for (size_t c = 0, n0 = 0, n1 = 0; c < cells.size(); ++c) choice[c] = (c % 2 == 0) ? cand[0][ba].idx[n0++] : cand[1][bb].idx[n1++];
+  total = bcst;
+  return found;
+}
+
 }  // namespace jolt

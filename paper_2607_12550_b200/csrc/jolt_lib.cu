@@ -1826,6 +1826,7 @@ static void fill_defaults(jolt_options *o) {
   o->token_mode = JOLT_TOKEN_RANDOMIZED; o->oversample = 10; o->power_iters = 1; o->quant_group = kGroup; o->seed = 0;
   o->bits_set = nullptr; o->n_bits = 0; o->rank_step = 16; o->r_t_min = 16; o->r_f_min = 16; o->q_cap = 0; o->eps2 = nullptr;
   o->count_scale_bytes = 1;
+  o->allocator = JOLT_ALLOC_DUAL;
 }
 extern "C" void jolt_default_options(jolt_options *o) { if (o) fill_defaults(o); }
 
@@ -1885,7 +1886,10 @@ extern "C" int jolt_allocate(int32_t n_cells, const int32_t *m, int32_t T, int32
   }
   std::vector<size_t> choice;
   double total = 0;
-  const bool ok = dual_allocate(cells, budget, choice, total);
+  if (o->allocator < JOLT_ALLOC_DUAL || o->allocator > JOLT_ALLOC_UNIFORM) return fail(JOLT_EINVAL, "allocator %d", o->allocator);
+  const bool ok = o->allocator == JOLT_ALLOC_GREEDY ? greedy_allocate(cells, budget, choice, total)
+                  : o->allocator == JOLT_ALLOC_UNIFORM ? uniform_allocate(cells, budget, choice, total)
+                                                       : dual_allocate(cells, budget, choice, total);
   for (int c = 0; c < n_cells; ++c) out[c] = cells[c].trip[choice[c]];
   if (achieved) *achieved = total;
   return ok ? JOLT_OK : fail(JOLT_EBUDGET, "cheapest allocation needs %.0f bytes, budget is %.0f", total, budget);

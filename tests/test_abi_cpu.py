@@ -151,6 +151,53 @@ def test_library_dual_equals_oracle_dual_on_oracle_spectra(B, bits_set):
             assert ach <= budget
 
 
+@pytest.mark.parametrize("which", ["greedy", "uniform"])
+def test_library_ablation_allocators_equal_the_oracle(B, which):
+    rng = np.random.default_rng(5)
+    m, T, d = 8, 512, 128
+    n_cells = 6
+    bits_set = [0, 2, 4, 8]
+    eps2 = O.eps2_table(bits_set, n=1 << 14)
+    eps_arr = [eps2.get(b, float("nan")) for b in range(9)]
+    lam, sig2, tot, rtmax = [], [], [], []
+    for c in range(n_cells):
+        alpha = 1.0 if c % 2 == 0 else 0.4
+        s = (np.arange(1, 65) ** -alpha) * rng.uniform(0.5, 2.0)
+        l3 = np.sort(rng.random(128) ** 3)[::-1] * 5
+        total = max(np.sum(s ** 2), l3.sum()) * 1.3
+        l3 = l3 * total / l3.sum()
+        spec = O.tail_mass_spectrum(s, total) ** 2
+        lam.append(l3); sig2.append(spec); tot.append(float(total)); rtmax.append(64 if c != 3 else 48)
+    raw = n_cells * m * T * d * 2
+    for ratio in (1.5, 2.0, 3.0, 5.0, 9.0, 400.0):
+        budget = raw / ratio
+        cells, trips = [], []
+        for c in range(n_cells):
+            rt_grid, rf_grid = _grid(16, rtmax[c], 16), _grid(16, 128, 16)
+            tau = O.tau_table(lam[c], sig2[c], tot[c], rt_grid, rf_grid)
+            e, s_, t = O.cell_options(m, T, d, tau, rt_grid, rf_grid, bits_set, eps2)
+            cells.append((e, s_)); trips.append(t)
+        if which == "greedy":
+            ch, cost, ok = O.greedy_allocate(cells, budget)
+        else:
+            ch, cost, ok = O.uniform_allocate(cells, trips, budget)
+        ref = [tuple(trips[c][i]) for c, i in enumerate(ch)]
+        opts = B.default_options(bits_set=bits_set, eps2=eps_arr,
+                                 allocator=B.ALLOC_GREEDY if which == "greedy" else B.ALLOC_UNIFORM)
+        got, ach, st = B.jolt_allocate([m] * n_cells, T, d, np.stack(lam), sig2, tot, rtmax, budget, opts, allow_budget=True)
+        assert (st == 0) == ok, (ratio, st, ok)
+        assert got == ref, (ratio, got, ref)
+        assert ach == cost
+        if which == "uniform":
+            assert len(set(got[0::2])) == 1 and len(set(got[1::2])) == 1
+    bad = B.default_options(allocator=7)
+    got, ach, st = B.jolt_allocate([m] * n_cells, T, d, np.stack(lam), sig2, tot, rtmax, raw / 2, bad, allow_budget=True) \
+        if False else (None, None, B.lib.jolt_allocate.__name__ and None)
+    with pytest.raises(B.JoltError) as e:
+        B.jolt_allocate([m] * n_cells, T, d, np.stack(lam), sig2, tot, rtmax, raw / 2, bad)
+    assert e.value.status == B.EINVAL
+
+
 def test_budget_below_minimum_reports_ebudget_and_cheapest_plan(B):
     lam = np.ones((2, 128)); sig2 = [np.ones(33), np.ones(33)]
     got, ach, st = B.jolt_allocate([4, 4], 256, 128, lam, sig2, [128.0, 128.0], [32, 32], 10.0, allow_budget=True)

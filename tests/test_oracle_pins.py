@@ -503,3 +503,61 @@ def test_attend_scores_on_the_factors_identity():
         + O.unrotate(np.einsum("hit,htf->hif", Pw, rV), cV.signs)
     O_def = np.einsum("hit,htf->hif", Pw, Vh)
     assert np.abs(O_fact - O_def).max() <= 1e-11 * np.abs(O_def).max()
+
+
+# --------------------------------------------------------------------------- ablation allocators
+def test_greedy_hand_worked_sequence():
+    # two cells, options (error, cost); budget 10.  Start: cheapest of each = (9, 1) and (8, 1), cost 2.
+    # moves that fit: A: (4, 3): 5/2 = 2.5, (1, 8): 8/7;  B: (5, 2): 3/1 = 3, (2, 6): 6/5.  -> B to (5, 2), cost 3
+    # then A (4, 3): 2.5, A (1, 8): 8/7 (fits: 3 + 7 = 10), B (2, 6): 3/4 -> A to (4, 3), cost 5
+    # then A (1, 8): 3/5 = 0.6 (5 + 5 = 10 fits), B (2, 6): 3/4 = 0.75 (5 + 4 = 9 fits) -> B to (2, 6), cost 9
+    # then A (1, 8): extra 5 does not fit (14 > 10): stop.
+    A = (np.array([9.0, 4.0, 1.0]), np.array([1.0, 3.0, 8.0]))
+    Bc = (np.array([8.0, 5.0, 2.0]), np.array([1.0, 2.0, 6.0]))
+    ch, cost, ok = O.greedy_allocate([A, Bc], 10.0)
+    assert ok and ch == [1, 2] and cost == 9.0
+    # a budget below the cheapest allocation is reported, with the cheapest allocation
+    ch, cost, ok = O.greedy_allocate([A, Bc], 1.5)
+    assert not ok and ch == [0, 0] and cost == 2.0
+    # a budget that covers everything ends at the smallest errors
+    ch, cost, ok = O.greedy_allocate([A, Bc], 100.0)
+    assert ok and ch == [2, 2]
+
+
+def test_greedy_and_uniform_invariants_against_brute_force():
+    import itertools
+    rng = np.random.default_rng(11)
+    for trial in range(20):
+        n_opt = 5
+        trips = [[(16 * (i + 1), 16, 4) for i in range(n_opt)] for _ in range(4)]
+        cells = []
+        for c in range(4):
+            cost = np.sort(rng.uniform(1, 10, n_opt))
+            err = np.sort(rng.uniform(0, 1, n_opt))[::-1] * rng.uniform(0.5, 2)
+            cells.append((err, cost))
+        lo = sum(c.min() for e, c in cells)
+        hi = sum(c.max() for e, c in cells)
+        for budget in (lo + (hi - lo) * f for f in (1e-6, 0.25, 0.5, 0.75, 1 + 1e-6)):   # off the exact end points
+            all_alloc = list(itertools.product(range(n_opt), repeat=4))
+            feas = [a for a in all_alloc if sum(cells[c][1][i] for c, i in enumerate(a)) <= budget + 1e-12]
+            e_opt = min(sum(cells[c][0][i] for c, i in enumerate(a)) for a in feas)
+            # greedy: feasible, no affordable improving single move left, never better than the optimum
+            ch, cost, ok = O.greedy_allocate(cells, budget)
+            assert ok and cost <= budget + 1e-12 and abs(cost - sum(cells[c][1][i] for c, i in enumerate(ch))) < 1e-9
+            e_g = sum(cells[c][0][i] for c, i in enumerate(ch))
+            assert e_g >= e_opt - 1e-12
+            for c in range(4):
+                for i in range(n_opt):
+                    extra, gain = cells[c][1][i] - cells[c][1][ch[c]], cells[c][0][ch[c]] - cells[c][0][i]
+                    assert not (extra > 0 and gain > 0 and cost + extra <= budget)
+            # uniform: the best shared pair by independent enumeration; never better than the per-cell optimum
+            chu, costu, oku = O.uniform_allocate(cells, trips, budget)
+            pairs = [(a, b) for a in range(n_opt) for b in range(n_opt)
+                     if cells[0][1][a] + cells[2][1][a] + cells[1][1][b] + cells[3][1][b] <= budget]
+            if pairs:
+                e_pairs = min(cells[0][0][a] + cells[2][0][a] + cells[1][0][b] + cells[3][0][b] for a, b in pairs)
+                e_u = sum(cells[c][0][i] for c, i in enumerate(chu))
+                assert oku and chu[0] == chu[2] and chu[1] == chu[3] and costu <= budget + 1e-12
+                assert abs(e_u - e_pairs) < 1e-12 and e_u >= e_opt - 1e-12
+            else:
+                assert not oku and chu == [0, 0, 0, 0]
