@@ -584,3 +584,24 @@ def test_serialized_cache_round_trip_is_bit_exact(B, synth):
     with pytest.raises(B.JoltError):
         B.jolt_deserialize(worse)
     h2.free()
+
+
+def test_plan_honours_the_allocator_option(B, synth):
+    cfg = synth.CacheConfig("t", 6, 2, 2, 512, n_terms=24, seed=71)
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2, 4, 6]
+    raw = 2 * K.numel() * 2
+    plans = {}
+    for name, alloc in (("dual", B.ALLOC_DUAL), ("greedy", B.ALLOC_GREEDY), ("uniform", B.ALLOC_UNIFORM)):
+        opts = B.default_options(seed=5, allocator=alloc)
+        plans[name], planned = B.jolt_plan(K, V, gs, raw / 3.0, opts)
+        assert planned <= raw / 3.0, name
+        assert planned == sum(B.cell_bytes(4, 512, 128, *p) for p in plans[name])
+    assert len(set(plans["uniform"][0::2])) == 1 and len(set(plans["uniform"][1::2])) == 1
+    # a plan from any allocator compresses and decodes
+    h = B.jolt_compress(K, V, gs, plans["greedy"], B.default_options(seed=5))
+    Ko, Vo = torch.empty_like(K), torch.empty_like(V)
+    B.jolt_decompress(h, Ko, Vo, gs)
+    torch.cuda.synchronize()
+    assert float((Ko.float() - K.float()).norm() / K.float().norm()) < 0.2
+    h.free()
