@@ -487,18 +487,18 @@ def test_rope_at_decode(B, synth, dtype, fused):
 
 
 # --------------------------------------------------------------------------- attention on the compressed cache
-@pytest.mark.parametrize("case", ["a", "b", "c"])
+@pytest.mark.parametrize("case", ["a", "b", "c", "d", "e"])
 def test_attend_on_the_factors(B, synth, case):
     # Injected factors (both sides hold the same stored backbone).  T = 384 leaves a 128-token tail chunk.
     cfg = synth.CacheConfig("t", 4, 2, 2, 384, n_terms=20, seed=51)
     K, V = synth.make_cache(cfg, device="cuda")
     gs = [0, 2, 4]
-    if case == "a":
-        plans, n_q = [(16, 64, 4), (16, 128, 2), (32, 96, 3), (0, 0, 8)], 4
+    if case in ("a", "d"):
+        plans, n_q = [(16, 64, 4), (16, 128, 2), (32, 96, 3), (0, 0, 8)], (4 if case == "a" else 1)
     elif case == "b":
         plans, n_q = [(0, 0, 4), (24, 96, 0), (16, 128, 1), (16, 64, 4)], 5
     else:
-        plans, n_q = [(16, 64, 8), (16, 128, 4), (32, 96, 2), (0, 0, 8)], 8
+        plans, n_q = [(16, 64, 8), (16, 128, 4), (32, 96, 2), (0, 0, 1)], (8 if case == "c" else 3)
     Knp, Vnp = _np(K), _np(V)
     UT, UF = [], []
     for c, (rt, rf, _) in enumerate(plans):
