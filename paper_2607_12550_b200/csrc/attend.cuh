@@ -345,9 +345,9 @@ __device__ __forceinline__ void att_mma_f16(float (&d)[4], const uint32_t (&a)[4
 
 // The score kernel for 1-, 2-, 4- and 8-bit codes with the code-times-query contraction on the tensor cores.
 // grid (ceil(n_chunks / 2), m, groups), kAttChunk threads = 8 warps; a CTA walks every gridDim.x-th chunk of its head, a
-// warp owns 32 tokens of the chunk = two 16-row MMA tiles.  Every lane
-// still loads its own token's packed row and scales (as in the CUDA-core kernel); the m16n8k16 A fragments are built from
-// words handed over by warp shuffles (the lane of row g holds that row), a pair of codes expanding to the exact fp16
+// warp owns 32 tokens of the chunk = two 16-row MMA tiles.  The chunk's
+// packed rows and scales are loaded coalesced and staged in shared memory; the m16n8k16 A fragments are built from
+// words read there (odd row pitch: the eight rows of a fragment column fall into eight banks), a pair of codes expanding to the exact fp16
 // integers 2u + 1 - 2^b (so the mid-rise half step is part of the operand and the product is twice the wanted sum).
 // B = the rotated query as hi + lo fp16, 8 query columns, staged once per CTA in shared memory (4 conflict-free word
 // reads per MMA pair).  Per 32-feature group the 16 x 8 partial product is scaled by Delta / 2 of its row.  Registers are
@@ -361,7 +361,7 @@ __device__ __forceinline__ uint32_t att_pair_f16(uint32_t x, int bits) {
 }
 
 template <int BITS>
-__global__ void __launch_bounds__(kAttChunk, BITS == 8 ? 2 : 3) attend_scores_mma_kernel(const AttendJob *__restrict__ jobs, int NQP, int n_chunks) {
+__global__ void __launch_bounds__(kAttChunk, BITS >= 4 ? 2 : 3) attend_scores_mma_kernel(const AttendJob *__restrict__ jobs, int NQP, int n_chunks) {
   static_assert(BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8, "codes that do not straddle words");
   const AttendJob &jb = jobs[blockIdx.z];
   if (jb.k.bits != BITS) return;
@@ -369,26 +369,32 @@ __global__ void __launch_bounds__(kAttChunk, BITS == 8 ? 2 : 3) attend_scores_mm
   if (h >= jb.m || (int)blockIdx.x * kAttChunk >= jb.T) return;
   __shared__ float red[2][kAttChunk / 32][kAttMaxQ];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
-  // the lane's own packed row and scales, requested one chunk ahead
-  uint32_t nrow[4 * BITS];
+  // the chunk's packed rows and scales, requested one chunk ahead: consecutive threads take consecutive 16-byte pieces
+  // (coalesced), and put them into shared memory with an odd row pitch, from where the fragment builders read words
+  constexpr int RP = 4 * BITS + 1;                 // words per staged row: rows g = 0..7 of one word fall into 8 banks
+  __shared__ uint32_t rows[kAttChunk][RP];
+  __shared__ uint2 scs[kAttChunk];
+  uint4 npc[BITS];                                 // pieces tid, tid + 256, ... of the chunk's kAttChunk * BITS
   uint2 nsc = make_uint2(0u, 0u);
   float2 nsb[4];                   // backbone scores of this lane's four (row, query pair) results
   const bool qok = 2 * c < NQP;
   auto fetch = [&](int chunk) {
-    const int t = chunk * kAttChunk + tid;
 #pragma unroll
     for (int r = 0; r < 4; ++r) nsb[r] = make_float2(0.f, 0.f);
-    if (chunk < n_chunks && chunk * kAttChunk + warp * 32 < jb.T) {
-      if (qok && jb.k.r_t > 0) {
+    if (chunk >= n_chunks) return;
+    const int t0 = chunk * kAttChunk, nt = min(kAttChunk, jb.T - t0);
+    if (qok && jb.k.r_t > 0 && warp * 32 < nt) {
 #pragma unroll
-        for (int r = 0; r < 4; ++r)
-          nsb[r] = *(const float2 *)(jb.p + ((size_t)h * jb.T + chunk * kAttChunk + warp * 32 + (r >> 1) * 16 + (r & 1) * 8 + g) * NQP + 2 * c);
-      }
-      const uint4 *wp = (const uint4 *)(jb.k.words + ((size_t)h * jb.T + t) * (4 * BITS));
-#pragma unroll
-      for (int i = 0; i < BITS; ++i) { const uint4 v = __ldg(wp + i); nrow[4 * i] = v.x; nrow[4 * i + 1] = v.y; nrow[4 * i + 2] = v.z; nrow[4 * i + 3] = v.w; }
-      nsc = __ldg((const uint2 *)(jb.k.scales + ((size_t)h * jb.T + t) * 4));
+      for (int r = 0; r < 4; ++r)
+        nsb[r] = *(const float2 *)(jb.p + ((size_t)h * jb.T + t0 + warp * 32 + (r >> 1) * 16 + (r & 1) * 8 + g) * NQP + 2 * c);
     }
+    const uint4 *wp = (const uint4 *)(jb.k.words + ((size_t)h * jb.T + t0) * (4 * BITS));
+#pragma unroll
+    for (int i = 0; i < BITS; ++i) {
+      const int idx = tid + i * kAttChunk;
+      npc[i] = idx < nt * BITS ? __ldg(wp + idx) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    nsc = tid < nt ? __ldg((const uint2 *)(jb.k.scales + ((size_t)h * jb.T + t0) * 4) + tid) : make_uint2(0u, 0u);
   };
   fetch(blockIdx.x);
   // B operand (rotated query, hi and lo) of the head in shared memory: [query][feature pair], 68 words per row so that
@@ -402,13 +408,17 @@ __global__ void __launch_bounds__(kAttChunk, BITS == 8 ? 2 : 3) attend_scores_mm
   __syncthreads();
   for (int chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
   const bool live = chunk * kAttChunk + warp * 32 < jb.T;      // T is a multiple of 128: a warp is all in or all out
-  uint32_t row[4 * BITS];
+  __syncthreads();                                       // the previous chunk's rows have been read
 #pragma unroll
-  for (int i = 0; i < 4 * BITS; ++i) row[i] = live ? nrow[i] : 0u;
-  const uint2 scw = nsc;
+  for (int i = 0; i < BITS; ++i) {
+    const int idx = tid + i * kAttChunk, r = idx / BITS, w4 = (idx % BITS) * 4;
+    rows[r][w4] = npc[i].x; rows[r][w4 + 1] = npc[i].y; rows[r][w4 + 2] = npc[i].z; rows[r][w4 + 3] = npc[i].w;
+  }
+  scs[tid] = nsc;
   float2 sb[4];
 #pragma unroll
   for (int r = 0; r < 4; ++r) sb[r] = nsb[r];
+  __syncthreads();
   fetch(chunk + gridDim.x);                              // in flight during this chunk's MMAs
   float sc[2][4];          // [tile][row g: queries 2c, 2c+1; row g + 8: queries 2c, 2c+1]
 #pragma unroll
@@ -417,9 +427,9 @@ __global__ void __launch_bounds__(kAttChunk, BITS == 8 ? 2 : 3) attend_scores_mm
     for (int j = 0; j < 4; ++j) sc[tl][j] = 0.f;
 #pragma unroll
   for (int tl = 0; tl < 2; ++tl) {
-    const int la = tl * 16 + g, lb = la + 8;           // lanes that hold rows g and g + 8 of this tile
-    const uint32_t sxa = __shfl_sync(0xffffffffu, scw.x, la), sya = __shfl_sync(0xffffffffu, scw.y, la);
-    const uint32_t sxb = __shfl_sync(0xffffffffu, scw.x, lb), syb = __shfl_sync(0xffffffffu, scw.y, lb);
+    const uint32_t *ra = rows[warp * 32 + tl * 16 + g], *rb = rows[warp * 32 + tl * 16 + g + 8];      // rows g and g + 8 of this tile
+    const uint2 sa = scs[warp * 32 + tl * 16 + g], sbw = scs[warp * 32 + tl * 16 + g + 8];
+    const uint32_t sxa = sa.x, sya = sa.y, sxb = sbw.x, syb = sbw.y;
 #pragma unroll
     for (int gq = 0; gq < 4; ++gq) {
       float d[4] = {0.f, 0.f, 0.f, 0.f};
@@ -428,27 +438,19 @@ __global__ void __launch_bounds__(kAttChunk, BITS == 8 ? 2 : 3) attend_scores_mm
         const int s8 = gq * 2 + s2;
         uint32_t a[4];
         if constexpr (BITS == 8) {            // 16 bits at bit 128 s2 + 16 c: word 4 s2 + (c >> 1), half c & 1; + 8 columns: two words on
-          const int w0 = gq * 8 + s2 * 4;
-          const uint32_t a00 = __shfl_sync(0xffffffffu, row[w0], la), a01 = __shfl_sync(0xffffffffu, row[w0 + 1], la);
-          const uint32_t a02 = __shfl_sync(0xffffffffu, row[w0 + 2], la), a03 = __shfl_sync(0xffffffffu, row[w0 + 3], la);
-          const uint32_t b00 = __shfl_sync(0xffffffffu, row[w0], lb), b01 = __shfl_sync(0xffffffffu, row[w0 + 1], lb);
-          const uint32_t b02 = __shfl_sync(0xffffffffu, row[w0 + 2], lb), b03 = __shfl_sync(0xffffffffu, row[w0 + 3], lb);
-          const int sh = 16 * (c & 1);
-          a[0] = att_pair_f16(((c & 2) ? a01 : a00) >> sh, 8); a[1] = att_pair_f16(((c & 2) ? b01 : b00) >> sh, 8);
-          a[2] = att_pair_f16(((c & 2) ? a03 : a02) >> sh, 8); a[3] = att_pair_f16(((c & 2) ? b03 : b02) >> sh, 8);
+          const int w0 = gq * 8 + s2 * 4 + (c >> 1), sh = 16 * (c & 1);
+          a[0] = att_pair_f16(ra[w0] >> sh, 8); a[1] = att_pair_f16(rb[w0] >> sh, 8);
+          a[2] = att_pair_f16(ra[w0 + 2] >> sh, 8); a[3] = att_pair_f16(rb[w0 + 2] >> sh, 8);
         } else if constexpr (BITS == 4) {     // 8 bits at bit 64 s2 + 8 c: word 2 s2, byte c; + 8 columns: the next word
           const int w0 = gq * 4 + s2 * 2;
-          const uint32_t a0 = __shfl_sync(0xffffffffu, row[w0], la), a1 = __shfl_sync(0xffffffffu, row[w0 + 1], la);
-          const uint32_t b0 = __shfl_sync(0xffffffffu, row[w0], lb), b1 = __shfl_sync(0xffffffffu, row[w0 + 1], lb);
-          a[0] = att_pair_f16(a0 >> (8 * c), 4); a[1] = att_pair_f16(b0 >> (8 * c), 4);
-          a[2] = att_pair_f16(a1 >> (8 * c), 4); a[3] = att_pair_f16(b1 >> (8 * c), 4);
+          a[0] = att_pair_f16(ra[w0] >> (8 * c), 4); a[1] = att_pair_f16(rb[w0] >> (8 * c), 4);
+          a[2] = att_pair_f16(ra[w0 + 1] >> (8 * c), 4); a[3] = att_pair_f16(rb[w0 + 1] >> (8 * c), 4);
         } else if constexpr (BITS == 2) {     // 4 bits at bit 32 s2 + 4 c: word s2, nibble c; + 8 columns: 16 bits on
-          const int w0 = gq * 2 + s2;
-          const uint32_t a0 = __shfl_sync(0xffffffffu, row[w0], la), b0 = __shfl_sync(0xffffffffu, row[w0], lb);
+          const uint32_t a0 = ra[gq * 2 + s2], b0 = rb[gq * 2 + s2];
           a[0] = att_pair_f16(a0 >> (4 * c), 2); a[1] = att_pair_f16(b0 >> (4 * c), 2);
           a[2] = att_pair_f16(a0 >> (4 * c + 16), 2); a[3] = att_pair_f16(b0 >> (4 * c + 16), 2);
         } else {                              // 2 bits at bit 16 s2 + 2 c of the group's single word; + 8 columns: 8 bits on
-          const uint32_t a0 = __shfl_sync(0xffffffffu, row[gq], la), b0 = __shfl_sync(0xffffffffu, row[gq], lb);
+          const uint32_t a0 = ra[gq], b0 = rb[gq];
           a[0] = att_pair_f16(a0 >> (16 * s2 + 2 * c), 1); a[1] = att_pair_f16(b0 >> (16 * s2 + 2 * c), 1);
           a[2] = att_pair_f16(a0 >> (16 * s2 + 2 * c + 8), 1); a[3] = att_pair_f16(b0 >> (16 * s2 + 2 * c + 8), 1);
         }
