@@ -242,7 +242,11 @@ def main():
     t0 = time.perf_counter()
     plans, planned_bytes = B.jolt_plan(K, V, gs, cache_bytes / ratio, opts)
     torch.cuda.synchronize()
-    plan_ms = (time.perf_counter() - t0) * 1e3
+    plan_ms = (time.perf_counter() - t0) * 1e3          # first call: includes one-time workspace and module set-up
+    t0 = time.perf_counter()
+    B.jolt_plan(K, V, gs, cache_bytes / ratio, opts)
+    torch.cuda.synchronize()
+    plan_ms_warm = (time.perf_counter() - t0) * 1e3
     Ko, Vo = torch.empty_like(K), torch.empty_like(V)
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
@@ -404,7 +408,7 @@ def main():
                                    + (f"randomized q={q}" if args.token_mode == "randomized" else "exact (converged block iteration)"),
                        "cache_bytes": cache_bytes, "compressed_bytes": planned_bytes, "achieved_ratio": cache_bytes / planned_bytes,
                        "rope_at_decode": bool(args.rope), "plan": plans, "l2": f"inputs ({cache_bytes / 1e6:.0f} MB) exceed L2; no flush"},
-            "compress_ms": tc, "decompress_ms": td, "plan_ms": plan_ms,
+            "compress_ms": tc, "decompress_ms": td, "plan_ms": plan_ms, "plan_ms_warm": plan_ms_warm,
             "compress_ms_min_med_max": [tc_all[0], tc_all[len(tc_all) // 2], tc_all[-1]],
             "decompress_ms_min_med_max": [td_all[0], td_all[len(td_all) // 2], td_all[-1]],
             "compress_gbs": world * cache_bytes / (tc * 1e-3) / 1e9, "decompress_gbs": world * cache_bytes / (td * 1e-3) / 1e9,
