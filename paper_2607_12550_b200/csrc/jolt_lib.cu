@@ -20,6 +20,7 @@
 #include "simt_gemm.cuh"
 #include "small_solvers.cuh"
 #include "block_jacobi.cuh"
+#include "cluster_jacobi.cuh"
 #include "rope.cuh"
 #include "attend.cuh"
 
@@ -30,8 +31,8 @@ thread_local std::string g_err;
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_eig_smem{1};
 long long *g_dbg_stamps = nullptr;   // device buffer for kernel cycle stamps (profiling aid)
-std::atomic<int> g_fast{15};  // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores,
-                              // bit 3: rotary embedding inside the decode kernel
+std::atomic<int> g_fast{31};  // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores,
+                              // bit 3: rotary embedding inside the decode kernel, bit 4: cluster-resident eigen-solver
 
 int fail(int code, const char *fmt, ...) {
   char buf[512];
@@ -330,7 +331,20 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
   // problems that fit one CTA's shared memory take the resident kernel, the rest the global-memory one
   std::vector<EigTask> small64, small32, big;
   std::vector<BJTask> bj;
+  std::vector<CholFactorTask> cf;
+  std::vector<CJTask> cj;                  // one launch: rows per lane follow the largest matrix
   for (auto &t : tasks) {
+    // singular values of B (w_sqrt): single-precision cluster solver; the mode-3 Gram, whose spectrum spans 1e6 and more
+    // when the cache has outlier channels, stays on the fp64 block solver
+    if (t.bjA && t.w_sqrt && t.n > 32 && t.n <= kCJMaxN && (g_fast.load() & 16)) {
+      // Cholesky factor in the block solver's scratch, then the cluster-resident one-sided Jacobi on its columns
+      cf.push_back({t.A, t.bjA, t.n, t.status});
+      CJTask c; memset(&c, 0, sizeof c);
+      c.L = t.bjA; c.n = t.n; c.U_out = t.U_out; c.ld_out = t.ld_out; c.r_out = t.r_out; c.w_out = t.w_out; c.w_sqrt = t.w_sqrt;
+      c.status = t.status; c.sweeps_out = t.bjDone;
+      cj.push_back(c);
+      continue;
+    }
     if (t.bjA && t.n > 32 && g_eig_smem.load() != 2) {
       BJTask b; memset(&b, 0, sizeof b);
       b.A_in = t.A; b.A = t.bjA; b.V = t.bjV; b.J = t.bjJ; b.off = t.bjOff; b.done = t.bjDone; b.ticket = (unsigned *)(t.bjDone + 1);
@@ -345,6 +359,27 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
     else if (eig_smem_bytes(t.n, 8) <= kSmemOptIn - 1024) small64.push_back(t);   // fp64 eigenvector accumulator fits
     else if (eig_smem_bytes(t.n, 4) <= kSmemOptIn - 1024) small32.push_back(t);
     else big.push_back(t);
+  }
+  if (!cf.empty()) {
+    const size_t off = P.push(cf);
+    const int n = (int)cf.size();
+    int cmn = 0;
+    for (auto &c : cf) cmn = std::max(cmn, c.n);
+    const size_t cshm = std::max(chol_factor_smem_bytes(kCholFactorSmemN), chol_factor_smem_bytes(cmn));
+    static bool cattr = false;
+    if (!cattr) { cudaFuncSetAttribute(chol_factor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemOptIn - 2048)); cattr = true; }
+    P.add(stage, [=](char *dev, cudaStream_t s) {
+      chol_factor_kernel<<<n, kCholFactorThreads, cshm, s>>>((const CholFactorTask *)(dev + off)); LAUNCHED();
+    });
+    static bool cjattr = false;
+    if (!cjattr) { cj_opt_in_smem(); cjattr = true; }
+    {
+      int mn = 0;
+      for (auto &c : cj) mn = std::max(mn, c.n);
+      const int nr = cj_rows_per_lane(mn), nt = (int)cj.size();
+      const size_t o2 = P.push(cj);
+      P.add(stage, [=](char *dev, cudaStream_t s) { cj_launch((const CJTask *)(dev + o2), nt, mn, nr, s); LAUNCHED(); });
+    }
   }
   if (!bj.empty()) {
     int max_nbe = 0, max_nP = 0;
@@ -2029,7 +2064,7 @@ extern "C" int jolt_debug_stamps(long long *host_out, int n) {
   return cudaMemcpy(host_out, g_dbg_stamps, sizeof(long long) * n, cudaMemcpyDeviceToHost) == cudaSuccess ? JOLT_OK : JOLT_ECUDA;
 }
 extern "C" int64_t jolt_launch_count(void) { return g_launches.load(); }
-extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled & 15); }
+extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled & 31); }
 extern "C" int jolt_last_stage_ms(float *out, int32_t cap, int32_t *n) {
   if (!out || !n) return fail(JOLT_EINVAL, "null argument");
   *n = std::min<int>(cap, kNumStages);
