@@ -5,6 +5,7 @@
 #include "tc_backbone.cuh"
 #include "tc_decode.cuh"
 #include "tc_gemm.cuh"
+#include "tc_orth.cuh"
 
 namespace {
 
@@ -210,7 +211,7 @@ inline void add_tok_tc(Program &P, int stage, std::vector<CellWork> &ws, const s
       if (src[i] == 2) { in = w.ufI ? w.Z : w.W; se = ilog2_floor((long long)c.N) / 2; }
       tc::SplitJob j;
       j.in = in; j.hi = w.Bhi; j.lo = w.Blo; j.batch = c.m; j.rows = kD; j.cols = c.k; j.ld_in = c.k;
-      j.kp = w.kp; j.scale_exp = se;
+      j.kp = w.kp; j.scale_exp = se; j.absmax = nullptr;
       sp.push_back(j);
     }
     std::vector<std::pair<int, int>> ch;
@@ -246,7 +247,7 @@ inline void add_feat_tc(Program &P, int stage, std::vector<CellWork> &ws) {
     const int se = ilog2_floor(c.T) / 2;
     if (w.split_ready != 1) {      // else the triangular solve of orth(S) has written the operand already
       tc::SplitJob j;
-      j.in = w.S; j.hi = w.Bhi; j.lo = w.Blo; j.batch = 1; j.rows = c.T; j.cols = c.k; j.ld_in = c.k; j.kp = w.kp; j.scale_exp = se;
+      j.in = w.S; j.hi = w.Bhi; j.lo = w.Blo; j.batch = 1; j.rows = c.T; j.cols = c.k; j.ld_in = c.k; j.kp = w.kp; j.scale_exp = se; j.absmax = nullptr;
       sp.push_back(j);
     }
     w.split_ready = 0;
@@ -298,6 +299,96 @@ inline void add_sketch_gen_tc(Program &P, int stage, std::vector<CellWork> &ws, 
     tc::gen_sketch_f16_kernel<<<dim3(148, n), 256, 0, s>>>((const tc::SketchJob *)(dev_t + off), stream_id, seed);
     LAUNCHED();
   });
+}
+
+// ------------------------------------------------------------------ CholeskyQR on tensor cores
+// Cells whose basis is already kept as the hi + lo operand of the sweeps (tensor-core cells with r_f = d, sketch
+// width up to OR_MAX_K) orthonormalise it there: Gram and Q = R L^-T are tcgen05 GEMMs, the Cholesky factor and its
+// inverse one fp64 CTA per cell.
+inline bool orth_tc_ok(const CellWork &w) {
+  return w.active && w.tc && w.ufI && w.c.k <= tc::OR_MAX_K && w.kp <= tc::OR_MAX_KP && w.c.T % 128 == 0 && w.orthPart != nullptr;
+}
+
+inline void add_orth_tc(Program &P, int stage, std::vector<CellWork> &ws, const std::vector<int> &idx, bool token_side, int passes,
+                        bool want_fp32) {
+  if (idx.empty()) return;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaFuncSetAttribute(tc::orth_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::OR_SMEM_LIMIT);
+    cudaFuncSetAttribute(tc::orth_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::OR_SMEM_LIMIT);
+    cudaFuncSetAttribute(tc::cholinv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::cholinv_smem_bytes(tc::kCholInvMaxN));
+    attr_done = true;
+  }
+  // the sweep left the raw basis as fp32 rows: measure its magnitude, split it into the operand layout
+  std::vector<tc::AbsMaxJob> am;
+  std::vector<tc::SplitJob> sp;
+  std::vector<tc::OrthCell> oc, oc_last;      // the fp32 rows of Q are only written by the last pass, and only if someone reads them
+  std::vector<tc::CholInvTask> ci;
+  int max_chunks = 0, max_tiles = 0, max_kp = 0, max_k = 0;
+  for (int i : idx) {
+    CellWork &w = ws[i];
+    const CellDesc &c = w.c;
+    const int rpp = token_side ? c.T : kD, panels = token_side ? 1 : c.m;
+    float *src = token_side ? w.S : w.Z;
+    unsigned *slot = w.orthMax + (w.orthMaxUsed++ % kOrthMaxSlots);
+    am.push_back({src, (long long)rpp * panels * c.k, slot});
+    tc::SplitJob j;
+    j.in = src; j.hi = w.Bhi; j.lo = w.Blo; j.batch = panels; j.rows = rpp; j.cols = c.k; j.ld_in = c.k; j.kp = w.kp; j.scale_exp = 0;
+    j.absmax = slot;
+    sp.push_back(j);
+    tc::OrthCell o;
+    memset(&o, 0, sizeof o);
+    {
+      const uint64_t dims[3] = {(uint64_t)rpp, (uint64_t)w.kp, (uint64_t)panels};
+      const uint64_t str[2] = {(uint64_t)rpp * 2, (uint64_t)w.kp * rpp * 2};
+      const uint32_t box[3] = {64, (uint32_t)w.kp, 1};
+      make_tmap_f16(&o.tmHi, w.Bhi, 3, dims, str, box);
+      make_tmap_f16(&o.tmLo, w.Blo, 3, dims, str, box);
+    }
+    {
+      const uint64_t dims[2] = {(uint64_t)w.kp, (uint64_t)w.kp};
+      const uint64_t str[1] = {(uint64_t)w.kp * 2};
+      const uint32_t box[2] = {64, (uint32_t)w.kp};
+      make_tmap_f16(&o.tmLhi, w.orthLhi, 2, dims, str, box);
+      make_tmap_f16(&o.tmLlo, w.orthLlo, 2, dims, str, box);
+    }
+    const int steps = panels * (rpp / 64);
+    o.part = w.orthPart; o.Lhi = w.orthLhi; o.Llo = w.orthLlo; o.l_exp = w.orthExp;
+    o.out32 = nullptr; o.ld = c.k; o.k = c.k; o.kp = w.kp; o.rpp = rpp; o.panels = panels;
+    o.n_chunks = (steps + tc::OR_STEPS_PER_CTA - 1) / tc::OR_STEPS_PER_CTA;
+    o.out_exp = ilog2_floor((long long)rpp * panels) / 2;
+    o.status = w.status;
+    oc.push_back(o);
+    o.out32 = want_fp32 ? src : nullptr;
+    oc_last.push_back(o);
+    ci.push_back({w.orthPart, o.n_chunks, w.kp, nullptr, c.k, w.orthLhi, w.orthLlo, w.orthExp, nullptr, w.status, 1e-10});
+    max_chunks = std::max(max_chunks, o.n_chunks);
+    max_tiles = std::max(max_tiles, panels * (rpp / 128));
+    max_kp = std::max(max_kp, w.kp); max_k = std::max(max_k, c.k);
+    w.split_ready = token_side ? 1 : 2;
+  }
+  const size_t o_am = P.push(am), o_oc = P.push(oc), o_ocl = P.push(oc_last), o_ci = P.push(ci);
+  const int n = (int)idx.size();
+  {
+    const size_t o_sp = P.push(sp);
+    P.add(stage, [=](char *dev_t, cudaStream_t s) {
+      tc::absmax_kernel<<<dim3(32, n), 256, 0, s>>>((const tc::AbsMaxJob *)(dev_t + o_am)); LAUNCHED();
+      tc::split_transpose_kernel<<<dim3(148, 1, n), 256, 0, s>>>((const tc::SplitJob *)(dev_t + o_sp)); LAUNCHED();
+    });
+  }
+  const uint32_t tile = (uint32_t)max_kp * 128u;
+  const int g_stages = std::max(2, std::min(6, (int)((tc::OR_SMEM_LIMIT - 16384 - 2048) / (2 * tile))));
+  const size_t g_smem = (size_t)g_stages * 2 * tile + 16384 + 1024 + 1024;
+  const size_t a_smem = (size_t)(4 + 2 * ((max_kp + 63) / 64)) * tile + 1024 + 1024;
+  const size_t c_smem = tc::cholinv_smem_bytes(max_k);
+  for (int pass = 0; pass < passes; ++pass) {
+    const size_t o_app = pass + 1 == passes ? o_ocl : o_oc;
+    P.add(stage, [=](char *dev_t, cudaStream_t s) {
+      tc::orth_gram_kernel<<<dim3(max_chunks, n), tc::OR_THREADS, g_smem, s>>>((const tc::OrthCell *)(dev_t + o_oc), g_stages); LAUNCHED();
+      tc::cholinv_kernel<<<n, tc::kCholInvThreads, c_smem, s>>>((const tc::CholInvTask *)(dev_t + o_ci)); LAUNCHED();
+      tc::orth_apply_kernel<<<dim3(max_tiles, n), tc::OR_THREADS, a_smem, s>>>((const tc::OrthCell *)(dev_t + o_app)); LAUNCHED();
+    });
+  }
 }
 
 }  // namespace

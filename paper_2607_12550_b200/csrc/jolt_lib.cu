@@ -21,6 +21,7 @@
 #include "small_solvers.cuh"
 #include "block_jacobi.cuh"
 #include "cluster_jacobi.cuh"
+#include "tc_orth.cuh"
 #include "rope.cuh"
 #include "attend.cuh"
 
@@ -31,8 +32,9 @@ thread_local std::string g_err;
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_eig_smem{1};
 long long *g_dbg_stamps = nullptr;   // device buffer for kernel cycle stamps (profiling aid)
-std::atomic<int> g_fast{31};  // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores,
-                              // bit 3: rotary embedding inside the decode kernel, bit 4: cluster-resident eigen-solver
+std::atomic<int> g_fast{63};  // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores,
+                              // bit 3: rotary embedding inside the decode kernel, bit 4: cluster-resident eigen-solver,
+                              // bit 5: CholeskyQR on tensor cores
 
 int fail(int code, const char *fmt, ...) {
   char buf[512];
@@ -331,14 +333,16 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
   // problems that fit one CTA's shared memory take the resident kernel, the rest the global-memory one
   std::vector<EigTask> small64, small32, big;
   std::vector<BJTask> bj;
-  std::vector<CholFactorTask> cf;
+  std::vector<CholFactorTask> cf;          // Cholesky factor for the cluster solver: work matrix in global memory (n > 152)
+  std::vector<tc::CholInvTask> cfs;        // ... in shared memory
   std::vector<CJTask> cj;                  // one launch: rows per lane follow the largest matrix
   for (auto &t : tasks) {
     // singular values of B (w_sqrt): single-precision cluster solver; the mode-3 Gram, whose spectrum spans 1e6 and more
     // when the cache has outlier channels, stays on the fp64 block solver
     if (t.bjA && t.w_sqrt && t.n > 32 && t.n <= kCJMaxN && (g_fast.load() & 16)) {
       // Cholesky factor in the block solver's scratch, then the cluster-resident one-sided Jacobi on its columns
-      cf.push_back({t.A, t.bjA, t.n, t.status});
+      if (t.n <= tc::kCholInvMaxN) cfs.push_back({nullptr, 0, 0, t.A, t.n, nullptr, nullptr, nullptr, t.bjA, t.status, 1e-13});
+      else cf.push_back({t.A, t.bjA, t.n, t.status});
       CJTask c; memset(&c, 0, sizeof c);
       c.L = t.bjA; c.n = t.n; c.U_out = t.U_out; c.ld_out = t.ld_out; c.r_out = t.r_out; c.w_out = t.w_out; c.w_sqrt = t.w_sqrt;
       c.status = t.status; c.sweeps_out = t.bjDone;
@@ -360,6 +364,18 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
     else if (eig_smem_bytes(t.n, 4) <= kSmemOptIn - 1024) small32.push_back(t);
     else big.push_back(t);
   }
+  if (!cfs.empty()) {
+    const size_t off = P.push(cfs);
+    const int n = (int)cfs.size();
+    int cmn = 0;
+    for (auto &c : cfs) cmn = std::max(cmn, c.k);
+    const size_t cshm = tc::cholinv_smem_bytes(cmn);
+    static bool cattr = false;
+    if (!cattr) { cudaFuncSetAttribute(tc::cholinv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::cholinv_smem_bytes(tc::kCholInvMaxN)); cattr = true; }
+    P.add(stage, [=](char *dev, cudaStream_t s) {
+      tc::cholinv_kernel<<<n, tc::kCholInvThreads, cshm, s>>>((const tc::CholInvTask *)(dev + off)); LAUNCHED();
+    });
+  }
   if (!cf.empty()) {
     const size_t off = P.push(cf);
     const int n = (int)cf.size();
@@ -371,6 +387,8 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
     P.add(stage, [=](char *dev, cudaStream_t s) {
       chol_factor_kernel<<<n, kCholFactorThreads, cshm, s>>>((const CholFactorTask *)(dev + off)); LAUNCHED();
     });
+  }
+  if (!cj.empty()) {
     static bool cjattr = false;
     if (!cjattr) { cj_opt_in_smem(); cjattr = true; }
     {
@@ -474,10 +492,14 @@ struct CellWork {      // device scratch of one cell
   bool skip_feat = false;    // no mode-3 Gram / eigen-solve needed
   int kp = 0;                // sketch width padded to a multiple of 16
   __half *Bhi = nullptr, *Blo = nullptr;
+  // CholeskyQR on tensor cores: Gram partials, L^-1 as fp16 hi + lo, its exponent, slots for measured magnitudes
+  float *orthPart = nullptr; __half *orthLhi = nullptr, *orthLlo = nullptr; int *orthExp = nullptr;
+  unsigned *orthMax = nullptr; int orthMaxUsed = 0;
   int split_ready = 0;       // 1 / 2: Bhi, Blo already hold the split of S / Z (written by the last triangular solve)
 };
 
 enum FactorMode { FM_RANDOMIZED = 0, FM_EXACT = 1, FM_INJECTED = 2 };
+constexpr int kOrthMaxSlots = 32;
 constexpr int kGramChunks = 32;   // row chunks of a tall Gram (fp64 partial per chunk, summed in order)
 
 // Scratch layout of one cell; run with b.base == nullptr to size it.
@@ -514,6 +536,12 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
         const size_t nb = std::max((size_t)c.m * w.kp * kD, (size_t)w.kp * T);
         w.Bhi = b.take<__half>(nb); w.Blo = b.take<__half>(nb);
         if (tok_segments(c.T) > 1) w.Zpart = b.take<float>((size_t)tok_segments(c.T) * c.m * kD * k);
+        if (w.ufI && k <= 152 && w.kp <= 160) {
+          const size_t steps = std::max((size_t)T / 64, (size_t)c.m * 2);
+          w.orthPart = b.take<float>(((steps + 7) / 8) * w.kp * w.kp);
+          w.orthLhi = b.take<__half>((size_t)w.kp * w.kp); w.orthLlo = b.take<__half>((size_t)w.kp * w.kp);
+          w.orthExp = b.take<int>(4); w.orthMax = b.take<unsigned>(kOrthMaxSlots);
+        }
       }
       w.Gs = b.take<double>(k * k); w.Lwork = k > (size_t)kCholSmemMaxN ? b.take<double>(k * (k + 1)) : nullptr;
       w.gpart = b.take<double>(kGramChunks * k * k); w.LT32 = b.take<float>(k * (k + 8)); w.invd = b.take<float>(k + 8);
@@ -582,7 +610,11 @@ void add_tall_gram(Program &P, int stage, const std::vector<TallGram> &jobs) {
 
 // orth(S) for every active cell by CholeskyQR2: twice {Gs = S^T S (fp64), Gs = L L^T, S <- S L^-T}.
 // token_side selects S (T rows) or Z (N rows); the result is left in the source buffer.
-void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side, int passes) {
+void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side, int passes, bool final_basis = false) {
+  std::vector<int> on_tc;
+  if (g_fast.load() & 32)
+    for (size_t i = 0; i < ws.size(); ++i) if (orth_tc_ok(ws[i])) on_tc.push_back((int)i);
+  add_orth_tc(P, stage, ws, on_tc, token_side, passes, final_basis);
   for (int pass = 0; pass < 2; ++pass) {
     // cls 0: Cholesky work matrix and L^T resident in shared memory (k <= kCholSmemMaxN); cls 1: both in global memory
     std::vector<TallGram> tg;
@@ -592,6 +624,7 @@ void add_orth(Program &P, int stage, std::vector<CellWork> &ws, bool token_side,
     if (pass >= passes) continue;          // the triangular solve works in place, so one pass is possible
     for (auto &w : ws) {
       if (!w.active) continue;
+      if ((g_fast.load() & 32) && orth_tc_ok(w)) continue;
       const int k = w.c.k, rows = token_side ? w.c.T : w.c.N;
       const int cls = k <= kCholSmemMaxN ? 0 : 1;
       float *buf = token_side ? w.S : w.Z;
@@ -759,6 +792,10 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
   if (act.empty()) return;
   const int na = (int)act.size();
   if (mode == FM_RANDOMIZED) {
+    std::vector<unsigned *> slots;
+    for (int i : act) if (ws[i].orthMax) slots.push_back(ws[i].orthMax);
+    if (!slots.empty())
+      P.add(ST_SKGEN, [=](char *, cudaStream_t s) { for (unsigned *p : slots) cudaMemsetAsync(p, 0, sizeof(unsigned) * kOrthMaxSlots, s); });
     std::vector<CellDesc> cd; std::vector<float *> om; std::vector<long long> cnt;
     for (int i : act) {
       if (ws[i].tc && ws[i].ufI) continue;
@@ -820,12 +857,12 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
     // only the range of the intermediate bases matters (one Cholesky-QR pass keeps them well conditioned);
     // the final basis is orthonormalised twice
     add_sketch(P, ST_SKETCH, ws, true);
-    add_orth(P, ST_ORTH, ws, true, power_iters == 0 ? 2 : 1);
+    add_orth(P, ST_ORTH, ws, true, power_iters == 0 ? 2 : 1, power_iters == 0);
     for (int it = 0; it < power_iters; ++it) {
       add_project(P, ST_POWER, ws);
       add_orth(P, ST_POWER, ws, false, 1);
       add_sketch(P, ST_POWER, ws, false);
-      add_orth(P, ST_POWER, ws, true, it + 1 == power_iters ? 2 : 1);
+      add_orth(P, ST_POWER, ws, true, it + 1 == power_iters ? 2 : 1, it + 1 == power_iters);
     }
     add_project(P, ST_PROJ, ws);          // Z now holds B^T (N x k)
     std::vector<TallGram> tgb; std::vector<EigTask> eg; std::vector<GemmTask> g2, g3;
@@ -2064,7 +2101,7 @@ extern "C" int jolt_debug_stamps(long long *host_out, int n) {
   return cudaMemcpy(host_out, g_dbg_stamps, sizeof(long long) * n, cudaMemcpyDeviceToHost) == cudaSuccess ? JOLT_OK : JOLT_ECUDA;
 }
 extern "C" int64_t jolt_launch_count(void) { return g_launches.load(); }
-extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled & 31); }
+extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled & 63); }
 extern "C" int jolt_last_stage_ms(float *out, int32_t cap, int32_t *n) {
   if (!out || !n) return fail(JOLT_EINVAL, "null argument");
   *n = std::min<int>(cap, kNumStages);

@@ -178,6 +178,7 @@ struct SplitJob {
   const float *in;      // [batch][rows][cols], pitch `ld_in`
   __half *hi, *lo;      // [batch][kp][rows]
   int batch, rows, cols, ld_in, kp, scale_exp;
+  const unsigned *absmax;   // optional: bit pattern of max |in| (measured on the device); the scale is then 2^-(exponent + 1)
 };
 
 __global__ void __launch_bounds__(256) split_transpose_kernel(const SplitJob *__restrict__ jobs) {
@@ -185,7 +186,8 @@ __global__ void __launch_bounds__(256) split_transpose_kernel(const SplitJob *__
   __shared__ float tile[32][33];
   const int tiles_r = (j.rows + 31) / 32, tiles_c = (j.kp + 31) / 32;
   const int per_batch = tiles_r * tiles_c;
-  const float sc = ldexpf(1.0f, j.scale_exp);
+  float sc = ldexpf(1.0f, j.scale_exp);
+  if (j.absmax) { const float mx = __uint_as_float(*j.absmax); sc = (mx > 0.f && isfinite(mx)) ? ldexpf(1.0f, -(ilogbf(mx) + 1)) : 1.0f; }
   for (int w = blockIdx.x; w < per_batch * j.batch; w += gridDim.x) {
     const int b = w / per_batch, t = w - b * per_batch;
     const int r0 = (t / tiles_c) * 32, c0 = (t % tiles_c) * 32;
