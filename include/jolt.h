@@ -255,8 +255,9 @@ int64_t jolt_launch_count(void);
  * kernels (decode, residual) and the tensor-core forms of jolt_attend's code streams, bit 1 = tcgen05 factor sweeps (sketch, projection), bit 2 = tcgen05 mode-3
  * Gram, bit 3 = rotary embedding inside the decode kernel (jolt_decompress_rope; otherwise a separate pass),
  * bit 4 = eigen-solver resident in a thread-block cluster (otherwise one launch per Jacobi round),
- * bit 5 = CholeskyQR of the range finder on tensor cores (otherwise fp64 SIMT Gram and row-wise triangular solve);
- * 63 (default) = all, where the shapes allow.  Returns the previous mask. */
+ * bit 5 = CholeskyQR of the range finder on tensor cores (otherwise fp64 SIMT Gram and row-wise triangular solve),
+ * bit 6 = factor sweeps with two output tiles per CTA (otherwise one);
+ * 127 (default) = all, where the shapes allow.  Returns the previous mask. */
 int jolt_set_fast_path(int enabled);
 
 /* Wall-clock-free per-stage device timing of the last compress / decompress on this thread

@@ -153,6 +153,38 @@ inline void launch_tc_gemm(Program &P, int stage, std::vector<tc::GemmCell> &cel
   });
 }
 
+template <int MODE>
+inline void launch_tc_gemm2(Program &P, int stage, std::vector<tc::Gemm2Cell> &cells) {
+  if (cells.empty()) return;
+  uint32_t max_stage = 0;
+  int gx = 0;
+  for (auto &c : cells) {
+    const uint32_t b_pitch = ((uint32_t)c.kp * 128u + 1023u) & ~1023u;
+    max_stage = std::max(max_stage, 32768u + (c.has_lo ? 2 * b_pitch : b_pitch));
+    gx = std::max(gx, MODE == tc::GM_TOK ? (c.T / 128 + 1) / 2 : c.m / 2);
+  }
+  const int n_stages = std::min(8, (int)((tc::GM_SMEM_LIMIT - 1536) / max_stage));
+  const size_t smem = (size_t)n_stages * max_stage + 1024 + 512;
+  static bool attr[3] = {false, false, false};
+  if (!attr[MODE]) {
+    cudaFuncSetAttribute(tc::tc_gemm2_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::GM_SMEM_LIMIT);
+    attr[MODE] = true;
+  }
+  const size_t off = P.push(cells);
+  const int n = (int)cells.size();
+  P.add(stage, [=](char *dev_t, cudaStream_t s) {
+    tc::tc_gemm2_kernel<MODE><<<dim3(gx, n), tc::GM_THREADS, smem, s>>>((const tc::Gemm2Cell *)(dev_t + off), n_stages);
+    LAUNCHED();
+  });
+}
+
+inline bool make_x_map4(CUtensorMap *tm, const CellDesc &c, uint32_t box_tok, uint32_t box_heads) {
+  const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)c.T, (uint64_t)c.n_heads, (uint64_t)(c.m / c.n_heads)};
+  const uint64_t str[3] = {(uint64_t)c.st * 2, (uint64_t)c.sh * 2, (uint64_t)c.sl * 2};
+  const uint32_t box[4] = {64, box_tok, box_heads, 1};
+  return make_tmap_f16(tm, c.X, 4, dims, str, box);
+}
+
 inline void launch_split(Program &P, int stage, const std::vector<tc::SplitJob> &jobs) {
   if (jobs.empty()) return;
   const size_t off = P.push(jobs);
@@ -195,9 +227,11 @@ inline void add_gram_tc(Program &P, int stage, std::vector<CellWork> &ws) {
 
 // S = sum_h X_h W_h for the tensor-core cells.  src: 0 = fp16 sketch already in Bhi, 1 = split W (fp32,
 // [h][128][k]), 2 = split Z (fp32, [h][128][k], orthonormal columns over N rows).
+inline bool orth_tc_ok(const CellWork &w);
 inline void add_tok_tc(Program &P, int stage, std::vector<CellWork> &ws, const std::vector<int> &src) {
   std::vector<tc::SplitJob> sp;
   std::vector<tc::GemmCell> gc;
+  std::vector<tc::Gemm2Cell> gc2;
   for (size_t i = 0; i < ws.size(); ++i) {
     CellWork &w = ws[i];
     if (!w.active || !w.tc) continue;
@@ -216,6 +250,22 @@ inline void add_tok_tc(Program &P, int stage, std::vector<CellWork> &ws, const s
     }
     std::vector<std::pair<int, int>> ch;
     sketch_chunks(w.kp, ch);
+    if (ch.size() == 1 && (g_fast.load() & 64)) {
+      // one column chunk: two token tiles per CTA share every operand tile
+      tc::Gemm2Cell g;
+      memset(&g, 0, sizeof g);
+      const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)w.kp, (uint64_t)c.m};
+      const uint64_t str[2] = {(uint64_t)kD * 2, (uint64_t)w.kp * kD * 2};
+      const uint32_t box[3] = {64, (uint32_t)w.kp, 1};
+      bool okm = make_x_map4(&g.tmX, c, 256, 1) && make_tmap_f16(&g.tmBhi, w.Bhi, 3, dims, str, box) &&
+                 make_tmap_f16(&g.tmBlo, w.Blo, 3, dims, str, box);
+      (void)okm;
+      g.C = w.S; g.ldc = c.k; g.ncols = c.k; g.kp = w.kp; g.has_lo = src[i] != 0; g.scale_exp = se;
+      g.m = c.m; g.n_heads = c.n_heads; g.T = c.T; g.status = w.status;
+      if (orth_tc_ok(w)) { g.absmax = w.orthMax + (w.orthMaxUsed % kOrthMaxSlots); w.absmax_ready = true; }
+      gc2.push_back(g);
+      continue;
+    }
     for (auto &cc : ch) {
       const int c0 = cc.first, kc = cc.second;
       if (c0 >= c.k) break;
@@ -234,12 +284,14 @@ inline void add_tok_tc(Program &P, int stage, std::vector<CellWork> &ws, const s
   }
   launch_split(P, stage, sp);
   launch_tc_gemm<tc::GM_TOK>(P, stage, gc);
+  launch_tc_gemm2<tc::GM_TOK>(P, stage, gc2);
 }
 
 // Z'_h = X_h^T Q for the tensor-core cells (Q = w.S, T x k with orthonormal columns).
 inline void add_feat_tc(Program &P, int stage, std::vector<CellWork> &ws) {
   std::vector<tc::SplitJob> sp;
   std::vector<tc::GemmCell> gc;
+  std::vector<tc::Gemm2Cell> gc2;
   std::vector<tc::SumJob> sums;
   for (auto &w : ws) {
     if (!w.active || !w.tc) continue;
@@ -253,6 +305,28 @@ inline void add_feat_tc(Program &P, int stage, std::vector<CellWork> &ws) {
     w.split_ready = 0;
     std::vector<std::pair<int, int>> ch;
     sketch_chunks(w.kp, ch);
+    if (ch.size() == 1 && c.n_heads % 2 == 0 && (g_fast.load() & 64)) {
+      // one column chunk: two heads of a layer per CTA share every tile of Q
+      tc::Gemm2Cell g;
+      memset(&g, 0, sizeof g);
+      const uint64_t dims[2] = {(uint64_t)c.T, (uint64_t)w.kp};
+      const uint64_t str[1] = {(uint64_t)c.T * 2};
+      const uint32_t box[2] = {64, (uint32_t)w.kp};
+      bool okm = make_x_map4(&g.tmX, c, 64, 2) && make_tmap_f16(&g.tmBhi, w.Bhi, 2, dims, str, box) &&
+                 make_tmap_f16(&g.tmBlo, w.Blo, 2, dims, str, box);
+      (void)okm;
+      g.ldc = c.k; g.ncols = c.k; g.kp = w.kp; g.has_lo = 1; g.scale_exp = se;
+      g.m = c.m; g.n_heads = c.n_heads; g.T = c.T; g.status = w.status;
+      const int nseg = tok_segments(c.T);
+      if (nseg == 1 && orth_tc_ok(w)) { g.absmax = w.orthMax + (w.orthMaxUsed % kOrthMaxSlots); w.absmax_ready = true; }
+      for (int sg = 0; sg < nseg; ++sg) {
+        g.C = nseg > 1 ? w.Zpart + (size_t)sg * c.m * kD * c.k : w.Zp;
+        g.t0 = sg * kTokSegment; g.n_tok = std::min(kTokSegment, c.T - g.t0);
+        gc2.push_back(g);
+      }
+      if (nseg > 1) sums.push_back({w.Zpart, w.Zp, (long long)c.m * kD * c.k, (long long)c.m * kD * c.k, nseg});
+      continue;
+    }
     for (auto &cc : ch) {
       const int c0 = cc.first, kc = cc.second;
       if (c0 >= c.k) break;
@@ -277,6 +351,7 @@ inline void add_feat_tc(Program &P, int stage, std::vector<CellWork> &ws) {
   }
   launch_split(P, stage, sp);
   launch_tc_gemm<tc::GM_FEAT>(P, stage, gc);
+  launch_tc_gemm2<tc::GM_FEAT>(P, stage, gc2);
   if (!sums.empty()) {
     const size_t off = P.push(sums);
     const int n = (int)sums.size();
@@ -331,7 +406,8 @@ inline void add_orth_tc(Program &P, int stage, std::vector<CellWork> &ws, const 
     const int rpp = token_side ? c.T : kD, panels = token_side ? 1 : c.m;
     float *src = token_side ? w.S : w.Z;
     unsigned *slot = w.orthMax + (w.orthMaxUsed++ % kOrthMaxSlots);
-    am.push_back({src, (long long)rpp * panels * c.k, slot});
+    if (!w.absmax_ready) am.push_back({src, (long long)rpp * panels * c.k, slot});      // else the sweep's epilogue measured it
+    w.absmax_ready = false;
     tc::SplitJob j;
     j.in = src; j.hi = w.Bhi; j.lo = w.Blo; j.batch = panels; j.rows = rpp; j.cols = c.k; j.ld_in = c.k; j.kp = w.kp; j.scale_exp = 0;
     j.absmax = slot;
@@ -368,11 +444,11 @@ inline void add_orth_tc(Program &P, int stage, std::vector<CellWork> &ws, const 
     w.split_ready = token_side ? 1 : 2;
   }
   const size_t o_am = P.push(am), o_oc = P.push(oc), o_ocl = P.push(oc_last), o_ci = P.push(ci);
-  const int n = (int)idx.size();
+  const int n = (int)idx.size(), n_am = (int)am.size();
   {
     const size_t o_sp = P.push(sp);
     P.add(stage, [=](char *dev_t, cudaStream_t s) {
-      tc::absmax_kernel<<<dim3(32, n), 256, 0, s>>>((const tc::AbsMaxJob *)(dev_t + o_am)); LAUNCHED();
+      if (n_am) { tc::absmax_kernel<<<dim3(32, n_am), 256, 0, s>>>((const tc::AbsMaxJob *)(dev_t + o_am)); LAUNCHED(); }
       tc::split_transpose_kernel<<<dim3(148, 1, n), 256, 0, s>>>((const tc::SplitJob *)(dev_t + o_sp)); LAUNCHED();
     });
   }

@@ -32,9 +32,9 @@ thread_local std::string g_err;
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_eig_smem{1};
 long long *g_dbg_stamps = nullptr;   // device buffer for kernel cycle stamps (profiling aid)
-std::atomic<int> g_fast{63};  // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores,
+std::atomic<int> g_fast{127};  // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores,
                               // bit 3: rotary embedding inside the decode kernel, bit 4: cluster-resident eigen-solver,
-                              // bit 5: CholeskyQR on tensor cores
+                              // bit 5: CholeskyQR on tensor cores, bit 6: two output tiles per CTA in the factor sweeps
 
 int fail(int code, const char *fmt, ...) {
   char buf[512];
@@ -494,7 +494,7 @@ struct CellWork {      // device scratch of one cell
   __half *Bhi = nullptr, *Blo = nullptr;
   // CholeskyQR on tensor cores: Gram partials, L^-1 as fp16 hi + lo, its exponent, slots for measured magnitudes
   float *orthPart = nullptr; __half *orthLhi = nullptr, *orthLlo = nullptr; int *orthExp = nullptr;
-  unsigned *orthMax = nullptr; int orthMaxUsed = 0;
+  unsigned *orthMax = nullptr; int orthMaxUsed = 0; bool absmax_ready = false;
   int split_ready = 0;       // 1 / 2: Bhi, Blo already hold the split of S / Z (written by the last triangular solve)
 };
 
@@ -2101,7 +2101,7 @@ extern "C" int jolt_debug_stamps(long long *host_out, int n) {
   return cudaMemcpy(host_out, g_dbg_stamps, sizeof(long long) * n, cudaMemcpyDeviceToHost) == cudaSuccess ? JOLT_OK : JOLT_ECUDA;
 }
 extern "C" int64_t jolt_launch_count(void) { return g_launches.load(); }
-extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled & 63); }
+extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled & 127); }
 extern "C" int jolt_last_stage_ms(float *out, int32_t cap, int32_t *n) {
   if (!out || !n) return fail(JOLT_EINVAL, "null argument");
   *n = std::min<int>(cap, kNumStages);
