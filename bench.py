@@ -114,6 +114,25 @@ def roof_time(flops, nbytes, pk):
     return max(flops / (pk["tensor"] * 1e12), nbytes / (pk["hbm"] * 1e9))
 
 
+# The plan jolt_plan gives for the c1 workload (seed 1, 2x budget, bits {0, 2, 4, 8}); the reference arm, which has no
+# GPU to plan with, times the oracle on this plan, and the GPU arm reports whether its own plan equals it.
+C1_PLAN = [(128, 128, 4), (96, 128, 8), (16, 48, 8), (96, 128, 8), (128, 128, 4), (96, 128, 8), (16, 64, 8), (96, 128, 8),
+           (128, 128, 4), (96, 128, 8), (128, 128, 4), (96, 128, 8), (16, 48, 8), (96, 128, 8), (128, 128, 4), (96, 128, 8)]
+
+
+def dram_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch of `kernel` on `workload`, from the table kept beside the ncu summaries
+    (profiles/dram_traffic.txt: kernel, workload, cells captured, bytes read, bytes written); scaled by the caller."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    for line in open(path):
+        f = line.split("#")[0].split()
+        if len(f) >= 5 and f[0] == kernel and f[1] == workload:
+            return {"cells": int(f[2]), "read": float(f[3]), "write": float(f[4])}
+    return None
+
+
 def run_reference(args):
     """The CPU oracle, as it stands, on a bounded sample of the same workload (rank 0 only)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -125,7 +144,7 @@ def run_reference(args):
     from paper_2607_12550_b200 import synth
     cfg = synth.CONFIGS["c1"]
     # sample: the K and the V cell of group 0, with plans typical of the 2x allocation
-    plans = {0: (128, 128, 4), 1: (112, 128, 8)}
+    plans = {0: C1_PLAN[0], 1: C1_PLAN[1]}
     cells = {w: synth.make_cell(cfg, 0, w).to(torch.float16).numpy() for w in (0, 1)}
     cell_bytes = cells[0].size * 2
     n_cells_total = 2 * cfg.n_groups
@@ -160,7 +179,8 @@ def run_reference(args):
             "warmup": args.warmup_ref, "ms_per_step": (tc + td) * 1e3 * n_cells_total / 2, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": "c1: GQA 32 layers / 4 per group, 8 KV heads, T=4096, d=128, fp16, 2x budget",
-                       "sample": "2 of 16 cells (group 0: K at (128,128,4), V at (112,128,8)); ms_per_step scaled to 16 cells"},
+                       "sample": f"2 of 16 cells (group 0: K at {C1_PLAN[0]}, V at {C1_PLAN[1]}, the plan jolt_plan gives this cache); "
+                                 "ms_per_step scaled to 16 cells", "plan": [list(p) for p in C1_PLAN]},
             "compress_gbs": sample_bytes / tc / 1e9, "decompress_gbs": sample_bytes / td / 1e9,
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": "group 0 K and V cells (2 of 16), numpy fp64"},
@@ -297,6 +317,23 @@ def main():
     tc, td = max_over_ranks(dist, [tc, td], "cuda")
     ms = tc + td
 
+    # per-kernel durations for the roofline entries: the same compress with one cell group, i.e. every stage for all
+    # cells before the next one starts, so that the library's CUDA-event stage timer (on the launching stream)
+    # attributes the call to its stages; not part of the timed steps above
+    lock = {}
+    prev_groups = B.set_stream_groups(1)
+    try:
+        n_lock = 3
+        for i in range(n_lock + 1):
+            h = B.jolt_compress(K, V, gs, plans, opts)
+            torch.cuda.synchronize()
+            if i:       # the first call warms the single-group path up
+                for k_, v_ in B.stage_ms().items():
+                    lock[k_] = lock.get(k_, 0.0) + v_ / n_lock
+            h.free()
+    finally:
+        B.set_stream_groups(prev_groups)
+
     # accuracy of the benchmarked configuration (mean relative Frobenius error over cells)
     errs = []
     for c in range(2 * ng):
@@ -386,9 +423,9 @@ def main():
     fd, bd = tot["decompress"]
     t_dec = stages.get("decode_rows", td)
     dec_bound = "hbm" if bd / (pk["hbm"] * 1e9) >= fd / (pk["tensor"] * 1e12) else "tensor"
-    # DRAM traffic of one launch: ncu capture of the first 2 groups (profiles/decode_kernel_config1_2groups.md:
-    # 60.4 MB read + 78.5 MB written for 4 of the 16 cells), scaled by the cells of this run
-    traffic = (60.440e6 + 78.180e6) * (2 * ng) / 4 if cfg.name == "c1" else None
+    # DRAM traffic of one launch: ncu capture of a few cells (profiles/dram_traffic.txt), scaled by the cells of this run
+    tr = dram_traffic("tc::decode_kernel", cfg.name)
+    traffic = (tr["read"] + tr["write"]) * (2 * ng) / tr["cells"] if tr else None
     if dec_bound == "hbm":
         ach = bd / (t_dec * 1e-3) / 1e9
         roofline = {"kernel": "tc::decode_kernel", "bound": "hbm", "achieved": ach, "peak": pk["hbm"], "unit": "GB/s",
@@ -400,9 +437,32 @@ def main():
                     "frac": ach / pk["tensor"], "traffic": traffic, "algorithmic_flops": fd, "kernel_ms": t_dec,
                     "peak_source": pk["source"] + " (MEASURED_PEAKS.json bf16_tflops, burst)"}
 
+    # compress: its largest GPU-filling kernel is the fused residual pass (tc::backbone_kernel<true>: X in, codes and
+    # scales out), HBM-bound; the factor sweeps (tc::tc_gemm2_kernel) read X once each and are bound by the tensor
+    # pipe once the dense operand is split in hi + lo (two MMAs per K step)
+    fr, br_ = tot["residual_quant"]
+    t_res = lock.get("residual_quant")
+    roof_c = None
+    if t_res:
+        tr = dram_traffic("tc::backbone_kernel<1>", cfg.name)
+        ach = br_ / (t_res * 1e-3) / 1e9
+        roof_c = {"kernel": "tc::backbone_kernel<1>", "bound": "hbm", "achieved": ach, "peak": pk["hbm"], "unit": "GB/s",
+                  "frac": ach / pk["hbm"], "traffic": (tr["read"] + tr["write"]) * (2 * ng) / tr["cells"] if tr else None,
+                  "algorithmic_bytes": br_, "kernel_ms": t_res,
+                  "peak_source": pk["source"] + " (MEASURED_PEAKS.json hbm_gbs)"}
+    roof_s = None
+    t_sw = lock.get("project")
+    if t_sw:
+        fs, bs = tot["project"]
+        # split operand: the sweep issues two MMAs per K step for every cell (the algorithmic count has one)
+        t_hbm, t_tc = bs / (pk["hbm"] * 1e9), 2 * fs / (pk["tensor"] * 1e12)
+        roof_s = {"kernel": "tc::tc_gemm2_kernel<FEAT> (projection sweep)", "bound": "tensor" if t_tc > t_hbm else "hbm",
+                  "achieved_gbs": bs / (t_sw * 1e-3) / 1e9, "achieved_tflops_issued": 2 * fs / (t_sw * 1e-3) / 1e12,
+                  "frac": max(t_hbm, t_tc) * 1e3 / t_sw, "kernel_ms": t_sw, "algorithmic_bytes": bs, "algorithmic_flops": fs}
+
     line = {"metric": METRIC, "value": job_throughput(world, cache_bytes, ms), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f16 operands, f32 accumulate (f64 small solvers)", "data": "synthetic",
+            "vs_baseline": None, "dtype": "f16 operands, f32 accumulate (f64 Cholesky, f32 Jacobi)", "data": "synthetic",
             "config": {"workload": f"{cfg.name}: {ng * cfg.layers_per_group} layers / {cfg.layers_per_group} per group, "
                                    f"{cfg.n_kv_heads} KV heads, T={cfg.seq_len}, d=128, fp16, budget {ratio}x, "
                                    + (f"randomized q={q}" if args.token_mode == "randomized" else "exact (converged block iteration)"),
@@ -415,7 +475,9 @@ def main():
             "compress_roofline_frac": t_roof_c * 1e3 / tc, "decompress_roofline_frac": t_roof_d * 1e3 / td,
             "compress_roofline_ms": t_roof_c * 1e3, "decompress_roofline_ms": t_roof_d * 1e3,
             "rel_frobenius_error": {"K": rel_k, "V": rel_v},
-            "stages_ms": stages, "roofline": roofline, "gpu_launches": launches, "clocks": clocks, "e2e": e2e}
+            "stages_ms": stages, "compress_stages_ms_one_group": lock, "roofline": roofline, "roofline_compress": roof_c,
+            "roofline_sweep": roof_s, "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
+            "same_plan_as_reference_arm": (cfg.name == "c1" and ng == cfg.n_groups and [tuple(p) for p in plans] == C1_PLAN)}
     if attend:
         line["attend"] = attend
 

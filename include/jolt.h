@@ -10,6 +10,13 @@
  * All work is issued on the CUDA stream passed in (a cudaStream_t cast to void*, NULL = default
  * stream); jolt_plan and jolt_compress synchronise that stream before they return (they read back
  * spectra / a status word), jolt_decompress only when the destination is host memory.
+ *
+ * Concurrency.  Scratch memory and kernel argument tables are one cached arena per device.  Calls may be issued on
+ * different streams: every call makes its stream wait (an event, no host synchronisation) for the last launch of the
+ * previous call that used the arena, so the GPU work of two library calls on one device never overlaps.  Calls from
+ * several host threads on one device must still be serialised by the caller (the event is recorded when a call
+ * returns; a second thread that enters in between would build its tables in the same arena).  jolt_decompress_static
+ * has a scratch array of its own and the rules stated there.
  */
 #ifndef JOLT_H
 #define JOLT_H
@@ -161,7 +168,8 @@ int jolt_decompress_rope(const jolt_handle *h, const jolt_layout *out_layout, vo
  *   contraction).  Scratch comes from the library's per-device workspace (grown on first use).  The first call on a
  *   handle also forms the projected cores P_h = fp16(G_h U_F^T) of all cells (m * r_t * 128 fp16 values per cell,
  *   about 5 % of the compressed size on the benchmark workload) in a device buffer that stays with the handle
- *   until jolt_free; later calls, on any stream, reuse them.  Errors: JOLT_EINVAL
+ *   until jolt_free; later calls, on any stream, reuse them (a first call that fails leaves nothing behind; the next
+ *   call forms them again).  Errors: JOLT_EINVAL
  *   (null / misaligned pointers, n_q out of range, wrong device), JOLT_EUNSUPPORTED (ranks that are not multiples
  *   of 8; sequences beyond about 3 million tokens), JOLT_ENOMEM, JOLT_ECUDA.  Asynchronous on `stream`.  Arithmetic:
  *   fp32; the contractions that run on the tensor cores take their fp32 operand as hi + lo fp16 (about 22 bits) and
@@ -200,7 +208,9 @@ int jolt_serialized_bytes(const jolt_handle *h, int64_t *bytes);
 int jolt_serialize(const jolt_handle *h, void *host_dst, int64_t cap, void *stream);
 int jolt_deserialize(const void *host_src, int64_t bytes, void *stream, jolt_handle **out);
 
-/* Release a handle and all buffers it owns.  NULL is accepted. */
+/* Release a handle and all buffers it owns.  NULL is accepted.  The compressed buffers are returned to the
+ * stream-ordered pool after the last call that read them (ordered on that call's stream; if that stream no longer
+ * exists, after the device has gone idle), so a decode that is still running keeps its data. */
 int jolt_free(jolt_handle *h);
 
 /* Stored bytes of the compressed cache: factors + core + packed codes + scales, i.e. Eq. (1) plus
@@ -259,6 +269,26 @@ int64_t jolt_launch_count(void);
  * bit 6 = factor sweeps with two output tiles per CTA (otherwise one);
  * 127 (default) = all, where the shapes allow.  Returns the previous mask. */
 int jolt_set_fast_path(int enabled);
+
+/* Number of cell groups whose factor stages jolt_compress runs side by side on internal streams (1..8, default 4):
+ * the small solvers between the sweeps are latency chains, which overlap with the GPU-filling kernels of other groups.
+ * 1 runs every stage for all cells before the next one starts (the setting under which jolt_last_stage_ms attributes
+ * the whole call to its stages).  Returns the previous value. */
+int jolt_set_stream_groups(int n);
+
+/* jolt_check_status -- device-side outcome of the last decode on this handle (jolt_decompress, jolt_decompress_rope,
+ * jolt_decompress_static; these are asynchronous and return before their kernels have run).  Every device-side wait of
+ * the kernels is bounded (a wait that runs out raises a status bit, the kernel drains and exits), and a quantisation step that is not finite in fp16 raises another.  Copies the handle's status
+ * words back on `stream`, synchronises that stream, and returns JOLT_OK, JOLT_ETIMEOUT or JOLT_ENUMERIC.  Decodes into
+ * host memory synchronise anyway and return this status themselves. */
+int jolt_check_status(const jolt_handle *h, void *stream);
+
+/* Test hook.  cycles > 0 replaces the limit of every bounded device-side wait (default 10^9 SM cycles, about half a
+ * second); skip_first_load != 0 makes the TMA thread of the two-tile sweep kernel leave out its first load, so that
+ * the consumer's wait runs out: the kernel must drain, release its tensor memory and report JOLT_ETIMEOUT through
+ * jolt_compress, and the next call on the same context must work.  cycles <= 0 and skip_first_load = 0 restore the
+ * defaults.  Applies to the current device. */
+int jolt_test_set_wait_limit(int64_t cycles, int32_t skip_first_load);
 
 /* Wall-clock-free per-stage device timing of the last compress / decompress on this thread
  * (milliseconds, CUDA events): out[0..n) in stage order, names via jolt_stage_name. */

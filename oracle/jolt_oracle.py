@@ -4,8 +4,7 @@ TEST INFRASTRUCTURE ONLY.  This module is the slow, obviously-correct statement 
 what the library computes.  It shares no code with the CUDA path, imports nothing
 from the package, and may be imported only by the tests, by the smoke check and by
 the benchmark's CPU-baseline leg.  Everything is numpy in float64 unless a passage
-below fixes a narrower type (fp16 storage of factors and scales, fp32 decision
-precision of the quantiser).
+below fixes a narrower type (fp16 storage of factors and scales).
 
 Each function names the passage of the paper it follows:
 
@@ -148,27 +147,30 @@ def fp16_round(x):
 
 
 def quantize_rows(Rp, bits: int, group: int = 32):
-    """Mid-rise symmetric quantiser on groups of `group` consecutive rotated features.
+    """Mid-rise symmetric quantiser on groups of `group` consecutive rotated features
+    (Sec. 4 "Rotated residual": the rotated residual is quantised uniformly at b bits, with a stored scale).
 
-    a = max |r'| over the group; Delta = fp16(a / 2^(b-1)); Delta == 0 -> all codes 2^(b-1);
-    otherwise u = clamp(floor(r' * (1/Delta)), -2^(b-1), 2^(b-1)-1) + 2^(b-1).
-    The decision (reciprocal, product, floor) is taken in fp32, the precision of the kernel.
+    a = max |r'| over the group; Delta = fp16(a / 2^(b-1)) (the stored scale, rounded to nearest even);
+    Delta == 0 -> all codes 2^(b-1); otherwise u = clamp(floor(r' / Delta), -2^(b-1), 2^(b-1) - 1) + 2^(b-1).
+    Everything but the rounding of the stored scale is float64: this is the definition, not any kernel's
+    arithmetic (a single-precision reciprocal-multiply evaluation of the same formula moves a code by one
+    only where r' / Delta lies within rounding distance of an integer; tests/test_oracle_pins.py bounds how often).
     Returns (codes uint8 [..., d], scales float16 [..., d/group]).
     """
     assert bits in (1, 2, 3, 4, 8)
+    Rp = np.asarray(Rp, dtype=np.float64)
     shp = Rp.shape
     d = shp[-1]
     assert d % group == 0
     g = Rp.reshape(shp[:-1] + (d // group, group))
     half = float(1 << (bits - 1))
-    a32 = np.abs(g).max(axis=-1).astype(np.float32)
+    a = np.abs(g).max(axis=-1)
     with np.errstate(over="ignore"):
-        delta16 = (a32 * np.float32(1.0 / half)).astype(np.float16)
-    delta32 = delta16.astype(np.float32)
-    zero = delta32 == 0
+        delta16 = (a / half).astype(np.float16)
+    delta = delta16.astype(np.float64)
+    zero = delta == 0
     with np.errstate(divide="ignore", over="ignore", invalid="ignore"):
-        inv = np.where(zero, np.float32(0), np.float32(1.0) / np.where(zero, np.float32(1), delta32)).astype(np.float32)
-        q = np.floor(g.astype(np.float32) * inv[..., None])
+        q = np.floor(g / np.where(zero, 1.0, delta)[..., None])
     q = np.clip(q, -half, half - 1.0) + half
     q = np.where(zero[..., None], half, q)
     return q.astype(np.uint8).reshape(shp), delta16

@@ -84,6 +84,9 @@ lib.jolt_release_workspace.argtypes = []
 lib.jolt_launch_count.argtypes = []
 lib.jolt_launch_count.restype = C.c_int64
 lib.jolt_set_fast_path.argtypes = [C.c_int]
+lib.jolt_set_stream_groups.argtypes = [C.c_int]
+lib.jolt_check_status.argtypes = [_vp, _vp]
+lib.jolt_test_set_wait_limit.argtypes = [C.c_int64, C.c_int32]
 lib.jolt_last_stage_ms.argtypes = [C.POINTER(C.c_float), C.c_int32, C.POINTER(C.c_int32)]
 lib.jolt_stage_name.argtypes = [C.c_int32]
 lib.jolt_stage_name.restype = C.c_char_p
@@ -336,6 +339,21 @@ def set_fast_path(enabled) -> int:
     if enabled is True:
         enabled = 127
     return lib.jolt_set_fast_path(int(enabled))
+
+
+def set_stream_groups(n: int) -> int:
+    """Number of cell groups jolt_compress runs side by side (1 = stage by stage); returns the previous value."""
+    return lib.jolt_set_stream_groups(int(n))
+
+
+def check_status(handle: "Handle", stream=None):
+    """Device-side outcome of the last decode on the handle (synchronises the stream); raises JoltError on failure."""
+    _check(lib.jolt_check_status(handle.ptr, _stream_ptr(stream)))
+
+
+def set_test_wait_limit(cycles: int = 0, skip_first_load: bool = False):
+    """Test hook of the bounded device-side waits; see include/jolt.h."""
+    _check(lib.jolt_test_set_wait_limit(int(cycles), 1 if skip_first_load else 0))
 
 
 def release_workspace():

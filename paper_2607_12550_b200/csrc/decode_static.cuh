@@ -4,8 +4,9 @@
 // memory to its own pool and forbids further driver allocations, a thread inside a region where a
 // device allocation would synchronise the whole context, or a host process whose allocator hooks
 // reject anything outside start-up.  For them this entry point keeps ALL of its scratch (the per-head
-// projected core, the fp32 backbone tile buffer, the status words and the kernel argument tables) in
-// one fixed array that is part of the loaded library image.
+// projected core, the fp32 backbone tile buffer and the kernel argument tables) in one fixed array that
+// is part of the loaded library image.  The status words its kernels write are the handle's own (made
+// with the handle), so a numerical failure seen by these kernels is reported by jolt_check_status.
 #pragma once
 
 namespace {
@@ -50,12 +51,12 @@ extern "C" int jolt_decompress_static(const jolt_handle *H, const jolt_layout *L
   const int nc = (int)H->cells.size();
   const size_t esz = L->dtype == JOLT_F16 ? 2 : 4;
 
-  // size the scratch before touching the GPU: status words, per cell P (fp16) and the fp32 backbone
+  // size the scratch before touching the GPU: per cell P (fp16) and the fp32 backbone (the status words live with the
+  // handle, allocated when it was made, so that jolt_check_status can report what these kernels saw)
   std::vector<CellWork> ws(nc);
   size_t work_bytes = 0;
   {
     Bump b;
-    b.take<int>(4 * (size_t)nc);
     for (int i = 0; i < nc; ++i) { ws[i].c = H->cells[i].c; ws[i].active = false; carve(b, ws[i], FM_INJECTED, true); }
     work_bytes = (b.off + 255) & ~(size_t)255;
   }
@@ -65,7 +66,7 @@ extern "C" int jolt_decompress_static(const jolt_handle *H, const jolt_layout *L
   if ((rc = static_scratch_address(dev, &base))) return rc;
   Bump b;
   b.base = base;
-  int *d_status = b.take<int>(4 * (size_t)nc);
+  int *d_status = H->d_status;
   for (int i = 0; i < nc; ++i) { ws[i].status = d_status + 4 * i; carve(b, ws[i], FM_INJECTED, true); }
 
   Program P;
@@ -98,8 +99,9 @@ extern "C" int jolt_decompress_static(const jolt_handle *H, const jolt_layout *L
   if (total > kStaticScratchBytes)
     return fail(JOLT_EINVAL, "cache needs %zu bytes of decode scratch, the static scratch holds %zu", total, kStaticScratchBytes);
   char *d_tab = base + work_bytes;
-  // the array keeps the previous call's contents: only the status words must start at zero (every other
-  // region is fully written before it is read)
+  // the array keeps the previous call's contents; every region of it is fully written before it is read.  The status
+  // words (the handle's) start at zero.
+  H->last_stream = st;
   CU(cudaMemsetAsync(d_status, 0, sizeof(int) * 4 * nc, st));
   if (!P.host.empty()) CU(cudaMemcpyAsync(d_tab, P.host.data(), P.host.size(), cudaMemcpyHostToDevice, st));
   for (auto &s : P.steps) s.run(d_tab, st);

@@ -31,7 +31,10 @@ namespace jolt {
 thread_local std::string g_err;
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_eig_smem{1};
+#ifdef JOLT_DEBUG
 long long *g_dbg_stamps = nullptr;   // device buffer for kernel cycle stamps (profiling aid)
+#endif
+std::atomic<int> g_n_cell_groups{4};        // concurrent cell groups of jolt_compress (jolt_set_stream_groups)
 std::atomic<int> g_fast{127};  // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores,
                               // bit 3: rotary embedding inside the decode kernel, bit 4: cluster-resident eigen-solver,
                               // bit 5: CholeskyQR on tensor cores, bit 6: two output tiles per CTA in the factor sweeps
@@ -92,6 +95,23 @@ static int ws_reserve(int dev, size_t bytes, void **out) {
   }
   *out = w.base;
   return JOLT_OK;
+}
+
+// The workspace and the argument-table arena are shared by every call on a device.  A call makes its stream wait for
+// the last launch of the previous call that used them (whatever stream that ran on) and leaves an event behind.
+static cudaEvent_t g_arena_ev[64] = {};
+static int arena_acquire(int dev, cudaStream_t st) {
+  std::lock_guard<std::mutex> lk(g_ws_mu);
+  if (!g_arena_ev[dev]) {
+    if (cudaEventCreateWithFlags(&g_arena_ev[dev], cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); g_arena_ev[dev] = nullptr; return fail(JOLT_ECUDA, "event"); }
+    return JOLT_OK;        // first use: nothing to wait for
+  }
+  if (cudaStreamWaitEvent(st, g_arena_ev[dev], 0) != cudaSuccess) { cudaGetLastError(); return fail(JOLT_ECUDA, "cudaStreamWaitEvent"); }
+  return JOLT_OK;
+}
+static void arena_release(int dev, cudaStream_t st) {
+  std::lock_guard<std::mutex> lk(g_ws_mu);
+  if (g_arena_ev[dev]) { if (cudaEventRecord(g_arena_ev[dev], st) != cudaSuccess) cudaGetLastError(); }
 }
 
 struct Bump {
@@ -212,6 +232,8 @@ struct jolt_handle {
   uint64_t seed = 0;
   int64_t stored_bytes = 0;
   bool subspace = false;     // token factors came from the converged block iteration (exact mode, large T)
+  int *d_status = nullptr;   // 4 words per cell, written by the decode kernels of the last call on this handle (jolt_check_status)
+  mutable cudaStream_t last_stream = nullptr;   // stream of the last call that read the handle's buffers (jolt_free orders after it)
   // jolt_attend: P_h = fp16(G_h U_F^T) of every cell, formed on the first call and kept until jolt_free
   mutable std::mutex att_mu;
   mutable __half *att_P = nullptr;
@@ -355,7 +377,6 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
       b.n = t.n; b.nbe = (((t.n + kBJBlock - 1) / kBJBlock) + 1) & ~1; b.nP = b.nbe * kBJBlock;
       b.w = t.w; b.U_out = t.U_out; b.ld_out = t.ld_out; b.r_out = t.r_out; b.w_out = t.w_out; b.w_sqrt = t.w_sqrt; b.status = t.status;
       b.tol = kBJTol;
-      if (const char *e = getenv("JOLT_BJ_TOL")) b.tol = atof(e);      // experiments only
       bj.push_back(b);
       continue;
     }
@@ -417,11 +438,6 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
       cfg.gridDim = dim3(gx + np, n); cfg.blockDim = dim3(kBJThreads); cfg.stream = s; cfg.attrs = &pdl; cfg.numAttrs = 1;
       for (int step = 0; step <= n_steps; ++step) { cudaLaunchKernelEx(&cfg, bj_round_kernel, d, step, n_steps, gx); LAUNCHED(); }
       bj_finish_kernel<<<n, 256, 0, s>>>(d, n_steps & 1); LAUNCHED();
-      if (getenv("JOLT_DEBUG_EIG")) {
-        cudaStreamSynchronize(s);
-        for (auto &b : copy) { double o[4]; int dn; cudaMemcpy(o, b.off, 32, cudaMemcpyDeviceToHost); cudaMemcpy(&dn, b.done, 4, cudaMemcpyDeviceToHost);
-          fprintf(stderr, "[jolt] bj n=%d nbe=%d last_off=%g total=%g done=%d rounds=%g\n", b.n, b.nbe, o[2], o[1], dn, o[3]); }
-      }
     });
   }
   static bool attr_done = false;
@@ -983,7 +999,6 @@ int run_program(Program &P, char *d_tables, cudaStream_t st, bool timed = true) 
 
 // Side streams on which independent groups of cells run their (latency-bound) factor stages concurrently.
 constexpr int kMaxGroups = 8;
-constexpr int kDefaultGroups = 4;
 struct GroupStreams { bool have = false; cudaStream_t s[kMaxGroups]; cudaEvent_t fork, join[kMaxGroups]; };
 GroupStreams g_groups[64];
 GroupStreams *group_streams(int dev) {
@@ -1003,8 +1018,7 @@ GroupStreams *group_streams(int dev) {
 // Cells whose factor stages may run side by side.  Cells that need the feature eigen-solve (the longest chain)
 // and the others never share a group.
 int assign_groups(const std::vector<CellWork> &ws, std::vector<int> &group) {
-  int want = kDefaultGroups;
-  if (const char *e = getenv("JOLT_GROUPS")) want = std::max(1, std::min(kMaxGroups, atoi(e)));
+  const int want = std::max(1, std::min(kMaxGroups, g_n_cell_groups.load()));
   group.assign(ws.size(), -1);
   int n_active = 0, n_long = 0;
   for (auto &w : ws) if (w.active) { ++n_active; if (!w.ufI) ++n_long; }
@@ -1132,9 +1146,13 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   if (out) *out = nullptr;
   if (!out || !plan || !K || !V) return fail(JOLT_EINVAL, "null argument");
   int rc;
+#ifdef JOLT_DEBUG
   const bool dbg = getenv("JOLT_DEBUG_TIMING") != nullptr;
   auto t_start = std::chrono::steady_clock::now();
   auto lap = [&](const char *what) { if (dbg) { auto n = std::chrono::steady_clock::now(); fprintf(stderr, "[jolt] %s: %.3f ms\n", what, std::chrono::duration<double, std::milli>(n - t_start).count()); t_start = n; } };
+#else
+  auto lap = [](const char *) {};
+#endif
   if ((rc = check_layout(L)) || (rc = check_options(o)) || (rc = check_device_alignment(L, K, V))) return rc;
   const bool injected = inUT != nullptr || inUF != nullptr;
   if (injected && (!inUT || !inUF)) return fail(JOLT_EINVAL, "both factor arrays are needed");
@@ -1182,7 +1200,12 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
       if (cudaMallocAsync(&H->blob, H->blob_bytes, st) != cudaSuccess) { cudaGetLastError(); return fail(JOLT_ENOMEM, "compressed cache of %zu bytes", H->blob_bytes); }
     }
   }
-  auto free_blob = [&]() { cudaFreeAsync(H->blob, st); H->blob = nullptr; };
+  if (cudaMalloc(&H->d_status, sizeof(int) * 4 * (size_t)nc) != cudaSuccess) {
+    cudaGetLastError(); cudaFreeAsync(H->blob, st); H->blob = nullptr; H->d_status = nullptr;
+    return fail(JOLT_ENOMEM, "status words");
+  }
+  auto free_blob = [&]() { cudaFreeAsync(H->blob, st); H->blob = nullptr; cudaFree(H->d_status); H->d_status = nullptr; };
+  H->last_stream = st;
   lap("validate+blob");
 
   // ---- workspace
@@ -1330,8 +1353,10 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   lap("residual program");
 
   // ---- run
+  if ((rc = arena_acquire(dev, st))) { free_blob(); return rc; }
   g_timer.begin(st);
   cudaError_t ce = cudaMemsetAsync(d_status, 0, sizeof(int) * 4 * nc, st);
+  if (ce == cudaSuccess) ce = cudaMemsetAsync(H->d_status, 0, sizeof(int) * 4 * nc, st);
   if (subspace) for (int i = 0; i < nc && ce == cudaSuccess; ++i) ce = cudaMemsetAsync(H->cells[i].e, 0, 4 * sizeof(int), st);
   for (int i = 0; i < nc && ce == cudaSuccess; ++i)
     if (cells[i].r_t == 0 || cells[i].r_f == kD || injected) ce = cudaMemsetAsync(H->cells[i].lam, 0, sizeof(float) * kD, st);
@@ -1365,19 +1390,24 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     // enqueue the groups' steps round-robin, so every side stream has work from the start
     size_t max_steps = 0;
     for (int g = 0; g < n_groups; ++g) max_steps = std::max(max_steps, PG[g].steps.size());
+#ifdef JOLT_DEBUG
     const bool tl = getenv("JOLT_DEBUG_TIMELINE") != nullptr;      // per-group stage boundaries, printed after the call
     struct TL { int g, stage; cudaEvent_t ev; };
     std::vector<TL> tls;
     cudaEvent_t tl0 = nullptr;
     if (tl) { cudaEventCreate(&tl0); cudaEventRecord(tl0, st); }
+#endif
     for (size_t si = 0; si < max_steps && ce == cudaSuccess; ++si)
       for (int g = 0; g < n_groups; ++g)
         if (si < PG[g].steps.size()) {
           PG[g].steps[si].run((char *)d_tab + tab_off[g], gs->s[g]);
+#ifdef JOLT_DEBUG
           if (tl && (si + 1 == PG[g].steps.size() || PG[g].steps[si + 1].stage != PG[g].steps[si].stage)) {
             TL t{g, PG[g].steps[si].stage, nullptr}; cudaEventCreate(&t.ev); cudaEventRecord(t.ev, gs->s[g]); tls.push_back(t);
           }
+#endif
         }
+#ifdef JOLT_DEBUG
     if (tl) {
       cudaDeviceSynchronize();
       for (int g = 0; g < n_groups; ++g) {
@@ -1388,6 +1418,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
       for (auto &t : tls) cudaEventDestroy(t.ev);
       cudaEventDestroy(tl0);
     }
+#endif
     if (ce == cudaSuccess) ce = cudaGetLastError();
     for (int g = 0; g < n_groups && ce == cudaSuccess; ++g) {
       ce = cudaEventRecord(gs->join[g], gs->s[g]);
@@ -1397,6 +1428,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     g_timer.mark(ST_FACT, st);
   }
   if ((rc = run_program(P, (char *)d_tab + tab_off.back(), st))) { free_blob(); return rc; }
+  arena_release(dev, st);
   lap("launches");
   std::vector<int> hstat(4 * nc);
   ce = cudaMemcpyAsync(hstat.data(), d_status, sizeof(int) * 4 * nc, cudaMemcpyDeviceToHost, st);
@@ -1456,10 +1488,10 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
   void *ws_base = nullptr;
   char *stage_K = nullptr, *stage_V = nullptr;
   int *d_status = nullptr;
+  d_status = H->d_status;          // the handle's own words: jolt_check_status reads them after the call
   for (int pass = 0; pass < 2; ++pass) {
     Bump b;
     b.base = (char *)ws_base;
-    d_status = b.take<int>(4 * (size_t)nc);
     if (L->mem_space == JOLT_MEM_HOST) { stage_K = b.take<char>(span); stage_V = b.take<char>(span); }
     if (n_rope_fused) rope_tab = b.take<float2>((size_t)(kD / 2) * L->seq_len);
     for (int i = 0; i < nc; ++i) {
@@ -1491,7 +1523,9 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
       b.out = obase; b.out_dtype = L->dtype == JOLT_F16 ? DT_F16 : DT_F32;
       b.osl = L->stride_layer; b.osh = L->stride_head; b.ost = L->stride_token;
       b.tma_out = 0;
+#ifdef JOLT_DEBUG
       b.dbg = g_dbg_stamps;
+#endif
       b.rope = rope_fused[i] ? rope_tab : nullptr;
       if (L->dtype == JOLT_F16 && L->stride_token % 8 == 0 && L->stride_head % 8 == 0 && L->stride_layer % 8 == 0 &&
           ((uintptr_t)obase % 16 == 0)) {
@@ -1560,17 +1594,37 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
   }
   void *d_tab = nullptr;
   if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
+  if ((rc = arena_acquire(dev, st))) return rc;
+  H->last_stream = st;
   g_timer.begin(st);
   CU(cudaMemsetAsync(d_status, 0, sizeof(int) * 4 * nc, st));
   if ((rc = run_program(P, (char *)d_tab, st))) return rc;
   if (L->mem_space == JOLT_MEM_HOST) {
+    std::vector<int> hstat(4 * (size_t)nc);
     CU(cudaMemcpyAsync(Kout, stage_K, span, cudaMemcpyDeviceToHost, st));
     CU(cudaMemcpyAsync(Vout, stage_V, span, cudaMemcpyDeviceToHost, st));
+    CU(cudaMemcpyAsync(hstat.data(), d_status, sizeof(int) * 4 * nc, cudaMemcpyDeviceToHost, st));
+    arena_release(dev, st);
     g_timer.mark(ST_OUT, st);
     CU(cudaStreamSynchronize(st));
     g_timer.finish();
+    return status_to_code(hstat);     // a host destination synchronises anyway: the device status comes back with it
   }
+  arena_release(dev, st);
   return JOLT_OK;
+}
+
+extern "C" int jolt_check_status(const jolt_handle *H, void *stream) {
+  if (!H) return fail(JOLT_EINVAL, "null argument");
+  if (!H->d_status) return JOLT_OK;
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
+  if (dev != H->device) return fail(JOLT_EINVAL, "handle belongs to device %d, current device is %d", H->device, dev);
+  std::vector<int> hstat(4 * H->cells.size());
+  cudaStream_t st = (cudaStream_t)stream;
+  CU(cudaMemcpyAsync(hstat.data(), H->d_status, sizeof(int) * hstat.size(), cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  return status_to_code(hstat);
 }
 
 extern "C" int jolt_decompress(const jolt_handle *H, const jolt_layout *L, void *Kout, void *Vout, void *stream) {
@@ -1641,9 +1695,18 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
   const int p_blocks = (m_max * std::max(krt, vrt) + kAttPRows - 1) / kAttPRows;
   if (shm_comb > 48 * 1024) return fail(JOLT_EUNSUPPORTED, "sequence of %d tokens: the chunk merge needs %zu bytes of shared memory", T, shm_comb);
   // the projected cores do not depend on the queries: formed by the first call on this handle, kept with it
+  // The mutex is held until the first call has issued the kernel that forms the cores and recorded `att_ready`; a
+  // call that fails before that point leaves no half-initialised state behind.
   bool first_call = false;
+  std::unique_lock<std::mutex> att_lk(H->att_mu);
+  auto att_reset = [&]() {
+    if (first_call) {
+      cudaDeviceSynchronize();
+      if (H->att_P) { cudaFree(H->att_P); H->att_P = nullptr; }
+      if (H->att_ready) { cudaEventDestroy(H->att_ready); H->att_ready = nullptr; }
+    }
+  };
   {
-    std::lock_guard<std::mutex> lk(H->att_mu);
     if (!H->att_P) {
       size_t halves = 0;
       H->att_P_off.assign(2 * ng, 0);
@@ -1655,6 +1718,7 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
       first_call = true;
     }
   }
+  if (!first_call) att_lk.unlock();
   std::vector<AttendJob> jobs(ng);
   void *ws_base = nullptr;
   int rc;
@@ -1686,7 +1750,7 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
       j.y = b.take<float>((size_t)j.m * n_chunks * std::max(j.v.r_t, 1) * NQP);
       j.a = b.take<float>((size_t)j.m * n_chunks * kD * NQP);
     }
-    if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) return rc;
+    if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) { att_reset(); return rc; }
   }
   Program P;
   const size_t off = P.push(jobs);
@@ -1746,9 +1810,12 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
     LAUNCHED();
   });
   void *d_tab = nullptr;
-  if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
+  if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) { att_reset(); return rc; }
+  if ((rc = arena_acquire(dev, st))) { att_reset(); return rc; }
+  H->last_stream = st;
   g_timer.begin(st);
-  if ((rc = run_program(P, (char *)d_tab, st))) return rc;
+  if ((rc = run_program(P, (char *)d_tab, st))) { att_reset(); return rc; }
+  arena_release(dev, st);
   return JOLT_OK;
 }
 
@@ -1809,7 +1876,8 @@ extern "C" int jolt_deserialize(const void *host_src, int64_t bytes, void *strea
   memcpy(&hd, p, sizeof hd); p += sizeof hd;
   if (hd.magic != kBlobMagic || hd.version != 1 || hd.head_dim != (uint32_t)kD) return fail(JOLT_EINVAL, "not a compressed-cache image of this library version");
   if (hd.n_groups <= 0 || hd.n_cells != 2 * hd.n_groups || hd.n_layers <= 0 || hd.n_kv_heads <= 0 || hd.T <= 0) return fail(JOLT_EINVAL, "corrupt image header");
-  const size_t need = sizeof hd + sizeof(int32_t) * (hd.n_groups + 1) + sizeof(BlobCell) * (size_t)hd.n_cells + hd.blob_bytes;
+  if (hd.blob_bytes > (uint64_t)bytes) return fail(JOLT_EINVAL, "image of %lld bytes, header names a payload of %llu", (long long)bytes, (unsigned long long)hd.blob_bytes);
+  const size_t need = sizeof hd + sizeof(int32_t) * ((size_t)hd.n_groups + 1) + sizeof(BlobCell) * (size_t)hd.n_cells + (size_t)hd.blob_bytes;
   if ((size_t)bytes < need) return fail(JOLT_EINVAL, "image of %lld bytes, header asks for %zu", (long long)bytes, need);
   int dev = 0;
   CU(cudaGetDevice(&dev));
@@ -1819,6 +1887,8 @@ extern "C" int jolt_deserialize(const void *host_src, int64_t bytes, void *strea
   H->group_start.resize(hd.n_groups + 1);
   memcpy(H->group_start.data(), p, sizeof(int32_t) * (hd.n_groups + 1)); p += sizeof(int32_t) * (hd.n_groups + 1);
   if (H->group_start[0] != 0 || H->group_start[hd.n_groups] != hd.n_layers) return fail(JOLT_EINVAL, "corrupt layer grouping");
+  for (int g = 0; g < hd.n_groups; ++g)
+    if (H->group_start[g + 1] <= H->group_start[g]) return fail(JOLT_EINVAL, "corrupt layer grouping (not ascending)");
   H->cells.resize(hd.n_cells);
   for (int i = 0; i < hd.n_cells; ++i) {
     BlobCell bc;
@@ -1838,6 +1908,9 @@ extern "C" int jolt_deserialize(const void *host_src, int64_t bytes, void *strea
   cudaError_t ce = cudaMemcpyAsync(H->blob, p, H->blob_bytes, cudaMemcpyHostToDevice, st);
   if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
   if (ce != cudaSuccess) { cudaGetLastError(); cudaFreeAsync(H->blob, st); return fail(JOLT_ECUDA, "upload: %s", cudaGetErrorString(ce)); }
+  if (cudaMalloc(&H->d_status, sizeof(int) * 4 * (size_t)hd.n_cells) != cudaSuccess) { cudaGetLastError(); cudaFreeAsync(H->blob, st); return fail(JOLT_ENOMEM, "status words"); }
+  cudaMemset(H->d_status, 0, sizeof(int) * 4 * (size_t)hd.n_cells);
+  H->last_stream = st;
   for (auto &cs : H->cells) encode_store_maps(cs);          // tensor maps point into the new buffer
   *out = H.release();
   return JOLT_OK;
@@ -1851,7 +1924,9 @@ extern "C" int jolt_free(jolt_handle *H) {
     if (cur != H->device) cudaSetDevice(H->device);
     if (H->att_P) { cudaFree(H->att_P); H->att_P = nullptr; }       // cudaFree waits for the kernels that read it
     if (H->att_ready) { cudaEventDestroy(H->att_ready); H->att_ready = nullptr; }
-    cudaFreeAsync(H->blob, 0);
+    if (H->d_status) { cudaFree(H->d_status); H->d_status = nullptr; }
+    // ordered after the last call that read the buffers (its stream may be gone by now: then wait for the device)
+    if (cudaFreeAsync(H->blob, H->last_stream) != cudaSuccess) { cudaGetLastError(); cudaDeviceSynchronize(); cudaFreeAsync(H->blob, 0); }
     if (cur != H->device) cudaSetDevice(cur);
   }
   delete H;
@@ -2027,6 +2102,7 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
   build_factor_program(P, ws, mode, true, power_iters, o->seed, fast);
   void *d_tab = nullptr;
   if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
+  if ((rc = arena_acquire(dev, st))) return rc;
   g_timer.begin(st);
   CU(cudaMemsetAsync(d_status, 0, sizeof(int) * 4 * nc, st));
   if (L->mem_space == JOLT_MEM_HOST) {
@@ -2034,6 +2110,7 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
     CU(cudaMemcpyAsync(stage_V, V, span, cudaMemcpyHostToDevice, st));
   }
   if ((rc = run_program(P, (char *)d_tab, st))) return rc;
+  arena_release(dev, st);
   std::vector<int> hstat(4 * nc);
   std::vector<float> lam((size_t)nc * kD);
   std::vector<std::vector<float>> sig(nc);
@@ -2090,6 +2167,7 @@ extern "C" int jolt_release_workspace(void) {
   if (g_tab[dev].base) { cudaFree(g_tab[dev].base); g_tab[dev] = Workspace(); }
   return JOLT_OK;
 }
+#ifdef JOLT_DEBUG
 extern "C" int jolt_debug_stamps(long long *host_out, int n) {
   // n > 0 and host_out == nullptr: (re)allocate and zero a device stamp buffer of n entries; host_out != nullptr: read it back
   if (!host_out) {
@@ -2100,7 +2178,16 @@ extern "C" int jolt_debug_stamps(long long *host_out, int n) {
   if (!g_dbg_stamps) return JOLT_EINVAL;
   return cudaMemcpy(host_out, g_dbg_stamps, sizeof(long long) * n, cudaMemcpyDeviceToHost) == cudaSuccess ? JOLT_OK : JOLT_ECUDA;
 }
+#endif
 extern "C" int64_t jolt_launch_count(void) { return g_launches.load(); }
+extern "C" int jolt_test_set_wait_limit(int64_t cycles, int32_t skip_first_load) {
+  const long long lim = cycles > 0 ? (long long)cycles : tc::kSpinCycles;
+  const int skip = skip_first_load ? 1 : 0;
+  CU(cudaMemcpyToSymbol(tc::g_spin_limit, &lim, sizeof lim));
+  CU(cudaMemcpyToSymbol(tc::g_test_skip_first_load, &skip, sizeof skip));
+  return JOLT_OK;
+}
+extern "C" int jolt_set_stream_groups(int n) { return g_n_cell_groups.exchange(std::max(1, std::min(8, n))); }
 extern "C" int jolt_set_fast_path(int enabled) { return g_fast.exchange(enabled & 127); }
 extern "C" int jolt_last_stage_ms(float *out, int32_t cap, int32_t *n) {
   if (!out || !n) return fail(JOLT_EINVAL, "null argument");

@@ -1,4 +1,4 @@
-// sm_100a building blocks: mbarrier, TMA (cp.async.bulk.tensor, no multicast), tcgen05 MMA with TMEM
+// sm_100a building blocks: mbarrier, plain per-CTA TMA tile loads (cp.async.bulk.tensor), tcgen05 MMA with TMEM
 // accumulators, shared-memory matrix descriptors for the 128-byte swizzle, and host-side tensor maps.
 // Every wait is bounded: after kSpinCycles the waiter raises the CTA's abort flag and returns, all
 // roles then drain to the common exit where TMEM is released.
@@ -10,6 +10,10 @@ namespace jolt {
 namespace tc {
 
 constexpr long long kSpinCycles = 1000000000ll;   // about half a second at 2 GHz
+// The limit the waits use (kSpinCycles unless jolt_test_set_wait_limit changed it) and a test switch that makes the TMA
+// thread of the two-tile sweep kernel leave out its first load, so that a wait runs out without anything faulting.
+__device__ long long g_spin_limit = kSpinCycles;
+__device__ int g_test_skip_first_load = 0;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -34,11 +38,11 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false if the CTA is aborting (this waiter timed out or another role did).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
   if (mbar_try(bar, parity)) return true;
-  const long long t0 = clock64();
+  const long long t0 = clock64(), limit = g_spin_limit;
   while (true) {
     if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kSpinCycles) { *abort_flag = 1; return false; }
+    if (clock64() - t0 > limit) { *abort_flag = 1; return false; }
   }
 }
 

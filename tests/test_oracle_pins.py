@@ -32,7 +32,7 @@ def test_mix64_is_splitmix64():
     assert outs == [0xE220A8397B1DCDAF, 0x6E789E6AA1B965F4, 0x06C45D188009454F]
 
 
-def test_gaussian_moments_and_fp32_exactness():
+def test_gaussian_moments_and_fp16_grid():
     g = O.gaussian_sketch(7, 3, 4096, 64)
     assert g.shape == (4096, 64)
     assert np.array_equal(g, g.astype(np.float16).astype(np.float64))     # defined on the fp16 grid
@@ -105,6 +105,23 @@ def test_quantiser_is_floor_of_ratio():
     assert np.array_equal(xh[0, :12], expect - 4 + 0.5)
     # all-zero groups: mid code, dequantises to 0
     assert np.all(codes[0, 32:] == 4) and np.all(xh[0, 32:] == 0)
+
+
+def test_single_precision_reciprocal_form_is_within_the_code_tolerance():
+    """The definition takes floor(r' / Delta) in float64.  A kernel that multiplies by a single-precision reciprocal
+    lands in the neighbouring bin only where r' / Delta is within rounding distance of an integer: never by more
+    than one code, and on far fewer than the 0.1 % of entries the code-parity gate allows."""
+    x = np.random.default_rng(77).standard_normal((4096, 128)) * 0.37
+    for bits in (1, 2, 3, 4, 8):
+        codes, sc = O.quantize_rows(x, bits)
+        half = float(1 << (bits - 1))
+        g = x.reshape(4096, 4, 32).astype(np.float32)
+        d32 = sc.astype(np.float32)
+        inv = (np.float32(1.0) / d32).astype(np.float32)
+        q = np.clip(np.floor(g * inv[..., None]), -half, half - 1.0) + half
+        diff = np.abs(q.reshape(4096, 128).astype(np.int64) - codes.astype(np.int64))
+        assert diff.max() <= 1
+        assert (diff != 0).mean() <= 2e-4
 
 
 def test_one_bit_is_sign_quantiser():
@@ -294,6 +311,55 @@ def test_bits_zero_stores_no_residual():
     assert np.allclose(Xh, O.stored_backbone(c.Gs16, c.e, c.UT16, c.UF16).astype(np.float32))
 
 
+def test_stored_backbone_decodes_an_exactly_low_rank_cell_at_any_magnitude():
+    """bits = 0 and an input of exact multilinear rank (r_t, r_f): the stored backbone IS the decode, so it must give
+    X back to fp16-storage accuracy -- also when the core has to be scaled down (entries above the fp16 range) or up
+    (entries below the fp16 normal range) by the per-cell exponent, which a wrong sign or offset of that exponent
+    would miss by orders of magnitude."""
+    base = _lowrank(3, 96, 128, 6, 12, noise=0.0, rng=np.random.default_rng(5))
+    for scale in (1.0, 3.0e4, 2.0e-7):
+        X = base * scale
+        c = O.compress_cell(X, 6, 12, 0, token_mode="exact", out_dtype="f32")
+        mx = np.abs(c.ideal["G"]).max()
+        if scale > 1e3:
+            assert mx > 65504 and c.e > 0          # would overflow fp16 unscaled
+        if scale < 1e-3:
+            assert mx < 2.0 ** -14 and c.e < 0     # would be subnormal unscaled
+        assert np.abs(c.Gs16).max() < 2048 and np.abs(c.Gs16).max() >= 1024
+        Xh = O.stored_backbone(c.Gs16, c.e, c.UT16, c.UF16)
+        # three fp16 roundings (core, two factors) and one of P_h: a few 2^-11 relative
+        assert O.rel_frobenius(X, Xh) <= 2.5e-3
+        assert O.rel_frobenius(X, O.decompress_cell(c)) <= 2.5e-3
+    # independent restatement with explicit loops on a tiny cell
+    c = O.compress_cell(base[:, :16] * 50.0, 4, 8, 0, token_mode="exact", out_dtype="f32")
+    Xh = O.stored_backbone(c.Gs16, c.e, c.UT16, c.UF16)
+    h, t, f = 1, 5, 77
+    P = [float(np.float16(sum(c.Gs16[h, r, s_] * c.UF16[f, s_] for s_ in range(8)))) for r in range(4)]
+    assert abs(Xh[h, t, f] - 2.0 ** c.e * sum(c.UT16[t, r] * P[r] for r in range(4))) <= 1e-12 * abs(Xh[h, t, f]) + 1e-300
+
+
+def test_plan_spectra_are_the_mode_spectra():
+    """What the allocator consumes: exact mode gives the squared singular values of the two unfoldings (both sum to
+    ||X||^2); the randomized probe gives the same leading values plus a zero tail once its cap covers the rank."""
+    X = _lowrank(3, 64, 128, 9, 128, noise=0.0, rng=np.random.default_rng(8)) * 2.0
+    tot = float(np.sum(X * X))
+    lam, s2, total = O.plan_spectra(X, 16, token_mode="exact")
+    assert abs(total - tot) <= 1e-12 * tot
+    assert abs(np.sum(s2) - tot) <= 1e-10 * tot and abs(np.sum(lam) - tot) <= 1e-10 * tot
+    s3 = np.linalg.svd(X.reshape(-1, 128), compute_uv=False)
+    assert np.allclose(lam, s3 ** 2, rtol=1e-9, atol=1e-9 * tot)
+    s2_ref = np.linalg.svd(np.transpose(X, (1, 0, 2)).reshape(64, -1), compute_uv=False) ** 2
+    assert np.allclose(s2[:9], s2_ref[:9], rtol=1e-10)
+    lam_r, s2_r, total_r = O.plan_spectra(X, 16, token_mode="randomized", seed=3, cell=1, power_iters=1)
+    assert len(s2_r) == 17 and total_r == total
+    assert np.allclose(s2_r[:9], s2_ref[:9], rtol=1e-9)          # the cap (16) covers the token rank (9)
+    assert np.all(s2_r[9:] <= 1e-9 * tot)                        # nothing is left for the synthetic tail value
+    # with a cap below the rank the tail value carries exactly the omitted mass
+    lam_c, s2_c, _ = O.plan_spectra(X, 4, token_mode="randomized", seed=3, cell=1, power_iters=2)
+    assert len(s2_c) == 5 and abs(np.sum(s2_c) - tot) <= 1e-10 * tot
+    assert s2_c[4] >= np.sum(s2_ref[4:9]) * (1 - 1e-6)
+
+
 # ----------------------------------------------------------------------------- bytes, cap policy
 def test_eq1_closed_form_and_printed_cache_size():
     g = _golden()
@@ -430,7 +496,7 @@ def test_rope_invariants():
     # the defining property: <rope(q, m), rope(k, n)> depends on m - n only
     q, k = RNG.standard_normal((1, 128)), RNG.standard_normal((1, 128))
     def score(m, n):
-        return float(O.rope_rotate(q, 10000.0, m) @ O.rope_rotate(k, 10000.0, n).T)
+        return float((O.rope_rotate(q, 10000.0, m) @ O.rope_rotate(k, 10000.0, n).T).item())
     assert abs(score(5, 2) - score(105, 102)) < 1e-10
     assert abs(score(5, 2) - score(5, 3)) > 1e-6
     # composition of shifts: rotating by a then by b is rotating by a + b

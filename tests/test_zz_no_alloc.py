@@ -39,8 +39,15 @@ def test_static_decode_matches_regular_decode_twice(B):
     torch.cuda.synchronize()
     for call in range(2):
         Ks, Vs = torch.full_like(K, float("nan")), torch.full_like(V, float("nan"))
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         B.jolt_decompress_static(h, Ks, Vs, gs)
         torch.cuda.synchronize()
+        if call == 1:
+            # "allocates nothing": the driver's free-memory figure does not move across the call (the first call on a
+            # device may still load the module and look the array's address up, so the second one is the one measured)
+            assert torch.cuda.mem_get_info()[0] == free_before
+        B.check_status(h)
         assert torch.isfinite(Ks).all() and torch.isfinite(Vs).all()
         assert _rel(Ks, Kr) <= REL_RECON, (call, _rel(Ks, Kr))
         assert _rel(Vs, Vr) <= REL_RECON, (call, _rel(Vs, Vr))
