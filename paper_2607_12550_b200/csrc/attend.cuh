@@ -13,8 +13,7 @@
 //
 // Kernels of a call (the contractions with a tensor-core shape are warp-level fp16 MMAs with fp32 accumulation, an fp32
 // operand entering as hi + lo fp16; the rest is CUDA-core fp32):
-//   attend_p16_kernel      P_h = fp16(G_h U_F^T) of every head of both cells (what the decoder's set-up also forms);
-//                          first call on a handle only
+//   (P_h = fp16(G_h U_F^T), the projected core the decoder also reads, is kept with the handle since compress)
 //   attend_prep_kernel     per (group, head, query): rotated scaled query (fp32, and scaled hi + lo fp16), w = P_h q
 //   attend_bscore_kernel   backbone scores U_T w of all heads of a cell as one dense product (U_T is shared by the heads)
 //   attend_scores_mma_kernel / attend_scores_kernel   per (group, head, 256-token chunk): residual scores added (codes
@@ -81,48 +80,6 @@ __device__ __forceinline__ float att_sign(uint64_t seed, int cell, int f) {
   uint32_t sw[4];
   cell_sign_words(seed, cell, sw);
   return ((sw[f >> 5] >> (f & 31)) & 1u) ? -1.f : 1.f;
-}
-
-// U_F of a cell transposed into shared memory: ufs[s * 128 + f]
-__device__ __forceinline__ void att_stage_uf(const AttendCell &c, __half *ufs, int tid, int nthr) {
-  for (int i = tid; i < 128 * c.r_f; i += nthr) {
-    const int f = i / c.r_f, s = i - f * c.r_f;
-    ufs[s * 128 + f] = c.UF[i];
-  }
-}
-
-// P_h[k][f] = fp16( sum_s G_h[k][s] U_F[f][s] ), the decoder's projected core in scaled units, for both cells of every
-// group.  grid (row blocks of kAttPRows, 2 * groups), 128 threads (thread = feature); dynamic shared memory: 128 * r_f halves.
-constexpr int kAttPRows = 32;
-__global__ void __launch_bounds__(128) attend_p16_kernel(const AttendJob *__restrict__ jobs) {
-  const AttendJob &jb = jobs[blockIdx.y >> 1];
-  const AttendCell &c = (blockIdx.y & 1) ? jb.v : jb.k;
-  __half *P = (blockIdx.y & 1) ? jb.vP : jb.kP;
-  const int rows = jb.m * c.r_t, r0 = blockIdx.x * kAttPRows, f = threadIdx.x;
-  if (r0 >= rows) return;
-  extern __shared__ unsigned char att_smem[];
-  __half *ufs = (__half *)att_smem;
-  att_stage_uf(c, ufs, f, 128);
-  __syncthreads();
-  const int r_f = c.r_f;
-  for (int rb = r0; rb < min(r0 + kAttPRows, rows); rb += 8) {      // rows are a multiple of 8 (r_t is)
-    float acc[8];
-#pragma unroll
-    for (int r = 0; r < 8; ++r) acc[r] = 0.f;
-    for (int s = 0; s < r_f; s += 8) {
-      uint4 g8[8];
-#pragma unroll
-      for (int r = 0; r < 8; ++r) g8[r] = __ldg((const uint4 *)(c.G + (size_t)(rb + r) * r_f + s));
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float u = __half2float(ufs[(s + j) * 128 + f]);
-#pragma unroll
-        for (int r = 0; r < 8; ++r) acc[r] = fmaf(__half2float(((const __half *)&g8[r])[j]), u, acc[r]);
-      }
-    }
-#pragma unroll
-    for (int r = 0; r < 8; ++r) P[(size_t)(rb + r) * 128 + f] = __float2half_rn(acc[r]);
-  }
 }
 
 // grid (m, groups, NQP), 128 threads (thread = feature), 128 floats of dynamic shared memory.  CTA z rotates query z

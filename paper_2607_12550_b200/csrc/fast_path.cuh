@@ -26,17 +26,12 @@ inline bool encode_store_maps(CellStore &cs) {
     const uint32_t box[2] = {64, 128};
     if (!make_tmap_f16(&cs.tmUT, cs.UT16, 2, dims, str, box)) return false;
   }
-  {
-    const uint64_t dims[2] = {(uint64_t)c.r_f, (uint64_t)kD};
-    const uint64_t str[1] = {(uint64_t)c.r_f * 2};
-    const uint32_t box[2] = {64, 128};
-    if (!make_tmap_f16(&cs.tmUF, cs.UF16, 2, dims, str, box)) return false;
-  }
-  {
-    const uint64_t dims[2] = {(uint64_t)c.r_f, (uint64_t)c.m * c.r_t};
-    const uint64_t str[1] = {(uint64_t)c.r_f * 2};
+  {  // projected core P[m * r_t][128]: a box is one head's r_t rows by 64 features (one MN-major operand panel)
+    if (!cs.P16) return false;
+    const uint64_t dims[2] = {(uint64_t)kD, (uint64_t)c.m * c.r_t};
+    const uint64_t str[1] = {(uint64_t)kD * 2};
     const uint32_t box[2] = {64, (uint32_t)c.r_t};
-    if (!make_tmap_f16(&cs.tmG, cs.G16, 2, dims, str, box)) return false;
+    if (!make_tmap_f16(&cs.tmP, cs.P16, 2, dims, str, box)) return false;
   }
   cs.tc_ok = true;
   return true;
@@ -87,7 +82,7 @@ inline void add_decode_tc(Program &P, int stage, const std::vector<tc::BBCell> &
 
 inline void fill_bb_common(tc::BBCell &b, const CellStore &cs, int *status) {
   memset(&b, 0, sizeof b);
-  b.tmUT = cs.tmUT; b.tmUF = cs.tmUF; b.tmG = cs.tmG;
+  b.tmUT = cs.tmUT; b.tmP = cs.tmP;
   b.words = cs.words; b.scales = cs.scales; b.e = cs.e;
   const CellDesc &c = cs.c;
   b.m = c.m; b.n_heads = c.n_heads; b.T = c.T; b.r_t = c.r_t; b.r_f = c.r_f; b.bits = c.bits; b.cell = c.cell;

@@ -198,6 +198,35 @@ __global__ void store_factors_kernel(const StoreJob *jobs) {
   for (long long i = i0; i < j.nUF; i += stride) j.UF16[i] = __float2half_rn(j.UF32[i]);
 }
 
+// P_h[k][f] = fp16( sum_s G_h[k][s] U_F[f][s] ), the projected core of the decoder in the core's scaled units, for every
+// (head, k) row of a cell: [m * r_t][128].  Formed once, when the stored factors exist, and kept with the handle: the
+// residual pass, the decode pass and the attention kernels all read THIS array, so the backbone the residual was taken
+// against is bit for bit the backbone the decoder adds back (closed loop).  grid (row blocks of 32, cells), 128 threads
+// (thread = feature); dynamic shared memory: 128 * r_f halves (U_F, staged as [s][f]).
+struct ProjJob { const __half *G, *UF; __half *P; int rows, r_f; };
+__global__ void __launch_bounds__(128) project_core_kernel(const ProjJob *__restrict__ jobs) {
+  const ProjJob j = jobs[blockIdx.y];
+  const int r0 = blockIdx.x * 32, f = threadIdx.x;
+  if (r0 >= j.rows) return;
+  extern __shared__ __half pc_uf[];
+  for (int e = f; e < 128 * j.r_f; e += 128) { const int ff = e / j.r_f, s = e - ff * j.r_f; pc_uf[s * 128 + ff] = j.UF[e]; }
+  __syncthreads();
+  for (int rb = r0; rb < min(r0 + 32, j.rows); rb += 8) {      // rows are a multiple of 8 (r_t is, or the tail is masked)
+    float acc[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) acc[r] = 0.f;
+    for (int s = 0; s < j.r_f; ++s) {
+      const float u = __half2float(pc_uf[s * 128 + f]);
+#pragma unroll
+      for (int r = 0; r < 8; ++r)
+        if (rb + r < j.rows) acc[r] = fmaf(__half2float(j.G[(size_t)(rb + r) * j.r_f + s]), u, acc[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < 8; ++r)
+      if (rb + r < j.rows) j.P[(size_t)(rb + r) * 128 + f] = __float2half_rn(acc[r]);
+  }
+}
+
 __global__ void round_to_half_inplace_kernel(float *const *ptrs, const long long *counts) {
   const int ci = blockIdx.y;
   float *p = ptrs[ci];
@@ -218,8 +247,9 @@ struct CellStore {
   float *lam = nullptr;    // 128
   int n_sigma = 0;
   const float *dbg_UT32 = nullptr;   // fp32 token factor in the workspace (valid until the next library call)
+  __half *P16 = nullptr;   // projected core [m * r_t][128] (decode-side scratch kept with the handle, not part of the stored bytes)
   bool tc_ok = false;      // tensor maps below are valid
-  alignas(64) CUtensorMap tmUT, tmUF, tmG;
+  alignas(64) CUtensorMap tmUT, tmP;
 };
 
 struct jolt_handle {
@@ -234,11 +264,7 @@ struct jolt_handle {
   bool subspace = false;     // token factors came from the converged block iteration (exact mode, large T)
   int *d_status = nullptr;   // 4 words per cell, written by the decode kernels of the last call on this handle (jolt_check_status)
   mutable cudaStream_t last_stream = nullptr;   // stream of the last call that read the handle's buffers (jolt_free orders after it)
-  // jolt_attend: P_h = fp16(G_h U_F^T) of every cell, formed on the first call and kept until jolt_free
-  mutable std::mutex att_mu;
-  mutable __half *att_P = nullptr;
-  mutable std::vector<size_t> att_P_off;     // per cell, in halves
-  mutable cudaEvent_t att_ready = nullptr;
+  __half *P_all = nullptr;   // the projected cores P_h = fp16(G_h U_F^T) of every cell (CellStore::P16 point into it)
 };
 
 // ------------------------------------------------------------------ validation
@@ -1140,6 +1166,36 @@ static size_t carve_handle_blob(jolt_handle &H) {
   return b.off + 256;
 }
 
+// Device buffer of the projected cores of the cells with a backbone (CellStore::P16 point into it).  A cell whose
+// feature factor is exactly the identity (`identity_uf[c]`: r_f = d, factors not injected) needs none: P = G there.
+static int alloc_projected_cores(jolt_handle &H, const std::vector<char> *identity_uf) {
+  size_t halves = 0;
+  const size_t nc = H.cells.size();
+  std::vector<size_t> off(nc, 0);
+  auto alias = [&](size_t c) { return identity_uf && (*identity_uf)[c]; };
+  for (size_t c = 0; c < nc; ++c) {
+    off[c] = halves;
+    if (H.cells[c].c.r_t > 0 && !alias(c)) halves += ((size_t)H.cells[c].c.m * H.cells[c].c.r_t * kD + 127) & ~(size_t)127;
+  }
+  if (halves) {
+    void *p = nullptr;
+    if (cudaMalloc(&p, halves * sizeof(__half)) != cudaSuccess) { cudaGetLastError(); return fail(JOLT_ENOMEM, "projected cores: %zu bytes", halves * sizeof(__half)); }
+    H.P_all = (__half *)p;
+  }
+  for (size_t c = 0; c < nc; ++c) {
+    CellStore &cs = H.cells[c];
+    cs.P16 = cs.c.r_t == 0 ? nullptr : (alias(c) ? cs.G16 : H.P_all + off[c]);
+  }
+  return JOLT_OK;
+}
+
+static void launch_project_cores(const ProjJob *d_jobs, int n, int max_rows, int max_rf, cudaStream_t s) {
+  static bool attr = false;
+  if (!attr) { cudaFuncSetAttribute(project_core_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 128 * 2); attr = true; }
+  project_core_kernel<<<dim3((max_rows + 31) / 32, n), 128, (size_t)128 * max_rf * sizeof(__half), s>>>(d_jobs);
+  LAUNCHED();
+}
+
 static int compress_impl(const jolt_layout *L, const void *K, const void *V, const jolt_cell_plan *plan,
                          const jolt_options *o, const float *const *inUT, const float *const *inUF, void *stream,
                          jolt_handle **out) {
@@ -1204,7 +1260,15 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     cudaGetLastError(); cudaFreeAsync(H->blob, st); H->blob = nullptr; H->d_status = nullptr;
     return fail(JOLT_ENOMEM, "status words");
   }
-  auto free_blob = [&]() { cudaFreeAsync(H->blob, st); H->blob = nullptr; cudaFree(H->d_status); H->d_status = nullptr; };
+  auto free_blob = [&]() {
+    cudaFreeAsync(H->blob, st); H->blob = nullptr; cudaFree(H->d_status); H->d_status = nullptr;
+    if (H->P_all) { cudaFree(H->P_all); H->P_all = nullptr; }
+  };
+  {
+    std::vector<char> identity_uf(nc, 0);
+    for (int i = 0; i < nc; ++i) identity_uf[i] = mode != FM_INJECTED && cells[i].r_t > 0 && cells[i].r_f == kD;
+    if ((rc = alloc_projected_cores(*H, &identity_uf))) { free_blob(); return rc; }
+  }
   H->last_stream = st;
   lap("validate+blob");
 
@@ -1284,9 +1348,20 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
     if (!sj.empty()) {
       const size_t off = PP.push(sj);
       const int n = (int)sj.size();
+      std::vector<ProjJob> pj;
+      int max_rows = 0, max_rf = 0;
+      for (int i : idx) {
+        const CellDesc &c = cells[i];
+        if (c.r_t == 0 || H->cells[i].P16 == H->cells[i].G16) continue;
+        pj.push_back({H->cells[i].G16, H->cells[i].UF16, H->cells[i].P16, c.m * c.r_t, c.r_f});
+        max_rows = std::max(max_rows, c.m * c.r_t); max_rf = std::max(max_rf, c.r_f);
+      }
+      const size_t poff = PP.push(pj);
+      const int np_ = (int)pj.size();
       PP.add(ST_STORE, [=](char *dev_t, cudaStream_t s) {
         core_exponent_kernel<<<dim3(kCoreMaxParts, n), 256, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
         store_factors_kernel<<<dim3(64, n), 256, 0, s>>>((const StoreJob *)(dev_t + off)); LAUNCHED();
+        if (np_) launch_project_cores((const ProjJob *)(dev_t + poff), np_, max_rows, max_rf, s);
       });
     }
     int tc_heads = 0;
@@ -1532,7 +1607,8 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
         const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)c.T, (uint64_t)c.n_heads, (uint64_t)(c.m / c.n_heads)};
         const uint64_t str[3] = {(uint64_t)L->stride_token * 2, (uint64_t)L->stride_head * 2, (uint64_t)L->stride_layer * 2};
         const uint32_t box[4] = {64, 128, 1, 1};
-        if (make_tmap_f16(&b.tmOut, obase, 4, dims, str, box)) b.tma_out = 1;
+        const uint32_t boxw[4] = {64, 32, 1, 1};
+        if (make_tmap_f16(&b.tmOut, obase, 4, dims, str, box) && make_tmap_f16(&b.tmOutW, obase, 4, dims, str, boxw)) b.tma_out = 1;
       }
       bbc.push_back(b);
       continue;
@@ -1688,37 +1764,11 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
     kbits |= 1u << ck.bits; vbits |= 1u << cv.bits;
     if ((ck.r_t % 8) || (cv.r_t % 8) || (ck.r_f % 8) || (cv.r_f % 8)) return fail(JOLT_EUNSUPPORTED, "ranks must be multiples of 8");
   }
-  const size_t shm_p16 = (size_t)128 * std::max(krf, vrf) * sizeof(__half);
   const size_t shm_prep = 128 * sizeof(float);
   const size_t shm_sc = (size_t)128 * NQP * sizeof(float);
   const size_t shm_comb = (size_t)(n_chunks + vrt + 136) * sizeof(float);
-  const int p_blocks = (m_max * std::max(krt, vrt) + kAttPRows - 1) / kAttPRows;
   if (shm_comb > 48 * 1024) return fail(JOLT_EUNSUPPORTED, "sequence of %d tokens: the chunk merge needs %zu bytes of shared memory", T, shm_comb);
-  // the projected cores do not depend on the queries: formed by the first call on this handle, kept with it
-  // The mutex is held until the first call has issued the kernel that forms the cores and recorded `att_ready`; a
-  // call that fails before that point leaves no half-initialised state behind.
-  bool first_call = false;
-  std::unique_lock<std::mutex> att_lk(H->att_mu);
-  auto att_reset = [&]() {
-    if (first_call) {
-      cudaDeviceSynchronize();
-      if (H->att_P) { cudaFree(H->att_P); H->att_P = nullptr; }
-      if (H->att_ready) { cudaEventDestroy(H->att_ready); H->att_ready = nullptr; }
-    }
-  };
-  {
-    if (!H->att_P) {
-      size_t halves = 0;
-      H->att_P_off.assign(2 * ng, 0);
-      for (int c = 0; c < 2 * ng; ++c) { H->att_P_off[c] = halves; halves += ((size_t)H->cells[c].c.m * std::max(H->cells[c].c.r_t, 1) * kD + 127) & ~(size_t)127; }
-      void *pbuf = nullptr;
-      if (cudaMalloc(&pbuf, halves * sizeof(__half)) != cudaSuccess) { cudaGetLastError(); return fail(JOLT_ENOMEM, "projected cores: %zu bytes", halves * sizeof(__half)); }
-      H->att_P = (__half *)pbuf;
-      if (cudaEventCreateWithFlags(&H->att_ready, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); cudaFree(pbuf); H->att_P = nullptr; return fail(JOLT_ECUDA, "event"); }
-      first_call = true;
-    }
-  }
-  if (!first_call) att_lk.unlock();
+  // the projected cores do not depend on the queries: compress (or deserialize) formed them, the handle keeps them
   std::vector<AttendJob> jobs(ng);
   void *ws_base = nullptr;
   int rc;
@@ -1736,8 +1786,8 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
       j.m = sk.c.m; j.T = T;
       const size_t row0 = (size_t)H->group_start[g] * nh * n_q * kD;
       j.q = (const float *)dQ + row0; j.out = (float *)dOut + row0;
-      j.kP = H->att_P + H->att_P_off[2 * g];
-      j.vP = H->att_P + H->att_P_off[2 * g + 1];
+      j.kP = sk.P16;
+      j.vP = sv.P16;
       j.wh = b.take<__half>((size_t)j.m * NQP * std::max(j.k.r_t, 8));
       j.wl = b.take<__half>((size_t)j.m * NQP * std::max(j.k.r_t, 8));
       j.we = b.take<float>((size_t)j.m * NQP);
@@ -1750,26 +1800,16 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
       j.y = b.take<float>((size_t)j.m * n_chunks * std::max(j.v.r_t, 1) * NQP);
       j.a = b.take<float>((size_t)j.m * n_chunks * kD * NQP);
     }
-    if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) { att_reset(); return rc; }
+    if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) return rc;
   }
   Program P;
   const size_t off = P.push(jobs);
   const uint64_t seed = H->seed;
   const float fscale = (float)scale;
-  cudaEvent_t att_ready = H->att_ready;
   const bool mma = (g_fast.load() & 1) != 0;        // warp-MMA forms of the two code streams (the CUDA-core forms stay as the portable path)
   const bool vmma = mma;
   P.add(ST_ATT, [=](char *dev_t, cudaStream_t s) {
     const AttendJob *d = (const AttendJob *)(dev_t + off);
-    if (first_call) {
-      if (p_blocks > 0) {
-        attend_p16_kernel<<<dim3(p_blocks, 2 * ng), 128, shm_p16, s>>>(d);
-        LAUNCHED();
-      }
-      cudaEventRecord(att_ready, s);
-    } else {
-      cudaStreamWaitEvent(s, att_ready, 0);      // a call on another stream must see the finished cores
-    }
     attend_prep_kernel<<<dim3(m_max, ng, NQP), 128, shm_prep, s>>>(d, n_q, NQP, fscale, seed);
     LAUNCHED();
     const dim3 grid(n_chunks, m_max, ng);
@@ -1810,11 +1850,11 @@ extern "C" int jolt_attend(const jolt_handle *H, const void *dQ, int32_t n_q, do
     LAUNCHED();
   });
   void *d_tab = nullptr;
-  if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) { att_reset(); return rc; }
-  if ((rc = arena_acquire(dev, st))) { att_reset(); return rc; }
+  if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
+  if ((rc = arena_acquire(dev, st))) return rc;
   H->last_stream = st;
   g_timer.begin(st);
-  if ((rc = run_program(P, (char *)d_tab, st))) { att_reset(); return rc; }
+  if ((rc = run_program(P, (char *)d_tab, st))) return rc;
   arena_release(dev, st);
   return JOLT_OK;
 }
@@ -1911,7 +1951,30 @@ extern "C" int jolt_deserialize(const void *host_src, int64_t bytes, void *strea
   if (cudaMalloc(&H->d_status, sizeof(int) * 4 * (size_t)hd.n_cells) != cudaSuccess) { cudaGetLastError(); cudaFreeAsync(H->blob, st); return fail(JOLT_ENOMEM, "status words"); }
   cudaMemset(H->d_status, 0, sizeof(int) * 4 * (size_t)hd.n_cells);
   H->last_stream = st;
-  for (auto &cs : H->cells) encode_store_maps(cs);          // tensor maps point into the new buffer
+  {  // projected cores of the uploaded cells (not part of the image: a function of the stored core and feature factor)
+    int rc = alloc_projected_cores(*H, nullptr);
+    std::vector<ProjJob> pj;
+    int max_rows = 0, max_rf = 0;
+    for (auto &cs : H->cells)
+      if (cs.c.r_t > 0) {
+        pj.push_back({cs.G16, cs.UF16, cs.P16, cs.c.m * cs.c.r_t, cs.c.r_f});
+        max_rows = std::max(max_rows, cs.c.m * cs.c.r_t); max_rf = std::max(max_rf, cs.c.r_f);
+      }
+    void *d_jobs = nullptr;
+    if (rc == JOLT_OK && !pj.empty()) {
+      ce = cudaMalloc(&d_jobs, pj.size() * sizeof(ProjJob));
+      if (ce == cudaSuccess) ce = cudaMemcpyAsync(d_jobs, pj.data(), pj.size() * sizeof(ProjJob), cudaMemcpyHostToDevice, st);
+      if (ce == cudaSuccess) { launch_project_cores((const ProjJob *)d_jobs, (int)pj.size(), max_rows, max_rf, st); ce = cudaStreamSynchronize(st); }
+      if (d_jobs) cudaFree(d_jobs);
+      if (ce != cudaSuccess) { cudaGetLastError(); rc = fail(JOLT_ECUDA, "projected cores: %s", cudaGetErrorString(ce)); }
+    }
+    if (rc != JOLT_OK) {
+      if (H->P_all) cudaFree(H->P_all);
+      cudaFree(H->d_status); cudaFreeAsync(H->blob, st);
+      return rc;
+    }
+  }
+  for (auto &cs : H->cells) encode_store_maps(cs);          // tensor maps point into the new buffers
   *out = H.release();
   return JOLT_OK;
 }
@@ -1922,8 +1985,7 @@ extern "C" int jolt_free(jolt_handle *H) {
     int cur = 0;
     cudaGetDevice(&cur);
     if (cur != H->device) cudaSetDevice(H->device);
-    if (H->att_P) { cudaFree(H->att_P); H->att_P = nullptr; }       // cudaFree waits for the kernels that read it
-    if (H->att_ready) { cudaEventDestroy(H->att_ready); H->att_ready = nullptr; }
+    if (H->P_all) { cudaFree(H->P_all); H->P_all = nullptr; }       // cudaFree waits for the kernels that read it
     if (H->d_status) { cudaFree(H->d_status); H->d_status = nullptr; }
     // ordered after the last call that read the buffers (its stream may be gone by now: then wait for the device)
     if (cudaFreeAsync(H->blob, H->last_stream) != cudaSuccess) { cudaGetLastError(); cudaDeviceSynchronize(); cudaFreeAsync(H->blob, 0); }

@@ -3,10 +3,11 @@
 //   DECODE  : X^  = 2^e U_T P_h + s . H(dequant(codes)) / sqrt(d)       -> fp16 / fp32 rows
 //   RESIDUAL: r   = x - 2^e U_T P_h ; rotate ; quantise ; pack            -> codes + scales
 //
-// One CTA owns a (cell, head, run of 128-token tiles).  It first forms P_h^T = fp16(U_F G_h^T) with one
-// MMA chain (TMA-fed, accumulator in TMEM, rounded into a K-major 128B-swizzled shared tile), then streams
-// U_T tiles through a TMA ring into  D = U_T[tile] P_h  with two TMEM accumulators, so the epilogue of one
-// tile overlaps the MMA of the next.  Two epilogue warpgroups alternate tiles; each thread owns one
+// One CTA owns a (cell, head, run of 128-token tiles).  The projected core P_h = fp16(G_h U_F^T) was formed once
+// when the cell was compressed and is kept with the handle: the CTA fetches its head's [r_t][128] block by TMA as
+// two 64-feature panels (an MN-major B operand) and streams U_T tiles through a TMA ring into  D = U_T[tile] P_h
+// with two TMEM accumulators, so the epilogue of one tile overlaps the MMA of the next.  Residual and decode read
+// the SAME stored P, so the backbone the residual is taken against is bit for bit the one the decoder adds back.  Two epilogue warpgroups alternate tiles; each thread owns one
 // 128-feature row in registers (TMEM lane = token).
 #pragma once
 #include "rowquant.cuh"
@@ -16,8 +17,8 @@ namespace jolt {
 namespace tc {
 
 constexpr int BB_THREADS = 384;
-constexpr int BB_P_BYTES = 65536;            // P^T: up to 4 K-blocks of [128 rows][128 B]
-constexpr int BB_BIG_BYTES = 131072;         // set-up operands, then ring (+ X tiles)
+constexpr int BB_P_BYTES = 65536;            // P: two panels of [r_t rows][128 B], r_t <= 256
+constexpr int BB_BIG_BYTES = 131072;         // ring (+ X tiles)
 constexpr int BB_STAGE_BYTES = 16384;        // one [128 tokens][64 fp16] box of U_T
 constexpr int BB_XTILE_BYTES = 32768;        // two [128 tokens][64 fp16] boxes of X
 constexpr int BB_SMEM_BYTES = BB_P_BYTES + BB_BIG_BYTES + 1024 /*align*/ + 512 /*barriers*/;
@@ -25,10 +26,10 @@ constexpr int BB_TMEM_COLS = 256;
 
 struct alignas(64) BBCell {
   CUtensorMap tmUT;     // fp16 [T][r_t]           dims {r_t, T},       box {64, 128}
-  CUtensorMap tmUF;     // fp16 [128][r_f]         dims {r_f, 128},     box {64, 128}
-  CUtensorMap tmG;      // fp16 [m*r_t][r_f]       dims {r_f, m*r_t},   box {64, r_t}
+  CUtensorMap tmP;      // fp16 [m*r_t][128]       dims {128, m*r_t},   box {64, r_t}
   CUtensorMap tmX;      // fp16 [L][n_h][T][128]   dims {128, T, n_h, L}, box {64, 128, 1, 1}   (RESIDUAL)
   CUtensorMap tmOut;    // same shape over the output tensor (DECODE, fp16 destinations TMA can address)
+  CUtensorMap tmOutW;   // the output tensor again with box {64, 32, 1, 1}: the 32 rows one warp stages and stores
   int tma_out;
   long long *dbg;       // optional: cycle stamps of CTA 0 (profiling aid), 8 per tile per warpgroup
   uint32_t *words;      // [m][T][4*bits]
@@ -102,7 +103,7 @@ __global__ void __launch_bounds__(BB_THREADS, 1) backbone_kernel(const BBCell *_
   const uint32_t sRing = sBig;
   const uint32_t sX = sBig + 4 * BB_STAGE_BYTES;       // RESIDUAL: two X tiles behind a 4-stage ring
   // barrier slots (8 bytes each)
-  const uint32_t bSetup = sBar + 0, bPdone = sBar + 8, bPready = sBar + 16;
+  const uint32_t bSetup = sBar + 0;
   auto bFull = [=](int s) { return sBar + 24 + 8 * s; };
   auto bEmpty = [=](int s) { return sBar + 24 + 64 + 8 * s; };
   auto bTfull = [=](int b) { return sBar + 152 + 8 * b; };
@@ -112,11 +113,12 @@ __global__ void __launch_bounds__(BB_THREADS, 1) backbone_kernel(const BBCell *_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = warp >> 2;
-  const int nkt = (c.r_t + 63) / 64, nkf = (c.r_f + 63) / 64;
+  const int nkt = (c.r_t + 63) / 64;
+  const uint32_t panel = (uint32_t)c.r_t * 128u;       // bytes of one 64-feature panel of P (r_t is a multiple of 16)
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
-    mbar_init(bSetup, 1); mbar_init(bPdone, 1); mbar_init(bPready, 256);
+    mbar_init(bSetup, 1);
     for (int s = 0; s < 8; ++s) { mbar_init(bFull(s), 1); mbar_init(bEmpty(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(bTfull(b), 1); mbar_init(bTempty(b), 128); mbar_init(bXfull(b), 1); mbar_init(bXempty(b), 128); }
     fence_barrier_init();
@@ -131,15 +133,12 @@ __global__ void __launch_bounds__(BB_THREADS, 1) backbone_kernel(const BBCell *_
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (warp == 8 && lane == 0) {
       // ---------------- TMA producer
-      tma_prefetch_desc(&c.tmUT); tma_prefetch_desc(&c.tmUF); tma_prefetch_desc(&c.tmG);
+      tma_prefetch_desc(&c.tmUT); tma_prefetch_desc(&c.tmP);
       if (RESIDUAL) tma_prefetch_desc(&c.tmX);
-      const uint32_t g_rows_bytes = (uint32_t)c.r_t * 128u;
-      mbar_expect_tx(bSetup, (uint32_t)nkf * (16384u + g_rows_bytes));
-      for (int kb = 0; kb < nkf; ++kb) {
-        tma_load_2d(sBig + kb * 16384, &c.tmUF, bSetup, kb * 64, 0);
-        tma_load_2d(sBig + 32768 + kb * 32768, &c.tmG, bSetup, kb * 64, h * c.r_t);
-      }
-      bool ok = mbar_wait(bPdone, 0, abort_flag);   // set-up operands consumed: the big region is free
+      mbar_expect_tx(bSetup, 2u * panel);
+      tma_load_2d(sP, &c.tmP, bSetup, 0, h * c.r_t);
+      tma_load_2d(sP + panel, &c.tmP, bSetup, 64, h * c.r_t);
+      bool ok = true;
       int cnt = 0;
       const int l = h / c.n_heads, hd = h - l * c.n_heads;
       for (int i = 0; ok && i < n_tiles; ++i) {
@@ -161,22 +160,11 @@ __global__ void __launch_bounds__(BB_THREADS, 1) backbone_kernel(const BBCell *_
       }
     } else if (warp == 9 && lane == 0) {
       // ---------------- MMA issuer
-      bool ok = mbar_wait(bSetup, 0, abort_flag);
+      bool ok = mbar_wait(bSetup, 0, abort_flag);      // the head's projected core has landed
       if (ok) {
         tc_fence_after();
-        const uint32_t idescP = umma_idesc_f16(128, c.r_t, 0, 0);
-        for (int kb = 0; kb < nkf; ++kb)
-          for (int k4 = 0; k4 < 4; ++k4) {
-            const uint64_t da = umma_desc_sw128(sBig + kb * 16384 + k4 * 32, 16, 1024);
-            const uint64_t db = umma_desc_sw128(sBig + 32768 + kb * 32768 + k4 * 32, 16, 1024);
-            umma_f16(tmem_base, da, db, idescP, (kb | k4) != 0);
-          }
-        umma_commit(bPdone);
-        ok = mbar_wait(bPready, 0, abort_flag);
-      }
-      if (ok) {
-        tc_fence_after();
-        const uint32_t idesc = umma_idesc_f16(128, 128, 0, 0);
+        const uint32_t idesc = umma_idesc_f16(128, 128, 0, 1);   // A = U_T tile, K-major; B = P panels, MN-major
+        const int ksteps = c.r_t / 16;
         int cnt = 0;
         for (int i = 0; ok && i < n_tiles; ++i) {
           const int b = i & 1, nb = i >> 1;
@@ -188,9 +176,10 @@ __global__ void __launch_bounds__(BB_THREADS, 1) backbone_kernel(const BBCell *_
             ok = mbar_wait(bFull(s), n & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            for (int k4 = 0; k4 < 4; ++k4) {
+            for (int k4 = 0; k4 < 4 && kb * 4 + k4 < ksteps; ++k4) {
               const uint64_t da = umma_desc_sw128(sRing + s * BB_STAGE_BYTES + k4 * 32, 16, 1024);
-              const uint64_t db = umma_desc_sw128(sP + kb * 16384 + k4 * 32, 16, 1024);
+              // 16 contraction rows of P = 2048 B per step; the second 64 features one panel further
+              const uint64_t db = umma_desc_sw128(sP + (kb * 4 + k4) * 2048, panel, 1024);
               umma_f16(tmem_base + b * 128, da, db, idesc, (kb | k4) != 0);
             }
             umma_commit(bEmpty(s));
@@ -205,36 +194,8 @@ __global__ void __launch_bounds__(BB_THREADS, 1) backbone_kernel(const BBCell *_
     const int q = warp & 3;
     const int row_in_tile = q * 32 + lane;
     const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
-    bool ok = __all_sync(0xffffffffu, mbar_wait(bPdone, 0, abort_flag));
-    if (ok) {
-      tc_fence_after();
-      // P^T (fp32 in TMEM, lane = feature, column = r) -> fp16, K-major 128B-swizzled rows in shared memory
-      for (int ch = wg; ch < 2 * nkt; ch += 2) {
-        float v[32];
-        tmem_ld32(t_lane + ch * 32, v);
-        tmem_wait_ld();
-        const int kb = ch >> 1;
-        unsigned char *rowp = sm + kb * 16384 + row_in_tile * 128;
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          uint4 pk;
-          __half2 *hp = (__half2 *)&pk;
-#pragma unroll
-          for (int e2 = 0; e2 < 4; ++e2) {
-            const int col = ch * 32 + jj * 8 + e2 * 2;
-            const float a = col < c.r_t ? v[jj * 8 + e2 * 2] : 0.f;
-            const float b2 = col + 1 < c.r_t ? v[jj * 8 + e2 * 2 + 1] : 0.f;
-            hp[e2] = __floats2half2_rn(a, b2);
-          }
-          const int chunk = (ch & 1) * 4 + jj;
-          *(uint4 *)(rowp + ((chunk ^ (row_in_tile & 7)) << 4)) = pk;
-        }
-      }
-      fence_proxy_async();
-      tc_fence_before();
-      mbar_arrive(bPready);
-    }
-    const float scale = ok ? ldexpf(1.0f, *c.e) : 0.f;
+    bool ok = true;
+    const float scale = ldexpf(1.0f, *c.e);
     const int l = h / c.n_heads, hd = h - l * c.n_heads;
     for (int i = wg; ok && i < n_tiles; i += 2) {
       const int tt = tile0 + i, nb = i >> 1;

@@ -7,8 +7,8 @@
 // residual (K = 128, B operand = the +-1 Hadamard matrix with the sign flips folded in, exact in fp16) go into
 // the same TMEM accumulator.  The epilogue threads only unpack codes into a half-precision operand tile
 // (pre-scaled by Delta / sqrt(128) * 2^-e) and, after the MMA, scale, convert and store their row: no
-// Hadamard butterflies on the CUDA cores.  P_h^T = fp16(U_F G_h^T) is formed once per CTA as in the residual
-// kernel.  Rounding the dequantised residual to fp16 before the rotation costs 2^-11 of the residual, i.e.
+// Hadamard butterflies on the CUDA cores.  P_h = fp16(G_h U_F^T) is the block stored with the handle at compress
+// time, fetched by TMA as an MN-major operand exactly as in the residual kernel.  Rounding the dequantised residual to fp16 before the rotation costs 2^-11 of the residual, i.e.
 // ~1e-5 of the cache entries, far below the fp16 rounding of the output itself.
 #pragma once
 #include "tc_backbone.cuh"
@@ -36,7 +36,8 @@ struct DecLayout {
   static constexpr int P_BYTES = 65536;
   static constexpr int NS = 4;                                          // ring stages in the ring region proper
   static constexpr int BIG_BYTES = NS * 16384 + DEC_NWG * 32768;        // ring + operand tiles (set-up operands first)
-  static constexpr int SMEM_BYTES = P_BYTES + DEC_H_BYTES + BIG_BYTES + 1024 + 512;
+  static constexpr int SMEM_BYTES = P_BYTES + DEC_H_BYTES + BIG_BYTES + 1024 /*align*/ + 512 /*barriers*/ + 1024 /*cell descriptor*/;
+  static_assert(sizeof(BBCell) <= 1024, "the cell descriptor is staged in 1 KB of shared memory");
   static constexpr int TMEM_COLS = 512;     // two accumulators per warpgroup when r_t <= 128
   // registers move from the producer warpgroup to the epilogue ones (12 warps: the register file has the slack a
   // blocking re-partition needs)
@@ -227,13 +228,43 @@ __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+// B operand of the inverse rotation: Hs[f][f'] = s_f * (-1)^popcount(f & f'), fp16, K-major, swizzled; built by the
+// 256 epilogue threads (et = thread index among them), then announced on bHready.  Thread et owns 16-byte chunk
+// et & 15 (features f' = 8 chunk .. 8 chunk + 7) of rows f = (et >> 4) + 16 k: popcount(f & f') splits into the part
+// from f's low three bits, the same for all of the thread's rows (f & 7 is), and popcount(f & 8 chunk), one sign per row.
+__device__ __forceinline__ void dec_build_rotation(unsigned char *smH, uint64_t seed, int cell, int et, uint32_t bHready) {
+  uint32_t sw[4];
+  cell_sign_words(seed, cell, sw);
+  const int chunk = et & 15, f0 = et >> 4;
+  uint32_t basew[4];
+#pragma unroll
+  for (int e2 = 0; e2 < 4; ++e2) {
+    const uint32_t n0 = __popc(f0 & 7 & (2 * e2)) & 1u, n1 = __popc(f0 & 7 & (2 * e2 + 1)) & 1u;
+    basew[e2] = (0x3C00u | (n0 << 15)) | ((0x3C00u | (n1 << 15)) << 16);      // +-1.0 in fp16
+  }
+  unsigned char *colp = smH + (chunk >> 3) * 16384;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int f = f0 + 16 * k;
+    const uint32_t flip = ((__popc(f & (chunk << 3)) & 1u) ^ ((sw[f >> 5] >> (f & 31)) & 1u)) * 0x80008000u;
+    *(uint4 *)(colp + f * 128 + (((chunk & 7) ^ (f & 7)) << 4)) = make_uint4(basew[0] ^ flip, basew[1] ^ flip, basew[2] ^ flip, basew[3] ^ flip);
+  }
+  fence_proxy_async();
+  mbar_arrive(bHready);
+}
+
 struct DecCtx {
-  uint32_t bTfull, bTempty, bRready, t_acc, s_obuf;
-  unsigned char *rbuf, *obuf;
+  uint32_t bTfull, bTempty, bRready, bHready, t_acc, s_obuf;
+  unsigned char *rbuf, *obuf, *smH;
+  const BBCell *cg;       // the descriptor in global memory: tensor maps are addressed there
   volatile int *abort_flag;
   int wg, nwg, rit, h, tile0, n_tiles, l, hd;
-  float scale, pre;
+  int ex;                 // core exponent: loaded at kernel start, first USED after the rotation operand is built
+  uint64_t seed;
 };
+// output scale 2^e and the residual operand's pre-scale (the operand is kept in the accumulator's units)
+struct DecScales { float scale, pre; };
+__device__ __forceinline__ DecScales dec_scales(int ex) { return {ldexpf(1.0f, ex), ldexpf(kInvSqrtD, -ex)}; }
 
 // The per-tile loop of one epilogue warpgroup (tiles wg, wg+2, ...) with one accumulator per warpgroup (r_t > 128).
 template <int BITS>
@@ -242,7 +273,9 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
   bool ok = true;
   const bool tma_out = c.tma_out != 0;
   if (x.wg < x.n_tiles) dec_load_codes<BITS>(c, (long long)x.h * c.T + (x.tile0 + x.wg) * 128 + x.rit, cur);
-  JOLT_DBG(const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;)
+  dec_build_rotation(x.smH, x.seed, c.cell, x.wg * 128 + x.rit, x.bHready);     // the first codes are in flight meanwhile
+  const DecScales sc = dec_scales(x.ex);
+  JOLT_DBG(const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == gridDim.y / 2 && x.rit == 0;)
   for (int i = x.wg; i < x.n_tiles; i += x.nwg) {
     const int tt = x.tile0 + i, nb = i / x.nwg;
     const int token = tt * 128 + x.rit;
@@ -254,7 +287,7 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
     }
     JOLT_DBG(if (dbg) dbg[1] = clock64();)
     if constexpr (BITS > 0) {
-      if (ok) dec_unpack_row<BITS>(cur, x.pre, x.rbuf, x.rit);
+      if (ok) dec_unpack_row<BITS>(cur, sc.pre, x.rbuf, x.rit);
       fence_proxy_async();
       mbar_arrive(x.bRready);
       JOLT_DBG(if (dbg) dbg[2] = clock64();)
@@ -281,7 +314,7 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
         for (int k8 = 0; k8 < 4; ++k8) {
           __half2 *hp = (__half2 *)&o[k8];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) hp[j] = __floats2half2_rn(v[k8 * 8 + 2 * j] * x.scale, v[k8 * 8 + 2 * j + 1] * x.scale);
+          for (int j = 0; j < 4; ++j) hp[j] = __floats2half2_rn(v[k8 * 8 + 2 * j] * sc.scale, v[k8 * 8 + 2 * j + 1] * sc.scale);
         }
         if (tma_out) {      // stage the row, same swizzled layout as a loaded X tile
           unsigned char *rowp = x.obuf + (ch >> 1) * 16384 + x.rit * 128;
@@ -296,7 +329,7 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
         float4 *p = (float4 *)((float *)c.out + off + ch * 32);
 #pragma unroll
         for (int k4 = 0; k4 < 8; ++k4)
-          p[k4] = make_float4(v[4 * k4] * x.scale, v[4 * k4 + 1] * x.scale, v[4 * k4 + 2] * x.scale, v[4 * k4 + 3] * x.scale);
+          p[k4] = make_float4(v[4 * k4] * sc.scale, v[4 * k4 + 1] * sc.scale, v[4 * k4 + 2] * sc.scale, v[4 * k4 + 3] * sc.scale);
       }
     }
     JOLT_DBG(if (dbg) dbg[5] = clock64();)
@@ -305,8 +338,8 @@ __device__ __forceinline__ bool dec_tile_loop(const BBCell &c, const DecCtx &x) 
       named_bar_sync(1 + x.wg, 128);
       JOLT_DBG(if (dbg) dbg[6] = clock64();)
       if (x.rit == 0 && ok) {
-        tma_store_4d(&c.tmOut, x.s_obuf, 0, tt * 128, x.hd, x.l);
-        tma_store_4d(&c.tmOut, x.s_obuf + 16384, 64, tt * 128, x.hd, x.l);
+        tma_store_4d(&x.cg->tmOut, x.s_obuf, 0, tt * 128, x.hd, x.l);
+        tma_store_4d(&x.cg->tmOut, x.s_obuf + 16384, 64, tt * 128, x.hd, x.l);
         tma_store_commit();
       }
     }
@@ -329,17 +362,26 @@ __device__ __forceinline__ bool dec_tile_loop_acc4(const BBCell &c, const DecCtx
   bool ok = true;
   const long long row0 = (long long)x.h * c.T + x.tile0 * 128 + x.rit;
   if (x.wg < x.n_tiles) dec_load_codes<BITS>(c, row0 + x.wg * 128, cur);
+  dec_build_rotation(x.smH, x.seed, c.cell, x.wg * 128 + x.rit, x.bHready);     // the first codes are in flight meanwhile
+  const DecScales sc = dec_scales(x.ex);
   const int lane = x.rit & 31, wrow0 = x.rit & ~31;       // this warp's rows of the tile: wrow0 .. wrow0 + 31
   unsigned char *obuf = x.rbuf;
+  const bool tma_out = c.tma_out != 0 && c.out_dtype == DT_F16;
+  const uint32_t s_wrows = x.s_obuf + (uint32_t)wrow0 * 128u;      // this warp's 32 staging rows (first 64 features)
   int n = 0;
-  JOLT_DBG(const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;)
+  JOLT_DBG(const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == gridDim.y / 2 && x.rit == 0;)
   for (int i = x.wg; i < x.n_tiles; i += 2, ++n) {
     const int acc = n & 1, ph = n >> 1;
     const int tt = x.tile0 + i, token = tt * 128 + x.rit;
     JOLT_DBG(long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;)
     JOLT_DBG(if (dbg) dbg[0] = clock64();)
+    if (tma_out && n > 0) {      // the previous tile's store must have read this warp's staging rows
+      if (lane == 0) tma_store_wait_read();
+      __syncwarp();
+    }
+    JOLT_DBG(if (dbg) dbg[1] = clock64();)
     if constexpr (BITS > 0) {
-      if (ok) dec_unpack_row<BITS>(cur, x.pre, obuf, x.rit);
+      if (ok) dec_unpack_row<BITS>(cur, sc.pre, obuf, x.rit);
       fence_proxy_async();
       mbar_arrive(x.bRready + 16 * acc);
       if (i + 2 < x.n_tiles) dec_load_codes<BITS>(c, row0 + (i + 2) * 128, cur);      // in flight during the MMA and the epilogue
@@ -372,34 +414,48 @@ __device__ __forceinline__ bool dec_tile_loop_acc4(const BBCell &c, const DecCtx
             uint4 o;
             __half2 *hp = (__half2 *)&o;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) hp[j] = __floats2half2_rn(v[k8 * 8 + 2 * j] * x.scale, v[k8 * 8 + 2 * j + 1] * x.scale);
+            for (int j = 0; j < 4; ++j) hp[j] = __floats2half2_rn(v[k8 * 8 + 2 * j] * sc.scale, v[k8 * 8 + 2 * j + 1] * sc.scale);
             *(uint4 *)(rowp + ((((ch & 1) * 4 + k8) ^ (x.rit & 7)) << 4)) = o;
           }
         }
-        __syncwarp();
-        JOLT_DBG(if (dbg) dbg[5] = clock64();)
-        // read back: lane l takes 16-byte chunk l & 15 of rows 2 it + (l >> 4); a row is 256 contiguous bytes of output
-        const int q16 = lane & 15;
-        __half *obase = (__half *)c.out + (long long)x.l * c.osl + (long long)x.hd * c.osh;
+        if (tma_out) {
+          // the warp's 32 staged rows leave as two bulk tensor stores (64 features each) issued by one lane: no thread
+          // waits for the global writes, only (before the rows are overwritten) for the copy engine to have read them
+          fence_proxy_async();
+          __syncwarp();
+          JOLT_DBG(if (dbg) dbg[5] = clock64();)
+          if (lane == 0) {
+            tma_store_4d(&x.cg->tmOutW, s_wrows, 0, tt * 128 + wrow0, x.hd, x.l);
+            tma_store_4d(&x.cg->tmOutW, s_wrows + 16384, 64, tt * 128 + wrow0, x.hd, x.l);
+            tma_store_commit();
+          }
+        } else {
+          __syncwarp();
+          JOLT_DBG(if (dbg) dbg[5] = clock64();)
+          // read back: lane l takes 16-byte chunk l & 15 of rows 2 it + (l >> 4); a row is 256 contiguous bytes of output
+          const int q16 = lane & 15;
+          __half *obase = (__half *)c.out + (long long)x.l * c.osl + (long long)x.hd * c.osh;
 #pragma unroll 4
-        for (int it = 0; it < 16; ++it) {
-          const int r = wrow0 + 2 * it + (lane >> 4);
-          const uint4 o = *(const uint4 *)(obuf + (q16 >> 3) * 16384 + r * 128 + (((q16 & 7) ^ (r & 7)) << 4));
-          *(uint4 *)(obase + (long long)(tt * 128 + r) * c.ost + q16 * 8) = o;
+          for (int it = 0; it < 16; ++it) {
+            const int r = wrow0 + 2 * it + (lane >> 4);
+            const uint4 o = *(const uint4 *)(obuf + (q16 >> 3) * 16384 + r * 128 + (((q16 & 7) ^ (r & 7)) << 4));
+            *(uint4 *)(obase + (long long)(tt * 128 + r) * c.ost + q16 * 8) = o;
+          }
+          __syncwarp();
         }
-        __syncwarp();
       } else {
         float4 *p = (float4 *)((float *)c.out + off);
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch)
 #pragma unroll
           for (int k4 = 0; k4 < 8; ++k4)
-            p[ch * 8 + k4] = make_float4(va[ch][4 * k4] * x.scale, va[ch][4 * k4 + 1] * x.scale, va[ch][4 * k4 + 2] * x.scale,
-                                         va[ch][4 * k4 + 3] * x.scale);
+            p[ch * 8 + k4] = make_float4(va[ch][4 * k4] * sc.scale, va[ch][4 * k4 + 1] * sc.scale, va[ch][4 * k4 + 2] * sc.scale,
+                                         va[ch][4 * k4 + 3] * sc.scale);
       }
     }
     JOLT_DBG(if (dbg) dbg[7] = clock64();)
   }
+  if (tma_out && lane == 0) tma_store_wait_all();
   return ok;
 }
 
@@ -414,17 +470,26 @@ __device__ __forceinline__ bool dec_tile_loop_acc4_rope(const BBCell &c, const D
   bool ok = true;
   const long long row0 = (long long)x.h * c.T + x.tile0 * 128 + x.rit;
   if (x.wg < x.n_tiles) dec_load_codes<BITS>(c, row0 + x.wg * 128, cur);
+  dec_build_rotation(x.smH, x.seed, c.cell, x.wg * 128 + x.rit, x.bHready);     // the first codes are in flight meanwhile
+  const DecScales sc = dec_scales(x.ex);
   const int lane = x.rit & 31, wrow0 = x.rit & ~31;       // this warp's rows of the tile: wrow0 .. wrow0 + 31
   unsigned char *obuf = x.rbuf;
+  const bool tma_out = c.tma_out != 0 && c.out_dtype == DT_F16;
+  const uint32_t s_wrows = x.s_obuf + (uint32_t)wrow0 * 128u;      // this warp's 32 staging rows (first 64 features)
   int n = 0;
-  JOLT_DBG(const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && x.rit == 0;)
+  JOLT_DBG(const bool stamp = c.dbg && blockIdx.x == 0 && blockIdx.y == gridDim.y / 2 && x.rit == 0;)
   for (int i = x.wg; i < x.n_tiles; i += 2, ++n) {
     const int acc = n & 1, ph = n >> 1;
     const int tt = x.tile0 + i, token = tt * 128 + x.rit;
     JOLT_DBG(long long *dbg = stamp ? c.dbg + (size_t)i * 8 : nullptr;)
     JOLT_DBG(if (dbg) dbg[0] = clock64();)
+    if (tma_out && n > 0) {      // the previous tile's store must have read this warp's staging rows
+      if (lane == 0) tma_store_wait_read();
+      __syncwarp();
+    }
+    JOLT_DBG(if (dbg) dbg[1] = clock64();)
     if constexpr (BITS > 0) {
-      if (ok) dec_unpack_row<BITS>(cur, x.pre, obuf, x.rit);
+      if (ok) dec_unpack_row<BITS>(cur, sc.pre, obuf, x.rit);
       fence_proxy_async();
       mbar_arrive(x.bRready + 16 * acc);
       if (i + 2 < x.n_tiles) dec_load_codes<BITS>(c, row0 + (i + 2) * 128, cur);      // in flight during the MMA and the epilogue
@@ -452,14 +517,14 @@ __device__ __forceinline__ bool dec_tile_loop_acc4_rope(const BBCell &c, const D
           uint4 o;
           __half2 *hp = (__half2 *)&o;
 #pragma unroll
-          for (int j = 0; j < 4; ++j) hp[j] = __floats2half2_rn(v[k8 * 8 + 2 * j] * x.scale, v[k8 * 8 + 2 * j + 1] * x.scale);
+          for (int j = 0; j < 4; ++j) hp[j] = __floats2half2_rn(v[k8 * 8 + 2 * j] * sc.scale, v[k8 * 8 + 2 * j + 1] * sc.scale);
           *(uint4 *)(rowp + ((((ch & 1) * 4 + k8) ^ (x.rit & 7)) << 4)) = o;
         }
       } else {
         float4 *p = (float4 *)((float *)c.out + off);
 #pragma unroll
         for (int k4 = 0; k4 < 8; ++k4)
-          p[ch * 8 + k4] = make_float4(v[4 * k4] * x.scale, v[4 * k4 + 1] * x.scale, v[4 * k4 + 2] * x.scale, v[4 * k4 + 3] * x.scale);
+          p[ch * 8 + k4] = make_float4(v[4 * k4] * sc.scale, v[4 * k4 + 1] * sc.scale, v[4 * k4 + 2] * sc.scale, v[4 * k4 + 3] * sc.scale);
       }
     };
     {
@@ -486,7 +551,16 @@ __device__ __forceinline__ bool dec_tile_loop_acc4_rope(const BBCell &c, const D
       }
       JOLT_DBG(if (dbg) dbg[4] = clock64();)
     }
-    if (ok && c.out_dtype == DT_F16) {
+    if (ok && tma_out) {
+      fence_proxy_async();
+      __syncwarp();
+      JOLT_DBG(if (dbg) dbg[5] = clock64();)
+      if (lane == 0) {
+        tma_store_4d(&x.cg->tmOutW, s_wrows, 0, tt * 128 + wrow0, x.hd, x.l);
+        tma_store_4d(&x.cg->tmOutW, s_wrows + 16384, 64, tt * 128 + wrow0, x.hd, x.l);
+        tma_store_commit();
+      }
+    } else if (ok && c.out_dtype == DT_F16) {
       __syncwarp();
       JOLT_DBG(if (dbg) dbg[5] = clock64();)
       // read back: lane l takes 16-byte chunk l & 15 of rows 2 it + (l >> 4); a row is 256 contiguous bytes of output
@@ -502,6 +576,7 @@ __device__ __forceinline__ bool dec_tile_loop_acc4_rope(const BBCell &c, const D
     }
     JOLT_DBG(if (dbg) dbg[7] = clock64();)
   }
+  if (tma_out && lane == 0) tma_store_wait_all();
   return ok;
 }
 
@@ -510,13 +585,16 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
   constexpr int NWG = DEC_NWG;
   constexpr int DEC_P_BYTES = LY::P_BYTES, DEC_BIG_BYTES = LY::BIG_BYTES, DEC_NS = LY::NS;
   extern __shared__ unsigned char smem_raw[];
-  const BBCell &c = cells[blockIdx.y];
-  const int items = c.m * c.items_per_head;
-  if ((int)blockIdx.x >= items) return;
-  const int h = blockIdx.x / c.items_per_head;
-  const int item = blockIdx.x - h * c.items_per_head;
-  const int tile0 = item * c.tiles_per_item;
-  const int n_tiles = min(c.tiles_per_item, c.T / 128 - tile0);
+  // The cell's descriptor is read from global memory ONCE, cooperatively, into shared memory: the scalar fields are
+  // used all over the kernel and each first touch from global would be a dependent L2 round trip on the critical
+  // path of the CTA's start.  Only the tensor maps are addressed in global memory (the copy engine requires that).
+  const BBCell &cg = cells[blockIdx.y];
+  const int items_per_head = cg.items_per_head, tiles_per_item = cg.tiles_per_item, n_tok_tiles = cg.T / 128;
+  if ((int)blockIdx.x >= cg.m * items_per_head) return;
+  const int h = blockIdx.x / items_per_head;
+  const int item = blockIdx.x - h * items_per_head;
+  const int tile0 = item * tiles_per_item;
+  const int n_tiles = min(tiles_per_item, n_tok_tiles - tile0);
   if (n_tiles <= 0) return;
 
   const uint32_t raw = smem_u32(smem_raw);
@@ -528,7 +606,7 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
   unsigned char *smH = sm + DEC_P_BYTES, *smR = sm + DEC_P_BYTES + DEC_H_BYTES + DEC_NS * BB_STAGE_BYTES;
   volatile int *abort_flag = (volatile int *)(sm + DEC_P_BYTES + DEC_H_BYTES + DEC_BIG_BYTES + 256);
   uint32_t *tmem_slot = (uint32_t *)(sm + DEC_P_BYTES + DEC_H_BYTES + DEC_BIG_BYTES + 264);
-  const uint32_t bSetup = sBar + 0, bPdone = sBar + 8, bPready = sBar + 16;
+  const uint32_t bSetup = sBar + 0, bHready = sBar + 16;
   auto bFull = [=](int s) { return sBar + 24 + 8 * s; };          // up to 6 ring stages
   auto bEmpty = [=](int s) { return sBar + 72 + 8 * s; };
   auto bTfull = [=](int b) { return sBar + 120 + 8 * b; };        // up to 4 accumulators
@@ -537,20 +615,14 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = warp >> 2;
-  JOLT_DBG(long long *kdbg = (c.dbg && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ? c.dbg + 16 * 8 : nullptr;)
+  JOLT_DBG(long long *kdbg = (cg.dbg && blockIdx.x == 0 && blockIdx.y == gridDim.y / 2 && threadIdx.x == 0) ? cg.dbg + 16 * 8 : nullptr;)
   JOLT_DBG(if (kdbg) { kdbg[0] = clock64(); long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); kdbg[6] = gt; })
-  const int nkt = (c.r_t + 63) / 64, nkf = (c.r_f + 63) / 64;
-  const bool has_res = c.bits > 0;
-  // r_t <= 128 leaves half of the P region and half of the ring free: each warpgroup then stages its output in a
-  // buffer of its own, so a tile's unpack never waits for the previous tile's TMA store to drain
-  // r_t <= 128 with two warpgroups: four accumulators and a six-stage ring (see the top of the file)
-  const bool acc4 = nkt <= 2;
-  const int ns = acc4 ? 6 : DEC_NS;
-  auto sStage = [=](int s) { return s < 4 ? sRing + (uint32_t)s * BB_STAGE_BYTES : sP + 32768u + (uint32_t)(s - 4) * BB_STAGE_BYTES; };
+  BBCell *sc_cell = (BBCell *)(sm + DEC_P_BYTES + DEC_H_BYTES + DEC_BIG_BYTES + 512);
+  for (int i = threadIdx.x; i < (int)(sizeof(BBCell) / 16); i += LY::THREADS) ((uint4 *)sc_cell)[i] = __ldg((const uint4 *)&cg + i);
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
-    mbar_init(bSetup, 1); mbar_init(bPdone, 1); mbar_init(bPready, NWG * 128);
+    mbar_init(bSetup, 1); mbar_init(bHready, NWG * 128);
     for (int s = 0; s < 6; ++s) { mbar_init(bFull(s), 1); mbar_init(bEmpty(s), 1); }
     for (int b = 0; b < 4; ++b) { mbar_init(bTfull(b), 1); mbar_init(bTempty(b), 128); mbar_init(bRready(b), 128); }
     fence_barrier_init();
@@ -560,18 +632,25 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  JOLT_DBG(if (kdbg) kdbg[1] = clock64();)
+  const BBCell &c = *sc_cell;            // scalar fields from here on; tensor maps through cg
+  const int nkt = (c.r_t + 63) / 64;
+  const uint32_t panel = (uint32_t)c.r_t * 128u;       // bytes of one 64-feature panel of P (r_t is a multiple of 16)
+  const bool has_res = c.bits > 0;
+  // r_t <= 128 leaves half of the P region free: it extends the ring to six stages, and each warpgroup owns two
+  // accumulators (see the top of the file)
+  const bool acc4 = nkt <= 2;
+  const int ns = acc4 ? 6 : DEC_NS;
+  auto sStage = [=](int s) { return s < 4 ? sRing + (uint32_t)s * BB_STAGE_BYTES : sP + 32768u + (uint32_t)(s - 4) * BB_STAGE_BYTES; };
 
   if (wg == NWG) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(LY::PROD_REGS));
     if (warp == NWG * 4 && lane == 0) {
       // ---------------- TMA producer
-      tma_prefetch_desc(&c.tmUT); tma_prefetch_desc(&c.tmUF); tma_prefetch_desc(&c.tmG);
-      mbar_expect_tx(bSetup, (uint32_t)nkf * (16384u + (uint32_t)c.r_t * 128u));
-      for (int kb = 0; kb < nkf; ++kb) {
-        tma_load_2d(sBig + kb * 16384, &c.tmUF, bSetup, kb * 64, 0);
-        tma_load_2d(sBig + 32768 + kb * 32768, &c.tmG, bSetup, kb * 64, h * c.r_t);
-      }
-      bool ok = mbar_wait(bPdone, 0, abort_flag);
+      mbar_expect_tx(bSetup, 2u * panel);
+      tma_load_2d(sP, &cg.tmP, bSetup, 0, h * c.r_t);
+      tma_load_2d(sP + panel, &cg.tmP, bSetup, 64, h * c.r_t);
+      bool ok = true;
       int cnt = 0;
       for (int i = 0; ok && i < n_tiles; ++i) {
         const int tt = tile0 + i;
@@ -580,140 +659,100 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
           ok = mbar_wait(bEmpty(s), (n & 1) ^ 1, abort_flag);
           if (!ok) break;
           mbar_expect_tx(bFull(s), BB_STAGE_BYTES);
-          tma_load_2d(sStage(s), &c.tmUT, bFull(s), kb * 64, tt * 128);
+          tma_load_2d(sStage(s), &cg.tmUT, bFull(s), kb * 64, tt * 128);
         }
       }
     } else if (warp == NWG * 4 + 1 && lane == 0) {
       // ---------------- MMA issuer (one thread, tiles in order: the ring's phase parities stay unambiguous)
-      bool ok = mbar_wait(bSetup, 0, abort_flag);
+      bool ok = mbar_wait(bSetup, 0, abort_flag);        // the head's projected core has landed
+      if (ok) ok = mbar_wait(bHready, 0, abort_flag);    // the rotation operand is built
       if (ok) {
         tc_fence_after();
-        const uint32_t idescP = umma_idesc_f16(128, c.r_t, 0, 0);
-        for (int kb = 0; kb < nkf; ++kb) {
-          const uint64_t da = umma_desc_sw128(sBig + kb * 16384, 16, 1024), db = umma_desc_sw128(sBig + 32768 + kb * 32768, 16, 1024);
-#pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4) umma_f16(tmem_base, umma_desc_kslice(da, k4), umma_desc_kslice(db, k4), idescP, (kb | k4) != 0);
-        }
-        umma_commit(bPdone);
-        ok = mbar_wait(bPready, 0, abort_flag);
-      }
-      if (ok) {
-        tc_fence_after();
-        const uint32_t idesc = umma_idesc_f16(128, 128, 0, 0);
-        // With four accumulators the backbone MMAs run `lead` tiles ahead of the rotation MMAs: a ring stage is
-        // released (and the next U_T tile requested) that much earlier, so the load latency hides behind the
-        // tiles whose backbone already waits in TMEM.  MMAs on one accumulator are still issued in order.
-        const int lead = acc4 ? 2 : 0;
-        // tile descriptors built once; per MMA only the K-slice step remains
-        const uint64_t dP0 = umma_desc_sw128(sP, 16, 1024), dH0 = umma_desc_sw128(sH, 16, 1024);
+        const uint32_t idesc = umma_idesc_f16(128, 128, 0, 0);      // rotation: both operands K-major
+        const uint32_t idescB = umma_idesc_f16(128, 128, 0, 1);     // backbone: B = P panels, MN-major
+        const int ksteps = c.r_t / 16;
+        // Two streams of work share this thread: the backbone of tile jb (needs its accumulator released and its
+        // U_T stages landed) and the rotation of tile jr < jb (needs the warpgroup's operand tile).  Whichever is
+        // ready goes first, the rotation preferred since an epilogue warpgroup waits for it: a late U_T stage then
+        // never holds back a rotation whose operands are complete.  With four accumulators the backbone runs up to
+        // three tiles ahead, so backbones wait in TMEM instead of U_T tiles in shared memory.  MMAs on one
+        // accumulator are still issued in order (backbone, then rotation, of the same tile).
+        // Tile descriptors are built once; per MMA only the K-slice step remains.
+        // P: 16 contraction rows = 2048 B per step, the second 64 features one panel further
+        const uint64_t dP0 = umma_desc_sw128(sP, panel, 1024), dH0 = umma_desc_sw128(sH, 16, 1024);
         const uint64_t dS0 = umma_desc_sw128(sRing, 16, 1024), dS4 = umma_desc_sw128(sP + 32768, 16, 1024);
         const uint64_t dR0 = umma_desc_sw128(sR, 16, 1024);
         constexpr uint64_t kStep16K = 16384 >> 4, kStep32K = 32768 >> 4;      // address-field steps
-        int cnt = 0;
-        for (int j = 0; ok && j < n_tiles + lead; ++j) {
-          if (j < n_tiles) {
-            // accumulator / barrier index b and how often it has been used (nb)
-            const int wgi = j % NWG, ni = j / NWG;
-            const int b = acc4 ? wgi + 2 * (ni & 1) : wgi, nb = acc4 ? ni >> 1 : ni;
-            ok = mbar_wait(bTempty(b), (nb & 1) ^ 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t tacc = tmem_base + b * 128;
-            for (int kb = 0; kb < nkt; ++kb, ++cnt) {
-              const int s = cnt % ns, n = cnt / ns;
-              ok = mbar_wait(bFull(s), n & 1, abort_flag);
-              if (!ok) break;
-              tc_fence_after();
-              const uint64_t da = s < 4 ? dS0 + (uint64_t)s * kStep16K : dS4 + (uint64_t)(s - 4) * kStep16K;
-              const uint64_t db = dP0 + (uint64_t)kb * kStep16K;
+        auto acc_of = [=](int t, int &b, int &nb) {      // accumulator / barrier index of tile t and how often it was used before
+          const int wgi = t % NWG, ni = t / NWG;
+          b = acc4 ? wgi + 2 * (ni & 1) : wgi; nb = acc4 ? ni >> 1 : ni;
+        };
+        int jb = 0, jr = 0, kb = 0, cnt = 0;
+        bool acc_free = false;
+        long long t_last = clock64();
+        const long long limit = g_spin_limit;
+        while (jr < n_tiles) {
+          bool progressed = false;
+          if (jr < jb) {
+            int b, nb;
+            acc_of(jr, b, nb);
+            if (!has_res || mbar_test(bRready(b), nb & 1)) {
+              if (has_res) {
+                tc_fence_after();
+                const uint32_t tacc = tmem_base + b * 128;
+                const uint64_t dR = dR0 + (uint64_t)(jr % NWG) * kStep32K;
 #pragma unroll
-              for (int k4 = 0; k4 < 4; ++k4) umma_f16(tacc, umma_desc_kslice(da, k4), umma_desc_kslice(db, k4), idesc, (kb | k4) != 0);
-              umma_commit(bEmpty(s));
+                for (int k2 = 0; k2 < 2; ++k2)
+#pragma unroll
+                  for (int k4 = 0; k4 < 4; ++k4)
+                    umma_f16(tacc, umma_desc_kslice(dR + k2 * kStep16K, k4), umma_desc_kslice(dH0 + k2 * kStep16K, k4), idesc, 1);
+              }
+              umma_commit(bTfull(b));
+              ++jr;
+              progressed = true;
             }
-            if (!ok) break;
           }
-          if (j >= lead) {
-            const int t = j - lead;
-            const int wgi = t % NWG, ni = t / NWG;
-            const int b = acc4 ? wgi + 2 * (ni & 1) : wgi, nb = acc4 ? ni >> 1 : ni;
-            if (has_res) {
-              ok = mbar_wait(bRready(b), nb & 1, abort_flag);
-              if (!ok) break;
+          if (jb < n_tiles) {
+            int b, nb;
+            acc_of(jb, b, nb);
+            if (!acc_free && mbar_test(bTempty(b), (nb & 1) ^ 1)) acc_free = true;
+            const int s = cnt % ns, n = cnt / ns;
+            if (acc_free && mbar_test(bFull(s), n & 1)) {
               tc_fence_after();
               const uint32_t tacc = tmem_base + b * 128;
-              const uint64_t dR = dR0 + (uint64_t)wgi * kStep32K;
+              const uint64_t da = s < 4 ? dS0 + (uint64_t)s * kStep16K : dS4 + (uint64_t)(s - 4) * kStep16K;
+              const uint64_t db = dP0 + (uint64_t)kb * (8192 >> 4);
 #pragma unroll
-              for (int kb = 0; kb < 2; ++kb)
-#pragma unroll
-                for (int k4 = 0; k4 < 4; ++k4)
-                  umma_f16(tacc, umma_desc_kslice(dR + kb * kStep16K, k4), umma_desc_kslice(dH0 + kb * kStep16K, k4), idesc, 1);
+              for (int k4 = 0; k4 < 4; ++k4)
+                if (kb * 4 + k4 < ksteps) umma_f16(tacc, umma_desc_kslice(da, k4), db + (uint64_t)k4 * (2048 >> 4), idescB, (kb | k4) != 0);
+              umma_commit(bEmpty(s));
+              ++cnt;
+              if (++kb == nkt) { kb = 0; acc_free = false; ++jb; }
+              progressed = true;
             }
-            umma_commit(bTfull(b));
           }
+          if (progressed) { t_last = clock64(); continue; }
+          if (*abort_flag) break;
+          if (clock64() - t_last > limit) { *abort_flag = 1; break; }
         }
       }
     }
   } else {
     // ---------------- epilogue warpgroups
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(LY::EPI_REGS));
+    JOLT_DBG(if (kdbg) kdbg[2] = clock64();)
     const int q = warp & 3;
     const int rit = q * 32 + lane;                 // row in tile
     const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
-    {  // B operand of the inverse rotation: Hs[f][f'] = s_f * (-1)^popcount(f & f'), fp16, K-major, swizzled
-      uint32_t sw[4];
-      cell_sign_words(seed, c.cell, sw);
-      const int et = wg * 128 + rit;               // 2048 16-byte chunks over all epilogue threads
-      for (int ci = et; ci < 2048; ci += NWG * 128) {
-        const int f = ci >> 4, chunk = ci & 15;
-        const uint32_t sgn = (sw[f >> 5] >> (f & 31)) & 1u;
-        uint4 pk;
-        uint32_t *pw = (uint32_t *)&pk;
-#pragma unroll
-        for (int e2 = 0; e2 < 4; ++e2) {
-          const int fp = chunk * 8 + e2 * 2;
-          const uint32_t n0 = (__popc(f & fp) & 1u) ^ sgn, n1 = (__popc(f & (fp + 1)) & 1u) ^ sgn;
-          pw[e2] = (0x3C00u | (n0 << 15)) | ((0x3C00u | (n1 << 15)) << 16);      // +-1.0 in fp16
-        }
-        *(uint4 *)(smH + (chunk >> 3) * 16384 + f * 128 + (((chunk & 7) ^ (f & 7)) << 4)) = pk;
-      }
-    }
-    JOLT_DBG(if (kdbg) kdbg[1] = clock64();)
-    bool ok = __all_sync(0xffffffffu, mbar_wait(bPdone, 0, abort_flag));
-    JOLT_DBG(if (kdbg) kdbg[2] = clock64();)
-    if (ok) {
-      tc_fence_after();
-      for (int ch = wg; ch < 2 * nkt; ch += NWG) {
-        float v[32];
-        tmem_ld32(t_lane + ch * 32, v);
-        tmem_wait_ld();
-        unsigned char *rowp = sm + (ch >> 1) * 16384 + rit * 128;
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          uint4 pk;
-          __half2 *hp = (__half2 *)&pk;
-#pragma unroll
-          for (int e2 = 0; e2 < 4; ++e2) {
-            const int col = ch * 32 + jj * 8 + e2 * 2;
-            hp[e2] = __floats2half2_rn(col < c.r_t ? v[jj * 8 + e2 * 2] : 0.f, col + 1 < c.r_t ? v[jj * 8 + e2 * 2 + 1] : 0.f);
-          }
-          *(uint4 *)(rowp + ((((ch & 1) * 4 + jj) ^ (rit & 7)) << 4)) = pk;
-        }
-      }
-      fence_proxy_async();
-      tc_fence_before();
-      mbar_arrive(bPready);
-    }
-    JOLT_DBG(if (kdbg) kdbg[3] = clock64();)
-    const int ex = ok ? *c.e : 0;
-    const float scale = ldexpf(1.0f, ex);
-    const float pre = ldexpf(kInvSqrtD, -ex);        // residual operand is kept in the accumulator's units
-    if (ok) {
+    {
       DecCtx x;
-      x.bTfull = bTfull(wg); x.bTempty = bTempty(wg); x.bRready = bRready(wg);
-      x.t_acc = t_lane + wg * 128; x.rbuf = smR + wg * 32768;
+      x.cg = &cg;
+      x.ex = *c.e;             // requested now, first used after the rotation operand is built
+      x.bTfull = bTfull(wg); x.bTempty = bTempty(wg); x.bRready = bRready(wg); x.bHready = bHready;
+      x.t_acc = t_lane + wg * 128; x.rbuf = smR + wg * 32768; x.smH = smH; x.seed = seed;
       x.s_obuf = sR + wg * 32768; x.obuf = x.rbuf;
       x.abort_flag = abort_flag; x.wg = wg; x.nwg = NWG; x.rit = rit; x.h = h; x.tile0 = tile0; x.n_tiles = n_tiles;
-      x.l = h / c.n_heads; x.hd = h - x.l * c.n_heads; x.scale = scale; x.pre = pre;
+      x.l = h / c.n_heads; x.hd = h - x.l * c.n_heads;
       if (acc4 && c.rope) {
         switch (c.bits) {
           case 0: dec_tile_loop_acc4_rope<0>(c, x); break;

@@ -204,7 +204,9 @@ __global__ void __launch_bounds__(OR_THREADS, 1) orth_gram_kernel(const OrthCell
 // upper triangle X, the diagonal of X in `invd`).  Per panel: (1) warp 0 factors the 8 x 8 diagonal block in
 // registers, (2) one thread per row solves its 8 panel entries against the block (rows above the panel are rows of X,
 // rows below are rows of L, the same recurrence), (3) the trailing update W[i][j] -= sum_c P[i][c] P[j][c] for the
-// rows of X (i < panel end) and of the Schur complement (i >= j), four columns per warp pass.  Three barriers per panel.
+// rows of X (i < panel end) and of the Schur complement (i >= j): first the next panel's eight columns, then -- while
+// warp 0 already factors the next diagonal block (look-ahead) -- the rest, four columns per warp pass.  Three barriers
+// per panel.
 // A pivot not above `dead_rel` of its original diagonal entry belongs to a direction that is dependent to working
 // accuracy: its column of L and its row / column of L^-1 are zero, status bit 1.
 // Input: fp32 row-chunk partials of the Gram kernel (summed here in fp64) or an fp64 matrix.  Output: L^-1 as fp16
@@ -261,48 +263,52 @@ __global__ void __launch_bounds__(kCholInvThreads, 1) cholinv_kernel(const CholI
   __syncthreads();
   for (int i = tid; i < n; i += nt) diag0[i] = W[(size_t)i * n + i];
   __syncthreads();
-  for (int j0 = 0; j0 < n; j0 += 8) {
+  // (1) the 8 x 8 diagonal block at j0: every lane of warp 0 factors it in registers (broadcast loads, no shuffles on
+  // the dependent chain), then publishes the block and the reciprocal pivots
+  auto factor_block = [&](int j0) {
     const int w = min(8, n - j0);
-    if (tid < 32) {
-      double Lb[8][8], piv[8];
-      int dead = 0;
+    double Lb[8][8], piv[8];
+    int dead = 0;
 #pragma unroll
-      for (int r = 0; r < 8; ++r)
+    for (int r = 0; r < 8; ++r)
 #pragma unroll
-        for (int cc = 0; cc <= r; ++cc) Lb[r][cc] = (r < w && cc < w) ? W[(size_t)(j0 + cc) * n + j0 + r] : (r == cc ? 1.0 : 0.0);
+      for (int cc = 0; cc <= r; ++cc) Lb[r][cc] = (r < w && cc < w) ? W[(size_t)(j0 + cc) * n + j0 + r] : (r == cc ? 1.0 : 0.0);
 #pragma unroll
-      for (int cc = 0; cc < 8; ++cc) {
-        piv[cc] = 0.0;
-        if (cc < w) {
-          const double d = Lb[cc][cc], dg = diag0[j0 + cc];
-          const bool bad = !(d > t.dead_rel * dg) || !(dg > 0);
-          const double rs = bad ? 0.0 : rsqrt_pos(d);
-          Lb[cc][cc] = bad ? 0.0 : d * rs;
-          dead |= bad ? 1 : 0;
-          piv[cc] = rs;
+    for (int cc = 0; cc < 8; ++cc) {
+      piv[cc] = 0.0;
+      if (cc < w) {
+        const double d = Lb[cc][cc], dg = diag0[j0 + cc];
+        const bool bad = !(d > t.dead_rel * dg) || !(dg > 0);
+        const double rs = bad ? 0.0 : rsqrt_pos(d);
+        Lb[cc][cc] = bad ? 0.0 : d * rs;
+        dead |= bad ? 1 : 0;
+        piv[cc] = rs;
 #pragma unroll
-          for (int r = cc + 1; r < 8; ++r) Lb[r][cc] *= rs;
+        for (int r = cc + 1; r < 8; ++r) Lb[r][cc] *= rs;
 #pragma unroll
-          for (int c2 = cc + 1; c2 < 8; ++c2)
+        for (int c2 = cc + 1; c2 < 8; ++c2)
 #pragma unroll
-            for (int r = c2; r < 8; ++r) Lb[r][c2] = fma(-Lb[r][cc], Lb[c2][cc], Lb[r][c2]);
-        }
-      }
-      if (tid < 8) {
-#pragma unroll
-        for (int rr = 0; rr < 8; ++rr)
-          if (rr == tid) {
-#pragma unroll
-            for (int cc = 0; cc < 8; ++cc) blkd[rr][cc] = cc <= rr ? Lb[rr][cc] : 0.0;
-          }
-      }
-      if (tid == 0) {
-#pragma unroll
-        for (int cc = 0; cc < 8; ++cc) ipiv[cc] = piv[cc];
-        if (dead) s_dead = 1;
+          for (int r = c2; r < 8; ++r) Lb[r][c2] = fma(-Lb[r][cc], Lb[c2][cc], Lb[r][c2]);
       }
     }
-    __syncthreads();
+    if (lane < 8) {
+#pragma unroll
+      for (int rr = 0; rr < 8; ++rr)
+        if (rr == lane) {
+#pragma unroll
+          for (int cc = 0; cc < 8; ++cc) blkd[rr][cc] = cc <= rr ? Lb[rr][cc] : 0.0;
+        }
+    }
+    if (lane == 0) {
+#pragma unroll
+      for (int cc = 0; cc < 8; ++cc) ipiv[cc] = piv[cc];
+      if (dead) s_dead = 1;
+    }
+  };
+  if (warp == 0) factor_block(0);
+  __syncthreads();
+  for (int j0 = 0; j0 < n; j0 += 8) {
+    const int w = min(8, n - j0);
     // (2) the panel entries of every row: x_c = (p_c - sum_{l<c} x_l L[c][l]) / L[c][c]
     for (int i = tid; i < n; i += nt) {
       const int r = i - j0;                   // row inside the panel when 0 <= r < w
@@ -331,27 +337,51 @@ __global__ void __launch_bounds__(kCholInvThreads, 1) cholinv_kernel(const CholI
       }
     }
     __syncthreads();
-    // (3) trailing update, four columns per warp pass; rows i < m0 belong to X, rows i >= column to the Schur complement
     const int m0 = j0 + w;
-    for (int j = m0 + 4 * warp; j < n; j += 4 * nw) {
-      double pj[4][8];
+    if (m0 >= n) break;
+    // (3a) trailing update of the NEXT panel's columns only (one thread per row), so that warp 0 can factor the next
+    // diagonal block while the other warps finish the update (look-ahead)
+    const int wn = min(8, n - m0);
+    for (int i = tid; i < n; i += nt) {
+      double pi[8];
 #pragma unroll
-      for (int q = 0; q < 4; ++q)
+      for (int cc = 0; cc < 8; ++cc) pi[cc] = pan[cc * n + i];
 #pragma unroll
-        for (int cc = 0; cc < 8; ++cc) pj[q][cc] = (j + q < n) ? pan[cc * n + j + q] : 0.0;
-      const int nv = m0 + (n - j);
-      for (int v = lane; v < nv; v += 32) {
-        const int i = v < m0 ? v : j + (v - m0);
-        double acc[4] = {0, 0, 0, 0};
+      for (int q = 0; q < 8; ++q) {
+        const int j = m0 + q;
+        if (q < wn && (i < m0 || i >= j)) {
+          double a0 = 0, a1 = 0;
 #pragma unroll
-        for (int cc = 0; cc < 8; ++cc) {
-          const double pv = pan[cc * n + i];
-#pragma unroll
-          for (int q = 0; q < 4; ++q) acc[q] = fma(pv, pj[q][cc], acc[q]);
+          for (int cc = 0; cc < 8; cc += 2) { a0 = fma(pi[cc], pan[cc * n + j], a0); a1 = fma(pi[cc + 1], pan[(cc + 1) * n + j], a1); }
+          W[(size_t)j * n + i] -= a0 + a1;
         }
+      }
+    }
+    __syncthreads();
+    // (1') next diagonal block on warp 0 || (3b) the other columns on the other warps, four columns per warp pass;
+    // rows i < m0 belong to X, rows i >= column to the Schur complement
+    if (warp == 0) factor_block(m0);
+    else {
+      for (int j = m0 + wn + 4 * (warp - 1); j < n; j += 4 * (nw - 1)) {
+        double pj[4][8];
 #pragma unroll
         for (int q = 0; q < 4; ++q)
-          if (j + q < n && (i < m0 || i >= j + q)) W[(size_t)(j + q) * n + i] -= acc[q];
+#pragma unroll
+          for (int cc = 0; cc < 8; ++cc) pj[q][cc] = (j + q < n) ? pan[cc * n + j + q] : 0.0;
+        const int nv = m0 + (n - j);
+        for (int v = lane; v < nv; v += 32) {
+          const int i = v < m0 ? v : j + (v - m0);
+          double acc[4] = {0, 0, 0, 0};
+#pragma unroll
+          for (int cc = 0; cc < 8; ++cc) {
+            const double pv = pan[cc * n + i];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[q] = fma(pv, pj[q][cc], acc[q]);
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (j + q < n && (i < m0 || i >= j + q)) W[(size_t)(j + q) * n + i] -= acc[q];
+        }
       }
     }
     __syncthreads();
