@@ -138,6 +138,21 @@ __device__ __forceinline__ void dec_unpack_row_row(const DecCodesRow<BITS> &d, f
 // sectors per load instruction), BITS neighbouring lanes fetch the BITS chunks of one row: a warp instruction then
 // reads 512 contiguous bytes, and after BITS instructions the warp holds the codes of its 32 rows.  Each lane
 // dequantises the 128 / BITS features of the chunks it holds and writes them into the operand tile itself.
+// Which chunk of which of the instruction's rows a lane fetches.  Any assignment covers the same 512 contiguous
+// bytes per load instruction; this one is chosen for the 16-byte shared-memory stores of the dequantised values,
+// which the hardware serves a quarter-warp (8 lanes) at a time: the 8 lanes of a quarter must hit 8 different
+// 16-byte columns of the swizzled operand tile, i.e. (column ^ row) & 7 all different.
+//   8-bit: a quarter takes 4 chunks (one 64-feature panel) of 2 rows;  4-bit: 2 chunks of 4 rows;
+//   2-bit: 1 chunk of 8 rows;  1-bit: the single chunk of 8 rows.
+template <int BITS>
+__device__ __forceinline__ void dec_lane_map(int lane, int &chunk, int &rsub) {
+  const int q = lane >> 3, i = lane & 7;
+  if constexpr (BITS == 8) { chunk = (q & 1) * 4 + (i & 3); rsub = (q >> 1) * 2 + (i >> 2); }
+  else if constexpr (BITS == 4) { chunk = (q >> 1) * 2 + (i >> 2); rsub = (q & 1) * 4 + (i & 3); }
+  else if constexpr (BITS == 2) { chunk = q & 1; rsub = (q >> 1) * 8 + i; }
+  else { chunk = 0; rsub = lane; }
+}
+
 template <int BITS>
 struct DecCodes {
   static constexpr bool kCoop = BITS == 8 || BITS == 4 || BITS == 2 || BITS == 1;
@@ -157,7 +172,8 @@ __device__ __forceinline__ void dec_load_codes(const BBCell &c, long long row, D
     constexpr int RPI = 32 / BITS;                            // rows per load instruction
     const int lane = threadIdx.x & 31;
     const long long wrow = row - lane;                        // first row of this warp's 32-row slab
-    const int chunk = lane % BITS, rsub = lane / BITS;
+    int chunk, rsub;
+    dec_lane_map<BITS>(lane, chunk, rsub);
 #pragma unroll
     for (int it = 0; it < BITS; ++it) {
       const long long r = wrow + it * RPI + rsub;
@@ -187,7 +203,8 @@ __device__ __forceinline__ void dec_unpack_row(const DecCodes<BITS> &d, float pr
     constexpr int RPI = 32 / BITS, NV = 128 / BITS;           // rows per instruction, values per chunk
     constexpr float c0 = -(8388608.0f + (float)(1 << (BITS - 1)));
     const int lane = rit & 31, wrow0 = rit & ~31;
-    const int chunk = lane % BITS, rsub = lane / BITS;
+    int chunk, rsub;
+    dec_lane_map<BITS>(lane, chunk, rsub);
 #pragma unroll
     for (int it = 0; it < BITS; ++it) {
       const int row = wrow0 + it * RPI + rsub;                // row of the tile this chunk belongs to
@@ -612,6 +629,7 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
   auto bTfull = [=](int b) { return sBar + 120 + 8 * b; };        // up to 4 accumulators
   auto bTempty = [=](int b) { return sBar + 152 + 8 * b; };
   auto bRready = [=](int b) { return sBar + 184 + 8 * b; };
+  auto bBB = [=](int b) { return sBar + 216 + 8 * b; };           // backbone of the accumulator's tile complete
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = warp >> 2;
@@ -624,7 +642,7 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
     *abort_flag = 0;
     mbar_init(bSetup, 1); mbar_init(bHready, NWG * 128);
     for (int s = 0; s < 6; ++s) { mbar_init(bFull(s), 1); mbar_init(bEmpty(s), 1); }
-    for (int b = 0; b < 4; ++b) { mbar_init(bTfull(b), 1); mbar_init(bTempty(b), 128); mbar_init(bRready(b), 128); }
+    for (int b = 0; b < 4; ++b) { mbar_init(bTfull(b), 1); mbar_init(bTempty(b), 128); mbar_init(bRready(b), 128); mbar_init(bBB(b), 1); }
     fence_barrier_init();
   }
   if (warp == NWG * 4) { tmem_alloc(smem_u32(tmem_slot), LY::TMEM_COLS); tmem_relinquish(); }
@@ -663,77 +681,71 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_kernel(const BBC
         }
       }
     } else if (warp == NWG * 4 + 1 && lane == 0) {
-      // ---------------- MMA issuer (one thread, tiles in order: the ring's phase parities stay unambiguous)
+      // ---------------- backbone MMA issuer.  Issuing an MMA costs its thread tens of cycles of dependent
+      // instructions, and a tile needs sixteen of them: the two halves of a tile's accumulation (backbone, rotation)
+      // are issued by two threads on different schedulers, ordered per accumulator through bBB.  The backbone thread
+      // runs ahead as far as free accumulators and landed U_T stages allow (two accumulators per warpgroup when
+      // r_t <= 128), so backbones wait in TMEM instead of U_T tiles in shared memory, and a late U_T stage never
+      // holds back a rotation whose operands are complete.
       bool ok = mbar_wait(bSetup, 0, abort_flag);        // the head's projected core has landed
-      if (ok) ok = mbar_wait(bHready, 0, abort_flag);    // the rotation operand is built
       if (ok) {
         tc_fence_after();
-        const uint32_t idesc = umma_idesc_f16(128, 128, 0, 0);      // rotation: both operands K-major
-        const uint32_t idescB = umma_idesc_f16(128, 128, 0, 1);     // backbone: B = P panels, MN-major
+        const uint32_t idescB = umma_idesc_f16(128, 128, 0, 1);     // A = U_T tile, K-major; B = P panels, MN-major
         const int ksteps = c.r_t / 16;
-        // Two streams of work share this thread: the backbone of tile jb (needs its accumulator released and its
-        // U_T stages landed) and the rotation of tile jr < jb (needs the warpgroup's operand tile).  Whichever is
-        // ready goes first, the rotation preferred since an epilogue warpgroup waits for it: a late U_T stage then
-        // never holds back a rotation whose operands are complete.  With four accumulators the backbone runs up to
-        // three tiles ahead, so backbones wait in TMEM instead of U_T tiles in shared memory.  MMAs on one
-        // accumulator are still issued in order (backbone, then rotation, of the same tile).
-        // Tile descriptors are built once; per MMA only the K-slice step remains.
         // P: 16 contraction rows = 2048 B per step, the second 64 features one panel further
-        const uint64_t dP0 = umma_desc_sw128(sP, panel, 1024), dH0 = umma_desc_sw128(sH, 16, 1024);
+        const uint64_t dP0 = umma_desc_sw128(sP, panel, 1024);
         const uint64_t dS0 = umma_desc_sw128(sRing, 16, 1024), dS4 = umma_desc_sw128(sP + 32768, 16, 1024);
-        const uint64_t dR0 = umma_desc_sw128(sR, 16, 1024);
-        constexpr uint64_t kStep16K = 16384 >> 4, kStep32K = 32768 >> 4;      // address-field steps
-        auto acc_of = [=](int t, int &b, int &nb) {      // accumulator / barrier index of tile t and how often it was used before
-          const int wgi = t % NWG, ni = t / NWG;
-          b = acc4 ? wgi + 2 * (ni & 1) : wgi; nb = acc4 ? ni >> 1 : ni;
-        };
-        int jb = 0, jr = 0, kb = 0, cnt = 0;
-        bool acc_free = false;
-        long long t_last = clock64();
-        const long long limit = g_spin_limit;
-        while (jr < n_tiles) {
-          bool progressed = false;
-          if (jr < jb) {
-            int b, nb;
-            acc_of(jr, b, nb);
-            if (!has_res || mbar_test(bRready(b), nb & 1)) {
-              if (has_res) {
-                tc_fence_after();
-                const uint32_t tacc = tmem_base + b * 128;
-                const uint64_t dR = dR0 + (uint64_t)(jr % NWG) * kStep32K;
-#pragma unroll
-                for (int k2 = 0; k2 < 2; ++k2)
-#pragma unroll
-                  for (int k4 = 0; k4 < 4; ++k4)
-                    umma_f16(tacc, umma_desc_kslice(dR + k2 * kStep16K, k4), umma_desc_kslice(dH0 + k2 * kStep16K, k4), idesc, 1);
-              }
-              umma_commit(bTfull(b));
-              ++jr;
-              progressed = true;
-            }
-          }
-          if (jb < n_tiles) {
-            int b, nb;
-            acc_of(jb, b, nb);
-            if (!acc_free && mbar_test(bTempty(b), (nb & 1) ^ 1)) acc_free = true;
+        constexpr uint64_t kStep16K = 16384 >> 4;      // address-field step
+        int cnt = 0;
+        for (int j = 0; ok && j < n_tiles; ++j) {
+          // accumulator / barrier index b of tile j and how often it was used before (nb)
+          const int wgi = j % NWG, ni = j / NWG;
+          const int b = acc4 ? wgi + 2 * (ni & 1) : wgi, nb = acc4 ? ni >> 1 : ni;
+          ok = mbar_wait(bTempty(b), (nb & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t tacc = tmem_base + b * 128;
+          for (int kb = 0; kb < nkt; ++kb, ++cnt) {
             const int s = cnt % ns, n = cnt / ns;
-            if (acc_free && mbar_test(bFull(s), n & 1)) {
-              tc_fence_after();
-              const uint32_t tacc = tmem_base + b * 128;
-              const uint64_t da = s < 4 ? dS0 + (uint64_t)s * kStep16K : dS4 + (uint64_t)(s - 4) * kStep16K;
-              const uint64_t db = dP0 + (uint64_t)kb * (8192 >> 4);
+            ok = mbar_wait(bFull(s), n & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t da = s < 4 ? dS0 + (uint64_t)s * kStep16K : dS4 + (uint64_t)(s - 4) * kStep16K;
+            const uint64_t db = dP0 + (uint64_t)kb * (8192 >> 4);
 #pragma unroll
-              for (int k4 = 0; k4 < 4; ++k4)
-                if (kb * 4 + k4 < ksteps) umma_f16(tacc, umma_desc_kslice(da, k4), db + (uint64_t)k4 * (2048 >> 4), idescB, (kb | k4) != 0);
-              umma_commit(bEmpty(s));
-              ++cnt;
-              if (++kb == nkt) { kb = 0; acc_free = false; ++jb; }
-              progressed = true;
-            }
+            for (int k4 = 0; k4 < 4; ++k4)
+              if (kb * 4 + k4 < ksteps) umma_f16(tacc, umma_desc_kslice(da, k4), db + (uint64_t)k4 * (2048 >> 4), idescB, (kb | k4) != 0);
+            umma_commit(bEmpty(s));
           }
-          if (progressed) { t_last = clock64(); continue; }
-          if (*abort_flag) break;
-          if (clock64() - t_last > limit) { *abort_flag = 1; break; }
+          if (ok) umma_commit(bBB(b));
+        }
+      }
+    } else if (warp == NWG * 4 + 2 && lane == 0) {
+      // ---------------- rotation MMA issuer: A = the warpgroup's dequantised residual tile, B = H
+      bool ok = mbar_wait(bHready, 0, abort_flag);    // the rotation operand is built
+      if (ok) {
+        tc_fence_after();
+        const uint32_t idesc = umma_idesc_f16(128, 128, 0, 0);      // both operands K-major
+        const uint64_t dH0 = umma_desc_sw128(sH, 16, 1024), dR0 = umma_desc_sw128(sR, 16, 1024);
+        constexpr uint64_t kStep16K = 16384 >> 4, kStep32K = 32768 >> 4;      // address-field steps
+        uint64_t dH[8];
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) dH[ks] = umma_desc_kslice(dH0 + (uint64_t)(ks >> 2) * kStep16K, ks & 3);
+        for (int j = 0; ok && j < n_tiles; ++j) {
+          const int wgi = j % NWG, ni = j / NWG;
+          const int b = acc4 ? wgi + 2 * (ni & 1) : wgi, nb = acc4 ? ni >> 1 : ni;
+          ok = mbar_wait(bBB(b), nb & 1, abort_flag);                 // the tile's backbone is in the accumulator
+          if (ok && has_res) ok = mbar_wait(bRready(b), nb & 1, abort_flag);
+          if (!ok) break;
+          if (has_res) {
+            tc_fence_after();
+            const uint32_t tacc = tmem_base + b * 128;
+            const uint64_t dR = dR0 + (uint64_t)wgi * kStep32K;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+              umma_f16(tacc, umma_desc_kslice(dR + (uint64_t)(ks >> 2) * kStep16K, ks & 3), dH[ks], idesc, 1);
+          }
+          umma_commit(bTfull(b));
         }
       }
     }
