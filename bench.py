@@ -485,19 +485,36 @@ def main():
         from oracle import jolt_oracle as O
         t0 = time.perf_counter()
         sample = {}
+        jolt_err = {}
         for w_ in (0, 1):
             X = (K, V)[w_][gs[0]:gs[1]].reshape(cfg.m, cfg.seq_len, 128).cpu().numpy()
             a = time.perf_counter()
             oc = O.compress_cell(X, *plans[w_], seed=cfg.seed, cell=w_, token_mode="randomized", power_iters=q)
             b_ = time.perf_counter()
-            O.decompress_cell(oc)
+            Xo = O.decompress_cell(oc)
             c_ = time.perf_counter()
             sample[w_] = (b_ - a, c_ - b_)
+            jolt_err["KV"[w_]] = O.rel_frobenius(X, Xo)
         sc = sum(v[0] for v in sample.values()); sd = sum(v[1] for v in sample.values())
         sb = 2 * cfg.m * cfg.seq_len * 128 * 2
         line["cpu_baseline"] = {"value": sb / (sc + sd) / 1e9, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                                 "sample": "cells 0 and 1 (group 0, K and V) of the same cache and plan, numpy fp64",
                                 "compress_gbs": sb / sc / 1e9, "decompress_gbs": sb / sd / 1e9}
+        # error context of the paper's reconstruction table (Sec. 6): the two baselines it lists, restated in the oracle,
+        # on the first 1024 tokens (the table's length) of layer group 0; not timed, not part of the metric
+        from oracle import baselines as BL
+        Tc = min(1024, cfg.seq_len)
+        ctx = {"tokens": Tc, "ratio_target": ratio, "jolt_oracle_full_length": jolt_err,
+               "int4_per_channel": {"ratio": BL.int4_per_channel_ratio(Tc)}, "cross_layer_svd": {}}
+        for w_ in (0, 1):
+            Xg = (K, V)[w_][gs[0]:gs[1], :, :Tc].cpu().numpy().astype("float64")
+            Xh, _ = BL.int4_per_channel(Xg.reshape(-1, Tc, 128))
+            ctx["int4_per_channel"]["KV"[w_]] = BL.rel_frobenius(Xg.reshape(-1, Tc, 128), Xh)
+            Xs, stored, r = BL.cross_layer_svd(Xg, ratio)
+            ctx["cross_layer_svd"]["KV"[w_]] = BL.rel_frobenius(Xg, Xs)
+            ctx["cross_layer_svd"]["rank"] = r
+            ctx["cross_layer_svd"]["ratio"] = Xg.size * 2 / stored
+        line["cpu_baseline"]["error_context"] = ctx
     print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
