@@ -113,6 +113,24 @@ void jolt_default_options(jolt_options *o);
 int jolt_plan(const jolt_layout *layout, const void *dK, const void *dV, double byte_budget,
               const jolt_options *opts, void *stream, jolt_cell_plan *out, double *achieved_bytes);
 
+/* The two halves of jolt_plan, for callers that plan one cache at several budgets or with several allocators (the
+ * ratio sweeps and allocator ablations of Sec. 6): the spectra are measured once and every further plan is host work.
+ * jolt_probe -- Sec. 5: mode-3 Gram eigenvalues and the leading q_cap token-mode singular values of every cell (plus the
+ *   tail-mass value of the randomized probe), measured by one GPU program per cell group on concurrent streams and
+ *   copied to the host in one transfer.  q_cap = opts->q_cap if positive, else the cap policy at `ratio_hint`
+ *   (uncompressed bytes over the byte budget the caller has in mind).  *out: a host object, free with
+ *   jolt_spectra_free; NULL on error.
+ * jolt_plan_from_spectra -- Sec. 4, Eq. (3)/(4) on the kept spectra; no GPU work, token ranks bounded by the probed cap.
+ *   JOLT_EINVAL if the cap policy of this budget asks for more token directions than were probed (probe again with a
+ *   larger q_cap); JOLT_EBUDGET as jolt_plan.
+ * jolt_plan(budget) == jolt_probe(ratio of that budget) followed by jolt_plan_from_spectra(budget). */
+typedef struct jolt_spectra jolt_spectra;
+int jolt_probe(const jolt_layout *layout, const void *dK, const void *dV, double ratio_hint, const jolt_options *opts,
+               void *stream, jolt_spectra **out);
+int jolt_plan_from_spectra(const jolt_spectra *spectra, double byte_budget, const jolt_options *opts,
+                           jolt_cell_plan *out, double *achieved_bytes);
+int jolt_spectra_free(jolt_spectra *spectra);
+
 /* jolt_compress -- paper Sec. 4 "Partial Tucker backbone" + "Rotated residual", Sec. 5 for the
  * randomized token factor.  For every cell: U_F from the mode-3 Gram, U_T (exact or randomized),
  * core G, residual against the stored fp16 backbone, sign-flip + 128-point Hadamard rotation along

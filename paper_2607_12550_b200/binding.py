@@ -50,6 +50,9 @@ lib.jolt_default_options.argtypes = [C.POINTER(Options)]
 lib.jolt_default_options.restype = None
 lib.jolt_plan.argtypes = [C.POINTER(Layout), _vp, _vp, C.c_double, C.POINTER(Options), _vp, C.POINTER(CellPlan),
                           C.POINTER(C.c_double)]
+lib.jolt_probe.argtypes = [C.POINTER(Layout), _vp, _vp, C.c_double, C.POINTER(Options), _vp, C.POINTER(_vp)]
+lib.jolt_plan_from_spectra.argtypes = [_vp, C.c_double, C.POINTER(Options), C.POINTER(CellPlan), C.POINTER(C.c_double)]
+lib.jolt_spectra_free.argtypes = [_vp]
 lib.jolt_compress.argtypes = [C.POINTER(Layout), _vp, _vp, C.POINTER(CellPlan), C.POINTER(Options), _vp, C.POINTER(_vp)]
 lib.jolt_compress_with_factors.argtypes = [C.POINTER(Layout), _vp, _vp, C.POINTER(CellPlan), C.POINTER(Options),
                                            C.POINTER(_vp), C.POINTER(_vp), _vp, C.POINTER(_vp)]
@@ -172,6 +175,40 @@ def jolt_plan(K, V, group_start, byte_budget: float, opts: Options | None = None
                        C.byref(ach))
     _check(st, allow=(EBUDGET,) if allow_budget else ())
     return [(p.r_t, p.r_f, p.bits) for p in out], ach.value
+
+
+class Spectra:
+    """The measured spectra of a cache (host object); plan it at any budget with `plan`."""
+
+    def __init__(self, ptr, n_cells):
+        self.ptr = ptr
+        self.n_cells = n_cells
+
+    def plan(self, byte_budget: float, opts: Options | None = None, allow_budget=False):
+        opts = opts or default_options()
+        out = (CellPlan * self.n_cells)()
+        ach = C.c_double(0)
+        st = lib.jolt_plan_from_spectra(self.ptr, byte_budget, C.byref(opts), out, C.byref(ach))
+        _check(st, allow=(EBUDGET,) if allow_budget else ())
+        return [(p.r_t, p.r_f, p.bits) for p in out], ach.value
+
+    def free(self):
+        if self.ptr:
+            lib.jolt_spectra_free(self.ptr)
+            self.ptr = None
+
+    def __del__(self):
+        if lib is not None:
+            self.free()
+
+
+def jolt_probe(K, V, group_start, ratio_hint: float, opts: Options | None = None, stream=None) -> Spectra:
+    lay = make_layout(K, group_start, V)
+    opts = opts or default_options()
+    ptr = C.c_void_p()
+    _check(lib.jolt_probe(C.byref(lay), K.data_ptr(), V.data_ptr(), float(ratio_hint), C.byref(opts), _stream_ptr(stream),
+                          C.byref(ptr)))
+    return Spectra(ptr, 2 * lay.n_groups)
 
 
 class Handle:

@@ -516,6 +516,8 @@ struct CellWork {      // device scratch of one cell
   double *Gs = nullptr, *Lwork = nullptr;      // Gram of the basis, Cholesky work matrix (k x (k+1)) for k > kCholSmemMaxN
   double *gpart = nullptr; float *LT32 = nullptr, *invd = nullptr;
   double *bjA = nullptr, *bjV = nullptr, *bjJ = nullptr, *bjOff = nullptr; int *bjDone = nullptr;
+  // eigen-solver scratch of the feature stage: its own, since the probe runs that stage concurrently with the token stage
+  double *bjfA = nullptr, *bjfV = nullptr, *bjfJ = nullptr, *bjfOff = nullptr; int *bjfDone = nullptr;
   double *BBt = nullptr, *BBv = nullptr, *BBw = nullptr;
   float *Ut = nullptr, *sigma = nullptr;
   float *UT32 = nullptr, *G32 = nullptr;
@@ -563,6 +565,11 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
         const size_t nbe = (((nmax + kBJBlock - 1) / kBJBlock) + 1) & ~(size_t)1, nP = nbe * kBJBlock;
         w.bjA = b.take<double>(2 * nP * nP); w.bjV = b.take<double>(nP * nP); w.bjJ = b.take<double>(2 * (nbe / 2) * 1024);
         w.bjOff = b.take<double>(4); w.bjDone = b.take<int>(4);
+      }
+      {
+        const size_t nbe = (((kD + kBJBlock - 1) / kBJBlock) + 1) & ~(size_t)1, nP = nbe * kBJBlock;
+        w.bjfA = b.take<double>(2 * nP * nP); w.bjfV = b.take<double>(nP * nP); w.bjfJ = b.take<double>(2 * (nbe / 2) * 1024);
+        w.bjfOff = b.take<double>(4); w.bjfDone = b.take<int>(4);
       }
       w.gram_part = b.take<double>((size_t)c.m * kD * kD * std::max(1, (tok_segments(c.T) + 1) / 2));
       w.C = b.take<double>(kD * kD); w.Cv = b.take<double>(kD * kD); w.Cw = b.take<double>(kD);
@@ -826,14 +833,16 @@ __global__ void __launch_bounds__(1024) subspace_residual_kernel(const ResidJob 
 }
 
 // Stages that produce U_F (fp32), U_T (fp32) and the core (fp32) of every active cell.
+// parts: 1 = the feature stage (mode-3 Gram, eigen-solve), 2 = the token stage and the core, 3 = both.  The two halves
+// may go into different programs only where the token stage does not read U_F (the randomized probe).
 void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool probe, int power_iters, uint64_t seed, bool fast,
-                          bool check_subspace = false) {
+                          bool check_subspace = false, int parts = 3) {
   (void)fast;
   std::vector<int> act;
   for (size_t i = 0; i < ws.size(); ++i) if (ws[i].active) act.push_back((int)i);
   if (act.empty()) return;
   const int na = (int)act.size();
-  if (mode == FM_RANDOMIZED) {
+  if (mode == FM_RANDOMIZED && (parts & 2)) {
     std::vector<unsigned *> slots;
     for (int i : act) if (ws[i].orthMax) slots.push_back(ws[i].orthMax);
     if (!slots.empty())
@@ -853,7 +862,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
       LAUNCHED();
     });
   }
-  if (mode != FM_INJECTED) {
+  if (mode != FM_INJECTED && (parts & 1)) {
     // mode-3 Gram: per-head partials in fp64, deterministic reduction, Jacobi
     std::vector<GemmTask> g;
     std::vector<const double *> parts; std::vector<double *> outs; std::vector<int> counts;
@@ -871,7 +880,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
         parts.push_back(w.gram_part); outs.push_back(w.C); counts.push_back(c.m);
       }
       EigTask e; memset(&e, 0, sizeof e);
-      e.bjA = w.bjA; e.bjV = w.bjV; e.bjJ = w.bjJ; e.bjOff = w.bjOff; e.bjDone = w.bjDone;
+      e.bjA = w.bjfA; e.bjV = w.bjfV; e.bjJ = w.bjfJ; e.bjOff = w.bjfOff; e.bjDone = w.bjfDone;
       e.A = w.C; e.Vt = w.Cv; e.w = w.Cw; e.n = kD; e.status = w.status; e.w_out = w.lam; e.w_sqrt = 0;
       if (!probe) { e.U_out = w.UF32; e.ld_out = c.r_f; e.r_out = c.r_f; }
       eg.push_back(e);
@@ -895,6 +904,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
       });
     }
   }
+  if (!(parts & 2)) return;
   if (mode == FM_RANDOMIZED) {
     // only the range of the intermediate bases matters (one Cholesky-QR pass keeps them well conditioned);
     // the final basis is orthonormalised twice
@@ -1164,6 +1174,61 @@ static size_t carve_handle_blob(jolt_handle &H) {
   }
   H.stored_bytes = stored;
   return b.off + 256;
+}
+
+// Runs the programs of the cell groups concurrently, one side stream per group, forked from and joined back into the
+// caller's stream; the groups' steps are enqueued round-robin, so every side stream has work from the start.
+static int run_group_programs(int dev, cudaStream_t st, std::vector<Program> &PG, int n_groups, void *d_tab,
+                              const std::vector<size_t> &tab_off) {
+  {
+    GroupStreams *gs = group_streams(dev);
+    if (!gs) return fail(JOLT_ECUDA, "cannot create side streams");
+    cudaError_t ce = cudaEventRecord(gs->fork, st);
+    for (int g = 0; g < n_groups && ce == cudaSuccess; ++g) {
+      ce = cudaStreamWaitEvent(gs->s[g], gs->fork, 0);
+      if (ce == cudaSuccess && !PG[g].host.empty())
+        ce = cudaMemcpyAsync((char *)d_tab + tab_off[g], PG[g].host.data(), PG[g].host.size(), cudaMemcpyHostToDevice, gs->s[g]);
+    }
+    // enqueue the groups' steps round-robin, so every side stream has work from the start
+    size_t max_steps = 0;
+    for (int g = 0; g < n_groups; ++g) max_steps = std::max(max_steps, PG[g].steps.size());
+#ifdef JOLT_DEBUG
+    const bool tl = getenv("JOLT_DEBUG_TIMELINE") != nullptr;      // per-group stage boundaries, printed after the call
+    struct TL { int g, stage; cudaEvent_t ev; };
+    std::vector<TL> tls;
+    cudaEvent_t tl0 = nullptr;
+    if (tl) { cudaEventCreate(&tl0); cudaEventRecord(tl0, st); }
+#endif
+    for (size_t si = 0; si < max_steps && ce == cudaSuccess; ++si)
+      for (int g = 0; g < n_groups; ++g)
+        if (si < PG[g].steps.size()) {
+          PG[g].steps[si].run((char *)d_tab + tab_off[g], gs->s[g]);
+#ifdef JOLT_DEBUG
+          if (tl && (si + 1 == PG[g].steps.size() || PG[g].steps[si + 1].stage != PG[g].steps[si].stage)) {
+            TL t{g, PG[g].steps[si].stage, nullptr}; cudaEventCreate(&t.ev); cudaEventRecord(t.ev, gs->s[g]); tls.push_back(t);
+          }
+#endif
+        }
+#ifdef JOLT_DEBUG
+    if (tl) {
+      cudaDeviceSynchronize();
+      for (int g = 0; g < n_groups; ++g) {
+        fprintf(stderr, "[jolt] group %d:", g);
+        for (auto &t : tls) if (t.g == g) { float ms = 0; cudaEventElapsedTime(&ms, tl0, t.ev); fprintf(stderr, " %s@%.2f", kStageNames[t.stage], ms); }
+        fprintf(stderr, "\n");
+      }
+      for (auto &t : tls) cudaEventDestroy(t.ev);
+      cudaEventDestroy(tl0);
+    }
+#endif
+    if (ce == cudaSuccess) ce = cudaGetLastError();
+    for (int g = 0; g < n_groups && ce == cudaSuccess; ++g) {
+      ce = cudaEventRecord(gs->join[g], gs->s[g]);
+      if (ce == cudaSuccess) ce = cudaStreamWaitEvent(st, gs->join[g], 0);
+    }
+    if (ce != cudaSuccess) { cudaDeviceSynchronize(); return fail(JOLT_ECUDA, "side streams: %s", cudaGetErrorString(ce)); }
+  }
+  return JOLT_OK;
 }
 
 // Device buffer of the projected cores of the cells with a backbone (CellStore::P16 point into it).  A cell whose
@@ -1454,52 +1519,7 @@ static int compress_impl(const jolt_layout *L, const void *K, const void *V, con
   if (n_groups <= 1) {
     if (n_groups == 1 && (rc = run_program(PG[0], (char *)d_tab, st))) { free_blob(); return rc; }
   } else {
-    GroupStreams *gs = group_streams(dev);
-    if (!gs) { free_blob(); return fail(JOLT_ECUDA, "cannot create side streams"); }
-    ce = cudaEventRecord(gs->fork, st);
-    for (int g = 0; g < n_groups && ce == cudaSuccess; ++g) {
-      ce = cudaStreamWaitEvent(gs->s[g], gs->fork, 0);
-      if (ce == cudaSuccess && !PG[g].host.empty())
-        ce = cudaMemcpyAsync((char *)d_tab + tab_off[g], PG[g].host.data(), PG[g].host.size(), cudaMemcpyHostToDevice, gs->s[g]);
-    }
-    // enqueue the groups' steps round-robin, so every side stream has work from the start
-    size_t max_steps = 0;
-    for (int g = 0; g < n_groups; ++g) max_steps = std::max(max_steps, PG[g].steps.size());
-#ifdef JOLT_DEBUG
-    const bool tl = getenv("JOLT_DEBUG_TIMELINE") != nullptr;      // per-group stage boundaries, printed after the call
-    struct TL { int g, stage; cudaEvent_t ev; };
-    std::vector<TL> tls;
-    cudaEvent_t tl0 = nullptr;
-    if (tl) { cudaEventCreate(&tl0); cudaEventRecord(tl0, st); }
-#endif
-    for (size_t si = 0; si < max_steps && ce == cudaSuccess; ++si)
-      for (int g = 0; g < n_groups; ++g)
-        if (si < PG[g].steps.size()) {
-          PG[g].steps[si].run((char *)d_tab + tab_off[g], gs->s[g]);
-#ifdef JOLT_DEBUG
-          if (tl && (si + 1 == PG[g].steps.size() || PG[g].steps[si + 1].stage != PG[g].steps[si].stage)) {
-            TL t{g, PG[g].steps[si].stage, nullptr}; cudaEventCreate(&t.ev); cudaEventRecord(t.ev, gs->s[g]); tls.push_back(t);
-          }
-#endif
-        }
-#ifdef JOLT_DEBUG
-    if (tl) {
-      cudaDeviceSynchronize();
-      for (int g = 0; g < n_groups; ++g) {
-        fprintf(stderr, "[jolt] group %d:", g);
-        for (auto &t : tls) if (t.g == g) { float ms = 0; cudaEventElapsedTime(&ms, tl0, t.ev); fprintf(stderr, " %s@%.2f", kStageNames[t.stage], ms); }
-        fprintf(stderr, "\n");
-      }
-      for (auto &t : tls) cudaEventDestroy(t.ev);
-      cudaEventDestroy(tl0);
-    }
-#endif
-    if (ce == cudaSuccess) ce = cudaGetLastError();
-    for (int g = 0; g < n_groups && ce == cudaSuccess; ++g) {
-      ce = cudaEventRecord(gs->join[g], gs->s[g]);
-      if (ce == cudaSuccess) ce = cudaStreamWaitEvent(st, gs->join[g], 0);
-    }
-    if (ce != cudaSuccess) { cudaDeviceSynchronize(); free_blob(); return fail(JOLT_ECUDA, "side streams: %s", cudaGetErrorString(ce)); }
+    if ((rc = run_group_programs(dev, st, PG, n_groups, d_tab, tab_off))) { free_blob(); return rc; }
     g_timer.mark(ST_FACT, st);
   }
   if ((rc = run_program(P, (char *)d_tab + tab_off.back(), st))) { free_blob(); return rc; }
@@ -2104,12 +2124,32 @@ extern "C" int jolt_allocate(int32_t n_cells, const int32_t *m, int32_t T, int32
   return ok ? JOLT_OK : fail(JOLT_EBUDGET, "cheapest allocation needs %.0f bytes, budget is %.0f", total, budget);
 }
 
-extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, double budget, const jolt_options *o, void *stream,
-                         jolt_cell_plan *out, double *achieved) {
+// The measured spectra of a cache (host memory): what the allocator needs, kept so that the cache can be planned again
+// at another budget or with another allocator without touching the GPU.
+struct jolt_spectra {
+  int32_t nc = 0, T = 0, q_cap = 0;
+  bool exact = false, cap_from_policy = false;
+  double raw = 0;                              // bytes of the uncompressed fp16 cache
+  std::vector<double> lam3, s2all, total;
+  std::vector<int64_t> off;
+  std::vector<int32_t> len, mm, rtmax;
+};
+
+namespace {
+struct PackJob { const float *src; float *dst; int n; };
+__global__ void pack_spectra_kernel(const PackJob *__restrict__ jobs) {
+  const PackJob j = jobs[blockIdx.x];
+  for (int i = threadIdx.x; i < j.n; i += blockDim.x) j.dst[i] = j.src[i];
+}
+}  // namespace
+
+extern "C" int jolt_probe(const jolt_layout *L, const void *K, const void *V, double ratio_hint, const jolt_options *o, void *stream,
+                          jolt_spectra **out) {
+  if (out) *out = nullptr;
   if (!out || !K || !V) return fail(JOLT_EINVAL, "null argument");
   int rc;
   if ((rc = check_layout(L)) || (rc = check_options(o)) || (rc = check_device_alignment(L, K, V))) return rc;
-  if (!(budget > 0)) return fail(JOLT_EINVAL, "byte budget must be positive");
+  if (!(ratio_hint > 0) && o->q_cap <= 0) return fail(JOLT_EINVAL, "the cap needs a compression ratio or opts->q_cap");
   cudaStream_t st = (cudaStream_t)stream;
   int dev = 0;
   CU(cudaGetDevice(&dev));
@@ -2121,7 +2161,7 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
   const bool exact = o->token_mode == JOLT_TOKEN_EXACT && !subspace;
   const int oversample = subspace ? std::max(o->oversample, kSubspaceOversample) : o->oversample;
   const int power_iters = subspace ? std::max(o->power_iters, kSubspaceIters) : o->power_iters;
-  const int q_cap = o->q_cap > 0 ? o->q_cap : cap_policy(L->seq_len, raw / budget);
+  const int q_cap = o->q_cap > 0 ? o->q_cap : cap_policy(L->seq_len, ratio_hint);
   std::vector<jolt_cell_plan> probe(nc);
   std::vector<CellDesc> cells;
   for (int i = 0; i < nc; ++i) {
@@ -2139,7 +2179,9 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
   std::vector<CellWork> ws(nc);
   void *ws_base = nullptr;
   int *d_status = nullptr;
+  float *d_pack = nullptr;
   char *stage_K = nullptr, *stage_V = nullptr;
+  size_t pack_floats = 0;
   for (int pass = 0; pass < 2; ++pass) {
     Bump b;
     b.base = (char *)ws_base;
@@ -2153,6 +2195,8 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
       ws[i].ufI = true;
       carve(b, ws[i], mode, false);
     }
+    if (pass == 0) { pack_floats = 0; for (int i = 0; i < nc; ++i) pack_floats += kD + (size_t)ws[i].n_sigma; }
+    d_pack = b.take<float>(pack_floats);
     if (pass == 0 && (rc = ws_reserve(dev, b.off + 256, &ws_base))) return rc;
   }
   if (L->mem_space == JOLT_MEM_HOST)
@@ -2160,10 +2204,40 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
       const char *hb = (const char *)(i % 2 == 0 ? K : V);
       ws[i].c.X = (i % 2 == 0 ? stage_K : stage_V) + ((const char *)ws[i].c.X - hb);
     }
+  // one program per cell group, run on concurrent streams like the factor stage of jolt_compress; then the spectra of
+  // all cells are gathered into one buffer and leave the device in a single copy
+  std::vector<int> cell_group(nc, -1);
+  int n_groups = assign_groups(ws, cell_group);
+  // the randomized token probe runs on X itself, so the feature spectra (Gram + eigen-solve of all cells) form a
+  // program of their own on one more stream instead of lengthening every group's chain
+  const bool split = mode == FM_RANDOMIZED && n_groups > 1 && n_groups < kMaxGroups;
+  std::vector<Program> PG(std::max(n_groups, 1) + (split ? 1 : 0));
+  for (int g = 0; g < n_groups; ++g) {
+    std::vector<CellWork> sub = ws;
+    for (int i = 0; i < nc; ++i) if (cell_group[i] != g) sub[i].active = false;
+    build_factor_program(PG[g], sub, mode, true, power_iters, o->seed, fast, false, split ? 2 : 3);
+  }
+  if (split) {
+    std::vector<CellWork> sub = ws;
+    build_factor_program(PG[n_groups], sub, mode, true, power_iters, o->seed, fast, false, 1);
+    ++n_groups;
+  }
   Program P;
-  build_factor_program(P, ws, mode, true, power_iters, o->seed, fast);
+  {
+    std::vector<PackJob> pj;
+    size_t at = 0;
+    for (int i = 0; i < nc; ++i) {
+      pj.push_back({ws[i].lam, d_pack + at, kD}); at += kD;
+      pj.push_back({ws[i].sigma, d_pack + at, ws[i].n_sigma}); at += ws[i].n_sigma;
+    }
+    const size_t poff = P.push(pj);
+    const int n = (int)pj.size();
+    P.add(ST_SVD, [=](char *dev_t, cudaStream_t s) { pack_spectra_kernel<<<n, 128, 0, s>>>((const PackJob *)(dev_t + poff)); LAUNCHED(); });
+  }
   void *d_tab = nullptr;
-  if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
+  std::vector<size_t> tab_off(PG.size() + 1, 0);
+  for (size_t g = 0; g < PG.size(); ++g) tab_off[g + 1] = tab_off[g] + ((PG[g].host.size() + 255) & ~(size_t)255);
+  if ((rc = tab_reserve(dev, tab_off.back() + P.host.size() + 256, &d_tab))) return rc;
   if ((rc = arena_acquire(dev, st))) return rc;
   g_timer.begin(st);
   CU(cudaMemsetAsync(d_status, 0, sizeof(int) * 4 * nc, st));
@@ -2171,39 +2245,66 @@ extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, dou
     CU(cudaMemcpyAsync(stage_K, K, span, cudaMemcpyHostToDevice, st));
     CU(cudaMemcpyAsync(stage_V, V, span, cudaMemcpyHostToDevice, st));
   }
-  if ((rc = run_program(P, (char *)d_tab, st))) return rc;
+  if (n_groups <= 1) {
+    if (n_groups == 1 && (rc = run_program(PG[0], (char *)d_tab, st))) return rc;
+  } else if ((rc = run_group_programs(dev, st, PG, n_groups, d_tab, tab_off))) return rc;
+  if ((rc = run_program(P, (char *)d_tab + tab_off.back(), st))) return rc;
   arena_release(dev, st);
   std::vector<int> hstat(4 * nc);
-  std::vector<float> lam((size_t)nc * kD);
-  std::vector<std::vector<float>> sig(nc);
+  std::vector<float> pack(pack_floats);
   CU(cudaMemcpyAsync(hstat.data(), d_status, sizeof(int) * 4 * nc, cudaMemcpyDeviceToHost, st));
-  for (int i = 0; i < nc; ++i) {
-    sig[i].resize(ws[i].n_sigma);
-    CU(cudaMemcpyAsync(lam.data() + (size_t)i * kD, ws[i].lam, sizeof(float) * kD, cudaMemcpyDeviceToHost, st));
-    CU(cudaMemcpyAsync(sig[i].data(), ws[i].sigma, sizeof(float) * ws[i].n_sigma, cudaMemcpyDeviceToHost, st));
-  }
+  CU(cudaMemcpyAsync(pack.data(), d_pack, sizeof(float) * pack_floats, cudaMemcpyDeviceToHost, st));
   CU(cudaStreamSynchronize(st));
   g_timer.finish();
   if ((rc = status_to_code(hstat))) return rc;
   // spectra -> allocator inputs (tail-mass accounting of Sec. 5 for the randomized probe)
-  std::vector<double> lam3((size_t)nc * kD), s2all, total(nc);
-  std::vector<int64_t> off(nc);
-  std::vector<int32_t> len(nc), mm(nc), rtmax(nc);
+  std::unique_ptr<jolt_spectra> S(new jolt_spectra);
+  S->nc = nc; S->T = L->seq_len; S->q_cap = q_cap; S->exact = exact; S->cap_from_policy = o->q_cap <= 0; S->raw = raw;
+  S->lam3.resize((size_t)nc * kD); S->total.resize(nc); S->off.resize(nc); S->len.resize(nc); S->mm.resize(nc); S->rtmax.resize(nc);
+  size_t at = 0;
   for (int i = 0; i < nc; ++i) {
+    const float *lam = pack.data() + at; at += kD;
+    const float *sig = pack.data() + at; at += ws[i].n_sigma;
     double tot = 0;
-    for (int j = 0; j < kD; ++j) { lam3[(size_t)i * kD + j] = lam[(size_t)i * kD + j]; tot += lam[(size_t)i * kD + j]; }
-    total[i] = tot;
-    off[i] = (int64_t)s2all.size();
-    const int keep = exact ? (int)sig[i].size() : std::min((int)sig[i].size(), cells[i].r_t);
+    for (int j = 0; j < kD; ++j) { S->lam3[(size_t)i * kD + j] = lam[j]; tot += lam[j]; }
+    S->total[i] = tot;
+    S->off[i] = (int64_t)S->s2all.size();
+    const int keep = exact ? ws[i].n_sigma : std::min(ws[i].n_sigma, cells[i].r_t);
     double acc = 0;
-    for (int j = 0; j < keep; ++j) { const double v = (double)sig[i][j] * sig[i][j]; s2all.push_back(v); acc += v; }
-    if (!exact) s2all.push_back(std::max(0.0, tot - acc));
-    len[i] = keep + (exact ? 0 : 1);
-    mm[i] = cells[i].m;
-    rtmax[i] = cells[i].r_t;
+    for (int j = 0; j < keep; ++j) { const double v = (double)sig[j] * sig[j]; S->s2all.push_back(v); acc += v; }
+    if (!exact) S->s2all.push_back(std::max(0.0, tot - acc));
+    S->len[i] = keep + (exact ? 0 : 1);
+    S->mm[i] = cells[i].m;
+    S->rtmax[i] = cells[i].r_t;
   }
-  return jolt_allocate(nc, mm.data(), L->seq_len, kD, lam3.data(), s2all.data(), off.data(), len.data(), total.data(),
-                       rtmax.data(), budget, o, out, achieved);
+  *out = S.release();
+  return JOLT_OK;
+}
+
+extern "C" int jolt_plan_from_spectra(const jolt_spectra *S, double budget, const jolt_options *o, jolt_cell_plan *out, double *achieved) {
+  if (!S || !out || !o) return fail(JOLT_EINVAL, "null argument");
+  if (!(budget > 0)) return fail(JOLT_EINVAL, "byte budget must be positive");
+  // the probe stopped at its cap: a budget whose own cap (Sec. 5 "Cap selection") is larger needs a new probe
+  if (S->cap_from_policy && !S->exact && o->q_cap <= 0 && cap_policy(S->T, S->raw / budget) > S->q_cap)
+    return fail(JOLT_EINVAL, "this budget's cap %d exceeds the probed cap %d", cap_policy(S->T, S->raw / budget), S->q_cap);
+  return jolt_allocate(S->nc, S->mm.data(), S->T, kD, S->lam3.data(), S->s2all.data(), S->off.data(), S->len.data(), S->total.data(),
+                       S->rtmax.data(), budget, o, out, achieved);
+}
+
+extern "C" int jolt_spectra_free(jolt_spectra *S) { delete S; return JOLT_OK; }
+
+extern "C" int jolt_plan(const jolt_layout *L, const void *K, const void *V, double budget, const jolt_options *o, void *stream,
+                         jolt_cell_plan *out, double *achieved) {
+  if (!out || !K || !V) return fail(JOLT_EINVAL, "null argument");
+  int rc;
+  if ((rc = check_layout(L)) || (rc = check_options(o))) return rc;
+  if (!(budget > 0)) return fail(JOLT_EINVAL, "byte budget must be positive");
+  const double raw = 2.0 * 2.0 * (double)L->n_layers * L->n_kv_heads * L->seq_len * kD;
+  jolt_spectra *S = nullptr;
+  if ((rc = jolt_probe(L, K, V, raw / budget, o, stream, &S))) return rc;
+  rc = jolt_plan_from_spectra(S, budget, o, out, achieved);
+  delete S;
+  return rc;
 }
 
 // ------------------------------------------------------------------ misc exports

@@ -247,15 +247,18 @@ __global__ void __launch_bounds__(kCholInvThreads, 1) cholinv_kernel(const CholI
     if (i >= j) {
       if (t.A64) v = 0.5 * (t.A64[(size_t)i * n + j] + t.A64[(size_t)j * n + i]);
       else {
-        const size_t idx = (i < 128 || j >= 128) ? (size_t)i * kp + j : (size_t)j * kp + i;
-        const float *p = t.part + idx;
+        // G is symmetric: entry (i, j), i >= j, is read as (row j, column i) of the partials, which is stored for every
+        // such pair (row j < 128 holds all columns; j >= 128 implies i >= 128) and contiguous in i across the threads
+        const float *p = t.part + (size_t)j * kp + i;
         const size_t cs = (size_t)kp * kp;
         int ch = 0;
-        for (; ch + 4 <= t.n_chunks; ch += 4) {
-          const float a = p[(size_t)ch * cs], b = p[(size_t)(ch + 1) * cs], c2 = p[(size_t)(ch + 2) * cs], d = p[(size_t)(ch + 3) * cs];
-          v += ((double)a + (double)b) + ((double)c2 + (double)d);
+        for (; ch + 8 <= t.n_chunks; ch += 8) {
+          float a[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) a[q] = __ldg(p + (size_t)(ch + q) * cs);
+          v += (((double)a[0] + (double)a[1]) + ((double)a[2] + (double)a[3])) + (((double)a[4] + (double)a[5]) + ((double)a[6] + (double)a[7]));
         }
-        for (; ch < t.n_chunks; ++ch) v += (double)p[(size_t)ch * cs];
+        for (; ch < t.n_chunks; ++ch) v += (double)__ldg(p + (size_t)ch * cs);
       }
     }
     W[e] = v;

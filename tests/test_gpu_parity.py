@@ -455,6 +455,42 @@ def test_plan_spectra_and_allocation(B, synth):
     h.free()
 
 
+def test_spectra_are_measured_once_and_planned_at_several_budgets(B, synth):
+    """jolt_probe + jolt_plan_from_spectra: the plan of jolt_plan at the probed budget, and at other budgets the
+    oracle's dual on the oracle's spectra (Sec. 4 Eq. (3)/(4), Sec. 5 tail-mass accounting), with no further GPU work."""
+    cfg = synth.CacheConfig("t", 4, 2, 2, 512, n_terms=48, seed=8)
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2, 4]
+    raw = 2 * K.numel() * 2
+    opts = B.default_options(seed=6, power_iters=1)
+    sp = B.jolt_probe(K, V, gs, 2.0, opts)
+    launches = B.lib.jolt_launch_count()
+    plans2, ach2 = sp.plan(raw / 2.0, opts)
+    assert (plans2, ach2) == B.jolt_plan(K, V, gs, raw / 2.0, opts)
+    launches = B.lib.jolt_launch_count()
+    Knp, Vnp = _np(K), _np(V)
+    q_cap = O.cap_policy(512, 2.0)
+    eps2 = O.eps2_table([0, 2, 4, 8])
+    cells, trips = [], []
+    for c in range(4):
+        X = cell_view(Knp, Vnp, gs, c).astype(np.float64)
+        lam, s2, tot = O.plan_spectra(X, q_cap, seed=6, cell=c, power_iters=1)
+        rt_grid, rf_grid = list(range(16, q_cap + 1, 16)), list(range(16, 129, 16))
+        tau = O.tau_table(lam, s2, tot, rt_grid, rf_grid)
+        e, s, t = O.cell_options(4, 512, 128, tau, rt_grid, rf_grid, [0, 2, 4, 8], eps2)
+        cells.append((e, s)); trips.append(t)
+    for ratio in (1.5, 3.0, 4.0):
+        plans, ach = sp.plan(raw / ratio, opts)
+        assert ach <= raw / ratio
+        ch, cost, lam_star, ok = O.dual_allocate(cells, raw / ratio)
+        e_ref = sum(cells[c][0][ch[c]] for c in range(4))
+        e_got = sum(cells[c][0][trips[c].index(tuple(plans[c]))] for c in range(4))
+        print(f"[parity] replan at {ratio}x: plan {plans}, modelled error {e_got:.6e} vs oracle {e_ref:.6e}")
+        assert abs(e_got - e_ref) <= 1e-3 * e_ref + 1e-9, (ratio, plans)
+    assert B.lib.jolt_launch_count() == launches          # planning from kept spectra launches nothing
+    sp.free()
+
+
 def test_tensor_core_and_portable_paths_agree(B, synth):
     """The tcgen05 kernels and the portable SIMT kernels are two implementations of the same path."""
     cfg = synth.CacheConfig("t", 2, 2, 4, 512, n_terms=32, seed=44)
