@@ -33,6 +33,8 @@ struct BJTask {
   float *U_out; int ld_out, r_out; float *w_out; int w_sqrt;
   int *status;
   double tol;           // convergence: off-diagonal mass <= tol * total mass (squared norms)
+  const float *V0;      // optional starting basis (n x n, row-major, column j = j-th vector): A_in is then V0^T M V0 and
+                        // the eigenvectors come out as V0 J; null: identity
 };
 
 __global__ void bj_init_kernel(const BJTask *__restrict__ tasks) {
@@ -44,7 +46,7 @@ __global__ void bj_init_kernel(const BJTask *__restrict__ tasks) {
     double v = 0;
     if (i < n && j < n) v = 0.5 * (t.A_in[(size_t)i * n + j] + t.A_in[(size_t)j * n + i]);
     t.A[e] = v;
-    t.V[e] = (i == j) ? 1.0 : 0.0;
+    t.V[e] = (t.V0 && i < n && j < n) ? (double)t.V0[(size_t)i * n + j] : ((i == j) ? 1.0 : 0.0);
     tot += v * v;
   }
   for (int o = 16; o; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);

@@ -94,8 +94,14 @@ __device__ __forceinline__ void cj_rotate(float (&a)[NR], float (&b)[NR], float 
     const float ta = __shfl_xor_sync(0xffffffffu, al, o), tb = __shfl_xor_sync(0xffffffffu, be, o), tg = __shfl_xor_sync(0xffffffffu, ga, o);
     al += ta; be += tb; ga += tg;
   }
+  // the angle depends on the ratios of (al, be, ga) only: bring the larger norm into [1/2, 1) by a power of two first, so
+  // that two columns that are both tiny against the rest (the null directions of a rank-deficient factor) do not push
+  // the products below into the denormal range, where the approximate reciprocal square root returns infinity
+  const float big = fmaxf(al, be);
+  const float sc = __uint_as_float(0x7E800000u - (__float_as_uint(big) & 0x7F800000u));
+  al *= sc; be *= sc; ga *= sc;
   const float ab = al * be, g2 = ga * ga;
-  if (!(ab > 1e-36f)) return;                       // a zero (padding or deflated) column
+  if (!(ab > 1e-36f)) return;                       // a zero (padding or deflated) column, or one 1e-36 of the other
   mx2 = fmaxf(mx2, g2 * __frcp_rn(ab));
   if (!(g2 > 1e-14f * ab)) return;                   // already orthogonal to single precision
   const float d = 0.5f * (be - al);

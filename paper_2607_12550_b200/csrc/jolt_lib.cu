@@ -21,6 +21,7 @@
 #include "small_solvers.cuh"
 #include "block_jacobi.cuh"
 #include "cluster_jacobi.cuh"
+#include "eig_presolve.cuh"
 #include "tc_orth.cuh"
 #include "rope.cuh"
 #include "attend.cuh"
@@ -211,19 +212,22 @@ __global__ void __launch_bounds__(128) project_core_kernel(const ProjJob *__rest
   extern __shared__ __half pc_uf[];
   for (int e = f; e < 128 * j.r_f; e += 128) { const int ff = e / j.r_f, s = e - ff * j.r_f; pc_uf[s * 128 + ff] = j.UF[e]; }
   __syncthreads();
-  for (int rb = r0; rb < min(r0 + 32, j.rows); rb += 8) {      // rows are a multiple of 8 (r_t is, or the tail is masked)
-    float acc[8];
+  // fp64 accumulation: products of two fp16 numbers are exact in it and the sum of <= 128 of them is far inside its
+  // precision, so the one rounding to fp16 is the rounding of the exact value (the definition), not of an fp32 sum
+  // that may sit on the other side of a rounding boundary
+  for (int rb = r0; rb < min(r0 + 32, j.rows); rb += 8) {
+    double acc[8];
 #pragma unroll
-    for (int r = 0; r < 8; ++r) acc[r] = 0.f;
+    for (int r = 0; r < 8; ++r) acc[r] = 0.0;
     for (int s = 0; s < j.r_f; ++s) {
-      const float u = __half2float(pc_uf[s * 128 + f]);
+      const double u = (double)__half2float(pc_uf[s * 128 + f]);
 #pragma unroll
       for (int r = 0; r < 8; ++r)
-        if (rb + r < j.rows) acc[r] = fmaf(__half2float(j.G[(size_t)(rb + r) * j.r_f + s]), u, acc[r]);
+        if (rb + r < j.rows) acc[r] = fma((double)__half2float(j.G[(size_t)(rb + r) * j.r_f + s]), u, acc[r]);
     }
 #pragma unroll
     for (int r = 0; r < 8; ++r)
-      if (rb + r < j.rows) j.P[(size_t)(rb + r) * 128 + f] = __float2half_rn(acc[r]);
+      if (rb + r < j.rows) j.P[(size_t)(rb + r) * 128 + f] = __double2half(acc[r]);
   }
 }
 
@@ -384,6 +388,7 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
   std::vector<CholFactorTask> cf;          // Cholesky factor for the cluster solver: work matrix in global memory (n > 152)
   std::vector<tc::CholInvTask> cfs;        // ... in shared memory
   std::vector<CJTask> cj;                  // one launch: rows per lane follow the largest matrix
+  std::vector<PresolveTask> pre;           // block-solver problems that start from a single-precision basis
   for (auto &t : tasks) {
     // singular values of B (w_sqrt): single-precision cluster solver; the mode-3 Gram, whose spectrum spans 1e6 and more
     // when the cache has outlier channels, stays on the fp64 block solver
@@ -399,7 +404,18 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
     }
     if (t.bjA && t.n > 32 && g_eig_smem.load() != 2) {
       BJTask b; memset(&b, 0, sizeof b);
-      b.A_in = t.A; b.A = t.bjA; b.V = t.bjV; b.J = t.bjJ; b.off = t.bjOff; b.done = t.bjDone; b.ticket = (unsigned *)(t.bjDone + 1);
+      const bool presolve = t.preL && !t.w_sqrt && t.n <= tc::kCholInvMaxN && (g_fast.load() & 16);
+      if (presolve) {
+        // A + shift -> Cholesky factor -> single-precision one-sided Jacobi: U; then A' = U^T A U, block solver from V = U
+        pre.push_back({t.A, t.preA, t.preU, t.preT, t.n});
+        cfs.push_back({nullptr, 0, 0, t.preA, t.n, nullptr, nullptr, nullptr, t.preL, nullptr, 0.0});
+        CJTask c; memset(&c, 0, sizeof c);
+        c.L = t.preL; c.n = t.n; c.U_out = t.preU; c.ld_out = t.n; c.r_out = t.n;
+        c.status = nullptr;      // only a starting basis: if this iteration stops short, the block solver sweeps more
+        cj.push_back(c);
+        b.V0 = t.preU;
+      }
+      b.A_in = presolve ? t.preA : t.A; b.A = t.bjA; b.V = t.bjV; b.J = t.bjJ; b.off = t.bjOff; b.done = t.bjDone; b.ticket = (unsigned *)(t.bjDone + 1);
       b.n = t.n; b.nbe = (((t.n + kBJBlock - 1) / kBJBlock) + 1) & ~1; b.nP = b.nbe * kBJBlock;
       b.w = t.w; b.U_out = t.U_out; b.ld_out = t.ld_out; b.r_out = t.r_out; b.w_out = t.w_out; b.w_sqrt = t.w_sqrt; b.status = t.status;
       b.tol = kBJTol;
@@ -411,6 +427,13 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
     else if (eig_smem_bytes(t.n, 4) <= kSmemOptIn - 1024) small32.push_back(t);
     else big.push_back(t);
   }
+  const size_t o_pre = P.push(pre);
+  const int n_pre = (int)pre.size();
+  int pre_n = 0;
+  for (auto &q : pre) pre_n = std::max(pre_n, q.n);
+  if (n_pre) P.add(stage, [=](char *dev, cudaStream_t s) {
+    presolve_shift_kernel<<<n_pre, 256, 0, s>>>((const PresolveTask *)(dev + o_pre)); LAUNCHED();
+  });
   if (!cfs.empty()) {
     const size_t off = P.push(cfs);
     const int n = (int)cfs.size();
@@ -446,7 +469,15 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
       P.add(stage, [=](char *dev, cudaStream_t s) { cj_launch((const CJTask *)(dev + o2), nt, mn, nr, s); LAUNCHED(); });
     }
   }
+  if (n_pre) P.add(stage, [=](char *dev, cudaStream_t s) {
+    const dim3 grid((pre_n + 15) / 16, n_pre);
+    presolve_mul_kernel<false><<<grid, 256, 0, s>>>((const PresolveTask *)(dev + o_pre)); LAUNCHED();
+    presolve_mul_kernel<true><<<grid, 256, 0, s>>>((const PresolveTask *)(dev + o_pre)); LAUNCHED();
+  });
   if (!bj.empty()) {
+    // with a single-precision starting basis for every problem one sweep converges (launches after convergence are
+    // no-ops of a few microseconds); eight are allowed for starting bases that came out poor
+    if (n_pre == (int)bj.size()) bj_sweeps = std::min(bj_sweeps, 8);
     int max_nbe = 0, max_nP = 0;
     for (auto &b : bj) { max_nbe = std::max(max_nbe, b.nbe); max_nP = std::max(max_nP, b.nP); }
     const size_t off = P.push(bj);
@@ -518,6 +549,7 @@ struct CellWork {      // device scratch of one cell
   double *bjA = nullptr, *bjV = nullptr, *bjJ = nullptr, *bjOff = nullptr; int *bjDone = nullptr;
   // eigen-solver scratch of the feature stage: its own, since the probe runs that stage concurrently with the token stage
   double *bjfA = nullptr, *bjfV = nullptr, *bjfJ = nullptr, *bjfOff = nullptr; int *bjfDone = nullptr;
+  double *preL = nullptr, *preT = nullptr, *preA = nullptr; float *preU = nullptr;      // pre-solve of the feature eigenproblem
   double *BBt = nullptr, *BBv = nullptr, *BBw = nullptr;
   float *Ut = nullptr, *sigma = nullptr;
   float *UT32 = nullptr, *G32 = nullptr;
@@ -570,6 +602,8 @@ void carve(Bump &b, CellWork &w, int mode, bool need_backbone_scratch) {
         const size_t nbe = (((kD + kBJBlock - 1) / kBJBlock) + 1) & ~(size_t)1, nP = nbe * kBJBlock;
         w.bjfA = b.take<double>(2 * nP * nP); w.bjfV = b.take<double>(nP * nP); w.bjfJ = b.take<double>(2 * (nbe / 2) * 1024);
         w.bjfOff = b.take<double>(4); w.bjfDone = b.take<int>(4);
+        w.preL = b.take<double>(kD * kD + 8); w.preT = b.take<double>(kD * kD); w.preA = b.take<double>(kD * kD);
+        w.preU = b.take<float>(kD * kD);
       }
       w.gram_part = b.take<double>((size_t)c.m * kD * kD * std::max(1, (tok_segments(c.T) + 1) / 2));
       w.C = b.take<double>(kD * kD); w.Cv = b.take<double>(kD * kD); w.Cw = b.take<double>(kD);
@@ -882,6 +916,7 @@ void build_factor_program(Program &P, std::vector<CellWork> &ws, int mode, bool 
       EigTask e; memset(&e, 0, sizeof e);
       e.bjA = w.bjfA; e.bjV = w.bjfV; e.bjJ = w.bjfJ; e.bjOff = w.bjfOff; e.bjDone = w.bjfDone;
       e.A = w.C; e.Vt = w.Cv; e.w = w.Cw; e.n = kD; e.status = w.status; e.w_out = w.lam; e.w_sqrt = 0;
+      e.preL = w.preL; e.preU = w.preU; e.preT = w.preT; e.preA = w.preA;
       if (!probe) { e.U_out = w.UF32; e.ld_out = c.r_f; e.r_out = c.r_f; }
       eg.push_back(e);
     }

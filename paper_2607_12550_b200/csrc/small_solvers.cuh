@@ -18,6 +18,9 @@ struct EigTask {
   int *status;      // set to 1 if not converged
   // optional scratch of the multi-launch block solver (null: single-CTA kernels)
   double *bjA, *bjV, *bjJ, *bjOff; int *bjDone;
+  // optional scratch of the single-precision pre-solve that gives the block solver its starting basis (null: start
+  // from the identity): preL n*n+8 doubles, preU n*n floats, preT and preA n*n doubles each
+  double *preL; float *preU; double *preT, *preA;
 };
 
 constexpr int kEigThreads = 1024;

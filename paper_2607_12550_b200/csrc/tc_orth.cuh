@@ -241,27 +241,30 @@ __global__ void __launch_bounds__(kCholInvThreads, 1) cholinv_kernel(const CholI
   __shared__ int s_exp, s_dead;
   const int tid = threadIdx.x, nt = blockDim.x, warp = tid >> 5, lane = tid & 31, nw = nt >> 5;
   if (tid == 0) s_dead = 0;
-  for (int e = tid; e < n * n; e += nt) {
-    const int j = e / n, i = e - j * n;      // column j, row i
-    double v = 0.0;
-    if (i >= j) {
-      if (t.A64) v = 0.5 * (t.A64[(size_t)i * n + j] + t.A64[(size_t)j * n + i]);
-      else {
-        // G is symmetric: entry (i, j), i >= j, is read as (row j, column i) of the partials, which is stored for every
-        // such pair (row j < 128 holds all columns; j >= 128 implies i >= 128) and contiguous in i across the threads
-        const float *p = t.part + (size_t)j * kp + i;
-        const size_t cs = (size_t)kp * kp;
-        int ch = 0;
-        for (; ch + 8 <= t.n_chunks; ch += 8) {
-          float a[8];
+  // a warp per column j, lanes over the rows i >= j: both the fp64 input (its upper triangle, (row j, column i): the
+  // matrix is symmetric) and the Gram partials are then read along contiguous addresses
+  for (int j = warp; j < n; j += nw) {
+    for (int i = lane; i < n; i += 32) {
+      double v = 0.0;
+      if (i >= j) {
+        if (t.A64) v = t.A64[(size_t)j * n + i];
+        else {
+          // entry (i, j), i >= j, is read as (row j, column i) of the partials, which is stored for every such pair
+          // (row j < 128 holds all columns; j >= 128 implies i >= 128)
+          const float *p = t.part + (size_t)j * kp + i;
+          const size_t cs = (size_t)kp * kp;
+          int ch = 0;
+          for (; ch + 8 <= t.n_chunks; ch += 8) {
+            float a[8];
 #pragma unroll
-          for (int q = 0; q < 8; ++q) a[q] = __ldg(p + (size_t)(ch + q) * cs);
-          v += (((double)a[0] + (double)a[1]) + ((double)a[2] + (double)a[3])) + (((double)a[4] + (double)a[5]) + ((double)a[6] + (double)a[7]));
+            for (int q = 0; q < 8; ++q) a[q] = __ldg(p + (size_t)(ch + q) * cs);
+            v += (((double)a[0] + (double)a[1]) + ((double)a[2] + (double)a[3])) + (((double)a[4] + (double)a[5]) + ((double)a[6] + (double)a[7]));
+          }
+          for (; ch < t.n_chunks; ++ch) v += (double)__ldg(p + (size_t)ch * cs);
         }
-        for (; ch < t.n_chunks; ++ch) v += (double)__ldg(p + (size_t)ch * cs);
       }
+      W[(size_t)j * n + i] = v;
     }
-    W[e] = v;
   }
   __syncthreads();
   for (int i = tid; i < n; i += nt) diag0[i] = W[(size_t)i * n + i];
@@ -391,10 +394,8 @@ __global__ void __launch_bounds__(kCholInvThreads, 1) cholinv_kernel(const CholI
   }
   if (tid == 0 && s_dead && t.status) atomicOr(t.status, 2);
   if (t.L64) {
-    for (int e = tid; e < n * n; e += nt) {
-      const int j = e / n, i = e - j * n;
-      t.L64[e] = i >= j ? W[e] : 0.0;
-    }
+    for (int j = warp; j < n; j += nw)
+      for (int i = lane; i < n; i += 32) t.L64[(size_t)j * n + i] = i >= j ? W[(size_t)j * n + i] : 0.0;
     if (tid == 0) {      // max |L_ij|^2 <= max G_ii: exponent for the single-precision Jacobi iteration
       double mxd = 0.0;
       for (int i = 0; i < n; ++i) mxd = fmax(mxd, diag0[i]);
@@ -406,10 +407,9 @@ __global__ void __launch_bounds__(kCholInvThreads, 1) cholinv_kernel(const CholI
   if (!t.Lhi) return;
   // ---- L^-1: (L^-1)_ic = X[c][i] for c < i, diagonal invd.  Scaled so that the largest entry lies in [2^9, 2^10).
   float mx = 0.f;
-  for (int e = tid; e < n * n; e += nt) {
-    const int i = e / n, cidx = e - i * n;       // column i of W, row cidx
-    if (cidx < i) mx = fmaxf(mx, fabsf((float)W[e]));
-    else if (cidx == i) mx = fmaxf(mx, (float)invd[i]);
+  for (int i = warp; i < n; i += nw) {           // column i of W, rows cidx < i hold row i of L^-1
+    for (int cidx = lane; cidx < i; cidx += 32) mx = fmaxf(mx, fabsf((float)W[(size_t)i * n + cidx]));
+    if (lane == 0) mx = fmaxf(mx, (float)invd[i]);
   }
   for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
   if (lane == 0) s_red[warp] = mx;
@@ -423,15 +423,22 @@ __global__ void __launch_bounds__(kCholInvThreads, 1) cholinv_kernel(const CholI
   }
   __syncthreads();
   const double sc = ldexp(1.0, s_exp);
-  for (int e = tid; e < kp * kp; e += nt) {
-    const int i = e / kp, cidx = e - i * kp;     // row i (output column of Q), column cidx (contraction index)
-    double v = 0.0;
-    if (i < n && cidx < i) v = W[(size_t)i * n + cidx];
-    else if (i < n && cidx == i) v = invd[i];
-    const float f = (float)(v * sc);
-    const __half h = __float2half_rn(f);
-    t.Lhi[e] = h;
-    t.Llo[e] = __float2half_rn(f - __half2float(h));
+  for (int i = warp; i < kp; i += nw) {          // row i (output column of Q), a pair of columns cidx (contraction index) per lane
+    for (int c2 = 2 * lane; c2 < kp; c2 += 64) {
+      float f[2];
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int cidx = c2 + u;
+        double v = 0.0;
+        if (i < n && cidx < i) v = W[(size_t)i * n + cidx];
+        else if (i < n && cidx == i) v = invd[i];
+        f[u] = (float)(v * sc);
+      }
+      const __half2 h = __floats2half2_rn(f[0], f[1]);
+      const float2 hf = __half22float2(h);
+      *(__half2 *)(t.Lhi + (size_t)i * kp + c2) = h;
+      *(__half2 *)(t.Llo + (size_t)i * kp + c2) = __floats2half2_rn(f[0] - hf.x, f[1] - hf.y);
+    }
   }
 }
 
