@@ -424,16 +424,17 @@ def main():
     t_dec = stages.get("decode_rows", td)
     dec_bound = "hbm" if bd / (pk["hbm"] * 1e9) >= fd / (pk["tensor"] * 1e12) else "tensor"
     # DRAM traffic of one launch: ncu capture of a few cells (profiles/dram_traffic.txt), scaled by the cells of this run
-    tr = dram_traffic("tc::decode_kernel", cfg.name)
+    dec_kernel = "tc::decode_kernel" if args.rope else "tc::decode_persistent_kernel"
+    tr = dram_traffic(dec_kernel, cfg.name)
     traffic = (tr["read"] + tr["write"]) * (2 * ng) / tr["cells"] if tr else None
     if dec_bound == "hbm":
         ach = bd / (t_dec * 1e-3) / 1e9
-        roofline = {"kernel": "tc::decode_kernel", "bound": "hbm", "achieved": ach, "peak": pk["hbm"], "unit": "GB/s",
+        roofline = {"kernel": dec_kernel, "bound": "hbm", "achieved": ach, "peak": pk["hbm"], "unit": "GB/s",
                     "frac": ach / pk["hbm"], "traffic": traffic, "algorithmic_bytes": bd, "kernel_ms": t_dec,
                     "peak_source": pk["source"] + " (MEASURED_PEAKS.json hbm_gbs)"}
     else:
         ach = fd / (t_dec * 1e-3) / 1e12
-        roofline = {"kernel": "tc::decode_kernel", "bound": "tensor", "achieved": ach, "peak": pk["tensor"], "unit": "TFLOP/s",
+        roofline = {"kernel": dec_kernel, "bound": "tensor", "achieved": ach, "peak": pk["tensor"], "unit": "TFLOP/s",
                     "frac": ach / pk["tensor"], "traffic": traffic, "algorithmic_flops": fd, "kernel_ms": t_dec,
                     "peak_source": pk["source"] + " (MEASURED_PEAKS.json bf16_tflops, burst)"}
 

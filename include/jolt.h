@@ -285,7 +285,10 @@ int64_t jolt_launch_count(void);
  * bit 4 = eigen-solver resident in a thread-block cluster (otherwise one launch per Jacobi round),
  * bit 5 = CholeskyQR of the range finder on tensor cores (otherwise fp64 SIMT Gram and row-wise triangular solve),
  * bit 6 = factor sweeps with two output tiles per CTA (otherwise one);
- * 127 (default) = all, where the shapes allow.  Returns the previous mask. */
+ * bit 7 = persistent decode kernel (one CTA per SM walks a share of all tiles; otherwise one CTA per 16-tile item;
+ *         launches with a cell of r_t > 128, with keys rotated at decode or with cells of different sequence
+ *         lengths always take the per-item kernel);
+ * 255 (default) = all, where the shapes allow.  Returns the previous mask. */
 int jolt_set_fast_path(int enabled);
 
 /* Number of cell groups whose factor stages jolt_compress runs side by side on internal streams (1..8, default 4):

@@ -370,11 +370,12 @@ def launch_count() -> int:
 
 
 def set_fast_path(enabled) -> int:
-    """False / 0: portable kernels only; True / 127: every sm_100a kernel; other ints: bit mask
+    """False / 0: portable kernels only; True / 255: every sm_100a kernel; other ints: bit mask
     (1 = fused backbone kernels, 2 = factor sweeps, 4 = Gram, 8 = rotary embedding inside the decode kernel,
-    16 = cluster-resident eigen-solver, 32 = CholeskyQR on tensor cores, 64 = two output tiles per CTA in the factor sweeps).  Returns the previous mask."""
+    16 = cluster-resident eigen-solver, 32 = CholeskyQR on tensor cores, 64 = two output tiles per CTA in the factor sweeps,
+    128 = persistent decode kernel).  Returns the previous mask."""
     if enabled is True:
-        enabled = 127
+        enabled = 255
     return lib.jolt_set_fast_path(int(enabled))
 
 

@@ -4,6 +4,7 @@
 #pragma once
 #include "tc_backbone.cuh"
 #include "tc_decode.cuh"
+#include "tc_decode_p.cuh"
 #include "tc_gemm.cuh"
 #include "tc_orth.cuh"
 
@@ -62,20 +63,51 @@ inline void add_backbone_tc(Program &P, int stage, const std::vector<tc::BBCell>
   });
 }
 
-inline void add_decode_tc(Program &P, int stage, const std::vector<tc::BBCell> &cells, uint64_t seed) {
+inline void add_decode_tc(Program &P, int stage, std::vector<tc::BBCell> cells, uint64_t seed) {
   if (cells.empty()) return;
   using LY = tc::DecLayout;
   static bool attr_done = false;
+  static int n_sm = 0;
   if (!attr_done) {
     cudaFuncSetAttribute(tc::decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
+    cudaFuncSetAttribute(tc::decode_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
     attr_done = true;
   }
+  // persistent form: every cell with r_t <= 128, the same sequence length and no rotation of keys at decode
+  bool persistent = (g_fast.load() & 128) != 0 && n_sm > 0;
+  long long total = 0;
+  for (auto &c : cells) {
+    if (c.r_t > 128 || c.T != cells[0].T) persistent = false;
+    if (c.rope) persistent = false;
+    c.tile_base = (int)total;
+    total += (long long)c.m * (c.T / 128);
+  }
+  if (total >= (1ll << 30)) persistent = false;
   int gx = 0;
   for (auto &c : cells) gx = std::max(gx, c.m * c.items_per_head);
+  const int nt = cells[0].T / 128, tot = (int)total;
   const size_t off = P.push(cells);
   const int n = (int)cells.size();
+  const int grid_p = (int)std::min<long long>(n_sm, total);
+  // The persistent kernel takes a fixed contiguous share per CTA and can hand a tail of the list out in chunks through
+  // a counter (zero at every launch: it travels in the argument table).  The tail is empty here: measured on the
+  // benchmark mix, a 5 % tail in 8-tile chunks made the launch slower (0.199 against 0.192 ms), because every chunk
+  // reloads its head's projected core into the single P buffer and restarts the unpack -> rotation pipeline.
+  const size_t off_cnt = P.push(std::vector<int>(4, 0));
+  std::vector<int2> run0(std::max(grid_p, 1), make_int2(tot, tot));
+  for (int i = 0; i < grid_p; ++i) run0[i] = make_int2((int)((long long)tot * i / grid_p), (int)((long long)tot * (i + 1) / grid_p));
+  const int pool = tot, chunk = 8;
+  const size_t off_run0 = P.push(run0);
   P.add(stage, [=](char *dev_t, cudaStream_t s) {
-    tc::decode_kernel<<<dim3(gx, n), LY::THREADS, LY::SMEM_BYTES, s>>>((const tc::BBCell *)(dev_t + off), seed);
+    if (persistent) {
+      tc::DecPArgs a{(const tc::BBCell *)(dev_t + off), n, nt, tot, seed, (const int2 *)(dev_t + off_run0), pool, chunk, (int *)(dev_t + off_cnt)};
+      tc::decode_persistent_kernel<<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
+    } else {
+      tc::decode_kernel<<<dim3(gx, n), LY::THREADS, LY::SMEM_BYTES, s>>>((const tc::BBCell *)(dev_t + off), seed);
+    }
     LAUNCHED();
   });
 }

@@ -40,6 +40,7 @@ struct alignas(64) BBCell {
   int out_dtype;
   int m, n_heads, T, r_t, r_f, bits, cell;
   int tiles_per_item, items_per_head;
+  int tile_base;        // persistent decode: first tile of this cell in the launch's linear (cell, head, tile) order
   int *status;
   const float2 *rope;   // DECODE of key cells: (cos, sin) of feature pair j at token t in rope[j * T + t]; null = no rotation
 };

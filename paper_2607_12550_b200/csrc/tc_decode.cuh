@@ -160,14 +160,39 @@ struct DecCodes {
   alignas(8) __half sc[8];                     // coop: the scales those chunks need; else sc[0..3] = the row's scales
 };
 
+// Read-only global loads that stay where they are written: the codes of the NEXT tile are requested a whole tile
+// ahead of their use, and a plain load may be moved by the compiler down to its first use (it did, where registers
+// were short: the unpack then waited a full memory round trip per tile).  A volatile asm keeps its place among the
+// other volatile statements (barrier arrivals and waits).
+__device__ __forceinline__ uint4 dec_ldg_v4(const void *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint2 dec_ldg_v2(const void *p) {
+  uint2 v;
+  asm volatile("ld.global.nc.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint32_t dec_ldg_u32(const void *p) {
+  uint32_t v;
+  asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ __half dec_ldg_h(const void *p) {
+  unsigned short v;
+  asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
+  return __ushort_as_half(v);
+}
+
 template <int BITS>
 __device__ __forceinline__ void dec_load_codes(const BBCell &c, long long row, DecCodes<BITS> &d) {
   if constexpr (BITS == 0) return;
   else if constexpr (!DecCodes<BITS>::kCoop) {
     const uint4 *wp = (const uint4 *)(c.words + row * (4 * BITS));
 #pragma unroll
-    for (int i = 0; i < BITS; ++i) { const uint4 v = __ldg(wp + i); d.words[4 * i] = v.x; d.words[4 * i + 1] = v.y; d.words[4 * i + 2] = v.z; d.words[4 * i + 3] = v.w; }
-    *(uint2 *)d.sc = __ldg((const uint2 *)(c.scales + row * 4));
+    for (int i = 0; i < BITS; ++i) { const uint4 v = dec_ldg_v4(wp + i); d.words[4 * i] = v.x; d.words[4 * i + 1] = v.y; d.words[4 * i + 2] = v.z; d.words[4 * i + 3] = v.w; }
+    *(uint2 *)d.sc = dec_ldg_v2(c.scales + row * 4);
   } else {
     constexpr int RPI = 32 / BITS;                            // rows per load instruction
     const int lane = threadIdx.x & 31;
@@ -177,13 +202,13 @@ __device__ __forceinline__ void dec_load_codes(const BBCell &c, long long row, D
 #pragma unroll
     for (int it = 0; it < BITS; ++it) {
       const long long r = wrow + it * RPI + rsub;
-      const uint4 v = __ldg((const uint4 *)(c.words + r * (4 * BITS)) + chunk);
+      const uint4 v = dec_ldg_v4((const uint4 *)(c.words + r * (4 * BITS)) + chunk);
       d.words[4 * it] = v.x; d.words[4 * it + 1] = v.y; d.words[4 * it + 2] = v.z; d.words[4 * it + 3] = v.w;
       const __half *sp = c.scales + r * 4;
-      if constexpr (BITS == 8) d.sc[it] = __ldg(sp + (chunk >> 1));
-      else if constexpr (BITS == 4) d.sc[it] = __ldg(sp + chunk);
-      else if constexpr (BITS == 2) *(uint32_t *)&d.sc[2 * it] = __ldg((const uint32_t *)(sp + 2 * chunk));
-      else *(uint2 *)&d.sc[0] = __ldg((const uint2 *)sp);
+      if constexpr (BITS == 8) d.sc[it] = dec_ldg_h(sp + (chunk >> 1));
+      else if constexpr (BITS == 4) d.sc[it] = dec_ldg_h(sp + chunk);
+      else if constexpr (BITS == 2) *(uint32_t *)&d.sc[2 * it] = dec_ldg_u32(sp + 2 * chunk);
+      else *(uint2 *)&d.sc[0] = dec_ldg_v2(sp);
     }
   }
 }
