@@ -311,6 +311,12 @@ int jolt_check_status(const jolt_handle *h, void *stream);
  * defaults.  Applies to the current device. */
 int jolt_test_set_wait_limit(int64_t cycles, int32_t skip_first_load);
 
+/* Test hook for the persistent decode kernel.  Its CTAs take fixed shares of the launch's tile list; the kernel can
+ * also hand the last `percent` % of the list out in chunks of `chunk_tiles` tiles to whichever CTA asks first.  The
+ * library leaves that tail empty (it measured slower); this switch turns it on so that tests cover the path.
+ * percent in [0, 100], chunk_tiles >= 1; (0, anything) restores the default.  Returns JOLT_EINVAL otherwise. */
+int jolt_test_set_decode_tail(int32_t percent, int32_t chunk_tiles);
+
 /* Wall-clock-free per-stage device timing of the last compress / decompress on this thread
  * (milliseconds, CUDA events): out[0..n) in stage order, names via jolt_stage_name. */
 int jolt_last_stage_ms(float *out, int32_t cap, int32_t *n);

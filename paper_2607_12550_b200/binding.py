@@ -90,6 +90,7 @@ lib.jolt_set_fast_path.argtypes = [C.c_int]
 lib.jolt_set_stream_groups.argtypes = [C.c_int]
 lib.jolt_check_status.argtypes = [_vp, _vp]
 lib.jolt_test_set_wait_limit.argtypes = [C.c_int64, C.c_int32]
+lib.jolt_test_set_decode_tail.argtypes = [C.c_int32, C.c_int32]
 lib.jolt_last_stage_ms.argtypes = [C.POINTER(C.c_float), C.c_int32, C.POINTER(C.c_int32)]
 lib.jolt_stage_name.argtypes = [C.c_int32]
 lib.jolt_stage_name.restype = C.c_char_p
@@ -392,6 +393,11 @@ def check_status(handle: "Handle", stream=None):
 def set_test_wait_limit(cycles: int = 0, skip_first_load: bool = False):
     """Test hook of the bounded device-side waits; see include/jolt.h."""
     _check(lib.jolt_test_set_wait_limit(int(cycles), 1 if skip_first_load else 0))
+
+
+def set_test_decode_tail(percent: int = 0, chunk_tiles: int = 8):
+    """Test hook: chunked tail of the persistent decode kernel's tile list; see include/jolt.h."""
+    _check(lib.jolt_test_set_decode_tail(int(percent), int(chunk_tiles)))
 
 
 def release_workspace():

@@ -93,13 +93,13 @@ inline void add_decode_tc(Program &P, int stage, std::vector<tc::BBCell> cells, 
   const int n = (int)cells.size();
   const int grid_p = (int)std::min<long long>(n_sm, total);
   // The persistent kernel takes a fixed contiguous share per CTA and can hand a tail of the list out in chunks through
-  // a counter (zero at every launch: it travels in the argument table).  The tail is empty here: measured on the
+  // a counter (zero at every launch: it travels in the argument table).  The tail is empty unless a test asks for one: measured on the
   // benchmark mix, a 5 % tail in 8-tile chunks made the launch slower (0.199 against 0.192 ms), because every chunk
   // reloads its head's projected core into the single P buffer and restarts the unpack -> rotation pipeline.
   const size_t off_cnt = P.push(std::vector<int>(4, 0));
   std::vector<int2> run0(std::max(grid_p, 1), make_int2(tot, tot));
-  for (int i = 0; i < grid_p; ++i) run0[i] = make_int2((int)((long long)tot * i / grid_p), (int)((long long)tot * (i + 1) / grid_p));
-  const int pool = tot, chunk = 8;
+  const int pool = (int)((long long)tot * (100 - g_dec_tail_pct.load()) / 100), chunk = std::max(1, g_dec_tail_chunk.load());
+  for (int i = 0; i < grid_p; ++i) run0[i] = make_int2((int)((long long)pool * i / grid_p), (int)((long long)pool * (i + 1) / grid_p));
   const size_t off_run0 = P.push(run0);
   P.add(stage, [=](char *dev_t, cudaStream_t s) {
     if (persistent) {

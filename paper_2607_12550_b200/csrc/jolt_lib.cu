@@ -36,6 +36,7 @@ std::atomic<int> g_eig_smem{1};
 long long *g_dbg_stamps = nullptr;   // device buffer for kernel cycle stamps (profiling aid)
 #endif
 std::atomic<int> g_n_cell_groups{4};        // concurrent cell groups of jolt_compress (jolt_set_stream_groups)
+std::atomic<int> g_dec_tail_pct{0}, g_dec_tail_chunk{8};   // test switch: chunked tail of the persistent decode (off)
 std::atomic<int> g_fast{255};  // bit 0: fused backbone kernels, bit 1: factor sweeps, bit 2: Gram on tensor cores,
                               // bit 3: rotary embedding inside the decode kernel, bit 4: cluster-resident eigen-solver,
                               // bit 5: CholeskyQR on tensor cores, bit 6: two output tiles per CTA in the factor sweeps,
@@ -2388,6 +2389,12 @@ extern "C" int jolt_test_set_wait_limit(int64_t cycles, int32_t skip_first_load)
   const int skip = skip_first_load ? 1 : 0;
   CU(cudaMemcpyToSymbol(tc::g_spin_limit, &lim, sizeof lim));
   CU(cudaMemcpyToSymbol(tc::g_test_skip_first_load, &skip, sizeof skip));
+  return JOLT_OK;
+}
+extern "C" int jolt_test_set_decode_tail(int32_t percent, int32_t chunk_tiles) {
+  if (percent < 0 || percent > 100 || (percent > 0 && chunk_tiles < 1)) return fail(JOLT_EINVAL, "decode tail %d %% in chunks of %d", percent, chunk_tiles);
+  g_dec_tail_pct.store(percent);
+  g_dec_tail_chunk.store(percent > 0 ? chunk_tiles : 8);
   return JOLT_OK;
 }
 extern "C" int jolt_set_stream_groups(int n) { return g_n_cell_groups.exchange(std::max(1, std::min(8, n))); }

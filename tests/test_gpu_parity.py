@@ -516,6 +516,51 @@ def test_tensor_core_and_portable_paths_agree(B, synth):
         assert np.allclose(outs[False][2][i][:32], outs[True][2][i][:32], rtol=1e-4)
 
 
+@pytest.mark.parametrize("case", ["mixed", "many_cells", "one_tile_heads"])
+def test_persistent_and_per_item_decode_kernels_agree_bit_for_bit(B, synth, case):
+    """The persistent decode kernel (one CTA per SM over a share of all tiles) and the per-item kernel compute every
+    output element with the same operations in the same order: their outputs are identical, in fp16 and in fp32, with
+    dense and with padded strides.  (The default path is checked against the oracle by the tests above.)"""
+    if case == "mixed":          # five tiles per head: warpgroups change parity from head to head; all bit widths
+        cfg = synth.CacheConfig("t", 6, 2, 4, 640, n_terms=24, seed=12)
+        gs = [0, 2, 4, 6]
+        plans = [(48, 128, 4), (40, 128, 8), (32, 96, 0), (56, 112, 3), (128, 128, 1), (16, 64, 2)]
+    elif case == "many_cells":   # 160 one-tile cells on 148 SMs: some CTAs' shares span two cells
+        cfg = synth.CacheConfig("t", 80, 1, 1, 128, n_terms=8, seed=13)
+        gs = list(range(81))
+        plans = [((16, 128, 4), (24, 128, 8), (8, 64, 2), (0, 0, 4))[c % 4] for c in range(160)]
+    else:                        # T = 128: every tile is a head of its own (a new projected core per tile)
+        cfg = synth.CacheConfig("t", 24, 8, 8, 128, n_terms=8, seed=14)
+        gs = [0, 8, 16, 24]
+        plans = [(32, 128, 4), (16, 96, 8)] * 3
+    K, V = synth.make_cache(cfg, device="cuda")
+    h = B.jolt_compress(K, V, gs, plans, B.default_options(seed=5, power_iters=1))
+    L, nh, T, d = K.shape
+    outs = {}
+    for mask in (255, 127, "tail"):     # "tail": the persistent kernel with 40 % of the tiles handed out in chunks of 3
+        prev = B.set_fast_path(255 if mask == "tail" else mask)
+        if mask == "tail":
+            B.set_test_decode_tail(40, 3)
+        try:
+            res = []
+            for dtype, pad in ((torch.float16, 0), (torch.float32, 0), (torch.float16, 32)):
+                Ko = torch.full((L, nh, T, d + pad), 7.0, dtype=dtype, device="cuda")[..., :d]
+                Vo = torch.full((L, nh, T, d + pad), 7.0, dtype=dtype, device="cuda")[..., :d]
+                B.jolt_decompress(h, Ko, Vo, gs)
+                B.check_status(h)
+                torch.cuda.synchronize()
+                res.append((Ko.clone(), Vo.clone()))
+            outs[mask] = res
+        finally:
+            B.set_fast_path(prev)
+            B.set_test_decode_tail(0)
+    for other in (127, "tail"):
+        for (Ka, Va), (Kb, Vb) in zip(outs[255], outs[other]):
+            assert torch.equal(Ka, Kb) and torch.equal(Va, Vb), (case, other)
+    assert torch.isfinite(outs[255][0][0].float()).all()
+    h.free()
+
+
 def test_degenerate_inputs(B):
     """All-zero cache, a constant cache and the largest legal token rank."""
     gs = [0, 1]
