@@ -1606,6 +1606,13 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
   int dev = 0;
   CU(cudaGetDevice(&dev));
   if (dev != H->device) return fail(JOLT_EINVAL, "handle belongs to device %d, current device is %d", H->device, dev);
+#ifdef JOLT_DEBUG
+  const bool dbg_t = getenv("JOLT_DEBUG_TIMING") != nullptr;
+  auto t_start = std::chrono::steady_clock::now();
+  auto lap = [&](const char *what) { if (dbg_t) { auto n = std::chrono::steady_clock::now(); fprintf(stderr, "[jolt] decode %s: %.1f us\n", what, std::chrono::duration<double, std::micro>(n - t_start).count()); t_start = n; } };
+#else
+  auto lap = [](const char *) {};
+#endif
   const int nc = (int)H->cells.size();
   const size_t esz = L->dtype == JOLT_F16 ? 2 : 4;
   const size_t span = layout_span_elems(L) * esz;
@@ -1640,6 +1647,7 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
   }
   char *Kd = L->mem_space == JOLT_MEM_HOST ? stage_K : (char *)Kout;
   char *Vd = L->mem_space == JOLT_MEM_HOST ? stage_V : (char *)Vout;
+  lap("workspace");
   Program P;
   std::vector<BackboneRef> br;
   std::vector<RowJob> rj;
@@ -1685,6 +1693,7 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
     rows += (long long)c.m * c.T;
     rj.push_back(j);
   }
+  lap("descriptors");
   // the costliest cells (most residual bits, then largest r_t) first: the last wave of CTAs is then the cheapest one
   std::stable_sort(bbc.begin(), bbc.end(), [](const tc::BBCell &x, const tc::BBCell &y) {
     return x.bits != y.bits ? x.bits > y.bits : x.r_t > y.r_t;
@@ -1729,13 +1738,16 @@ static int decompress_impl(const jolt_handle *H, const jolt_layout *L, void *Kou
       LAUNCHED();
     });
   }
+  lap("program");
   void *d_tab = nullptr;
   if ((rc = tab_reserve(dev, P.host.size() + 256, &d_tab))) return rc;
   if ((rc = arena_acquire(dev, st))) return rc;
   H->last_stream = st;
   g_timer.begin(st);
   CU(cudaMemsetAsync(d_status, 0, sizeof(int) * 4 * nc, st));
+  lap("acquire+memset");
   if ((rc = run_program(P, (char *)d_tab, st))) return rc;
+  lap("upload+launch");
   if (L->mem_space == JOLT_MEM_HOST) {
     std::vector<int> hstat(4 * (size_t)nc);
     CU(cudaMemcpyAsync(Kout, stage_K, span, cudaMemcpyDeviceToHost, st));
