@@ -70,18 +70,23 @@ inline void add_decode_tc(Program &P, int stage, std::vector<tc::BBCell> cells, 
   static int n_sm = 0;
   if (!attr_done) {
     cudaFuncSetAttribute(tc::decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
-    cudaFuncSetAttribute(tc::decode_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
+    cudaFuncSetAttribute(tc::decode_persistent_kernel<false, 0x11Fu>, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
+    cudaFuncSetAttribute(tc::decode_persistent_kernel<true, 0x11Fu>, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
+    cudaFuncSetAttribute(tc::decode_persistent_kernel<true, 0x110u>, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
     attr_done = true;
   }
   // persistent form: every cell with r_t <= 128, the same sequence length and no rotation of keys at decode
-  bool persistent = (g_fast.load() & 128) != 0 && n_sm > 0;
+  bool persistent = (g_fast.load() & 128) != 0 && n_sm > 0, tma_only = true;
+  unsigned bitmask = 0;
   long long total = 0;
   for (auto &c : cells) {
     if (c.r_t > 128 || c.T != cells[0].T) persistent = false;
     if (c.rope) persistent = false;
+    if (!(c.tma_out != 0 && c.out_dtype == DT_F16)) tma_only = false;
+    bitmask |= 1u << c.bits;
     c.tile_base = (int)total;
     total += (long long)c.m * (c.T / 128);
   }
@@ -104,7 +109,9 @@ inline void add_decode_tc(Program &P, int stage, std::vector<tc::BBCell> cells, 
   P.add(stage, [=](char *dev_t, cudaStream_t s) {
     if (persistent) {
       tc::DecPArgs a{(const tc::BBCell *)(dev_t + off), n, nt, tot, seed, (const int2 *)(dev_t + off_run0), pool, chunk, (int *)(dev_t + off_cnt)};
-      tc::decode_persistent_kernel<<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
+      if (tma_only && (bitmask & ~0x110u) == 0) tc::decode_persistent_kernel<true, 0x110u><<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
+      else if (tma_only) tc::decode_persistent_kernel<true, 0x11Fu><<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
+      else tc::decode_persistent_kernel<false, 0x11Fu><<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
     } else {
       tc::decode_kernel<<<dim3(gx, n), LY::THREADS, LY::SMEM_BYTES, s>>>((const tc::BBCell *)(dev_t + off), seed);
     }

@@ -87,14 +87,14 @@ __device__ __forceinline__ void tma_prefetch_l2_2d(const void *tmap, int c0, int
 // scale, round to fp16, stage the warp's 32 rows and hand them to one bulk tensor store per half.  `pending` says
 // whether a bulk store of this warp may still be reading its staging rows.
 // returns bit 0: no wait ran out, bit 1: a bulk store of this warp is still pending
-template <int BITS>
+template <int BITS, bool TMA_ONLY>
 __device__ __forceinline__ int dec_tile_loop_p(const BBCell &c, const DecPCtx &x, int p0, int p_end, bool pending) {
   DecCodes<BITS> cur;
   bool ok = true;
   const DecScales sc = dec_scales(x.ex);
   const int lane = x.rit & 31, wrow0 = x.rit & ~31;
-  const bool f16 = c.out_dtype == DT_F16;
-  const bool tma_out = c.tma_out != 0 && f16;
+  const bool f16 = TMA_ONLY || c.out_dtype == DT_F16;
+  const bool tma_out = TMA_ONLY || (c.tma_out != 0 && f16);
   unsigned char *rowp = x.stg + lane * 128;
   // (head, tile in head) of the tile being finished and of the next tile whose codes are to be requested
   int h = (p0 - x.base) / x.nt, tt = (p0 - x.base) - h * x.nt;
@@ -228,6 +228,11 @@ struct DecRunQ {
   }
 };
 
+// TMA_ONLY: every cell of the launch writes fp16 through bulk tensor stores (the common case gets a tile loop without
+// the fp32 and read-back paths)
+// BITMASK: bit b set = the tile loop for b-bit cells is compiled in (a launch takes the smallest instantiated superset
+// of its cells' bit widths: fewer tile loops, a smaller instruction footprint)
+template <bool TMA_ONLY, unsigned BITMASK>
 __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_persistent_kernel(const DecPArgs a) {
   using LY = DecLayout;
   constexpr int NWG = DEC_NWG, NS = LY::NS;
@@ -489,15 +494,14 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_persistent_kerne
           x.s_stg = sStg + (uint32_t)(wg * 16384 + qd * 4096); x.stg = smStg + wg * 16384 + qd * 4096;
           x.abort_flag = abort_flag; x.wg = wg; x.rit = rit; x.nt = nt; x.base = c.tile_base; x.joff = j - p;
           const int p0 = p + (((j & 1) == wg) ? 0 : 1);      // this warpgroup's first tile of the piece
-          int rcode;
-          switch (c.bits) {
-            case 0: rcode = dec_tile_loop_p<0>(c, x, p0, cell_end, pending); break;
-            case 1: rcode = dec_tile_loop_p<1>(c, x, p0, cell_end, pending); break;
-            case 2: rcode = dec_tile_loop_p<2>(c, x, p0, cell_end, pending); break;
-            case 3: rcode = dec_tile_loop_p<3>(c, x, p0, cell_end, pending); break;
-            case 4: rcode = dec_tile_loop_p<4>(c, x, p0, cell_end, pending); break;
-            default: rcode = dec_tile_loop_p<8>(c, x, p0, cell_end, pending); break;
-          }
+          int rcode = pending ? 2 : 0;      // a bit width that is not compiled in: reported as a failed launch
+          const int bits = c.bits;
+          if ((BITMASK & 1u) && bits == 0) rcode = dec_tile_loop_p<0, TMA_ONLY>(c, x, p0, cell_end, pending);
+          if ((BITMASK & 2u) && bits == 1) rcode = dec_tile_loop_p<1, TMA_ONLY>(c, x, p0, cell_end, pending);
+          if ((BITMASK & 4u) && bits == 2) rcode = dec_tile_loop_p<2, TMA_ONLY>(c, x, p0, cell_end, pending);
+          if ((BITMASK & 8u) && bits == 3) rcode = dec_tile_loop_p<3, TMA_ONLY>(c, x, p0, cell_end, pending);
+          if ((BITMASK & 16u) && bits == 4) rcode = dec_tile_loop_p<4, TMA_ONLY>(c, x, p0, cell_end, pending);
+          if ((BITMASK & 256u) && bits == 8) rcode = dec_tile_loop_p<8, TMA_ONLY>(c, x, p0, cell_end, pending);
           ok = (rcode & 1) != 0; pending = (rcode & 2) != 0;
         }
         j += cell_end - p;
