@@ -73,12 +73,19 @@ inline void add_decode_tc(Program &P, int stage, std::vector<tc::BBCell> cells, 
     cudaFuncSetAttribute(tc::decode_persistent_kernel<false, 0x11Fu>, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
     cudaFuncSetAttribute(tc::decode_persistent_kernel<true, 0x11Fu>, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
     cudaFuncSetAttribute(tc::decode_persistent_kernel<true, 0x110u>, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
+    cudaFuncSetAttribute(tc::decode_persistent_kernel<true, 0x010u>, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
+    cudaFuncSetAttribute(tc::decode_persistent_kernel<true, 0x100u>, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
+    cudaFuncSetAttribute(tc::decode_persistent_kernel<true, 0x014u>, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
+    cudaFuncSetAttribute(tc::decode_persistent_kernel<true, 0x018u>, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES);
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
     attr_done = true;
   }
-  // persistent form: every cell with r_t <= 128, the same sequence length and no rotation of keys at decode
+  // persistent form: every cell with r_t <= 128, the same sequence length and no rotation of keys at decode.  It is
+  // instantiated per output mode and per set of bit widths: with at most two tile loops compiled in (and fp16 output
+  // through bulk tensor stores only) ptxas keeps the whole epilogue in registers; with three or more it spills 50-60
+  // bytes, and a spill reload inside the tile loop costs several per cent of the launch.
   bool persistent = (g_fast.load() & 128) != 0 && n_sm > 0, tma_only = true;
   unsigned bitmask = 0;
   long long total = 0;
@@ -109,7 +116,11 @@ inline void add_decode_tc(Program &P, int stage, std::vector<tc::BBCell> cells, 
   P.add(stage, [=](char *dev_t, cudaStream_t s) {
     if (persistent) {
       tc::DecPArgs a{(const tc::BBCell *)(dev_t + off), n, nt, tot, seed, (const int2 *)(dev_t + off_run0), pool, chunk, (int *)(dev_t + off_cnt)};
-      if (tma_only && (bitmask & ~0x110u) == 0) tc::decode_persistent_kernel<true, 0x110u><<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
+      if (tma_only && bitmask == 0x010u) tc::decode_persistent_kernel<true, 0x010u><<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
+      else if (tma_only && bitmask == 0x100u) tc::decode_persistent_kernel<true, 0x100u><<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
+      else if (tma_only && (bitmask & ~0x110u) == 0) tc::decode_persistent_kernel<true, 0x110u><<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
+      else if (tma_only && (bitmask & ~0x014u) == 0) tc::decode_persistent_kernel<true, 0x014u><<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
+      else if (tma_only && (bitmask & ~0x018u) == 0) tc::decode_persistent_kernel<true, 0x018u><<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
       else if (tma_only) tc::decode_persistent_kernel<true, 0x11Fu><<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
       else tc::decode_persistent_kernel<false, 0x11Fu><<<grid_p, LY::THREADS, LY::SMEM_BYTES, s>>>(a);
     } else {
