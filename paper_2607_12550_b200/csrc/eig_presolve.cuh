@@ -23,8 +23,9 @@ struct PresolveTask {
 // Ash = A + (1e-12 * trace / n) I: every pivot of the factorisation stays positive, the null directions of a rank
 // deficient A become tiny columns of L that the one-sided Jacobi still orthogonalises (it works relative to each
 // column's own norm), so U is a complete basis.  The shift never reaches the eigenvalues: A' is formed from A itself.
+// grid (slices, matrices): every CTA sums the diagonal itself and shifts its slice of the rows.
 __global__ void presolve_shift_kernel(const PresolveTask *__restrict__ tasks) {
-  const PresolveTask t = tasks[blockIdx.x];
+  const PresolveTask t = tasks[blockIdx.y];
   const int n = t.n;
   __shared__ double red[32];
   double tr = 0.0;
@@ -35,7 +36,8 @@ __global__ void presolve_shift_kernel(const PresolveTask *__restrict__ tasks) {
   tr = 0.0;
   for (int w = 0; w < (int)blockDim.x / 32; ++w) tr += red[w];
   const double shift = 1e-12 * fabs(tr) / n;
-  for (int e = threadIdx.x; e < n * n; e += blockDim.x) {
+  const int per = (n * n + gridDim.x - 1) / gridDim.x, e0 = blockIdx.x * per, e1 = min(n * n, e0 + per);
+  for (int e = e0 + threadIdx.x; e < e1; e += blockDim.x) {
     const int i = e / n, j = e - i * n;
     t.Ash[e] = t.A[e] + (i == j ? shift : 0.0);
   }
@@ -60,6 +62,9 @@ __global__ void __launch_bounds__(256) presolve_mul_kernel(const PresolveTask *_
   double *out = SECOND ? t.Ash : t.T;
   for (int c0 = 0; c0 < n; c0 += 128) {
     double acc[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+    // unrolled: the loads of eight steps are in flight together (one step at a time left the kernel waiting on an L2
+    // round trip per step)
+#pragma unroll 8
     for (int k = 0; k < n; ++k) {
       const double a0 = lhs[2 * ty][k], a1 = lhs[2 * ty + 1][k];
 #pragma unroll

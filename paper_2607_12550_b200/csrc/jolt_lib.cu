@@ -434,7 +434,7 @@ void add_eig(Program &P, int stage, const std::vector<EigTask> &tasks, int bj_sw
   int pre_n = 0;
   for (auto &q : pre) pre_n = std::max(pre_n, q.n);
   if (n_pre) P.add(stage, [=](char *dev, cudaStream_t s) {
-    presolve_shift_kernel<<<n_pre, 256, 0, s>>>((const PresolveTask *)(dev + o_pre)); LAUNCHED();
+    presolve_shift_kernel<<<dim3(16, n_pre), 256, 0, s>>>((const PresolveTask *)(dev + o_pre)); LAUNCHED();
   });
   if (!cfs.empty()) {
     const size_t off = P.push(cfs);

@@ -13,7 +13,8 @@
 // -> read and stage(i) -> bulk store reads the rows -> unpack(i + 2): longer than the tensor pipe needs for two
 // tiles, and the pipe idles.  Here the output is staged in a region of its own (half a tile per warpgroup, one
 // 64-feature box per warp at a time), so the operand tile is free as soon as the rotation MMAs of tile i complete:
-// the warpgroup unpacks tile i + 2 FIRST and reads, converts and stores tile i while the rotation of i + 2 runs.
+// the warpgroup stores the first 64 features of tile i, unpacks tile i + 2 (while that store reads the staging rows),
+// then converts and stores the second 64 features of tile i while the rotation of i + 2 runs.
 //
 // What changes at a boundary:
 //   head   the projected core P_h (one 32 KB buffer; the 32 KB next to it is the staging region): a thread of its own
