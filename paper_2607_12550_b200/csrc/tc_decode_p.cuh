@@ -244,7 +244,7 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_persistent_kerne
   const int run0_first = my_run0.x, run0_end = my_run0.y;
   const int pool = a.pool;
   JOLT_DBG(long long *cta_dbg = cells[0].dbg ? cells[0].dbg + 128 + blockIdx.x * 4 : nullptr;)
-  JOLT_DBG(if (cta_dbg && threadIdx.x == 0) { long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); cta_dbg[0] = g; cta_dbg[2] = clock64(); })
+  JOLT_DBG(if (cta_dbg && threadIdx.x == 0) { long long g; unsigned sm; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); asm volatile("mov.u32 %0, %%smid;" : "=r"(sm)); cta_dbg[0] = g; cta_dbg[2] = sm; })
 
   // shared memory: P block (32 KB) | output staging (2 x 16 KB) | rotation operand H | U_T ring | operand tiles | barriers
   const uint32_t raw = smem_u32(smem_raw);
@@ -515,7 +515,7 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_persistent_kerne
   }
   tc_fence_before();
   __syncthreads();
-  JOLT_DBG(if (cta_dbg && threadIdx.x == 0) { long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); cta_dbg[1] = g; cta_dbg[3] = clock64(); })
+  JOLT_DBG(if (cta_dbg && threadIdx.x == 0) { long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); cta_dbg[1] = g; cta_dbg[3] = 0; })
   if (*abort_flag) {
     if (threadIdx.x == 0) atomicOr(cells[0].status, 8);
     const long long t0 = clock64();
