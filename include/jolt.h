@@ -305,10 +305,11 @@ int jolt_set_stream_groups(int n);
 int jolt_check_status(const jolt_handle *h, void *stream);
 
 /* Test hook.  cycles > 0 replaces the limit of every bounded device-side wait (default 10^9 SM cycles, about half a
- * second); skip_first_load != 0 makes the TMA thread of the two-tile sweep kernel leave out its first load, so that
- * the consumer's wait runs out: the kernel must drain, release its tensor memory and report JOLT_ETIMEOUT through
- * jolt_compress, and the next call on the same context must work.  cycles <= 0 and skip_first_load = 0 restore the
- * defaults.  Applies to the current device. */
+ * second).  skip_first_load = 1 makes the TMA thread of the two-tile sweep kernel leave out its first load, so that the
+ * consumer's wait runs out: the kernel must drain, release its tensor memory and report JOLT_ETIMEOUT through
+ * jolt_compress, and the next call on the same context must work.  skip_first_load = 2 does the same to the U_T thread
+ * of the persistent decode kernel: the launch ends, jolt_check_status reports JOLT_ETIMEOUT, the next decode works.
+ * cycles <= 0 and skip_first_load = 0 restore the defaults.  Applies to the current device. */
 int jolt_test_set_wait_limit(int64_t cycles, int32_t skip_first_load);
 
 /* Test hook for the persistent decode kernel.  Its CTAs take fixed shares of the launch's tile list; the kernel can

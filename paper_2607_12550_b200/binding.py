@@ -390,9 +390,10 @@ def check_status(handle: "Handle", stream=None):
     _check(lib.jolt_check_status(handle.ptr, _stream_ptr(stream)))
 
 
-def set_test_wait_limit(cycles: int = 0, skip_first_load: bool = False):
-    """Test hook of the bounded device-side waits; see include/jolt.h."""
-    _check(lib.jolt_test_set_wait_limit(int(cycles), 1 if skip_first_load else 0))
+def set_test_wait_limit(cycles: int = 0, skip_first_load=False):
+    """Test hook of the bounded device-side waits (skip_first_load: False / True = the sweep kernel / 2 = the persistent
+    decode kernel); see include/jolt.h."""
+    _check(lib.jolt_test_set_wait_limit(int(cycles), int(skip_first_load)))
 
 
 def set_test_decode_tail(percent: int = 0, chunk_tiles: int = 8):

@@ -2398,7 +2398,7 @@ extern "C" int jolt_debug_stamps(long long *host_out, int n) {
 extern "C" int64_t jolt_launch_count(void) { return g_launches.load(); }
 extern "C" int jolt_test_set_wait_limit(int64_t cycles, int32_t skip_first_load) {
   const long long lim = cycles > 0 ? (long long)cycles : tc::kSpinCycles;
-  const int skip = skip_first_load ? 1 : 0;
+  const int skip = skip_first_load == 2 ? 2 : (skip_first_load ? 1 : 0);
   CU(cudaMemcpyToSymbol(tc::g_spin_limit, &lim, sizeof lim));
   CU(cudaMemcpyToSymbol(tc::g_test_skip_first_load, &skip, sizeof skip));
   return JOLT_OK;

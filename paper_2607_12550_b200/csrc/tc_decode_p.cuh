@@ -320,6 +320,7 @@ __global__ void __launch_bounds__(DecLayout::THREADS, 1) decode_persistent_kerne
               const int s = cnt % NS, n = cnt / NS;
               ok = mbar_wait(bEmpty(s), (n & 1) ^ 1, abort_flag);
               if (!ok) break;
+              if (cnt == 0 && g_test_skip_first_load == 2) continue;      // test switch: the backbone thread's wait runs out
               mbar_expect_tx(bFull(s), BB_STAGE_BYTES);
               tma_load_2d(sRing + s * BB_STAGE_BYTES, &cg.tmUT, bFull(s), kb * 64, tt * 128);
             }

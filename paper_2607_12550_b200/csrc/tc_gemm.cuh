@@ -237,7 +237,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1) tc_gemm2_kernel(const Gemm2Cell
       ok = mbar_wait(bEmpty(s), (n & 1) ^ 1, abort_flag);
       if (!ok) break;
       const uint32_t st = sStages + s * stage_bytes;
-      if (j == 0 && g_test_skip_first_load) continue;       // test switch: this stage never fills, its consumer's wait runs out
+      if (j == 0 && g_test_skip_first_load == 1) continue;       // test switch: this stage never fills, its consumer's wait runs out
       mbar_expect_tx(bFull(s), a_bytes + (c.has_lo ? 2 : 1) * b_bytes);
       if (MODE == GM_TOK) {
         const int h = j >> 1, kf = j & 1;

@@ -810,6 +810,33 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_survives(B, synth):
     h.free()
 
 
+def test_a_wait_that_runs_out_in_the_persistent_decode_is_reported(B, synth):
+    """The same for the persistent decode kernel: its U_T thread leaves out the first ring stage, the backbone thread's
+    wait for it runs out after about a millisecond, every role of every CTA leaves its loops (the chunk queue gets its
+    end marker, the epilogue warpgroups still meet at their barriers), tensor memory is released, the launch ends and
+    jolt_check_status reports JOLT_ETIMEOUT; the next decode on the same context gives the usual output."""
+    cfg = synth.CacheConfig("t", 4, 2, 4, 512, n_terms=16, seed=21)
+    K, V = synth.make_cache(cfg, device="cuda")
+    gs = [0, 2, 4]
+    plans = [(32, 128, 4), (16, 128, 8), (32, 96, 4), (48, 128, 8)]
+    h, Ko, Vo = _roundtrip(B, K, V, gs, plans, B.default_options(seed=4))
+    B.check_status(h)
+    Kb, Vb = torch.empty_like(K), torch.empty_like(V)
+    B.set_test_wait_limit(2_000_000, 2)
+    try:
+        B.jolt_decompress(h, Kb, Vb, gs)
+        with pytest.raises(B.JoltError) as e:
+            B.check_status(h)
+        assert e.value.status == B.ETIMEOUT, e.value
+    finally:
+        B.set_test_wait_limit(0, False)
+    torch.cuda.synchronize()
+    B.jolt_decompress(h, Kb, Vb, gs)
+    B.check_status(h)
+    assert torch.equal(Kb, Ko) and torch.equal(Vb, Vo)
+    h.free()
+
+
 def test_decode_status_is_surfaced(B):
     """A stored quantisation step that is not a finite fp16 number cannot come out of jolt_compress, but it can sit in
     a damaged serialised image: the decode kernels raise a status bit, jolt_check_status (and a decode into host memory,
