@@ -418,8 +418,8 @@ def main():
     t_roof_d = sum(roof_time(*cell_work(cfg.m, cfg.seq_len, cfg.head_dim, rt, rf, b, min(rt + 10, cfg.seq_len, cfg.m * rf), q, 2)["decompress"], pk)
                    for rt, rf, b in plans)
     stages = {k_: v_ / len(rec) for k_, v_ in stage_acc.items()}
-    # roofline of the dominant kernel of the headline (decompress) call: decode_kernel is the only kernel of
-    # jolt_decompress; its duration is the library's own CUDA-event stage timer on the launching stream
+    # roofline of the dominant kernel of the headline (decompress) call: the decode kernel (persistent form, or the
+    # per-item one) is the only kernel of jolt_decompress; its duration is the library's own CUDA-event stage timer on the launching stream
     fd, bd = tot["decompress"]
     t_dec = stages.get("decode_rows", td)
     dec_bound = "hbm" if bd / (pk["hbm"] * 1e9) >= fd / (pk["tensor"] * 1e12) else "tensor"
