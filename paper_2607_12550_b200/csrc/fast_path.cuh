@@ -38,6 +38,27 @@ inline bool encode_store_maps(CellStore &cs) {
   return true;
 }
 
+// Launch with an explicit execution priority (the least one for the kernels that fill the machine: a cell group's
+// cache-wide sweeps and its residual pass then yield to the other groups' small latency-bound kernels, whose side
+// streams run at a higher priority).  Outside the concurrent cell groups the priority has nothing to compete with.
+inline int heavy_kernel_priority() {
+  static int lo = 0, hi = 0;
+  static bool have = false;
+  if (!have) { cudaDeviceGetStreamPriorityRange(&lo, &hi); have = true; }
+  return lo;
+}
+template <typename... KArgs, typename... Args>
+inline void launch_heavy(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute at;
+  memset(&at, 0, sizeof at);
+  at.id = cudaLaunchAttributePriority; at.val.priority = heavy_kernel_priority();
+  cfg.attrs = &at; cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 inline void bb_split(int total_heads, int n_tiles, int &tiles_per_item, int &items_per_head) {
   int per_head = (888 + total_heads / 2) / std::max(total_heads, 1);
   per_head = std::max(1, std::min(per_head, n_tiles));
@@ -58,7 +79,7 @@ inline void add_backbone_tc(Program &P, int stage, const std::vector<tc::BBCell>
   const size_t off = P.push(cells);
   const int n = (int)cells.size();
   P.add(stage, [=](char *dev_t, cudaStream_t s) {
-    tc::backbone_kernel<RESIDUAL><<<dim3(gx, n), tc::BB_THREADS, tc::BB_SMEM_BYTES, s>>>((const tc::BBCell *)(dev_t + off), seed);
+    launch_heavy(tc::backbone_kernel<RESIDUAL>, dim3(gx, n), dim3(tc::BB_THREADS), (size_t)tc::BB_SMEM_BYTES, s, (const tc::BBCell *)(dev_t + off), seed);
     LAUNCHED();
   });
 }
@@ -193,7 +214,7 @@ inline void launch_tc_gemm(Program &P, int stage, std::vector<tc::GemmCell> &cel
   const size_t off = P.push(cells);
   const int n = (int)cells.size();
   P.add(stage, [=](char *dev_t, cudaStream_t s) {
-    tc::tc_gemm_kernel<MODE><<<dim3(gx, n), tc::GM_THREADS, smem, s>>>((const tc::GemmCell *)(dev_t + off), n_stages);
+    launch_heavy(tc::tc_gemm_kernel<MODE>, dim3(gx, n), dim3(tc::GM_THREADS), smem, s, (const tc::GemmCell *)(dev_t + off), n_stages);
     LAUNCHED();
   });
 }
@@ -218,7 +239,7 @@ inline void launch_tc_gemm2(Program &P, int stage, std::vector<tc::Gemm2Cell> &c
   const size_t off = P.push(cells);
   const int n = (int)cells.size();
   P.add(stage, [=](char *dev_t, cudaStream_t s) {
-    tc::tc_gemm2_kernel<MODE><<<dim3(gx, n), tc::GM_THREADS, smem, s>>>((const tc::Gemm2Cell *)(dev_t + off), n_stages);
+    launch_heavy(tc::tc_gemm2_kernel<MODE>, dim3(gx, n), dim3(tc::GM_THREADS), smem, s, (const tc::Gemm2Cell *)(dev_t + off), n_stages);
     LAUNCHED();
   });
 }
@@ -416,7 +437,7 @@ inline void add_sketch_gen_tc(Program &P, int stage, std::vector<CellWork> &ws, 
   const size_t off = P.push(jobs);
   const int n = (int)jobs.size();
   P.add(stage, [=](char *dev_t, cudaStream_t s) {
-    tc::gen_sketch_f16_kernel<<<dim3(148, n), 256, 0, s>>>((const tc::SketchJob *)(dev_t + off), stream_id, seed);
+    launch_heavy(tc::gen_sketch_f16_kernel, dim3(148, n), dim3(256), (size_t)0, s, (const tc::SketchJob *)(dev_t + off), stream_id, seed);
     LAUNCHED();
   });
 }

@@ -1086,10 +1086,12 @@ GroupStreams *group_streams(int dev) {
       // Group 0 holds the cells whose chain is the longest (those with a feature eigen-solve, when there are any): its
       // stream gets the greatest priority, so its small latency-bound kernels are placed ahead of the other groups'
       // cache-wide sweeps instead of waiting for a wave of their CTAs to drain (measured on config 1: median of the call
-      // 3.04 -> 2.87 ms, and a quarter of the spread between calls).
+      // 3.04 -> 2.87 ms, and a quarter of the spread between calls).  The other groups' streams sit in the middle of the
+      // range and the kernels that fill the machine are launched at the least priority whatever their stream
+      // (launch_heavy): 2.87 -> 2.84 ms.
       int lo = 0, hi = 0;
       cudaDeviceGetStreamPriorityRange(&lo, &hi);      // (least, greatest)
-      if (cudaStreamCreateWithPriority(&g.s[i], cudaStreamNonBlocking, i == 0 ? hi : lo) != cudaSuccess) return nullptr;
+      if (cudaStreamCreateWithPriority(&g.s[i], cudaStreamNonBlocking, i == 0 ? hi : (hi + lo) / 2) != cudaSuccess) return nullptr;
       if (cudaEventCreateWithFlags(&g.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
     }
     if (cudaEventCreateWithFlags(&g.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
