@@ -217,15 +217,23 @@ __global__ void __launch_bounds__(128) project_core_kernel(const ProjJob *__rest
   // fp64 accumulation: products of two fp16 numbers are exact in it and the sum of <= 128 of them is far inside its
   // precision, so the one rounding to fp16 is the rounding of the exact value (the definition), not of an fp32 sum
   // that may sit on the other side of a rounding boundary
+  // eight rows of G at a time, staged in shared memory (read straight from global memory the loop waited for one
+  // broadcast load per row and step: 76 us for three small cells on the critical chain of the call)
+  __shared__ __half gs[8][128];
   for (int rb = r0; rb < min(r0 + 32, j.rows); rb += 8) {
+    __syncthreads();
+    for (int e = f; e < 8 * j.r_f; e += 128) {
+      const int r = e / j.r_f, s = e - r * j.r_f;
+      gs[r][s] = rb + r < j.rows ? j.G[(size_t)(rb + r) * j.r_f + s] : __float2half(0.f);
+    }
+    __syncthreads();
     double acc[8];
 #pragma unroll
     for (int r = 0; r < 8; ++r) acc[r] = 0.0;
     for (int s = 0; s < j.r_f; ++s) {
       const double u = (double)__half2float(pc_uf[s * 128 + f]);
 #pragma unroll
-      for (int r = 0; r < 8; ++r)
-        if (rb + r < j.rows) acc[r] = fma((double)__half2float(j.G[(size_t)(rb + r) * j.r_f + s]), u, acc[r]);
+      for (int r = 0; r < 8; ++r) acc[r] = fma((double)__half2float(gs[r][s]), u, acc[r]);
     }
 #pragma unroll
     for (int r = 0; r < 8; ++r)
